@@ -1,0 +1,243 @@
+/*
+ * tb.h -- C ABI of the B200 phrase-boosting decode library.
+ *
+ * The library implements the hot path of per-stream shallow-fusion phrase boosting inside
+ * batched Transducer (RNNT / TDT) decoding: every stream of a batch owns a compiled
+ * case-insensitive boosting graph; each decode step turns the hypothesis's graph state into
+ * a bonus over the vocabulary, adds lambda * bonus to the joint logits, selects tokens
+ * (argmax, or top-K over beam x vocabulary) and advances the graph state; blank leaves the
+ * state unchanged.
+ *
+ * Conventions
+ *   - Every call returns an int: TB_OK (0) or a negative TB_ERR_* code; tb_strerror() names
+ *     it.  No exception crosses this boundary and the library keeps no global state.
+ *   - "host" pointers are read or written by the CPU during the call.  "device" pointers are
+ *     caller-owned device memory on the batch's GPU; the library never frees or resizes
+ *     them.  The library owns only what tb_batch_create allocates (graph arena, slot table,
+ *     per-slot decode state, hypothesis tree, status word).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  GPU
+ *     work is enqueued on it and returns before it has run; device outputs may be read after
+ *     the stream has been synchronised.  All calls on one batch must be issued to one
+ *     stream, or be ordered by the caller, because a re-bind may reuse arena space that
+ *     earlier decode calls read.
+ *   - Token ids are 0..vocab-1, blank = vocab.  Graph states are graph-local (root = 0); a
+ *     slot without a graph reports state -1.
+ *   - Logits must not contain NaN (the selection is then undefined); infinities are fine.
+ *   - Arithmetic contract: a candidate's value is fl(x + fl(lambda * bonus)) in float32 (a
+ *     rounded multiply, then a rounded add, never fused); blank and unbound slots use x
+ *     itself; bf16 logits are widened exactly.  Ties go to the lowest token id.
+ */
+#ifndef TB_H_
+#define TB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TB_OK 0
+#define TB_ERR_INVALID_ARG (-1)   /* a bad pointer, size, token, weight, stride, dtype */
+#define TB_ERR_OOM (-2)           /* host or device allocation failed */
+#define TB_ERR_CUDA (-3)          /* a CUDA runtime call failed */
+#define TB_ERR_ARENA_FULL (-4)    /* the graph does not fit into the arena's free space */
+#define TB_ERR_BAD_SLOT (-5)      /* slot index outside the batch */
+#define TB_ERR_DEVICE_STATUS (-6) /* a kernel recorded a violated bound (see tb_batch_status) */
+
+#define TB_BF16 0 /* logits are bfloat16 */
+#define TB_F32 1  /* logits are float32 */
+
+/* Bits of the device status word (tb_batch_status). */
+#define TB_STATUS_WALK_TOO_DEEP 1   /* a suffix-link walk exceeded the graph's depth bound */
+#define TB_STATUS_BAD_STATE 2       /* a graph state outside [0, n_states) was met */
+#define TB_STATUS_STEP_LIMIT 4      /* a decode loop hit its static iteration bound */
+#define TB_STATUS_WAIT_TIMEOUT 8    /* a bounded wait inside a kernel ran out */
+
+/* Limits of this build. */
+#define TB_MAX_VOCAB 8192           /* non-blank tokens */
+#define TB_MAX_PHRASE_LEN 255       /* tokens per phrase (graph depth is stored in a byte) */
+#define TB_MAX_BEAM 32
+
+typedef struct tb_graph tb_graph; /* immutable compiled graph, host memory */
+typedef struct tb_batch tb_batch; /* device arena + slot table + per-slot state */
+
+/*
+ * Read-only view of a compiled graph as flat arrays in host memory: the arc arrays (label =
+ * case class, target state, weight) and state arrays (outgoing-arc range, suffix-link
+ * target, suffix-link weight, final weight) of Sec. 2.2 para. 2.  States are numbered
+ * breadth-first from root = 0 with a state's children in ascending class order, so arcs are
+ * sorted by (source state, class).  The pointers stay valid until tb_graph_free.
+ */
+typedef struct {
+  int32_t n_states, n_arcs, n_classes, vocab, max_depth;
+  float lambda;
+  const int32_t *state_arc_begin; /* [n_states+1] */
+  const int32_t *arc_class;       /* [n_arcs] ascending within a state */
+  const int32_t *arc_dst;         /* [n_arcs] */
+  const float *arc_w;             /* [n_arcs] */
+  const int32_t *state_fail;      /* [n_states] suffix-link target */
+  const float *state_bw;          /* [n_states] suffix-link weight */
+  const float *state_final;       /* [n_states] final weight (exported, not applied) */
+  const uint8_t *state_depth;     /* [n_states] */
+  const int32_t *case_class;      /* [vocab] token -> class */
+} tb_graph_view;
+
+const char *tb_strerror(int code);
+
+/*
+ * Compile one phrase list into a boosting graph (host only, no GPU needed).
+ * Sec. 2.1 para. 1-2 (phrase tree with suffix links; one arc per case class stands for all
+ * case variants of a token), the potential rule above Eq. 1 (arc score = destination potential
+ * minus source potential; one token per arc, so Eq. 1's split is Delta = w_k), Sec. 2.2 para. 2
+ * (array layout).
+ *   phrase_tokens  host int32 [phrase_offsets[n_phrases]]: the phrases' tokens, back to back
+ *   phrase_offsets host int64 [n_phrases+1], non-decreasing, first entry 0
+ *   token_weights  host float [as phrase_tokens] or NULL (= 1.0): score of each phrase token;
+ *                  must be finite and >= 0; where phrases share a prefix the largest weight
+ *                  given to a position wins; phrases equal after case folding are merged
+ *   case_class     host int32 [vocab] or NULL (= identity, case-sensitive): tokens with the
+ *                  same class are case variants of each other; classes are >= 0
+ *   lambda         boosting weight of this list (Sec. 2.2 para. 2), finite
+ *   flags          must be 0
+ *   out            receives the graph; free it with tb_graph_free
+ * Empty phrases are skipped.  Errors: TB_ERR_INVALID_ARG (token outside [0, vocab), bad
+ * weight or class, phrase longer than TB_MAX_PHRASE_LEN, vocab outside [1, TB_MAX_VOCAB]),
+ * TB_ERR_OOM.
+ */
+int tb_graph_compile(const int32_t *phrase_tokens, const int64_t *phrase_offsets, int32_t n_phrases,
+                     const float *token_weights, const int32_t *case_class, int32_t vocab, float lambda,
+                     uint32_t flags, tb_graph **out);
+
+/* Fill *out with pointers into g (host).  TB_ERR_INVALID_ARG on NULL. */
+int tb_graph_view_get(const tb_graph *g, tb_graph_view *out);
+
+/* Free a graph.  Safe right after tb_batch_bind_stream returned: bind copies what it needs. */
+void tb_graph_free(tb_graph *g);
+
+/*
+ * Create a batch on `device`: the merged multi-model storage of Sec. 2.2 para. 2 (one arena
+ * holding every bound graph's arrays behind a per-slot offset table), plus per-slot decode
+ * state.  All slots start unbound (model id -1).
+ *   vocab, case_class  as for tb_graph_compile; one token -> class map per batch
+ *   n_slots            number of stream slots (>= 1)
+ *   max_beam           largest K tb_beam_step will be called with (1..TB_MAX_BEAM)
+ *   max_tree_steps     capacity, in beam steps, of the hypothesis tree (0 = no tree)
+ *   arena_bytes        size of the graph arena
+ * Errors: TB_ERR_INVALID_ARG, TB_ERR_OOM, TB_ERR_CUDA.
+ */
+int tb_batch_create(int32_t vocab, const int32_t *case_class, int32_t n_slots, int32_t max_beam,
+                    int32_t max_tree_steps, size_t arena_bytes, int device, tb_batch **out);
+
+/* Free everything the batch owns (synchronises the device first). */
+void tb_batch_destroy(tb_batch *b);
+
+/*
+ * Attach graph g to `slot`, or detach with g == NULL (model id -1: zero bonus, state -1;
+ * Sec. 2.2 para. 3).  Adding and removing lists while other streams keep running is Sec. 2.2
+ * para. 4; here the slot index is the stable id, and no other slot's graph moves or changes.
+ * The graph is copied through pinned host memory with an asynchronous host-to-device copy
+ * on `stream`; the slot's offsets are published and its streaming state is reset (state =
+ * root or -1, frame cursor 0, score 0) in stream order.  The previous graph's arena space is
+ * reused by later binds.  g must have been compiled with the batch's vocab and class map.
+ * Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG (vocab / class map mismatch),
+ * TB_ERR_ARENA_FULL (nothing was changed), TB_ERR_CUDA.
+ */
+int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *stream);
+
+/*
+ * Copy the device status word to *device_status (host) after synchronising `stream`, and
+ * clear it.  Returns TB_OK if it was 0, else TB_ERR_DEVICE_STATUS (bits: TB_STATUS_*).
+ */
+int tb_batch_status(tb_batch *b, int32_t *device_status, void *stream);
+
+/*
+ * Greedy RNNT decoding of B streams, slot i serving stream i, all on the device with no
+ * host synchronisation per frame (Sec. 2.2 para. 3 for the boosted scores, Sec. 3.4 for greedy
+ * label-looping decoding, Sec. 2.3 for GPU-resident execution).
+ * Per stream: t = 0, k = 0, state = root; while t < length: take row (t, k), select the
+ * argmax of the boosted row; blank: t++, k = 0; else emit (token, t), advance the state,
+ * k++, and k == S closes the frame (t++, k = 0) adding nothing to the score.  The score is
+ * the float32 sum, in step order, of the selected values.
+ *   logits       device, dtype TB_BF16 or TB_F32, logical shape [B, T, S, vocab+1]
+ *   strides      host int64 [4]: element strides of the four dimensions
+ *   lengths      device int32 [B] or NULL (= T); values are clamped to [0, T]
+ *   out_tokens   device int32 [B, T*S]: emitted tokens of stream i at [i*T*S ...]
+ *   out_frames   device int32 [B, T*S]: frame of each emitted token
+ *   out_counts   device int32 [B]: tokens emitted
+ *   out_scores   device float [B]
+ *   out_states   device int32 [B]: final graph state (-1 for unbound slots)
+ * Does not read or change the slots' streaming state.  Errors: TB_ERR_INVALID_ARG
+ * (B > n_slots, bad dtype, NULL pointers, non-positive sizes), TB_ERR_CUDA.
+ */
+int tb_greedy_decode(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t T, int32_t S,
+                     const int64_t *strides, const int32_t *lengths, int32_t *out_tokens,
+                     int32_t *out_frames, int32_t *out_counts, float *out_scores, int32_t *out_states,
+                     void *stream);
+
+/*
+ * One streaming chunk for slots 0..n_slots-1, RNNT (n_dur = 0) or TDT (n_dur > 0), resuming
+ * from and updating each slot's persistent state {graph state, frame cursor, symbols in the
+ * current frame, score, emitted count} (Sec. 2.3: decoding state is kept across chunk
+ * boundaries; Sec. 2.2 para. 4: slots are re-bound between chunks).  The call covers the
+ * slot's frames [c, c + chunk), c = chunk * (number of tb_stream_chunk calls since the
+ * slot's last bind... counted per slot); frames at or beyond valid_frames[slot] are not
+ * decoded; a cursor that a TDT duration moved beyond the chunk is carried over.
+ * TDT row: vocab+1 token logits, then n_dur duration logits for durations 0..n_dur-1; the
+ * duration is their argmax (lowest on ties); score += value[token] + x_dur[duration];
+ * blank: t += max(duration, 1); token: emit, advance the state, then duration > 0 ?
+ * t += duration : next row of the same frame (the S-th symbol closes the frame).
+ *   logits        device [n_slots, chunk, S, vocab+1+n_dur], strides as above (host int64 [4])
+ *   valid_frames  device int32 [n_slots]: total frames of the slot's stream known so far
+ *   out_tokens / out_frames / out_durs  device int32 [n_slots, chunk*S]; out_durs may be NULL
+ *   out_counts    device int32 [n_slots]: tokens emitted in this chunk
+ *   out_scores    device float [n_slots]: running score
+ *   out_states    device int32 [n_slots]: graph state after the chunk
+ *   out_cursors   device int32 [n_slots] or NULL: frame cursor after the chunk
+ * Errors: as tb_greedy_decode.
+ */
+int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots, int32_t chunk, int32_t S,
+                    int32_t n_dur, const int64_t *strides, const int32_t *valid_frames,
+                    int32_t *out_tokens, int32_t *out_frames, int32_t *out_durs, int32_t *out_counts,
+                    float *out_scores, int32_t *out_states, int32_t *out_cursors, void *stream);
+
+/* Forget the hypothesis tree (step counter = 0).  Call before the first step of an utterance. */
+int tb_beam_reset(tb_batch *b);
+
+/*
+ * One beam expansion for streams 0..B-1 (Sec. 2.3 / Sec. 3.4 beam search; Sec. 2.2 para. 3 for
+ * the scores), each hypothesis carrying its own graph state.
+ * Per stream, candidates: each live hypothesis k with score > -inf and each token v in
+ * 0..vocab scores fl(score_k + value_k(v)); each frozen hypothesis with score > -inf is
+ * carried as one candidate with its score and token -1.  The K best in the order (score
+ * descending, token ascending with the carried token counted as vocab+1, parent ascending)
+ * become the new hypotheses, best first: score, state = token non-blank ? next(state_parent,
+ * token) : state_parent, live = live_parent and token non-blank.  Unfilled places get score
+ * -inf, state -1, live 0, parent -1, token -1.  (parent, token) is appended to the
+ * hypothesis tree when the batch has one.
+ *   logits         device; hypothesis k of stream i reads the vocab+1 contiguous elements
+ *                  at element offset i*stream_stride + k*hyp_stride (hyp_stride 0: all
+ *                  hypotheses of a stream share one row)
+ *   new_frame      non-zero: before expanding, every hypothesis with score > -inf becomes live
+ *   scores/states/live  device float / int32 / uint8 [B, K], updated in place
+ *   out_parent/out_token  device int32 [B, K]
+ * Errors: TB_ERR_INVALID_ARG (K > max_beam, tree full, ...), TB_ERR_CUDA.
+ */
+int tb_beam_step(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t K, int64_t stream_stride,
+                 int64_t hyp_stride, int32_t new_frame, float *scores, int32_t *states, uint8_t *live,
+                 int32_t *out_parent, int32_t *out_token, void *stream);
+
+/*
+ * Walk the hypothesis tree back from the hypotheses of the latest step and write each one's
+ * non-blank tokens in emission order (Sec. 2.3: hypotheses live in a flattened tree).
+ *   out_tokens  device int32 [B, K, max_len]; sequences longer than max_len are truncated
+ *   out_lens    device int32 [B, K]: full lengths (0 for empty places)
+ * Errors: TB_ERR_INVALID_ARG (no tree, no steps, K/B different from the steps recorded).
+ */
+int tb_beam_backtrace(tb_batch *b, int32_t B, int32_t K, int32_t max_len, int32_t *out_tokens,
+                      int32_t *out_lens, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TB_H_ */

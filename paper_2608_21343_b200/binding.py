@@ -1,0 +1,270 @@
+"""Python side of the C-ABI library ``libtb.so``: the same calls with the same names, taking
+torch tensors for device memory and numpy arrays for host memory.  Argument marshalling only --
+every step of the decode path runs in the library's CUDA kernels.  There is no CPU fallback: if
+the library cannot be loaded, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtb.so")
+
+if not os.path.exists(LIB_PATH):
+    raise RuntimeError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2608_21343_b200.build` "
+        "(or __graft_entry__.build()); this package has no fallback path")
+_lib = C.CDLL(LIB_PATH)
+
+TB_OK = 0
+TB_ERR_INVALID_ARG, TB_ERR_OOM, TB_ERR_CUDA, TB_ERR_ARENA_FULL, TB_ERR_BAD_SLOT, TB_ERR_DEVICE_STATUS = -1, -2, -3, -4, -5, -6
+TB_BF16, TB_F32 = 0, 1
+
+
+class TbError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {tb_strerror(code)} ({code})")
+
+
+class _GraphView(C.Structure):
+    _fields_ = [
+        ("n_states", C.c_int32), ("n_arcs", C.c_int32), ("n_classes", C.c_int32), ("vocab", C.c_int32),
+        ("max_depth", C.c_int32), ("lambda_", C.c_float),
+        ("state_arc_begin", C.POINTER(C.c_int32)), ("arc_class", C.POINTER(C.c_int32)),
+        ("arc_dst", C.POINTER(C.c_int32)), ("arc_w", C.POINTER(C.c_float)),
+        ("state_fail", C.POINTER(C.c_int32)), ("state_bw", C.POINTER(C.c_float)),
+        ("state_final", C.POINTER(C.c_float)), ("state_depth", C.POINTER(C.c_uint8)),
+        ("case_class", C.POINTER(C.c_int32)),
+    ]
+
+
+_vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
+_SIGS = {
+    "tb_strerror": (C.c_char_p, [C.c_int]),
+    "tb_graph_compile": (C.c_int, [_vp, _vp, _i32, _vp, _vp, _i32, C.c_float, C.c_uint32, C.POINTER(_vp)]),
+    "tb_graph_view_get": (C.c_int, [_vp, C.POINTER(_GraphView)]),
+    "tb_graph_free": (None, [_vp]),
+    "tb_batch_create": (C.c_int, [_i32, _vp, _i32, _i32, _i32, C.c_size_t, C.c_int, C.POINTER(_vp)]),
+    "tb_batch_destroy": (None, [_vp]),
+    "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
+    "tb_batch_status": (C.c_int, [_vp, C.POINTER(_i32), _vp]),
+    "tb_greedy_decode": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "tb_stream_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
+                                  _vp, _vp, _vp]),
+    "tb_beam_reset": (C.c_int, [_vp]),
+    "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _fn = getattr(_lib, _name)       # AttributeError here = the library lacks a declared symbol
+    _fn.restype, _fn.argtypes = _res, _args
+
+EXPORTED = tuple(_SIGS)
+
+
+def tb_strerror(code: int) -> str:
+    return _lib.tb_strerror(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != TB_OK:
+        raise TbError(code, where)
+
+
+def _host(a, dtype):
+    return None if a is None else np.ascontiguousarray(a, dtype=dtype)
+
+
+def _hp(a):
+    return None if a is None else a.ctypes.data_as(_vp)
+
+
+def _dp(t):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda):
+        raise TypeError("expected a CUDA tensor")
+    return _vp(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return _vp(stream.cuda_stream)
+
+
+def _logit_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return TB_BF16
+    if t.dtype == torch.float32:
+        return TB_F32
+    raise TypeError("logits must be bfloat16 or float32")
+
+
+class Graph:
+    """A compiled boosting graph (host object)."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def view(self) -> dict:
+        v = _GraphView()
+        _check(_lib.tb_graph_view_get(self.handle, C.byref(v)), "tb_graph_view_get")
+        n, a = v.n_states, v.n_arcs
+
+        def arr(p, cnt, dt):
+            return np.ctypeslib.as_array(p, shape=(cnt,)).astype(dt, copy=True) if cnt else np.zeros(0, dtype=dt)
+
+        return dict(
+            n_states=n, n_arcs=a, n_classes=v.n_classes, vocab=v.vocab, max_depth=v.max_depth, lam=v.lambda_,
+            state_arc_begin=arr(v.state_arc_begin, n + 1, np.int32), arc_class=arr(v.arc_class, a, np.int32),
+            arc_dst=arr(v.arc_dst, a, np.int32), arc_w=arr(v.arc_w, a, np.float32),
+            state_fail=arr(v.state_fail, n, np.int32), state_bw=arr(v.state_bw, n, np.float32),
+            state_final=arr(v.state_final, n, np.float32), state_depth=arr(v.state_depth, n, np.uint8),
+            case_class=arr(v.case_class, v.vocab, np.int32))
+
+    def free(self):
+        if self.handle:
+            _lib.tb_graph_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.free()
+
+
+def tb_graph_compile(phrases, vocab: int, case_class=None, token_weights=None, lam: float = 1.0, flags: int = 0) -> Graph:
+    """phrases: list of token lists, or a (tokens, offsets) pair of arrays."""
+    if isinstance(phrases, tuple):
+        toks, offs = _host(phrases[0], np.int32), _host(phrases[1], np.int64)
+        n = len(offs) - 1
+        w = _host(token_weights, np.float32)
+    else:
+        n = len(phrases)
+        offs = np.zeros(n + 1, dtype=np.int64)
+        if n:
+            offs[1:] = np.cumsum([len(p) for p in phrases])
+        toks = np.array([t for p in phrases for t in p], dtype=np.int32)
+        w = None if token_weights is None else np.array([x for p in token_weights for x in p], dtype=np.float32)
+    cc = _host(case_class, np.int32)
+    h = _vp()
+    _check(_lib.tb_graph_compile(_hp(toks), _hp(offs), n, _hp(w), _hp(cc), vocab, float(lam), flags, C.byref(h)),
+           "tb_graph_compile")
+    return Graph(h)
+
+
+class Batch:
+    """Device arena + slot table + per-slot decode state."""
+
+    def __init__(self, handle, vocab, n_slots, max_beam, device):
+        self.handle, self.vocab, self.n_slots, self.max_beam, self.device = handle, vocab, n_slots, max_beam, device
+
+    def destroy(self):
+        if self.handle:
+            _lib.tb_batch_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.destroy()
+
+
+def tb_batch_create(vocab: int, case_class, n_slots: int, max_beam: int = 1, max_tree_steps: int = 0,
+                    arena_bytes: int = 64 << 20, device: int = 0) -> Batch:
+    cc = _host(case_class, np.int32)
+    h = _vp()
+    _check(_lib.tb_batch_create(vocab, _hp(cc), n_slots, max_beam, max_tree_steps, arena_bytes, device, C.byref(h)),
+           "tb_batch_create")
+    return Batch(h, vocab, n_slots, max_beam, device)
+
+
+def tb_batch_destroy(batch: Batch):
+    batch.destroy()
+
+
+def tb_batch_bind_stream(batch: Batch, slot: int, graph, stream=None):
+    _check(_lib.tb_batch_bind_stream(batch.handle, slot, None if graph is None else graph.handle, _stream(stream)),
+           "tb_batch_bind_stream")
+
+
+def tb_batch_status(batch: Batch, stream=None) -> int:
+    st = _i32(0)
+    rc = _lib.tb_batch_status(batch.handle, C.byref(st), _stream(stream))
+    if rc not in (TB_OK, TB_ERR_DEVICE_STATUS):
+        raise TbError(rc, "tb_batch_status")
+    return st.value
+
+
+def _strides4(t: torch.Tensor):
+    assert t.dim() == 4
+    return np.array(t.stride(), dtype=np.int64)
+
+
+def tb_greedy_decode(batch: Batch, logits: torch.Tensor, lengths=None, out=None, stream=None) -> dict:
+    """logits [B, T, S, vocab+1] on the batch's device.  Returns device tensors."""
+    B, T, S, W = logits.shape
+    if W != batch.vocab + 1:
+        raise ValueError("last dimension must be vocab + 1")
+    dev = logits.device
+    if out is None:
+        out = dict(tokens=torch.empty((B, T * S), dtype=torch.int32, device=dev),
+                   frames=torch.empty((B, T * S), dtype=torch.int32, device=dev),
+                   counts=torch.empty(B, dtype=torch.int32, device=dev),
+                   scores=torch.empty(B, dtype=torch.float32, device=dev),
+                   states=torch.empty(B, dtype=torch.int32, device=dev))
+    st = _strides4(logits)
+    _check(_lib.tb_greedy_decode(batch.handle, _dp(logits), _logit_dtype(logits), B, T, S, _hp(st), _dp(lengths),
+                                 _dp(out["tokens"]), _dp(out["frames"]), _dp(out["counts"]), _dp(out["scores"]),
+                                 _dp(out["states"]), _stream(stream)), "tb_greedy_decode")
+    return out
+
+
+def tb_stream_chunk(batch: Batch, logits: torch.Tensor, n_dur: int, valid_frames: torch.Tensor, out=None,
+                    stream=None) -> dict:
+    """logits [n_slots, chunk, S, vocab+1+n_dur].  Returns device tensors."""
+    n, chunk, S, W = logits.shape
+    if W != batch.vocab + 1 + n_dur:
+        raise ValueError("last dimension must be vocab + 1 + n_dur")
+    dev = logits.device
+    if out is None:
+        out = dict(tokens=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   frames=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   durs=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   counts=torch.empty(n, dtype=torch.int32, device=dev),
+                   scores=torch.empty(n, dtype=torch.float32, device=dev),
+                   states=torch.empty(n, dtype=torch.int32, device=dev),
+                   cursors=torch.empty(n, dtype=torch.int32, device=dev))
+    st = _strides4(logits)
+    _check(_lib.tb_stream_chunk(batch.handle, _dp(logits), _logit_dtype(logits), n, chunk, S, n_dur, _hp(st),
+                                _dp(valid_frames), _dp(out["tokens"]), _dp(out["frames"]), _dp(out.get("durs")),
+                                _dp(out["counts"]), _dp(out["scores"]), _dp(out["states"]), _dp(out.get("cursors")),
+                                _stream(stream)), "tb_stream_chunk")
+    return out
+
+
+def tb_beam_reset(batch: Batch):
+    _check(_lib.tb_beam_reset(batch.handle), "tb_beam_reset")
+
+
+def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_stride: int, new_frame: bool,
+                 scores: torch.Tensor, states: torch.Tensor, live: torch.Tensor, out_parent: torch.Tensor,
+                 out_token: torch.Tensor, stream=None, offset: int = 0):
+    """logits: any tensor; hypothesis k of stream i reads vocab+1 contiguous elements at element
+    offset ``offset + i*stream_stride + k*hyp_stride``.  scores/states/live [B, K] are updated in place."""
+    B, K = scores.shape
+    ptr = _vp(logits.data_ptr() + offset * logits.element_size())
+    _check(_lib.tb_beam_step(batch.handle, ptr, _logit_dtype(logits), B, K, stream_stride, hyp_stride,
+                             1 if new_frame else 0, _dp(scores), _dp(states), _dp(live), _dp(out_parent),
+                             _dp(out_token), _stream(stream)), "tb_beam_step")
+
+
+def tb_beam_backtrace(batch: Batch, B: int, K: int, max_len: int, stream=None):
+    dev = torch.device("cuda", batch.device)
+    toks = torch.zeros((B, K, max_len), dtype=torch.int32, device=dev)
+    lens = torch.zeros((B, K), dtype=torch.int32, device=dev)
+    _check(_lib.tb_beam_backtrace(batch.handle, B, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
+           "tb_beam_backtrace")
+    return toks, lens

@@ -1,0 +1,80 @@
+"""Builds the CUDA library in-tree: ``paper_2608_21343_b200/libtb.so`` (sm_100a only)."""
+from __future__ import annotations
+
+import glob
+import hashlib
+import os
+import shutil
+import subprocess
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_HERE)
+CSRC = os.path.join(_HERE, "csrc")
+INCLUDE = os.path.join(_ROOT, "include")
+LIB = os.path.join(_HERE, "libtb.so")
+_STAMP = LIB + ".srchash"
+
+NVCC_FLAGS = [
+    "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+    "--fmad=false",  # the arithmetic contract forbids fusing x + lambda*bonus
+    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+]
+
+
+def sources():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")) + glob.glob(os.path.join(CSRC, "*.cpp")))
+
+
+def _src_hash() -> str:
+    h = hashlib.sha256()
+    files = sources() + sorted(glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
+                               glob.glob(os.path.join(INCLUDE, "*.h")))
+    for f in files:
+        h.update(os.path.basename(f).encode())
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()
+
+
+def is_current() -> bool:
+    if not (os.path.exists(LIB) and os.path.exists(_STAMP)):
+        return False
+    with open(_STAMP) as f:
+        return f.read().strip() == _src_hash()
+
+
+def nvcc_path():
+    return shutil.which("nvcc") or ("/usr/local/cuda/bin/nvcc" if os.path.exists("/usr/local/cuda/bin/nvcc") else None)
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    if not force and is_current():
+        return LIB
+    nvcc = nvcc_path()
+    if nvcc is None:
+        raise RuntimeError("nvcc not found: cannot build libtb.so")
+    cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", LIB, *sources()]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.run(cmd, check=True)
+    with open(_STAMP, "w") as f:
+        f.write(_src_hash())
+    return LIB
+
+
+def ensure_built() -> str:
+    """Build if the library is missing or stale and a compiler is present; otherwise require the
+    library to exist (a machine without nvcc uses the one that was built beforehand)."""
+    if is_current():
+        return LIB
+    if nvcc_path() is not None:
+        return build_library()
+    if os.path.exists(LIB):
+        return LIB
+    raise RuntimeError("libtb.so is missing and nvcc is not available to build it")
+
+
+if __name__ == "__main__":
+    import sys
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))

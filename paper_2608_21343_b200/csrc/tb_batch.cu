@@ -1,0 +1,299 @@
+// Batch object: the merged multi-model storage (one device arena for all bound graphs behind a
+// per-slot offset table, Sec. 2.2 para. 2), graph add / swap / remove (Sec. 2.2 para. 4) with
+// asynchronous host-to-device copies through pinned staging, and the C-ABI entry points that
+// validate arguments and launch the decode kernels.
+#include <cstring>
+#include <map>
+#include <new>
+#include <vector>
+
+#include "tb_launch.h"
+
+namespace {
+
+constexpr size_t kArenaAlign = 256;
+constexpr int kStagingRing = 4;
+
+struct DeviceGuard {  // makes the batch's device current for the duration of a call
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; cudaGetLastError(); return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) { ok = false; cudaGetLastError(); }
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// First-fit free list over the arena with coalescing.  Live graphs never move: a slot keeps its
+// block until it is re-bound, so no decode in flight ever sees its arrays shift.  (The paper
+// compacts the merged tensors on removal; with a free list the physical offsets of the other
+// models stay put and the slot index plays the role of the stable model id.)
+struct ArenaAllocator {
+  std::map<size_t, size_t> free_blocks;  // offset -> size
+  size_t capacity = 0;
+  void init(size_t bytes) { capacity = bytes; free_blocks.clear(); if (bytes) free_blocks[0] = bytes; }
+  bool alloc(size_t bytes, size_t* off) {
+    for (auto it = free_blocks.begin(); it != free_blocks.end(); ++it) {
+      if (it->second >= bytes) {
+        *off = it->first;
+        size_t rest = it->second - bytes, start = it->first;
+        free_blocks.erase(it);
+        if (rest) free_blocks[start + bytes] = rest;
+        return true;
+      }
+    }
+    return false;
+  }
+  void release(size_t off, size_t bytes) {
+    auto next = free_blocks.lower_bound(off);
+    if (next != free_blocks.begin()) {
+      auto prev = std::prev(next);
+      if (prev->first + prev->second == off) { off = prev->first; bytes += prev->second; free_blocks.erase(prev); }
+    }
+    if (next != free_blocks.end() && off + bytes == next->first) { bytes += next->second; free_blocks.erase(next); }
+    free_blocks[off] = bytes;
+  }
+  size_t free_bytes() const { size_t s = 0; for (auto& kv : free_blocks) s += kv.second; return s; }
+};
+
+struct Staging {
+  unsigned char* host = nullptr;
+  size_t cap = 0;
+  cudaEvent_t done = nullptr;
+  bool pending = false;
+};
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct tb_batch {
+  int device = 0;
+  int32_t vocab = 0, n_classes = 0, n_slots = 0, max_beam = 0, max_tree_steps = 0;
+  uint64_t class_map_hash = 0;
+  unsigned char* arena = nullptr;
+  size_t arena_bytes = 0;
+  TbSlotRec* d_slots = nullptr;
+  TbSlotState* d_sstate = nullptr;
+  int32_t* d_cls = nullptr;
+  int32_t* d_status = nullptr;
+  int2* d_tree = nullptr;
+  int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
+  ArenaAllocator alloc;
+  std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
+  Staging staging[kStagingRing];
+  int next_staging = 0;
+};
+
+static void destroy_batch(tb_batch* b) {
+  if (!b) return;
+  cudaDeviceSynchronize();
+  cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
+  cudaFree(b->d_status); cudaFree(b->d_tree);
+  for (auto& s : b->staging) {
+    if (s.host) cudaFreeHost(s.host);
+    if (s.done) cudaEventDestroy(s.done);
+  }
+  cudaGetLastError();
+  delete b;
+}
+
+extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t n_slots, int32_t max_beam,
+                               int32_t max_tree_steps, size_t arena_bytes, int device, tb_batch** out) {
+  if (!out) return TB_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (vocab < 1 || vocab > TB_MAX_VOCAB || n_slots < 1 || max_beam < 1 || max_beam > TB_MAX_BEAM ||
+      max_tree_steps < 0 || arena_bytes == 0)
+    return TB_ERR_INVALID_ARG;
+  std::vector<int32_t> cls(vocab);
+  int32_t n_classes = 0;
+  for (int32_t v = 0; v < vocab; ++v) {
+    cls[v] = case_class ? case_class[v] : v;
+    if (cls[v] < 0) return TB_ERR_INVALID_ARG;
+    n_classes = cls[v] + 1 > n_classes ? cls[v] + 1 : n_classes;
+  }
+  DeviceGuard guard(device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  tb_batch* b = new (std::nothrow) tb_batch();
+  if (!b) return TB_ERR_OOM;
+  b->device = device; b->vocab = vocab; b->n_classes = n_classes; b->n_slots = n_slots;
+  b->max_beam = max_beam; b->max_tree_steps = max_tree_steps;
+  b->class_map_hash = tb_hash_class_map(case_class, vocab);
+  b->arena_bytes = round_up(arena_bytes, kArenaAlign);
+  b->alloc.init(b->arena_bytes);
+  b->slot_block.assign(n_slots, {0, 0});
+  bool ok = true;
+  ok = ok && cudaMalloc(&b->arena, b->arena_bytes) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_slots, sizeof(TbSlotRec) * n_slots) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_sstate, sizeof(TbSlotState) * n_slots) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_cls, sizeof(int32_t) * vocab) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_status, sizeof(int32_t)) == cudaSuccess;
+  if (ok && max_tree_steps > 0)
+    ok = cudaMalloc(&b->d_tree, sizeof(int2) * static_cast<size_t>(max_tree_steps) * n_slots * max_beam) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); destroy_batch(b); return TB_ERR_OOM; }
+  // every slot starts unbound: n_states = 0, streaming state = {-1, 0, 0, 0, 0, 0}
+  std::vector<TbSlotState> init(n_slots);
+  for (auto& s : init) { std::memset(&s, 0, sizeof s); s.state = -1; }
+  ok = ok && cudaMemset(b->d_slots, 0, sizeof(TbSlotRec) * n_slots) == cudaSuccess;
+  ok = ok && cudaMemcpy(b->d_sstate, init.data(), sizeof(TbSlotState) * n_slots, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(b->d_cls, cls.data(), sizeof(int32_t) * vocab, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemset(b->d_status, 0, sizeof(int32_t)) == cudaSuccess;
+  for (auto& s : b->staging) ok = ok && cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); destroy_batch(b); return TB_ERR_CUDA; }
+  *out = b;
+  return TB_OK;
+}
+
+extern "C" void tb_batch_destroy(tb_batch* b) {
+  if (!b) return;
+  DeviceGuard guard(b->device);
+  destroy_batch(b);
+}
+
+extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g, void* stream_) {
+  if (!b) return TB_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= b->n_slots) return TB_ERR_BAD_SLOT;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  TbSlotRec rec;
+  std::memset(&rec, 0, sizeof rec);
+  size_t off = 0, bytes = 0;
+  if (g) {
+    if (g->vocab != b->vocab || g->class_map_hash != b->class_map_hash) return TB_ERR_INVALID_ARG;
+    bytes = round_up(g->blob.size(), kArenaAlign);
+    if (!b->alloc.alloc(bytes, &off)) return TB_ERR_ARENA_FULL;
+    // pinned staging: wait only if this ring entry's previous copy has not finished yet
+    Staging& s = b->staging[b->next_staging];
+    b->next_staging = (b->next_staging + 1) % kStagingRing;
+    bool ok = true;
+    if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
+    if (ok && s.cap < g->blob.size()) {
+      if (s.host) cudaFreeHost(s.host);
+      s.host = nullptr; s.cap = 0;
+      size_t want = round_up(g->blob.size() * 2, 1 << 16);
+      ok = cudaMallocHost(&s.host, want) == cudaSuccess;
+      if (ok) s.cap = want;
+    }
+    if (ok) {
+      std::memcpy(s.host, g->blob.data(), g->blob.size());
+      ok = cudaMemcpyAsync(b->arena + off, s.host, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+      ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;
+      s.pending = ok;
+    }
+    if (!ok) { cudaGetLastError(); b->alloc.release(off, bytes); return TB_ERR_CUDA; }
+    rec.off_arc_begin = static_cast<int64_t>(off) + g->off_arc_begin;
+    rec.off_fail = static_cast<int64_t>(off) + g->off_fail;
+    rec.off_bw = static_cast<int64_t>(off) + g->off_bw;
+    rec.off_arc_cls = static_cast<int64_t>(off) + g->off_arc_cls;
+    rec.off_arc_w = static_cast<int64_t>(off) + g->off_arc_w;
+    rec.off_arc_dst = static_cast<int64_t>(off) + g->off_arc_dst;
+    rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
+  }
+  int rc = tb_launch_publish_slot(b->d_slots, b->d_sstate, slot, rec, stream);
+  if (rc != TB_OK) { if (bytes) b->alloc.release(off, bytes); return rc; }
+  // The old block goes back to the free list now; anything that reuses it is enqueued on the
+  // same stream after the decode calls that still read it.
+  auto& blk = b->slot_block[slot];
+  if (blk.second) b->alloc.release(blk.first, blk.second);
+  blk = {off, bytes};
+  return TB_OK;
+}
+
+extern "C" int tb_batch_status(tb_batch* b, int32_t* device_status, void* stream_) {
+  if (!b || !device_status) return TB_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  int32_t st = 0;
+  bool ok = cudaMemcpyAsync(&st, b->d_status, sizeof st, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(b->d_status, 0, sizeof st, stream) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return TB_ERR_CUDA; }
+  *device_status = st;
+  return st == 0 ? TB_OK : TB_ERR_DEVICE_STATUS;
+}
+
+static int fill_decode_params(tb_batch* b, const void* logits, int dtype, int32_t n, int32_t frames, int32_t S,
+                              int32_t n_dur, const int64_t* strides, TbDecodeParams* p) {
+  if (!b || !logits || !strides || (dtype != TB_BF16 && dtype != TB_F32)) return TB_ERR_INVALID_ARG;
+  if (n < 1 || n > b->n_slots || frames < 1 || S < 1 || n_dur < 0 || n_dur > 32) return TB_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(frames) * S > INT32_MAX) return TB_ERR_INVALID_ARG;
+  std::memset(p, 0, sizeof *p);
+  p->logits = logits; p->dtype = dtype; p->n_streams = n; p->frames = frames; p->S = S; p->V = b->vocab;
+  p->n_dur = n_dur; p->C = b->n_classes;
+  p->sb = strides[0]; p->st = strides[1]; p->ss = strides[2]; p->sv = strides[3];
+  p->out_cap = frames * S;
+  p->slots = b->d_slots; p->sstate = b->d_sstate; p->arena = b->arena; p->cls = b->d_cls; p->status = b->d_status;
+  return TB_OK;
+}
+
+extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int32_t B, int32_t T, int32_t S,
+                                const int64_t* strides, const int32_t* lengths, int32_t* out_tokens,
+                                int32_t* out_frames, int32_t* out_counts, float* out_scores, int32_t* out_states,
+                                void* stream_) {
+  TbDecodeParams p;
+  int rc = fill_decode_params(b, logits, dtype, B, T, S, 0, strides, &p);
+  if (rc != TB_OK) return rc;
+  if (!out_tokens || !out_frames || !out_counts || !out_scores || !out_states) return TB_ERR_INVALID_ARG;
+  p.lengths = lengths; p.persistent = 0;
+  p.out_tokens = out_tokens; p.out_frames = out_frames; p.out_counts = out_counts;
+  p.out_scores = out_scores; p.out_states = out_states;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32_t n_slots, int32_t chunk,
+                               int32_t S, int32_t n_dur, const int64_t* strides, const int32_t* valid_frames,
+                               int32_t* out_tokens, int32_t* out_frames, int32_t* out_durs, int32_t* out_counts,
+                               float* out_scores, int32_t* out_states, int32_t* out_cursors, void* stream_) {
+  TbDecodeParams p;
+  int rc = fill_decode_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, &p);
+  if (rc != TB_OK) return rc;
+  if (!valid_frames || !out_tokens || !out_frames || !out_counts || !out_scores || !out_states) return TB_ERR_INVALID_ARG;
+  p.lengths = valid_frames; p.persistent = 1;
+  p.out_tokens = out_tokens; p.out_frames = out_frames; p.out_durs = out_durs; p.out_counts = out_counts;
+  p.out_scores = out_scores; p.out_states = out_states; p.out_cursors = out_cursors;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_beam_reset(tb_batch* b) {
+  if (!b) return TB_ERR_INVALID_ARG;
+  b->tree_steps = 0; b->tree_B = 0; b->tree_K = 0;
+  return TB_OK;
+}
+
+extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t B, int32_t K, int64_t stream_stride,
+                            int64_t hyp_stride, int32_t new_frame, float* scores, int32_t* states, uint8_t* live,
+                            int32_t* out_parent, int32_t* out_token, void* stream_) {
+  if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
+  if ((dtype != TB_BF16 && dtype != TB_F32) || B < 1 || B > b->n_slots || K < 1 || K > b->max_beam) return TB_ERR_INVALID_ARG;
+  if (b->d_tree) {
+    if (b->tree_steps >= b->max_tree_steps) return TB_ERR_INVALID_ARG;
+    if (b->tree_steps > 0 && (b->tree_B != B || b->tree_K != K)) return TB_ERR_INVALID_ARG;
+  }
+  TbBeamParams p;
+  std::memset(&p, 0, sizeof p);
+  p.logits = logits; p.dtype = dtype; p.B = B; p.K = K; p.V = b->vocab; p.C = b->n_classes;
+  p.new_frame = new_frame; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = hyp_stride;
+  p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;
+  p.tree = b->d_tree; p.slots = b->d_slots; p.arena = b->arena; p.cls = b->d_cls; p.status = b->d_status;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  int rc = tb_launch_beam_step(p, static_cast<cudaStream_t>(stream_));
+  if (rc == TB_OK && b->d_tree) { b->tree_steps++; b->tree_B = B; b->tree_K = K; }
+  return rc;
+}
+
+extern "C" int tb_beam_backtrace(tb_batch* b, int32_t B, int32_t K, int32_t max_len, int32_t* out_tokens,
+                                 int32_t* out_lens, void* stream_) {
+  if (!b || !out_tokens || !out_lens || max_len < 1) return TB_ERR_INVALID_ARG;
+  if (!b->d_tree || b->tree_steps == 0 || b->tree_B != B || b->tree_K != K) return TB_ERR_INVALID_ARG;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  return tb_launch_beam_backtrace(b->d_tree, b->tree_steps, B, K, b->vocab, max_len, out_tokens, out_lens,
+                                  static_cast<cudaStream_t>(stream_));
+}

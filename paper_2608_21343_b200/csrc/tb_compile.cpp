@@ -1,0 +1,238 @@
+// Host-side graph compiler: phrase lists -> flat arc/state arrays (Sec. 2.1 para. 1-2, the
+// potential rule above Eq. 1, Sec. 2.2 para. 2).  Sort-based: the case-folded phrases are
+// sorted lexicographically, which makes the distinct prefixes of every length appear in
+// breadth-first order (a state's children in ascending class order), so states and arcs are
+// numbered directly without building a pointer tree.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "tb_internal.h"
+
+namespace {
+
+struct Folded {
+  const int32_t* tok;  // into the caller's array
+  const float* w;      // may be null
+  int32_t len;
+};
+
+inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
+
+template <typename T>
+int64_t append_section(std::vector<unsigned char>& blob, const std::vector<T>& v) {
+  size_t off = align16(blob.size());
+  blob.resize(off + v.size() * sizeof(T));
+  if (!v.empty()) std::memcpy(blob.data() + off, v.data(), v.size() * sizeof(T));
+  return static_cast<int64_t>(off);
+}
+
+}  // namespace
+
+uint64_t tb_hash_class_map(const int32_t* case_class, int32_t vocab) {
+  uint64_t h = 1469598103934665603ull ^ static_cast<uint64_t>(vocab);
+  for (int32_t v = 0; v < vocab; ++v) {
+    uint64_t c = case_class ? static_cast<uint64_t>(case_class[v]) : static_cast<uint64_t>(v);
+    h = (h ^ c) * 1099511628211ull;
+  }
+  return h;
+}
+
+extern "C" const char* tb_strerror(int code) {
+  switch (code) {
+    case TB_OK: return "ok";
+    case TB_ERR_INVALID_ARG: return "invalid argument";
+    case TB_ERR_OOM: return "out of memory";
+    case TB_ERR_CUDA: return "CUDA runtime error";
+    case TB_ERR_ARENA_FULL: return "graph arena full";
+    case TB_ERR_BAD_SLOT: return "slot index out of range";
+    case TB_ERR_DEVICE_STATUS: return "a kernel recorded a violated bound";
+    default: return "unknown error";
+  }
+}
+
+static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,
+                        const float* token_weights, const int32_t* case_class, int32_t vocab, float lambda,
+                        tb_graph* g) {
+  // ---- validation -------------------------------------------------------------------------
+  int32_t n_classes = vocab;
+  if (case_class) {
+    n_classes = 0;
+    for (int32_t v = 0; v < vocab; ++v) {
+      if (case_class[v] < 0) return TB_ERR_INVALID_ARG;
+      n_classes = std::max(n_classes, case_class[v] + 1);
+    }
+  }
+  if (n_phrases > 0 && phrase_offsets[0] != 0) return TB_ERR_INVALID_ARG;
+  std::vector<Folded> ph;
+  ph.reserve(n_phrases);
+  int32_t max_len = 0;
+  for (int32_t p = 0; p < n_phrases; ++p) {
+    int64_t b = phrase_offsets[p], e = phrase_offsets[p + 1];
+    if (e < b) return TB_ERR_INVALID_ARG;
+    if (e - b > TB_MAX_PHRASE_LEN) return TB_ERR_INVALID_ARG;
+    for (int64_t i = b; i < e; ++i) {
+      if (phrase_tokens[i] < 0 || phrase_tokens[i] >= vocab) return TB_ERR_INVALID_ARG;
+      if (token_weights && !(std::isfinite(token_weights[i]) && token_weights[i] >= 0.0f)) return TB_ERR_INVALID_ARG;
+    }
+    if (e == b) continue;  // empty phrases are skipped
+    ph.push_back({phrase_tokens + b, token_weights ? token_weights + b : nullptr, static_cast<int32_t>(e - b)});
+    max_len = std::max(max_len, static_cast<int32_t>(e - b));
+  }
+  auto cls_of = [&](int32_t tok) { return case_class ? case_class[tok] : tok; };
+
+  // ---- sort the folded phrases, longest-common-prefix with the predecessor -----------------
+  const size_t P = ph.size();
+  std::vector<uint32_t> order(P);
+  std::iota(order.begin(), order.end(), 0u);
+  std::sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+    const Folded &x = ph[a], &y = ph[b];
+    int32_t n = std::min(x.len, y.len);
+    for (int32_t i = 0; i < n; ++i) {
+      int32_t cx = cls_of(x.tok[i]), cy = cls_of(y.tok[i]);
+      if (cx != cy) return cx < cy;
+    }
+    return x.len < y.len;
+  });
+  std::vector<int32_t> lcp(P, 0);
+  std::vector<size_t> node_base(P + 1, 0);  // where phrase i's node ids start in `node_of`
+  for (size_t i = 0; i < P; ++i) {
+    const Folded& x = ph[order[i]];
+    node_base[i + 1] = node_base[i] + x.len;
+    if (i == 0) continue;
+    const Folded& y = ph[order[i - 1]];
+    int32_t n = std::min(x.len, y.len), l = 0;
+    while (l < n && cls_of(x.tok[l]) == cls_of(y.tok[l])) ++l;
+    lcp[i] = l;
+  }
+
+  // ---- states: distinct prefixes, depth by depth = breadth-first order ----------------------
+  std::vector<int32_t> node_of(node_base[P]);   // node id of phrase i's prefix of length d+1
+  std::vector<int32_t> parent(1, -1), cls(1, -1);
+  std::vector<uint8_t> depth(1, 0), is_end(1, 0);
+  std::vector<double> wt(1, 0.0);
+  for (int32_t d = 1; d <= max_len; ++d) {
+    for (size_t i = 0; i < P; ++i) {
+      const Folded& x = ph[order[i]];
+      if (x.len < d) continue;
+      double w = x.w ? static_cast<double>(x.w[d - 1]) : 1.0;
+      int32_t id;
+      if (lcp[i] >= d) {  // same prefix as the predecessor, which therefore has this node
+        id = node_of[node_base[i - 1] + d - 1];
+        wt[id] = std::max(wt[id], w);
+      } else {
+        id = static_cast<int32_t>(parent.size());
+        parent.push_back(d == 1 ? 0 : node_of[node_base[i] + d - 2]);
+        cls.push_back(cls_of(x.tok[d - 1]));
+        depth.push_back(static_cast<uint8_t>(d));
+        is_end.push_back(0);
+        wt.push_back(w);
+      }
+      node_of[node_base[i] + d - 1] = id;
+      if (x.len == d) is_end[id] = 1;
+    }
+  }
+  const int32_t N = static_cast<int32_t>(parent.size());
+  const int32_t A = N - 1;
+
+  // ---- arcs: arc a enters state a+1; a state's arcs are contiguous --------------------------
+  g->n_states = N; g->n_arcs = A; g->n_classes = n_classes; g->vocab = vocab;
+  g->max_depth = max_len; g->lambda = lambda;
+  g->state_arc_begin.assign(N + 1, 0);
+  g->arc_class.resize(A); g->arc_dst.resize(A); g->arc_w.resize(A);
+  g->state_fail.assign(N, 0); g->state_bw.assign(N, 0.0f); g->state_final.assign(N, 0.0f);
+  g->state_depth.assign(depth.begin(), depth.end());
+  for (int32_t id = 1; id < N; ++id) {
+    g->state_arc_begin[parent[id] + 1]++;
+    g->arc_class[id - 1] = cls[id];
+    g->arc_dst[id - 1] = id;
+  }
+  for (int32_t u = 0; u < N; ++u) g->state_arc_begin[u + 1] += g->state_arc_begin[u];
+
+  auto find_arc = [&](int32_t u, int32_t c) -> int32_t {
+    const int32_t* b = g->arc_class.data() + g->state_arc_begin[u];
+    const int32_t* e = g->arc_class.data() + g->state_arc_begin[u + 1];
+    const int32_t* it = std::lower_bound(b, e, c);
+    return (it != e && *it == c) ? static_cast<int32_t>(it - g->arc_class.data()) : -1;
+  };
+
+  // ---- suffix links (ids ascend breadth-first, so the parent's link is ready) ---------------
+  for (int32_t id = 1; id < N; ++id) {
+    int32_t f = 0;
+    if (parent[id] != 0) {
+      int32_t q = g->state_fail[parent[id]];
+      for (;;) {
+        int32_t a = find_arc(q, cls[id]);
+        if (a >= 0) { f = g->arc_dst[a]; break; }
+        if (q == 0) break;
+        q = g->state_fail[q];
+      }
+    }
+    g->state_fail[id] = f;
+  }
+
+  // ---- potentials in double, stored values rounded once --------------------------------------
+  // loan: credit of the partial match since the last completed phrase (returned on back-off);
+  // outp: everything banked on arriving at a state (phrases ending there, own or as suffixes).
+  std::vector<double> loan(N, 0.0), outp(N, 0.0);
+  for (int32_t id = 1; id < N; ++id) {
+    double through = loan[parent[id]] + wt[id];
+    loan[id] = is_end[id] ? 0.0 : through;
+    outp[id] = (is_end[id] ? through : 0.0) + outp[g->state_fail[id]];
+  }
+  for (int32_t id = 0; id < N; ++id) {
+    g->state_final[id] = static_cast<float>(-loan[id]);
+    if (id) {
+      g->state_bw[id] = static_cast<float>(loan[g->state_fail[id]] - loan[id]);
+      g->arc_w[id - 1] = static_cast<float>(loan[id] - loan[parent[id]] + outp[id]);
+    }
+  }
+  g->case_class.resize(vocab);
+  for (int32_t v = 0; v < vocab; ++v) g->case_class[v] = cls_of(v);
+  g->class_map_hash = tb_hash_class_map(case_class, vocab);
+
+  // ---- device blob ---------------------------------------------------------------------------
+  g->blob.clear();
+  g->off_arc_begin = append_section(g->blob, g->state_arc_begin);
+  g->off_fail = append_section(g->blob, g->state_fail);
+  g->off_bw = append_section(g->blob, g->state_bw);
+  g->off_arc_cls = append_section(g->blob, g->arc_class);
+  g->off_arc_w = append_section(g->blob, g->arc_w);
+  g->off_arc_dst = append_section(g->blob, g->arc_dst);
+  g->blob.resize(align16(g->blob.size()) + 16);  // tail padding so vector loads may overrun a section
+  return TB_OK;
+}
+
+extern "C" int tb_graph_compile(const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,
+                                const float* token_weights, const int32_t* case_class, int32_t vocab,
+                                float lambda, uint32_t flags, tb_graph** out) {
+  if (!out) return TB_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (flags != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda)) return TB_ERR_INVALID_ARG;
+  if (n_phrases > 0 && (!phrase_offsets || (phrase_offsets[n_phrases] > 0 && !phrase_tokens))) return TB_ERR_INVALID_ARG;
+  try {
+    tb_graph* g = new tb_graph();
+    int rc = compile_impl(phrase_tokens, phrase_offsets, n_phrases, token_weights, case_class, vocab, lambda, g);
+    if (rc != TB_OK) { delete g; return rc; }
+    *out = g;
+    return TB_OK;
+  } catch (const std::bad_alloc&) {
+    return TB_ERR_OOM;
+  }
+}
+
+extern "C" int tb_graph_view_get(const tb_graph* g, tb_graph_view* out) {
+  if (!g || !out) return TB_ERR_INVALID_ARG;
+  out->n_states = g->n_states; out->n_arcs = g->n_arcs; out->n_classes = g->n_classes;
+  out->vocab = g->vocab; out->max_depth = g->max_depth; out->lambda = g->lambda;
+  out->state_arc_begin = g->state_arc_begin.data(); out->arc_class = g->arc_class.data();
+  out->arc_dst = g->arc_dst.data(); out->arc_w = g->arc_w.data();
+  out->state_fail = g->state_fail.data(); out->state_bw = g->state_bw.data();
+  out->state_final = g->state_final.data(); out->state_depth = g->state_depth.data();
+  out->case_class = g->case_class.data();
+  return TB_OK;
+}
+
+extern "C" void tb_graph_free(tb_graph* g) { delete g; }

@@ -1,0 +1,40 @@
+// Kernel parameter blocks and launch entry points (host side of the kernels).
+#ifndef TB_LAUNCH_H_
+#define TB_LAUNCH_H_
+
+#include <cuda_runtime.h>
+
+#include "tb_internal.h"
+
+struct TbDecodeParams {
+  const void* logits;        // device
+  int dtype;                 // TB_BF16 / TB_F32
+  int32_t n_streams, frames, S, V, n_dur, C;
+  int64_t sb, st, ss, sv;    // element strides: stream, frame, row-in-frame, token
+  const int32_t* lengths;    // device [n_streams] or null
+  int32_t persistent;        // 0: offline greedy (fresh state); 1: streaming (TbSlotState)
+  int32_t* out_tokens; int32_t* out_frames; int32_t* out_durs; int32_t* out_counts;
+  float* out_scores; int32_t* out_states; int32_t* out_cursors;
+  int32_t out_cap;           // tokens per stream the output arrays can hold
+  const TbSlotRec* slots; TbSlotState* sstate; const unsigned char* arena;
+  const int32_t* cls;        // device [V] token -> class
+  int32_t* status;
+};
+
+struct TbBeamParams {
+  const void* logits; int dtype;
+  int32_t B, K, V, C, new_frame, step;
+  int64_t stream_stride, hyp_stride;
+  float* scores; int32_t* states; uint8_t* live; int32_t* out_parent; int32_t* out_token;
+  int2* tree;                // [steps, B, K] (parent, token) or null
+  const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
+};
+
+int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
+int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
+int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
+                             int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
+int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
+                           cudaStream_t stream);
+
+#endif  // TB_LAUNCH_H_

@@ -1,0 +1,164 @@
+"""GPU parity for tb_beam_step / tb_beam_backtrace and tb_stream_chunk against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_21343_b200 import workloads as W
+from helpers import SCORE_TOL, make_batch, oracle_graph, to_device, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_beam(tb, w, data, K, phrase_lists=None):
+    """Frame-synchronous driver: E = w.S rows per frame shared by all hypotheses of a stream."""
+    phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
+    B, T, E, Wd = data["logits"].shape
+    batch, _ = make_batch(tb, w, phrase_lists, max_beam=K, max_tree_steps=T * E)
+    logits = to_device(data["logits"])
+    dev = logits.device
+    scores = torch.full((B, K), float("-inf"), device=dev)
+    scores[:, 0] = 0.0
+    states = torch.full((B, K), -1, dtype=torch.int32, device=dev)
+    states[:, 0] = torch.tensor([0 if p is not None else -1 for p in phrase_lists], dtype=torch.int32, device=dev)
+    live = torch.zeros((B, K), dtype=torch.uint8, device=dev)
+    par = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tok = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tb.tb_beam_reset(batch)
+    tree = []
+    sb, st, se, _ = logits.stride()
+    for t in range(T):
+        for e in range(E):
+            tb.tb_beam_step(batch, logits, sb, 0, e == 0, scores, states, live, par, tok, offset=t * st + e * se)
+            tree.append(torch.stack([par, tok], dim=-1).clone())
+    toks, lens = tb.tb_beam_backtrace(batch, B, K, T * E)
+    assert tb.tb_batch_status(batch) == 0
+    torch.cuda.synchronize()
+    return dict(scores=scores.cpu().numpy(), states=states.cpu().numpy(), live=live.cpu().numpy(),
+                tree=torch.stack(tree, dim=1).cpu().numpy(), tokens=toks.cpu().numpy(), lens=lens.cpu().numpy())
+
+
+def compare_beam(w, data, out, K, streams, phrase_lists=None):
+    phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
+    for i in streams:
+        ref = O.beam_decode(oracle_graph(w, phrase_lists[i]), data["logits"][i], K)
+        assert np.array_equal(out["tree"][i], ref["tree"]), f"stream {i}: (parent, token) tree"
+        assert np.array_equal(out["states"][i], ref["states"]), f"stream {i}: states"
+        assert np.array_equal(out["lens"][i], ref["lens"]), f"stream {i}: lengths"
+        for k in range(K):
+            assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k]), f"stream {i} hyp {k}"
+        fin = np.isfinite(ref["scores"])
+        assert np.array_equal(np.isfinite(out["scores"][i]), fin)
+        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL), f"stream {i}: scores"
+
+
+def test_workload4_beam_reduced(tb):
+    w = W.get_workload(4, B=5, T=60, n_plants=6)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[2] = None
+    out = run_beam(tb, w, data, w.K, lists)
+    compare_beam(w, data, out, w.K, range(w.B), lists)
+
+
+@pytest.mark.parametrize("K", [1, 2, 7])
+def test_beam_other_widths_fp32(tb, K):
+    w = W.get_workload(1, B=3, T=25, S=2)
+    data = W.batch_inputs(w)
+    out = run_beam(tb, w, data, K)
+    compare_beam(w, data, out, K, range(w.B))
+    if K == 1:       # a beam of one is greedy decoding
+        for i in range(w.B):
+            ref = O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i])
+            n = len(ref["tokens"])
+            assert out["lens"][i, 0] == n and np.array_equal(out["tokens"][i, 0, :n], ref["tokens"])
+
+
+def test_workload4_full_size_sampled_streams(tb):
+    w = W.get_workload(4)
+    data = W.batch_inputs(w)
+    out = run_beam(tb, w, data, w.K)
+    compare_beam(w, data, out, w.K, [0, 13, 31])
+
+
+def test_beam_step_frozen_and_empty(tb):
+    """One step by hand: ordering of equal scores, a frozen hypothesis carried, empty places."""
+    w = W.get_workload(1, B=1, T=1)
+    batch, _ = make_batch(tb, w, [[[0]]], max_beam=3)
+    V = w.V
+    rows = torch.full((1, 3, V + 1), -5.0, device="cuda:0")
+    rows[0, 0, 0] = 1.0           # +1 bonus for class 0 -> 2.0
+    rows[0, 0, 4] = 2.0
+    rows[0, 0, V] = 2.0
+    rows[0, 1, :] = 9.0           # frozen hypothesis: its row must not be read
+    scores = torch.tensor([[0.0, 2.0, float("-inf")]], device="cuda:0")
+    states = torch.tensor([[0, 0, -1]], dtype=torch.int32, device="cuda:0")
+    live = torch.tensor([[1, 0, 0]], dtype=torch.uint8, device="cuda:0")
+    par = torch.empty((1, 3), dtype=torch.int32, device="cuda:0")
+    tok = torch.empty((1, 3), dtype=torch.int32, device="cuda:0")
+    tb.tb_beam_step(batch, rows, 3 * (V + 1), V + 1, False, scores, states, live, par, tok)
+    torch.cuda.synchronize()
+    assert par.tolist() == [[0, 0, 0]] and tok.tolist() == [[0, 4, V]]
+    assert scores.tolist() == [[2.0, 2.0, 2.0]] and states.tolist() == [[1, 0, 0]] and live.tolist() == [[1, 1, 0]]
+    ref_scores = np.array([0.0, 2.0, -np.inf], dtype=np.float32)
+    ref_states = np.array([0, 0, -1], dtype=np.int32)
+    ref_live = np.array([1, 0, 0], dtype=np.uint8)
+    rp, rt = O.beam_step(O.Graph([[0]], V, case_class=w.vocab.case_class), rows[0].cpu().numpy(), ref_scores, ref_states, ref_live)
+    assert rp.tolist() == [0, 0, 0] and rt.tolist() == [0, 4, V]
+
+
+def run_stream(tb, w, n_chunks, weights_lam=None):
+    """Streaming decode with stream churn on both sides; compares after every chunk."""
+    sched_gpu = W.ChurnSchedule(w)
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=8 << 20)
+    slots = [dict(graph=None, st=None, t0=0) for _ in range(w.B)]
+    n_binds = 0
+    for c in range(n_chunks):
+        chunk, lengths, binds = sched_gpu.next_chunk()
+        for slot, stream_id, phrases in binds:
+            g = tb.tb_graph_compile(phrases, w.V, case_class=w.vocab.case_class)
+            tb.tb_batch_bind_stream(batch, slot, g)
+            og = oracle_graph(w, phrases)
+            slots[slot] = dict(graph=og, st=O.StreamState(0, 0, 0, 0.0, 0), t0=0)
+            n_binds += 1
+        out = to_host(tb.tb_stream_chunk(batch, to_device(chunk), w.n_dur,
+                                         torch.from_numpy(lengths).to("cuda:0")))
+        for i in range(w.B):
+            sl = slots[i]
+            ref = O.stream_chunk(sl["graph"], chunk[i], w.n_dur, sl["t0"], int(lengths[i]), sl["st"])
+            sl["t0"] += w.chunk
+            n = int(out["counts"][i])
+            assert n == len(ref["tokens"]), (c, i)
+            assert np.array_equal(out["tokens"][i, :n], ref["tokens"]), (c, i)
+            assert np.array_equal(out["frames"][i, :n], ref["frames"]), (c, i)
+            assert np.array_equal(out["durs"][i, :n], ref["durs"]), (c, i)
+            assert out["states"][i] == sl["st"].state and out["cursors"][i] == sl["st"].t, (c, i)
+            assert abs(float(out["scores"][i]) - float(sl["st"].score)) <= SCORE_TOL, (c, i)
+    assert tb.tb_batch_status(batch) == 0
+    return n_binds
+
+
+def test_workload5_streaming_tdt_with_churn_reduced(tb):
+    w = W.get_workload(5, B=12, T=90, T_lo=20, n_phrases=60, n_phrases_lo=10)
+    n_binds = run_stream(tb, w, n_chunks=30)
+    assert n_binds > 2 * w.B          # slots were refilled while others kept running
+
+
+def test_streaming_rnnt_chunked_equals_offline(tb):
+    """Sec. 2.3: state carried across chunk boundaries -- chunks of 8 frames give the offline result."""
+    w = W.get_workload(2, B=4, T=64, n_phrases=50, n_plants=6)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    logits = to_device(data["logits"])
+    off = to_host(tb.tb_greedy_decode(batch, logits))
+    valid = torch.full((w.B,), w.T, dtype=torch.int32, device="cuda:0")
+    toks = [[] for _ in range(w.B)]
+    for c in range(0, w.T, 8):
+        out = to_host(tb.tb_stream_chunk(batch, logits[:, c:c + 8], 0, valid))
+        for i in range(w.B):
+            toks[i] += list(zip(out["tokens"][i, :out["counts"][i]], out["frames"][i, :out["counts"][i]]))
+    for i in range(w.B):
+        n = int(off["counts"][i])
+        assert toks[i] == list(zip(off["tokens"][i, :n], off["frames"][i, :n]))
+        assert out["states"][i] == off["states"][i] and out["scores"][i] == off["scores"][i]
+        assert out["cursors"][i] == w.T

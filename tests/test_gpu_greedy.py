@@ -1,0 +1,173 @@
+"""GPU parity, greedy RNNT (tb_greedy_decode) against the CPU oracle on the same seeded inputs:
+tokens, frames and graph states bit-exact, scores within 1e-4 absolute."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_21343_b200 import workloads as W
+from helpers import SCORE_TOL, check_greedy, make_batch, oracle_graph, to_device, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_compare(tb, w, data, lengths=None, phrase_lists=None, weights=None, lam=None, what=""):
+    phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
+    batch, _ = make_batch(tb, w, phrase_lists, weights=weights, lam=lam)
+    logits = to_device(data["logits"])
+    dl = None if lengths is None else torch.tensor(lengths, dtype=torch.int32, device="cuda:0")
+    out = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(phrase_lists):
+        g = oracle_graph(w, p, None if weights is None else weights[i], lam)
+        ref = O.greedy_rnnt(g, data["logits"][i], None if lengths is None else lengths[i])
+        check_greedy(out, i, ref, what)
+    return out, batch
+
+
+def test_workload1_tiny_greedy_full(tb):
+    w = W.get_workload(1)
+    data = W.batch_inputs(w)
+    out, _ = run_and_compare(tb, w, data, what="w1")
+    assert out["counts"].min() > 5
+    # per-stream independence (Sec. 2.2 para. 3): each stream alone gives the same result
+    for i in range(w.B):
+        batch1, _ = make_batch(tb, w, [data["phrases"][i]])
+        solo = to_host(tb.tb_greedy_decode(batch1, to_device(data["logits"][i:i + 1])))
+        n = int(out["counts"][i])
+        assert int(solo["counts"][0]) == n
+        assert np.array_equal(solo["tokens"][0, :n], out["tokens"][i, :n])
+        assert np.array_equal(solo["frames"][0, :n], out["frames"][i, :n])
+        assert solo["states"][0] == out["states"][i] and solo["scores"][0] == out["scores"][i]
+
+
+def test_workload2_reduced_and_unbound_mix(tb):
+    w = W.get_workload(2, B=12, T=160)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[3] = None            # model id -1
+    lists[7] = []              # an empty list: root only
+    out, _ = run_and_compare(tb, w, data, phrase_lists=lists, what="w2r")
+    assert out["states"][3] == -1
+
+
+def test_workload2_full_size_sampled_streams(tb):
+    """The benchmark's configuration (B=128, T=750, bf16): every stream decoded on the GPU,
+    a sample of streams decoded one by one by the oracle."""
+    w = W.get_workload(2)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    logits = to_device(data["logits"])
+    out = to_host(tb.tb_greedy_decode(batch, logits))
+    assert tb.tb_batch_status(batch) == 0
+    for i in list(range(0, w.B, 9)) + [w.B - 1]:
+        ref = O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i])
+        check_greedy(out, i, ref, "w2")
+    # unboosted: every slot unbound
+    for i in range(w.B):
+        tb.tb_batch_bind_stream(batch, i, None)
+    out0 = to_host(tb.tb_greedy_decode(batch, logits))
+    for i in (0, 64, 127):
+        check_greedy(out0, i, O.greedy_rnnt(None, data["logits"][i]), "w2-unboosted")
+    assert (out0["states"] == -1).all()
+
+
+def test_workload3_large_lists(tb):
+    w = W.get_workload(3, B=3, T=300)
+    data = W.batch_inputs(w)
+    out, _ = run_and_compare(tb, w, data, what="w3")
+
+
+@pytest.mark.parametrize("lam", [0.5, 2.0, 0.0])
+def test_weighted_lists_and_lambda(tb, lam):
+    w = W.get_workload(2, B=5, T=120, n_phrases=40)
+    data = W.batch_inputs(w)
+    rng = np.random.default_rng(1)
+    weights = [[[float(rng.choice([0.5, 1.0, 1.5, 2.0])) for _ in p] for p in lst] for lst in data["phrases"]]
+    run_and_compare(tb, w, data, weights=weights, lam=lam, what=f"lam{lam}")
+
+
+def test_lengths_strides_and_edges(tb):
+    w = W.get_workload(1, B=5, T=40)
+    data = W.batch_inputs(w)
+    lengths = [40, 0, 1, 17, 39]
+    run_and_compare(tb, w, data, lengths=lengths, what="lengths")
+    # non-contiguous logits: rows padded to 272 elements, streams reversed in memory
+    batch, _ = make_batch(tb, w, data["phrases"])
+    big = torch.zeros((w.B, w.T, w.S, 272), dtype=torch.float32, device="cuda:0")
+    big[..., 5:5 + w.V + 1] = to_device(data["logits"])
+    view = big[..., 5:5 + w.V + 1]
+    assert not view.is_contiguous()
+    out = to_host(tb.tb_greedy_decode(batch, view))
+    for i in range(w.B):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]), "strided")
+    # S = 1 and T = 1
+    for T, S in ((1, 3), (9, 1)):
+        w2 = W.get_workload(1, B=2, T=T, S=S, n_plants=0)
+        d2 = W.batch_inputs(w2)
+        run_and_compare(tb, w2, d2, what=f"T{T}S{S}")
+
+
+def test_exact_ties_go_to_lowest_id(tb):
+    w = W.get_workload(1, B=2, T=30, n_plants=0)
+    data = W.batch_inputs(w)
+    x = data["logits"]
+    x[:, ::2, 0, :] = np.round(x[:, ::2, 0, :] * 2) / 2           # coarse grid: many exact ties
+    x[0, 1, 0, 10] = x[0, 1, 0, 200] = x[0, 1, 0, w.V] = 9.0      # token tie that also ties with blank
+    run_and_compare(tb, w, data, what="ties")
+
+
+def test_rebind_one_slot_leaves_others_alone(tb):
+    """Sec. 2.2 para. 4: lists are swapped while other streams keep theirs."""
+    w = W.get_workload(2, B=6, T=100)
+    data = W.batch_inputs(w)
+    batch, graphs = make_batch(tb, w, data["phrases"], arena_bytes=1 << 20)
+    logits = to_device(data["logits"])
+    before = to_host(tb.tb_greedy_decode(batch, logits))
+    other = W.stream_phrases(w, 77)
+    g_new = tb.tb_graph_compile(other, w.V, case_class=w.vocab.case_class)
+    tb.tb_batch_bind_stream(batch, 2, g_new)
+    g_new.free()                                   # bind copied what it needs
+    tb.tb_batch_bind_stream(batch, 4, None)
+    after = to_host(tb.tb_greedy_decode(batch, logits))
+    for i in (0, 1, 3, 5):
+        for k in before:
+            assert np.array_equal(before[k][i], after[k][i]), (i, k)
+    check_greedy(after, 2, O.greedy_rnnt(oracle_graph(w, other), data["logits"][2]), "rebound")
+    check_greedy(after, 4, O.greedy_rnnt(None, data["logits"][4]), "unbound")
+    # churn the arena: many swaps into a small arena must keep working (free list reuse)
+    for r in range(40):
+        g = tb.tb_graph_compile(W.stream_phrases(w, 100 + r), w.V, case_class=w.vocab.case_class)
+        tb.tb_batch_bind_stream(batch, r % w.B, g)
+    final = to_host(tb.tb_greedy_decode(batch, logits))
+    for i in range(w.B):
+        r = max(r for r in range(40) if r % w.B == i)
+        check_greedy(final, i, O.greedy_rnnt(oracle_graph(w, W.stream_phrases(w, 100 + r)), data["logits"][i]), "churn")
+
+
+def test_error_codes(tb):
+    w = W.get_workload(1, B=2, T=8)
+    data = W.batch_inputs(w)
+    batch, graphs = make_batch(tb, w, data["phrases"], arena_bytes=4096)
+
+    def code(fn, *a, **k):
+        with pytest.raises(tb.TbError) as e:
+            fn(*a, **k)
+        return e.value.code
+    assert code(tb.tb_batch_bind_stream, batch, 2, graphs[0]) == tb.TB_ERR_BAD_SLOT
+    assert code(tb.tb_batch_bind_stream, batch, -1, graphs[0]) == tb.TB_ERR_BAD_SLOT
+    other_vocab = tb.tb_graph_compile([[1, 2]], w.V - 1)
+    assert code(tb.tb_batch_bind_stream, batch, 0, other_vocab) == tb.TB_ERR_INVALID_ARG
+    other_map = tb.tb_graph_compile([[1, 2]], w.V)          # identity class map
+    assert code(tb.tb_batch_bind_stream, batch, 0, other_map) == tb.TB_ERR_INVALID_ARG
+    big = tb.tb_graph_compile(W.stream_phrases(W.get_workload(1, n_phrases=400), 0), w.V, case_class=w.vocab.case_class)
+    logits = to_device(data["logits"])
+    before = to_host(tb.tb_greedy_decode(batch, logits))
+    assert code(tb.tb_batch_bind_stream, batch, 0, big) == tb.TB_ERR_ARENA_FULL
+    after = to_host(tb.tb_greedy_decode(batch, logits))       # a failed bind changes nothing
+    for k in before:
+        assert np.array_equal(before[k], after[k])
+    three = torch.zeros((3, 8, 3, w.V + 1), device="cuda:0")
+    assert code(tb.tb_greedy_decode, batch, three) == tb.TB_ERR_INVALID_ARG   # B > n_slots
+    assert code(tb.tb_batch_create, 0, None, 1) == tb.TB_ERR_INVALID_ARG
+    assert code(tb.tb_batch_create, 8, None, 1, max_beam=99) == tb.TB_ERR_INVALID_ARG

@@ -1,0 +1,90 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, and its graph compiler emits arrays identical to the oracle's compiler (both
+use the breadth-first canonical numbering, so equality is element for element)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2608_21343_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ARRAYS = ("state_arc_begin", "arc_class", "arc_dst", "arc_w", "state_fail", "state_bw", "state_final",
+          "state_depth", "case_class")
+
+
+def declared_functions():
+    names = []
+    for fn in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names += re.findall(r"\b(tb_[a-z_0-9]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol(tb):
+    lib = ctypes.CDLL(tb.LIB_PATH)
+    names = declared_functions()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(tb.EXPORTED)
+    assert tb.tb_strerror(0) == "ok" and "arena" in tb.tb_strerror(tb.TB_ERR_ARENA_FULL)
+
+
+def assert_same_graph(tb, phrases, V, cc, weights=None, lam=1.0):
+    go = O.Graph(phrases, V, case_class=cc, weights=weights, lam=lam)
+    gl = tb.tb_graph_compile(phrases, V, case_class=cc, token_weights=weights, lam=lam).view()
+    for k in ("n_states", "n_arcs", "n_classes", "vocab", "max_depth"):
+        assert gl[k] == getattr(go, k), k
+    assert gl["lam"] == go.lam
+    for k in ARRAYS:
+        a, b = gl[k], getattr(go, k)
+        assert a.dtype == b.dtype and a.shape == b.shape and a.tobytes() == b.tobytes(), k
+    return go
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_compiler_matches_oracle_random_lists(tb, seed):
+    rng = np.random.default_rng(seed)
+    V = int(rng.integers(3, 40))
+    cc = None if seed % 3 == 0 else rng.integers(0, max(1, V // 2), size=V).astype(np.int32)
+    n = int(rng.integers(0, 60))
+    phrases = [[int(t) for t in rng.integers(0, V, size=rng.integers(0, 7))] for _ in range(n)]
+    weights = None
+    if seed % 2:
+        weights = [[float(rng.choice([0.25, 0.5, 1.0, 1.3, 2.0])) for _ in p] for p in phrases]
+    assert_same_graph(tb, phrases, V, cc, weights, lam=[1.0, 0.5, 2.0][seed % 3])
+
+
+def test_compiler_matches_oracle_on_workload_lists(tb):
+    for cid, b in ((1, 0), (1, 3), (2, 5), (4, 1), (5, 7)):
+        w = W.get_workload(cid)
+        g = assert_same_graph(tb, W.stream_phrases(w, b), w.V, w.vocab.case_class)
+        assert g.n_states > 10
+    w = W.get_workload(3)
+    g = assert_same_graph(tb, W.stream_phrases(w, 2), w.V, w.vocab.case_class)
+    assert 15000 < g.n_states < 40000          # "about 20-30k states and arcs per stream"
+
+
+def test_compile_error_codes(tb):
+    def code(*a, **k):
+        with pytest.raises(tb.TbError) as e:
+            tb.tb_graph_compile(*a, **k)
+        return e.value.code
+    assert code([[0, 9]], 4) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, -1]], 4) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, token_weights=[[1.0, -1.0]]) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, token_weights=[[1.0, float("inf")]]) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, case_class=[0, -2, 1, 1]) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, lam=float("nan")) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 0) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 100000) == tb.TB_ERR_INVALID_ARG
+    assert code([[0] * 300], 4) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, flags=1) == tb.TB_ERR_INVALID_ARG
+    g = tb.tb_graph_compile([], 4).view()
+    assert g["n_states"] == 1 and g["n_arcs"] == 0
