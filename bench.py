@@ -226,13 +226,14 @@ def main():
         "graph_compile_ms_per_list": compile_s * 1e3 / w.B,
     }
 
-    if not args.no_extras and rank == 0:
+    if rank == 0:
         # unboosted: the same call with every slot unbound
         out0 = tb.tb_greedy_decode(plain, logits)
         p_ms, _ = timed(lambda: tb.tb_greedy_decode(plain, logits, out=out0), args.steps, args.warmup)
         p_ms /= args.steps
         result["unboosted"] = {"ms_per_step": p_ms, "frames_per_s": w.B * w.T / (p_ms * 1e-3),
                                "boosted_overhead_pct": 100.0 * (total_ms / args.steps / p_ms - 1.0)}
+    if not args.no_extras and rank == 0:
         # end to end through the public call with host buffers: H2D of the logits, decode, D2H of results
         dl = torch.empty_like(logits)
         host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}

@@ -54,6 +54,9 @@ extern "C" {
 #define TB_STATUS_STEP_LIMIT 4      /* a decode loop hit its static iteration bound */
 #define TB_STATUS_WAIT_TIMEOUT 8    /* a bounded wait inside a kernel ran out */
 
+/* tb_batch_set_flags */
+#define TB_FLAG_GENERAL_KERNELS 1   /* always use the general decode kernel (any layout), never the pipelined one */
+
 /* Limits of this build. */
 #define TB_MAX_VOCAB 8192           /* non-blank tokens */
 #define TB_MAX_PHRASE_LEN 255       /* tokens per phrase (graph depth is stored in a byte) */
@@ -146,6 +149,15 @@ void tb_batch_destroy(tb_batch *b);
 int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *stream);
 
 /*
+ * Set behaviour flags of the batch (TB_FLAG_*; 0 = defaults).  With the defaults
+ * tb_greedy_decode picks the pipelined kernel whenever the call fits it (bf16 logits, token
+ * stride 1, the S rows of a frame contiguous, vocab <= 2048, S <= 4) and the general kernel
+ * otherwise; both give identical results.  The paper has no counterpart of this call.
+ * Errors: TB_ERR_INVALID_ARG (unknown bits).
+ */
+int tb_batch_set_flags(tb_batch *b, uint32_t flags);
+
+/*
  * Copy the device status word to *device_status (host) after synchronising `stream`, and
  * clear it.  Returns TB_OK if it was 0, else TB_ERR_DEVICE_STATUS (bits: TB_STATUS_*).
  */
@@ -180,8 +192,8 @@ int tb_greedy_decode(tb_batch *b, const void *logits, int dtype, int32_t B, int3
  * from and updating each slot's persistent state {graph state, frame cursor, symbols in the
  * current frame, score, emitted count} (Sec. 2.3: decoding state is kept across chunk
  * boundaries; Sec. 2.2 para. 4: slots are re-bound between chunks).  The call covers the
- * slot's frames [c, c + chunk), c = chunk * (number of tb_stream_chunk calls since the
- * slot's last bind... counted per slot); frames at or beyond valid_frames[slot] are not
+ * slot's frames [c, c + chunk), c = the number of frames that earlier
+ * tb_stream_chunk calls covered since the slot's last bind; frames at or beyond valid_frames[slot] are not
  * decoded; a cursor that a TDT duration moved beyond the chunk is carried over.
  * TDT row: vocab+1 token logits, then n_dur duration logits for durations 0..n_dur-1; the
  * duration is their argmax (lowest on ties); score += value[token] + x_dur[duration];

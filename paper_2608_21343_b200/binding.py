@@ -12,7 +12,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtb.so")
+LIB_PATH = os.environ.get("TB_LIB_PATH") or os.path.join(_HERE, "libtb.so")
 
 if not os.path.exists(LIB_PATH):
     raise RuntimeError(
@@ -53,6 +53,7 @@ _SIGS = {
     "tb_batch_destroy": (None, [_vp]),
     "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
     "tb_batch_status": (C.c_int, [_vp, C.POINTER(_i32), _vp]),
+    "tb_batch_set_flags": (C.c_int, [_vp, C.c_uint32]),
     "tb_greedy_decode": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_stream_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                   _vp, _vp, _vp]),
@@ -129,7 +130,7 @@ class Graph:
             case_class=arr(v.case_class, v.vocab, np.int32))
 
     def free(self):
-        if self.handle:
+        if self.handle and _lib is not None:
             _lib.tb_graph_free(self.handle)
             self.handle = None
 
@@ -164,7 +165,7 @@ class Batch:
         self.handle, self.vocab, self.n_slots, self.max_beam, self.device = handle, vocab, n_slots, max_beam, device
 
     def destroy(self):
-        if self.handle:
+        if self.handle and _lib is not None:
             _lib.tb_batch_destroy(self.handle)
             self.handle = None
 
@@ -188,6 +189,13 @@ def tb_batch_destroy(batch: Batch):
 def tb_batch_bind_stream(batch: Batch, slot: int, graph, stream=None):
     _check(_lib.tb_batch_bind_stream(batch.handle, slot, None if graph is None else graph.handle, _stream(stream)),
            "tb_batch_bind_stream")
+
+
+TB_FLAG_GENERAL_KERNELS = 1
+
+
+def tb_batch_set_flags(batch: Batch, flags: int):
+    _check(_lib.tb_batch_set_flags(batch.handle, flags), "tb_batch_set_flags")
 
 
 def tb_batch_status(batch: Batch, stream=None) -> int:

@@ -17,7 +17,7 @@ _STAMP = LIB + ".srchash"
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "--fmad=false",  # the arithmetic contract forbids fusing x + lambda*bonus
-    "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+    "-Xcompiler", "-fPIC", "-Xcompiler", "-ffp-contract=off", "-shared", "-cudart", "static",
 ]
 
 

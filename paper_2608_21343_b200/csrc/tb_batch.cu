@@ -53,7 +53,6 @@ struct ArenaAllocator {
     if (next != free_blocks.end() && off + bytes == next->first) { bytes += next->second; free_blocks.erase(next); }
     free_blocks[off] = bytes;
   }
-  size_t free_bytes() const { size_t s = 0; for (auto& kv : free_blocks) s += kv.second; return s; }
 };
 
 struct Staging {
@@ -76,11 +75,14 @@ struct tb_batch {
   TbSlotRec* d_slots = nullptr;
   TbSlotState* d_sstate = nullptr;
   int32_t* d_cls = nullptr;
+  uint32_t flags = 0;
   int32_t* d_status = nullptr;
   int2* d_tree = nullptr;
   int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
   ArenaAllocator alloc;
   std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
+  std::vector<int32_t> slot_cache_bytes;               // bytes of the sections the pipelined kernel caches
+  std::vector<int32_t> slot_n_states;
   Staging staging[kStagingRing];
   int next_staging = 0;
 };
@@ -122,6 +124,8 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   b->arena_bytes = round_up(arena_bytes, kArenaAlign);
   b->alloc.init(b->arena_bytes);
   b->slot_block.assign(n_slots, {0, 0});
+  b->slot_cache_bytes.assign(n_slots, 0);
+  b->slot_n_states.assign(n_slots, 0);
   bool ok = true;
   ok = ok && cudaMalloc(&b->arena, b->arena_bytes) == cudaSuccess;
   ok = ok && cudaMalloc(&b->d_slots, sizeof(TbSlotRec) * n_slots) == cudaSuccess;
@@ -182,12 +186,12 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
       s.pending = ok;
     }
     if (!ok) { cudaGetLastError(); b->alloc.release(off, bytes); return TB_ERR_CUDA; }
-    rec.off_arc_begin = static_cast<int64_t>(off) + g->off_arc_begin;
-    rec.off_fail = static_cast<int64_t>(off) + g->off_fail;
-    rec.off_bw = static_cast<int64_t>(off) + g->off_bw;
-    rec.off_arc_cls = static_cast<int64_t>(off) + g->off_arc_cls;
-    rec.off_arc_w = static_cast<int64_t>(off) + g->off_arc_w;
-    rec.off_arc_dst = static_cast<int64_t>(off) + g->off_arc_dst;
+    rec.blob_off = static_cast<int64_t>(off);
+    rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
+    rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
+    rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
+    rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
+    rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
     rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
   }
   int rc = tb_launch_publish_slot(b->d_slots, b->d_sstate, slot, rec, stream);
@@ -197,6 +201,9 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
   auto& blk = b->slot_block[slot];
   if (blk.second) b->alloc.release(blk.first, blk.second);
   blk = {off, bytes};
+  b->slot_n_states[slot] = g ? g->n_states : 0;
+  // what the pipelined kernel caches in shared memory: the resolved lists, else the state records + token arcs
+  b->slot_cache_bytes[slot] = !g ? 0 : static_cast<int32_t>(g->blob.size()) - (g->n_rsent >= 0 ? g->off_rsrec : g->off_strec);
   return TB_OK;
 }
 
@@ -241,7 +248,22 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   p.out_scores = out_scores; p.out_states = out_states;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
+  if (!(b->flags & TB_FLAG_GENERAL_KERNELS)) {
+    int32_t max_cache = 0, max_states = 0;
+    for (int32_t i = 0; i < B; ++i) {
+      max_cache = b->slot_cache_bytes[i] > max_cache ? b->slot_cache_bytes[i] : max_cache;
+      max_states = b->slot_n_states[i] > max_states ? b->slot_n_states[i] : max_states;
+    }
+    rc = tb_launch_greedy_fast(p, max_cache, max_states, static_cast<cudaStream_t>(stream_));
+    if (rc != 1) return rc;
+  }
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {
+  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS))) return TB_ERR_INVALID_ARG;
+  b->flags = flags;
+  return TB_OK;
 }
 
 extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32_t n_slots, int32_t chunk,

@@ -22,11 +22,11 @@ struct Folded {
 inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
 
 template <typename T>
-int64_t append_section(std::vector<unsigned char>& blob, const std::vector<T>& v) {
+int32_t append_section(std::vector<unsigned char>& blob, const std::vector<T>& v) {
   size_t off = align16(blob.size());
   blob.resize(off + v.size() * sizeof(T));
   if (!v.empty()) std::memcpy(blob.data() + off, v.data(), v.size() * sizeof(T));
-  return static_cast<int64_t>(off);
+  return static_cast<int32_t>(off);
 }
 
 }  // namespace
@@ -201,6 +201,74 @@ static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offs
   g->off_arc_cls = append_section(g->blob, g->arc_class);
   g->off_arc_w = append_section(g->blob, g->arc_w);
   g->off_arc_dst = append_section(g->blob, g->arc_dst);
+  {  // per-state records and token-expanded arcs (tokens of a class in ascending id order)
+    std::vector<int32_t> ctb(n_classes + 1, 0), ctk(vocab);
+    for (int32_t v = 0; v < vocab; ++v) ctb[g->case_class[v] + 1]++;
+    for (int32_t c = 0; c < n_classes; ++c) ctb[c + 1] += ctb[c];
+    std::vector<int32_t> fill(ctb.begin(), ctb.end() - 1);
+    for (int32_t v = 0; v < vocab; ++v) ctk[fill[g->case_class[v]]++] = v;
+    std::vector<TbStateRec> recs(N);
+    std::vector<TbTokEnt> ents;
+    for (int32_t u = 0; u < N; ++u) {
+      recs[u].tok_begin = static_cast<int32_t>(ents.size());
+      for (int32_t a = g->state_arc_begin[u]; a < g->state_arc_begin[u + 1]; ++a) {
+        const int32_t c = g->arc_class[a];
+        for (int32_t j = ctb[c]; j < ctb[c + 1]; ++j)
+          ents.push_back({static_cast<uint32_t>(ctk[j]) | (static_cast<uint32_t>(c) << 16), g->arc_w[a], g->arc_dst[a], 0});
+      }
+      recs[u].tok_end = static_cast<int32_t>(ents.size());
+      recs[u].fail = g->state_fail[u];
+      recs[u].bw = g->state_bw[u];
+    }
+    g->off_strec = append_section(g->blob, recs);
+    g->off_tokent = append_section(g->blob, ents);
+    g->n_tokent = static_cast<int32_t>(ents.size());
+
+    // resolved lists (see TbRsRec): the walk the kernels would do, done once here in float
+    float root_w_max = 0.0f;
+    for (int32_t a = g->state_arc_begin[0]; a < g->state_arc_begin[1]; ++a) root_w_max = std::max(root_w_max, std::fabs(g->arc_w[a]));
+    std::vector<TbRsRec> rrecs(N);
+    std::vector<TbRsEnt> rents;
+    std::vector<int32_t> seen(n_classes, -1);   // class -> state that listed it during the current walk
+    bool fits = vocab < (1 << TB_RS_TOK_BITS) && N < (1 << (32 - TB_RS_TOK_BITS));
+    g->d_max = 0.0f;
+    for (int32_t s = 0; s < N; ++s) {
+      float acc = 0.0f;
+      const size_t first = rents.size();
+      for (int32_t u = s; u != 0; u = g->state_fail[u]) {
+        if (fits) {
+          for (int32_t a = g->state_arc_begin[u]; a < g->state_arc_begin[u + 1]; ++a) {
+            const int32_t c = g->arc_class[a];
+            if (seen[c] == s) continue;           // shadowed by a chain state closer to s
+            seen[c] = s;
+            const float bonus = acc + g->arc_w[a];
+            const float lb = lambda * bonus;
+            for (int32_t j = ctb[c]; j < ctb[c + 1]; ++j)
+              rents.push_back({(static_cast<uint32_t>(g->arc_dst[a]) << TB_RS_TOK_BITS) | static_cast<uint32_t>(ctk[j]), lb});
+          }
+          if (rents.size() > TB_RS_MAX_ENTRIES) fits = false;
+        }
+        acc = acc + g->state_bw[u];
+      }
+      g->d_max = std::max(g->d_max, std::fabs(acc));
+      rrecs[s].begin = static_cast<int32_t>(first);
+      rrecs[s].count = static_cast<int32_t>(rents.size() - first);
+      rrecs[s].D = acc;
+      rrecs[s].bmag = std::fabs(lambda) * (std::fabs(acc) + root_w_max);
+      if (fits)
+        std::sort(rents.begin() + first, rents.end(), [](const TbRsEnt& x, const TbRsEnt& y) {
+          return (x.dst_tok & ((1u << TB_RS_TOK_BITS) - 1)) < (y.dst_tok & ((1u << TB_RS_TOK_BITS) - 1));
+        });
+    }
+    if (fits) {
+      g->off_rsrec = append_section(g->blob, rrecs);
+      g->off_rsent = append_section(g->blob, rents);
+      g->n_rsent = static_cast<int32_t>(rents.size());
+    } else {
+      g->off_rsrec = g->off_rsent = 0;
+      g->n_rsent = -1;
+    }
+  }
   g->blob.resize(align16(g->blob.size()) + 16);  // tail padding so vector loads may overrun a section
   return TB_OK;
 }

@@ -25,12 +25,13 @@ struct GraphPtrs {
 // "Read the state and arc offsets of the model id and shift the pointers" (Sec. 2.2 para. 3).
 __device__ __forceinline__ GraphPtrs graph_of(const unsigned char* arena, const TbSlotRec& r) {
   GraphPtrs g;
-  g.arc_begin = reinterpret_cast<const int32_t*>(arena + r.off_arc_begin);
-  g.fail = reinterpret_cast<const int32_t*>(arena + r.off_fail);
-  g.bw = reinterpret_cast<const float*>(arena + r.off_bw);
-  g.arc_cls = reinterpret_cast<const int32_t*>(arena + r.off_arc_cls);
-  g.arc_w = reinterpret_cast<const float*>(arena + r.off_arc_w);
-  g.arc_dst = reinterpret_cast<const int32_t*>(arena + r.off_arc_dst);
+  const unsigned char* blob = arena + r.blob_off;
+  g.arc_begin = reinterpret_cast<const int32_t*>(blob + r.off_arc_begin);
+  g.fail = reinterpret_cast<const int32_t*>(blob + r.off_fail);
+  g.bw = reinterpret_cast<const float*>(blob + r.off_bw);
+  g.arc_cls = reinterpret_cast<const int32_t*>(blob + r.off_arc_cls);
+  g.arc_w = reinterpret_cast<const float*>(blob + r.off_arc_w);
+  g.arc_dst = reinterpret_cast<const int32_t*>(blob + r.off_arc_dst);
   g.n_states = r.n_states; g.n_arcs = r.n_arcs; g.max_depth = r.max_depth; g.lambda = r.lambda;
   return g;
 }

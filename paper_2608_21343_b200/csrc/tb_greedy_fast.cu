@@ -1,0 +1,856 @@
+// Pipelined greedy RNNT decode for packed bf16 logits: one persistent thread block per stream.
+//
+//   producer warp : streams the stream's frames (S rows each) from HBM into a shared-memory ring
+//                   with bulk asynchronous copies (16-byte aligned supersets of each frame) that
+//                   complete on an mbarrier;
+//   helper warps  : reduce every row, ahead of time and independently of the graph state, to a
+//                   summary {best root-boosted value y1, its token id1, an upper bound y2b on
+//                   every other token's root-boosted value, the blank logit, ...};
+//   decider warp  : the only sequential part -- walks the rows the decode visits, resolves each
+//                   from its summary plus the few tokens boosted by the current non-root graph
+//                   state, advances the graph state and the frame cursor, writes the outputs.
+// The decider shares its warp scheduler with no helper: warps are spread over the SM's four
+// schedulers by warp index, and every fourth warp other than the decider and the producer just
+// waits at the final barrier.
+//
+// Exactness.  Values follow the arithmetic contract (val = fl(x + fl(lambda * bonus)), ties to
+// the lowest id).  y(v) = fl(x[v] + fl(lambda * w_root(cls v))) is the exact value of token v in
+// the root state.  In a non-root state s every token whose class has no arc on the non-root part
+// of the suffix chain ("plain" tokens) has value fl(x + fl(lambda * fl(D + w_root))) with D the
+// summed suffix-link weights of the whole chain; in real arithmetic that is y + lambda*D, so the
+// order among plain tokens is the order of y up to rounding.  The decider accepts the summary's
+// winner as the best plain token only when y1 exceeds the bound on all other tokens by more
+// than a margin tau that dominates every rounding error involved, or shows that no plain token
+// can reach the best of {blank, the state's own tokens}; the tokens the chain boosts are always
+// evaluated exactly; otherwise the whole row is rescanned exactly from shared memory.
+//
+// Every wait is bounded; a wait that runs out raises TB_STATUS_WAIT_TIMEOUT, makes all roles of
+// the block leave their loops, and the block still waits (bounded) for its copies in flight.
+#include <cuda_bf16.h>
+
+#include "tb_device.cuh"
+#include "tb_launch.h"
+
+namespace {
+
+constexpr int kWarpsF = 20;     // warp 0 decider, warp 4 producer, warps 8/12/16 parked, 15 helpers
+constexpr int kHelpers = kWarpsF - kWarpsF / 4;
+constexpr int kThreadsF = kWarpsF * 32;
+constexpr int kSMax = 4;        // rows per frame the ring bookkeeping is sized for
+constexpr int kNitMax = 8;      // 256 tokens per pass iteration: V <= 2048 (kernel instantiated for 1, 2, 4, 8)
+constexpr int kWindow = 16;     // rows the decider looks at per round
+constexpr int kLaneDeep = 96;   // up to this many boosted tokens, each decider lane resolves a row alone
+constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
+constexpr uint32_t kSpinLimit = 1u << 20;
+
+#ifdef TB_PROFILE
+__device__ unsigned long long tb_prof[16];
+__device__ unsigned long long tb_prof_blk[4 * 1024];
+#define PROF_DECL() long long _pacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; long long _pt = 0
+#define PROF_T0() _pt = clock64()
+#define PROF_ADD(slot) do { long long _n = clock64(); _pacc[slot] += _n - _pt; _pt = _n; } while (0)
+#define PROF_COUNT(slot) _pacc[slot] += 1
+#define PROF_FLUSH() do { if ((threadIdx.x & 31) == 0) { for (int _i = 0; _i < 16; ++_i) if (_pacc[_i]) atomicAdd(&tb_prof[_i], (unsigned long long)_pacc[_i]); } } while (0)
+#else
+#define PROF_DECL() do {} while (0)
+#define PROF_T0() do {} while (0)
+#define PROF_ADD(slot) do {} while (0)
+#define PROF_COUNT(slot) do {} while (0)
+#define PROF_FLUSH() do {} while (0)
+#endif
+
+// What a helper leaves for the decider about one row (32 bytes, read as two 16-byte loads).
+struct RowSummary {
+  float y1;          // best root-boosted token value of the row (ties: lowest id)
+  float y2b;         // upper bound on the root-boosted value of every other token
+  float xb;          // blank logit
+  float x1;          // raw logit of the best token
+  float rootcw1;     // root arc weight of the best token's class (0 if none)
+  int32_t rootdst1;  // root arc target of the best token's class (0 if none)
+  uint32_t packed;   // id1 | overflow << 16 | gap_ok << 17  (gap_ok: y1 clears y2b by the rounding margin of any state)
+  uint32_t seq;      // frame number + 1: written last; the decider takes the summary as valid when it matches
+};
+constexpr uint32_t kSumOvf = 1u << 16, kSumGap = 1u << 17;
+// Summaries of one ring stage are kSMax * 32 bytes; stages are spaced 16 bytes further apart so that the
+// decider's lanes (one stage each) read their 16-byte halves from distinct shared-memory banks.
+constexpr int kSumStageBytes = kSMax * 32 + 16;
+
+// ---- mbarrier / bulk-copy primitives --------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Arrival without release ordering.  The decider uses it to hand a ring slot back: it has only
+// read the slot, and every such read has completed (its value fed a ballot) before the arrival,
+// so nothing needs to be made visible -- while a releasing arrival would also wait for the
+// decider's earlier global stores (emitted tokens) to be acknowledged by the memory system.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// The same test, letting the hardware park the warp for up to `ns` before it answers "not yet".
+__device__ __forceinline__ bool mbar_try_wait_park(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the block is aborting or the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicOr(status, TB_STATUS_WAIT_TIMEOUT);
+  return false;
+}
+// Bounded wait for the roles that are not latency critical: parks the warp between polls so that
+// it does not take issue slots or shared-memory pipeline cycles from the decider.
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (uint32_t it = 0; it < (kSpinLimit >> 2); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(256);
+    if ((it & 63u) == 63u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicOr(status, TB_STATUS_WAIT_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+__device__ __forceinline__ float row_at(const unsigned char* rowp, int idx) {
+  return bf16_bits_to_float(*reinterpret_cast<const uint16_t*>(rowp + 2 * idx));
+}
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) {
+  __nv_bfloat162 r;
+  *reinterpret_cast<uint32_t*>(&r) = w;
+  return r;
+}
+// Order-preserving map float -> uint32 (-0 is folded into +0 first, so equal floats get equal keys).
+__device__ __forceinline__ uint32_t fkey(float v) {
+  const uint32_t u = __float_as_uint(v + 0.0f);
+  return u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float fkey_inv(uint32_t k) {
+  return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+
+// Shared-memory accesses by 32-bit shared address (keeps the decider's address arithmetic short).
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds_v2(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint4 lds_v4_volatile(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_v4_volatile(uint32_t a, uint4 v) {
+  asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ bool mbar_test_addr(uint32_t bar_addr, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_relaxed_addr(uint32_t bar_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+}
+
+struct Smem {  // byte offsets into dynamic shared memory, computed identically on host and device
+  int ring, bars, summ, cls16, rootcb, rootcw, rootdst, lbuf, cls_seen, tokidx, misc, cache, total;
+};
+__host__ __device__ inline int up16(int x) { return (x + 15) & ~15; }
+__host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes) {
+  Smem s;
+  int o = 0;
+  s.ring = o; o += nst * slot_bytes;
+  s.bars = o; o += up16(8 * (2 * nst));
+  s.summ = o; o += nst * kSumStageBytes;
+  s.cls16 = o; o += up16(2 * V);
+  s.rootcb = o; o += up16(4 * C);
+  s.rootcw = o; o += up16(4 * C);
+  s.rootdst = o; o += up16(4 * C);
+  s.lbuf = o; o += up16(8 * V);       // boosted-token list of the current state when it is not read from the cache
+  s.cls_seen = o; o += up16(2 * C);   // class -> position in lbuf while a list is being built
+  s.tokidx = o; o += up16(2 * V);     // token -> position in the current list (filled only for an exact rescan)
+  s.misc = o; o += 64;
+  s.cache = o; o += up16(cache_bytes);
+  s.total = o;
+  return s;
+}
+
+struct FastParams {
+  TbDecodeParams d;
+  int32_t nst, slot_bytes, cache_bytes;  // cache_bytes > 0: every bound graph's lists (resolved, else state records + token arcs) fit in shared memory
+  const unsigned char* tensor_lo;        // first / one-past-last byte of the logits tensor
+  const unsigned char* tensor_hi;
+};
+
+// ---- helper: one row -> summary ----------------------------------------------------------------
+struct HelperCtx {
+  const uint16_t* cls16;
+  const float* rootcb;
+  const float* rootcw;
+  const int32_t* rootdst;
+  float beta_min, beta_max, dbeta;
+  float bmag_max;   // bound on |lambda| * (|D(s)| + largest root weight) over all states s
+  int V, nit;
+};
+
+template <int NIT>
+__device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned char* slot, int off_bytes,
+                                              uint32_t out_a, uint32_t seq, int lane) {
+  const int p = (off_bytes & 15) >> 1;                    // elements of the first 16-byte block that precede the row
+  const uint4* blk = reinterpret_cast<const uint4*>(slot + (off_bytes & ~15));
+  const unsigned char* rowp = slot + off_bytes;
+  const int V = h.V;
+  uint32_t w[4 * NIT];
+  const uint32_t NEG2 = 0xFF80FF80u;                      // two bf16 -inf
+#pragma unroll
+  for (int j = 0; j < NIT; ++j) {
+    if (j < h.nit) {
+      const int b = j * 32 + lane;
+      uint4 q = blk[b];
+      const int idx0 = b * 8 - p;                         // token id of the block's first element
+      if (idx0 < 0 || idx0 + 8 > V) {                     // head / tail block: mask what is not a token of this row
+        uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i0 = idx0 + 2 * e;
+          if (i0 < 0 || i0 >= V) qq[e] = (qq[e] & 0xFFFF0000u) | 0xFF80u;
+          if (i0 + 1 < 0 || i0 + 1 >= V) qq[e] = (qq[e] & 0x0000FFFFu) | 0xFF800000u;
+        }
+      }
+      w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+    } else {
+      w[4 * j] = w[4 * j + 1] = w[4 * j + 2] = w[4 * j + 3] = NEG2;
+    }
+  }
+  // tokens after the last full pass (at most 7): one element per lane
+  const int tail_idx = h.nit * 256 - p + lane;
+  const bool tail_ok = tail_idx < V && tail_idx >= 0;
+  uint32_t tail_bits = 0xFF80u;
+  if (tail_ok) tail_bits = *reinterpret_cast<const uint16_t*>(rowp + 2 * tail_idx);
+
+  // pass 1: raw maximum of the row's token logits (tree of packed maxima, then across the warp)
+  __nv_bfloat162 mm[4 * NIT];
+#pragma unroll
+  for (int i = 0; i < 4 * NIT; ++i) mm[i] = as_bf162(w[i]);
+#pragma unroll
+  for (int n = 2 * NIT; n >= 1; n >>= 1) {
+#pragma unroll
+    for (int i = 0; i < n; ++i) mm[i] = __hmax2(mm[i], mm[i + n]);
+  }
+  const __nv_bfloat162 m2 = __hmax2(mm[0], as_bf162(tail_bits | 0xFF800000u));
+  __nv_bfloat16 m = __hmax(__low2bfloat16(m2), __high2bfloat16(m2));
+  {
+    // order-preserving integer image of a bf16, so that one warp-wide integer max does the reduction
+    const uint32_t u = __bfloat16_as_ushort(m);
+    const uint32_t key = (u & 0x8000u) ? (0xFFFFu ^ u) : (u | 0x8000u);
+    const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+    const uint32_t ub = (kmax & 0x8000u) ? (kmax ^ 0x8000u) : (0xFFFFu ^ kmax);
+    m = __ushort_as_bfloat16(static_cast<unsigned short>(ub));
+  }
+  const float mf = __bfloat162float(m);
+  // Every token whose root-boosted value can reach that of the raw maximum has x >= m - dbeta;
+  // gamma keeps a strict margin over all roundings.  thr is rounded down.
+  const float gamma = (fabsf(mf) + fabsf(h.beta_max) + fabsf(h.beta_min)) * 0.0009765625f + 1e-30f;
+  const float thr_f = __fsub_rn(__fsub_rn(mf, h.dbeta), gamma);
+  const __nv_bfloat16 thr = __float2bfloat16_rd(thr_f);
+  const __nv_bfloat162 thr2 = __halves2bfloat162(thr, thr);
+
+  // pass 2: each lane notes its candidates (token id << 16 | logit bits); four fit, more flag the row
+  int nc = 0;
+  uint32_t cd[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int i = 0; i < 4 * NIT; ++i) {
+    const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);
+    if (mk) {
+      const uint32_t idx = static_cast<uint32_t>(((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 - p);
+      if (mk & 0xFFFFu) { cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = (idx << 16) | (w[i] & 0xFFFFu); ++nc; }
+      if (mk >> 16) { cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = ((idx + 1) << 16) | (w[i] >> 16); ++nc; }
+    }
+  }
+  if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
+    cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = (static_cast<uint32_t>(tail_idx) << 16) | tail_bits; ++nc;
+  }
+  // exact root-boosted values of this lane's candidates: best (value, lowest id) and runner-up value
+  ValId b{-INFINITY, INT32_MAX};
+  float sec = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (j < nc) {
+      const int id = static_cast<int>(cd[j] >> 16);
+      const ValId c{__fadd_rn(bf16_bits_to_float(cd[j] & 0xFFFFu), h.rootcb[h.cls16[id]]), id};
+      if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+    }
+  }
+  // across the warp: best (value, lowest id) and the runner-up value
+  const uint32_t key = fkey(b.v);
+  const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+  const int idmin = static_cast<int>(__reduce_min_sync(0xffffffffu, key == kmax ? static_cast<uint32_t>(b.i) : 0x7FFFFFFFu));
+  const bool mine = (key == kmax) && (b.i == idmin);
+  const uint32_t k2 = __reduce_max_sync(0xffffffffu, fkey(mine ? sec : b.v));
+  const bool ovf = __any_sync(0xffffffffu, nc > 4) || idmin >= V;
+  if (mine || (ovf && lane == 0)) {
+    // tokens that are not candidates have x < thr, hence root-boosted value <= fl(thr + beta_max)
+    const float ncb = __fadd_rn(__bfloat162float(thr), h.beta_max);
+    const int id1 = ovf ? 0 : b.i;
+    const int cl1 = h.cls16[id1];
+    RowSummary r;
+    r.y1 = b.v; r.y2b = fmaxf(fkey_inv(k2), ncb); r.xb = row_at(rowp, V); r.x1 = row_at(rowp, id1);
+    r.rootcw1 = h.rootcw[cl1]; r.rootdst1 = h.rootdst[cl1];
+    // same margin as the decider's, with the largest scale any state can have
+    const float tau = (fabsf(r.y1) + 4.0f * h.bmag_max) * 1.9073486328125e-6f + 1e-30f;
+    r.packed = static_cast<uint32_t>(id1) | (ovf ? kSumOvf : 0u) | ((r.y1 - r.y2b > tau) ? kSumGap : 0u);
+    r.seq = seq;
+    if (!ovf || lane == 0) {
+      // first half, fence, then the half that carries the sequence word
+      sts_v4_volatile(out_a, make_uint4(__float_as_uint(r.y1), __float_as_uint(r.y2b), __float_as_uint(r.xb), __float_as_uint(r.x1)));
+      __threadfence_block();
+      sts_v4_volatile(out_a + 16u, make_uint4(__float_as_uint(r.rootcw1), static_cast<uint32_t>(r.rootdst1), r.packed, r.seq));
+    }
+  }
+  __syncwarp();
+}
+
+// ---- decider ------------------------------------------------------------------------------------
+// The tokens boosted by the non-root part of the suffix chain of the current state, as 8-byte
+// entries {target state << 11 | token, lb} with lb = fl(lambda * fl(acc + w)).  Either a slice of
+// the graph's resolved lists cached in shared memory (sorted by token id), or a list assembled in
+// `lbuf`: copied from the resolved lists in the arena, or built by walking the chain (unsorted).
+struct CurList {
+  uint32_t addr;   // shared address of the first entry
+  int n;
+  bool sorted;
+  float D, bmag;
+};
+constexpr uint32_t kTokMask = (1u << TB_RS_TOK_BITS) - 1u;
+
+// Chain walk for graphs without resolved lists: closest chain state first, a class already
+// listed by a closer state is shadowed.  acc = suffix-link weights crossed so far, in walk order.
+__device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokEnt* tokent, int n_states, int max_depth,
+                                           int s, float lam, float R, TbRsEnt* lbuf, int16_t* cls_seen,
+                                           const uint16_t* cls16, CurList& L, int lane, int32_t* status) {
+  int n = 0;
+  float acc = 0.0f;
+  int u = s;
+  if (u < 0 || u >= n_states) { if (lane == 0) atomicOr(status, TB_STATUS_BAD_STATE); u = 0; }
+  for (int it = 0; u != 0; ++it) {
+    if (it > max_depth + 1) { if (lane == 0) atomicOr(status, TB_STATUS_WALK_TOO_DEEP); break; }
+    const TbStateRec rec = strec[u];
+    const int n_start = n;
+    for (int e0 = rec.tok_begin; e0 < rec.tok_end; e0 += 32) {
+      const int e = e0 + lane;
+      const bool have = e < rec.tok_end;
+      TbTokEnt ent{0u, 0.0f, 0, 0};
+      if (have) ent = tokent[e];
+      const int c = static_cast<int>(ent.tok_cls >> 16);
+      const int seen = have ? cls_seen[c] : 0;
+      const bool fresh = have && (seen < 0 || seen >= n_start);   // same class again only as a sibling from this state
+      const unsigned mask = __ballot_sync(0xffffffffu, fresh);
+      if (fresh) {
+        const int pos = n + __popc(mask & ((1u << lane) - 1u));
+        lbuf[pos].dst_tok = (static_cast<uint32_t>(ent.dst) << TB_RS_TOK_BITS) | (ent.tok_cls & 0xFFFFu);
+        lbuf[pos].lb = __fmul_rn(lam, __fadd_rn(acc, ent.w));
+        cls_seen[c] = static_cast<int16_t>(pos);
+      }
+      n += __popc(mask);
+      __syncwarp();
+    }
+    acc = __fadd_rn(acc, rec.bw);
+    u = rec.fail;
+  }
+  for (int i = lane; i < n; i += 32) cls_seen[cls16[lbuf[i].dst_tok & kTokMask]] = -1;   // leave the map clean
+  __syncwarp();
+  L.addr = smem_u32(lbuf); L.n = n; L.sorted = false; L.D = acc;
+  L.bmag = fabsf(lam) * (fabsf(acc) + R);
+}
+
+struct Pick {
+  ValId win;
+  int next;
+};
+
+// Warp-wide best of per-lane (value, id, next): two integer reductions and a shuffle.
+__device__ __forceinline__ Pick warp_pick(ValId v, int next) {
+  const uint32_t key = fkey(v.v);
+  const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+  const uint32_t idmin = __reduce_min_sync(0xffffffffu, key == kmax ? static_cast<uint32_t>(v.i) : 0xFFFFFFFFu);
+  const unsigned who = __ballot_sync(0xffffffffu, key == kmax && static_cast<uint32_t>(v.i) == idmin);
+  const int src = __ffs(who) - 1;
+  Pick p;
+  p.win.v = __shfl_sync(0xffffffffu, v.v, src);
+  p.win.i = static_cast<int>(idmin);
+  p.next = __shfl_sync(0xffffffffu, next, src);
+  return p;
+}
+
+template <int NIT>
+__global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
+  extern __shared__ __align__(128) unsigned char dyn[];
+#ifdef TB_PROFILE
+  const long long _kstart = clock64();
+#endif
+  const TbDecodeParams& p = P.d;
+  const int V = p.V, C = p.C, S = p.S, W = V + 1, nst = P.nst;
+  const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes);
+  unsigned char* ring = dyn + so.ring;
+  uint64_t* full = reinterpret_cast<uint64_t*>(dyn + so.bars);
+  uint64_t* freeb = full + nst;
+  const uint32_t summ_a = smem_u32(dyn + so.summ);
+  uint16_t* cls16 = reinterpret_cast<uint16_t*>(dyn + so.cls16);
+  float* rootcb = reinterpret_cast<float*>(dyn + so.rootcb);
+  float* rootcw = reinterpret_cast<float*>(dyn + so.rootcw);
+  int32_t* rootdst = reinterpret_cast<int32_t*>(dyn + so.rootdst);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(dyn + so.misc);
+  float* root_stats = reinterpret_cast<float*>(dyn + so.misc + 16);   // beta_min, beta_max, R
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TbSlotRec rec = p.slots[b];
+  const bool bound = rec.n_states > 0;
+  const bool resolved = bound && rec.n_rsent >= 0;
+  const bool cached = bound && P.cache_bytes > 0;
+  const GraphPtrs g = graph_of(p.arena, rec);
+  const float lam = bound ? rec.lambda : 0.0f;
+  const unsigned char* blob = p.arena + rec.blob_off;
+
+  int end = p.lengths ? p.lengths[b] : p.frames;
+  end = max(0, min(end, p.frames));
+
+  // ---- set-up: tables, root vectors, graph cache, barriers ----------------------------------------
+  for (int v = tid; v < V; v += kThreadsF) {
+    cls16[v] = static_cast<uint16_t>(p.cls[v]);
+    reinterpret_cast<int16_t*>(dyn + so.tokidx)[v] = -1;
+  }
+  for (int c = tid; c < C; c += kThreadsF) {
+    rootcb[c] = 0.0f; rootcw[c] = 0.0f; rootdst[c] = 0;
+    reinterpret_cast<int16_t*>(dyn + so.cls_seen)[c] = -1;
+  }
+  for (int i = tid; i < nst * kSumStageBytes / 4; i += kThreadsF) reinterpret_cast<uint32_t*>(dyn + so.summ)[i] = 0u;   // no sequence word matches yet
+  if (tid == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < nst; ++i) { mbar_init(&full[i], 1); mbar_init(&freeb[i], S + 1); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (cached) {
+    // the lists the decider reads are the tail of the blob: one contiguous 16-byte aligned range
+    const int from = resolved ? rec.off_rsrec : rec.off_strec;
+    const uint4* src = reinterpret_cast<const uint4*>(blob + from);
+    uint4* dst = reinterpret_cast<uint4*>(dyn + so.cache);
+    for (int i = tid; i < ((rec.blob_bytes - from) >> 4); i += kThreadsF) dst[i] = src[i];
+  }
+  __syncthreads();
+  if (bound) {
+    const int e = g.arc_begin[1];
+    for (int a = g.arc_begin[0] + tid; a < e; a += kThreadsF) {
+      const int c = g.arc_cls[a];
+      const float wv = __fadd_rn(0.0f, g.arc_w[a]);        // the walk's fl(acc + w) with acc = 0
+      rootcw[c] = wv; rootcb[c] = __fmul_rn(lam, wv); rootdst[c] = g.arc_dst[a];
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    float bmin = 0.0f, bmax = 0.0f, R = 0.0f;               // tokens without a root arc have beta = 0
+    if (bound) {
+      const int e = g.arc_begin[1];
+      for (int a = g.arc_begin[0]; a < e; ++a) {
+        const int c = g.arc_cls[a];
+        bmin = fminf(bmin, rootcb[c]); bmax = fmaxf(bmax, rootcb[c]); R = fmaxf(R, fabsf(rootcw[c]));
+      }
+    }
+    root_stats[0] = bmin; root_stats[1] = bmax; root_stats[2] = R;
+  }
+  __syncthreads();
+
+  const unsigned char* base = reinterpret_cast<const unsigned char*>(p.logits) + 2 * static_cast<int64_t>(b) * p.sb;
+  const int64_t frame_stride_bytes = 2 * p.st;
+  const int row_bytes = 2 * W;
+  const int frame_bytes = S * row_bytes;
+  const int lead0 = static_cast<int>(reinterpret_cast<uintptr_t>(base) & 15);
+  const int lead_step = static_cast<int>(frame_stride_bytes & 15);
+
+  PROF_DECL();
+  if (warp == 4) {
+    // ================================ producer ================================================
+    int issued = 0, st = 0, use = 0;
+    for (int f = 0; f < end; ++f) {
+      PROF_T0();
+      if (use > 0 && !mbar_wait_parked(&freeb[st], (use - 1) & 1, abort_flag, p.status)) break;
+      PROF_ADD(6);
+      const unsigned char* src = base + static_cast<int64_t>(f) * frame_stride_bytes;
+      const int lead = static_cast<int>(reinterpret_cast<uintptr_t>(src) & 15);
+      const unsigned char* a0 = src - lead;
+      const uint32_t bytes = static_cast<uint32_t>(up16(lead + frame_bytes));
+      unsigned char* dst = ring + static_cast<size_t>(st) * P.slot_bytes;
+      if (a0 >= P.tensor_lo && a0 + bytes <= P.tensor_hi) {
+        if (lane == 0) { mbar_arrive_expect_tx(&full[st], bytes); bulk_load(dst, a0, bytes, &full[st]); }
+      } else {  // the aligned superset would leave the tensor: copy the frame's own elements
+        const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
+        uint16_t* d16 = reinterpret_cast<uint16_t*>(dst + lead);
+        for (int i = lane; i < S * W; i += 32) d16[i] = __ldg(s16 + i);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[st]);
+      }
+      issued = f + 1;
+      if (++st == nst) { st = 0; ++use; }
+      __syncwarp();
+    }
+    PROF_FLUSH();
+    // no copy may be in flight when the block exits
+    for (int f = max(0, issued - nst); f < issued; ++f) {
+      const int fs = f % nst;
+      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&full[fs], (f / nst) & 1); ++it) {}
+    }
+  } else if ((warp & 3) != 0) {
+    // ================================ helpers =================================================
+    const int hid = warp - 1 - (warp >> 2);               // 0 .. kHelpers-1 over the warps that are not multiples of 4
+    HelperCtx h;
+    h.cls16 = cls16; h.rootcb = rootcb; h.rootcw = rootcw; h.rootdst = rootdst; h.V = V; h.nit = (V + 255) / 256;
+    h.beta_min = root_stats[0]; h.beta_max = root_stats[1]; h.dbeta = __fsub_rn(root_stats[1], root_stats[0]);
+    h.bmag_max = fabsf(lam) * ((bound ? rec.d_max : 0.0f) + root_stats[2]);
+    const int64_t n_rows = static_cast<int64_t>(end) * S;
+    for (int64_t r = hid; r < n_rows; r += kHelpers) {
+      const int f = static_cast<int>(r / S), k = static_cast<int>(r - static_cast<int64_t>(f) * S);
+      const int st = f % nst;
+      const uint32_t ph = (f / nst) & 1;
+      PROF_T0();
+      if (!mbar_wait_parked(&full[st], ph, abort_flag, p.status)) break;
+      PROF_ADD(0);
+      const int lead = static_cast<int>((lead0 + static_cast<int64_t>(f) * lead_step) & 15);
+      const unsigned char* slot = ring + static_cast<size_t>(st) * P.slot_bytes;
+      summarize_row<NIT>(h, slot, lead + k * row_bytes, summ_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
+      if (lane == 0) mbar_arrive(&freeb[st]);
+      PROF_ADD(1);
+    }
+    PROF_FLUSH();
+  } else if (warp == 0) {
+    // ================================ decider =================================================
+    // Works in rounds.  Decider lane L (L < number of ring stages) owns ring stage L for the
+    // whole decode and keeps that stage's frame number, barrier parity and row address in
+    // registers.  In a round every lane whose frame lies in the window [t, t + win_rows)
+    // resolves one row on its own, under the current graph state and with no cross-lane
+    // reduction: the lane holding frame t resolves the current row (t, k), the others row 0 of
+    // their frame, the row the decode reaches there if everything before it is blank.  One ballot
+    // tells how many leading rows are blank; they are consumed at once, and the first row that
+    // selects a token ends the round, because the graph state changes there.
+    const float R = root_stats[2];
+    const uint32_t ring_a = smem_u32(ring), freeb_a = smem_u32(freeb);
+    const uint32_t cache_a = smem_u32(dyn + so.cache);
+    TbRsEnt* lbuf = reinterpret_cast<TbRsEnt*>(dyn + so.lbuf);
+    int16_t* cls_seen = reinterpret_cast<int16_t*>(dyn + so.cls_seen);
+    int16_t* tokidx = reinterpret_cast<int16_t*>(dyn + so.tokidx);
+    const TbStateRec* strec = cached && !resolved ? reinterpret_cast<const TbStateRec*>(dyn + so.cache)
+                                                  : reinterpret_cast<const TbStateRec*>(blob + rec.off_strec);
+    const TbTokEnt* tokent = cached && !resolved ? reinterpret_cast<const TbTokEnt*>(dyn + so.cache + (rec.off_tokent - rec.off_strec))
+                                                 : reinterpret_cast<const TbTokEnt*>(blob + rec.off_tokent);
+    const TbRsRec* rsrec_g = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec);
+    const TbRsEnt* rsent_g = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
+    const uint32_t rsent_cache_a = cache_a + static_cast<uint32_t>(rec.off_rsent - rec.off_rsrec);
+
+    CurList L;
+    L.addr = smem_u32(lbuf); L.n = 0; L.sorted = true; L.D = 0.0f; L.bmag = fabsf(lam) * R;
+
+    // the stage this lane owns
+    const bool own = lane < nst;
+    const uint32_t ol = own ? static_cast<uint32_t>(lane) : 0u;   // lanes without a stage alias stage 0 and never act on it
+    const uint32_t my_slot_a = ring_a + ol * P.slot_bytes;
+    const uint32_t my_sum_a = summ_a + ol * kSumStageBytes;
+    const uint32_t my_free_a = freeb_a + ol * 8u;
+    const int lead_wrap = (nst * lead_step) & 15;
+    int my_f = lane;
+    int my_lead = (lead0 + lane * lead_step) & 15;
+    uint32_t spins = 0;
+
+    const int win_rows = min(kWindow, nst - 1);
+    const uint32_t nst_mask = (1u << nst) - 1u;
+    int t = 0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0;
+    float score = 0.0f;
+    int32_t* out_tok = p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
+    int32_t* out_frm = p.out_frames + static_cast<int64_t>(b) * p.out_cap;
+    const int max_rounds = p.frames * S + p.frames + 8;
+    bool failed = false;
+    for (int it = 0; t < end; ++it) {
+      if (it >= max_rounds) { if (lane == 0) atomicOr(p.status, TB_STATUS_STEP_LIMIT); break; }
+      PROF_T0();
+      // ---- everything that depends on nothing computed in this round is issued first --------------
+      const int rank = my_f - t;                            // >= 0 for every owning lane
+      const bool in_win = own && rank < win_rows && my_f < end;
+      const uint32_t koff = rank == 0 ? static_cast<uint32_t>(k) : 0u;
+      // the half with the sequence word is read first: when it matches, the other half is complete
+      const uint4 q1 = lds_v4_volatile(my_sum_a + koff * 32u + 16u);
+      const uint4 q0 = lds_v4_volatile(my_sum_a + koff * 32u);
+      const uint32_t row_a = my_slot_a + my_lead + koff * row_bytes;
+      bool ready = in_win && q1.w == static_cast<uint32_t>(my_f) + 1u;
+      if (!__shfl_sync(0xffffffffu, ready, st)) {          // the current row itself is not summarised yet: poll
+        if (++spins > kSpinLimit || ((spins & 255u) == 0u && *abort_flag)) {
+          if (spins > kSpinLimit) { *abort_flag = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
+          failed = true; break;
+        }
+        --it;                                               // a poll is not a round
+        continue;
+      }
+      spins = 0;
+      PROF_ADD(2);
+      const bool lane_eval = L.n <= kLaneDeep;              // few boosted tokens: every lane resolves its own row
+      ready = ready && (lane_eval || rank == 0);            // otherwise only the current row is looked at
+      const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+      const uint32_t id1 = q1.z & 0xFFFFu;
+      bool rescan = (q1.z & kSumOvf) != 0 || !lane_eval;
+#ifdef TB_PROFILE
+      int cause = rescan ? 1 : 0;
+#endif
+      // the tokens the state's chain boosts: exact values, four entries in flight at a time
+      float wv = -INFINITY;
+      uint32_t wdt = static_cast<uint32_t>(V);
+      bool in_deep = false;
+      if (lane_eval) {
+        for (int i0 = 0; i0 < L.n; i0 += 4) {
+          uint2 e[4];
+          uint32_t xr[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) e[j] = lds_v2(L.addr + 8u * min(i0 + j, L.n - 1));   // past the end: the last entry again
+#pragma unroll
+          for (int j = 0; j < 4; ++j) xr[j] = lds_u16(row_a + 2u * (e[j].x & kTokMask));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t tk = e[j].x & kTokMask;
+            const float v = __fadd_rn(bf16_bits_to_float(xr[j]), __uint_as_float(e[j].y));
+            in_deep |= tk == id1;
+            // sorted lists ascend in token id, so the first maximum is the lowest id
+            const bool take = L.sorted ? v > wv : (v > wv || (v == wv && tk < (wdt & kTokMask)));
+            if (take) { wv = v; wdt = e[j].x; }
+          }
+        }
+      }
+      PROF_ADD(3);
+      int wtok = static_cast<int>(wdt & kTokMask);
+      int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
+      {
+        // the best plain token: exact when the summary's winner is plain and clears the others by the
+        // rounding margin (at the root it is exact by construction); else bounded from above
+        const bool plain_ok = !in_deep && ((q1.z & kSumGap) != 0 || s <= 0);
+        const float nd = __fadd_rn(x1, __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
+        if (plain_ok) {
+          if (nd > wv || (nd == wv && static_cast<int>(id1) < wtok)) { wv = nd; wtok = static_cast<int>(id1); wnext = bound ? static_cast<int>(q1.y) : -1; }
+        } else {
+          const float ub = (in_deep ? y2b : y1) + lam * L.D;
+          const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
+          if (!(fmaxf(wv, xb) > ub + tau)) {
+            rescan = true;
+#ifdef TB_PROFILE
+            cause |= in_deep ? 2 : 4;
+#endif
+          }
+        }
+      }
+      const bool is_blank = ready && !rescan && !(wv >= xb);   // a tie with blank goes to the token
+      const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank);
+      const unsigned rot = ((blank_m >> st) | (blank_m << (nst - st))) & nst_mask;   // bit r: the lane of frame t + r
+      const int nb = __ffs(~rot) - 1;                       // leading blank rows (at most win_rows)
+      PROF_ADD(7);
+      // ---- the leading blanks, then the row after them ------------------------------------------------
+      const int l1 = st + 1 >= nst ? st + 1 - nst : st + 1;
+      const int jl = st + nb >= nst ? st + nb - nst : st + nb;
+      const float xb0 = __shfl_sync(0xffffffffu, xb, st), xb1 = __shfl_sync(0xffffffffu, xb, l1);
+      const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
+      const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
+      const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
+      const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+      const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
+      if (nb > 0) score = __fadd_rn(score, xb0);
+      if (nb > 1) score = __fadd_rn(score, xb1);
+      for (int r = 2; r < nb; ++r) {
+        const int src = st + r >= nst ? st + r - nst : st + r;
+        score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, src));
+      }
+      PROF_ADD(4);
+      int tok = V;                                          // V: no token selected in this round
+      float tval = 0.0f;
+      int tnext = s, adv = nb;                              // adv: frames fully passed in this round
+      if (nb < win_rows && j_ready) {
+        const int k_row = nb == 0 ? k : 0;                  // symbols already emitted in that row's frame
+        if (!j_rescan) {
+          tok = j_tok; tval = j_val; tnext = j_next;
+        } else {
+          // exact evaluation of that row by the whole warp from shared memory
+          PROF_COUNT(9);
+#ifdef TB_PROFILE
+          { const int cz = __shfl_sync(0xffffffffu, cause, jl); if (cz & 1) _pacc[12] += 1; if (cz & 2) _pacc[13] += 1; if (cz & 4) _pacc[14] += 1; }
+#endif
+          const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
+          for (int i = lane; i < L.n; i += 32) tokidx[lds_v2(L.addr + 8u * i).x & kTokMask] = static_cast<int16_t>(i);
+          __syncwarp();
+          ValId best{bf16_bits_to_float(lds_u16(rrow + 2u * V)), V};
+          int bn = s;
+          for (int tk = lane; tk < V; tk += 32) {
+            const int i = tokidx[tk];
+            float lbv; int nx;
+            if (i >= 0) { const uint2 e = lds_v2(L.addr + 8u * i); lbv = __uint_as_float(e.y); nx = static_cast<int>(e.x >> TB_RS_TOK_BITS); }
+            else { const int c = cls16[tk]; lbv = __fmul_rn(lam, __fadd_rn(L.D, rootcw[c])); nx = rootdst[c]; }
+            const float x = bf16_bits_to_float(lds_u16(rrow + 2u * tk));
+            const ValId c2{bound ? __fadd_rn(x, lbv) : x, tk};
+            if (better(c2, best)) { best = c2; bn = bound ? nx : -1; }
+          }
+          __syncwarp();
+          for (int i = lane; i < L.n; i += 32) tokidx[lds_v2(L.addr + 8u * i).x & kTokMask] = -1;
+          const Pick pk = warp_pick(best, bn);
+          tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
+          if (tok == V) { score = __fadd_rn(score, tval); ++adv; }   // blank after all: that frame is passed too
+        }
+        if (tok != V) {
+          score = __fadd_rn(score, tval);
+          if (lane == 0 && n_out < p.out_cap) { out_tok[n_out] = tok; out_frm[n_out] = t + nb; }
+          ++n_out;
+          k = k_row + 1;
+          if (k == S) ++adv;                                // the frame closes by force
+        }
+      }
+      PROF_ADD(10);
+      PROF_COUNT(8);
+      // ---- hand the passed frames' slots back, move on -------------------------------------------------
+      if (own && rank < adv) {
+        mbar_arrive_relaxed_addr(my_free_a);
+        my_f += nst; my_lead = (my_lead + lead_wrap) & 15;
+      }
+      if (adv > 0 && (tok == V || k == S)) k = 0;
+      t += adv;
+      st += adv; if (st >= nst) st -= nst;
+      PROF_ADD(5);
+      if (tok != V && bound && tnext != s) {
+        s = tnext;
+        if (s <= 0) {
+          L.n = 0; L.D = 0.0f; L.bmag = fabsf(lam) * R; L.sorted = true;
+        } else if (resolved) {
+          if (s >= rec.n_states) { if (lane == 0) atomicOr(p.status, TB_STATUS_BAD_STATE); s = 0; }
+          if (cached) {
+            const uint4 r4 = lds_v4(cache_a + 16u * s);
+            L.addr = rsent_cache_a + 8u * r4.x; L.n = static_cast<int>(r4.y);
+            L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w);
+          } else {
+            const TbRsRec r4 = rsrec_g[s];
+            for (int i = lane; i < r4.count && i < V; i += 32) lbuf[i] = rsent_g[r4.begin + i];
+            __syncwarp();
+            L.addr = smem_u32(lbuf); L.n = r4.count; L.D = r4.D; L.bmag = r4.bmag;
+          }
+          L.sorted = true;
+        } else {
+          build_list(strec, tokent, rec.n_states, rec.max_depth, s, lam, R, lbuf, cls_seen, cls16, L, lane, p.status);
+        }
+      }
+      PROF_ADD(11);
+    }
+    PROF_FLUSH();
+#ifdef TB_PROFILE
+    if (lane == 0 && blockIdx.x < 1024) {
+      tb_prof_blk[4 * blockIdx.x] = _pacc[2] + _pacc[3] + _pacc[4] + _pacc[5] + _pacc[7] + _pacc[10] + _pacc[11];
+      tb_prof_blk[4 * blockIdx.x + 1] = clock64() - _kstart;
+      tb_prof_blk[4 * blockIdx.x + 2] = n_out;
+      tb_prof_blk[4 * blockIdx.x + 3] = _pacc[9];
+    }
+#endif
+    if (failed || t < end) *abort_flag = 1;   // left early: let the other roles stop too
+    if (lane == 0) {
+      p.out_counts[b] = n_out; p.out_scores[b] = score; p.out_states[b] = s;
+      if (p.out_cursors) p.out_cursors[b] = t;
+    }
+  }
+  __syncthreads();
+}
+
+}  // namespace
+
+#ifdef TB_PROFILE
+extern "C" int tb_debug_prof(unsigned long long* out16, int reset) {
+  if (cudaMemcpyFromSymbol(out16, tb_prof, sizeof(unsigned long long) * 16) != cudaSuccess) return -1;
+  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(tb_prof, z, sizeof z); }
+  return 0;
+}
+extern "C" int tb_debug_prof_blk(unsigned long long* out, int n) {
+  return cudaMemcpyFromSymbol(out, tb_prof_blk, sizeof(unsigned long long) * 4 * n) == cudaSuccess ? 0 : -1;
+}
+#endif
+
+// Returns TB_OK if the launch was made, 1 if this path does not cover the call (the caller then
+// uses the general kernel), or an error code.
+int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int32_t max_states, cudaStream_t stream) {
+  const int W = d.V + 1;
+  if (d.dtype != TB_BF16 || d.persistent || d.n_dur != 0) return 1;
+  if (d.sv != 1 || d.ss != W || d.st < static_cast<int64_t>(d.S) * W || d.sb < 0) return 1;
+  if (d.S > kSMax || d.V > 256 * kNitMax || d.V >= (1 << TB_RS_TOK_BITS) || max_states >= (1 << (32 - TB_RS_TOK_BITS))) return 1;
+  if (reinterpret_cast<uintptr_t>(d.logits) & 1) return 1;
+  FastParams P;
+  P.d = d;
+  // 16 bytes past a multiple of 128: the decider's lanes (one slot each) then spread over the shared-memory banks
+  P.slot_bytes = ((up16(d.S * W * 2 + 16) + 127) & ~127) + 16;
+  P.tensor_lo = reinterpret_cast<const unsigned char*>(d.logits);
+  const int64_t last = static_cast<int64_t>(d.n_streams - 1) * d.sb + static_cast<int64_t>(d.frames - 1) * d.st +
+                       static_cast<int64_t>(d.S - 1) * d.ss + d.V;
+  P.tensor_hi = P.tensor_lo + 2 * (last + 1);
+  int dev = 0, max_smem = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return TB_ERR_CUDA;
+  }
+  const int budget = max_smem - 1024;
+  P.cache_bytes = (max_cache_bytes > 0 && max_cache_bytes <= 48 * 1024) ? max_cache_bytes : 0;
+  const int fixed = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes).total;
+  const int per_stage = P.slot_bytes + 16 + kSumStageBytes;
+  int nst = (budget - fixed - 64) / per_stage;
+  if (nst > kStagesMax) nst = kStagesMax;
+  if (nst < 4) return 1;
+  P.nst = nst;
+  const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes);
+  if (so.total > budget) return 1;
+  const int nit = (d.V + 255) / 256;
+  void (*fn)(FastParams) = nit <= 1 ? k_greedy_fast<1> : nit <= 2 ? k_greedy_fast<2> : nit <= 4 ? k_greedy_fast<4> : k_greedy_fast<8>;
+  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess) {
+    cudaGetLastError();
+    return 1;
+  }
+  fn<<<d.n_streams, kThreadsF, so.total, stream>>>(P);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}

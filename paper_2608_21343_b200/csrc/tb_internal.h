@@ -19,8 +19,47 @@ struct tb_graph {
   uint64_t class_map_hash = 0;  // to reject a bind against a batch with another class map
   // Device blob: sections at 16-byte aligned offsets, all ids graph-local.
   std::vector<unsigned char> blob;
-  int64_t off_arc_begin = 0, off_fail = 0, off_bw = 0, off_arc_cls = 0, off_arc_w = 0, off_arc_dst = 0;
+  int32_t off_arc_begin = 0, off_fail = 0, off_bw = 0, off_arc_cls = 0, off_arc_w = 0, off_arc_dst = 0;
+  int32_t off_strec = 0, off_tokent = 0, n_tokent = 0;
+  int32_t off_rsrec = 0, off_rsent = 0, n_rsent = 0;  // resolved per-state lists (n_rsent < 0: not built)
+  float d_max = 0.0f;                                  // largest |sum of suffix-link weights| over all states
 };
+
+// Two derived sections of the blob serve the pipelined kernel.  TbStateRec packs what a
+// suffix-link walk needs from one state into one 16-byte load; TbTokEnt lists, per state, its
+// outgoing arcs expanded to tokens (every case sibling of the arc's class), so that the tokens
+// a state boosts can be scored without going through the class -> tokens table.
+struct TbStateRec {
+  int32_t tok_begin, tok_end;  // range in the TbTokEnt section
+  int32_t fail;                // suffix-link target
+  float bw;                    // suffix-link weight
+};
+struct TbTokEnt {
+  uint32_t tok_cls;            // token | class << 16
+  float w;                     // arc weight
+  int32_t dst;                 // arc target
+  int32_t pad;
+};
+static_assert(sizeof(TbStateRec) == 16 && sizeof(TbTokEnt) == 16, "16-byte records");
+
+// Resolved lists: for every state, all tokens that the non-root part of its suffix chain boosts,
+// shadowing already applied (the chain state closest to the state wins a class), sorted by token
+// id, each with its finished additive term lb = fl(lambda * fl(acc + w)) (acc = suffix-link
+// weights crossed before the arc's chain state, added in walk order) and the arc's target.  With
+// them a state change costs the pipelined kernel one record load instead of a chain walk.  Built
+// only for graphs whose lists stay small (TB_RS_MAX_ENTRIES) and whose ids fit the packing.
+struct TbRsRec {
+  int32_t begin, count;  // range in the TbRsEnt section
+  float D;               // sum of the suffix-link weights of the whole chain, in walk order
+  float bmag;            // |lambda| * (|D| + largest root arc weight): scale of the rounding margin
+};
+struct TbRsEnt {
+  uint32_t dst_tok;      // target state << 11 | token
+  float lb;
+};
+static_assert(sizeof(TbRsRec) == 16 && sizeof(TbRsEnt) == 8, "record sizes");
+#define TB_RS_MAX_ENTRIES (1 << 18)
+#define TB_RS_TOK_BITS 11
 
 uint64_t tb_hash_class_map(const int32_t* case_class, int32_t vocab);
 
@@ -28,11 +67,16 @@ uint64_t tb_hash_class_map(const int32_t* case_class, int32_t vocab);
 // offsets from the arena base) and the scalars a walk needs.  n_states == 0 marks an unbound
 // slot (model id -1).
 struct TbSlotRec {
-  int64_t off_arc_begin, off_fail, off_bw, off_arc_cls, off_arc_w, off_arc_dst;
+  int64_t blob_off;  // byte offset of the graph's blob inside the arena
+  int32_t off_arc_begin, off_fail, off_bw, off_arc_cls, off_arc_w, off_arc_dst, off_strec, off_tokent;  // within the blob
   int32_t n_states, n_arcs, max_depth;
   float lambda;
+  int32_t n_tokent, blob_bytes;
+  int32_t off_rsrec, off_rsent, n_rsent;  // resolved lists; n_rsent < 0: the graph has none
+  float d_max;
+  int32_t pad[12];
 };
-static_assert(sizeof(TbSlotRec) == 64, "slot record is one 64-byte line");
+static_assert(sizeof(TbSlotRec) == 128, "slot record is 128 bytes");
 
 // Per-slot streaming state kept on the device between tb_stream_chunk calls.
 struct TbSlotState {

@@ -29,7 +29,7 @@ def make_batch(tb, w, phrase_lists, n_slots=None, weights=None, lam=None, arena_
                                 lam=w.lam if lam is None else lam)
         graphs.append(g)
         v = g.view()
-        total += 64 * (v["n_states"] + v["n_arcs"]) + 4096
+        total += 512 * (v["n_states"] + v["n_arcs"]) + 8192
     batch = tb.tb_batch_create(w.V, w.vocab.case_class, n_slots, arena_bytes=arena_bytes or max(1 << 20, total), **kw)
     for i, g in enumerate(graphs):
         tb.tb_batch_bind_stream(batch, i, g)

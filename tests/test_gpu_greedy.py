@@ -148,7 +148,7 @@ def test_rebind_one_slot_leaves_others_alone(tb):
 def test_error_codes(tb):
     w = W.get_workload(1, B=2, T=8)
     data = W.batch_inputs(w)
-    batch, graphs = make_batch(tb, w, data["phrases"], arena_bytes=4096)
+    batch, graphs = make_batch(tb, w, data["phrases"], arena_bytes=8192)
 
     def code(fn, *a, **k):
         with pytest.raises(tb.TbError) as e:
@@ -171,3 +171,73 @@ def test_error_codes(tb):
     assert code(tb.tb_greedy_decode, batch, three) == tb.TB_ERR_INVALID_ARG   # B > n_slots
     assert code(tb.tb_batch_create, 0, None, 1) == tb.TB_ERR_INVALID_ARG
     assert code(tb.tb_batch_create, 8, None, 1, max_beam=99) == tb.TB_ERR_INVALID_ARG
+
+
+# ---------------------------------------------------------------------------------------------
+# the pipelined kernel (packed bf16) against the oracle and against the general kernel
+# ---------------------------------------------------------------------------------------------
+
+def both_kernels(tb, w, data, phrase_lists=None, weights=None, lam=None, lengths=None, logits=None, what=""):
+    phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
+    batch, _ = make_batch(tb, w, phrase_lists, weights=weights, lam=lam)
+    logits = to_device(data["logits"]) if logits is None else logits
+    dl = None if lengths is None else torch.tensor(lengths, dtype=torch.int32, device="cuda:0")
+    fast = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
+    gen = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+    tb.tb_batch_set_flags(batch, 0)
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(phrase_lists):
+        g = oracle_graph(w, p, None if weights is None else weights[i], lam)
+        ref = O.greedy_rnnt(g, data["logits"][i], None if lengths is None else lengths[i])
+        check_greedy(fast, i, ref, what + " pipelined")
+        check_greedy(gen, i, ref, what + " general")
+        assert fast["scores"][i] == gen["scores"][i]
+    return fast
+
+
+@pytest.mark.parametrize("V,S,T", [(1024, 3, 150), (300, 4, 70), (256, 1, 90), (2048, 2, 40), (700, 3, 33)])
+def test_pipelined_kernel_shapes(tb, V, S, T):
+    w = W.get_workload(2, B=7, T=T, S=S, V=V, n_phrases=60, n_plants=8)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[1] = None
+    lists[4] = []
+    lengths = [T, T - 1, 0, 1, T // 2, T, 3]
+    both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"V{V}S{S}")
+
+
+@pytest.mark.parametrize("lam", [0.5, 2.0, -1.0])
+def test_pipelined_kernel_weights_and_ties(tb, lam):
+    """Coarse logits (many exact ties), mixed weights, lambda of either sign: the exact rescan path."""
+    w = W.get_workload(2, B=6, T=120, n_phrases=80, n_plants=10)
+    data = W.batch_inputs(w)
+    x = W.bf16_bits_to_f32(data["logits"])
+    x[:, ::3] = np.round(x[:, ::3] * 4) / 4
+    data["logits"] = W.f32_to_bf16_bits(x)
+    rng = np.random.default_rng(3)
+    weights = [[[float(rng.choice([0.5, 1.0, 1.5, 2.0])) for _ in p] for p in lst] for lst in data["phrases"]]
+    both_kernels(tb, w, data, weights=weights, lam=lam, what=f"ties lam{lam}")
+
+
+def test_pipelined_kernel_unaligned_and_padded_frames(tb):
+    w = W.get_workload(2, B=4, T=50, n_phrases=40, n_plants=5)
+    data = W.batch_inputs(w)
+    Wd = w.V + 1
+    for shift, pad in ((1, 0), (3, 0), (0, 7), (5, 64)):
+        flat = torch.zeros(shift + w.B * w.T * (w.S * Wd + pad) + 8, dtype=torch.bfloat16, device="cuda:0")
+        view = flat[shift:shift + w.B * w.T * (w.S * Wd + pad)].view(w.B, w.T, w.S * Wd + pad)[:, :, :w.S * Wd]
+        view = view.reshape(w.B, w.T, w.S, Wd) if pad == 0 else view.unflatten(2, (w.S, Wd))
+        view.copy_(to_device(data["logits"]))
+        assert view.data_ptr() % 16 == (flat.data_ptr() + 2 * shift) % 16
+        both_kernels(tb, w, data, logits=view, what=f"shift{shift}pad{pad}")
+    # the last stream's last frame ends exactly at the end of the allocation's tensor
+    exact = to_device(data["logits"]).clone()
+    both_kernels(tb, w, data, logits=exact, what="exact end")
+
+
+def test_pipelined_kernel_large_lists_not_cached(tb):
+    """Graphs too large for the shared-memory cache are walked in the arena (workload 3 lists)."""
+    w = W.get_workload(3, B=2, T=150)
+    data = W.batch_inputs(w)
+    both_kernels(tb, w, data, what="w3")
