@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <limits>
 #include <new>
 #include <numeric>
 
@@ -230,7 +231,7 @@ static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offs
     std::vector<TbRsRec> rrecs(N);
     std::vector<TbRsEnt> rents;
     std::vector<int32_t> seen(n_classes, -1);   // class -> state that listed it during the current walk
-    bool fits = vocab < (1 << TB_RS_TOK_BITS) && N < (1 << (32 - TB_RS_TOK_BITS));
+    bool fits = 2 * (vocab + 1) <= (1 << TB_RS_TOK_BITS) && N < (1 << (32 - TB_RS_TOK_BITS));
     g->d_max = 0.0f;
     for (int32_t s = 0; s < N; ++s) {
       float acc = 0.0f;
@@ -244,21 +245,24 @@ static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offs
             const float bonus = acc + g->arc_w[a];
             const float lb = lambda * bonus;
             for (int32_t j = ctb[c]; j < ctb[c + 1]; ++j)
-              rents.push_back({(static_cast<uint32_t>(g->arc_dst[a]) << TB_RS_TOK_BITS) | static_cast<uint32_t>(ctk[j]), lb});
+              rents.push_back({(static_cast<uint32_t>(g->arc_dst[a]) << TB_RS_TOK_BITS) | static_cast<uint32_t>(2 * ctk[j]), lb});
           }
           if (rents.size() > TB_RS_MAX_ENTRIES) fits = false;
         }
         acc = acc + g->state_bw[u];
       }
       g->d_max = std::max(g->d_max, std::fabs(acc));
+      if (fits) {
+        std::sort(rents.begin() + first, rents.end(), [](const TbRsEnt& x, const TbRsEnt& y) {
+          return (x.dst_tok & ((1u << TB_RS_TOK_BITS) - 1)) < (y.dst_tok & ((1u << TB_RS_TOK_BITS) - 1));
+        });
+        while ((rents.size() - first) % 4 != 0)   // sentinels: the blank column with lb = -inf
+          rents.push_back({static_cast<uint32_t>(2 * vocab), -std::numeric_limits<float>::infinity()});
+      }
       rrecs[s].begin = static_cast<int32_t>(first);
       rrecs[s].count = static_cast<int32_t>(rents.size() - first);
       rrecs[s].D = acc;
       rrecs[s].bmag = std::fabs(lambda) * (std::fabs(acc) + root_w_max);
-      if (fits)
-        std::sort(rents.begin() + first, rents.end(), [](const TbRsEnt& x, const TbRsEnt& y) {
-          return (x.dst_tok & ((1u << TB_RS_TOK_BITS) - 1)) < (y.dst_tok & ((1u << TB_RS_TOK_BITS) - 1));
-        });
     }
     if (fits) {
       g->off_rsrec = append_section(g->blob, rrecs);

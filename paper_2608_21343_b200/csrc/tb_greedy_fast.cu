@@ -38,8 +38,7 @@ constexpr int kHelpers = kWarpsF - kWarpsF / 4;
 constexpr int kThreadsF = kWarpsF * 32;
 constexpr int kSMax = 4;        // rows per frame the ring bookkeeping is sized for
 constexpr int kNitMax = 8;      // 256 tokens per pass iteration: V <= 2048 (kernel instantiated for 1, 2, 4, 8)
-constexpr int kWindow = 16;     // rows the decider looks at per round
-constexpr int kLaneDeep = 96;   // up to this many boosted tokens, each decider lane resolves a row alone
+constexpr int kGroupDeep = 32;  // up to this many boosted tokens, the decider resolves eight rows per round, four lanes each
 constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -199,7 +198,7 @@ __device__ __forceinline__ void mbar_arrive_relaxed_addr(uint32_t bar_addr) {
 }
 
 struct Smem {  // byte offsets into dynamic shared memory, computed identically on host and device
-  int ring, bars, summ, cls16, rootcb, rootcw, rootdst, lbuf, cls_seen, tokidx, misc, cache, total;
+  int ring, bars, summ, cls16, rootcb, rootcw, rootdst, lbuf, cls_seen, tokidx, emit, misc, cache, total;
 };
 __host__ __device__ inline int up16(int x) { return (x + 15) & ~15; }
 __host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes) {
@@ -212,9 +211,10 @@ __host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int
   s.rootcb = o; o += up16(4 * C);
   s.rootcw = o; o += up16(4 * C);
   s.rootdst = o; o += up16(4 * C);
-  s.lbuf = o; o += up16(8 * V);       // boosted-token list of the current state when it is not read from the cache
+  s.lbuf = o; o += up16(8 * (V + 4)); // boosted-token list of the current state when it is not read from the cache
   s.cls_seen = o; o += up16(2 * C);   // class -> position in lbuf while a list is being built
   s.tokidx = o; o += up16(2 * V);     // token -> position in the current list (filled only for an exact rescan)
+  s.emit = o; o += 32 * 8;            // emitted (token, frame) pairs waiting for a coalesced store
   s.misc = o; o += 64;
   s.cache = o; o += up16(cache_bytes);
   s.total = o;
@@ -319,11 +319,34 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
   // exact root-boosted values of this lane's candidates: best (value, lowest id) and runner-up value
   ValId b{-INFINITY, INT32_MAX};
   float sec = -INFINITY;
+  if (!__any_sync(0xffffffffu, nc > 4)) {
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    if (j < nc) {
-      const int id = static_cast<int>(cd[j] >> 16);
-      const ValId c{__fadd_rn(bf16_bits_to_float(cd[j] & 0xFFFFu), h.rootcb[h.cls16[id]]), id};
+    for (int j = 0; j < 4; ++j) {
+      if (j < nc) {
+        const int id = static_cast<int>(cd[j] >> 16);
+        const ValId c{__fadd_rn(bf16_bits_to_float(cd[j] & 0xFFFFu), h.rootcb[h.cls16[id]]), id};
+        if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+      }
+    }
+  } else {
+    // some lane met more candidates than it can note (a low row maximum): evaluate every hit in place
+#pragma unroll
+    for (int i = 0; i < 4 * NIT; ++i) {
+      const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);
+      if (mk) {
+        const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 - p;
+        if (mk & 0xFFFFu) {
+          const ValId c{__fadd_rn(bf16_bits_to_float(w[i] & 0xFFFFu), h.rootcb[h.cls16[idx]]), idx};
+          if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+        }
+        if (mk >> 16) {
+          const ValId c{__fadd_rn(bf16_bits_to_float(w[i] >> 16), h.rootcb[h.cls16[idx + 1]]), idx + 1};
+          if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+        }
+      }
+    }
+    if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
+      const ValId c{__fadd_rn(bf16_bits_to_float(tail_bits), h.rootcb[h.cls16[tail_idx]]), tail_idx};
       if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
     }
   }
@@ -333,7 +356,7 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
   const int idmin = static_cast<int>(__reduce_min_sync(0xffffffffu, key == kmax ? static_cast<uint32_t>(b.i) : 0x7FFFFFFFu));
   const bool mine = (key == kmax) && (b.i == idmin);
   const uint32_t k2 = __reduce_max_sync(0xffffffffu, fkey(mine ? sec : b.v));
-  const bool ovf = __any_sync(0xffffffffu, nc > 4) || idmin >= V;
+  const bool ovf = idmin >= V;   // no candidate at all (cannot happen with finite logits)
   if (mine || (ovf && lane == 0)) {
     // tokens that are not candidates have x < thr, hence root-boosted value <= fl(thr + beta_max)
     const float ncb = __fadd_rn(__bfloat162float(thr), h.beta_max);
@@ -367,12 +390,13 @@ struct CurList {
   bool sorted;
   float D, bmag;
 };
-constexpr uint32_t kTokMask = (1u << TB_RS_TOK_BITS) - 1u;
+constexpr uint32_t kTokMask = (1u << TB_RS_TOK_BITS) - 1u;   // low bits of an entry: 2 * token
 
 // Chain walk for graphs without resolved lists: closest chain state first, a class already
 // listed by a closer state is shadowed.  acc = suffix-link weights crossed so far, in walk order.
+// The list is padded to a multiple of four with sentinels (blank column, lb = -inf).
 __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokEnt* tokent, int n_states, int max_depth,
-                                           int s, float lam, float R, TbRsEnt* lbuf, int16_t* cls_seen,
+                                           int s, float lam, float R, int V, TbRsEnt* lbuf, int16_t* cls_seen,
                                            const uint16_t* cls16, CurList& L, int lane, int32_t* status) {
   int n = 0;
   float acc = 0.0f;
@@ -393,7 +417,7 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
       const unsigned mask = __ballot_sync(0xffffffffu, fresh);
       if (fresh) {
         const int pos = n + __popc(mask & ((1u << lane) - 1u));
-        lbuf[pos].dst_tok = (static_cast<uint32_t>(ent.dst) << TB_RS_TOK_BITS) | (ent.tok_cls & 0xFFFFu);
+        lbuf[pos].dst_tok = (static_cast<uint32_t>(ent.dst) << TB_RS_TOK_BITS) | (2u * (ent.tok_cls & 0xFFFFu));
         lbuf[pos].lb = __fmul_rn(lam, __fadd_rn(acc, ent.w));
         cls_seen[c] = static_cast<int16_t>(pos);
       }
@@ -403,9 +427,11 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
     acc = __fadd_rn(acc, rec.bw);
     u = rec.fail;
   }
-  for (int i = lane; i < n; i += 32) cls_seen[cls16[lbuf[i].dst_tok & kTokMask]] = -1;   // leave the map clean
+  for (int i = lane; i < n; i += 32) cls_seen[cls16[(lbuf[i].dst_tok & kTokMask) >> 1]] = -1;   // leave the map clean
+  const int n_pad = (n + 3) & ~3;
+  if (lane < n_pad - n) { lbuf[n + lane].dst_tok = 2u * static_cast<uint32_t>(V); lbuf[n + lane].lb = -INFINITY; }
   __syncwarp();
-  L.addr = smem_u32(lbuf); L.n = n; L.sorted = false; L.D = acc;
+  L.addr = smem_u32(lbuf); L.n = n_pad; L.sorted = false; L.D = acc;
   L.bmag = fabsf(lam) * (fabsf(acc) + R);
 }
 
@@ -568,20 +594,21 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     PROF_FLUSH();
   } else if (warp == 0) {
     // ================================ decider =================================================
-    // Works in rounds.  Decider lane L (L < number of ring stages) owns ring stage L for the
-    // whole decode and keeps that stage's frame number, barrier parity and row address in
-    // registers.  In a round every lane whose frame lies in the window [t, t + win_rows)
-    // resolves one row on its own, under the current graph state and with no cross-lane
-    // reduction: the lane holding frame t resolves the current row (t, k), the others row 0 of
-    // their frame, the row the decode reaches there if everything before it is blank.  One ballot
-    // tells how many leading rows are blank; they are consumed at once, and the first row that
-    // selects a token ends the round, because the graph state changes there.
+    // Works in rounds.  With few boosted tokens in the current state (the usual case) the warp is
+    // eight groups of four lanes; group q looks at one row: group 0 at the current row (t, k),
+    // group q >= 1 at row (t + q, 0), the row the decode reaches if everything before it is blank.
+    // The four lanes share the state's boosted tokens, combine with two shuffles, and every group
+    // resolves its row under the current graph state.  One ballot tells how many leading rows are
+    // blank; they are consumed at once, and the first row that selects a token ends the round,
+    // because the graph state changes there.  With many boosted tokens all 32 lanes share them and
+    // only the current row is resolved.
     const float R = root_stats[2];
     const uint32_t ring_a = smem_u32(ring), freeb_a = smem_u32(freeb);
     const uint32_t cache_a = smem_u32(dyn + so.cache);
     TbRsEnt* lbuf = reinterpret_cast<TbRsEnt*>(dyn + so.lbuf);
     int16_t* cls_seen = reinterpret_cast<int16_t*>(dyn + so.cls_seen);
     int16_t* tokidx = reinterpret_cast<int16_t*>(dyn + so.tokidx);
+    int2* emit_buf = reinterpret_cast<int2*>(dyn + so.emit);
     const TbStateRec* strec = cached && !resolved ? reinterpret_cast<const TbStateRec*>(dyn + so.cache)
                                                   : reinterpret_cast<const TbStateRec*>(blob + rec.off_strec);
     const TbTokEnt* tokent = cached && !resolved ? reinterpret_cast<const TbTokEnt*>(dyn + so.cache + (rec.off_tokent - rec.off_strec))
@@ -593,38 +620,29 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     CurList L;
     L.addr = smem_u32(lbuf); L.n = 0; L.sorted = true; L.D = 0.0f; L.bmag = fabsf(lam) * R;
 
-    // the stage this lane owns
-    const bool own = lane < nst;
-    const uint32_t ol = own ? static_cast<uint32_t>(lane) : 0u;   // lanes without a stage alias stage 0 and never act on it
-    const uint32_t my_slot_a = ring_a + ol * P.slot_bytes;
-    const uint32_t my_sum_a = summ_a + ol * kSumStageBytes;
-    const uint32_t my_free_a = freeb_a + ol * 8u;
-    const int lead_wrap = (nst * lead_step) & 15;
-    int my_f = lane;
-    int my_lead = (lead0 + lane * lead_step) & 15;
-    uint32_t spins = 0;
-
-    const int win_rows = min(kWindow, nst - 1);
-    const uint32_t nst_mask = (1u << nst) - 1u;
-    int t = 0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0;
+    const int q = lane >> 2, ql = lane & 3;                 // group and lane within the group
+    const int win_rows = min(8, nst - 1);
+    int t = 0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0, lead = lead0;
     float score = 0.0f;
     int32_t* out_tok = p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
     int32_t* out_frm = p.out_frames + static_cast<int64_t>(b) * p.out_cap;
     const int max_rounds = p.frames * S + p.frames + 8;
+    uint32_t spins = 0;
     bool failed = false;
     for (int it = 0; t < end; ++it) {
       if (it >= max_rounds) { if (lane == 0) atomicOr(p.status, TB_STATUS_STEP_LIMIT); break; }
       PROF_T0();
-      // ---- everything that depends on nothing computed in this round is issued first --------------
-      const int rank = my_f - t;                            // >= 0 for every owning lane
-      const bool in_win = own && rank < win_rows && my_f < end;
-      const uint32_t koff = rank == 0 ? static_cast<uint32_t>(k) : 0u;
+      const bool wide = L.n > kGroupDeep;                   // many boosted tokens: the whole warp takes the current row
+      const int rq = wide ? 0 : q;                          // window row of this lane
+      int stq = st + rq; if (stq >= nst) stq -= nst;
+      const uint32_t koff = rq == 0 ? static_cast<uint32_t>(k) : 0u;
+      const uint32_t sum_a = summ_a + stq * kSumStageBytes + koff * 32u;
       // the half with the sequence word is read first: when it matches, the other half is complete
-      const uint4 q1 = lds_v4_volatile(my_sum_a + koff * 32u + 16u);
-      const uint4 q0 = lds_v4_volatile(my_sum_a + koff * 32u);
-      const uint32_t row_a = my_slot_a + my_lead + koff * row_bytes;
-      bool ready = in_win && q1.w == static_cast<uint32_t>(my_f) + 1u;
-      if (!__shfl_sync(0xffffffffu, ready, st)) {          // the current row itself is not summarised yet: poll
+      const uint4 q1 = lds_v4_volatile(sum_a + 16u);
+      const uint4 q0 = lds_v4_volatile(sum_a);
+      const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + rq * lead_step) & 15) + koff * row_bytes;
+      const bool ready = rq < win_rows && t + rq < end && q1.w == static_cast<uint32_t>(t + rq) + 1u;
+      if (!__shfl_sync(0xffffffffu, ready, 0)) {           // the current row itself is not summarised yet: poll
         if (++spins > kSpinLimit || ((spins & 255u) == 0u && *abort_flag)) {
           if (spins > kSpinLimit) { *abort_flag = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
           failed = true; break;
@@ -634,47 +652,68 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       }
       spins = 0;
       PROF_ADD(2);
-      const bool lane_eval = L.n <= kLaneDeep;              // few boosted tokens: every lane resolves its own row
-      ready = ready && (lane_eval || rank == 0);            // otherwise only the current row is looked at
       const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
-      const uint32_t id1 = q1.z & 0xFFFFu;
-      bool rescan = (q1.z & kSumOvf) != 0 || !lane_eval;
-#ifdef TB_PROFILE
-      int cause = rescan ? 1 : 0;
-#endif
-      // the tokens the state's chain boosts: exact values, four entries in flight at a time
+      const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
+      bool rescan = (q1.z & kSumOvf) != 0;
+      // ---- the tokens the state's chain boosts: exact values; this lane takes every 4th (or 32nd) entry
       float wv = -INFINITY;
-      uint32_t wdt = static_cast<uint32_t>(V);
+      uint32_t wdt = 2u * static_cast<uint32_t>(V);
       bool in_deep = false;
-      if (lane_eval) {
-        for (int i0 = 0; i0 < L.n; i0 += 4) {
-          uint2 e[4];
-          uint32_t xr[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) e[j] = lds_v2(L.addr + 8u * min(i0 + j, L.n - 1));   // past the end: the last entry again
-#pragma unroll
-          for (int j = 0; j < 4; ++j) xr[j] = lds_u16(row_a + 2u * (e[j].x & kTokMask));
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t tk = e[j].x & kTokMask;
-            const float v = __fadd_rn(bf16_bits_to_float(xr[j]), __uint_as_float(e[j].y));
-            in_deep |= tk == id1;
-            // sorted lists ascend in token id, so the first maximum is the lowest id
-            const bool take = L.sorted ? v > wv : (v > wv || (v == wv && tk < (wdt & kTokMask)));
-            if (take) { wv = v; wdt = e[j].x; }
-          }
+      {
+        const int lstep = wide ? 32 : 4, l0 = wide ? lane : ql;
+        int i = l0;
+        for (; i + lstep < L.n; i += 2 * lstep) {           // two entries in flight
+          const uint2 e0 = lds_v2(L.addr + 8u * i), e1 = lds_v2(L.addr + 8u * (i + lstep));
+          const uint32_t x0 = lds_u16(row_a + (e0.x & kTokMask)), x1r = lds_u16(row_a + (e1.x & kTokMask));
+          const float v0 = __fadd_rn(bf16_bits_to_float(x0), __uint_as_float(e0.y));
+          const float v1 = __fadd_rn(bf16_bits_to_float(x1r), __uint_as_float(e1.y));
+          in_deep |= (e0.x & kTokMask) == id1x2 || (e1.x & kTokMask) == id1x2;
+          if (v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask))) { wv = v0; wdt = e0.x; }
+          if (v1 > wv || (v1 == wv && (e1.x & kTokMask) < (wdt & kTokMask))) { wv = v1; wdt = e1.x; }
+        }
+        if (i < L.n) {
+          const uint2 e0 = lds_v2(L.addr + 8u * i);
+          const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16(row_a + (e0.x & kTokMask))), __uint_as_float(e0.y));
+          in_deep |= (e0.x & kTokMask) == id1x2;
+          if (v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask))) { wv = v0; wdt = e0.x; }
         }
       }
       PROF_ADD(3);
-      int wtok = static_cast<int>(wdt & kTokMask);
+      // combine over the lanes that share the row
+      if (L.n > 0) {
+        if (wide) {
+          const uint32_t key = fkey(wv);
+          const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+          const uint32_t tmin = __reduce_min_sync(0xffffffffu, key == kmax ? (wdt & kTokMask) : 0xFFFFFFFFu);
+          const unsigned who = __ballot_sync(0xffffffffu, key == kmax && (wdt & kTokMask) == tmin);
+          const int src = __ffs(who) - 1;
+          wv = __shfl_sync(0xffffffffu, wv, src); wdt = __shfl_sync(0xffffffffu, wdt, src);
+          in_deep = __any_sync(0xffffffffu, in_deep);
+        } else {
+#pragma unroll
+          for (int off = 1; off <= 2; off <<= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, wv, off);
+            const uint32_t od = __shfl_xor_sync(0xffffffffu, wdt, off);
+            const bool oi = __shfl_xor_sync(0xffffffffu, in_deep, off);
+            if (ov > wv || (ov == wv && (od & kTokMask) < (wdt & kTokMask))) { wv = ov; wdt = od; }
+            in_deep |= oi;
+          }
+        }
+      }
+      PROF_ADD(15);
+      int wtok = static_cast<int>((wdt & kTokMask) >> 1);
       int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
+#ifdef TB_PROFILE
+      int cause = rescan ? 1 : 0;
+#endif
       {
         // the best plain token: exact when the summary's winner is plain and clears the others by the
         // rounding margin (at the root it is exact by construction); else bounded from above
         const bool plain_ok = !in_deep && ((q1.z & kSumGap) != 0 || s <= 0);
         const float nd = __fadd_rn(x1, __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
+        const int id1 = static_cast<int>(id1x2 >> 1);
         if (plain_ok) {
-          if (nd > wv || (nd == wv && static_cast<int>(id1) < wtok)) { wv = nd; wtok = static_cast<int>(id1); wnext = bound ? static_cast<int>(q1.y) : -1; }
+          if (nd > wv || (nd == wv && id1 < wtok)) { wv = nd; wtok = id1; wnext = bound ? static_cast<int>(q1.y) : -1; }
         } else {
           const float ub = (in_deep ? y2b : y1) + lam * L.D;
           const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
@@ -687,14 +726,14 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         }
       }
       const bool is_blank = ready && !rescan && !(wv >= xb);   // a tie with blank goes to the token
-      const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank);
-      const unsigned rot = ((blank_m >> st) | (blank_m << (nst - st))) & nst_mask;   // bit r: the lane of frame t + r
-      const int nb = __ffs(~rot) - 1;                       // leading blank rows (at most win_rows)
+      const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank) & 0x11111111u;   // one bit per group
+      const unsigned stop_m = ~blank_m & 0x11111111u;
+      int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : 8;          // leading blank rows
+      if (wide) nb = (blank_m & 1u) ? 1 : 0;
       PROF_ADD(7);
       // ---- the leading blanks, then the row after them ------------------------------------------------
-      const int l1 = st + 1 >= nst ? st + 1 - nst : st + 1;
-      const int jl = st + nb >= nst ? st + nb - nst : st + nb;
-      const float xb0 = __shfl_sync(0xffffffffu, xb, st), xb1 = __shfl_sync(0xffffffffu, xb, l1);
+      const int jl = wide ? 0 : 4 * min(nb, 7);
+      const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
       const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
       const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
       const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
@@ -702,15 +741,12 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
       if (nb > 0) score = __fadd_rn(score, xb0);
       if (nb > 1) score = __fadd_rn(score, xb1);
-      for (int r = 2; r < nb; ++r) {
-        const int src = st + r >= nst ? st + r - nst : st + r;
-        score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, src));
-      }
+      for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, 4 * r));
       PROF_ADD(4);
       int tok = V;                                          // V: no token selected in this round
       float tval = 0.0f;
       int tnext = s, adv = nb;                              // adv: frames fully passed in this round
-      if (nb < win_rows && j_ready) {
+      if (!(wide && nb == 1) && nb < win_rows && j_ready) {
         const int k_row = nb == 0 ? k : 0;                  // symbols already emitted in that row's frame
         if (!j_rescan) {
           tok = j_tok; tval = j_val; tnext = j_next;
@@ -721,7 +757,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           { const int cz = __shfl_sync(0xffffffffu, cause, jl); if (cz & 1) _pacc[12] += 1; if (cz & 2) _pacc[13] += 1; if (cz & 4) _pacc[14] += 1; }
 #endif
           const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
-          for (int i = lane; i < L.n; i += 32) tokidx[lds_v2(L.addr + 8u * i).x & kTokMask] = static_cast<int16_t>(i);
+          for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = static_cast<int16_t>(i); }
           __syncwarp();
           ValId best{bf16_bits_to_float(lds_u16(rrow + 2u * V)), V};
           int bn = s;
@@ -735,14 +771,22 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             if (better(c2, best)) { best = c2; bn = bound ? nx : -1; }
           }
           __syncwarp();
-          for (int i = lane; i < L.n; i += 32) tokidx[lds_v2(L.addr + 8u * i).x & kTokMask] = -1;
+          for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = -1; }
           const Pick pk = warp_pick(best, bn);
           tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
           if (tok == V) { score = __fadd_rn(score, tval); ++adv; }   // blank after all: that frame is passed too
         }
         if (tok != V) {
           score = __fadd_rn(score, tval);
-          if (lane == 0 && n_out < p.out_cap) { out_tok[n_out] = tok; out_frm[n_out] = t + nb; }
+          // emitted tokens are staged in shared memory and written out 32 at a time, coalesced
+          if (lane == 0) emit_buf[n_out & 31] = make_int2(tok, t + nb);
+          if ((n_out & 31) == 31) {
+            __syncwarp();
+            const int2 e = emit_buf[lane];
+            const int o = (n_out & ~31) + lane;
+            if (o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+            __syncwarp();
+          }
           ++n_out;
           k = k_row + 1;
           if (k == S) ++adv;                                // the frame closes by force
@@ -751,13 +795,14 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       PROF_ADD(10);
       PROF_COUNT(8);
       // ---- hand the passed frames' slots back, move on -------------------------------------------------
-      if (own && rank < adv) {
-        mbar_arrive_relaxed_addr(my_free_a);
-        my_f += nst; my_lead = (my_lead + lead_wrap) & 15;
+      if (lane < adv) {                                     // lane r frees the slot of frame t + r
+        const int sr = st + lane >= nst ? st + lane - nst : st + lane;
+        mbar_arrive_relaxed_addr(freeb_a + 8u * sr);
       }
       if (adv > 0 && (tok == V || k == S)) k = 0;
       t += adv;
       st += adv; if (st >= nst) st -= nst;
+      lead = (lead + adv * lead_step) & 15;
       PROF_ADD(5);
       if (tok != V && bound && tnext != s) {
         s = tnext;
@@ -771,13 +816,13 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w);
           } else {
             const TbRsRec r4 = rsrec_g[s];
-            for (int i = lane; i < r4.count && i < V; i += 32) lbuf[i] = rsent_g[r4.begin + i];
+            for (int i = lane; i < r4.count && i < V + 4; i += 32) lbuf[i] = rsent_g[r4.begin + i];
             __syncwarp();
             L.addr = smem_u32(lbuf); L.n = r4.count; L.D = r4.D; L.bmag = r4.bmag;
           }
           L.sorted = true;
         } else {
-          build_list(strec, tokent, rec.n_states, rec.max_depth, s, lam, R, lbuf, cls_seen, cls16, L, lane, p.status);
+          build_list(strec, tokent, rec.n_states, rec.max_depth, s, lam, R, V, lbuf, cls_seen, cls16, L, lane, p.status);
         }
       }
       PROF_ADD(11);
@@ -791,6 +836,12 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       tb_prof_blk[4 * blockIdx.x + 3] = _pacc[9];
     }
 #endif
+    if ((n_out & 31) != 0) {                  // the tokens still staged
+      __syncwarp();
+      const int2 e = emit_buf[lane];
+      const int o = (n_out & ~31) + lane;
+      if (lane < (n_out & 31) && o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+    }
     if (failed || t < end) *abort_flag = 1;   // left early: let the other roles stop too
     if (lane == 0) {
       p.out_counts[b] = n_out; p.out_scores[b] = score; p.out_states[b] = s;
@@ -819,7 +870,7 @@ int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int3
   const int W = d.V + 1;
   if (d.dtype != TB_BF16 || d.persistent || d.n_dur != 0) return 1;
   if (d.sv != 1 || d.ss != W || d.st < static_cast<int64_t>(d.S) * W || d.sb < 0) return 1;
-  if (d.S > kSMax || d.V > 256 * kNitMax || d.V >= (1 << TB_RS_TOK_BITS) || max_states >= (1 << (32 - TB_RS_TOK_BITS))) return 1;
+  if (d.S > kSMax || d.V > 256 * kNitMax || 2 * (d.V + 1) > (1 << TB_RS_TOK_BITS) || max_states >= (1 << (32 - TB_RS_TOK_BITS))) return 1;
   if (reinterpret_cast<uintptr_t>(d.logits) & 1) return 1;
   FastParams P;
   P.d = d;
@@ -841,7 +892,7 @@ int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int3
   const int per_stage = P.slot_bytes + 16 + kSumStageBytes;
   int nst = (budget - fixed - 64) / per_stage;
   if (nst > kStagesMax) nst = kStagesMax;
-  if (nst < 4) return 1;
+  if (nst < 9) return 1;   // the decider's window spans eight stages
   P.nst = nst;
   const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes);
   if (so.total > budget) return 1;

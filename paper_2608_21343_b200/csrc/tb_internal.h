@@ -48,18 +48,21 @@ static_assert(sizeof(TbStateRec) == 16 && sizeof(TbTokEnt) == 16, "16-byte recor
 // weights crossed before the arc's chain state, added in walk order) and the arc's target.  With
 // them a state change costs the pipelined kernel one record load instead of a chain walk.  Built
 // only for graphs whose lists stay small (TB_RS_MAX_ENTRIES) and whose ids fit the packing.
+// Every list is padded to a multiple of four entries with sentinels {token = vocab (the blank
+// column), lb = -inf, target 0}, which can never be selected, so that readers may take four
+// entries at a time without a bounds test.
 struct TbRsRec {
-  int32_t begin, count;  // range in the TbRsEnt section
+  int32_t begin, count;  // range in the TbRsEnt section (count includes the padding)
   float D;               // sum of the suffix-link weights of the whole chain, in walk order
   float bmag;            // |lambda| * (|D| + largest root arc weight): scale of the rounding margin
 };
 struct TbRsEnt {
-  uint32_t dst_tok;      // target state << 11 | token
+  uint32_t dst_tok;      // target state << 12 | 2 * token (the token's byte offset in a bf16 row)
   float lb;
 };
 static_assert(sizeof(TbRsRec) == 16 && sizeof(TbRsEnt) == 8, "record sizes");
 #define TB_RS_MAX_ENTRIES (1 << 18)
-#define TB_RS_TOK_BITS 11
+#define TB_RS_TOK_BITS 12   /* 2 * token < 4096, i.e. vocab + 1 <= 2048 */
 
 uint64_t tb_hash_class_map(const int32_t* case_class, int32_t vocab);
 
