@@ -32,6 +32,9 @@ from paper_2608_21343_b200 import workloads as W  # noqa: E402
 
 METRIC = "boosted_greedy_decode_frames_per_s_B128"
 UNIT = "frames/s"
+# DRAM read + write bytes per logits row of the decode kernel, from an ncu capture of a 32-stream launch
+# (152.9 MB for 72000 rows); the kernel runs one block per stream, so traffic scales with the stream count.
+NCU_DRAM_BYTES_PER_ROW = 2123.0
 
 
 def load_peaks():
@@ -218,7 +221,9 @@ def main():
         "gpu_launches": args.steps * 1,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "greedy decode",
+                     "traffic": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S,
+                     "traffic_note": "ncu dram read+write of a 32-stream launch scaled by streams",
+                     "peak_kind": f"of {peak_kind}", "kernel": "k_greedy_fast (one launch per decode)",
                      "rows_visited": visited, "bytes_per_row": row_bytes,
                      "all_rows_GBs": streamed, "all_rows_frac": streamed / peak},
         "rows_visited_per_frame": visited / (w.B * w.T),

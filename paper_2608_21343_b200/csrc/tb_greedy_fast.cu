@@ -39,6 +39,7 @@ constexpr int kThreadsF = kWarpsF * 32;
 constexpr int kSMax = 4;        // rows per frame the ring bookkeeping is sized for
 constexpr int kNitMax = 8;      // 256 tokens per pass iteration: V <= 2048 (kernel instantiated for 1, 2, 4, 8)
 constexpr int kGroupDeep = 32;  // up to this many boosted tokens, the decider resolves eight rows per round, four lanes each
+constexpr int kAllRowsDeep = 64; // all-rows mode in a state that just repeated itself: at most this many boosted tokens
 constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -594,14 +595,19 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     PROF_FLUSH();
   } else if (warp == 0) {
     // ================================ decider =================================================
-    // Works in rounds.  With few boosted tokens in the current state (the usual case) the warp is
-    // eight groups of four lanes; group q looks at one row: group 0 at the current row (t, k),
-    // group q >= 1 at row (t + q, 0), the row the decode reaches if everything before it is blank.
-    // The four lanes share the state's boosted tokens, combine with two shuffles, and every group
-    // resolves its row under the current graph state.  One ballot tells how many leading rows are
-    // blank; they are consumed at once, and the first row that selects a token ends the round,
-    // because the graph state changes there.  With many boosted tokens all 32 lanes share them and
-    // only the current row is resolved.
+    // Works in rounds over a window of eight frames.  The warp is eight groups of four lanes; group q
+    // stands for frame t + q.  A round resolves rows in parallel under the current graph state and then
+    // consumes as many of them, in decode order, as the state allows:
+    //   shared mode (the usual case: the state's chain boosts a few tokens and the last token changed
+    //     the state): group q resolves one row -- group 0 the current row (t, k), group q >= 1 row
+    //     (t + q, 0), the row the decode reaches there if everything before it is blank; the four lanes
+    //     share the boosted tokens and combine with two shuffles.  One ballot tells how many leading
+    //     rows are blank; they are consumed at once and the first row that selects a token ends the
+    //     round, because the graph state changes there.
+    //   all-rows mode (no boosted tokens -- root state or unboosted stream -- or the last token left the
+    //     state unchanged): lane ql of group q resolves row (t + q, ql) on its own, so a round can walk
+    //     through tokens too, as long as they leave the state unchanged.
+    //   wide mode (many boosted tokens): all 32 lanes share them and resolve the current row only.
     const float R = root_stats[2];
     const uint32_t ring_a = smem_u32(ring), freeb_a = smem_u32(freeb);
     const uint32_t cache_a = smem_u32(dyn + so.cache);
@@ -621,46 +627,40 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     L.addr = smem_u32(lbuf); L.n = 0; L.sorted = true; L.D = 0.0f; L.bmag = fabsf(lam) * R;
 
     const int q = lane >> 2, ql = lane & 3;                 // group and lane within the group
-    const int win_rows = min(8, nst - 1);
+    constexpr int kWin = 8;                                 // frames per window (the launcher guarantees nst > kWin)
     int t = 0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0, lead = lead0;
     float score = 0.0f;
     int32_t* out_tok = p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
     int32_t* out_frm = p.out_frames + static_cast<int64_t>(b) * p.out_cap;
     const int max_rounds = p.frames * S + p.frames + 8;
     uint32_t spins = 0;
-    bool failed = false;
+    bool failed = false, stable = false, no_allrows = false;
     for (int it = 0; t < end; ++it) {
       if (it >= max_rounds) { if (lane == 0) atomicOr(p.status, TB_STATUS_STEP_LIMIT); break; }
       PROF_T0();
-      const bool wide = L.n > kGroupDeep;                   // many boosted tokens: the whole warp takes the current row
-      const int rq = wide ? 0 : q;                          // window row of this lane
+      // ---- mode and this lane's row --------------------------------------------------------------------
+      const bool allrows = !no_allrows && (L.n == 0 || (stable && L.n <= kAllRowsDeep));
+      const bool wide = !allrows && L.n > kGroupDeep;
+      const int rq = wide ? 0 : q;                          // window frame of this lane
+      const int rk = allrows ? ql : (rq == 0 ? k : 0);      // row of that frame
       int stq = st + rq; if (stq >= nst) stq -= nst;
-      const uint32_t koff = rq == 0 ? static_cast<uint32_t>(k) : 0u;
-      const uint32_t sum_a = summ_a + stq * kSumStageBytes + koff * 32u;
+      const uint32_t sum_a = summ_a + stq * kSumStageBytes + min(rk, kSMax - 1) * 32u;
       // the half with the sequence word is read first: when it matches, the other half is complete
       const uint4 q1 = lds_v4_volatile(sum_a + 16u);
       const uint4 q0 = lds_v4_volatile(sum_a);
-      const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + rq * lead_step) & 15) + koff * row_bytes;
-      const bool ready = rq < win_rows && t + rq < end && q1.w == static_cast<uint32_t>(t + rq) + 1u;
-      if (!__shfl_sync(0xffffffffu, ready, 0)) {           // the current row itself is not summarised yet: poll
-        if (++spins > kSpinLimit || ((spins & 255u) == 0u && *abort_flag)) {
-          if (spins > kSpinLimit) { *abort_flag = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
-          failed = true; break;
-        }
-        --it;                                               // a poll is not a round
-        continue;
-      }
-      spins = 0;
+      const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + rq * lead_step) & 15) + rk * row_bytes;
+      const bool in_row = rk < S && (rq > 0 || rk >= k);   // all-rows mode: rows before (t, k) are behind us
+      const bool ready = in_row && t + rq < end && q1.w == static_cast<uint32_t>(t + rq) + 1u;
       PROF_ADD(2);
       const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
       const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
       bool rescan = (q1.z & kSumOvf) != 0;
-      // ---- the tokens the state's chain boosts: exact values; this lane takes every 4th (or 32nd) entry
+      // ---- the tokens the state's chain boosts: exact values; the lanes that share a row split the list
       float wv = -INFINITY;
       uint32_t wdt = 2u * static_cast<uint32_t>(V);
       bool in_deep = false;
       {
-        const int lstep = wide ? 32 : 4, l0 = wide ? lane : ql;
+        const int lstep = allrows ? 1 : (wide ? 32 : 4), l0 = allrows ? 0 : (wide ? lane : ql);
         int i = l0;
         for (; i + lstep < L.n; i += 2 * lstep) {           // two entries in flight
           const uint2 e0 = lds_v2(L.addr + 8u * i), e1 = lds_v2(L.addr + 8u * (i + lstep));
@@ -680,7 +680,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       }
       PROF_ADD(3);
       // combine over the lanes that share the row
-      if (L.n > 0) {
+      if (L.n > 0 && !allrows) {
         if (wide) {
           const uint32_t key = fkey(wv);
           const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
@@ -726,60 +726,29 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         }
       }
       const bool is_blank = ready && !rescan && !(wv >= xb);   // a tie with blank goes to the token
-      const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank) & 0x11111111u;   // one bit per group
-      const unsigned stop_m = ~blank_m & 0x11111111u;
-      int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : 8;          // leading blank rows
-      if (wide) nb = (blank_m & 1u) ? 1 : 0;
-      PROF_ADD(7);
-      // ---- the leading blanks, then the row after them ------------------------------------------------
-      const int jl = wide ? 0 : 4 * min(nb, 7);
-      const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
-      const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
-      const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
-      const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
-      const float j_val = __shfl_sync(0xffffffffu, wv, jl);
-      const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
-      if (nb > 0) score = __fadd_rn(score, xb0);
-      if (nb > 1) score = __fadd_rn(score, xb1);
-      for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, 4 * r));
-      PROF_ADD(4);
-      int tok = V;                                          // V: no token selected in this round
+      const unsigned blank_all = __ballot_sync(0xffffffffu, is_blank);
+      int tok = V;                                          // V: the round's last row selected no token
       float tval = 0.0f;
-      int tnext = s, adv = nb;                              // adv: frames fully passed in this round
-      if (!(wide && nb == 1) && nb < win_rows && j_ready) {
-        const int k_row = nb == 0 ? k : 0;                  // symbols already emitted in that row's frame
-        if (!j_rescan) {
-          tok = j_tok; tval = j_val; tnext = j_next;
-        } else {
-          // exact evaluation of that row by the whole warp from shared memory
-          PROF_COUNT(9);
-#ifdef TB_PROFILE
-          { const int cz = __shfl_sync(0xffffffffu, cause, jl); if (cz & 1) _pacc[12] += 1; if (cz & 2) _pacc[13] += 1; if (cz & 4) _pacc[14] += 1; }
-#endif
-          const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
-          for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = static_cast<int16_t>(i); }
-          __syncwarp();
-          ValId best{bf16_bits_to_float(lds_u16(rrow + 2u * V)), V};
-          int bn = s;
-          for (int tk = lane; tk < V; tk += 32) {
-            const int i = tokidx[tk];
-            float lbv; int nx;
-            if (i >= 0) { const uint2 e = lds_v2(L.addr + 8u * i); lbv = __uint_as_float(e.y); nx = static_cast<int>(e.x >> TB_RS_TOK_BITS); }
-            else { const int c = cls16[tk]; lbv = __fmul_rn(lam, __fadd_rn(L.D, rootcw[c])); nx = rootdst[c]; }
-            const float x = bf16_bits_to_float(lds_u16(rrow + 2u * tk));
-            const ValId c2{bound ? __fadd_rn(x, lbv) : x, tk};
-            if (better(c2, best)) { best = c2; bn = bound ? nx : -1; }
+      int tnext = s, adv = 0;                               // adv: frames fully passed in this round
+      bool progress = false;
+      if (allrows) {
+        // ---- walk the window row by row, through tokens too, while the state stays what it is ----------
+        const unsigned ready_all = __ballot_sync(0xffffffffu, ready && !rescan);
+        const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
+        PROF_ADD(7);
+        int fq = 0, pos = k;
+        for (int guard = 0; guard < 4 * kWin && fq < kWin; ++guard) {
+          const int li = 4 * fq + pos;
+          if (!((ready_all >> li) & 1u)) break;
+          progress = true;
+          if ((blank_all >> li) & 1u) {
+            score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, li));
+            ++fq; pos = 0;
+            continue;
           }
-          __syncwarp();
-          for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = -1; }
-          const Pick pk = warp_pick(best, bn);
-          tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
-          if (tok == V) { score = __fadd_rn(score, tval); ++adv; }   // blank after all: that frame is passed too
-        }
-        if (tok != V) {
-          score = __fadd_rn(score, tval);
-          // emitted tokens are staged in shared memory and written out 32 at a time, coalesced
-          if (lane == 0) emit_buf[n_out & 31] = make_int2(tok, t + nb);
+          const int wt = __shfl_sync(0xffffffffu, wtok, li);
+          score = __fadd_rn(score, __shfl_sync(0xffffffffu, wv, li));
+          if (lane == 0) emit_buf[n_out & 31] = make_int2(wt, t + fq);
           if ((n_out & 31) == 31) {
             __syncwarp();
             const int2 e = emit_buf[lane];
@@ -788,22 +757,110 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             __syncwarp();
           }
           ++n_out;
-          k = k_row + 1;
-          if (k == S) ++adv;                                // the frame closes by force
+          const bool keep = (keep_all >> li) & 1u;
+          if (!keep) { tok = wt; tnext = __shfl_sync(0xffffffffu, wnext, li); }
+          if (++pos == S) { ++fq; pos = 0; }
+          if (!keep) break;
         }
+        adv = fq; k = pos;
+        if (!progress) {
+          // the current row is not summarised yet (poll), or it needs the exact rescan (next round, shared mode)
+          const unsigned resc_all = __ballot_sync(0xffffffffu, ready && rescan);
+          if ((resc_all >> k) & 1u) no_allrows = true;
+        }
+        PROF_ADD(4);
+        PROF_ADD(10);
+      } else {
+        // ---- the leading blanks, then the row after them --------------------------------------------------
+        const unsigned blank_m = blank_all & 0x11111111u;   // one bit per group
+        const unsigned stop_m = ~blank_m & 0x11111111u;
+        int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : kWin;
+        if (wide) nb = (blank_m & 1u) ? 1 : 0;
+        PROF_ADD(7);
+        const int jl = wide ? 0 : 4 * min(nb, kWin - 1);
+        const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
+        const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
+        const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
+        const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
+        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+        const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
+        if (nb > 0) score = __fadd_rn(score, xb0);
+        if (nb > 1) score = __fadd_rn(score, xb1);
+        for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, 4 * r));
+        adv = nb;
+        progress = nb > 0;
+        PROF_ADD(4);
+        if (!(wide && nb == 1) && nb < kWin && j_ready) {
+          progress = true;
+          const int k_row = nb == 0 ? k : 0;                // symbols already emitted in that row's frame
+          if (!j_rescan) {
+            tok = j_tok; tval = j_val; tnext = j_next;
+          } else {
+            // exact evaluation of that row by the whole warp from shared memory
+            PROF_COUNT(9);
+#ifdef TB_PROFILE
+            { const int cz = __shfl_sync(0xffffffffu, cause, jl); if (cz & 1) _pacc[12] += 1; if (cz & 2) _pacc[13] += 1; if (cz & 4) _pacc[14] += 1; }
+#endif
+            const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
+            for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = static_cast<int16_t>(i); }
+            __syncwarp();
+            ValId best{bf16_bits_to_float(lds_u16(rrow + 2u * V)), V};
+            int bn = s;
+            for (int tk = lane; tk < V; tk += 32) {
+              const int i = tokidx[tk];
+              float lbv; int nx;
+              if (i >= 0) { const uint2 e = lds_v2(L.addr + 8u * i); lbv = __uint_as_float(e.y); nx = static_cast<int>(e.x >> TB_RS_TOK_BITS); }
+              else { const int c = cls16[tk]; lbv = __fmul_rn(lam, __fadd_rn(L.D, rootcw[c])); nx = rootdst[c]; }
+              const float x = bf16_bits_to_float(lds_u16(rrow + 2u * tk));
+              const ValId c2{bound ? __fadd_rn(x, lbv) : x, tk};
+              if (better(c2, best)) { best = c2; bn = bound ? nx : -1; }
+            }
+            __syncwarp();
+            for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = -1; }
+            const Pick pk = warp_pick(best, bn);
+            tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
+            if (tok == V) { score = __fadd_rn(score, tval); ++adv; }   // blank after all: that frame is passed too
+          }
+          if (tok != V) {
+            score = __fadd_rn(score, tval);
+            // emitted tokens are staged in shared memory and written out 32 at a time, coalesced
+            if (lane == 0) emit_buf[n_out & 31] = make_int2(tok, t + nb);
+            if ((n_out & 31) == 31) {
+              __syncwarp();
+              const int2 e = emit_buf[lane];
+              const int o = (n_out & ~31) + lane;
+              if (o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+              __syncwarp();
+            }
+            ++n_out;
+            k = k_row + 1;
+            if (k == S) ++adv;                              // the frame closes by force
+          }
+        }
+        if (adv > 0 && (tok == V || k == S)) k = 0;
+        PROF_ADD(10);
       }
-      PROF_ADD(10);
       PROF_COUNT(8);
+      if (!progress) {                                      // the current row is not summarised yet: poll
+        if (++spins > kSpinLimit || ((spins & 255u) == 0u && *abort_flag)) {
+          if (spins > kSpinLimit) { *abort_flag = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
+          failed = true; break;
+        }
+        --it;                                               // a poll is not a round
+        continue;
+      }
+      spins = 0;
+      if (!allrows) no_allrows = false;
       // ---- hand the passed frames' slots back, move on -------------------------------------------------
       if (lane < adv) {                                     // lane r frees the slot of frame t + r
         const int sr = st + lane >= nst ? st + lane - nst : st + lane;
         mbar_arrive_relaxed_addr(freeb_a + 8u * sr);
       }
-      if (adv > 0 && (tok == V || k == S)) k = 0;
       t += adv;
       st += adv; if (st >= nst) st -= nst;
       lead = (lead + adv * lead_step) & 15;
       PROF_ADD(5);
+      if (tok != V) stable = (tnext == s);                  // the last token left the state unchanged
       if (tok != V && bound && tnext != s) {
         s = tnext;
         if (s <= 0) {
