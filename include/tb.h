@@ -61,6 +61,7 @@ extern "C" {
 #define TB_MAX_VOCAB 8192           /* non-blank tokens */
 #define TB_MAX_PHRASE_LEN 255       /* tokens per phrase (graph depth is stored in a byte) */
 #define TB_MAX_BEAM 32
+#define TB_NOALLOC_MAX_STREAMS 256 /* streams per tb_greedy_decode_noalloc call */
 
 typedef struct tb_graph tb_graph; /* immutable compiled graph, host memory */
 typedef struct tb_batch tb_batch; /* device arena + slot table + per-slot state */
@@ -248,6 +249,44 @@ int tb_beam_step(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t 
  */
 int tb_beam_backtrace(tb_batch *b, int32_t B, int32_t K, int32_t max_len, int32_t *out_tokens,
                       int32_t *out_lens, void *stream);
+
+/*
+ * Unboosted greedy RNNT decoding that allocates nothing.  (The paper has no counterpart; this is
+ * a service to one kind of caller.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the moment it decodes --
+ * a serving process whose device memory was divided up front among its models and that treats any
+ * later cudaMalloc as a fault, or a latency-critical thread that cannot afford cudaMalloc because
+ * it synchronises the device and would stall the other streams' decoding.  Such callers cannot use
+ * tb_batch_create (it allocates the arena, the slot table and the status word), and without a
+ * batch there is no graph, so this call decodes every stream as unbound (model id -1): per stream
+ * exactly what tb_greedy_decode returns for a slot without a graph.
+ *
+ * The decode kernel's own working memory (one status word and one "unbound" slot record per
+ * stream) lives in a fixed array inside the library, 33 KB, which every GPU that loads the library
+ * holds until the process exits; hence the limit of TB_NOALLOC_MAX_STREAMS streams per call.  The
+ * call makes no cudaMalloc / cudaFree and uses no allocating library routine.  Every call shares
+ * that one array: the call clears what it needs to start from zero, in stream order, but two calls
+ * that overlap on the GPU (different streams, or different host threads) race on it -- callers must
+ * serialise their calls per device.  The first call on a device looks up the array's device address
+ * (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *
+ *   device       the GPU that holds the caller's buffers
+ *   logits       device, dtype TB_BF16 or TB_F32, logical shape [B, T, S, vocab+1]
+ *   strides      host int64 [4], element strides (any layout)
+ *   lengths      device int32 [B] or NULL (= T)
+ *   out_tokens / out_frames   device int32 [B, T*S]
+ *   out_counts / out_states   device int32 [B] (states are all -1)
+ *   out_scores   device float [B]
+ *   out_status   device int32 [1] or NULL: receives the kernel's status word (TB_STATUS_* bits, 0 = fine)
+ * Asynchronous on `stream` like the other decode calls.  Errors: TB_ERR_INVALID_ARG (B outside
+ * [1, TB_NOALLOC_MAX_STREAMS], vocab outside [1, TB_MAX_VOCAB], bad dtype, NULL pointers, sizes
+ * < 1), TB_ERR_CUDA.
+ */
+int tb_greedy_decode_noalloc(int device, const void *logits, int dtype, int32_t B, int32_t T, int32_t S,
+                             int32_t vocab, const int64_t *strides, const int32_t *lengths,
+                             int32_t *out_tokens, int32_t *out_frames, int32_t *out_counts, float *out_scores,
+                             int32_t *out_states, int32_t *out_status, void *stream);
 
 #ifdef __cplusplus
 }

@@ -60,6 +60,8 @@ _SIGS = {
     "tb_beam_reset": (C.c_int, [_vp]),
     "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                           _vp, _vp, _vp]),
 }
 for _name, (_res, _args) in _SIGS.items():
     _fn = getattr(_lib, _name)       # AttributeError here = the library lacks a declared symbol
@@ -276,3 +278,22 @@ def tb_beam_backtrace(batch: Batch, B: int, K: int, max_len: int, stream=None):
     _check(_lib.tb_beam_backtrace(batch.handle, B, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
            "tb_beam_backtrace")
     return toks, lens
+
+
+TB_NOALLOC_MAX_STREAMS = 256
+
+
+def tb_greedy_decode_noalloc(logits: torch.Tensor, out: dict, lengths=None, stream=None) -> dict:
+    """Unboosted greedy decode for callers that must not allocate device memory at decode time
+    (a server with a fixed, pre-divided memory budget; a thread that cannot afford the device-wide
+    synchronisation of cudaMalloc).  The library's own working memory is a fixed array inside the
+    library, so the caller brings every buffer: ``out`` must hold preallocated device tensors
+    ``tokens`` / ``frames`` [B, T*S], ``counts`` / ``states`` [B] (int32), ``scores`` [B] (float32) and
+    optionally ``status`` [1] (int32).  Calls that overlap on one GPU race on the shared array."""
+    B, T, S, W = logits.shape
+    st = _strides4(logits)
+    _check(_lib.tb_greedy_decode_noalloc(logits.device.index or 0, _dp(logits), _logit_dtype(logits), B, T, S, W - 1,
+                                         _hp(st), _dp(lengths), _dp(out["tokens"]), _dp(out["frames"]),
+                                         _dp(out["counts"]), _dp(out["scores"]), _dp(out["states"]),
+                                         _dp(out.get("status")), _stream(stream)), "tb_greedy_decode_noalloc")
+    return out
