@@ -154,8 +154,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
+    from paper_2608_21343_b200 import sharding
+
     # ---- inputs: this rank's own 128 streams (stream ids offset by rank), graphs compiled and bound
-    streams = [rank * w.B + i for i in range(w.B)]
+    streams = sharding.rank_streams(rank, w.B)
     data = W.batch_inputs(w, streams)
     host_logits = torch.from_numpy(data["logits"]).view(torch.bfloat16).pin_memory()
     logits = host_logits.to(dev, non_blocking=True)
@@ -195,13 +197,8 @@ def main():
     total_ms, each_ms = timed(lambda: tb.tb_greedy_decode(batch, logits, out=out), args.steps, args.warmup)
     clocks = sampler.stop()
     assert tb.tb_batch_status(batch) == 0, "a kernel recorded a violated bound"
-    ms = total_ms / args.steps
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
-    frames_total = w.B * w.T * world
-    value = frames_total / (ms * 1e-3)
+    job = sharding.job_throughput(w.B * w.T, total_ms / args.steps, device=dev)   # max over ranks of the time
+    ms, value = job["ms"], job["value"]
 
     counts = out["counts"].cpu().numpy()
     frames = out["frames"].cpu().numpy()

@@ -85,13 +85,6 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Arrival without release ordering.  The decider uses it to hand a ring slot back: it has only
-// read the slot, and every such read has completed (its value fed a ballot) before the arrival,
-// so nothing needs to be made visible -- while a releasing arrival would also wait for the
-// decider's earlier global stores (emitted tokens) to be acknowledged by the memory system.
-__device__ __forceinline__ void mbar_arrive_relaxed(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
@@ -103,26 +96,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
-}
-// The same test, letting the hardware park the warp for up to `ns` before it answers "not yet".
-__device__ __forceinline__ bool mbar_try_wait_park(uint64_t* bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the block is aborting or the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 255u && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  atomicOr(status, TB_STATUS_WAIT_TIMEOUT);
-  return false;
 }
 // Bounded wait for the roles that are not latency critical: parks the warp between polls so that
 // it does not take issue slots or shared-memory pipeline cycles from the decider.
@@ -185,15 +158,10 @@ __device__ __forceinline__ uint4 lds_v4_volatile(uint32_t a) {
 __device__ __forceinline__ void sts_v4_volatile(uint32_t a, uint4 v) {
   asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
-__device__ __forceinline__ bool mbar_test_addr(uint32_t bar_addr, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar_addr), "r"(parity) : "memory");
-  return ok != 0;
-}
+// Arrival without release ordering.  The decider uses it to hand a ring slot back: it has only
+// read the slot, and every such read has completed (its value fed a ballot) before the arrival,
+// so nothing needs to be made visible -- while a releasing arrival would also wait for the
+// decider's earlier global stores (emitted tokens) to be acknowledged by the memory system.
 __device__ __forceinline__ void mbar_arrive_relaxed_addr(uint32_t bar_addr) {
   asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar_addr) : "memory");
 }
@@ -302,54 +270,46 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
   const __nv_bfloat16 thr = __float2bfloat16_rd(thr_f);
   const __nv_bfloat162 thr2 = __halves2bfloat162(thr, thr);
 
-  // pass 2: each lane notes its candidates (token id << 16 | logit bits); four fit, more flag the row
-  int nc = 0;
-  uint32_t cd[4] = {0u, 0u, 0u, 0u};
+  // pass 2: one bit per element of this lane that reaches the threshold (bit 2i + h: word i, half h)
+  uint32_t hits = 0;
 #pragma unroll
   for (int i = 0; i < 4 * NIT; ++i) {
-    const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);
-    if (mk) {
-      const uint32_t idx = static_cast<uint32_t>(((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 - p);
-      if (mk & 0xFFFFu) { cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = (idx << 16) | (w[i] & 0xFFFFu); ++nc; }
-      if (mk >> 16) { cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = ((idx + 1) << 16) | (w[i] >> 16); ++nc; }
-    }
-  }
-  if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
-    cd[3] = cd[2]; cd[2] = cd[1]; cd[1] = cd[0]; cd[0] = (static_cast<uint32_t>(tail_idx) << 16) | tail_bits; ++nc;
+    const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);          // 0xFFFF per half that passes
+    if (4 * NIT <= 16) hits |= ((mk & 1u) | ((mk >> 15) & 2u)) << (2 * i);
+    else if (mk) hits |= 1u << (i & 31);                             // NIT = 8: one bit per word, both halves re-tested below
   }
   // exact root-boosted values of this lane's candidates: best (value, lowest id) and runner-up value
   ValId b{-INFINITY, INT32_MAX};
   float sec = -INFINITY;
-  if (!__any_sync(0xffffffffu, nc > 4)) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (j < nc) {
-        const int id = static_cast<int>(cd[j] >> 16);
-        const ValId c{__fadd_rn(bf16_bits_to_float(cd[j] & 0xFFFFu), h.rootcb[h.cls16[id]]), id};
+  while (hits) {
+    const int bit = __ffs(hits) - 1;
+    hits &= hits - 1u;
+    if (4 * NIT <= 16) {
+      const int i = bit >> 1;
+      const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 + (bit & 1) - p;
+      if (idx >= 0 && idx < V) {                            // masked elements pass only a threshold of -inf
+        const ValId c{__fadd_rn(row_at(rowp, idx), h.rootcb[h.cls16[idx]]), idx};
         if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
       }
-    }
-  } else {
-    // some lane met more candidates than it can note (a low row maximum): evaluate every hit in place
+    } else {
+      const int i = bit;
+      const int idx0 = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 - p;
 #pragma unroll
-    for (int i = 0; i < 4 * NIT; ++i) {
-      const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);
-      if (mk) {
-        const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 - p;
-        if (mk & 0xFFFFu) {
-          const ValId c{__fadd_rn(bf16_bits_to_float(w[i] & 0xFFFFu), h.rootcb[h.cls16[idx]]), idx};
-          if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
-        }
-        if (mk >> 16) {
-          const ValId c{__fadd_rn(bf16_bits_to_float(w[i] >> 16), h.rootcb[h.cls16[idx + 1]]), idx + 1};
-          if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+      for (int hh = 0; hh < 2; ++hh) {
+        const int idx = idx0 + hh;
+        if (idx >= 0 && idx < V) {
+          const float x = row_at(rowp, idx);
+          if (x >= __bfloat162float(thr)) {
+            const ValId c{__fadd_rn(x, h.rootcb[h.cls16[idx]]), idx};
+            if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
+          }
         }
       }
     }
-    if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
-      const ValId c{__fadd_rn(bf16_bits_to_float(tail_bits), h.rootcb[h.cls16[tail_idx]]), tail_idx};
-      if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
-    }
+  }
+  if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
+    const ValId c{__fadd_rn(bf16_bits_to_float(tail_bits), h.rootcb[h.cls16[tail_idx]]), tail_idx};
+    if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
   }
   // across the warp: best (value, lowest id) and the runner-up value
   const uint32_t key = fkey(b.v);
@@ -519,16 +479,32 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    float bmin = 0.0f, bmax = 0.0f, R = 0.0f;               // tokens without a root arc have beta = 0
+  {
+    // extremes of the root arcs' lambda * w (tokens without a root arc have beta = 0) and of |w|
+    float bmin = 0.0f, bmax = 0.0f, R = 0.0f;
     if (bound) {
       const int e = g.arc_begin[1];
-      for (int a = g.arc_begin[0]; a < e; ++a) {
-        const int c = g.arc_cls[a];
-        bmin = fminf(bmin, rootcb[c]); bmax = fmaxf(bmax, rootcb[c]); R = fmaxf(R, fabsf(rootcw[c]));
+      for (int a = g.arc_begin[0] + tid; a < e; a += kThreadsF) {
+        const float wv = __fadd_rn(0.0f, g.arc_w[a]);
+        const float cb = __fmul_rn(lam, wv);
+        bmin = fminf(bmin, cb); bmax = fmaxf(bmax, cb); R = fmaxf(R, fabsf(wv));
       }
     }
-    root_stats[0] = bmin; root_stats[1] = bmax; root_stats[2] = R;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      bmin = fminf(bmin, __shfl_xor_sync(0xffffffffu, bmin, off));
+      bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, off));
+      R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, off));
+    }
+    float* part = reinterpret_cast<float*>(dyn + so.lbuf);   // not in use yet
+    if (lane == 0) { part[3 * warp] = bmin; part[3 * warp + 1] = bmax; part[3 * warp + 2] = R; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w2 = 1; w2 < kWarpsF; ++w2) {
+        bmin = fminf(bmin, part[3 * w2]); bmax = fmaxf(bmax, part[3 * w2 + 1]); R = fmaxf(R, part[3 * w2 + 2]);
+      }
+      root_stats[0] = bmin; root_stats[1] = bmax; root_stats[2] = R;
+    }
   }
   __syncthreads();
 
@@ -578,19 +554,25 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     h.cls16 = cls16; h.rootcb = rootcb; h.rootcw = rootcw; h.rootdst = rootdst; h.V = V; h.nit = (V + 255) / 256;
     h.beta_min = root_stats[0]; h.beta_max = root_stats[1]; h.dbeta = __fsub_rn(root_stats[1], root_stats[0]);
     h.bmag_max = fabsf(lam) * ((bound ? rec.d_max : 0.0f) + root_stats[2]);
-    const int64_t n_rows = static_cast<int64_t>(end) * S;
-    for (int64_t r = hid; r < n_rows; r += kHelpers) {
-      const int f = static_cast<int>(r / S), k = static_cast<int>(r - static_cast<int64_t>(f) * S);
-      const int st = f % nst;
-      const uint32_t ph = (f / nst) & 1;
+    // rows are dealt round-robin: this warp takes rows hid, hid + kHelpers, ... of the stream, in order
+    int f = hid / S, k = hid - f * S;                     // frame and row in frame
+    int st = f % nst;
+    uint32_t ph = (f / nst) & 1;
+    int lead = (lead0 + f * lead_step) & 15;
+    for (; f < end;) {
       PROF_T0();
       if (!mbar_wait_parked(&full[st], ph, abort_flag, p.status)) break;
       PROF_ADD(0);
-      const int lead = static_cast<int>((lead0 + static_cast<int64_t>(f) * lead_step) & 15);
       const unsigned char* slot = ring + static_cast<size_t>(st) * P.slot_bytes;
       summarize_row<NIT>(h, slot, lead + k * row_bytes, summ_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
       if (lane == 0) mbar_arrive(&freeb[st]);
       PROF_ADD(1);
+      k += kHelpers;
+      while (k >= S) {                                      // on to a later frame
+        k -= S; ++f;
+        lead = (lead + lead_step) & 15;
+        if (++st == nst) { st = 0; ph ^= 1u; }
+      }
     }
     PROF_FLUSH();
   } else if (warp == 0) {
