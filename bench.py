@@ -119,6 +119,103 @@ def run_reference(args, w):
     }))
 
 
+def side_measurement(args):
+    """Workloads 3-5 on one GPU: one JSON line each, with that workload's own metric (not the headline)."""
+    import torch
+    from paper_2608_21343_b200 import binding as tb
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+
+    def timed(fn, n, warm):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    if args.workload == 3:
+        w = W.get_workload(3, **({"B": args.streams} if args.streams else {}))
+        data = W.batch_inputs(w)
+        t0 = time.perf_counter()
+        graphs = [tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class) for p in data["phrases"]]
+        compile_ms = (time.perf_counter() - t0) * 1e3 / w.B
+        batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=int(4.5e6) * w.B + (1 << 20))
+        for i, g in enumerate(graphs):
+            tb.tb_batch_bind_stream(batch, i, g)
+        logits = torch.from_numpy(data["logits"]).view(torch.bfloat16).to(dev)
+        out = tb.tb_greedy_decode(batch, logits)
+        ms = timed(lambda: tb.tb_greedy_decode(batch, logits, out=out), args.steps, args.warmup)
+        assert tb.tb_batch_status(batch) == 0
+        print(json.dumps({"metric": "boosted_greedy_decode_frames_per_s_large_lists", "value": w.B * w.T / (ms * 1e-3),
+                          "unit": UNIT, "ms_per_step": ms, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                          "config": {"workload": w.name, "B": w.B, "T": w.T, "states_per_graph": graphs[0].view()["n_states"]},
+                          "graph_compile_ms_per_list": compile_ms, "data": "synthetic"}))
+    elif args.workload == 4:
+        w = W.get_workload(4)
+        data = W.batch_inputs(w)
+        B, T, E, _ = data["logits"].shape
+        K = w.K
+        batch = tb.tb_batch_create(w.V, w.vocab.case_class, B, max_beam=K, max_tree_steps=T * E, arena_bytes=64 << 20)
+        for i, p in enumerate(data["phrases"]):
+            tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class))
+        logits = torch.from_numpy(data["logits"]).view(torch.bfloat16).to(dev)
+        sb, st, se, _ = logits.stride()
+        scores = torch.empty((B, K), device=dev)
+        states = torch.empty((B, K), dtype=torch.int32, device=dev)
+        live = torch.zeros((B, K), dtype=torch.uint8, device=dev)
+        par = torch.empty((B, K), dtype=torch.int32, device=dev)
+        tok = torch.empty_like(par)
+
+        def run():
+            scores.fill_(float("-inf")); scores[:, 0] = 0.0
+            states.fill_(-1); states[:, 0] = 0
+            tb.tb_beam_reset(batch)
+            for t in range(T):
+                for e in range(E):
+                    tb.tb_beam_step(batch, logits, sb, 0, e == 0, scores, states, live, par, tok, offset=t * st + e * se)
+        ms = timed(run, max(2, args.steps // 5), 1)
+        print(json.dumps({"metric": "beam_decode_frames_per_s_K4_B32", "value": B * T / (ms * 1e-3), "unit": UNIT,
+                          "ms_per_decode": ms, "us_per_beam_step": ms * 1e3 / (T * E), "n_gpus": 1,
+                          "config": {"workload": w.name, "B": B, "K": K, "T": T, "E": E,
+                                     "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
+    else:
+        w = W.get_workload(5, **({"B": args.streams} if args.streams else {}))
+        sched = W.ChurnSchedule(w)
+        batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
+        n_chunks, lat, binds, t_compile = 40 + 10 * args.steps, [], 0, 0.0
+        bufs = []
+        for c in range(n_chunks):
+            chunk, lengths, bl = sched.next_chunk()
+            t0 = time.perf_counter()
+            gs = [(sl, tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class)) for sl, _, p in bl]
+            t_compile += time.perf_counter() - t0
+            dl = torch.from_numpy(chunk).view(torch.bfloat16).to(dev)      # a fresh buffer per chunk: nothing stays in L2
+            dv = torch.from_numpy(lengths).to(dev)
+            bufs = (bufs + [dl])[-8:]
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for sl, g in gs:
+                tb.tb_batch_bind_stream(batch, sl, g)
+            tb.tb_stream_chunk(batch, dl, w.n_dur, dv)
+            b.record()
+            torch.cuda.synchronize()
+            lat.append(a.elapsed_time(b))
+            binds += len(bl)
+        lat = np.array(lat[10:])
+        print(json.dumps({"metric": "streaming_tdt_chunk_latency_ms", "p50": float(np.percentile(lat, 50)),
+                          "p99": float(np.percentile(lat, 99)), "unit": "ms", "higher_is_better": False, "n_gpus": 1,
+                          "config": {"workload": w.name, "slots": w.B, "chunk_frames": w.chunk, "chunks": len(lat),
+                                     "binds_in_timed_region": True, "rebinds": binds - w.B},
+                          "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
+                          "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds), "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -128,7 +225,12 @@ def main():
     ap.add_argument("--streams", type=int, default=0, help="override B (profiling captures use a small case)")
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5],
+                    help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn: side measurements")
     args = ap.parse_args()
+    if args.workload != 2:
+        side_measurement(args)
+        return
     args.warmup = max(args.warmup, 3)
     over = {}
     if args.streams:

@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, off));
       R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, off));
     }
-    float* part = reinterpret_cast<float*>(dyn + so.lbuf);   // not in use yet
+    float* part = reinterpret_cast<float*>(dyn + so.ring);   // the ring is not in use yet (3 floats per warp)
     if (lane == 0) { part[3 * warp] = bmin; part[3 * warp + 1] = bmax; part[3 * warp + 2] = R; }
     __syncthreads();
     if (tid == 0) {

@@ -241,3 +241,69 @@ def test_pipelined_kernel_large_lists_not_cached(tb):
     w = W.get_workload(3, B=2, T=150)
     data = W.batch_inputs(w)
     both_kernels(tb, w, data, what="w3")
+
+
+@pytest.mark.parametrize("V,S", [(5, 3), (17, 2), (33, 4)])
+def test_pipelined_kernel_tiny_vocabularies(tb, V, S):
+    """Rows far shorter than one 16-byte-block pass of the helpers."""
+    rng = np.random.default_rng(V)
+    B, T = 5, 60
+    cc = (np.arange(V) // 2).astype(np.int32)
+    x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32)
+    x[..., V] += 0.5
+    xb = W.f32_to_bf16_bits(x)
+    lists = [[[int(t) for t in rng.integers(0, V, size=rng.integers(1, 4))] for _ in range(6)] for _ in range(B)]
+    lists[2] = None
+    batch = tb.tb_batch_create(V, cc, B + 2, arena_bytes=1 << 20)          # more slots than streams
+    for i, p in enumerate(lists):
+        tb.tb_batch_bind_stream(batch, i, None if p is None else tb.tb_graph_compile(p, V, case_class=cc))
+    lengths = torch.tensor([T, T + 50, 7, 0, T - 1], dtype=torch.int32, device="cuda:0")   # T + 50 is clamped to T
+    out = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=lengths))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(lists):
+        g = None if p is None else O.Graph(p, V, case_class=cc)
+        check_greedy(out, i, O.greedy_rnnt(g, xb[i], min(int(lengths[i]), T)), f"V{V}")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_pipelined_kernel_random_configurations(tb, seed):
+    """Random shapes, class maps, list sizes, weights, lambda, lengths and base offsets: both kernels
+    against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    V = int(rng.choice([9, 40, 255, 256, 257, 511, 1023, 1500, 2046]))
+    S = int(rng.integers(1, 5))
+    B, T = int(rng.integers(1, 7)), int(rng.integers(1, 70))
+    n_cls = int(rng.integers(1, V + 1))
+    cc = rng.integers(0, n_cls, size=V).astype(np.int32)
+    lam = float(rng.choice([1.0, 0.5, 2.0, -0.5]))
+    x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32) * float(rng.choice([0.3, 1.0, 3.0]))
+    x[..., V] += float(rng.choice([0.0, 1.0, 3.0]))
+    if seed % 3 == 0:
+        x = np.round(x * 2) / 2                                   # coarse grid: exact ties everywhere
+    xb = W.f32_to_bf16_bits(x)
+    lists, weights = [], []
+    hot = rng.integers(0, V, size=max(2, V // 20))                # a small pool makes phrases chain and repeat
+    for b in range(B):
+        n = int(rng.integers(0, 60))
+        ph = [[int(t) for t in rng.choice(hot, size=rng.integers(1, 6))] for _ in range(n)]
+        lists.append(None if (b == 1 and B > 1) else ph)
+        weights.append([[float(rng.choice([0.5, 1.0, 1.5, 2.0])) for _ in p] for p in ph])
+    batch = tb.tb_batch_create(V, cc, B, arena_bytes=8 << 20)
+    for i, p in enumerate(lists):
+        if p is not None:
+            tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc, token_weights=weights[i], lam=lam))
+    shift = int(rng.integers(0, 9))
+    flat = torch.zeros(shift + xb.size + 8, dtype=torch.bfloat16, device="cuda:0")
+    view = flat[shift:shift + xb.size].view(B, T, S, V + 1)
+    view.copy_(to_device(xb))
+    lens = rng.integers(0, T + 1, size=B).astype(np.int32)
+    dl = torch.from_numpy(lens).to("cuda:0")
+    fast = to_host(tb.tb_greedy_decode(batch, view, lengths=dl))
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
+    gen = to_host(tb.tb_greedy_decode(batch, view, lengths=dl))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(lists):
+        g = None if p is None else O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam)
+        ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
+        check_greedy(fast, i, ref, f"seed{seed} pipelined V{V} S{S}")
+        check_greedy(gen, i, ref, f"seed{seed} general V{V} S{S}")
