@@ -179,8 +179,24 @@ def side_measurement(args):
                 for e in range(E):
                     tb.tb_beam_step(batch, logits, sb, 0, e == 0, scores, states, live, par, tok, offset=t * st + e * se)
         ms = timed(run, max(2, args.steps // 5), 1)
+        # the same T*E steps captured once in a CUDA graph and replayed: no host work per step
+        graph_ms = None
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                run()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            cg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cg):
+                run()
+            graph_ms = timed(cg.replay, max(2, args.steps // 5), 1)
+        except Exception as exc:  # noqa: BLE001
+            graph_ms = f"capture failed: {exc}"
         print(json.dumps({"metric": "beam_decode_frames_per_s_K4_B32", "value": B * T / (ms * 1e-3), "unit": UNIT,
                           "ms_per_decode": ms, "us_per_beam_step": ms * 1e3 / (T * E), "n_gpus": 1,
+                          "cuda_graph_ms_per_decode": graph_ms,
                           "config": {"workload": w.name, "B": B, "K": K, "T": T, "E": E,
                                      "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
     else:

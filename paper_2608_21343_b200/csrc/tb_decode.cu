@@ -11,6 +11,7 @@
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kBeamList = 64;   // boosted tokens per hypothesis kept for the next-state lookup of the beam step
 
 struct ChainSmem {
   int32_t state[TB_CHAIN_MAX];
@@ -25,6 +26,61 @@ struct StepSmem {
   int32_t t, k, s, tok, go;
 };
 
+// Token view of the current graph state, for graphs that carry resolved lists (see TbRsRec):
+// instead of walking the suffix chain into a class-indexed bonus vector, the state's finished list
+// is scattered into two token-indexed arrays; a token that is not in the list ("plain") gets
+// fl(lambda * fl(D + root arc weight of its class)) and the root arc's target.
+struct TokView {
+  float* rootcw;      // [C] root arc weight per class (0 if none)
+  int32_t* rootdst;   // [C] root arc target per class (0 if none)
+  float* tok_lb;      // [V] finished additive term of a listed token
+  int32_t* tok_dst;   // [V] target state of a listed token, -1: not listed
+  uint16_t* cur_tok;  // tokens of the list now scattered (to undo it)
+  int32_t n;
+  float D;
+};
+__host__ __device__ inline size_t tokview_bytes(int V, int C) {
+  return static_cast<size_t>(C) * 8 + static_cast<size_t>(V) * 8 + ((static_cast<size_t>(V) * 2 + 8 + 15) & ~size_t(15));
+}
+__device__ inline void tokview_init(TokView& tv, unsigned char* mem, int V, int C, const GraphPtrs& g) {
+  tv.rootcw = reinterpret_cast<float*>(mem);
+  tv.rootdst = reinterpret_cast<int32_t*>(mem + 4 * static_cast<size_t>(C));
+  tv.tok_lb = reinterpret_cast<float*>(mem + 8 * static_cast<size_t>(C));
+  tv.tok_dst = reinterpret_cast<int32_t*>(mem + 8 * static_cast<size_t>(C) + 4 * static_cast<size_t>(V));
+  tv.cur_tok = reinterpret_cast<uint16_t*>(mem + 8 * static_cast<size_t>(C) + 8 * static_cast<size_t>(V));
+  tv.n = 0; tv.D = 0.0f;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) { tv.rootcw[c] = 0.0f; tv.rootdst[c] = 0; }
+  for (int v = threadIdx.x; v < V; v += blockDim.x) tv.tok_dst[v] = -1;
+  __syncthreads();
+  const int e = g.arc_begin[1];
+  for (int a = g.arc_begin[0] + threadIdx.x; a < e; a += blockDim.x) {
+    const int c = g.arc_cls[a];
+    if (c >= 0 && c < C) { tv.rootcw[c] = __fadd_rn(0.0f, g.arc_w[a]); tv.rootdst[c] = g.arc_dst[a]; }
+  }
+  __syncthreads();
+}
+// Block-wide: replace the scattered list by that of state s (the root's list is empty, D = 0).
+__device__ inline void tokview_enter(TokView& tv, const unsigned char* blob, const TbSlotRec& rec, int32_t s, int V,
+                                     int32_t* status) {
+  for (int i = threadIdx.x; i < tv.n; i += blockDim.x) {
+    const int tk = tv.cur_tok[i];
+    if (tk < V) tv.tok_dst[tk] = -1;
+  }
+  __syncthreads();
+  if (s < 0 || s >= rec.n_states) { if (threadIdx.x == 0) atomicOr(status, TB_STATUS_BAD_STATE); s = 0; }
+  const TbRsRec r = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[s];
+  const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent) + r.begin;
+  const int n = min(r.count, V + 4);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const TbRsEnt e = ent[i];
+    const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
+    if (tk < V) { tv.tok_lb[tk] = e.lb; tv.tok_dst[tk] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
+    tv.cur_tok[i] = static_cast<uint16_t>(tk);
+  }
+  __syncthreads();
+  tv.n = n; tv.D = r.D;
+}
+
 template <typename LT>
 __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
   extern __shared__ __align__(16) unsigned char dyn[];
@@ -36,6 +92,10 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
   const TbSlotRec rec = p.slots[b];
   const bool bound = rec.n_states > 0;
   const GraphPtrs g = graph_of(p.arena, rec);
+  const unsigned char* blob = p.arena + rec.blob_off;
+  const bool use_tv = bound && rec.n_rsent >= 0 && p.tokview;   // resolved lists: token view instead of a chain walk
+  TokView tv;
+  if (use_tv) tokview_init(tv, dyn, p.V, p.C, g);
   const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.sb;
   const int V = p.V;
 
@@ -63,14 +123,24 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
       break;
     }
     if (bound && built_for != s) {
-      build_bonus(g, s, p.C, bvec, nvec, sm.chain.state, sm.chain.acc, &sm.chain.len, p.status);
+      if (use_tv) tokview_enter(tv, blob, rec, s, V, p.status);
+      else build_bonus(g, s, p.C, bvec, nvec, sm.chain.state, sm.chain.acc, &sm.chain.len, p.status);
       built_for = s;
     }
     const LT* row = base + static_cast<int64_t>(t - t0) * p.st + static_cast<int64_t>(k) * p.ss;
     ValId best{-INFINITY, INT32_MAX};
     for (int v = threadIdx.x; v <= V; v += kThreads) {
       float x = LogitLoad<LT>::at(row + static_cast<int64_t>(v) * p.sv);
-      float val = (bound && v < V) ? __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)])) : x;
+      float val = x;
+      if (bound && v < V) {
+        if (use_tv) {
+          const float lb = tv.tok_dst[v] >= 0 ? tv.tok_lb[v]
+                                              : __fmul_rn(g.lambda, __fadd_rn(tv.D, tv.rootcw[__ldg(p.cls + v)]));
+          val = __fadd_rn(x, lb);
+        } else {
+          val = __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)]));
+        }
+      }
       ValId c{val, v};
       if (better(c, best)) best = c;
     }
@@ -99,7 +169,7 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
         if (p.out_durs) p.out_durs[o] = dur;
       }
       ++n_out;
-      if (bound) s = nvec[__ldg(p.cls + tok)];
+      if (bound) s = use_tv ? (tv.tok_dst[tok] >= 0 ? tv.tok_dst[tok] : tv.rootdst[__ldg(p.cls + tok)]) : nvec[__ldg(p.cls + tok)];
       if (p.n_dur > 0 && dur > 0) { t += dur; k = 0; }
       else { ++k; if (k == p.S) { ++t; k = 0; } }
     }
@@ -148,9 +218,14 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int V = p.V, K = p.K, W = V + 1;
   float* cand = reinterpret_cast<float*>(dyn);                         // [K, V+1]
-  float* bvec = cand + static_cast<size_t>(K) * W;                     // [C]
+  unsigned char* aux = dyn + ((static_cast<size_t>(K) * W * sizeof(float) + 15) & ~size_t(15));
+  float* bvec = reinterpret_cast<float*>(aux);                         // [C]   (chain-walk path)
   int32_t* nvec = reinterpret_cast<int32_t*>(bvec + p.C);              // [C]
   __shared__ ChainSmem chain;
+  // token-view path: per hypothesis a copy of its state's short list, to find the next state of a pick
+  __shared__ uint16_t hl_tok[TB_MAX_BEAM][kBeamList];
+  __shared__ int32_t hl_dst[TB_MAX_BEAM][kBeamList];
+  __shared__ int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
   __shared__ BeamKey red[kThreads / 32 + 1];
   __shared__ float h_score[TB_MAX_BEAM];
   __shared__ int32_t h_state[TB_MAX_BEAM];
@@ -162,6 +237,10 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   const bool bound = rec.n_states > 0;
   const GraphPtrs g = graph_of(p.arena, rec);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned char* blob = p.arena + rec.blob_off;
+  const bool use_tv = bound && rec.n_rsent >= 0 && p.tokview;
+  TokView tv;
+  if (use_tv) tokview_init(tv, aux, V, p.C, g);
 
   if (threadIdx.x < K) {
     const int64_t o = static_cast<int64_t>(b) * K + threadIdx.x;
@@ -175,13 +254,32 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   // all candidate values of the live hypotheses
   for (int k = 0; k < K; ++k) {
     if (h_score[k] == -INFINITY || !h_live[k]) continue;  // uniform across the block
-    if (bound) build_bonus(g, h_state[k], p.C, bvec, nvec, chain.state, chain.acc, &chain.len, p.status);
+    if (use_tv) {
+      tokview_enter(tv, blob, rec, h_state[k], V, p.status);
+      for (int i = threadIdx.x; i < tv.n && i < kBeamList; i += kThreads) {
+        const int tk = tv.cur_tok[i];
+        hl_tok[k][i] = static_cast<uint16_t>(tk);
+        hl_dst[k][i] = tk < V ? tv.tok_dst[tk] : 0;
+      }
+      if (threadIdx.x == 0) hl_n[k] = tv.n <= kBeamList ? tv.n : -1;
+    } else if (bound) {
+      build_bonus(g, h_state[k], p.C, bvec, nvec, chain.state, chain.acc, &chain.len, p.status);
+    }
     const LT* row = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride +
                     static_cast<int64_t>(k) * p.hyp_stride;
     const float sc = h_score[k];
     for (int v = threadIdx.x; v < W; v += kThreads) {
       float x = LogitLoad<LT>::at(row + v);
-      float val = (bound && v < V) ? __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)])) : x;
+      float val = x;
+      if (bound && v < V) {
+        if (use_tv) {
+          const float lb = tv.tok_dst[v] >= 0 ? tv.tok_lb[v]
+                                              : __fmul_rn(g.lambda, __fadd_rn(tv.D, tv.rootcw[__ldg(p.cls + v)]));
+          val = __fadd_rn(x, lb);
+        } else {
+          val = __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)]));
+        }
+      }
       cand[static_cast<size_t>(k) * W + v] = __fadd_rn(sc, val);
     }
     __syncthreads();
@@ -234,7 +332,14 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
       token = (c.tkey == V + 1) ? -1 : c.tkey;
       state = h_state[parent];
       if (token >= 0 && token != V) {
-        if (bound) state = walk_next(g, state, __ldg(p.cls + token), p.status);
+        if (use_tv && hl_n[parent] >= 0) {
+          int nx = tv.rootdst[__ldg(p.cls + token)];          // a pick that the parent's list does not hold is a plain token
+          for (int i = 0; i < hl_n[parent]; ++i)
+            if (hl_tok[parent][i] == token) { nx = hl_dst[parent][i]; break; }
+          state = nx;
+        } else if (bound) {
+          state = walk_next(g, state, __ldg(p.cls + token), p.status);
+        }
         lv = h_live[parent];
       }
     }
@@ -288,8 +393,12 @@ int set_smem(F* fn, size_t bytes) {
 
 }  // namespace
 
-int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream) {
-  const size_t smem = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+int tb_launch_decode_general(const TbDecodeParams& p_in, cudaStream_t stream) {
+  TbDecodeParams p = p_in;
+  size_t smem = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+  // graphs with resolved lists exist only for vocabularies whose token view fits comfortably
+  p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
+  if (p.tokview && tokview_bytes(p.V, p.C) > smem) smem = tokview_bytes(p.V, p.C);
   int rc;
   if (p.dtype == TB_BF16) {
     if ((rc = set_smem(k_decode_general<uint16_t>, smem)) != TB_OK) return rc;
@@ -301,9 +410,12 @@ int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream) {
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
-int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream) {
-  const size_t smem = static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) +
-                      static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
+  TbBeamParams p = p_in;
+  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+  p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
+  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
   int rc;
   if (p.dtype == TB_BF16) {

@@ -13,6 +13,7 @@ struct TbDecodeParams {
   int64_t sb, st, ss, sv;    // element strides: stream, frame, row-in-frame, token
   const int32_t* lengths;    // device [n_streams] or null
   int32_t persistent;        // 0: offline greedy (fresh state); 1: streaming (TbSlotState)
+  int32_t tokview;           // set by the launcher: shared memory is sized for the token view of resolved lists
   int32_t* out_tokens; int32_t* out_frames; int32_t* out_durs; int32_t* out_counts;
   float* out_scores; int32_t* out_states; int32_t* out_cursors;
   int32_t out_cap;           // tokens per stream the output arrays can hold
@@ -24,6 +25,7 @@ struct TbDecodeParams {
 struct TbBeamParams {
   const void* logits; int dtype;
   int32_t B, K, V, C, new_frame, step;
+  int32_t tokview;           // set by the launcher, as in TbDecodeParams
   int64_t stream_stride, hyp_stride;
   float* scores; int32_t* states; uint8_t* live; int32_t* out_parent; int32_t* out_token;
   int2* tree;                // [steps, B, K] (parent, token) or null
