@@ -198,21 +198,6 @@ struct BeamKey {  // order: value descending, token key ascending, parent ascend
   float v;
   int32_t tkey, par;
 };
-__device__ __forceinline__ bool before(const BeamKey& a, const BeamKey& b) {
-  return a.v > b.v || (a.v == b.v && (a.tkey < b.tkey || (a.tkey == b.tkey && a.par < b.par)));
-}
-__device__ __forceinline__ BeamKey warp_first(BeamKey x) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    BeamKey y;
-    y.v = __shfl_xor_sync(0xffffffffu, x.v, off);
-    y.tkey = __shfl_xor_sync(0xffffffffu, x.tkey, off);
-    y.par = __shfl_xor_sync(0xffffffffu, x.par, off);
-    if (before(y, x)) x = y;
-  }
-  return x;
-}
-
 template <typename LT>
 __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   extern __shared__ __align__(16) unsigned char dyn[];
@@ -226,7 +211,9 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   __shared__ uint16_t hl_tok[TB_MAX_BEAM][kBeamList];
   __shared__ int32_t hl_dst[TB_MAX_BEAM][kBeamList];
   __shared__ int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
-  __shared__ BeamKey red[kThreads / 32 + 1];
+  __shared__ int32_t h_beg[TB_MAX_BEAM], h_cnt[TB_MAX_BEAM];
+  __shared__ float h_D[TB_MAX_BEAM];
+  __shared__ unsigned long long red64[kThreads / 32];
   __shared__ float h_score[TB_MAX_BEAM];
   __shared__ int32_t h_state[TB_MAX_BEAM];
   __shared__ uint8_t h_live[TB_MAX_BEAM];
@@ -252,72 +239,109 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   __syncthreads();
 
   // all candidate values of the live hypotheses
-  for (int k = 0; k < K; ++k) {
-    if (h_score[k] == -INFINITY || !h_live[k]) continue;  // uniform across the block
-    if (use_tv) {
-      tokview_enter(tv, blob, rec, h_state[k], V, p.status);
-      for (int i = threadIdx.x; i < tv.n && i < kBeamList; i += kThreads) {
-        const int tk = tv.cur_tok[i];
-        hl_tok[k][i] = static_cast<uint16_t>(tk);
-        hl_dst[k][i] = tk < V ? tv.tok_dst[tk] : 0;
-      }
-      if (threadIdx.x == 0) hl_n[k] = tv.n <= kBeamList ? tv.n : -1;
-    } else if (bound) {
-      build_bonus(g, h_state[k], p.C, bvec, nvec, chain.state, chain.acc, &chain.len, p.status);
-    }
-    const LT* row = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride +
-                    static_cast<int64_t>(k) * p.hyp_stride;
-    const float sc = h_score[k];
-    for (int v = threadIdx.x; v < W; v += kThreads) {
-      float x = LogitLoad<LT>::at(row + v);
-      float val = x;
-      if (bound && v < V) {
-        if (use_tv) {
-          const float lb = tv.tok_dst[v] >= 0 ? tv.tok_lb[v]
-                                              : __fmul_rn(g.lambda, __fadd_rn(tv.D, tv.rootcw[__ldg(p.cls + v)]));
-          val = __fadd_rn(x, lb);
-        } else {
-          val = __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)]));
-        }
-      }
-      cand[static_cast<size_t>(k) * W + v] = __fadd_rn(sc, val);
+  if (use_tv) {
+    // every hypothesis at once: its state's record, then all plain values, then the listed tokens on top
+    if (threadIdx.x < K) {
+      const int k = threadIdx.x;
+      int32_t st = h_state[k];
+      if (st < 0 || st >= rec.n_states) { if (h_score[k] != -INFINITY && h_live[k]) atomicOr(p.status, TB_STATUS_BAD_STATE); st = 0; }
+      const TbRsRec r = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[st];
+      h_beg[k] = r.begin; h_cnt[k] = r.count; h_D[k] = r.D;
+      hl_n[k] = r.count <= kBeamList ? r.count : -1;
     }
     __syncthreads();
+    const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+    for (int v = threadIdx.x; v < W; v += kThreads) {
+      const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
+      for (int k = 0; k < K; ++k) {
+        if (h_score[k] == -INFINITY || !h_live[k]) continue;
+        const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
+        const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
+        cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+      }
+    }
+    __syncthreads();
+    const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
+    for (int k = 0; k < K; ++k) {
+      if (h_score[k] == -INFINITY || !h_live[k]) continue;
+      for (int i = threadIdx.x; i < h_cnt[k]; i += kThreads) {
+        const TbRsEnt e = ent[h_beg[k] + i];
+        const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
+        if (i < kBeamList) { hl_tok[k][i] = static_cast<uint16_t>(tk); hl_dst[k][i] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
+        if (tk < V) {
+          const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + tk);
+          cand[static_cast<size_t>(k) * W + tk] = __fadd_rn(h_score[k], __fadd_rn(x, e.lb));
+        }
+      }
+    }
+    __syncthreads();
+  } else {
+    for (int k = 0; k < K; ++k) {
+      if (h_score[k] == -INFINITY || !h_live[k]) continue;  // uniform across the block
+      if (bound) build_bonus(g, h_state[k], p.C, bvec, nvec, chain.state, chain.acc, &chain.len, p.status);
+      const LT* row = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride +
+                      static_cast<int64_t>(k) * p.hyp_stride;
+      const float sc = h_score[k];
+      for (int v = threadIdx.x; v < W; v += kThreads) {
+        float x = LogitLoad<LT>::at(row + v);
+        float val = (bound && v < V) ? __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)])) : x;
+        cand[static_cast<size_t>(k) * W + v] = __fadd_rn(sc, val);
+      }
+      __syncthreads();
+    }
   }
 
-  // K rounds: the first candidate, in order, that comes strictly after the previous pick
-  BeamKey prev{INFINITY, -2, -2};
-  const BeamKey none{-INFINITY, INT32_MAX, INT32_MAX};
-  for (int r = 0; r < K; ++r) {
-    BeamKey best = none;
+  // K rounds of selection.  A candidate's place in the order (value descending, token key ascending,
+  // parent ascending) is one 64-bit key: the order-preserving image of the value above the inverted
+  // (token key, parent) pair; keys are distinct, 0 means "none".  Every thread keeps the best key among
+  // its own candidates that has not been picked yet; after a round only the owner of the pick rescans.
+  auto make_key = [](float v, int tkey, int k) -> unsigned long long {
+    const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
+    const uint32_t hi = u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+    const uint32_t lo = 0xFFFFFFFFu - (static_cast<uint32_t>(tkey) * 32u + static_cast<uint32_t>(k));
+    return (static_cast<unsigned long long>(hi) << 32) | lo;
+  };
+  // best key below `limit` among this thread's candidates: tokens v = tid, tid + 256, ... of every live
+  // hypothesis, plus (thread k) the carried candidate of a frozen hypothesis k
+  auto scan_mine = [&](unsigned long long limit) -> unsigned long long {
+    unsigned long long m = 0ull;
     for (int k = 0; k < K; ++k) {
       if (h_score[k] == -INFINITY) continue;
       if (!h_live[k]) {
-        if (threadIdx.x == 0) {
-          BeamKey c{h_score[k], V + 1, k};
-          if (before(prev, c) && before(c, best)) best = c;
-        }
+        if (threadIdx.x == k) { const unsigned long long kk = make_key(h_score[k], V + 1, k); if (kk < limit && kk > m) m = kk; }
         continue;
       }
+      const float* ck = cand + static_cast<size_t>(k) * W;
       for (int v = threadIdx.x; v < W; v += kThreads) {
-        BeamKey c{cand[static_cast<size_t>(k) * W + v], v, k};
-        if (before(prev, c) && before(c, best)) best = c;
+        const unsigned long long kk = make_key(ck[v], v, k);
+        if (kk < limit && kk > m) m = kk;
       }
     }
-    best = warp_first(best);
-    if (lane == 0) red[warp] = best;
+    return m;
+  };
+  unsigned long long mine = scan_mine(~0ull);
+  for (int r = 0; r < K; ++r) {
+    unsigned long long m = mine;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) { const unsigned long long o = __shfl_xor_sync(0xffffffffu, m, off); if (o > m) m = o; }
+    if (lane == 0) red64[warp] = m;
     __syncthreads();
-    if (warp == 0) {
-      BeamKey y = lane < kThreads / 32 ? red[lane] : none;
-      y = warp_first(y);
-      if (lane == 0) red[kThreads / 32] = y;
+    unsigned long long best = red64[0];
+#pragma unroll
+    for (int w2 = 1; w2 < kThreads / 32; ++w2) { const unsigned long long o = red64[w2]; if (o > best) best = o; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      BeamKey c{-INFINITY, INT32_MAX, INT32_MAX};
+      if (best != 0ull) {
+        const uint32_t lo = 0xFFFFFFFFu - static_cast<uint32_t>(best & 0xFFFFFFFFull);
+        c.tkey = static_cast<int32_t>(lo >> 5); c.par = static_cast<int32_t>(lo & 31u);
+        c.v = c.tkey == V + 1 ? h_score[c.par] : cand[static_cast<size_t>(c.par) * W + c.tkey];
+      }
+      sel[r] = c;
     }
-    __syncthreads();
-    best = red[kThreads / 32];
-    if (threadIdx.x == 0) sel[r] = best;
-    prev = best;           // once `none` is reached every later round yields `none` again
-    __syncthreads();
+    if (best != 0ull && mine == best) mine = scan_mine(best);   // this thread owned the pick: find its next best
   }
+  __syncthreads();
 
   // new hypotheses, the hypothesis tree
   if (threadIdx.x < K) {
