@@ -38,7 +38,7 @@ constexpr int kHelpers = kWarpsF - kWarpsF / 4;
 constexpr int kThreadsF = kWarpsF * 32;
 constexpr int kSMax = 4;        // rows per frame the ring bookkeeping is sized for
 constexpr int kNitMax = 8;      // 256 tokens per pass iteration: V <= 2048 (kernel instantiated for 1, 2, 4, 8)
-constexpr int kGroupDeep = 32;  // up to this many boosted tokens, the decider resolves eight rows per round, four lanes each
+constexpr int kGroupDeep = 64;  // up to this many boosted tokens, the decider resolves eight rows per round, four lanes each
 constexpr int kAllRowsDeep = 64; // all-rows mode in a state that just repeated itself: at most this many boosted tokens
 constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
 constexpr uint32_t kSpinLimit = 1u << 20;
