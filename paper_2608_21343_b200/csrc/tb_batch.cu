@@ -85,13 +85,15 @@ struct tb_batch {
   std::vector<int32_t> slot_n_states;
   Staging staging[kStagingRing];
   int next_staging = 0;
+  void* seg_scratch = nullptr;      // working memory of the two-segment greedy decode (grown on demand)
+  size_t seg_scratch_bytes = 0;
 };
 
 static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch);
   for (auto& s : b->staging) {
     if (s.host) cudaFreeHost(s.host);
     if (s.done) cudaEventDestroy(s.done);
@@ -254,7 +256,17 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
       max_cache = b->slot_cache_bytes[i] > max_cache ? b->slot_cache_bytes[i] : max_cache;
       max_states = b->slot_n_states[i] > max_states ? b->slot_n_states[i] : max_states;
     }
-    rc = tb_launch_greedy_fast(p, max_cache, max_states, static_cast<cudaStream_t>(stream_));
+    // the two-segment decode keeps what its second segment produces in scratch memory of the batch; growing it
+    // frees the old block first (cudaFree waits for earlier work), so one decode per batch at a time
+    const size_t want = tb_greedy_fast_scratch_bytes(B, T, S);
+    if (want > b->seg_scratch_bytes && want <= (static_cast<size_t>(1) << 30)) {
+      cudaFree(b->seg_scratch);
+      b->seg_scratch = nullptr; b->seg_scratch_bytes = 0;
+      if (cudaMalloc(&b->seg_scratch, want) == cudaSuccess) b->seg_scratch_bytes = want;
+      else cudaGetLastError();
+    }
+    rc = tb_launch_greedy_fast(p, max_cache, max_states, b->seg_scratch, b->seg_scratch_bytes,
+                               static_cast<cudaStream_t>(stream_));
     if (rc != 1) return rc;
   }
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));

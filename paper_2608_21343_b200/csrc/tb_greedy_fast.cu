@@ -42,6 +42,8 @@ constexpr int kGroupDeep = 64;  // up to this many boosted tokens, the decider r
 constexpr int kAllRowsDeep = 64; // all-rows mode in a state that just repeated itself: at most this many boosted tokens
 constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr int kSegMinFrames = 192;  // streams at least this long are decoded as two segments (see the header)
+constexpr int kSegWarm = 32;        // frames the second segment decodes before the first frame it answers for
 
 #ifdef TB_PROFILE
 __device__ unsigned long long tb_prof[16];
@@ -99,13 +101,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait for the roles that are not latency critical: parks the warp between polls so that
 // it does not take issue slots or shared-memory pipeline cycles from the decider.
-__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait_parked(uint64_t* bar, uint32_t parity, volatile int* flags, int pipe, int32_t* status) {
   for (uint32_t it = 0; it < (kSpinLimit >> 2); ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     __nanosleep(256);
-    if ((it & 63u) == 63u && *abort_flag) return false;
+    if ((it & 7u) == 7u && flags[pipe]) return false;
   }
-  *abort_flag = 1;
+  flags[0] = 1; flags[1] = 1;
   atomicOr(status, TB_STATUS_WAIT_TIMEOUT);
   return false;
 }
@@ -168,9 +170,10 @@ __device__ __forceinline__ void mbar_arrive_relaxed_addr(uint32_t bar_addr) {
 
 struct Smem {  // byte offsets into dynamic shared memory, computed identically on host and device
   int ring, bars, summ, cls16, rootcb, rootcw, rootdst, lbuf, cls_seen, tokidx, emit, misc, cache, total;
+  int lbuf_sz, cls_seen_sz, tokidx_sz;   // the deciders' private areas exist once per segment, this far apart
 };
 __host__ __device__ inline int up16(int x) { return (x + 15) & ~15; }
-__host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes) {
+__host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes, int npipes) {
   Smem s;
   int o = 0;
   s.ring = o; o += nst * slot_bytes;
@@ -180,11 +183,12 @@ __host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int
   s.rootcb = o; o += up16(4 * C);
   s.rootcw = o; o += up16(4 * C);
   s.rootdst = o; o += up16(4 * C);
-  s.lbuf = o; o += up16(8 * (V + 4)); // boosted-token list of the current state when it is not read from the cache
-  s.cls_seen = o; o += up16(2 * C);   // class -> position in lbuf while a list is being built
-  s.tokidx = o; o += up16(2 * V);     // token -> position in the current list (filled only for an exact rescan)
-  s.emit = o; o += 32 * 8;            // emitted (token, frame) pairs waiting for a coalesced store
-  s.misc = o; o += 64;
+  s.lbuf_sz = up16(8 * (V + 4)); s.cls_seen_sz = up16(2 * C); s.tokidx_sz = up16(2 * V);
+  s.lbuf = o; o += npipes * s.lbuf_sz;         // boosted-token list of the current state when it is not read from the cache
+  s.cls_seen = o; o += npipes * s.cls_seen_sz; // class -> position in lbuf while a list is being built
+  s.tokidx = o; o += npipes * s.tokidx_sz;     // token -> position in the current list (filled only for an exact rescan)
+  s.emit = o; o += npipes * 32 * 8;            // emitted (token, frame) pairs waiting for a coalesced store
+  s.misc = o; o += 96;
   s.cache = o; o += up16(cache_bytes);
   s.total = o;
   return s;
@@ -195,6 +199,12 @@ struct FastParams {
   int32_t nst, slot_bytes, cache_bytes;  // cache_bytes > 0: every bound graph's lists (resolved, else state records + token arcs) fit in shared memory
   const unsigned char* tensor_lo;        // first / one-past-last byte of the logits tensor
   const unsigned char* tensor_hi;
+  // two-segment decode: per stream, what the second segment emits / adds to the score / its state at every frame start
+  int32_t npipes;                        // 2: long bound streams are decoded as two segments
+  int32_t scr_cap;                       // frames * S
+  int32_t* scr_tok;                      // [n_streams][2 * scr_cap]: tokens, then frames
+  float* scr_val;                        // [n_streams][scr_cap]: value of every row the segment visits, in order
+  int4* scr_trace;                       // [n_streams][frames + 1]: {state, tokens so far, values so far} at each frame start
 };
 
 // ---- helper: one row -> summary ----------------------------------------------------------------
@@ -270,12 +280,12 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
   const __nv_bfloat16 thr = __float2bfloat16_rd(thr_f);
   const __nv_bfloat162 thr2 = __halves2bfloat162(thr, thr);
 
-  // pass 2: one bit per element of this lane that reaches the threshold (bit 2i + h: word i, half h)
+  // pass 2: one bit per element of this lane that reaches the threshold (bit i + 16 h: word i, half h)
   uint32_t hits = 0;
 #pragma unroll
   for (int i = 0; i < 4 * NIT; ++i) {
     const uint32_t mk = __hge2_mask(as_bf162(w[i]), thr2);          // 0xFFFF per half that passes
-    if (4 * NIT <= 16) hits |= ((mk & 1u) | ((mk >> 15) & 2u)) << (2 * i);
+    if (4 * NIT <= 16) hits |= mk & (0x00010001u << i);
     else if (mk) hits |= 1u << (i & 31);                             // NIT = 8: one bit per word, both halves re-tested below
   }
   // exact root-boosted values of this lane's candidates: best (value, lowest id) and runner-up value
@@ -285,8 +295,8 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
     const int bit = __ffs(hits) - 1;
     hits &= hits - 1u;
     if (4 * NIT <= 16) {
-      const int i = bit >> 1;
-      const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 + (bit & 1) - p;
+      const int i = bit & 15;
+      const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 + (bit >> 4) - p;
       if (idx >= 0 && idx < V) {                            // masked elements pass only a threshold of -inf
         const ValId c{__fadd_rn(row_at(rowp, idx), h.rootcb[h.cls16[idx]]), idx};
         if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
@@ -423,7 +433,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
 #endif
   const TbDecodeParams& p = P.d;
   const int V = p.V, C = p.C, S = p.S, W = V + 1, nst = P.nst;
-  const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes);
+  const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes, P.npipes);
   unsigned char* ring = dyn + so.ring;
   uint64_t* full = reinterpret_cast<uint64_t*>(dyn + so.bars);
   uint64_t* freeb = full + nst;
@@ -432,7 +442,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   float* rootcb = reinterpret_cast<float*>(dyn + so.rootcb);
   float* rootcw = reinterpret_cast<float*>(dyn + so.rootcw);
   int32_t* rootdst = reinterpret_cast<int32_t*>(dyn + so.rootdst);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(dyn + so.misc);
+  volatile int* flags = reinterpret_cast<volatile int*>(dyn + so.misc);        // [2] stop flag per segment; [2] second segment's progress
+  int* seg_res = reinterpret_cast<int*>(dyn + so.misc + 32);                     // what the two deciders leave for the final merge
   float* root_stats = reinterpret_cast<float*>(dyn + so.misc + 16);   // beta_min, beta_max, R
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -451,14 +462,16 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   for (int v = tid; v < V; v += kThreadsF) {
     cls16[v] = static_cast<uint16_t>(p.cls[v]);
     reinterpret_cast<int16_t*>(dyn + so.tokidx)[v] = -1;
+    if (P.npipes == 2) reinterpret_cast<int16_t*>(dyn + so.tokidx + so.tokidx_sz)[v] = -1;
   }
   for (int c = tid; c < C; c += kThreadsF) {
     rootcb[c] = 0.0f; rootcw[c] = 0.0f; rootdst[c] = 0;
     reinterpret_cast<int16_t*>(dyn + so.cls_seen)[c] = -1;
+    if (P.npipes == 2) reinterpret_cast<int16_t*>(dyn + so.cls_seen + so.cls_seen_sz)[c] = -1;
   }
   for (int i = tid; i < nst * kSumStageBytes / 4; i += kThreadsF) reinterpret_cast<uint32_t*>(dyn + so.summ)[i] = 0u;   // no sequence word matches yet
   if (tid == 0) {
-    *abort_flag = 0;
+    flags[0] = 0; flags[1] = 0; flags[2] = 0;
     for (int i = 0; i < nst; ++i) { mbar_init(&full[i], 1); mbar_init(&freeb[i], S + 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -515,67 +528,94 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   const int lead0 = static_cast<int>(reinterpret_cast<uintptr_t>(base) & 15);
   const int lead_step = static_cast<int>(frame_stride_bytes & 15);
 
+  // ---- segments ------------------------------------------------------------------------------------------
+  // A long bound stream is decoded by two pipelines at once (each: producer, helpers, decider, a share of the
+  // ring).  Pipeline 0 starts at frame 0.  Pipeline 1 starts kSegWarm frames before frame f_mid in the root
+  // state and answers for the frames from f_mid on; from there it records, at every frame start, its graph
+  // state and how much it has emitted.  The decode from a given (frame start, graph state) is a function of
+  // those two alone, so once pipeline 0, which carries the true state, stands at a frame start >= f_mid in the
+  // state pipeline 1 recorded there, the rest of pipeline 1's output is the true continuation; until then
+  // pipeline 0 just keeps decoding.  The merge after the final barrier appends that continuation.
+  const bool seg = P.npipes == 2 && bound && end >= kSegMinFrames;
+  const int f_mid = seg ? (end + kSegWarm) / 2 : end;
+  // this warp's pipeline: warps 0 / 4 (decider, producer) and the first helpers belong to 0; warps 8 / 12 and the rest to 1
+  const int vw = warp;
+  const int hid_all = vw - 1 - (vw >> 2);                // helper index over the warps that are not multiples of 4
+  const int nh0 = seg ? (kHelpers + 1) / 2 : kHelpers;
+  const int pipe = !seg ? 0 : ((vw & 3) == 0 ? (vw >= 8 ? 1 : 0) : (hid_all >= nh0 ? 1 : 0));
+  const int nst0 = seg ? nst / 2 : nst;
+  const int pst_base = pipe ? nst0 : 0;                      // first ring stage of the pipeline
+  const int pnst = pipe ? nst - nst0 : nst0;
+  const int pf0 = pipe ? f_mid - kSegWarm : 0;               // first frame the pipeline fetches and decodes
+  unsigned char* pring = ring + static_cast<size_t>(pst_base) * P.slot_bytes;
+  uint64_t* pfull = full + pst_base;
+  uint64_t* pfree = freeb + pst_base;
+  const uint32_t psumm_a = summ_a + pst_base * kSumStageBytes;
+
   PROF_DECL();
-  if (warp == 4) {
+  if (vw == 4 || (seg && vw == 12)) {
     // ================================ producer ================================================
-    int issued = 0, st = 0, use = 0;
-    for (int f = 0; f < end; ++f) {
+    int issued = pf0, st = 0, use = 0;
+    for (int f = pf0; f < end; ++f) {
       PROF_T0();
-      if (use > 0 && !mbar_wait_parked(&freeb[st], (use - 1) & 1, abort_flag, p.status)) break;
+      if (flags[pipe]) break;
+      if (use > 0 && !mbar_wait_parked(&pfree[st], (use - 1) & 1, flags, pipe, p.status)) break;
       PROF_ADD(6);
       const unsigned char* src = base + static_cast<int64_t>(f) * frame_stride_bytes;
       const int lead = static_cast<int>(reinterpret_cast<uintptr_t>(src) & 15);
       const unsigned char* a0 = src - lead;
       const uint32_t bytes = static_cast<uint32_t>(up16(lead + frame_bytes));
-      unsigned char* dst = ring + static_cast<size_t>(st) * P.slot_bytes;
+      unsigned char* dst = pring + static_cast<size_t>(st) * P.slot_bytes;
       if (a0 >= P.tensor_lo && a0 + bytes <= P.tensor_hi) {
-        if (lane == 0) { mbar_arrive_expect_tx(&full[st], bytes); bulk_load(dst, a0, bytes, &full[st]); }
+        if (lane == 0) { mbar_arrive_expect_tx(&pfull[st], bytes); bulk_load(dst, a0, bytes, &pfull[st]); }
       } else {  // the aligned superset would leave the tensor: copy the frame's own elements
         const uint16_t* s16 = reinterpret_cast<const uint16_t*>(src);
         uint16_t* d16 = reinterpret_cast<uint16_t*>(dst + lead);
         for (int i = lane; i < S * W; i += 32) d16[i] = __ldg(s16 + i);
         __syncwarp();
-        if (lane == 0) mbar_arrive(&full[st]);
+        if (lane == 0) mbar_arrive(&pfull[st]);
       }
       issued = f + 1;
-      if (++st == nst) { st = 0; ++use; }
+      if (++st == pnst) { st = 0; ++use; }
       __syncwarp();
     }
     PROF_FLUSH();
     // no copy may be in flight when the block exits
-    for (int f = max(0, issued - nst); f < issued; ++f) {
-      const int fs = f % nst;
-      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&full[fs], (f / nst) & 1); ++it) {}
+    for (int f = max(pf0, issued - pnst); f < issued; ++f) {
+      const int fl = f - pf0, fs = fl % pnst;
+      for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(&pfull[fs], (fl / pnst) & 1); ++it) {}
     }
-  } else if ((warp & 3) != 0) {
+  } else if ((vw & 3) != 0) {
     // ================================ helpers =================================================
-    const int hid = warp - 1 - (warp >> 2);               // 0 .. kHelpers-1 over the warps that are not multiples of 4
+    const int ph0 = pipe ? nh0 : 0, pnh = seg ? (pipe ? kHelpers - nh0 : nh0) : kHelpers;
+    const int hid = hid_all - ph0;                        // 0 .. pnh-1 within the pipeline
     HelperCtx h;
     h.cls16 = cls16; h.rootcb = rootcb; h.rootcw = rootcw; h.rootdst = rootdst; h.V = V; h.nit = (V + 255) / 256;
     h.beta_min = root_stats[0]; h.beta_max = root_stats[1]; h.dbeta = __fsub_rn(root_stats[1], root_stats[0]);
     h.bmag_max = fabsf(lam) * ((bound ? rec.d_max : 0.0f) + root_stats[2]);
-    // rows are dealt round-robin: this warp takes rows hid, hid + kHelpers, ... of the stream, in order
-    int f = hid / S, k = hid - f * S;                     // frame and row in frame
-    int st = f % nst;
-    uint32_t ph = (f / nst) & 1;
+    // rows are dealt round-robin: this warp takes rows hid, hid + pnh, ... of the pipeline's frames, in order
+    int fl = hid / S, k = hid - fl * S;                   // frame (counted from the pipeline's first) and row in frame
+    int st = fl % pnst;
+    uint32_t ph = (fl / pnst) & 1;
+    int f = pf0 + fl;
     int lead = (lead0 + f * lead_step) & 15;
     for (; f < end;) {
       PROF_T0();
-      if (!mbar_wait_parked(&full[st], ph, abort_flag, p.status)) break;
+      if (!mbar_wait_parked(&pfull[st], ph, flags, pipe, p.status)) break;
       PROF_ADD(0);
-      const unsigned char* slot = ring + static_cast<size_t>(st) * P.slot_bytes;
-      summarize_row<NIT>(h, slot, lead + k * row_bytes, summ_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
-      if (lane == 0) mbar_arrive(&freeb[st]);
+      const unsigned char* slot = pring + static_cast<size_t>(st) * P.slot_bytes;
+      summarize_row<NIT>(h, slot, lead + k * row_bytes, psumm_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
+      if (lane == 0) mbar_arrive(&pfree[st]);
       PROF_ADD(1);
-      k += kHelpers;
+      k += pnh;
       while (k >= S) {                                      // on to a later frame
         k -= S; ++f;
         lead = (lead + lead_step) & 15;
-        if (++st == nst) { st = 0; ph ^= 1u; }
+        if (++st == pnst) { st = 0; ph ^= 1u; }
       }
     }
     PROF_FLUSH();
-  } else if (warp == 0) {
+  } else if (vw == 0 || (seg && vw == 8)) {
     // ================================ decider =================================================
     // Works in rounds over a window of eight frames.  The warp is eight groups of four lanes; group q
     // stands for frame t + q.  A round resolves rows in parallel under the current graph state and then
@@ -591,12 +631,14 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     //     through tokens too, as long as they leave the state unchanged.
     //   wide mode (many boosted tokens): all 32 lanes share them and resolve the current row only.
     const float R = root_stats[2];
-    const uint32_t ring_a = smem_u32(ring), freeb_a = smem_u32(freeb);
+    const uint32_t ring_a = smem_u32(pring), freeb_a = smem_u32(pfree);
+    const uint32_t summ_a = psumm_a;                        // (shadows the block-wide base: this pipeline's stages)
+    const int nst = pnst;
     const uint32_t cache_a = smem_u32(dyn + so.cache);
-    TbRsEnt* lbuf = reinterpret_cast<TbRsEnt*>(dyn + so.lbuf);
-    int16_t* cls_seen = reinterpret_cast<int16_t*>(dyn + so.cls_seen);
-    int16_t* tokidx = reinterpret_cast<int16_t*>(dyn + so.tokidx);
-    int2* emit_buf = reinterpret_cast<int2*>(dyn + so.emit);
+    TbRsEnt* lbuf = reinterpret_cast<TbRsEnt*>(dyn + so.lbuf + pipe * so.lbuf_sz);
+    int16_t* cls_seen = reinterpret_cast<int16_t*>(dyn + so.cls_seen + pipe * so.cls_seen_sz);
+    int16_t* tokidx = reinterpret_cast<int16_t*>(dyn + so.tokidx + pipe * so.tokidx_sz);
+    int2* emit_buf = reinterpret_cast<int2*>(dyn + so.emit + pipe * 256);
     const TbStateRec* strec = cached && !resolved ? reinterpret_cast<const TbStateRec*>(dyn + so.cache)
                                                   : reinterpret_cast<const TbStateRec*>(blob + rec.off_strec);
     const TbTokEnt* tokent = cached && !resolved ? reinterpret_cast<const TbTokEnt*>(dyn + so.cache + (rec.off_tokent - rec.off_strec))
@@ -610,10 +652,18 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
 
     const int q = lane >> 2, ql = lane & 3;                 // group and lane within the group
     constexpr int kWin = 8;                                 // frames per window (the launcher guarantees nst > kWin)
-    int t = 0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0, lead = lead0;
+    int t = pf0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0, lead = (lead0 + pf0 * lead_step) & 15;
     float score = 0.0f;
-    int32_t* out_tok = p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
-    int32_t* out_frm = p.out_frames + static_cast<int64_t>(b) * p.out_cap;
+    // pipeline 1 writes to scratch memory and keeps a log: rec_on
+    const bool rec_on = pipe == 1, chk_on = seg && pipe == 0;
+    const int out_cap = rec_on ? P.scr_cap : p.out_cap;
+    int32_t* out_tok = rec_on ? P.scr_tok + 2 * static_cast<int64_t>(b) * P.scr_cap : p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
+    int32_t* out_frm = rec_on ? out_tok + P.scr_cap : p.out_frames + static_cast<int64_t>(b) * p.out_cap;
+    float* vlog = rec_on ? P.scr_val + static_cast<int64_t>(b) * P.scr_cap : nullptr;
+    int4* trace = seg ? P.scr_trace + static_cast<int64_t>(b) * (p.frames + 1) : nullptr;
+    int nv = 0;                                             // values logged so far
+    int tc = -1;                                            // pipeline 0: the frame start at which it met pipeline 1's record
+    if (rec_on && pf0 >= f_mid && lane == 0) { trace[pf0] = make_int4(s, 0, 0, 0); __threadfence_block(); flags[2] = pf0 + 1; }
     const int max_rounds = p.frames * S + p.frames + 8;
     uint32_t spins = 0;
     bool failed = false, stable = false, no_allrows = false;
@@ -724,24 +774,34 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           if (!((ready_all >> li) & 1u)) break;
           progress = true;
           if ((blank_all >> li) & 1u) {
-            score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, li));
+            const float bv = __shfl_sync(0xffffffffu, xb, li);
+            score = __fadd_rn(score, bv);
             ++fq; pos = 0;
+            if (rec_on) {
+              if (lane == 0) { vlog[nv] = bv; if (t + fq >= f_mid) trace[t + fq] = make_int4(s, n_out, nv + 1, 0); }
+              ++nv;
+            }
             continue;
           }
           const int wt = __shfl_sync(0xffffffffu, wtok, li);
-          score = __fadd_rn(score, __shfl_sync(0xffffffffu, wv, li));
+          const float tv = __shfl_sync(0xffffffffu, wv, li);
+          score = __fadd_rn(score, tv);
           if (lane == 0) emit_buf[n_out & 31] = make_int2(wt, t + fq);
           if ((n_out & 31) == 31) {
             __syncwarp();
             const int2 e = emit_buf[lane];
             const int o = (n_out & ~31) + lane;
-            if (o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+            if (o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
             __syncwarp();
           }
           ++n_out;
           const bool keep = (keep_all >> li) & 1u;
           if (!keep) { tok = wt; tnext = __shfl_sync(0xffffffffu, wnext, li); }
           if (++pos == S) { ++fq; pos = 0; }
+          if (rec_on) {
+            if (lane == 0) { vlog[nv] = tv; if (pos == 0 && t + fq >= f_mid) trace[t + fq] = make_int4(keep ? s : tnext, n_out, nv + 1, 0); }
+            ++nv;
+          }
           if (!keep) break;
         }
         adv = fq; k = pos;
@@ -772,8 +832,10 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         adv = nb;
         progress = nb > 0;
         PROF_ADD(4);
+        bool took = false;                                  // the row after the blanks was consumed too
         if (!(wide && nb == 1) && nb < kWin && j_ready) {
           progress = true;
+          took = true;
           const int k_row = nb == 0 ? k : 0;                // symbols already emitted in that row's frame
           if (!j_rescan) {
             tok = j_tok; tval = j_val; tnext = j_next;
@@ -811,7 +873,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
               __syncwarp();
               const int2 e = emit_buf[lane];
               const int o = (n_out & ~31) + lane;
-              if (o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+              if (o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
               __syncwarp();
             }
             ++n_out;
@@ -819,13 +881,23 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             if (k == S) ++adv;                              // the frame closes by force
           }
         }
+        if (rec_on) {
+          // the values in visiting order, and the frame starts t + 1 .. t + adv this round reached
+          if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xb;
+          if (took && lane == 0) vlog[nv + nb] = tval;
+          if (lane < adv && t + lane + 1 >= f_mid) {
+            const bool viatok = lane >= nb && tok != V;     // reached because the token closed its frame
+            trace[t + lane + 1] = make_int4(viatok ? tnext : s, n_out - ((tok != V && !viatok) ? 1 : 0), nv + lane + 1, 0);
+          }
+          nv += nb + (took ? 1 : 0);
+        }
         if (adv > 0 && (tok == V || k == S)) k = 0;
         PROF_ADD(10);
       }
       PROF_COUNT(8);
       if (!progress) {                                      // the current row is not summarised yet: poll
-        if (++spins > kSpinLimit || ((spins & 255u) == 0u && *abort_flag)) {
-          if (spins > kSpinLimit) { *abort_flag = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
+        if (++spins > kSpinLimit || ((spins & 255u) == 0u && flags[pipe])) {
+          if (spins > kSpinLimit) { flags[0] = 1; flags[1] = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
           failed = true; break;
         }
         --it;                                               // a poll is not a round
@@ -864,6 +936,15 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           build_list(strec, tokent, rec.n_states, rec.max_depth, s, lam, R, V, lbuf, cls_seen, cls16, L, lane, p.status);
         }
       }
+      if (rec_on && adv > 0) {                              // publish how far the record reaches
+        __threadfence_block();
+        if (lane == 0) flags[2] = t + 1;
+      }
+      if (chk_on && k == 0 && t >= f_mid && t < end && t < flags[2]) {
+        // at a frame start pipeline 1 has recorded: the same graph state means the same decode from here on
+        const int rec_state = *reinterpret_cast<const volatile int*>(trace + t);
+        if (rec_state == s) { tc = t; break; }
+      }
       PROF_ADD(11);
     }
     PROF_FLUSH();
@@ -879,12 +960,54 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       __syncwarp();
       const int2 e = emit_buf[lane];
       const int o = (n_out & ~31) + lane;
-      if (lane < (n_out & 31) && o < p.out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+      if (lane < (n_out & 31) && o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
     }
-    if (failed || t < end) *abort_flag = 1;   // left early: let the other roles stop too
+    if (tc >= 0) flags[0] = 1;                // met the record: this pipeline's producer and helpers stop
+    else if (chk_on && !failed && t >= end) flags[1] = 1;   // decoded everything itself: pipeline 1 is not needed
+    else if (failed || t < end) { flags[0] = 1; flags[1] = 1; }   // left early: let the other roles stop too
     if (lane == 0) {
-      p.out_counts[b] = n_out; p.out_scores[b] = score; p.out_states[b] = s;
-      if (p.out_cursors) p.out_cursors[b] = t;
+      if (!seg) {
+        p.out_counts[b] = n_out; p.out_scores[b] = score; p.out_states[b] = s;
+        if (p.out_cursors) p.out_cursors[b] = t;
+      } else if (pipe == 0) {
+        seg_res[0] = n_out; seg_res[1] = __float_as_int(score); seg_res[2] = s; seg_res[3] = tc; seg_res[4] = t;
+      } else {
+        seg_res[8] = n_out; seg_res[9] = nv; seg_res[10] = s; seg_res[11] = t;
+      }
+    }
+  }
+  __syncthreads();
+  if (seg) {
+    // ---- merge: pipeline 0's output, then pipeline 1's from the frame start where the two met ----------------
+    const int nA = seg_res[0], tcm = seg_res[3];
+    int count = nA, s_fin = seg_res[2], t_fin = seg_res[4];
+    float score = __int_as_float(seg_res[1]);
+    if (tcm >= 0) {
+      const int nB = seg_res[8], nvB = seg_res[9];
+      const int4 tr = P.scr_trace[static_cast<int64_t>(b) * (p.frames + 1) + tcm];
+      const int n0 = tr.y, nv0 = tr.z;
+      const int32_t* scr_tok = P.scr_tok + 2 * static_cast<int64_t>(b) * P.scr_cap;
+      const int32_t* scr_frm = scr_tok + P.scr_cap;
+      int32_t* out_tok = p.out_tokens + static_cast<int64_t>(b) * p.out_cap;
+      int32_t* out_frm = p.out_frames + static_cast<int64_t>(b) * p.out_cap;
+      for (int j = n0 + tid; j < nB && j < P.scr_cap; j += kThreadsF) {
+        const int o = nA + j - n0;
+        if (o < p.out_cap) { out_tok[o] = scr_tok[j]; out_frm[o] = scr_frm[j]; }
+      }
+      if (warp == 0) {
+        // the score is the sum in visiting order: add pipeline 1's values one by one
+        const float* vlog = P.scr_val + static_cast<int64_t>(b) * P.scr_cap;
+        for (int i0 = nv0; i0 < nvB; i0 += 32) {
+          const float v = i0 + lane < nvB ? vlog[i0 + lane] : 0.0f;
+          const int m = min(32, nvB - i0);
+          for (int j = 0; j < m; ++j) score = __fadd_rn(score, __shfl_sync(0xffffffffu, v, j));
+        }
+      }
+      count = nA + nB - n0; s_fin = seg_res[10]; t_fin = seg_res[11];
+    }
+    if (tid == 0) {
+      p.out_counts[b] = count; p.out_scores[b] = score; p.out_states[b] = s_fin;
+      if (p.out_cursors) p.out_cursors[b] = t_fin;
     }
   }
   __syncthreads();
@@ -903,9 +1026,30 @@ extern "C" int tb_debug_prof_blk(unsigned long long* out, int n) {
 }
 #endif
 
+namespace {
+// scratch layout of the two-segment decode: tokens+frames, values, frame-start records
+struct ScratchLayout { size_t tok, val, trace, total; };
+ScratchLayout scratch_layout(int32_t n_streams, int32_t frames, int32_t S) {
+  ScratchLayout l;
+  const size_t cap = static_cast<size_t>(frames) * S, n = static_cast<size_t>(n_streams);
+  size_t o = 0;
+  l.tok = o; o += (n * 2 * cap * sizeof(int32_t) + 255) & ~static_cast<size_t>(255);
+  l.val = o; o += (n * cap * sizeof(float) + 255) & ~static_cast<size_t>(255);
+  l.trace = o; o += n * (static_cast<size_t>(frames) + 1) * sizeof(int4);
+  l.total = o;
+  return l;
+}
+}  // namespace
+
+size_t tb_greedy_fast_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S) {
+  if (n_streams <= 0 || frames < kSegMinFrames || S <= 0) return 0;
+  return scratch_layout(n_streams, frames, S).total;
+}
+
 // Returns TB_OK if the launch was made, 1 if this path does not cover the call (the caller then
 // uses the general kernel), or an error code.
-int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int32_t max_states, cudaStream_t stream) {
+int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int32_t max_states, void* scratch,
+                          size_t scratch_bytes, cudaStream_t stream) {
   const int W = d.V + 1;
   if (d.dtype != TB_BF16 || d.persistent || d.n_dur != 0) return 1;
   if (d.sv != 1 || d.ss != W || d.st < static_cast<int64_t>(d.S) * W || d.sb < 0) return 1;
@@ -927,13 +1071,32 @@ int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int3
   }
   const int budget = max_smem - 1024;
   P.cache_bytes = (max_cache_bytes > 0 && max_cache_bytes <= 48 * 1024) ? max_cache_bytes : 0;
-  const int fixed = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes).total;
   const int per_stage = P.slot_bytes + 16 + kSumStageBytes;
-  int nst = (budget - fixed - 64) / per_stage;
-  if (nst > kStagesMax) nst = kStagesMax;
+  // two segments per stream when the scratch memory is there and both halves of the ring can hold a window
+  P.npipes = 1; P.scr_cap = 0; P.scr_tok = nullptr; P.scr_val = nullptr; P.scr_trace = nullptr;
+  int nst = 0;
+  if (d.frames >= kSegMinFrames && scratch && (reinterpret_cast<uintptr_t>(scratch) & 15) == 0) {
+    const ScratchLayout l = scratch_layout(d.n_streams, d.frames, d.S);
+    const int fixed2 = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes, 2).total;
+    int nst2 = (budget - fixed2 - 64) / per_stage;
+    if (nst2 > kStagesMax) nst2 = kStagesMax;
+    if (l.total <= scratch_bytes && nst2 >= 18) {
+      P.npipes = 2; nst = nst2;
+      unsigned char* sb = static_cast<unsigned char*>(scratch);
+      P.scr_cap = d.frames * d.S;
+      P.scr_tok = reinterpret_cast<int32_t*>(sb + l.tok);
+      P.scr_val = reinterpret_cast<float*>(sb + l.val);
+      P.scr_trace = reinterpret_cast<int4*>(sb + l.trace);
+    }
+  }
+  if (P.npipes == 1) {
+    const int fixed = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes, 1).total;
+    nst = (budget - fixed - 64) / per_stage;
+    if (nst > kStagesMax) nst = kStagesMax;
+  }
   if (nst < 9) return 1;   // the decider's window spans eight stages
   P.nst = nst;
-  const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes);
+  const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes, P.npipes);
   if (so.total > budget) return 1;
   const int nit = (d.V + 255) / 256;
   void (*fn)(FastParams) = nit <= 1 ? k_greedy_fast<1> : nit <= 2 ? k_greedy_fast<2> : nit <= 4 ? k_greedy_fast<4> : k_greedy_fast<8>;
