@@ -307,3 +307,75 @@ def test_pipelined_kernel_random_configurations(tb, seed):
         ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
         check_greedy(fast, i, ref, f"seed{seed} pipelined V{V} S{S}")
         check_greedy(gen, i, ref, f"seed{seed} general V{V} S{S}")
+
+
+# ---------------------------------------------------------------------------------------------
+# streams long enough to be decoded as two segments that are merged at the end
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("V,S,T", [(1024, 3, 192), (1024, 3, 193), (300, 4, 260), (256, 1, 500), (700, 2, 333)])
+def test_two_segment_decode_shapes(tb, V, S, T):
+    """Lengths on both sides of the two-segment threshold in one batch, an unbound slot and an empty list."""
+    w = W.get_workload(2, B=8, T=T, S=S, V=V, n_phrases=60, n_plants=12)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[1] = None
+    lists[4] = []
+    lengths = [T, T, 191, 192, T, T - 1, 0, 200 if T >= 200 else T]
+    both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"two segments V{V}S{S}T{T}")
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_two_segment_decode_slow_to_meet(tb, seed):
+    """Heavy boosts over a small pool of tokens keep the decode inside phrases, so the segment that starts in the
+    root state takes long to fall in with the true one (or never does); coarse logits add exact ties."""
+    rng = np.random.default_rng(7000 + seed)
+    V, S = int(rng.choice([64, 257, 1024])), int(rng.integers(1, 4))
+    B, T = 5, int(rng.integers(192, 420))
+    cc = rng.integers(0, max(1, V // 2), size=V).astype(np.int32)
+    lam = float(rng.choice([1.0, 3.0, -2.0]))
+    x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32) * float(rng.choice([0.5, 1.0]))
+    x[..., V] += float(rng.choice([0.5, 2.0]))
+    if seed % 2 == 0:
+        x = np.round(x * 2) / 2
+    xb = W.f32_to_bf16_bits(x)
+    hot = rng.integers(0, V, size=6)
+    lists, weights = [], []
+    for b in range(B):
+        ph = [[int(t) for t in rng.choice(hot, size=rng.integers(2, 9))] for _ in range(int(rng.integers(5, 80)))]
+        lists.append(ph)
+        weights.append([[float(rng.choice([0.5, 1.0, 2.0, 4.0])) for _ in p] for p in ph])
+    batch = tb.tb_batch_create(V, cc, B, arena_bytes=16 << 20)
+    for i, p in enumerate(lists):
+        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc, token_weights=weights[i], lam=lam))
+    lens = np.array([T, T - 3, 192, T, 250 if T >= 250 else T], dtype=np.int32)
+    dl = torch.from_numpy(lens).to("cuda:0")
+    out = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=dl))
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
+    gen = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=dl))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(lists):
+        ref = O.greedy_rnnt(O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam), xb[i], int(lens[i]))
+        check_greedy(out, i, ref, f"seed {seed} pipelined")
+        check_greedy(gen, i, ref, f"seed {seed} general")
+        assert out["scores"][i] == gen["scores"][i]
+
+
+def test_two_segment_decode_repeats_and_rebinding(tb):
+    """The same batch decoded again after a slot changed its list, and twice in a row: the scratch memory of the
+    second segment carries nothing over."""
+    w = W.get_workload(2, B=6, T=300, n_phrases=50, n_plants=15)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"], arena_bytes=8 << 20)
+    logits = to_device(data["logits"])
+    first = to_host(tb.tb_greedy_decode(batch, logits))
+    again = to_host(tb.tb_greedy_decode(batch, logits))
+    for k in first:
+        assert np.array_equal(first[k], again[k]), k
+    other = W.stream_phrases(w, 17)
+    tb.tb_batch_bind_stream(batch, 2, tb.tb_graph_compile(other, w.V, case_class=w.vocab.case_class))
+    out = to_host(tb.tb_greedy_decode(batch, logits))
+    assert tb.tb_batch_status(batch) == 0
+    for i in range(w.B):
+        p = other if i == 2 else data["phrases"][i]
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, p), data["logits"][i]), "after rebinding")
