@@ -52,7 +52,10 @@ __device__ unsigned long long tb_prof_blk[4 * 1024];
 #define PROF_T0() _pt = clock64()
 #define PROF_ADD(slot) do { long long _n = clock64(); _pacc[slot] += _n - _pt; _pt = _n; } while (0)
 #define PROF_COUNT(slot) _pacc[slot] += 1
-#define PROF_FLUSH() do { if ((threadIdx.x & 31) == 0) { for (int _i = 0; _i < 16; ++_i) if (_pacc[_i]) atomicAdd(&tb_prof[_i], (unsigned long long)_pacc[_i]); } } while (0)
+#ifndef TB_PROF_PIPE
+#define TB_PROF_PIPE pipe
+#endif
+#define PROF_FLUSH() do { if ((threadIdx.x & 31) == 0 && pipe == TB_PROF_PIPE) { for (int _i = 0; _i < 16; ++_i) if (_pacc[_i]) atomicAdd(&tb_prof[_i], (unsigned long long)_pacc[_i]); } } while (0)
 #else
 #define PROF_DECL() do {} while (0)
 #define PROF_T0() do {} while (0)
@@ -735,9 +738,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       PROF_ADD(15);
       int wtok = static_cast<int>((wdt & kTokMask) >> 1);
       int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
-#ifdef TB_PROFILE
-      int cause = rescan ? 1 : 0;
-#endif
       {
         // the best plain token: exact when the summary's winner is plain and clears the others by the
         // rounding margin (at the root it is exact by construction); else bounded from above
@@ -751,9 +751,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
           if (!(fmaxf(wv, xb) > ub + tau)) {
             rescan = true;
-#ifdef TB_PROFILE
-            cause |= in_deep ? 2 : 4;
-#endif
           }
         }
       }
@@ -842,9 +839,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           } else {
             // exact evaluation of that row by the whole warp from shared memory
             PROF_COUNT(9);
-#ifdef TB_PROFILE
-            { const int cz = __shfl_sync(0xffffffffu, cause, jl); if (cz & 1) _pacc[12] += 1; if (cz & 2) _pacc[13] += 1; if (cz & 4) _pacc[14] += 1; }
-#endif
             const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
             for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = static_cast<int16_t>(i); }
             __syncwarp();
@@ -896,6 +890,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       }
       PROF_COUNT(8);
       if (!progress) {                                      // the current row is not summarised yet: poll
+        PROF_COUNT(12);
         if (++spins > kSpinLimit || ((spins & 255u) == 0u && flags[pipe])) {
           if (spins > kSpinLimit) { flags[0] = 1; flags[1] = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
           failed = true; break;
