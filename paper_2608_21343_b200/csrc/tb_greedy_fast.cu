@@ -765,42 +765,55 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const unsigned ready_all = __ballot_sync(0xffffffffu, ready && !rescan);
         const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
         PROF_ADD(7);
-        int fq = 0, pos = k;
-        for (int guard = 0; guard < 4 * kWin && fq < kWin; ++guard) {
-          const int li = 4 * fq + pos;
-          if (!((ready_all >> li) & 1u)) break;
-          progress = true;
-          if ((blank_all >> li) & 1u) {
-            const float bv = __shfl_sync(0xffffffffu, xb, li);
-            score = __fadd_rn(score, bv);
-            ++fq; pos = 0;
-            if (rec_on) {
-              if (lane == 0) { vlog[nv] = bv; if (t + fq >= f_mid) trace[t + fq] = make_int4(s, n_out, nv + 1, 0); }
-              ++nv;
-            }
-            continue;
-          }
-          const int wt = __shfl_sync(0xffffffffu, wtok, li);
-          const float tv = __shfl_sync(0xffffffffu, wv, li);
-          score = __fadd_rn(score, tv);
-          if (lane == 0) emit_buf[n_out & 31] = make_int2(wt, t + fq);
-          if ((n_out & 31) == 31) {
+        // Which rows the decode visits follows from the blank / token pattern alone while the state stays what
+        // it is: in a frame, row j is visited when rows 0 .. j-1 selected tokens.  All of it is bit arithmetic
+        // on the ballots (bit 4 q + j: row j of frame t + q); only the score is added up row by row.
+        const unsigned m1 = 0x11111111u;
+        const unsigned smask = S >= 4 ? 0xFFFFFFFFu : (m1 << S) - m1;          // rows j < S of every frame
+        const unsigned pre = (1u << k) - 1u;                                   // rows of frame t behind the cursor
+        const unsigned tok_all = ready_all & ~blank_all;
+        const unsigned tokx = tok_all | pre;
+        const unsigned a0 = tokx & m1, a1 = (tokx >> 1) & m1, a2 = (tokx >> 2) & m1;
+        const unsigned vis = (m1 | (a0 << 1) | ((a0 & a1) << 2) | ((a0 & a1 & a2) << 3)) & smask & ~pre;
+        // the walk ends before a row that is not ready (or needs the rescan) and after a token that changes the state
+        const unsigned bad = vis & (~ready_all | (tok_all & ~keep_all));
+        const int pb = bad ? __ffs(bad) - 1 : 32;
+        const bool last_tok = pb < 32 && ((tok_all >> pb) & 1u);                // that token is consumed too
+        const unsigned cm = (vis & (pb < 32 ? (1u << pb) - 1u : 0xFFFFFFFFu)) | (last_tok ? 1u << pb : 0u);
+        const unsigned tm = cm & tok_all, bm = cm & blank_all;
+        progress = cm != 0u;
+        if (last_tok) { tok = __shfl_sync(0xffffffffu, wtok, pb); tnext = __shfl_sync(0xffffffffu, wnext, pb); }
+        // frames closed: by a blank, or by a token in the frame's last row
+        const unsigned cl = bm | (tm & (m1 << (S - 1)));
+        const unsigned clf = (cl | (cl >> 1) | (cl >> 2) | (cl >> 3)) & m1;
+        const int fq = __popc(clf);
+        const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * fq)) & 0xFu) : 0;
+        const unsigned upto = 0xFFFFFFFFu >> (31 - lane);                       // bits 0 .. lane
+        const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
+        const float val = mine_t ? wv : xb;
+        if (rec_on) {
+          if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
+          if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
+            trace[t + q + 1] = make_int4((last_tok && lane == pb) ? tnext : s, n_out + __popc(tm & upto), nv + __popc(cm & upto), 0);
+          nv += __popc(cm);
+        }
+        // emitted tokens, in order, through the staging buffer (at most one block boundary is crossed)
+        const int nt = __popc(tm);
+        if (nt > 0) {
+          const int room = 32 - (n_out & 31);
+          const int rank = __popc(tm & upto) - 1;
+          if (mine_t && rank < room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
+          if (nt >= room) {
             __syncwarp();
             const int2 e = emit_buf[lane];
             const int o = (n_out & ~31) + lane;
             if (o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
             __syncwarp();
+            if (mine_t && rank >= room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
           }
-          ++n_out;
-          const bool keep = (keep_all >> li) & 1u;
-          if (!keep) { tok = wt; tnext = __shfl_sync(0xffffffffu, wnext, li); }
-          if (++pos == S) { ++fq; pos = 0; }
-          if (rec_on) {
-            if (lane == 0) { vlog[nv] = tv; if (pos == 0 && t + fq >= f_mid) trace[t + fq] = make_int4(keep ? s : tnext, n_out, nv + 1, 0); }
-            ++nv;
-          }
-          if (!keep) break;
+          n_out += nt;
         }
+        for (unsigned m = cm; m; m &= m - 1u) score = __fadd_rn(score, __shfl_sync(0xffffffffu, val, __ffs(m) - 1));
         adv = fq; k = pos;
         if (!progress) {
           // the current row is not summarised yet (poll), or it needs the exact rescan (next round, shared mode)
