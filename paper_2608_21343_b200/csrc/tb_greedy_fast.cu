@@ -42,8 +42,8 @@ constexpr int kGroupDeep = 64;  // up to this many boosted tokens, the decider r
 constexpr int kAllRowsDeep = 64; // all-rows mode in a state that just repeated itself: at most this many boosted tokens
 constexpr int kStagesMax = 24;  // ring stages; each decider lane below this number owns one stage
 constexpr uint32_t kSpinLimit = 1u << 20;
-constexpr int kSegMinFrames = 192;  // streams at least this long are decoded as two segments (see the header)
-constexpr int kSegWarm = 32;        // frames the second segment decodes before the first frame it answers for
+constexpr int kSegMinFrames = 128;  // streams at least this long are decoded as two segments (see the header)
+constexpr int kSegWarm = 16;        // frames the second segment decodes before the first frame it answers for
 
 #ifdef TB_PROFILE
 __device__ unsigned long long tb_prof[16];

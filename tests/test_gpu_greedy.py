@@ -313,7 +313,7 @@ def test_pipelined_kernel_random_configurations(tb, seed):
 # streams long enough to be decoded as two segments that are merged at the end
 # ---------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("V,S,T", [(1024, 3, 192), (1024, 3, 193), (300, 4, 260), (256, 1, 500), (700, 2, 333)])
+@pytest.mark.parametrize("V,S,T", [(1024, 3, 128), (1024, 3, 129), (1024, 3, 193), (300, 4, 260), (256, 1, 500), (700, 2, 333)])
 def test_two_segment_decode_shapes(tb, V, S, T):
     """Lengths on both sides of the two-segment threshold in one batch, an unbound slot and an empty list."""
     w = W.get_workload(2, B=8, T=T, S=S, V=V, n_phrases=60, n_plants=12)
@@ -321,7 +321,7 @@ def test_two_segment_decode_shapes(tb, V, S, T):
     lists = list(data["phrases"])
     lists[1] = None
     lists[4] = []
-    lengths = [T, T, 191, 192, T, T - 1, 0, 200 if T >= 200 else T]
+    lengths = [T, T, 127, 128, T, T - 1, 0, 200 if T >= 200 else T]
     both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"two segments V{V}S{S}T{T}")
 
 
@@ -331,7 +331,7 @@ def test_two_segment_decode_slow_to_meet(tb, seed):
     root state takes long to fall in with the true one (or never does); coarse logits add exact ties."""
     rng = np.random.default_rng(7000 + seed)
     V, S = int(rng.choice([64, 257, 1024])), int(rng.integers(1, 4))
-    B, T = 5, int(rng.integers(192, 420))
+    B, T = 5, int(rng.integers(128, 420))
     cc = rng.integers(0, max(1, V // 2), size=V).astype(np.int32)
     lam = float(rng.choice([1.0, 3.0, -2.0]))
     x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32) * float(rng.choice([0.5, 1.0]))
@@ -348,7 +348,7 @@ def test_two_segment_decode_slow_to_meet(tb, seed):
     batch = tb.tb_batch_create(V, cc, B, arena_bytes=16 << 20)
     for i, p in enumerate(lists):
         tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc, token_weights=weights[i], lam=lam))
-    lens = np.array([T, T - 3, 192, T, 250 if T >= 250 else T], dtype=np.int32)
+    lens = np.array([T, T - 3, 128, T, 250 if T >= 250 else T], dtype=np.int32)
     dl = torch.from_numpy(lens).to("cuda:0")
     out = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=dl))
     tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
