@@ -233,21 +233,33 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
 #pragma unroll
   for (int j = 0; j < NIT; ++j) {
     if (j < h.nit) {
-      const int b = j * 32 + lane;
-      uint4 q = blk[b];
-      const int idx0 = b * 8 - p;                         // token id of the block's first element
-      if (idx0 < 0 || idx0 + 8 > V) {                     // head / tail block: mask what is not a token of this row
-        uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int i0 = idx0 + 2 * e;
-          if (i0 < 0 || i0 >= V) qq[e] = (qq[e] & 0xFFFF0000u) | 0xFF80u;
-          if (i0 + 1 < 0 || i0 + 1 >= V) qq[e] = (qq[e] & 0x0000FFFFu) | 0xFF800000u;
-        }
-      }
+      const uint4 q = blk[j * 32 + lane];
       w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
     } else {
       w[4 * j] = w[4 * j + 1] = w[4 * j + 2] = w[4 * j + 3] = NEG2;
+    }
+  }
+  // What the 16-byte blocks hold beyond this row's tokens is masked to -inf: the p elements before the row in
+  // the first block (lane 0 only), and everything from element V on when the passes reach that far.
+  if (p > 0 && lane == 0) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (2 * e < p) w[e] = (w[e] & 0xFFFF0000u) | 0xFF80u;
+      if (2 * e + 1 < p) w[e] = (w[e] & 0x0000FFFFu) | 0xFF800000u;
+    }
+  }
+  if (V + p < h.nit * 256) {
+#pragma unroll
+    for (int j = 0; j < NIT; ++j) {
+      const int idx0 = (j * 32 + lane) * 8 - p;             // token id of the block's first element
+      if (j < h.nit && idx0 + 8 > V) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int i0 = idx0 + 2 * e;
+          if (i0 >= V) w[4 * j + e] = (w[4 * j + e] & 0xFFFF0000u) | 0xFF80u;
+          if (i0 + 1 >= V) w[4 * j + e] = (w[4 * j + e] & 0x0000FFFFu) | 0xFF800000u;
+        }
+      }
     }
   }
   // tokens after the last full pass (at most 7): one element per lane
