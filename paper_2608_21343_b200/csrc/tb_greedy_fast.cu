@@ -172,7 +172,7 @@ __device__ __forceinline__ void mbar_arrive_relaxed_addr(uint32_t bar_addr) {
 }
 
 struct Smem {  // byte offsets into dynamic shared memory, computed identically on host and device
-  int ring, bars, summ, cls16, rootcb, rootcw, rootdst, lbuf, cls_seen, tokidx, emit, misc, cache, total;
+  int ring, bars, summ, cls16, tokcb, rootcw, rootdst, lbuf, cls_seen, tokidx, emit, misc, cache, total;
   int lbuf_sz, cls_seen_sz, tokidx_sz;   // the deciders' private areas exist once per segment, this far apart
 };
 __host__ __device__ inline int up16(int x) { return (x + 15) & ~15; }
@@ -183,7 +183,7 @@ __host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int
   s.bars = o; o += up16(8 * (2 * nst));
   s.summ = o; o += nst * kSumStageBytes;
   s.cls16 = o; o += up16(2 * V);
-  s.rootcb = o; o += up16(4 * C);
+  s.tokcb = o; o += up16(4 * V);            // lambda * root-arc weight of every token (0 without a root arc)
   s.rootcw = o; o += up16(4 * C);
   s.rootdst = o; o += up16(4 * C);
   s.lbuf_sz = up16(8 * (V + 4)); s.cls_seen_sz = up16(2 * C); s.tokidx_sz = up16(2 * V);
@@ -213,7 +213,7 @@ struct FastParams {
 // ---- helper: one row -> summary ----------------------------------------------------------------
 struct HelperCtx {
   const uint16_t* cls16;
-  const float* rootcb;
+  const float* tokcb;
   const float* rootcw;
   const int32_t* rootdst;
   float beta_min, beta_max, dbeta;
@@ -313,7 +313,7 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
       const int i = bit & 15;
       const int idx = ((i >> 2) * 32 + lane) * 8 + (i & 3) * 2 + (bit >> 4) - p;
       if (idx >= 0 && idx < V) {                            // masked elements pass only a threshold of -inf
-        const ValId c{__fadd_rn(row_at(rowp, idx), h.rootcb[h.cls16[idx]]), idx};
+        const ValId c{__fadd_rn(row_at(rowp, idx), h.tokcb[idx]), idx};
         if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
       }
     } else {
@@ -325,7 +325,7 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
         if (idx >= 0 && idx < V) {
           const float x = row_at(rowp, idx);
           if (x >= __bfloat162float(thr)) {
-            const ValId c{__fadd_rn(x, h.rootcb[h.cls16[idx]]), idx};
+            const ValId c{__fadd_rn(x, h.tokcb[idx]), idx};
             if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
           }
         }
@@ -333,7 +333,7 @@ __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned
     }
   }
   if (tail_ok && __hge(__ushort_as_bfloat16(static_cast<unsigned short>(tail_bits)), thr)) {
-    const ValId c{__fadd_rn(bf16_bits_to_float(tail_bits), h.rootcb[h.cls16[tail_idx]]), tail_idx};
+    const ValId c{__fadd_rn(bf16_bits_to_float(tail_bits), h.tokcb[tail_idx]), tail_idx};
     if (better(c, b)) { sec = fmaxf(sec, b.v); b = c; } else { sec = fmaxf(sec, c.v); }
   }
   // across the warp: best (value, lowest id) and the runner-up value
@@ -454,7 +454,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   uint64_t* freeb = full + nst;
   const uint32_t summ_a = smem_u32(dyn + so.summ);
   uint16_t* cls16 = reinterpret_cast<uint16_t*>(dyn + so.cls16);
-  float* rootcb = reinterpret_cast<float*>(dyn + so.rootcb);
+  float* tokcb = reinterpret_cast<float*>(dyn + so.tokcb);
+  float* rootcb = reinterpret_cast<float*>(dyn + so.ring + 256);   // per class, only while the tables are set up (the ring is not in use yet)
   float* rootcw = reinterpret_cast<float*>(dyn + so.rootcw);
   int32_t* rootdst = reinterpret_cast<int32_t*>(dyn + so.rootdst);
   volatile int* flags = reinterpret_cast<volatile int*>(dyn + so.misc);        // [2] stop flag per segment; [2] second segment's progress
@@ -507,6 +508,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     }
   }
   __syncthreads();
+  for (int v = tid; v < V; v += kThreadsF) tokcb[v] = rootcb[cls16[v]];
   {
     // extremes of the root arcs' lambda * w (tokens without a root arc have beta = 0) and of |w|
     float bmin = 0.0f, bmax = 0.0f, R = 0.0f;
@@ -605,7 +607,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     const int ph0 = pipe ? nh0 : 0, pnh = seg ? (pipe ? kHelpers - nh0 : nh0) : kHelpers;
     const int hid = hid_all - ph0;                        // 0 .. pnh-1 within the pipeline
     HelperCtx h;
-    h.cls16 = cls16; h.rootcb = rootcb; h.rootcw = rootcw; h.rootdst = rootdst; h.V = V; h.nit = (V + 255) / 256;
+    h.cls16 = cls16; h.tokcb = tokcb; h.rootcw = rootcw; h.rootdst = rootdst; h.V = V; h.nit = (V + 255) / 256;
     h.beta_min = root_stats[0]; h.beta_max = root_stats[1]; h.dbeta = __fsub_rn(root_stats[1], root_stats[0]);
     h.bmag_max = fabsf(lam) * ((bound ? rec.d_max : 0.0f) + root_stats[2]);
     // rows are dealt round-robin: this warp takes rows hid, hid + pnh, ... of the pipeline's frames, in order
