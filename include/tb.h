@@ -180,8 +180,14 @@ int tb_batch_status(tb_batch *b, int32_t *device_status, void *stream);
  *   out_counts   device int32 [B]: tokens emitted
  *   out_scores   device float [B]
  *   out_states   device int32 [B]: final graph state (-1 for unbound slots)
- * Does not read or change the slots' streaming state.  Errors: TB_ERR_INVALID_ARG
- * (B > n_slots, bad dtype, NULL pointers, non-positive sizes), TB_ERR_CUDA.
+ * Does not read or change the slots' streaming state.  Working memory: the pipelined kernel
+ * decodes long bound streams as two segments at once and merges them (the result is that of the
+ * sequential decode, bit for bit); what the second segment produces passes through a device
+ * block owned by the batch, which this call allocates or grows (freeing the old block, which
+ * waits for the device) when B*T*S exceeds what an earlier call needed.  Hence one
+ * tb_greedy_decode per batch at a time; if the block cannot be had, streams are decoded whole.
+ * Errors: TB_ERR_INVALID_ARG (B > n_slots, bad dtype, NULL pointers, non-positive sizes),
+ * TB_ERR_CUDA.
  */
 int tb_greedy_decode(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t T, int32_t S,
                      const int64_t *strides, const int32_t *lengths, int32_t *out_tokens,

@@ -9,8 +9,8 @@
 //   decider warp  : the only sequential part -- walks the rows the decode visits, resolves each
 //                   from its summary plus the few tokens boosted by the current non-root graph
 //                   state, advances the graph state and the frame cursor, writes the outputs.
-// The decider shares its warp scheduler with no helper: warps are spread over the SM's four
-// schedulers by warp index, and every fourth warp other than the decider and the producer just
+// The deciders share their warp scheduler with no helper: warps are spread over the SM's four
+// schedulers by warp index, and every fourth warp that is neither a decider nor a producer just
 // waits at the final barrier.
 //
 // Exactness.  Values follow the arithmetic contract (val = fl(x + fl(lambda * bonus)), ties to
@@ -23,6 +23,9 @@
 // than a margin tau that dominates every rounding error involved, or shows that no plain token
 // can reach the best of {blank, the state's own tokens}; the tokens the chain boosts are always
 // evaluated exactly; otherwise the whole row is rescanned exactly from shared memory.
+//
+// Long bound streams are decoded as two segments at once, each by a pipeline of its own (producer,
+// helpers, decider, half of the ring), and merged at the end: see "segments" in the kernel.
 //
 // Every wait is bounded; a wait that runs out raises TB_STATUS_WAIT_TIMEOUT, makes all roles of
 // the block leave their loops, and the block still waits (bounded) for its copies in flight.
