@@ -156,7 +156,7 @@ class Graph:
 
     def __del__(self):
         h = getattr(self, "handle", None)
-        if h:
+        if h and lib is not None:          # at interpreter shutdown module globals may already be gone
             lib().orc_graph_free(h)
             self.handle = None
 
