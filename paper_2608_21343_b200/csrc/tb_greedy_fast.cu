@@ -556,8 +556,12 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   // those two alone, so once pipeline 0, which carries the true state, stands at a frame start >= f_mid in the
   // state pipeline 1 recorded there, the rest of pipeline 1's output is the true continuation; until then
   // pipeline 0 just keeps decoding.  The merge after the final barrier appends that continuation.
-  const bool seg = P.npipes == 2 && bound && end >= kSegMinFrames;
-  const int f_mid = seg ? (end + kSegWarm) / 2 : end;
+  // (an unbound stream has no graph state: its second pipeline starts exactly in the true state, with no
+  // warm-up, and the two meet at f_mid; it is split as well because one pipeline's ring turns over too slowly
+  // to keep the copies flowing)
+  const bool seg = P.npipes == 2 && end >= kSegMinFrames;
+  const int warm = bound ? kSegWarm : 0;
+  const int f_mid = seg ? (end + warm) / 2 : end;
   // this warp's pipeline: warps 0 / 4 (decider, producer) and the first helpers belong to 0; warps 8 / 12 and the rest to 1
   const int vw = warp;
   const int hid_all = vw - 1 - (vw >> 2);                // helper index over the warps that are not multiples of 4
@@ -566,7 +570,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   const int nst0 = seg ? nst / 2 : nst;
   const int pst_base = pipe ? nst0 : 0;                      // first ring stage of the pipeline
   const int pnst = pipe ? nst - nst0 : nst0;
-  const int pf0 = pipe ? f_mid - kSegWarm : 0;               // first frame the pipeline fetches and decodes
+  const int pf0 = pipe ? f_mid - warm : 0;                   // first frame the pipeline fetches and decodes
   unsigned char* pring = ring + static_cast<size_t>(pst_base) * P.slot_bytes;
   uint64_t* pfull = full + pst_base;
   uint64_t* pfree = freeb + pst_base;
