@@ -226,6 +226,19 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned char* blob = p.arena + rec.blob_off;
   const bool use_tv = bound && rec.n_rsent >= 0 && p.tokview;
+  // rows shared by the hypotheses of a stream (hyp_stride 0) depend on nothing that is loaded below: fetch this
+  // thread's elements now, so that their latency overlaps the loads of the slot record, states and lists
+  constexpr int kPref = 5;
+  const bool pref = use_tv && p.hyp_stride == 0 && W <= kPref * kThreads;
+  float xpre[kPref];
+  if (pref) {
+    const LT* row0 = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+#pragma unroll
+    for (int j = 0; j < kPref; ++j) {
+      const int v = threadIdx.x + j * kThreads;
+      xpre[j] = v < W ? LogitLoad<LT>::at(row0 + v) : 0.0f;
+    }
+  }
   TokView tv;
   if (use_tv) tokview_init(tv, aux, V, p.C, g);
 
@@ -251,11 +264,14 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     }
     __syncthreads();
     const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
-    for (int v = threadIdx.x; v < W; v += kThreads) {
+#pragma unroll
+    for (int j = 0; j < (W + kThreads - 1) / kThreads && (!pref || j < kPref); ++j) {
+      const int v = threadIdx.x + j * kThreads;
+      if (v >= W) break;
       const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
       for (int k = 0; k < K; ++k) {
         if (h_score[k] == -INFINITY || !h_live[k]) continue;
-        const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
+        const float x = pref ? xpre[j < kPref ? j : 0] : LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
         const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
         cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
       }
