@@ -379,3 +379,44 @@ def test_two_segment_decode_repeats_and_rebinding(tb):
     for i in range(w.B):
         p = other if i == 2 else data["phrases"][i]
         check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, p), data["logits"][i]), "after rebinding")
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_pipelined_kernel_soak_against_oracle(tb, block):
+    """Ten random configurations per case, lengths on both sides of the two-segment threshold, any alignment:
+    tokens, frames, states and the float32 score bit for bit as the oracle's."""
+    for seed in range(10 * block, 10 * block + 10):
+        rng = np.random.default_rng(50000 + seed)
+        V = int(rng.choice([9, 64, 255, 256, 257, 511, 1023, 1024, 1500, 2046]))
+        S = int(rng.integers(1, 5))
+        B = int(rng.integers(1, 6))
+        T = int(rng.choice([rng.integers(1, 128), rng.integers(128, 300), rng.integers(300, 700)]))
+        cc = rng.integers(0, int(rng.integers(1, V + 1)), size=V).astype(np.int32)
+        lam = float(rng.choice([1.0, 0.5, 2.0, 3.0, -0.5]))
+        x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32) * float(rng.choice([0.3, 1.0, 3.0]))
+        x[..., V] += float(rng.choice([0.0, 1.0, 3.0]))
+        if seed % 3 == 0:
+            x = np.round(x * 2) / 2
+        xb = W.f32_to_bf16_bits(x)
+        hot = rng.integers(0, V, size=max(2, int(rng.choice([4, V // 20 + 2, V // 4 + 2]))))
+        lists, weights = [], []
+        for b in range(B):
+            ph = [[int(t) for t in rng.choice(hot, size=rng.integers(1, 7))] for _ in range(int(rng.integers(0, 120)))]
+            lists.append(None if (b == 1 and B > 1 and seed % 2) else ph)
+            weights.append([[float(rng.choice([0.5, 1.0, 1.5, 2.0])) for _ in p] for p in ph])
+        batch = tb.tb_batch_create(V, cc, B, arena_bytes=32 << 20)
+        for i, p in enumerate(lists):
+            if p is not None:
+                tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc, token_weights=weights[i], lam=lam))
+        shift = int(rng.integers(0, 9))
+        flat = torch.zeros(shift + xb.size + 8, dtype=torch.bfloat16, device="cuda:0")
+        view = flat[shift:shift + xb.size].view(B, T, S, V + 1)
+        view.copy_(to_device(xb))
+        lens = rng.integers(max(0, T - 40), T + 1, size=B).astype(np.int32)
+        out = to_host(tb.tb_greedy_decode(batch, view, lengths=torch.from_numpy(lens).to("cuda:0")))
+        assert tb.tb_batch_status(batch) == 0
+        for i, p in enumerate(lists):
+            g = None if p is None else O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam)
+            ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
+            check_greedy(out, i, ref, f"seed {seed}")
+            assert float(out["scores"][i]) == float(ref["score"]), f"seed {seed} stream {i}: score bits"
