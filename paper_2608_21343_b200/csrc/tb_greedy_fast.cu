@@ -424,6 +424,8 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
   L.bmag = fabsf(lam) * (fabsf(acc) + R);
 }
 
+__device__ __forceinline__ void prog_publish(volatile int* flags, int v) { flags[2] = v; }
+
 struct Pick {
   ValId win;
   int next;
@@ -691,12 +693,134 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     const int max_rounds = p.frames * S + p.frames + 8;
     uint32_t spins = 0;
     bool failed = false, stable = false, no_allrows = false;
+    const bool fast_ok = bound && cached && resolved;       // the branch-free round reads lists from the cache only
     for (int it = 0; t < end; ++it) {
       if (it >= max_rounds) { if (lane == 0) atomicOr(p.status, TB_STATUS_STEP_LIMIT); break; }
       PROF_T0();
       // ---- mode and this lane's row --------------------------------------------------------------------
       const bool allrows = !no_allrows && (L.n == 0 || (stable && L.n <= kAllRowsDeep));
       const bool wide = !allrows && L.n > kGroupDeep;
+      // ---- the usual round, without branches -----------------------------------------------------------
+      // A lone warp pays tens of cycles for every branch whose condition was only just computed (nothing
+      // else can issue while it resolves).  The usual round -- shared mode, lists in the cache -- is therefore
+      // computed here as straight-line code with selects; everything unusual (a row that needs the rescan,
+      // nothing ready, a full staging block, a long blank run, a state out of range) is collected in one
+      // flag, and then the round falls through, having changed nothing, to the general code below.
+      if (fast_ok && !allrows && !wide && !(chk_on && t >= f_mid)) {
+        const int rk = q == 0 ? k : 0;
+        int stq = st + q; stq -= stq >= nst ? nst : 0;
+        const uint32_t sum_a = summ_a + stq * kSumStageBytes + rk * 32u;
+        const uint4 q1 = lds_v4_volatile(sum_a + 16u);
+        const uint4 q0 = lds_v4_volatile(sum_a);
+        const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + q * lead_step) & 15) + rk * row_bytes;
+        const bool ready = t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u;
+        const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+        const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
+        float wv = -INFINITY;
+        uint32_t wdt = 2u * static_cast<uint32_t>(V);
+        bool in_deep = false;
+        {
+          int i = ql;
+          for (; i + 4 < L.n; i += 8) {                      // two entries in flight
+            const uint2 e0 = lds_v2(L.addr + 8u * i), e1 = lds_v2(L.addr + 8u * (i + 4));
+            const uint32_t x0 = lds_u16(row_a + (e0.x & kTokMask)), x1r = lds_u16(row_a + (e1.x & kTokMask));
+            const float v0 = __fadd_rn(bf16_bits_to_float(x0), __uint_as_float(e0.y));
+            const float v1 = __fadd_rn(bf16_bits_to_float(x1r), __uint_as_float(e1.y));
+            in_deep |= (e0.x & kTokMask) == id1x2 || (e1.x & kTokMask) == id1x2;
+            const bool b0 = v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask));
+            wv = b0 ? v0 : wv; wdt = b0 ? e0.x : wdt;
+            const bool b1 = v1 > wv || (v1 == wv && (e1.x & kTokMask) < (wdt & kTokMask));
+            wv = b1 ? v1 : wv; wdt = b1 ? e1.x : wdt;
+          }
+          if (i < L.n) {
+            const uint2 e0 = lds_v2(L.addr + 8u * i);
+            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16(row_a + (e0.x & kTokMask))), __uint_as_float(e0.y));
+            in_deep |= (e0.x & kTokMask) == id1x2;
+            const bool b0 = v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask));
+            wv = b0 ? v0 : wv; wdt = b0 ? e0.x : wdt;
+          }
+        }
+#pragma unroll
+        for (int off = 1; off <= 2; off <<= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, wv, off);
+          const uint32_t od = __shfl_xor_sync(0xffffffffu, wdt, off);
+          const bool oi = __shfl_xor_sync(0xffffffffu, in_deep, off);
+          const bool bo = ov > wv || (ov == wv && (od & kTokMask) < (wdt & kTokMask));
+          wv = bo ? ov : wv; wdt = bo ? od : wdt;
+          in_deep |= oi;
+        }
+        int wtok = static_cast<int>((wdt & kTokMask) >> 1);
+        int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
+        // the best plain token (see the general code): exact when it clears the others by the margin, else bounded
+        const bool plain_ok = !in_deep && ((q1.z & kSumGap) != 0 || s <= 0);
+        const float nd = __fadd_rn(x1, __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
+        const int id1 = static_cast<int>(id1x2 >> 1);
+        const float ub = (in_deep ? y2b : y1) + lam * L.D;
+        const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
+        const bool rescan = (q1.z & kSumOvf) != 0 || (!plain_ok && !(fmaxf(wv, xb) > ub + tau));
+        const bool take_plain = plain_ok && (nd > wv || (nd == wv && id1 < wtok));
+        wv = take_plain ? nd : wv; wtok = take_plain ? id1 : wtok; wnext = take_plain ? static_cast<int>(q1.y) : wnext;
+        const bool is_blank = ready && !rescan && !(wv >= xb);
+        const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank) & 0x11111111u;
+        const unsigned stop_m = ~blank_m & 0x11111111u;
+        const int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : kWin;
+        const int jl = 4 * min(nb, kWin - 1);
+        const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
+        const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
+        const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
+        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+        const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
+        const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
+        const float xb2 = __shfl_sync(0xffffffffu, xb, 8), xb3 = __shfl_sync(0xffffffffu, xb, 12);
+        const bool took = nb < kWin && j_ready;             // the row after the blanks selects a token
+        const bool rare = (nb == 0 && !took) || (took && j_rescan) || (took && (n_out & 31) == 31) || nb > 4 ||
+                          (took && (j_next < 0 || j_next >= rec.n_states));
+        if (!rare) {
+          // ---- commit ----
+          score = nb > 0 ? __fadd_rn(score, xb0) : score;
+          score = nb > 1 ? __fadd_rn(score, xb1) : score;
+          score = nb > 2 ? __fadd_rn(score, xb2) : score;
+          score = nb > 3 ? __fadd_rn(score, xb3) : score;
+          score = took ? __fadd_rn(score, j_val) : score;
+          if (lane == 0 && took) emit_buf[n_out & 31] = make_int2(j_tok, t + nb);
+          const int k_row = nb == 0 ? k : 0;
+          const bool closes = took && k_row + 1 == S;       // the token fills its frame
+          const int adv = nb + (closes ? 1 : 0);
+          const int tnext = took ? j_next : s;
+          n_out += took ? 1 : 0;
+          if (rec_on) {
+            if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xb;
+            if (took && lane == 0) vlog[nv + nb] = j_val;
+            if (lane < adv && t + lane + 1 >= f_mid)
+              trace[t + lane + 1] = make_int4(lane >= nb ? tnext : s, n_out - ((took && lane < nb) ? 1 : 0), nv + lane + 1, 0);
+            nv += nb + (took ? 1 : 0);
+          }
+          k = (took && !closes) ? k_row + 1 : 0;
+          {
+            int sr = st + lane; sr -= sr >= nst ? nst : 0;
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];\n\t}"
+                         ::"r"(freeb_a + 8u * sr), "r"(lane < adv ? 1u : 0u) : "memory");
+          }
+          t += adv;
+          st += adv; st -= st >= nst ? nst : 0;
+          lead = (lead + adv * lead_step) & 15;
+          stable = took ? tnext == s : stable;
+          s = tnext;
+          {
+            const uint4 r4 = lds_v4(cache_a + 16u * static_cast<uint32_t>(max(s, 0)));   // the root's record is the empty list
+            L.addr = rsent_cache_a + 8u * r4.x; L.n = static_cast<int>(r4.y);
+            L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w); L.sorted = true;
+          }
+          if (rec_on) {
+            __threadfence_block();
+            if (lane == 0 && adv > 0) prog_publish(flags, t + 1);
+          }
+          spins = 0; no_allrows = false;
+          PROF_ADD(3);
+          PROF_COUNT(8);
+          continue;
+        }
+      }
       const int rq = wide ? 0 : q;                          // window frame of this lane
       const int rk = allrows ? ql : (rq == 0 ? k : 0);      // row of that frame
       int stq = st + rq; if (stq >= nst) stq -= nst;
