@@ -158,6 +158,18 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t a) {
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
   return v;
 }
+// The same loads as plain asm (not volatile): for the list cache and for rows of a held ring slot, which do not
+// change while the decider reads them, so that the compiler may schedule them freely.
+__device__ __forceinline__ uint32_t lds_u16_nv(uint32_t a) {
+  uint16_t v;
+  asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ uint2 lds_v2_nv(uint32_t a) {
+  uint2 v;
+  asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
 __device__ __forceinline__ uint4 lds_v4_volatile(uint32_t a) {
   uint4 v;
   asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
@@ -716,39 +728,43 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const bool ready = t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u;
         const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
         const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
+        // this lane's entries ql, ql + 4, ...: the cached lists are sorted by token, so within a lane a strict
+        // comparison keeps the lowest token among equal values; bit 0 of an entry word is free (2 * token) and
+        // carries "this is the summary's winner" through the reduction
         float wv = -INFINITY;
         uint32_t wdt = 2u * static_cast<uint32_t>(V);
-        bool in_deep = false;
         {
           int i = ql;
           for (; i + 4 < L.n; i += 8) {                      // two entries in flight
-            const uint2 e0 = lds_v2(L.addr + 8u * i), e1 = lds_v2(L.addr + 8u * (i + 4));
-            const uint32_t x0 = lds_u16(row_a + (e0.x & kTokMask)), x1r = lds_u16(row_a + (e1.x & kTokMask));
+            const uint2 e0 = lds_v2_nv(L.addr + 8u * i), e1 = lds_v2_nv(L.addr + 8u * (i + 4));
+            const uint32_t x0 = lds_u16_nv(row_a + (e0.x & kTokMask)), x1r = lds_u16_nv(row_a + (e1.x & kTokMask));
             const float v0 = __fadd_rn(bf16_bits_to_float(x0), __uint_as_float(e0.y));
             const float v1 = __fadd_rn(bf16_bits_to_float(x1r), __uint_as_float(e1.y));
-            in_deep |= (e0.x & kTokMask) == id1x2 || (e1.x & kTokMask) == id1x2;
-            const bool b0 = v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask));
-            wv = b0 ? v0 : wv; wdt = b0 ? e0.x : wdt;
-            const bool b1 = v1 > wv || (v1 == wv && (e1.x & kTokMask) < (wdt & kTokMask));
-            wv = b1 ? v1 : wv; wdt = b1 ? e1.x : wdt;
+            const uint32_t d0 = e0.x | ((e0.x & kTokMask) == id1x2 ? 1u : 0u), d1 = e1.x | ((e1.x & kTokMask) == id1x2 ? 1u : 0u);
+            const bool b01 = v1 > v0;                         // e1's token is the larger one
+            const float vm = b01 ? v1 : v0; const uint32_t dm = b01 ? d1 : d0;
+            const uint32_t seen = (d0 | d1 | wdt) & 1u;
+            const bool bw = vm > wv;
+            wv = bw ? vm : wv; wdt = (bw ? dm : wdt) | seen;
           }
           if (i < L.n) {
-            const uint2 e0 = lds_v2(L.addr + 8u * i);
-            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16(row_a + (e0.x & kTokMask))), __uint_as_float(e0.y));
-            in_deep |= (e0.x & kTokMask) == id1x2;
-            const bool b0 = v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask));
-            wv = b0 ? v0 : wv; wdt = b0 ? e0.x : wdt;
+            const uint2 e0 = lds_v2_nv(L.addr + 8u * i);
+            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + (e0.x & kTokMask))), __uint_as_float(e0.y));
+            const uint32_t d0 = e0.x | ((e0.x & kTokMask) == id1x2 ? 1u : 0u);
+            const uint32_t seen = (d0 | wdt) & 1u;
+            const bool bw = v0 > wv;
+            wv = bw ? v0 : wv; wdt = (bw ? d0 : wdt) | seen;
           }
         }
 #pragma unroll
         for (int off = 1; off <= 2; off <<= 1) {
           const float ov = __shfl_xor_sync(0xffffffffu, wv, off);
           const uint32_t od = __shfl_xor_sync(0xffffffffu, wdt, off);
-          const bool oi = __shfl_xor_sync(0xffffffffu, in_deep, off);
-          const bool bo = ov > wv || (ov == wv && (od & kTokMask) < (wdt & kTokMask));
-          wv = bo ? ov : wv; wdt = bo ? od : wdt;
-          in_deep |= oi;
+          const uint32_t seen = (od | wdt) & 1u;
+          const bool bo = ov > wv || (ov == wv && (od & kTokMask & ~1u) < (wdt & kTokMask & ~1u));
+          wv = bo ? ov : wv; wdt = (bo ? od : wdt) | seen;
         }
+        const bool in_deep = (wdt & 1u) != 0u;
         int wtok = static_cast<int>((wdt & kTokMask) >> 1);
         int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
         // the best plain token (see the general code): exact when it clears the others by the margin, else bounded
@@ -767,9 +783,9 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const int jl = 4 * min(nb, kWin - 1);
         const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
         const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
-        const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
+        const uint32_t j_tn = __shfl_sync(0xffffffffu, (static_cast<uint32_t>(wnext) << TB_RS_TOK_BITS) | static_cast<uint32_t>(wtok), jl);
+        const int j_tok = static_cast<int>(j_tn & kTokMask), j_next = static_cast<int>(j_tn >> TB_RS_TOK_BITS);
         const float j_val = __shfl_sync(0xffffffffu, wv, jl);
-        const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
         const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
         const float xb2 = __shfl_sync(0xffffffffu, xb, 8), xb3 = __shfl_sync(0xffffffffu, xb, 12);
         const bool took = nb < kWin && j_ready;             // the row after the blanks selects a token
@@ -818,8 +834,10 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           spins = 0; no_allrows = false;
           PROF_ADD(3);
           PROF_COUNT(8);
+          PROF_COUNT(13);
           continue;
         }
+        PROF_COUNT(14);
       }
       const int rq = wide ? 0 : q;                          // window frame of this lane
       const int rk = allrows ? ql : (rq == 0 ? k : 0);      // row of that frame
