@@ -756,13 +756,20 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             wv = bw ? v0 : wv; wdt = (bw ? d0 : wdt) | seen;
           }
         }
-#pragma unroll
-        for (int off = 1; off <= 2; off <<= 1) {
-          const float ov = __shfl_xor_sync(0xffffffffu, wv, off);
-          const uint32_t od = __shfl_xor_sync(0xffffffffu, wdt, off);
-          const uint32_t seen = (od | wdt) & 1u;
-          const bool bo = ov > wv || (ov == wv && (od & kTokMask & ~1u) < (wdt & kTokMask & ~1u));
-          wv = bo ? ov : wv; wdt = (bo ? od : wdt) | seen;
+        // the group's best: every lane fetches the other three lanes' results at once and reduces them itself
+        // (minima and maxima only; no predicate until the end).  Equal best values in two lanes -- the lowest
+        // token would decide -- are left to the general code.
+        bool tie;
+        {
+          const float o1 = __shfl_xor_sync(0xffffffffu, wv, 1), o2 = __shfl_xor_sync(0xffffffffu, wv, 2), o3 = __shfl_xor_sync(0xffffffffu, wv, 3);
+          const uint32_t d1 = __shfl_xor_sync(0xffffffffu, wdt, 1), d2 = __shfl_xor_sync(0xffffffffu, wdt, 2), d3 = __shfl_xor_sync(0xffffffffu, wdt, 3);
+          const float hi1 = fmaxf(wv, o1), lo1 = fminf(wv, o1), hi2 = fmaxf(o2, o3), lo2 = fminf(o2, o3);
+          const float gm = fmaxf(hi1, hi2), second = fmaxf(fminf(hi1, hi2), fmaxf(lo1, lo2));
+          tie = second == gm;
+          const uint32_t seen = (wdt | d1 | d2 | d3) & 1u;
+          const uint32_t dsel = wv == gm ? wdt : (o1 == gm ? d1 : (o2 == gm ? d2 : d3));
+          wdt = (dsel & ~1u) | seen;
+          wv = gm;
         }
         const bool in_deep = (wdt & 1u) != 0u;
         int wtok = static_cast<int>((wdt & kTokMask) >> 1);
@@ -773,8 +780,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const int id1 = static_cast<int>(id1x2 >> 1);
         const float ub = (in_deep ? y2b : y1) + lam * L.D;
         const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
-        const bool rescan = (q1.z & kSumOvf) != 0 || (!plain_ok && !(fmaxf(wv, xb) > ub + tau));
-        const bool take_plain = plain_ok && (nd > wv || (nd == wv && id1 < wtok));
+        const bool rescan = (q1.z & kSumOvf) != 0 || tie || (!plain_ok && !(fmaxf(wv, xb) > ub + tau)) || (plain_ok && nd == wv);
+        const bool take_plain = plain_ok && nd > wv;
         wv = take_plain ? nd : wv; wtok = take_plain ? id1 : wtok; wnext = take_plain ? static_cast<int>(q1.y) : wnext;
         const bool is_blank = ready && !rescan && !(wv >= xb);
         const unsigned blank_m = __ballot_sync(0xffffffffu, is_blank) & 0x11111111u;
