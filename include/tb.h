@@ -186,6 +186,8 @@ int tb_batch_status(tb_batch *b, int32_t *device_status, void *stream);
  * block owned by the batch, which this call allocates or grows (freeing the old block, which
  * waits for the device) when B*T*S exceeds what an earlier call needed.  Hence one
  * tb_greedy_decode per batch at a time; if the block cannot be had, streams are decoded whole.
+ * While `stream` is being captured into a CUDA graph nothing is allocated (the call works with
+ * the block an earlier call left, or decodes the streams whole).
  * Errors: TB_ERR_INVALID_ARG (B > n_slots, bad dtype, NULL pointers, non-positive sizes),
  * TB_ERR_CUDA.
  */

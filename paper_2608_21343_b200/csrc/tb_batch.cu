@@ -259,7 +259,11 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
     // the two-segment decode keeps what its second segment produces in scratch memory of the batch; growing it
     // frees the old block first (cudaFree waits for earlier work), so one decode per batch at a time
     const size_t want = tb_greedy_fast_scratch_bytes(B, T, S);
-    if (want > b->seg_scratch_bytes && want <= (static_cast<size_t>(1) << 30)) {
+    // (never while the caller's stream is being captured into a graph: allocation is not allowed there; the decode
+    // then runs with the block it has, or with one segment per stream)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream_), &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+    if (cap == cudaStreamCaptureStatusNone && want > b->seg_scratch_bytes && want <= (static_cast<size_t>(1) << 30)) {
       cudaFree(b->seg_scratch);
       b->seg_scratch = nullptr; b->seg_scratch_bytes = 0;
       if (cudaMalloc(&b->seg_scratch, want) == cudaSuccess) b->seg_scratch_bytes = want;

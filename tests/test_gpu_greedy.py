@@ -420,3 +420,35 @@ def test_pipelined_kernel_soak_against_oracle(tb, block):
             ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
             check_greedy(out, i, ref, f"seed {seed}")
             assert float(out["scores"][i]) == float(ref["score"]), f"seed {seed} stream {i}: score bits"
+
+
+def test_greedy_decode_in_a_cuda_graph(tb):
+    """One decode captured into a CUDA graph and replayed twice gives the outputs of the direct call -- both when
+    an earlier call has sized the batch's scratch memory and when the batch's first decode happens under capture
+    (nothing is allocated there; the streams are then decoded whole)."""
+    w = W.get_workload(2, B=6, T=300, n_phrases=50, n_plants=15)
+    data = W.batch_inputs(w)
+    logits = to_device(data["logits"])
+    refs = [O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]) for i in range(w.B)]
+    for warm in (True, False):
+        batch, _ = make_batch(tb, w, data["phrases"], arena_bytes=8 << 20)
+        n = w.T * w.S
+        out = dict(tokens=torch.zeros((w.B, n), dtype=torch.int32, device="cuda:0"),
+                   frames=torch.zeros((w.B, n), dtype=torch.int32, device="cuda:0"),
+                   counts=torch.zeros(w.B, dtype=torch.int32, device="cuda:0"),
+                   scores=torch.zeros(w.B, dtype=torch.float32, device="cuda:0"),
+                   states=torch.zeros(w.B, dtype=torch.int32, device="cuda:0"))
+        if warm:
+            tb.tb_greedy_decode(batch, logits, out=out)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            tb.tb_greedy_decode(batch, logits, out=out, stream=torch.cuda.current_stream())
+        for _ in range(2):
+            for v in out.values():
+                v.zero_()
+            graph.replay()
+            host = to_host(out)
+            for i in range(w.B):
+                check_greedy(host, i, refs[i], f"graph replay, warm={warm}")
+        assert tb.tb_batch_status(batch) == 0
