@@ -716,7 +716,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       // A lone warp pays tens of cycles for every branch whose condition was only just computed (nothing
       // else can issue while it resolves).  The usual round -- shared mode, lists in the cache -- is therefore
       // computed here as straight-line code with selects; everything unusual (a row that needs the rescan,
-      // nothing ready, a full staging block, a long blank run, a state out of range) is collected in one
+      // nothing ready, a state out of range) is collected in one
       // flag, and then the round falls through, having changed nothing, to the general code below.
       if (fast_ok && !allrows && !wide && !(chk_on && t >= f_mid)) {
         const int rk = q == 0 ? k : 0;
@@ -795,17 +795,31 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const float j_val = __shfl_sync(0xffffffffu, wv, jl);
         const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
         const float xb2 = __shfl_sync(0xffffffffu, xb, 8), xb3 = __shfl_sync(0xffffffffu, xb, 12);
+        const float xb4 = __shfl_sync(0xffffffffu, xb, 16), xb5 = __shfl_sync(0xffffffffu, xb, 20);
+        const float xb6 = __shfl_sync(0xffffffffu, xb, 24), xb7 = __shfl_sync(0xffffffffu, xb, 28);
         const bool took = nb < kWin && j_ready;             // the row after the blanks selects a token
-        const bool rare = (nb == 0 && !took) || (took && j_rescan) || (took && (n_out & 31) == 31) || nb > 4 ||
-                          (took && (j_next < 0 || j_next >= rec.n_states));
+        const bool rare = (nb == 0 && !took) || (took && j_rescan) || (took && (j_next < 0 || j_next >= rec.n_states));
         if (!rare) {
           // ---- commit ----
           score = nb > 0 ? __fadd_rn(score, xb0) : score;
           score = nb > 1 ? __fadd_rn(score, xb1) : score;
           score = nb > 2 ? __fadd_rn(score, xb2) : score;
           score = nb > 3 ? __fadd_rn(score, xb3) : score;
+          score = nb > 4 ? __fadd_rn(score, xb4) : score;
+          score = nb > 5 ? __fadd_rn(score, xb5) : score;
+          score = nb > 6 ? __fadd_rn(score, xb6) : score;
+          score = nb > 7 ? __fadd_rn(score, xb7) : score;
           score = took ? __fadd_rn(score, j_val) : score;
           if (lane == 0 && took) emit_buf[n_out & 31] = make_int2(j_tok, t + nb);
+          {
+            // a token that fills the staging block sends it out (every lane reads its slot in any case: no branch)
+            const bool full_blk = took && (n_out & 31) == 31;
+            __syncwarp();
+            const int2 e = emit_buf[lane];
+            const int o = (n_out & ~31) + lane;
+            if (full_blk && o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+            __syncwarp();
+          }
           const int k_row = nb == 0 ? k : 0;
           const bool closes = took && k_row + 1 == S;       // the token fills its frame
           const int adv = nb + (closes ? 1 : 0);
