@@ -718,6 +718,84 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       // computed here as straight-line code with selects; everything unusual (a row that needs the rescan,
       // nothing ready, a state out of range) is collected in one
       // flag, and then the round falls through, having changed nothing, to the general code below.
+      // ---- the same for a round in the root state (or of an unbound stream): no list, every lane its own row ---
+      if (allrows && L.n == 0 && (fast_ok || !bound) && !(chk_on && t >= f_mid)) {
+        int stq = st + q; stq -= stq >= nst ? nst : 0;
+        const uint32_t sum_a = summ_a + stq * kSumStageBytes + min(ql, kSMax - 1) * 32u;
+        const uint4 q1 = lds_v4_volatile(sum_a + 16u);
+        const uint4 q0 = lds_v4_volatile(sum_a);
+        const bool ready = ql < S && (q > 0 || ql >= k) && t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u &&
+                           (q1.z & kSumOvf) == 0;
+        const float xb = __uint_as_float(q0.z);
+        const float wv = __fadd_rn(__uint_as_float(q0.w), __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
+        const int wtok = static_cast<int>(q1.z & 0xFFFFu), wnext = bound ? static_cast<int>(q1.y) : -1;
+        const unsigned ready_all = __ballot_sync(0xffffffffu, ready);
+        const unsigned blank_all = __ballot_sync(0xffffffffu, ready && !(wv >= xb));
+        const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
+        const unsigned m1 = 0x11111111u;
+        const unsigned smask = S >= 4 ? 0xFFFFFFFFu : (m1 << S) - m1;
+        const unsigned pre = (1u << k) - 1u;
+        const unsigned tok_all = ready_all & ~blank_all;
+        const unsigned tokx = tok_all | pre;
+        const unsigned a0 = tokx & m1, a1 = (tokx >> 1) & m1, a2 = (tokx >> 2) & m1;
+        const unsigned vis = (m1 | (a0 << 1) | ((a0 & a1) << 2) | ((a0 & a1 & a2) << 3)) & smask & ~pre;
+        const unsigned bad = vis & (~ready_all | (tok_all & ~keep_all));
+        const int pb = bad ? __ffs(bad) - 1 : 32;
+        const bool last_tok = pb < 32 && ((tok_all >> (pb & 31)) & 1u);
+        const unsigned cm = (vis & (pb < 32 ? (1u << (pb & 31)) - 1u : 0xFFFFFFFFu)) | (last_tok ? 1u << (pb & 31) : 0u);
+        const unsigned tm = cm & tok_all, bm = cm & blank_all;
+        const int tn = __shfl_sync(0xffffffffu, wnext, pb & 31);
+        const int tnext = last_tok ? tn : s;
+        const int nt = __popc(tm);
+        const bool rare = cm == 0u || nt >= 32 - (n_out & 31) || (last_tok && bound && (tnext < 0 || tnext >= rec.n_states));
+        if (!rare) {
+          const unsigned cl = bm | (tm & (m1 << (S - 1)));
+          const unsigned clf = (cl | (cl >> 1) | (cl >> 2) | (cl >> 3)) & m1;
+          const int fq = __popc(clf);
+          const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * (fq & 7))) & 0xFu) : 0;
+          const unsigned upto = 0xFFFFFFFFu >> (31 - lane);
+          const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
+          const float val = mine_t ? wv : xb;
+          if (rec_on) {
+            if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
+            if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
+              trace[t + q + 1] = make_int4((last_tok && lane == pb) ? tnext : s, n_out + __popc(tm & upto), nv + __popc(cm & upto), 0);
+            nv += __popc(cm);
+          }
+          if (mine_t) emit_buf[(n_out + __popc(tm & upto) - 1) & 31] = make_int2(wtok, t + q);
+          n_out += nt;
+          // the score in visiting order; a row that was not consumed adds -0, which changes nothing
+          const float valm = mine_c ? val : -0.0f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) score = __fadd_rn(score, __shfl_sync(0xffffffffu, valm, i));
+          {
+            int sr = st + lane; sr -= sr >= nst ? nst : 0;
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];\n\t}"
+                         ::"r"(freeb_a + 8u * sr), "r"(lane < fq ? 1u : 0u) : "memory");
+          }
+          k = pos;
+          t += fq;
+          st += fq; st -= st >= nst ? nst : 0;
+          lead = (lead + fq * lead_step) & 15;
+          stable = last_tok ? false : stable;
+          s = tnext;
+          if (bound) {
+            const uint4 r4 = lds_v4(cache_a + 16u * static_cast<uint32_t>(max(s, 0)));
+            L.addr = rsent_cache_a + 8u * r4.x; L.n = static_cast<int>(r4.y);
+            L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w); L.sorted = true;
+          }
+          if (rec_on) {
+            __threadfence_block();
+            if (lane == 0 && fq > 0) prog_publish(flags, t + 1);
+          }
+          spins = 0;
+          PROF_ADD(3);
+          PROF_COUNT(8);
+          PROF_COUNT(13);
+          continue;
+        }
+        PROF_COUNT(14);
+      }
       if (fast_ok && !allrows && !wide && !(chk_on && t >= f_mid)) {
         const int rk = q == 0 ? k : 0;
         int stq = st + q; stq -= stq >= nst ? nst : 0;
