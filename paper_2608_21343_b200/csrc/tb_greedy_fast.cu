@@ -718,131 +718,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       // computed here as straight-line code with selects; everything unusual (a row that needs the rescan,
       // nothing ready, a state out of range) is collected in one
       // flag, and then the round falls through, having changed nothing, to the general code below.
-      // ---- the same for an all-rows round (root state, unbound stream, or a state that repeats itself): every
-      // lane its own row, and the whole list of the state, if it has one
-      if (allrows && (fast_ok || !bound) && !(chk_on && t >= f_mid)) {
-        int stq = st + q; stq -= stq >= nst ? nst : 0;
-        const uint32_t sum_a = summ_a + stq * kSumStageBytes + min(ql, kSMax - 1) * 32u;
-        const uint4 q1 = lds_v4_volatile(sum_a + 16u);
-        const uint4 q0 = lds_v4_volatile(sum_a);
-        const float xb = __uint_as_float(q0.z);
-        // the plain winner: at the root (no list) it is the row's winner
-        float wv = __fadd_rn(__uint_as_float(q0.w), __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
-        int wtok = static_cast<int>(q1.z & 0xFFFFu), wnext = bound ? static_cast<int>(q1.y) : -1;
-        bool rescan = (q1.z & kSumOvf) != 0;
-        if (L.n > 0) {
-          const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + q * lead_step) & 15) + min(ql, kSMax - 1) * row_bytes;
-          const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
-          float lv = -INFINITY;
-          uint32_t ld = 2u * static_cast<uint32_t>(V);
-          bool in_deep = false;
-          int i = 0;
-          for (; i + 3 < L.n; i += 4) {                       // sorted by token: strict comparisons, four in flight
-            const uint32_t ea = L.addr + 8u * i;
-            const uint2 e0 = lds_v2_nv(ea), e1 = lds_v2_nv(ea + 8u), e2 = lds_v2_nv(ea + 16u), e3 = lds_v2_nv(ea + 24u);
-            const uint32_t t0 = e0.x & kTokMask, t1 = e1.x & kTokMask, t2 = e2.x & kTokMask, t3 = e3.x & kTokMask;
-            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t0)), __uint_as_float(e0.y));
-            const float v1 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t1)), __uint_as_float(e1.y));
-            const float v2 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t2)), __uint_as_float(e2.y));
-            const float v3 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t3)), __uint_as_float(e3.y));
-            in_deep |= t0 == id1x2 || t1 == id1x2 || t2 == id1x2 || t3 == id1x2;
-            const bool b01 = v1 > v0, b23 = v3 > v2;
-            const float va = b01 ? v1 : v0, vb = b23 ? v3 : v2;
-            const uint32_t da = b01 ? e1.x : e0.x, db = b23 ? e3.x : e2.x;
-            const bool bab = vb > va;
-            const float vm = bab ? vb : va;
-            const uint32_t dm = bab ? db : da;
-            const bool bw = vm > lv;
-            lv = bw ? vm : lv; ld = bw ? dm : ld;
-          }                                                   // (cached lists are padded to multiples of four)
-          const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y);
-          const bool plain_ok = !in_deep && ((q1.z & kSumGap) != 0 || s <= 0);
-          const float ub = (in_deep ? y2b : y1) + lam * L.D;
-          const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
-          rescan = rescan || (!plain_ok && !(fmaxf(lv, xb) > ub + tau)) || (plain_ok && wv == lv);
-          const bool take_plain = plain_ok && wv > lv;
-          wv = take_plain ? wv : lv;
-          wtok = take_plain ? wtok : static_cast<int>((ld & kTokMask) >> 1);
-          wnext = take_plain ? wnext : static_cast<int>(ld >> TB_RS_TOK_BITS);
-        }
-        const bool ready = ql < S && (q > 0 || ql >= k) && t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u && !rescan;
-        const unsigned ready_all = __ballot_sync(0xffffffffu, ready);
-        const unsigned blank_all = __ballot_sync(0xffffffffu, ready && !(wv >= xb));
-        const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
-        const unsigned m1 = 0x11111111u;
-        const unsigned smask = S >= 4 ? 0xFFFFFFFFu : (m1 << S) - m1;
-        const unsigned pre = (1u << k) - 1u;
-        const unsigned tok_all = ready_all & ~blank_all;
-        const unsigned tokx = tok_all | pre;
-        const unsigned a0 = tokx & m1, a1 = (tokx >> 1) & m1, a2 = (tokx >> 2) & m1;
-        const unsigned vis = (m1 | (a0 << 1) | ((a0 & a1) << 2) | ((a0 & a1 & a2) << 3)) & smask & ~pre;
-        const unsigned bad = vis & (~ready_all | (tok_all & ~keep_all));
-        const int pb = bad ? __ffs(bad) - 1 : 32;
-        const bool last_tok = pb < 32 && ((tok_all >> (pb & 31)) & 1u);
-        const unsigned cm = (vis & (pb < 32 ? (1u << (pb & 31)) - 1u : 0xFFFFFFFFu)) | (last_tok ? 1u << (pb & 31) : 0u);
-        const unsigned tm = cm & tok_all, bm = cm & blank_all;
-        const int tn = __shfl_sync(0xffffffffu, wnext, pb & 31);
-        const int tnext = last_tok ? tn : s;
-        const int nt = __popc(tm);
-        const bool rare = cm == 0u || (last_tok && bound && (tnext < 0 || tnext >= rec.n_states));
-        if (!rare) {
-          const unsigned cl = bm | (tm & (m1 << (S - 1)));
-          const unsigned clf = (cl | (cl >> 1) | (cl >> 2) | (cl >> 3)) & m1;
-          const int fq = __popc(clf);
-          const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * (fq & 7))) & 0xFu) : 0;
-          const unsigned upto = 0xFFFFFFFFu >> (31 - lane);
-          const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
-          const float val = mine_t ? wv : xb;
-          if (rec_on) {
-            if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
-            if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
-              trace[t + q + 1] = make_int4((last_tok && lane == pb) ? tnext : s, n_out + __popc(tm & upto), nv + __popc(cm & upto), 0);
-            nv += __popc(cm);
-          }
-          {
-            // through the staging buffer; when these tokens fill the current block it goes out in between
-            const int room = 32 - (n_out & 31), rank = __popc(tm & upto) - 1;
-            if (mine_t && rank < room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
-            __syncwarp();
-            const int2 e = emit_buf[lane];
-            const int o = (n_out & ~31) + lane;
-            if (nt >= room && o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
-            __syncwarp();
-            if (mine_t && rank >= room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
-          }
-          n_out += nt;
-          // the score in visiting order; a row that was not consumed adds -0, which changes nothing
-          const float valm = mine_c ? val : -0.0f;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) score = __fadd_rn(score, __shfl_sync(0xffffffffu, valm, i));
-          {
-            int sr = st + lane; sr -= sr >= nst ? nst : 0;
-            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];\n\t}"
-                         ::"r"(freeb_a + 8u * sr), "r"(lane < fq ? 1u : 0u) : "memory");
-          }
-          k = pos;
-          t += fq;
-          st += fq; st -= st >= nst ? nst : 0;
-          lead = (lead + fq * lead_step) & 15;
-          stable = last_tok ? false : stable;
-          s = tnext;
-          if (bound) {
-            const uint4 r4 = lds_v4(cache_a + 16u * static_cast<uint32_t>(max(s, 0)));
-            L.addr = rsent_cache_a + 8u * r4.x; L.n = static_cast<int>(r4.y);
-            L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w); L.sorted = true;
-          }
-          if (rec_on) {
-            __threadfence_block();
-            if (lane == 0 && fq > 0) prog_publish(flags, t + 1);
-          }
-          spins = 0;
-          PROF_ADD(3);
-          PROF_COUNT(8);
-          PROF_COUNT(13);
-          continue;
-        }
-        PROF_COUNT(14);
-      }
       if (fast_ok && !allrows && !wide && !(chk_on && t >= f_mid)) {
         const int rk = q == 0 ? k : 0;
         int stq = st + q; stq -= stq >= nst ? nst : 0;
@@ -978,6 +853,131 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             if (lane == 0 && adv > 0) prog_publish(flags, t + 1);
           }
           spins = 0; no_allrows = false;
+          PROF_ADD(3);
+          PROF_COUNT(8);
+          PROF_COUNT(13);
+          continue;
+        }
+        PROF_COUNT(14);
+      }
+      // ---- the same for an all-rows round (root state, unbound stream, or a state that repeats itself): every
+      // lane its own row, and the whole list of the state, if it has one
+      if (allrows && (fast_ok || !bound) && !(chk_on && t >= f_mid)) {
+        int stq = st + q; stq -= stq >= nst ? nst : 0;
+        const uint32_t sum_a = summ_a + stq * kSumStageBytes + min(ql, kSMax - 1) * 32u;
+        const uint4 q1 = lds_v4_volatile(sum_a + 16u);
+        const uint4 q0 = lds_v4_volatile(sum_a);
+        const float xb = __uint_as_float(q0.z);
+        // the plain winner: at the root (no list) it is the row's winner
+        float wv = __fadd_rn(__uint_as_float(q0.w), __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
+        int wtok = static_cast<int>(q1.z & 0xFFFFu), wnext = bound ? static_cast<int>(q1.y) : -1;
+        bool rescan = (q1.z & kSumOvf) != 0;
+        if (L.n > 0) {
+          const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + q * lead_step) & 15) + min(ql, kSMax - 1) * row_bytes;
+          const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
+          float lv = -INFINITY;
+          uint32_t ld = 2u * static_cast<uint32_t>(V);
+          bool in_deep = false;
+          int i = 0;
+          for (; i + 3 < L.n; i += 4) {                       // sorted by token: strict comparisons, four in flight
+            const uint32_t ea = L.addr + 8u * i;
+            const uint2 e0 = lds_v2_nv(ea), e1 = lds_v2_nv(ea + 8u), e2 = lds_v2_nv(ea + 16u), e3 = lds_v2_nv(ea + 24u);
+            const uint32_t t0 = e0.x & kTokMask, t1 = e1.x & kTokMask, t2 = e2.x & kTokMask, t3 = e3.x & kTokMask;
+            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t0)), __uint_as_float(e0.y));
+            const float v1 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t1)), __uint_as_float(e1.y));
+            const float v2 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t2)), __uint_as_float(e2.y));
+            const float v3 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t3)), __uint_as_float(e3.y));
+            in_deep |= t0 == id1x2 || t1 == id1x2 || t2 == id1x2 || t3 == id1x2;
+            const bool b01 = v1 > v0, b23 = v3 > v2;
+            const float va = b01 ? v1 : v0, vb = b23 ? v3 : v2;
+            const uint32_t da = b01 ? e1.x : e0.x, db = b23 ? e3.x : e2.x;
+            const bool bab = vb > va;
+            const float vm = bab ? vb : va;
+            const uint32_t dm = bab ? db : da;
+            const bool bw = vm > lv;
+            lv = bw ? vm : lv; ld = bw ? dm : ld;
+          }                                                   // (cached lists are padded to multiples of four)
+          const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y);
+          const bool plain_ok = !in_deep && ((q1.z & kSumGap) != 0 || s <= 0);
+          const float ub = (in_deep ? y2b : y1) + lam * L.D;
+          const float tau = (fabsf(y1) + 4.0f * L.bmag) * 3.814697265625e-6f + 1e-30f;
+          rescan = rescan || (!plain_ok && !(fmaxf(lv, xb) > ub + tau)) || (plain_ok && wv == lv);
+          const bool take_plain = plain_ok && wv > lv;
+          wv = take_plain ? wv : lv;
+          wtok = take_plain ? wtok : static_cast<int>((ld & kTokMask) >> 1);
+          wnext = take_plain ? wnext : static_cast<int>(ld >> TB_RS_TOK_BITS);
+        }
+        const bool ready = ql < S && (q > 0 || ql >= k) && t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u && !rescan;
+        const unsigned ready_all = __ballot_sync(0xffffffffu, ready);
+        const unsigned blank_all = __ballot_sync(0xffffffffu, ready && !(wv >= xb));
+        const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
+        const unsigned m1 = 0x11111111u;
+        const unsigned smask = S >= 4 ? 0xFFFFFFFFu : (m1 << S) - m1;
+        const unsigned pre = (1u << k) - 1u;
+        const unsigned tok_all = ready_all & ~blank_all;
+        const unsigned tokx = tok_all | pre;
+        const unsigned a0 = tokx & m1, a1 = (tokx >> 1) & m1, a2 = (tokx >> 2) & m1;
+        const unsigned vis = (m1 | (a0 << 1) | ((a0 & a1) << 2) | ((a0 & a1 & a2) << 3)) & smask & ~pre;
+        const unsigned bad = vis & (~ready_all | (tok_all & ~keep_all));
+        const int pb = bad ? __ffs(bad) - 1 : 32;
+        const bool last_tok = pb < 32 && ((tok_all >> (pb & 31)) & 1u);
+        const unsigned cm = (vis & (pb < 32 ? (1u << (pb & 31)) - 1u : 0xFFFFFFFFu)) | (last_tok ? 1u << (pb & 31) : 0u);
+        const unsigned tm = cm & tok_all, bm = cm & blank_all;
+        const int tn = __shfl_sync(0xffffffffu, wnext, pb & 31);
+        const int tnext = last_tok ? tn : s;
+        const int nt = __popc(tm);
+        const bool rare = cm == 0u || (last_tok && bound && (tnext < 0 || tnext >= rec.n_states));
+        if (!rare) {
+          const unsigned cl = bm | (tm & (m1 << (S - 1)));
+          const unsigned clf = (cl | (cl >> 1) | (cl >> 2) | (cl >> 3)) & m1;
+          const int fq = __popc(clf);
+          const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * (fq & 7))) & 0xFu) : 0;
+          const unsigned upto = 0xFFFFFFFFu >> (31 - lane);
+          const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
+          const float val = mine_t ? wv : xb;
+          if (rec_on) {
+            if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
+            if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
+              trace[t + q + 1] = make_int4((last_tok && lane == pb) ? tnext : s, n_out + __popc(tm & upto), nv + __popc(cm & upto), 0);
+            nv += __popc(cm);
+          }
+          {
+            // through the staging buffer; when these tokens fill the current block it goes out in between
+            const int room = 32 - (n_out & 31), rank = __popc(tm & upto) - 1;
+            if (mine_t && rank < room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
+            __syncwarp();
+            const int2 e = emit_buf[lane];
+            const int o = (n_out & ~31) + lane;
+            if (nt >= room && o < out_cap) { out_tok[o] = e.x; out_frm[o] = e.y; }
+            __syncwarp();
+            if (mine_t && rank >= room) emit_buf[(n_out + rank) & 31] = make_int2(wtok, t + q);
+          }
+          n_out += nt;
+          // the score in visiting order; a row that was not consumed adds -0, which changes nothing
+          const float valm = mine_c ? val : -0.0f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) score = __fadd_rn(score, __shfl_sync(0xffffffffu, valm, i));
+          {
+            int sr = st + lane; sr -= sr >= nst ? nst : 0;
+            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];\n\t}"
+                         ::"r"(freeb_a + 8u * sr), "r"(lane < fq ? 1u : 0u) : "memory");
+          }
+          k = pos;
+          t += fq;
+          st += fq; st -= st >= nst ? nst : 0;
+          lead = (lead + fq * lead_step) & 15;
+          stable = last_tok ? false : stable;
+          s = tnext;
+          if (bound) {
+            const uint4 r4 = lds_v4(cache_a + 16u * static_cast<uint32_t>(max(s, 0)));
+            L.addr = rsent_cache_a + 8u * r4.x; L.n = static_cast<int>(r4.y);
+            L.D = __uint_as_float(r4.z); L.bmag = __uint_as_float(r4.w); L.sorted = true;
+          }
+          if (rec_on) {
+            __threadfence_block();
+            if (lane == 0 && fq > 0) prog_publish(flags, t + 1);
+          }
+          spins = 0;
           PROF_ADD(3);
           PROF_COUNT(8);
           PROF_COUNT(13);
