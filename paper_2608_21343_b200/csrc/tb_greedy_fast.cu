@@ -735,6 +735,24 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         uint32_t wdt = 2u * static_cast<uint32_t>(V);
         {
           int i = ql;
+          for (; i + 12 < L.n; i += 16) {                     // four entries in flight, compared as a tree
+            const uint32_t ea = L.addr + 8u * i;
+            const uint2 e0 = lds_v2_nv(ea), e1 = lds_v2_nv(ea + 32u), e2 = lds_v2_nv(ea + 64u), e3 = lds_v2_nv(ea + 96u);
+            const uint32_t t0 = e0.x & kTokMask, t1 = e1.x & kTokMask, t2 = e2.x & kTokMask, t3 = e3.x & kTokMask;
+            const float v0 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t0)), __uint_as_float(e0.y));
+            const float v1 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t1)), __uint_as_float(e1.y));
+            const float v2 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t2)), __uint_as_float(e2.y));
+            const float v3 = __fadd_rn(bf16_bits_to_float(lds_u16_nv(row_a + t3)), __uint_as_float(e3.y));
+            const uint32_t seen = ((t0 == id1x2 || t1 == id1x2 || t2 == id1x2 || t3 == id1x2) ? 1u : 0u) | (wdt & 1u);
+            const bool b01 = v1 > v0, b23 = v3 > v2;
+            const float va = b01 ? v1 : v0, vb = b23 ? v3 : v2;
+            const uint32_t da = b01 ? e1.x : e0.x, db = b23 ? e3.x : e2.x;
+            const bool bab = vb > va;
+            const float vm = bab ? vb : va;
+            const uint32_t dm = bab ? db : da;
+            const bool bw = vm > wv;
+            wv = bw ? vm : wv; wdt = (bw ? dm : wdt) | seen;
+          }
           for (; i + 4 < L.n; i += 8) {                      // two entries in flight
             const uint2 e0 = lds_v2_nv(L.addr + 8u * i), e1 = lds_v2_nv(L.addr + 8u * (i + 4));
             const uint32_t x0 = lds_u16_nv(row_a + (e0.x & kTokMask)), x1r = lds_u16_nv(row_a + (e1.x & kTokMask));
