@@ -403,9 +403,14 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
   float acc = 0.0f;
   int u = s;
   if (u < 0 || u >= n_states) { if (lane == 0) atomicOr(status, TB_STATUS_BAD_STATE); u = 0; }
+  TbStateRec rec{0, 0, 0, 0.0f};
+  if (u != 0) rec = strec[u];
   for (int it = 0; u != 0; ++it) {
     if (it > max_depth + 1) { if (lane == 0) atomicOr(status, TB_STATUS_WALK_TOO_DEEP); break; }
-    const TbStateRec rec = strec[u];
+    // the next chain state's record is requested before this state's arcs are: the two trips to L2 overlap
+    const int nu = rec.fail;
+    TbStateRec nrec = rec;
+    if (nu > 0 && nu < n_states) nrec = strec[nu];
     const int n_start = n;
     for (int e0 = rec.tok_begin; e0 < rec.tok_end; e0 += 32) {
       const int e = e0 + lane;
@@ -426,7 +431,8 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
       __syncwarp();
     }
     acc = __fadd_rn(acc, rec.bw);
-    u = rec.fail;
+    u = (nu > 0 && nu < n_states) ? nu : 0;
+    rec = nrec;
   }
   for (int i = lane; i < n; i += 32) cls_seen[cls16[(lbuf[i].dst_tok & kTokMask) >> 1]] = -1;   // leave the map clean
   const int n_pad = (n + 3) & ~3;
