@@ -412,11 +412,13 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
     TbStateRec nrec = rec;
     if (nu > 0 && nu < n_states) nrec = strec[nu];
     const int n_start = n;
+    TbTokEnt ahead{0u, 0.0f, 0, 0};
+    if (rec.tok_begin + lane < rec.tok_end) ahead = tokent[rec.tok_begin + lane];
     for (int e0 = rec.tok_begin; e0 < rec.tok_end; e0 += 32) {
       const int e = e0 + lane;
       const bool have = e < rec.tok_end;
-      TbTokEnt ent{0u, 0.0f, 0, 0};
-      if (have) ent = tokent[e];
+      const TbTokEnt ent = ahead;                           // (the next 32 arcs are requested before these are dealt with)
+      if (e + 32 < rec.tok_end) ahead = tokent[e + 32];
       const int c = static_cast<int>(ent.tok_cls >> 16);
       const int seen = have ? cls_seen[c] : 0;
       const bool fresh = have && (seen < 0 || seen >= n_start);   // same class again only as a sibling from this state
