@@ -452,3 +452,30 @@ def test_greedy_decode_in_a_cuda_graph(tb):
             for i in range(w.B):
                 check_greedy(host, i, refs[i], f"graph replay, warm={warm}")
         assert tb.tb_batch_status(batch) == 0
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_pipelined_kernel_masked_logits(tb, seed):
+    """Token logits of -inf (masked tokens), whole rows with every token masked: the decode picks blank there and
+    stays bit-exact with the oracle."""
+    rng = np.random.default_rng(8000 + seed)
+    V, S, B, T = int(rng.choice([257, 1024])), int(rng.integers(2, 4)), 4, int(rng.choice([90, 260]))
+    cc = (np.arange(V) // 3).astype(np.int32)
+    x = rng.standard_normal((B, T, S, V + 1)).astype(np.float32)
+    x[..., V] += 2.0
+    m = rng.random(x.shape) < 0.15
+    m[..., V] = False
+    x[m] = -np.inf
+    x[:, ::7, :, :V] = -np.inf
+    xb = W.f32_to_bf16_bits(x)
+    hot = rng.integers(0, V, size=12)
+    lists = [[[int(t) for t in rng.choice(hot, size=rng.integers(1, 6))] for _ in range(40)] for _ in range(B)]
+    batch = tb.tb_batch_create(V, cc, B, arena_bytes=8 << 20)
+    for i, p in enumerate(lists):
+        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc))
+    out = to_host(tb.tb_greedy_decode(batch, to_device(xb)))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(lists):
+        ref = O.greedy_rnnt(O.Graph(p, V, case_class=cc), xb[i])
+        check_greedy(out, i, ref, f"masked seed {seed}")
+        assert float(out["scores"][i]) == float(ref["score"]) or (np.isinf(ref["score"]) and np.isinf(out["scores"][i]))
