@@ -727,6 +727,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       // nothing ready, a state out of range) is collected in one
       // flag, and then the round falls through, having changed nothing, to the general code below.
       if (fast_ok && !allrows && !wide && !(chk_on && t >= f_mid)) {
+      fast_again:
         const int rk = q == 0 ? k : 0;
         int stq = st + q; stq -= stq >= nst ? nst : 0;
         const uint32_t sum_a = summ_a + stq * kSumStageBytes + rk * 32u;
@@ -882,6 +883,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           PROF_ADD(3);
           PROF_COUNT(8);
           PROF_COUNT(13);
+          // the next round is of the same kind more often than not: straight back, without the loop's bookkeeping
+          if (L.n > 0 && L.n <= kGroupDeep && !stable && t < end && it + 1 < max_rounds && !(chk_on && t >= f_mid)) { ++it; goto fast_again; }
           continue;
         }
         PROF_COUNT(14);
