@@ -168,6 +168,42 @@ class Graph:
         return b.value, nx.value
 
 
+class GraphFromArrays(Graph):
+    """A graph given as its arrays (built by another front end of the oracle, e.g. ``variative.py``); the decode
+    functions of the C file read it through the same structure as a graph the C file built itself."""
+
+    def __init__(self, a: dict):
+        self.n_states, self.n_arcs, self.n_classes = int(a["n_states"]), int(a["n_arcs"]), int(a["n_classes"])
+        self.vocab, self.max_depth, self.lam = int(a["vocab"]), int(a["max_depth"]), float(a["lam"])
+        self.state_arc_begin = np.ascontiguousarray(a["state_arc_begin"], dtype=np.int32)
+        self.arc_class = np.ascontiguousarray(a["arc_class"], dtype=np.int32)
+        self.arc_dst = np.ascontiguousarray(a["arc_dst"], dtype=np.int32)
+        self.arc_w = np.ascontiguousarray(a["arc_w"], dtype=np.float32)
+        self.state_fail = np.ascontiguousarray(a["state_fail"], dtype=np.int32)
+        self.state_bw = np.ascontiguousarray(a["state_bw"], dtype=np.float32)
+        self.state_final = np.ascontiguousarray(a["state_final"], dtype=np.float32)
+        self.state_depth = np.ascontiguousarray(a["state_depth"], dtype=np.uint8)
+        self.case_class = np.ascontiguousarray(a["case_class"], dtype=np.int32)
+        assert self.state_arc_begin.shape == (self.n_states + 1,) and self.arc_class.shape == (self.n_arcs,)
+        s = _GraphStruct()
+        s.n_states, s.n_arcs, s.n_classes = self.n_states, self.n_arcs, self.n_classes
+        s.vocab, s.max_depth, s.lambda_ = self.vocab, self.max_depth, self.lam
+
+        def p(x, t):
+            return x.ctypes.data_as(C.POINTER(t))
+
+        s.state_arc_begin = p(self.state_arc_begin, C.c_int32); s.arc_class = p(self.arc_class, C.c_int32)
+        s.arc_dst = p(self.arc_dst, C.c_int32); s.arc_w = p(self.arc_w, C.c_float)
+        s.state_fail = p(self.state_fail, C.c_int32); s.state_bw = p(self.state_bw, C.c_float)
+        s.state_final = p(self.state_final, C.c_float); s.state_depth = p(self.state_depth, C.c_uint8)
+        s.case_class = p(self.case_class, C.c_int32)
+        self._struct = s                       # the arrays above stay alive with this object
+        self.handle = C.cast(C.pointer(s), C.c_void_p)
+
+    def __del__(self):                         # nothing of this graph was allocated by the C file
+        self.handle = None
+
+
 def null_step(v: int):
     b = C.c_float()
     nx = C.c_int32()

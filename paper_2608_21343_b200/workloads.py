@@ -344,3 +344,69 @@ class ChurnSchedule:
                 self.next_stream += 1
                 self.pending.append(slot)
         return chunk, lengths, binds
+
+
+# ----------------------------------------------------------------------------------------------
+# piece vocabularies and phrases as strings (inputs of the variative compile; Sec. 2.1 para. 4-5)
+# ----------------------------------------------------------------------------------------------
+
+def make_piece_vocab(seed: int, letters: int = 12, merged: int = 200, max_len: int = 4) -> List[bytes]:
+    """A synthetic piece vocabulary (stand-in for a SentencePiece model's): every letter as a piece of its own
+    in both cases (a, A, b, B, ...), then ``merged`` distinct lower-case pieces of 2..max_len letters; about
+    half of them also have a Title-case piece and a quarter an UPPER-case one -- a vocabulary does not hold
+    every case variant of every piece."""
+    rng = np.random.default_rng([seed, 77001])
+    out: List[bytes] = []
+    for i in range(letters):
+        out.append(bytes([97 + i]))
+        out.append(bytes([65 + i]))
+    seen = set()
+    while len(seen) < merged:
+        n = int(rng.integers(2, max_len + 1))
+        seen.add(bytes(int(x) + 97 for x in rng.integers(0, letters, size=n)))
+    for p in sorted(seen):
+        out.append(p)
+        r = rng.random()
+        if r < 0.5:
+            out.append(bytes([p[0] - 32]) + p[1:])
+        if r < 0.25:
+            out.append(bytes(b - 32 for b in p))
+    return out
+
+
+def draw_string_phrases(seed: int, pieces: List[bytes], n: int, len_lo: int = 1, len_hi: int = 4) -> List[bytes]:
+    """``n`` phrases, each the concatenation of len_lo..len_hi pieces drawn from the lower-case pieces (so that
+    merged pieces occur inside phrases), given in lower case as user lists usually are."""
+    rng = np.random.default_rng([seed, 77002])
+    lower = [p for p in pieces if p == p.lower()]
+    out = []
+    for _ in range(n):
+        k = int(rng.integers(len_lo, len_hi + 1))
+        out.append(b"".join(lower[int(i)] for i in rng.integers(0, len(lower), size=k)))
+    return out
+
+
+def random_spelling(rng: np.random.Generator, phrase: bytes, pieces: List[bytes], casing: Optional[int] = None) -> List[int]:
+    """Token ids of one way the model could emit ``phrase``: a casing (0 lower, 1 UPPER, 2 Title, 3 random per
+    letter; drawn if None) and a random segmentation of that spelling into pieces the vocabulary holds."""
+    ids = {}
+    for t, p in enumerate(pieces):
+        ids.setdefault(p, t)
+    longest = max(len(p) for p in pieces)
+    mode = int(rng.integers(0, 4)) if casing is None else casing
+    low = phrase.lower()
+    if mode == 0:
+        s = low
+    elif mode == 1:
+        s = low.upper()
+    elif mode == 2:
+        s = low[:1].upper() + low[1:]
+    else:
+        s = bytes((b - 32 if (97 <= b <= 122 and rng.random() < 0.5) else b) for b in low)
+    toks, i = [], 0
+    while i < len(s):
+        cand = [m for m in range(1, min(longest, len(s) - i) + 1) if s[i:i + m] in ids]
+        m = cand[int(rng.integers(0, len(cand)))]
+        toks.append(ids[s[i:i + m]])
+        i += m
+    return toks
