@@ -60,6 +60,7 @@ extern "C" {
 /* Limits of this build. */
 #define TB_MAX_VOCAB 8192           /* non-blank tokens */
 #define TB_MAX_PHRASE_LEN 255       /* tokens per phrase (graph depth is stored in a byte) */
+#define TB_MAX_PIECE_LEN 32         /* characters (bytes) per vocabulary piece, variative compile */
 #define TB_MAX_BEAM 32
 #define TB_NOALLOC_MAX_STREAMS 256 /* streams per tb_greedy_decode_noalloc call */
 
@@ -112,6 +113,49 @@ const char *tb_strerror(int code);
 int tb_graph_compile(const int32_t *phrase_tokens, const int64_t *phrase_offsets, int32_t n_phrases,
                      const float *token_weights, const int32_t *case_class, int32_t vocab, float lambda,
                      uint32_t flags, tb_graph **out);
+
+/*
+ * Token -> class map of a piece vocabulary for case-insensitive matching (Sec. 2.1 para. 5: a piece
+ * counts wherever its lower-cased spelling matches): pieces with the same lower-cased spelling
+ * (ASCII letters are folded, other bytes compared as they are) share a class; classes are numbered in
+ * order of the lowest token id that has them.  Pass the result to tb_batch_create for a batch that
+ * binds graphs made by tb_graph_compile_variative over the same vocabulary.
+ *   piece_chars    host bytes [piece_offsets[vocab]]: the pieces' spellings, back to back
+ *   piece_offsets  host int64 [vocab+1], increasing, first entry 0; every piece 1..TB_MAX_PIECE_LEN bytes
+ *   out_case_class host int32 [vocab], written;  out_n_classes host int32 or NULL
+ * Errors: TB_ERR_INVALID_ARG, TB_ERR_OOM.
+ */
+int tb_piece_classes(const uint8_t *piece_chars, const int64_t *piece_offsets, int32_t vocab,
+                     int32_t *out_case_class, int32_t *out_n_classes);
+
+/*
+ * Compile one phrase list, given as text, into a variative case-insensitive boosting graph (host
+ * only).  Sec. 2.1 para. 4-7 and Eq. 1: the lower-cased phrase is a chain of its characters; every
+ * piece whose lower-cased spelling covers a contiguous stretch of the chain is an arc over it, so
+ * the graph accepts every casing and every segmentation of the phrase; states carry a cumulative
+ * potential and an arc scores the difference of the potentials of its ends.  The potentials come
+ * from the greedy segmentation of the lower-cased phrase (here: longest spelling first): a token of
+ * m characters with score w gives its character i (0-based) the share
+ * w * exp((i+1)^tau) / sum_j exp((j+1)^tau).  Phrases sharing a prefix share its states, a state
+ * taking the largest share given to it.  Suffix links and their weights are those of
+ * tb_graph_compile, taken over the characters; an arc over several characters weighs what the
+ * single-character arcs along it weigh together, so all spellings of a phrase earn the same total.
+ * The result has the same array layout and is bound, decoded and freed like any other graph; its
+ * classes are those of tb_piece_classes.
+ *   phrase_chars   host bytes [phrase_offsets[n_phrases]]: the phrases' text, any casing, back to back
+ *   phrase_offsets host int64 [n_phrases+1], non-decreasing, first entry 0; at most 255 bytes per phrase
+ *   phrase_weights host float [n_phrases] or NULL (= 1.0): score w of every token of the phrase's
+ *                  greedy segmentation; finite and >= 0
+ *   piece_chars, piece_offsets, vocab  the piece vocabulary, as for tb_piece_classes; every
+ *                  character of every phrase must be the spelling of some piece
+ *   tau            Eq. 1's exponent, finite and >= 0 (0: uniform split; large: all at the token's end)
+ *   lambda, flags, out  as for tb_graph_compile
+ * Empty phrases are skipped.  Errors: TB_ERR_INVALID_ARG, TB_ERR_OOM.
+ */
+int tb_graph_compile_variative(const uint8_t *phrase_chars, const int64_t *phrase_offsets, int32_t n_phrases,
+                               const float *phrase_weights, const uint8_t *piece_chars,
+                               const int64_t *piece_offsets, int32_t vocab, float tau, float lambda,
+                               uint32_t flags, tb_graph **out);
 
 /* Fill *out with pointers into g (host).  TB_ERR_INVALID_ARG on NULL. */
 int tb_graph_view_get(const tb_graph *g, tb_graph_view *out);

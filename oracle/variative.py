@@ -90,7 +90,9 @@ def eq1_split(w: float, m: int, tau: float):
 
 
 def build(phrases, pieces, weights=None, tau: float = 1.0, lam: float = 1.0) -> dict:
-    """Compile phrases (byte strings, any casing) over the piece vocabulary (byte strings)."""
+    """Compile phrases (byte strings, any casing) over the piece vocabulary (byte strings).
+    tau and the weights are taken at float32 precision (what a caller of the library can pass)."""
+    tau = float(np.float32(tau))
     case_class, spell = piece_classes(pieces)
     class_of = {c: i for i, c in enumerate(spell)}
     longest = max(len(c) for c in spell)
@@ -103,7 +105,7 @@ def build(phrases, pieces, weights=None, tau: float = 1.0, lam: float = 1.0) -> 
             continue
         if len(canon) > 255:
             raise ValueError("phrase longer than 255 characters")
-        w = 1.0 if weights is None else float(weights[pi])
+        w = 1.0 if weights is None else float(np.float32(weights[pi]))
         shares = [d for m in greedy_backbone(canon, class_of, longest) for d in eq1_split(w, m, tau)]
         u = 0
         for i, b in enumerate(canon):

@@ -47,6 +47,9 @@ _vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
 _SIGS = {
     "tb_strerror": (C.c_char_p, [C.c_int]),
     "tb_graph_compile": (C.c_int, [_vp, _vp, _i32, _vp, _vp, _i32, C.c_float, C.c_uint32, C.POINTER(_vp)]),
+    "tb_piece_classes": (C.c_int, [_vp, _vp, _i32, _vp, C.POINTER(_i32)]),
+    "tb_graph_compile_variative": (C.c_int, [_vp, _vp, _i32, _vp, _vp, _vp, _i32, C.c_float, C.c_float, C.c_uint32,
+                                             C.POINTER(_vp)]),
     "tb_graph_view_get": (C.c_int, [_vp, C.POINTER(_GraphView)]),
     "tb_graph_free": (None, [_vp]),
     "tb_batch_create": (C.c_int, [_i32, _vp, _i32, _i32, _i32, C.c_size_t, C.c_int, C.POINTER(_vp)]),
@@ -157,6 +160,36 @@ def tb_graph_compile(phrases, vocab: int, case_class=None, token_weights=None, l
     h = _vp()
     _check(_lib.tb_graph_compile(_hp(toks), _hp(offs), n, _hp(w), _hp(cc), vocab, float(lam), flags, C.byref(h)),
            "tb_graph_compile")
+    return Graph(h)
+
+
+def _flat_bytes(items):
+    """List of byte strings -> (bytes uint8, offsets int64)."""
+    offs = np.zeros(len(items) + 1, dtype=np.int64)
+    if len(items):
+        offs[1:] = np.cumsum([len(x) for x in items])
+    flat = np.frombuffer(b"".join(items), dtype=np.uint8).copy() if offs[-1] else np.zeros(0, dtype=np.uint8)
+    return flat, offs
+
+
+def tb_piece_classes(pieces):
+    """pieces: list of byte strings (the vocabulary's spellings).  Returns (case_class int32 [V], n_classes)."""
+    flat, offs = _flat_bytes(pieces)
+    cc = np.zeros(len(pieces), dtype=np.int32)
+    n = _i32()
+    _check(_lib.tb_piece_classes(_hp(flat), _hp(offs), len(pieces), _hp(cc), C.byref(n)), "tb_piece_classes")
+    return cc, n.value
+
+
+def tb_graph_compile_variative(phrases, pieces, phrase_weights=None, tau: float = 1.0, lam: float = 1.0,
+                               flags: int = 0) -> Graph:
+    """phrases, pieces: lists of byte strings (phrases in any casing)."""
+    pf, po = _flat_bytes(phrases)
+    vf, vo = _flat_bytes(pieces)
+    w = _host(phrase_weights, np.float32)
+    h = _vp()
+    _check(_lib.tb_graph_compile_variative(_hp(pf), _hp(po), len(phrases), _hp(w), _hp(vf), _hp(vo), len(pieces),
+                                           float(tau), float(lam), flags, C.byref(h)), "tb_graph_compile_variative")
     return Graph(h)
 
 
