@@ -410,3 +410,29 @@ def random_spelling(rng: np.random.Generator, phrase: bytes, pieces: List[bytes]
         toks.append(ids[s[i:i + m]])
         i += m
     return toks
+
+
+@dataclass
+class _RowShape:
+    V: int
+    S: int
+    dtype: str
+
+
+def variative_stream_logits(seed: int, b: int, pieces: List[bytes], phrases: List[bytes], T: int, S: int = 3,
+                            dtype: str = "bf16", n_plants: int = 20) -> np.ndarray:
+    """Logits [T, S, V+1] in storage format for stream ``b`` of a variative-list decode: the same recipe as the
+    token-list workloads (N(0,1) token logits, blank +3), with ``n_plants`` phrases planted as random spellings
+    (casing and segmentation drawn per plant), one piece per frame."""
+    shp = _RowShape(V=len(pieces), S=S, dtype=dtype)
+    rng = np.random.default_rng([seed, 77003, b])
+    x = rng.standard_normal((T, S, shp.V + 1), dtype=np.float32)
+    x[:, :, shp.V] += np.float32(BLANK_BIAS)
+    x = round_to_dtype(x, dtype)
+    if n_plants > 0 and len(phrases) > 0 and T >= n_plants:
+        seg = T // n_plants
+        for i in range(n_plants):
+            toks = random_spelling(rng, phrases[int(rng.integers(0, len(phrases)))], pieces)
+            t0 = i * seg + int(rng.integers(0, max(1, seg - len(toks))))
+            _plant_tokens(x, shp, toks, t0, rng)
+    return to_storage(x, dtype)

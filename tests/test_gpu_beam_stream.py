@@ -10,11 +10,13 @@ from helpers import SCORE_TOL, make_batch, oracle_graph, to_device, to_host
 pytestmark = pytest.mark.gpu
 
 
-def run_beam(tb, w, data, K, phrase_lists=None):
-    """Frame-synchronous driver: E = w.S rows per frame shared by all hypotheses of a stream."""
+def run_beam(tb, w, data, K, phrase_lists=None, batch=None):
+    """Frame-synchronous driver: E = w.S rows per frame shared by all hypotheses of a stream.
+    (batch: one made by the caller, with slot i bound unless phrase_lists[i] is None)"""
     phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
     B, T, E, Wd = data["logits"].shape
-    batch, _ = make_batch(tb, w, phrase_lists, max_beam=K, max_tree_steps=T * E)
+    if batch is None:
+        batch, _ = make_batch(tb, w, phrase_lists, max_beam=K, max_tree_steps=T * E)
     logits = to_device(data["logits"])
     dev = logits.device
     scores = torch.full((B, K), float("-inf"), device=dev)

@@ -88,3 +88,62 @@ def test_compile_error_codes(tb):
     assert code([[0, 1]], 4, flags=1) == tb.TB_ERR_INVALID_ARG
     g = tb.tb_graph_compile([], 4).view()
     assert g["n_states"] == 1 and g["n_arcs"] == 0
+
+
+# ---- variative, case-insensitive compile (Sec. 2.1 para. 4-7, Eq. 1) -------------------------------------
+
+def assert_same_variative_graph(tb, phrases, pieces, weights=None, tau=1.0, lam=1.0):
+    from oracle import variative as var
+    a = var.build(phrases, pieces, weights=weights, tau=tau, lam=lam)
+    gl = tb.tb_graph_compile_variative(phrases, pieces, phrase_weights=weights, tau=tau, lam=lam).view()
+    for k in ("n_states", "n_arcs", "n_classes", "vocab", "max_depth"):
+        assert gl[k] == a[k], k
+    for k in ARRAYS:
+        assert gl[k].dtype == a[k].dtype and gl[k].shape == a[k].shape and gl[k].tobytes() == a[k].tobytes(), k
+    return a
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_variative_compiler_matches_oracle(tb, seed):
+    rng = np.random.default_rng(seed)
+    pieces = W.make_piece_vocab(seed, letters=int(rng.integers(3, 12)), merged=int(rng.integers(0, 80)),
+                                max_len=int(rng.integers(2, 6)))
+    phrases = W.draw_string_phrases(seed, pieces, int(rng.integers(0, 90)), 1, 5)
+    if seed % 2:                                         # user lists in mixed casing, duplicates, an empty phrase
+        phrases = [p.upper() if i % 3 == 0 else p.title() if i % 3 == 1 else p for i, p in enumerate(phrases)]
+        phrases += phrases[:3] + [b""]
+    weights = None if seed % 3 == 0 else [float(rng.uniform(0.0, 2.5)) for _ in phrases]
+    a = assert_same_variative_graph(tb, phrases, pieces, weights, tau=float(rng.uniform(0.0, 3.0)),
+                                    lam=[1.0, 0.5, 2.0][seed % 3])
+    cc, n = tb.tb_piece_classes(pieces)
+    assert np.array_equal(cc, a["case_class"]) and n == a["n_classes"]
+
+
+def test_variative_compiler_on_a_production_sized_list(tb):
+    # 300 phrases over a 1024-piece vocabulary, the size of the per-stream lists of the decode workloads
+    pieces = W.make_piece_vocab(11, letters=26, merged=560, max_len=5)[:1024]
+    phrases = W.draw_string_phrases(11, pieces, 300, 1, 6)
+    a = assert_same_variative_graph(tb, phrases, pieces, tau=1.0)
+    assert a["n_states"] > 1000 and a["n_arcs"] > a["n_states"]          # not a tree: arcs converge
+
+
+def test_variative_compile_error_codes(tb):
+    pieces = [b"a", b"A", b"b", b"ab"]
+
+    def code(*a, **k):
+        with pytest.raises(tb.TbError) as e:
+            tb.tb_graph_compile_variative(*a, **k)
+        return e.value.code
+    assert code([b"abc"], pieces) == tb.TB_ERR_INVALID_ARG                   # 'c' has no piece
+    assert code([b"ab"], pieces, tau=-1.0) == tb.TB_ERR_INVALID_ARG
+    assert code([b"ab"], pieces, tau=float("nan")) == tb.TB_ERR_INVALID_ARG
+    assert code([b"ab"], pieces, lam=float("inf")) == tb.TB_ERR_INVALID_ARG
+    assert code([b"ab"], pieces, phrase_weights=[-1.0]) == tb.TB_ERR_INVALID_ARG
+    assert code([b"a" * 256], pieces) == tb.TB_ERR_INVALID_ARG
+    assert code([b"ab"], pieces + [b""]) == tb.TB_ERR_INVALID_ARG             # an empty piece
+    assert code([b"ab"], pieces + [b"a" * 33]) == tb.TB_ERR_INVALID_ARG       # a piece longer than TB_MAX_PIECE_LEN
+    assert code([b"ab"], pieces, flags=1) == tb.TB_ERR_INVALID_ARG
+    g = tb.tb_graph_compile_variative([], pieces).view()
+    assert g["n_states"] == 1 and g["n_arcs"] == 0
+    g = tb.tb_graph_compile_variative([b"AB"], pieces, tau=0.0).view()      # the hand-worked list, given in upper case
+    assert list(g["arc_class"]) == [0, 2, 1] and list(g["arc_w"]) == [0.5, 1.0, 0.5]
