@@ -156,6 +156,37 @@ def side_measurement(args):
                           "unit": UNIT, "ms_per_step": ms, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
                           "config": {"workload": w.name, "B": w.B, "T": w.T, "states_per_graph": graphs[0].view()["n_states"]},
                           "graph_compile_ms_per_list": compile_ms, "data": "synthetic"}))
+    elif args.workload == 6:
+        # variative, case-insensitive lists (Sec. 2.1, Eq. 1) at workload 2's shape: phrases as text over a synthetic
+        # piece vocabulary, compiled per stream; spellings planted in random casings and segmentations
+        B, T, S = (args.streams or 128), (args.frames or 750), 3
+        pieces = W.make_piece_vocab(6, letters=26, merged=560, max_len=5)
+        lists = [W.draw_string_phrases(6000 + b, pieces, 100, 1, 4) for b in range(B)]
+        x = np.stack([W.variative_stream_logits(6, b, pieces, lists[b], T, S) for b in range(B)])
+        cc, n_cls = tb.tb_piece_classes(pieces)
+        t0 = time.perf_counter()
+        graphs = [tb.tb_graph_compile_variative(p, pieces, tau=1.0) for p in lists]
+        compile_ms = (time.perf_counter() - t0) * 1e3 / B
+        v0 = graphs[0].view()
+        batch = tb.tb_batch_create(len(pieces), cc, B, arena_bytes=(1 << 20) * B + (1 << 20))
+        for i, g in enumerate(graphs):
+            tb.tb_batch_bind_stream(batch, i, g)
+        logits = torch.from_numpy(x).view(torch.bfloat16).to(dev)
+        out = tb.tb_greedy_decode(batch, logits)
+        ms = timed(lambda: tb.tb_greedy_decode(batch, logits, out=out), args.steps, args.warmup)
+        assert tb.tb_batch_status(batch) == 0
+        plain = tb.tb_batch_create(len(pieces), cc, B, arena_bytes=1 << 20)
+        out0 = tb.tb_greedy_decode(plain, logits)
+        ms0 = timed(lambda: tb.tb_greedy_decode(plain, logits, out=out0), args.steps, args.warmup)
+        print(json.dumps({"metric": "boosted_greedy_decode_frames_per_s_variative_lists", "value": B * T / (ms * 1e-3),
+                          "unit": UNIT, "ms_per_step": ms, "unboosted_ms_per_step": ms0, "n_gpus": 1, "steps": args.steps,
+                          "warmup": args.warmup,
+                          "config": {"workload": "variative_greedy_rnnt", "B": B, "T": T, "S": S, "V": len(pieces),
+                                     "classes": n_cls, "phrases_per_stream": 100, "tau": 1.0,
+                                     "states_per_graph": v0["n_states"], "arcs_per_graph": v0["n_arcs"]},
+                          "graph_compile_ms_per_list": compile_ms,
+                          "graph_compile_phrases_per_s": 100.0 / (compile_ms * 1e-3),
+                          "tokens_emitted": int(out["counts"].sum().item()), "data": "synthetic"}))
     elif args.workload == 4:
         w = W.get_workload(4)
         data = W.batch_inputs(w)
@@ -242,8 +273,8 @@ def main():
     ap.add_argument("--streams", type=int, default=0, help="override B (profiling captures use a small case)")
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
-    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5],
-                    help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn: side measurements")
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6],
+                    help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists: side measurements")
     args = ap.parse_args()
     if args.workload != 2:
         side_measurement(args)

@@ -82,6 +82,7 @@ struct tb_batch {
   ArenaAllocator alloc;
   std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
   std::vector<int32_t> slot_cache_bytes;               // bytes of the sections the pipelined kernel caches
+  std::vector<uint8_t> slot_resolved;                  // the bound graph carries resolved per-state lists (1 for an unbound slot)
   std::vector<int32_t> slot_n_states;
   Staging staging[kStagingRing];
   int next_staging = 0;
@@ -127,6 +128,7 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   b->alloc.init(b->arena_bytes);
   b->slot_block.assign(n_slots, {0, 0});
   b->slot_cache_bytes.assign(n_slots, 0);
+  b->slot_resolved.assign(n_slots, 1);
   b->slot_n_states.assign(n_slots, 0);
   bool ok = true;
   ok = ok && cudaMalloc(&b->arena, b->arena_bytes) == cudaSuccess;
@@ -206,6 +208,7 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
   b->slot_n_states[slot] = g ? g->n_states : 0;
   // what the pipelined kernel caches in shared memory: the resolved lists, else the state records + token arcs
   b->slot_cache_bytes[slot] = !g ? 0 : static_cast<int32_t>(g->blob.size()) - (g->n_rsent >= 0 ? g->off_rsrec : g->off_strec);
+  b->slot_resolved[slot] = (!g || g->n_rsent >= 0) ? 1 : 0;
   return TB_OK;
 }
 
@@ -251,10 +254,11 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   if (!(b->flags & TB_FLAG_GENERAL_KERNELS)) {
-    int32_t max_cache = 0, max_states = 0;
+    int32_t max_cache = 0, max_states = 0, all_resolved = 1;
     for (int32_t i = 0; i < B; ++i) {
       max_cache = b->slot_cache_bytes[i] > max_cache ? b->slot_cache_bytes[i] : max_cache;
       max_states = b->slot_n_states[i] > max_states ? b->slot_n_states[i] : max_states;
+      if (!b->slot_resolved[i]) all_resolved = 0;
     }
     // the two-segment decode keeps what its second segment produces in scratch memory of the batch; growing it
     // frees the old block first (cudaFree waits for earlier work), so one decode per batch at a time
@@ -269,7 +273,7 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
       if (cudaMalloc(&b->seg_scratch, want) == cudaSuccess) b->seg_scratch_bytes = want;
       else cudaGetLastError();
     }
-    rc = tb_launch_greedy_fast(p, max_cache, max_states, b->seg_scratch, b->seg_scratch_bytes,
+    rc = tb_launch_greedy_fast(p, max_cache, max_states, all_resolved, b->seg_scratch, b->seg_scratch_bytes,
                                static_cast<cudaStream_t>(stream_));
     if (rc != 1) return rc;
   }

@@ -191,7 +191,7 @@ struct Smem {  // byte offsets into dynamic shared memory, computed identically 
   int lbuf_sz, cls_seen_sz, tokidx_sz;   // the deciders' private areas exist once per segment, this far apart
 };
 __host__ __device__ inline int up16(int x) { return (x + 15) & ~15; }
-__host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes, int npipes) {
+__host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int cache_bytes, int npipes, int own_lists) {
   Smem s;
   int o = 0;
   s.ring = o; o += nst * slot_bytes;
@@ -201,7 +201,8 @@ __host__ __device__ inline Smem carve(int nst, int slot_bytes, int V, int C, int
   s.tokcb = o; o += up16(4 * V);            // lambda * root-arc weight of every token (0 without a root arc)
   s.rootcw = o; o += up16(4 * C);
   s.rootdst = o; o += up16(4 * C);
-  s.lbuf_sz = up16(8 * (V + 4)); s.cls_seen_sz = up16(2 * C); s.tokidx_sz = up16(2 * V);
+  // own_lists == 0: every bound graph's resolved lists are in the cache, no decider ever builds or stages a list
+  s.lbuf_sz = own_lists ? up16(8 * (V + 4)) : 16; s.cls_seen_sz = own_lists ? up16(2 * C) : 0; s.tokidx_sz = up16(2 * V);
   s.lbuf = o; o += npipes * s.lbuf_sz;         // boosted-token list of the current state when it is not read from the cache
   s.cls_seen = o; o += npipes * s.cls_seen_sz; // class -> position in lbuf while a list is being built
   s.tokidx = o; o += npipes * s.tokidx_sz;     // token -> position in the current list (filled only for an exact rescan)
@@ -219,6 +220,7 @@ struct FastParams {
   const unsigned char* tensor_hi;
   // two-segment decode: per stream, what the second segment emits / adds to the score / its state at every frame start
   int32_t npipes;                        // 2: long bound streams are decoded as two segments
+  int32_t own_lists;                     // 0: no graph of the batch needs a list built or staged outside the cache
   int32_t scr_cap;                       // frames * S
   int32_t* scr_tok;                      // [n_streams][2 * scr_cap]: tokens, then frames
   float* scr_val;                        // [n_streams][scr_cap]: value of every row the segment visits, in order
@@ -473,7 +475,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
 #endif
   const TbDecodeParams& p = P.d;
   const int V = p.V, C = p.C, S = p.S, W = V + 1, nst = P.nst;
-  const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes, P.npipes);
+  const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes, P.npipes, P.own_lists);
   unsigned char* ring = dyn + so.ring;
   uint64_t* full = reinterpret_cast<uint64_t*>(dyn + so.bars);
   uint64_t* freeb = full + nst;
@@ -498,6 +500,14 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
 
   int end = p.lengths ? p.lengths[b] : p.frames;
   end = max(0, min(end, p.frames));
+  if (bound && !P.own_lists && !(resolved && cached)) {      // the launch was laid out without room for this graph's lists
+    if (tid == 0) {
+      atomicOr(p.status, TB_STATUS_BAD_STATE);
+      p.out_counts[b] = 0; p.out_scores[b] = 0.0f; p.out_states[b] = 0;
+      if (p.out_cursors) p.out_cursors[b] = 0;
+    }
+    return;
+  }
 
   // ---- set-up: tables, root vectors, graph cache, barriers ----------------------------------------
   for (int v = tid; v < V; v += kThreadsF) {
@@ -507,8 +517,10 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   }
   for (int c = tid; c < C; c += kThreadsF) {
     rootcb[c] = 0.0f; rootcw[c] = 0.0f; rootdst[c] = 0;
-    reinterpret_cast<int16_t*>(dyn + so.cls_seen)[c] = -1;
-    if (P.npipes == 2) reinterpret_cast<int16_t*>(dyn + so.cls_seen + so.cls_seen_sz)[c] = -1;
+    if (P.own_lists) {
+      reinterpret_cast<int16_t*>(dyn + so.cls_seen)[c] = -1;
+      if (P.npipes == 2) reinterpret_cast<int16_t*>(dyn + so.cls_seen + so.cls_seen_sz)[c] = -1;
+    }
   }
   for (int i = tid; i < nst * kSumStageBytes / 4; i += kThreadsF) reinterpret_cast<uint32_t*>(dyn + so.summ)[i] = 0u;   // no sequence word matches yet
   if (tid == 0) {
@@ -697,7 +709,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     L.addr = smem_u32(lbuf); L.n = 0; L.sorted = true; L.D = 0.0f; L.bmag = fabsf(lam) * R;
 
     const int q = lane >> 2, ql = lane & 3;                 // group and lane within the group
-    constexpr int kWin = 8;                                 // frames per window (the launcher guarantees nst > kWin)
+    constexpr int kWin = 8;                                 // frames per window (the launcher guarantees nst >= kWin)
     int t = pf0, k = 0, s = bound ? 0 : -1, n_out = 0, st = 0, lead = (lead0 + pf0 * lead_step) & 15;
     float score = 0.0f;
     // pipeline 1 writes to scratch memory and keeps a log: rec_on
@@ -1424,8 +1436,8 @@ size_t tb_greedy_fast_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S
 
 // Returns TB_OK if the launch was made, 1 if this path does not cover the call (the caller then
 // uses the general kernel), or an error code.
-int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int32_t max_states, void* scratch,
-                          size_t scratch_bytes, cudaStream_t stream) {
+int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int32_t max_states, int32_t all_resolved,
+                          void* scratch, size_t scratch_bytes, cudaStream_t stream) {
   const int W = d.V + 1;
   if (d.dtype != TB_BF16 || d.persistent || d.n_dur != 0) return 1;
   if (d.sv != 1 || d.ss != W || d.st < static_cast<int64_t>(d.S) * W || d.sb < 0) return 1;
@@ -1446,33 +1458,40 @@ int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int3
     return TB_ERR_CUDA;
   }
   const int budget = max_smem - 1024;
-  P.cache_bytes = (max_cache_bytes > 0 && max_cache_bytes <= 48 * 1024) ? max_cache_bytes : 0;
   const int per_stage = P.slot_bytes + 16 + kSumStageBytes;
-  // two segments per stream when the scratch memory is there and both halves of the ring can hold a window
+  const bool seg_ok = d.frames >= kSegMinFrames && scratch && (reinterpret_cast<uintptr_t>(scratch) & 15) == 0 &&
+                      scratch_layout(d.n_streams, d.frames, d.S).total <= scratch_bytes;
+  // Layouts in order of preference: the graphs' lists cached in shared memory with two segments per stream (each
+  // half of the ring at least eight stages, the decider's window), cached with one segment, then not cached (lists read from the arena),
+  // again with two segments or one.
+  // A cache beyond 48 KB is only taken when no decider needs room to build or stage lists of its own.
   P.npipes = 1; P.scr_cap = 0; P.scr_tok = nullptr; P.scr_val = nullptr; P.scr_trace = nullptr;
   int nst = 0;
-  if (d.frames >= kSegMinFrames && scratch && (reinterpret_cast<uintptr_t>(scratch) & 15) == 0) {
-    const ScratchLayout l = scratch_layout(d.n_streams, d.frames, d.S);
-    const int fixed2 = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes, 2).total;
-    int nst2 = (budget - fixed2 - 64) / per_stage;
-    if (nst2 > kStagesMax) nst2 = kStagesMax;
-    if (l.total <= scratch_bytes && nst2 >= 18) {
-      P.npipes = 2; nst = nst2;
-      unsigned char* sb = static_cast<unsigned char*>(scratch);
-      P.scr_cap = d.frames * d.S;
-      P.scr_tok = reinterpret_cast<int32_t*>(sb + l.tok);
-      P.scr_val = reinterpret_cast<float*>(sb + l.val);
-      P.scr_trace = reinterpret_cast<int4*>(sb + l.trace);
-    }
+  for (int attempt = 0; attempt < 4 && nst == 0; ++attempt) {
+    const bool want_cache = attempt < 2, want_seg = (attempt & 1) == 0;
+    if (want_cache && !(max_cache_bytes > 0 && (max_cache_bytes <= 48 * 1024 || (all_resolved && max_cache_bytes <= 112 * 1024)))) continue;
+    if (want_seg && !seg_ok) continue;
+    P.cache_bytes = want_cache ? max_cache_bytes : 0;
+    P.own_lists = (all_resolved && (P.cache_bytes > 0 || max_states == 0)) ? 0 : 1;
+    const int np = want_seg ? 2 : 1;
+    const int fixed = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes, np, P.own_lists).total;
+    int n = (budget - fixed - 64) / per_stage;
+    if (n > kStagesMax) n = kStagesMax;
+    if (n < (np == 2 ? 16 : 9)) continue;     // a pipeline's part of the ring holds at least the decider's window
+    nst = n; P.npipes = np;
   }
-  if (P.npipes == 1) {
-    const int fixed = carve(0, P.slot_bytes, d.V, d.C, P.cache_bytes, 1).total;
-    nst = (budget - fixed - 64) / per_stage;
-    if (nst > kStagesMax) nst = kStagesMax;
+  if (nst == 0) return 1;
+  if (P.npipes == 2) {
+    const ScratchLayout l = scratch_layout(d.n_streams, d.frames, d.S);
+    unsigned char* sb = static_cast<unsigned char*>(scratch);
+    P.scr_cap = d.frames * d.S;
+    P.scr_tok = reinterpret_cast<int32_t*>(sb + l.tok);
+    P.scr_val = reinterpret_cast<float*>(sb + l.val);
+    P.scr_trace = reinterpret_cast<int4*>(sb + l.trace);
   }
   if (nst < 9) return 1;   // the decider's window spans eight stages
   P.nst = nst;
-  const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes, P.npipes);
+  const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes, P.npipes, P.own_lists);
   if (so.total > budget) return 1;
   const int nit = (d.V + 255) / 256;
   void (*fn)(FastParams) = nit <= 1 ? k_greedy_fast<1> : nit <= 2 ? k_greedy_fast<2> : nit <= 4 ? k_greedy_fast<4> : k_greedy_fast<8>;

@@ -36,11 +36,12 @@ struct TbBeamParams {
 int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
 // Returns TB_OK when it launched, 1 when the call is outside what the pipelined kernel covers.
 // max_cache_bytes: the largest cacheable list section among the slots decoded; max_states: their largest state count.
+// all_resolved: non-zero when every bound graph among them carries resolved per-state lists.
 // scratch / scratch_bytes: device memory for the two-segment decode (tb_greedy_fast_scratch_bytes says how
 // much a call needs); with less than that the kernel decodes every stream as one segment.
 size_t tb_greedy_fast_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S);
-int tb_launch_greedy_fast(const TbDecodeParams& p, int32_t max_cache_bytes, int32_t max_states, void* scratch,
-                          size_t scratch_bytes, cudaStream_t stream);
+int tb_launch_greedy_fast(const TbDecodeParams& p, int32_t max_cache_bytes, int32_t max_states, int32_t all_resolved,
+                          void* scratch, size_t scratch_bytes, cudaStream_t stream);
 int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
