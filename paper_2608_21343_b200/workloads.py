@@ -361,6 +361,7 @@ def make_piece_vocab(seed: int, letters: int = 12, merged: int = 200, max_len: i
         out.append(bytes([97 + i]))
         out.append(bytes([65 + i]))
     seen = set()
+    merged = min(merged, sum(letters ** n for n in range(2, max_len + 1)))   # no more than there are
     while len(seen) < merged:
         n = int(rng.integers(2, max_len + 1))
         seen.add(bytes(int(x) + 97 for x in rng.integers(0, letters, size=n)))

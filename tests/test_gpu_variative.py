@@ -82,3 +82,18 @@ def test_beam_decode_with_variative_graphs(tb):
             assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
         fin = np.isfinite(ref["scores"])
         assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
+
+
+@pytest.mark.parametrize("n_phrases,letters,merged", [(400, 26, 560), (30, 8, 40), (200, 12, 300)])
+def test_greedy_decode_variative_list_sizes(tb, n_phrases, letters, merged):
+    # from lists whose resolved per-state lists fit the kernel's shared-memory cache with room to spare, over
+    # ones that take most of it (shorter ring), to lists read from the arena
+    pieces = W.make_piece_vocab(21, letters=letters, merged=merged, max_len=4)
+    B, T, S = 4, 260, 3
+    lists = [W.draw_string_phrases(700 + b, pieces, n_phrases, 1, 5) for b in range(B)]
+    x = np.stack([W.variative_stream_logits(21, b, pieces, lists[b], T, S, n_plants=15) for b in range(B)])
+    batch = make_variative_batch(tb, pieces, lists, tau=1.5)
+    out = to_host(tb.tb_greedy_decode(batch, to_device(x)))
+    assert tb.tb_batch_status(batch) == 0
+    for b, g in enumerate(oracle_graphs(pieces, lists, 1.5)):
+        check_greedy(out, b, O.greedy_rnnt(g, x[b]), f"variative {n_phrases} phrases")
