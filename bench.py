@@ -35,7 +35,7 @@ UNIT = "frames/s"
 # DRAM read + write bytes per logits row of the decode kernel, from an ncu capture of a 32-stream launch
 # (160.2 MB for 72000 rows: each stream's second segment re-reads 16 warm-up frames, and what it emits goes
 # through scratch memory); the kernel runs one block per stream, so traffic scales with the stream count.
-NCU_DRAM_BYTES_PER_ROW = 2225.0
+NCU_DRAM_BYTES_PER_ROW = 2233.0
 
 
 def load_peaks():
