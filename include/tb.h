@@ -44,6 +44,7 @@ extern "C" {
 #define TB_ERR_ARENA_FULL (-4)    /* the graph does not fit into the arena's free space */
 #define TB_ERR_BAD_SLOT (-5)      /* slot index outside the batch */
 #define TB_ERR_DEVICE_STATUS (-6) /* a kernel recorded a violated bound (see tb_batch_status) */
+#define TB_ERR_IO (-7)            /* a file could not be opened, read or written */
 
 #define TB_BF16 0 /* logits are bfloat16 */
 #define TB_F32 1  /* logits are float32 */
@@ -66,6 +67,7 @@ extern "C" {
 
 typedef struct tb_graph tb_graph; /* immutable compiled graph, host memory */
 typedef struct tb_batch tb_batch; /* device arena + slot table + per-slot state */
+typedef struct tb_cache tb_cache; /* compiled graphs kept in host memory, by the content of their lists */
 
 /*
  * Read-only view of a compiled graph as flat arrays in host memory: the arc arrays (label =
@@ -164,6 +166,38 @@ int tb_graph_view_get(const tb_graph *g, tb_graph_view *out);
 void tb_graph_free(tb_graph *g);
 
 /*
+ * The host levels of the three-level cache of Sec. 2.2 para. 5 (the cost that remains with per-stream lists is
+ * compiling and transferring the models when streams are created).
+ *
+ * Disk: tb_graph_save writes a compiled graph (its arrays and its device blob) to `path`; tb_graph_load
+ * reads one back, identical in every array to the graph that was saved.  A file that is not such a file,
+ * was cut short or altered (magic, version, sizes, a checksum over the contents, the class map) is refused
+ * with TB_ERR_INVALID_ARG; a file that cannot be opened, read or written gives TB_ERR_IO.  Files are only
+ * meant for the machine and build that wrote them (native byte order, this build's blob layout).
+ */
+int tb_graph_save(const tb_graph *g, const char *path);
+int tb_graph_load(const char *path, tb_graph **out);
+
+/*
+ * Memory: a cache of compiled graphs in host memory, keyed by the content of everything the compiler
+ * reads (tokens, offsets, weights, class map, vocab, lambda, flags).  tb_cache_compile returns the graph
+ * tb_graph_compile would return for the same arguments -- from the cache when the same list was compiled
+ * through this cache before (*out_hit = 1), otherwise by compiling it and keeping it (least recently used
+ * graphs are dropped once `capacity_bytes` of host memory would be exceeded; a graph larger than that is
+ * returned but not kept).  The returned graph is the caller's to release with tb_graph_free as usual; it
+ * stays valid after the cache drops or is destroyed.  Calls on one cache may come from several threads.
+ *   out_hit  host int32 or NULL.   Errors: as tb_graph_compile.
+ * tb_cache_stats: any pointer may be NULL.
+ */
+int tb_cache_create(size_t capacity_bytes, tb_cache **out);
+void tb_cache_destroy(tb_cache *c);
+int tb_cache_compile(tb_cache *c, const int32_t *phrase_tokens, const int64_t *phrase_offsets, int32_t n_phrases,
+                     const float *token_weights, const int32_t *case_class, int32_t vocab, float lambda,
+                     uint32_t flags, tb_graph **out, int32_t *out_hit);
+int tb_cache_stats(tb_cache *c, int64_t *hits, int64_t *misses, int64_t *evictions, size_t *bytes_used,
+                   int64_t *entries);
+
+/*
  * Create a batch on `device`: the merged multi-model storage of Sec. 2.2 para. 2 (one arena
  * holding every bound graph's arrays behind a per-slot offset table), plus per-slot decode
  * state.  All slots start unbound (model id -1).
@@ -192,6 +226,23 @@ void tb_batch_destroy(tb_batch *b);
  * TB_ERR_ARENA_FULL (nothing was changed), TB_ERR_CUDA.
  */
 int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *stream);
+
+/*
+ * Decoder-level registration (Sec. 2.2 para. 5: models known before a recognition session are registered with
+ * the decoder, which takes the update cost out of the decoding loop).  tb_batch_register_model copies the
+ * graph into the arena once (asynchronously on `stream`, like a bind) and returns a model id >= 0;
+ * tb_batch_bind_model then points a slot at that model: no compile, no copy, no allocation -- one small
+ * kernel that writes the slot's record and resets its streaming state, ordered on `stream`.  Any number of
+ * slots may be bound to one model; model id -1 unbinds the slot (as tb_batch_bind_stream with NULL).  A slot
+ * bound either way can be re-bound either way.  tb_batch_unregister_model gives the model's arena block back;
+ * it fails with TB_ERR_INVALID_ARG while a slot is still bound to the model.  The caller orders it after the
+ * decode calls that may still read the model, as for re-binding a slot.
+ * Errors: TB_ERR_INVALID_ARG (NULL, a graph for another vocabulary or class map, an id that is not
+ * registered), TB_ERR_BAD_SLOT, TB_ERR_ARENA_FULL, TB_ERR_OOM, TB_ERR_CUDA.
+ */
+int tb_batch_register_model(tb_batch *b, const tb_graph *g, int32_t *out_model_id, void *stream);
+int tb_batch_bind_model(tb_batch *b, int32_t slot, int32_t model_id, void *stream);
+int tb_batch_unregister_model(tb_batch *b, int32_t model_id);
 
 /*
  * Set behaviour flags of the batch (TB_FLAG_*; 0 = defaults).  With the defaults

@@ -22,6 +22,7 @@ _lib = C.CDLL(LIB_PATH)
 
 TB_OK = 0
 TB_ERR_INVALID_ARG, TB_ERR_OOM, TB_ERR_CUDA, TB_ERR_ARENA_FULL, TB_ERR_BAD_SLOT, TB_ERR_DEVICE_STATUS = -1, -2, -3, -4, -5, -6
+TB_ERR_IO = -7
 TB_BF16, TB_F32 = 0, 1
 
 
@@ -52,6 +53,17 @@ _SIGS = {
                                              C.POINTER(_vp)]),
     "tb_graph_view_get": (C.c_int, [_vp, C.POINTER(_GraphView)]),
     "tb_graph_free": (None, [_vp]),
+    "tb_graph_save": (C.c_int, [_vp, C.c_char_p]),
+    "tb_graph_load": (C.c_int, [C.c_char_p, C.POINTER(_vp)]),
+    "tb_cache_create": (C.c_int, [C.c_size_t, C.POINTER(_vp)]),
+    "tb_cache_destroy": (None, [_vp]),
+    "tb_cache_compile": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, C.c_float, C.c_uint32, C.POINTER(_vp),
+                                   C.POINTER(_i32)]),
+    "tb_cache_stats": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(C.c_size_t),
+                                 C.POINTER(_i64)]),
+    "tb_batch_register_model": (C.c_int, [_vp, _vp, C.POINTER(_i32), _vp]),
+    "tb_batch_bind_model": (C.c_int, [_vp, _i32, _i32, _vp]),
+    "tb_batch_unregister_model": (C.c_int, [_vp, _i32]),
     "tb_batch_create": (C.c_int, [_i32, _vp, _i32, _i32, _i32, C.c_size_t, C.c_int, C.POINTER(_vp)]),
     "tb_batch_destroy": (None, [_vp]),
     "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
@@ -161,6 +173,83 @@ def tb_graph_compile(phrases, vocab: int, case_class=None, token_weights=None, l
     _check(_lib.tb_graph_compile(_hp(toks), _hp(offs), n, _hp(w), _hp(cc), vocab, float(lam), flags, C.byref(h)),
            "tb_graph_compile")
     return Graph(h)
+
+
+def _flatten_phrases(phrases, token_weights):
+    if isinstance(phrases, tuple):
+        toks, offs = _host(phrases[0], np.int32), _host(phrases[1], np.int64)
+        return toks, offs, len(offs) - 1, _host(token_weights, np.float32)
+    n = len(phrases)
+    offs = np.zeros(n + 1, dtype=np.int64)
+    if n:
+        offs[1:] = np.cumsum([len(p) for p in phrases])
+    toks = np.array([t for p in phrases for t in p], dtype=np.int32)
+    w = None if token_weights is None else np.array([x for p in token_weights for x in p], dtype=np.float32)
+    return toks, offs, n, w
+
+
+def tb_graph_save(graph: Graph, path: str):
+    _check(_lib.tb_graph_save(graph.handle, os.fsencode(path)), "tb_graph_save")
+
+
+def tb_graph_load(path: str) -> Graph:
+    h = _vp()
+    _check(_lib.tb_graph_load(os.fsencode(path), C.byref(h)), "tb_graph_load")
+    return Graph(h)
+
+
+class Cache:
+    """Compiled graphs kept in host memory (tb_cache)."""
+
+    def __init__(self, handle):
+        self.handle = handle
+
+    def stats(self) -> dict:
+        h, m, e, n = _i64(), _i64(), _i64(), _i64()
+        used = C.c_size_t()
+        _check(_lib.tb_cache_stats(self.handle, C.byref(h), C.byref(m), C.byref(e), C.byref(used), C.byref(n)),
+               "tb_cache_stats")
+        return dict(hits=h.value, misses=m.value, evictions=e.value, bytes_used=used.value, entries=n.value)
+
+    def destroy(self):
+        if self.handle and _lib is not None:
+            _lib.tb_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.destroy()
+
+
+def tb_cache_create(capacity_bytes: int) -> Cache:
+    h = _vp()
+    _check(_lib.tb_cache_create(capacity_bytes, C.byref(h)), "tb_cache_create")
+    return Cache(h)
+
+
+def tb_cache_compile(cache: Cache, phrases, vocab: int, case_class=None, token_weights=None, lam: float = 1.0,
+                     flags: int = 0):
+    """Returns (graph, hit)."""
+    toks, offs, n, w = _flatten_phrases(phrases, token_weights)
+    cc = _host(case_class, np.int32)
+    h, hit = _vp(), _i32()
+    _check(_lib.tb_cache_compile(cache.handle, _hp(toks), _hp(offs), n, _hp(w), _hp(cc), vocab, float(lam), flags,
+                                 C.byref(h), C.byref(hit)), "tb_cache_compile")
+    return Graph(h), bool(hit.value)
+
+
+def tb_batch_register_model(batch, graph: Graph, stream=None) -> int:
+    mid = _i32()
+    _check(_lib.tb_batch_register_model(batch.handle, graph.handle, C.byref(mid), _stream(stream)),
+           "tb_batch_register_model")
+    return mid.value
+
+
+def tb_batch_bind_model(batch, slot: int, model_id: int, stream=None):
+    _check(_lib.tb_batch_bind_model(batch.handle, slot, model_id, _stream(stream)), "tb_batch_bind_model")
+
+
+def tb_batch_unregister_model(batch, model_id: int):
+    _check(_lib.tb_batch_unregister_model(batch.handle, model_id), "tb_batch_unregister_model")
 
 
 def _flat_bytes(items):

@@ -84,6 +84,17 @@ struct tb_batch {
   std::vector<int32_t> slot_cache_bytes;               // bytes of the sections the pipelined kernel caches
   std::vector<uint8_t> slot_resolved;                  // the bound graph carries resolved per-state lists (1 for an unbound slot)
   std::vector<int32_t> slot_n_states;
+  // models registered ahead of a session (Sec. 2.2 para. 5, decoder-level registration): uploaded once, bound to
+  // slots by id without a copy
+  struct Model {
+    bool live = false;
+    size_t off = 0, bytes = 0;
+    TbSlotRec rec;
+    int32_t n_states = 0, cache_bytes = 0, users = 0;
+    uint8_t resolved = 1;
+  };
+  std::vector<Model> models;
+  std::vector<int32_t> slot_model;                     // registered model a slot is bound to, else -1
   Staging staging[kStagingRing];
   int next_staging = 0;
   void* seg_scratch = nullptr;      // working memory of the two-segment greedy decode (grown on demand)
@@ -130,6 +141,7 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   b->slot_cache_bytes.assign(n_slots, 0);
   b->slot_resolved.assign(n_slots, 1);
   b->slot_n_states.assign(n_slots, 0);
+  b->slot_model.assign(n_slots, -1);
   bool ok = true;
   ok = ok && cudaMalloc(&b->arena, b->arena_bytes) == cudaSuccess;
   ok = ok && cudaMalloc(&b->d_slots, sizeof(TbSlotRec) * n_slots) == cudaSuccess;
@@ -158,6 +170,62 @@ extern "C" void tb_batch_destroy(tb_batch* b) {
   destroy_batch(b);
 }
 
+// Copies a graph's blob into a fresh arena block (through the pinned staging ring, on `stream`) and fills the
+// slot record that points at it.
+static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, size_t* off_out, size_t* bytes_out,
+                        TbSlotRec* rec_out) {
+  if (g->vocab != b->vocab || g->class_map_hash != b->class_map_hash) return TB_ERR_INVALID_ARG;
+  size_t off = 0;
+  const size_t bytes = round_up(g->blob.size(), kArenaAlign);
+  if (!b->alloc.alloc(bytes, &off)) return TB_ERR_ARENA_FULL;
+  // pinned staging: wait only if this ring entry's previous copy has not finished yet
+  Staging& s = b->staging[b->next_staging];
+  b->next_staging = (b->next_staging + 1) % kStagingRing;
+  bool ok = true;
+  if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
+  if (ok && s.cap < g->blob.size()) {
+    if (s.host) cudaFreeHost(s.host);
+    s.host = nullptr; s.cap = 0;
+    size_t want = round_up(g->blob.size() * 2, 1 << 16);
+    ok = cudaMallocHost(&s.host, want) == cudaSuccess;
+    if (ok) s.cap = want;
+  }
+  if (ok) {
+    std::memcpy(s.host, g->blob.data(), g->blob.size());
+    ok = cudaMemcpyAsync(b->arena + off, s.host, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;
+    s.pending = ok;
+  }
+  if (!ok) { cudaGetLastError(); b->alloc.release(off, bytes); return TB_ERR_CUDA; }
+  TbSlotRec& rec = *rec_out;
+  std::memset(&rec, 0, sizeof rec);
+  rec.blob_off = static_cast<int64_t>(off);
+  rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
+  rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
+  rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
+  rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
+  rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
+  rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
+  *off_out = off; *bytes_out = bytes;
+  return TB_OK;
+}
+
+// what the pipelined kernel caches in shared memory: the resolved lists, else the state records + token arcs
+static int32_t cache_bytes_of(const tb_graph* g) {
+  return static_cast<int32_t>(g->blob.size()) - (g->n_rsent >= 0 ? g->off_rsrec : g->off_strec);
+}
+
+// The slot lets go of what it was bound to: its own block goes back to the free list (anything that reuses it is
+// enqueued on the same stream after the decode calls that still read it), a registered model loses a user.
+static void release_slot(tb_batch* b, int32_t slot) {
+  auto& blk = b->slot_block[slot];
+  if (blk.second) b->alloc.release(blk.first, blk.second);
+  blk = {0, 0};
+  const int32_t m = b->slot_model[slot];
+  if (m >= 0) b->models[m].users--;
+  b->slot_model[slot] = -1;
+}
+
 extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g, void* stream_) {
   if (!b) return TB_ERR_INVALID_ARG;
   if (slot < 0 || slot >= b->n_slots) return TB_ERR_BAD_SLOT;
@@ -168,47 +236,73 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
   std::memset(&rec, 0, sizeof rec);
   size_t off = 0, bytes = 0;
   if (g) {
-    if (g->vocab != b->vocab || g->class_map_hash != b->class_map_hash) return TB_ERR_INVALID_ARG;
-    bytes = round_up(g->blob.size(), kArenaAlign);
-    if (!b->alloc.alloc(bytes, &off)) return TB_ERR_ARENA_FULL;
-    // pinned staging: wait only if this ring entry's previous copy has not finished yet
-    Staging& s = b->staging[b->next_staging];
-    b->next_staging = (b->next_staging + 1) % kStagingRing;
-    bool ok = true;
-    if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
-    if (ok && s.cap < g->blob.size()) {
-      if (s.host) cudaFreeHost(s.host);
-      s.host = nullptr; s.cap = 0;
-      size_t want = round_up(g->blob.size() * 2, 1 << 16);
-      ok = cudaMallocHost(&s.host, want) == cudaSuccess;
-      if (ok) s.cap = want;
-    }
-    if (ok) {
-      std::memcpy(s.host, g->blob.data(), g->blob.size());
-      ok = cudaMemcpyAsync(b->arena + off, s.host, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
-      ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;
-      s.pending = ok;
-    }
-    if (!ok) { cudaGetLastError(); b->alloc.release(off, bytes); return TB_ERR_CUDA; }
-    rec.blob_off = static_cast<int64_t>(off);
-    rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
-    rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
-    rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
-    rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
-    rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
-    rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
+    int rc = upload_graph(b, g, stream, &off, &bytes, &rec);
+    if (rc != TB_OK) return rc;
   }
   int rc = tb_launch_publish_slot(b->d_slots, b->d_sstate, slot, rec, stream);
   if (rc != TB_OK) { if (bytes) b->alloc.release(off, bytes); return rc; }
-  // The old block goes back to the free list now; anything that reuses it is enqueued on the
-  // same stream after the decode calls that still read it.
-  auto& blk = b->slot_block[slot];
-  if (blk.second) b->alloc.release(blk.first, blk.second);
-  blk = {off, bytes};
+  release_slot(b, slot);
+  b->slot_block[slot] = {off, bytes};
   b->slot_n_states[slot] = g ? g->n_states : 0;
-  // what the pipelined kernel caches in shared memory: the resolved lists, else the state records + token arcs
-  b->slot_cache_bytes[slot] = !g ? 0 : static_cast<int32_t>(g->blob.size()) - (g->n_rsent >= 0 ? g->off_rsrec : g->off_strec);
+  b->slot_cache_bytes[slot] = !g ? 0 : cache_bytes_of(g);
   b->slot_resolved[slot] = (!g || g->n_rsent >= 0) ? 1 : 0;
+  return TB_OK;
+}
+
+extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* out_model_id, void* stream_) {
+  if (!b || !g || !out_model_id) return TB_ERR_INVALID_ARG;
+  *out_model_id = -1;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  tb_batch::Model m;
+  int rc = upload_graph(b, g, static_cast<cudaStream_t>(stream_), &m.off, &m.bytes, &m.rec);
+  if (rc != TB_OK) return rc;
+  m.live = true; m.n_states = g->n_states; m.cache_bytes = cache_bytes_of(g); m.resolved = g->n_rsent >= 0 ? 1 : 0;
+  int32_t id = -1;
+  for (size_t i = 0; i < b->models.size(); ++i)
+    if (!b->models[i].live) { id = static_cast<int32_t>(i); break; }
+  try {
+    if (id < 0) { b->models.emplace_back(); id = static_cast<int32_t>(b->models.size()) - 1; }
+  } catch (const std::bad_alloc&) {
+    b->alloc.release(m.off, m.bytes);
+    return TB_ERR_OOM;
+  }
+  b->models[id] = m;
+  *out_model_id = id;
+  return TB_OK;
+}
+
+extern "C" int tb_batch_bind_model(tb_batch* b, int32_t slot, int32_t model_id, void* stream_) {
+  if (!b) return TB_ERR_INVALID_ARG;
+  if (slot < 0 || slot >= b->n_slots) return TB_ERR_BAD_SLOT;
+  if (model_id < -1 || model_id >= static_cast<int32_t>(b->models.size()) || (model_id >= 0 && !b->models[model_id].live))
+    return TB_ERR_INVALID_ARG;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  TbSlotRec rec;
+  std::memset(&rec, 0, sizeof rec);
+  if (model_id >= 0) rec = b->models[model_id].rec;
+  int rc = tb_launch_publish_slot(b->d_slots, b->d_sstate, slot, rec, static_cast<cudaStream_t>(stream_));
+  if (rc != TB_OK) return rc;
+  release_slot(b, slot);
+  if (model_id >= 0) {
+    const tb_batch::Model& m = b->models[model_id];
+    b->models[model_id].users++;
+    b->slot_model[slot] = model_id;
+    b->slot_n_states[slot] = m.n_states; b->slot_cache_bytes[slot] = m.cache_bytes; b->slot_resolved[slot] = m.resolved;
+  } else {
+    b->slot_n_states[slot] = 0; b->slot_cache_bytes[slot] = 0; b->slot_resolved[slot] = 1;
+  }
+  return TB_OK;
+}
+
+extern "C" int tb_batch_unregister_model(tb_batch* b, int32_t model_id) {
+  if (!b || model_id < 0 || model_id >= static_cast<int32_t>(b->models.size()) || !b->models[model_id].live)
+    return TB_ERR_INVALID_ARG;
+  tb_batch::Model& m = b->models[model_id];
+  if (m.users > 0) return TB_ERR_INVALID_ARG;          // still bound to a slot
+  b->alloc.release(m.off, m.bytes);
+  m = tb_batch::Model();
   return TB_OK;
 }
 

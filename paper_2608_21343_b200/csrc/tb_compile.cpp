@@ -53,6 +53,7 @@ extern "C" const char* tb_strerror(int code) {
     case TB_ERR_ARENA_FULL: return "graph arena full";
     case TB_ERR_BAD_SLOT: return "slot index out of range";
     case TB_ERR_DEVICE_STATUS: return "a kernel recorded a violated bound";
+    case TB_ERR_IO: return "file could not be opened, read or written";
     default: return "unknown error";
   }
 }
@@ -555,4 +556,6 @@ extern "C" int tb_graph_view_get(const tb_graph* g, tb_graph_view* out) {
   return TB_OK;
 }
 
-extern "C" void tb_graph_free(tb_graph* g) { delete g; }
+extern "C" void tb_graph_free(tb_graph* g) {
+  if (g && g->refs.fetch_sub(1) == 1) delete g;   // a cache may still hold the graph
+}

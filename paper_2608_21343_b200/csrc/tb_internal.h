@@ -2,6 +2,7 @@
 #ifndef TB_INTERNAL_H_
 #define TB_INTERNAL_H_
 
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 #include <vector>
@@ -23,6 +24,7 @@ struct tb_graph {
   int32_t off_strec = 0, off_tokent = 0, n_tokent = 0;
   int32_t off_rsrec = 0, off_rsent = 0, n_rsent = 0;  // resolved per-state lists (n_rsent < 0: not built)
   float d_max = 0.0f;                                  // largest |sum of suffix-link weights| over all states
+  std::atomic<int32_t> refs{1};                        // holders: the caller's handle, plus one per cache that keeps the graph
 };
 
 // Two derived sections of the blob serve the pipelined kernel.  TbStateRec packs what a

@@ -1,0 +1,123 @@
+"""GPU checks of the model lifecycle (Sec. 2.2 para. 4-5): models registered with the decoder ahead of a
+session and bound to slots by id, graphs that went through a file, graphs from the host-memory cache -- every
+way of getting a list onto the device must decode exactly like compiling and binding it, i.e. like the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_21343_b200 import workloads as W
+from helpers import check_greedy, oracle_graph, to_device, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+def _decode_and_check(tb, w, batch, data, lists, what):
+    out = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"])))
+    assert tb.tb_batch_status(batch) == 0
+    for i, p in enumerate(lists):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, p), data["logits"][i]), what)
+
+
+def test_registered_models_decode_like_bound_graphs(tb):
+    w = W.get_workload(2, B=6, T=200)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    graphs = [tb.tb_graph_compile(p, w.V, case_class=cc) for p in data["phrases"]]
+    batch = tb.tb_batch_create(w.V, cc, w.B, arena_bytes=4 << 20)
+    ids = [tb.tb_batch_register_model(batch, g) for g in graphs]
+    assert sorted(ids) == list(range(w.B))
+    for i, m in enumerate(ids):
+        tb.tb_batch_bind_model(batch, i, m)
+    _decode_and_check(tb, w, batch, data, data["phrases"], "registered")
+    # several slots on one model, one slot unbound by id -1, one bound the ordinary way
+    plan = [ids[2], ids[2], -1, ids[0], ids[2], None]
+    lists = [data["phrases"][2], data["phrases"][2], None, data["phrases"][0], data["phrases"][2], data["phrases"][5]]
+    for i, m in enumerate(plan):
+        if m is None:
+            tb.tb_batch_bind_stream(batch, i, graphs[5])
+        else:
+            tb.tb_batch_bind_model(batch, i, m)
+    _decode_and_check(tb, w, batch, data, lists, "shared model")
+    # a model in use cannot be dropped; one that is not can, and its id is handed out again
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_batch_unregister_model(batch, ids[2])
+    assert e.value.code == tb.TB_ERR_INVALID_ARG
+    tb.tb_batch_unregister_model(batch, ids[4])
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_bind_model(batch, 0, ids[4])
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_unregister_model(batch, ids[4])
+    assert tb.tb_batch_register_model(batch, graphs[1]) == ids[4]
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_batch_bind_model(batch, 99, ids[0])
+    assert e.value.code == tb.TB_ERR_BAD_SLOT
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_bind_model(batch, 0, 12345)
+    # moving every slot off a model frees it for removal
+    for i in range(w.B):
+        tb.tb_batch_bind_model(batch, i, -1)
+    for m in set(ids):
+        tb.tb_batch_unregister_model(batch, m)
+    _decode_and_check(tb, w, batch, data, [None] * w.B, "all unbound")
+
+
+def test_registration_does_not_leak_arena_space(tb):
+    w = W.get_workload(2, B=2, T=130)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    g = tb.tb_graph_compile(data["phrases"][0], w.V, case_class=cc)
+    batch = tb.tb_batch_create(w.V, cc, 2, arena_bytes=256 << 10)       # room for a few such graphs only
+    for r in range(200):
+        m = tb.tb_batch_register_model(batch, g)
+        tb.tb_batch_bind_model(batch, r % 2, m)
+        tb.tb_batch_bind_model(batch, r % 2, -1)
+        tb.tb_batch_unregister_model(batch, m)
+    held = []
+    with pytest.raises(tb.TbError) as e:                                 # and the arena does fill up when models are kept
+        for _ in range(100):
+            held.append(tb.tb_batch_register_model(batch, g))
+    assert e.value.code == tb.TB_ERR_ARENA_FULL and len(held) >= 2
+    tb.tb_batch_bind_model(batch, 0, held[0])
+    tb.tb_batch_bind_stream(batch, 1, None)
+    _decode_and_check(tb, w, batch, data, [data["phrases"][0], None], "after churn")
+
+
+def test_graphs_from_file_and_from_the_cache_decode_the_same(tb, tmp_path):
+    w = W.get_workload(2, B=4, T=150)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    cache = tb.tb_cache_create(8 << 20)
+    batch = tb.tb_batch_create(w.V, cc, w.B, arena_bytes=4 << 20)
+    for i, p in enumerate(data["phrases"]):
+        if i % 2:
+            path = str(tmp_path / f"list{i}.tbg")
+            tb.tb_graph_save(tb.tb_graph_compile(p, w.V, case_class=cc), path)
+            g = tb.tb_graph_load(path)
+        else:
+            tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+            g, hit = tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+            assert hit
+        tb.tb_batch_bind_stream(batch, i, g)
+    cache.destroy()
+    _decode_and_check(tb, w, batch, data, data["phrases"], "file / cache")
+
+
+def test_streaming_with_registered_models(tb):
+    # chunked decoding of slots bound by id equals the offline decode of the same streams
+    w = W.get_workload(2, B=3, T=64)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    batch = tb.tb_batch_create(w.V, cc, w.B, arena_bytes=2 << 20)
+    for i, p in enumerate(data["phrases"]):
+        tb.tb_batch_bind_model(batch, i, tb.tb_batch_register_model(batch, tb.tb_graph_compile(p, w.V, case_class=cc)))
+    logits = to_device(data["logits"])
+    toks = [[] for _ in range(w.B)]
+    valid = torch.full((w.B,), w.T, dtype=torch.int32, device="cuda:0")
+    for c in range(w.T // 8):
+        out = to_host(tb.tb_stream_chunk(batch, logits[:, 8 * c:8 * c + 8].contiguous(), 0, valid))
+        for i in range(w.B):
+            toks[i] += list(out["tokens"][i, :out["counts"][i]])
+    for i, p in enumerate(data["phrases"]):
+        ref = O.greedy_rnnt(oracle_graph(w, p), data["logits"][i])
+        assert toks[i] == list(ref["tokens"])

@@ -147,3 +147,130 @@ def test_variative_compile_error_codes(tb):
     assert g["n_states"] == 1 and g["n_arcs"] == 0
     g = tb.tb_graph_compile_variative([b"AB"], pieces, tau=0.0).view()      # the hand-worked list, given in upper case
     assert list(g["arc_class"]) == [0, 2, 1] and list(g["arc_w"]) == [0.5, 1.0, 0.5]
+
+
+# ---- model lifecycle off the device: disk and memory levels (Sec. 2.2 para. 5) ---------------------------
+
+def _same_view(a, b):
+    for k in a:
+        if isinstance(a[k], np.ndarray):
+            assert a[k].dtype == b[k].dtype and a[k].tobytes() == b[k].tobytes(), k
+        else:
+            assert a[k] == b[k], k
+
+
+def test_graph_save_load_round_trip(tb, tmp_path):
+    w = W.get_workload(2)
+    for i, g in enumerate([tb.tb_graph_compile(W.stream_phrases(w, 3), w.V, case_class=w.vocab.case_class, lam=0.5),
+                           tb.tb_graph_compile([], 7),
+                           tb.tb_graph_compile_variative([b"hello", b"help"], [bytes([c]) for c in b"helopHELOP"] + [b"he", b"He", b"llo"])]):
+        path = str(tmp_path / f"g{i}.tbg")
+        tb.tb_graph_save(g, path)
+        _same_view(g.view(), tb.tb_graph_load(path).view())
+
+
+def test_graph_load_refuses_damaged_files(tb, tmp_path):
+    w = W.get_workload(1)
+    g = tb.tb_graph_compile(W.stream_phrases(w, 0), w.V, case_class=w.vocab.case_class)
+    path = str(tmp_path / "g.tbg")
+    tb.tb_graph_save(g, path)
+    raw = open(path, "rb").read()
+
+    def code(data):
+        p = str(tmp_path / "bad.tbg")
+        open(p, "wb").write(data)
+        with pytest.raises(tb.TbError) as e:
+            tb.tb_graph_load(p)
+        return e.value.code
+    assert code(raw[:-1]) == tb.TB_ERR_INVALID_ARG                       # cut short
+    assert code(raw + b"\0") == tb.TB_ERR_INVALID_ARG                    # longer than it says
+    assert code(b"XXXX" + raw[4:]) == tb.TB_ERR_INVALID_ARG              # not such a file
+    assert code(raw[:40]) == tb.TB_ERR_IO                                # not even a header
+    for pos in (8, len(raw) // 2, len(raw) - 3):                          # one altered byte: header field, payload
+        b = bytearray(raw)
+        b[pos] ^= 0x40
+        assert code(bytes(b)) == tb.TB_ERR_INVALID_ARG
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_graph_load(str(tmp_path / "missing.tbg"))
+    assert e.value.code == tb.TB_ERR_IO
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_graph_save(g, str(tmp_path / "no_such_dir" / "g.tbg"))
+    assert e.value.code == tb.TB_ERR_IO
+
+
+def test_cache_returns_what_the_compiler_returns(tb):
+    w = W.get_workload(2)
+    cc = w.vocab.case_class
+    cache = tb.tb_cache_create(1 << 20)
+    lists = [W.stream_phrases(w, b) for b in range(6)]
+    first = []
+    for p in lists:
+        g, hit = tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+        assert not hit
+        _same_view(g.view(), tb.tb_graph_compile(p, w.V, case_class=cc).view())
+        first.append(g)
+    for p, g0 in zip(lists, first):
+        g, hit = tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+        assert hit and g.handle.value == g0.handle.value               # the very same compiled graph
+    # anything the compiler reads is part of the key
+    assert not tb.tb_cache_compile(cache, lists[0], w.V, case_class=cc, lam=0.5)[1]
+    assert not tb.tb_cache_compile(cache, lists[0], w.V, case_class=None)[1]
+    assert not tb.tb_cache_compile(cache, lists[0], w.V, case_class=cc, token_weights=[[1.0] * len(p) for p in lists[0]])[1]
+    assert not tb.tb_cache_compile(cache, lists[0][:-1], w.V, case_class=cc)[1]
+    assert not tb.tb_cache_compile(cache, lists[0][:-2] + [lists[0][-2] + lists[0][-1]], w.V, case_class=cc)[1]   # same tokens, other phrase boundaries
+    st = cache.stats()
+    assert st["hits"] == 6 and st["misses"] == 11 and st["entries"] == 11 and st["evictions"] == 0
+    # errors pass through, nothing is kept for them
+    with pytest.raises(tb.TbError):
+        tb.tb_cache_compile(cache, [[0, w.V + 5]], w.V, case_class=cc)
+    assert cache.stats()["entries"] == 11
+    # a graph handed out stays valid when the cache goes away
+    cache.destroy()
+    assert first[2].view()["n_states"] > 10
+
+
+def test_cache_drops_least_recently_used(tb):
+    w = W.get_workload(2)
+    cc = w.vocab.case_class
+    lists = [W.stream_phrases(w, b) for b in range(5)]
+    probe = tb.tb_cache_create(1 << 24)
+    tb.tb_cache_compile(probe, lists[0], w.V, case_class=cc)
+    one = probe.stats()["bytes_used"]
+    cache = tb.tb_cache_create(int(3.5 * one))                           # room for three such graphs
+    for p in lists[:3]:
+        tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+    assert tb.tb_cache_compile(cache, lists[0], w.V, case_class=cc)[1]   # 0 is now the most recent
+    tb.tb_cache_compile(cache, lists[3], w.V, case_class=cc)             # drops 1, the least recent
+    assert cache.stats()["evictions"] >= 1
+    assert tb.tb_cache_compile(cache, lists[0], w.V, case_class=cc)[1]
+    assert not tb.tb_cache_compile(cache, lists[1], w.V, case_class=cc)[1]
+    tiny = tb.tb_cache_create(64)                                        # too small for any graph: compiles, keeps nothing
+    g, hit = tb.tb_cache_compile(tiny, lists[0], w.V, case_class=cc)
+    assert not hit and g.view()["n_states"] > 10 and tiny.stats()["entries"] == 0
+
+
+def test_cache_is_safe_from_several_threads(tb):
+    import threading
+    w = W.get_workload(2)
+    cc = w.vocab.case_class
+    lists = [W.stream_phrases(w, b) for b in range(8)]
+    want = [tb.tb_graph_compile(p, w.V, case_class=cc).view()["n_states"] for p in lists]
+    cache = tb.tb_cache_create(1 << 22)
+    errors = []
+
+    def work(tid):
+        try:
+            for r in range(30):
+                i = (tid + r) % len(lists)
+                g, _ = tb.tb_cache_compile(cache, lists[i], w.V, case_class=cc)
+                assert g.view()["n_states"] == want[i]
+        except Exception as e:              # noqa: BLE001
+            errors.append(e)
+    threads = [threading.Thread(target=work, args=(t,)) for t in range(8)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors
+    st = cache.stats()
+    assert st["hits"] + st["misses"] == 240 and st["entries"] == 8
