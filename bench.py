@@ -231,7 +231,7 @@ def side_measurement(args):
                           "cuda_graph_ms_per_decode": graph_ms,
                           "config": {"workload": w.name, "B": B, "K": K, "T": T, "E": E,
                                      "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
-    else:
+    elif args.workload == 5:
         w = W.get_workload(5, **({"B": args.streams} if args.streams else {}))
         sched = W.ChurnSchedule(w)
         batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
@@ -263,6 +263,74 @@ def side_measurement(args):
                           "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
                           "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds), "data": "synthetic"}))
 
+    elif args.workload == 7:
+        # Model lifecycle sweep in the manner of the paper's speed table (128 streams; cache: none / disk / memory /
+        # decoder): the streaming workload's churn with 128 slots, the same schedule for every mode; the timed region of
+        # a chunk is host wall clock from "the new streams' lists are known" to "the chunk is decoded".
+        import tempfile
+        w = W.get_workload(5, B=args.streams or 128)
+        cc = w.vocab.case_class
+        sched = W.ChurnSchedule(w)
+        n_chunks = 30 + max(args.steps, 100)
+        plan = [sched.next_chunk() for _ in range(n_chunks)]
+        def flat(p):                                     # the lists as arrays, as a server would hold them
+            offs = np.zeros(len(p) + 1, dtype=np.int64)
+            offs[1:] = np.cumsum([len(x) for x in p])
+            return (np.array([t for x in p for t in x], dtype=np.int32), offs)
+        plan = [(c, l, [(sl, sid, flat(p)) for sl, sid, p in bl]) for c, l, bl in plan]
+        lists = {sid: p for _, _, bl in plan for _, sid, p in bl}
+        tmp = tempfile.mkdtemp(prefix="tb_lists_")
+        rows = []
+        for mode in ("none", "disk", "memory", "decoder"):
+            batch = tb.tb_batch_create(w.V, cc, w.B, arena_bytes=1 << 30)
+            cache, model_of = None, {}
+            if mode == "disk":
+                for sid, p in lists.items():
+                    tb.tb_graph_save(tb.tb_graph_compile(p, w.V, case_class=cc), os.path.join(tmp, "%d.tbg" % sid))
+            elif mode == "memory":
+                cache = tb.tb_cache_create(1 << 30)
+                for p in lists.values():
+                    tb.tb_cache_compile(cache, p, w.V, case_class=cc)
+            elif mode == "decoder":
+                for sid, p in lists.items():
+                    model_of[sid] = tb.tb_batch_register_model(batch, tb.tb_graph_compile(p, w.V, case_class=cc))
+            torch.cuda.synchronize()
+            lat, binds = [], 0
+            for chunk, lengths, bl in plan:
+                dl = torch.from_numpy(chunk).view(torch.bfloat16).to(dev)
+                dv = torch.from_numpy(lengths).to(dev)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                for sl, sid, p in bl:
+                    if mode == "none":
+                        tb.tb_batch_bind_stream(batch, sl, tb.tb_graph_compile(p, w.V, case_class=cc))
+                    elif mode == "disk":
+                        tb.tb_batch_bind_stream(batch, sl, tb.tb_graph_load(os.path.join(tmp, "%d.tbg" % sid)))
+                    elif mode == "memory":
+                        tb.tb_batch_bind_stream(batch, sl, tb.tb_cache_compile(cache, p, w.V, case_class=cc)[0])
+                    else:
+                        tb.tb_batch_bind_model(batch, sl, model_of[sid])
+                tb.tb_stream_chunk(batch, dl, w.n_dur, dv)
+                torch.cuda.synchronize()
+                lat.append((time.perf_counter() - t0) * 1e3)
+                binds += len(bl)
+            assert tb.tb_batch_status(batch) == 0
+            steady = np.array(lat[30:])                      # the first chunks bind every slot at once
+            nb = sum(len(bl) for _, _, bl in plan[30:])
+            rows.append({"cache": mode, "ms_per_chunk_mean": float(steady.mean()), "ms_per_chunk_p50": float(np.percentile(steady, 50)),
+                         "ms_per_chunk_p99": float(np.percentile(steady, 99)),
+                         "frames_per_s": w.B * w.chunk * len(steady) / (float(steady.sum()) * 1e-3),
+                         "binds_per_chunk": nb / len(steady)})
+            batch.destroy()
+        base = rows[-1]["frames_per_s"]
+        for r in rows:
+            r["vs_decoder_level"] = r["frames_per_s"] / base
+        print(json.dumps({"metric": "model_lifecycle_sweep_streaming_tdt", "unit": UNIT, "n_gpus": 1, "rows": rows,
+                          "config": {"workload": w.name + " (128 slots)", "slots": w.B, "chunk_frames": w.chunk,
+                                     "chunks": n_chunks - 30, "lists": len(lists),
+                                     "timed": "host wall clock per chunk: obtain the new streams' graphs, bind, decode the chunk, synchronise"},
+                          "data": "synthetic"}))
+
 
 def main():
     ap = argparse.ArgumentParser()
@@ -273,8 +341,8 @@ def main():
     ap.add_argument("--streams", type=int, default=0, help="override B (profiling captures use a small case)")
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
-    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6],
-                    help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists: side measurements")
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
+                    help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists, 7 model lifecycle sweep: side measurements")
     args = ap.parse_args()
     if args.workload != 2:
         side_measurement(args)

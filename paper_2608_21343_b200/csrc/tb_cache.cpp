@@ -20,9 +20,17 @@ namespace {
 constexpr uint32_t kMagic = 0x31474254u;   // "TBG1"
 constexpr uint32_t kVersion = 1;
 
+// FNV-1a style checksum over 8-byte words (the tail byte by byte): detects damage, is not cryptographic
 uint64_t fnv1a(const void* p, size_t n, uint64_t h = 1469598103934665603ull) {
   const unsigned char* b = static_cast<const unsigned char*>(p);
-  for (size_t i = 0; i < n; ++i) h = (h ^ b[i]) * 1099511628211ull;
+  size_t i = 0;
+  for (; i + 8 <= n; i += 8) {
+    uint64_t w;
+    std::memcpy(&w, b + i, 8);
+    h = (h ^ w) * 1099511628211ull;
+    h ^= h >> 29;
+  }
+  for (; i < n; ++i) h = (h ^ b[i]) * 1099511628211ull;
   return h;
 }
 
