@@ -30,7 +30,9 @@
  * formulas (brute-force substring matching, explicit case expansion, exhaustive beam
  * enumeration, library argmax).  Not pinned beyond reduced cases ("parity unpinned"):
  * beam decoding with K smaller than the number of alignments on large inputs, TDT with
- * free durations, and the stream-churn schedule.
+ * durations that vary from row to row (pinned by a hand-worked case and by the reductions
+ * "all durations 0 = the RNNT rule" and "all durations d = the unit case on every d-th
+ * frame"), and the stream-churn schedule.
  *
  * Arithmetic: potentials in double, each stored value rounded once to float; every
  * run-time sum is a float add in the order written, compiled with -ffp-contract=off so

@@ -579,3 +579,47 @@ def test_chunked_equals_unchunked(n_dur):
         assert toks == list(ref["tokens"]) and frs == list(ref["frames"]) and durs == list(ref["durs"])
         assert (st.state, st.t, st.k, st.n_emitted) == (whole.state, whole.t, whole.k, whole.n_emitted)
         assert st.score == whole.score
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_tdt_with_zero_durations_is_the_rnnt_rule(seed):
+    """Durations rigged to 0 on every row: a token stays in its frame and moves to the next row, blank still
+    advances one frame, the S-th symbol closes the frame -- the label-looping RNNT rule, which is pinned on its own.
+    The duration logit that wins is 0, so even the scores agree bit for bit."""
+    rng = np.random.default_rng(40 + seed)
+    V, D, T, S = 12, 5, 50, 3
+    phrases, weights = random_list(rng, V, 6, 3, dyadic_weights=True)
+    g = O.Graph(phrases, V, weights=weights)
+    x = dyadic_logits(rng, (T, S, V + 1 + D), blank_bias=0.5)
+    x[:, :, V + 1:] = -1.0
+    x[:, :, V + 1] = 0.0
+    st = O.StreamState(0, 0, 0, 0.0, 0)
+    r = O.stream_chunk(g, x, D, 0, T, st)
+    ref = O.greedy_rnnt(g, np.ascontiguousarray(x[:, :, :V + 1]))
+    assert list(r["tokens"]) == list(ref["tokens"]) and list(r["frames"]) == list(ref["frames"])
+    assert set(r["durs"]) <= {0} and st.state == ref["state"] and st.t == T
+    assert np.float32(st.score) == ref["score"]
+
+
+@pytest.mark.parametrize("d", [2, 3, 4])
+def test_tdt_with_constant_durations_is_the_unit_case_on_every_dth_frame(d):
+    """Durations rigged to d on every row: only rows (0, 0), (d, 0), (2d, 0), ... are visited, each once -- the
+    unit-duration decode (pinned above against a per-frame argmax) of the tensor that keeps every d-th frame."""
+    rng = np.random.default_rng(50 + d)
+    V, D, T, S = 10, 5, 61, 2
+    phrases, _ = random_list(rng, V, 5, 3)
+    g = O.Graph(phrases, V)
+    x = dyadic_logits(rng, (T, S, V + 1 + D))
+    x[:, :, V + 1:] = 0.0
+    x[:, :, V + 1 + d] = 1.0
+    st = O.StreamState(0, 0, 0, 0.0, 0)
+    r = O.stream_chunk(g, x, D, 0, T, st)
+    y = np.ascontiguousarray(x[::d])
+    y[:, :, V + 1:] = 0.0
+    y[:, :, V + 2] = 1.0                                         # the same rows, duration 1
+    Ty = y.shape[0]
+    st1 = O.StreamState(0, 0, 0, 0.0, 0)
+    r1 = O.stream_chunk(g, y, D, 0, Ty, st1)
+    assert list(r["tokens"]) == list(r1["tokens"]) and list(r["frames"]) == [d * f for f in r1["frames"]]
+    assert set(r["durs"]) <= {d} and st.state == st1.state and st.score == st1.score
+    assert st.t == d * Ty and st.n_emitted == st1.n_emitted
