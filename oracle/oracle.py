@@ -78,6 +78,8 @@ def lib():
         _lib.orc_graph_get.argtypes = [C.c_void_p, C.POINTER(_GraphStruct)]
         _lib.orc_step.restype = None
         _lib.orc_step.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        _lib.orc_apply_final_weight.restype = C.c_float
+        _lib.orc_apply_final_weight.argtypes = [C.c_void_p, C.c_int32, C.c_float]
         _lib.orc_greedy_rnnt.restype = C.c_int64
         _lib.orc_greedy_rnnt.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
@@ -202,6 +204,11 @@ class GraphFromArrays(Graph):
 
     def __del__(self):                         # nothing of this graph was allocated by the C file
         self.handle = None
+
+
+def apply_final_weight(graph, state: int, score) -> np.float32:
+    """score + lambda * final(state): the end-of-stream charge of a hypothesis that stops in ``state``."""
+    return np.float32(lib().orc_apply_final_weight(graph.handle if graph is not None else None, int(state), float(score)))
 
 
 def null_step(v: int):

@@ -293,6 +293,20 @@ void orc_step(const orc_graph *g, int32_t s, int32_t v, float *bonus, int32_t *n
   }
 }
 
+/*
+ * End of stream (Sec. 2.2 para. 2 lists a final weight per state): a hypothesis that stops in
+ * state s is charged that state's final weight, score' = score + lambda * final(s), a rounded
+ * multiply and a rounded add like every other bonus.  final(s) = -loan(s): what a partial match
+ * had been lent is returned, so that a finished hypothesis keeps the bonus of the phrases it
+ * completed and nothing else.  READING: the paper names the tensor only; this is the one use
+ * that makes its value (the loan, negated) meaningful.  A NULL graph or state -1 changes nothing.
+ */
+float orc_apply_final_weight(const orc_graph *g, int32_t s, float score) {
+  if (!g || s < 0) return score;
+  float lam_f = g->lambda * g->state_final[s];
+  return score + lam_f;
+}
+
 /* ------------------------------------------------------------------------------------ */
 /* Logit access and the boosted value of one candidate.                                  */
 /* ------------------------------------------------------------------------------------ */

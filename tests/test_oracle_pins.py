@@ -623,3 +623,43 @@ def test_tdt_with_constant_durations_is_the_unit_case_on_every_dth_frame(d):
     assert list(r["tokens"]) == list(r1["tokens"]) and list(r["frames"]) == [d * f for f in r1["frames"]]
     assert set(r["durs"]) <= {d} and st.state == st1.state and st.score == st1.score
     assert st.t == d * Ty and st.n_emitted == st1.n_emitted
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_final_weight_leaves_exactly_the_completed_phrases(seed):
+    """After the end-of-stream charge the bonus a history has collected is the sum over the phrase occurrences
+    that were completed in it, found by plain substring matching (no automaton): the loan of an unfinished
+    match is gone.  Dyadic weights make every sum exact."""
+    rng = np.random.default_rng(70 + seed)
+    V = 6
+    phrases, weights = random_list(rng, V, 8, 4, dyadic_weights=True)
+    merged = {}
+    for p, wts in zip(phrases, weights):                       # duplicates: element-wise largest weight
+        if len(p):
+            merged[tuple(p)] = [max(a, b) for a, b in zip(merged.get(tuple(p), [0.0] * len(p)), wts)]
+    # weight of the node reached by a prefix = largest weight any phrase through it gives that position
+    node_w = {}
+    for p, wts in merged.items():
+        for i in range(len(p)):
+            node_w[p[:i + 1]] = max(node_w.get(p[:i + 1], 0.0), wts[i])
+    ends = sorted(merged, key=len)
+
+    def completed_value(p):
+        # what completing p banks: the node weights since the last phrase end strictly inside p
+        last = max([len(q) for q in ends if len(q) < len(p) and p[:len(q)] == q], default=0)
+        return sum(node_w[p[:i + 1]] for i in range(last, len(p)))
+    g = O.Graph(phrases, V, weights=weights, lam=2.0)
+    for _ in range(200):
+        h = [int(t) for t in rng.integers(0, V, size=int(rng.integers(0, 14)))]
+        s, total = 0, 0.0
+        for t in h:
+            b, s = g.step(s, t)
+            total += 2.0 * float(b)
+        total = float(O.apply_final_weight(g, s, total))
+        want = 0.0
+        for p in merged:
+            for i in range(len(h) - len(p) + 1):
+                if tuple(h[i:i + len(p)]) == p:
+                    want += 2.0 * completed_value(p)
+        assert total == want, (h, total, want)
+    assert float(O.apply_final_weight(None, -1, 3.5)) == 3.5 and float(O.apply_final_weight(g, -1, 3.5)) == 3.5
