@@ -344,6 +344,19 @@ int tb_beam_step(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t 
                  int32_t *out_parent, int32_t *out_token, void *stream);
 
 /*
+ * End of stream: charge every hypothesis the final weight of the graph state it stops in (Sec. 2.2 para. 2
+ * lists a final weight per state; it is the loan of the unfinished partial match, negated, so a finished
+ * hypothesis keeps the bonus of the phrases it completed and nothing else):
+ * scores[i, k] = fl(scores[i, k] + fl(lambda_i * final(states[i, k]))) for stream i = 0..B-1 bound to a graph,
+ * states[i, k] >= 0 and a score above -inf; everything else is left as it is.  Works on the [B, K] arrays of
+ * tb_beam_step (re-rank afterwards if the order matters) and, with K = 1, on out_scores / out_states of
+ * tb_greedy_decode or tb_stream_chunk.
+ *   scores  device float [B, K], updated in place;  states  device int32 [B, K]
+ * Errors: TB_ERR_INVALID_ARG, TB_ERR_CUDA; a state outside the graph sets TB_STATUS_BAD_STATE.
+ */
+int tb_apply_final_weights(tb_batch *b, int32_t B, int32_t K, float *scores, const int32_t *states, void *stream);
+
+/*
  * Walk the hypothesis tree back from the hypotheses of the latest step and write each one's
  * non-blank tokens in emission order (Sec. 2.3: hypotheses live in a flattened tree).
  *   out_tokens  device int32 [B, K, max_len]; sequences longer than max_len are truncated

@@ -75,6 +75,7 @@ _SIGS = {
     "tb_beam_reset": (C.c_int, [_vp]),
     "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "tb_apply_final_weights": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
                                            _vp, _vp, _vp]),
 }
@@ -391,6 +392,17 @@ def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_str
     _check(_lib.tb_beam_step(batch.handle, ptr, _logit_dtype(logits), B, K, stream_stride, hyp_stride,
                              1 if new_frame else 0, _dp(scores), _dp(states), _dp(live), _dp(out_parent),
                              _dp(out_token), _stream(stream)), "tb_beam_step")
+
+
+def tb_apply_final_weights(batch: Batch, scores: torch.Tensor, states: torch.Tensor, stream=None):
+    """scores float32 [B] or [B, K], states int32 of the same shape (device, contiguous); scores updated in place."""
+    assert scores.dtype == torch.float32 and states.dtype == torch.int32 and scores.shape == states.shape
+    assert scores.is_contiguous() and states.is_contiguous()
+    B = scores.shape[0]
+    K = 1 if scores.dim() == 1 else scores.shape[1]
+    _check(_lib.tb_apply_final_weights(batch.handle, B, K, _dp(scores), _dp(states), _stream(stream)),
+           "tb_apply_final_weights")
+    return scores
 
 
 def tb_beam_backtrace(batch: Batch, B: int, K: int, max_len: int, stream=None):

@@ -203,6 +203,7 @@ static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, siz
   rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
   rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
   rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
+  rec.off_final = g->off_final;
   rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
   rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
   rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
@@ -372,6 +373,14 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
     if (rc != 1) return rc;
   }
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* scores, const int32_t* states,
+                                      void* stream_) {
+  if (!b || !scores || !states || B < 1 || B > b->n_slots || K < 1) return TB_ERR_INVALID_ARG;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  return tb_launch_final_weights(b->d_slots, b->arena, B, K, scores, states, b->d_status, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {

@@ -18,7 +18,7 @@
 namespace {
 
 constexpr uint32_t kMagic = 0x31474254u;   // "TBG1"
-constexpr uint32_t kVersion = 1;
+constexpr uint32_t kVersion = 2;
 
 // FNV-1a style checksum over 8-byte words (the tail byte by byte): detects damage, is not cryptographic
 uint64_t fnv1a(const void* p, size_t n, uint64_t h = 1469598103934665603ull) {
@@ -42,7 +42,7 @@ struct FileHeader {
   int32_t off_arc_begin, off_fail, off_bw, off_arc_cls, off_arc_w, off_arc_dst, off_strec, off_tokent, n_tokent;
   int32_t off_rsrec, off_rsent, n_rsent;
   float d_max;
-  uint32_t pad;
+  int32_t off_final;
   uint64_t blob_bytes;
   uint64_t payload_hash;   // of everything after the header
 };
@@ -83,7 +83,7 @@ extern "C" int tb_graph_save(const tb_graph* g, const char* path) {
     h.off_arc_begin = g->off_arc_begin; h.off_fail = g->off_fail; h.off_bw = g->off_bw; h.off_arc_cls = g->off_arc_cls;
     h.off_arc_w = g->off_arc_w; h.off_arc_dst = g->off_arc_dst; h.off_strec = g->off_strec; h.off_tokent = g->off_tokent;
     h.n_tokent = g->n_tokent; h.off_rsrec = g->off_rsrec; h.off_rsent = g->off_rsent; h.n_rsent = g->n_rsent;
-    h.d_max = g->d_max; h.blob_bytes = g->blob.size();
+    h.d_max = g->d_max; h.off_final = g->off_final; h.blob_bytes = g->blob.size();
     h.payload_hash = fnv1a(payload.data(), payload.size());
     std::FILE* f = std::fopen(path, "wb");
     if (!f) return TB_ERR_IO;
@@ -135,11 +135,11 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
     g->off_arc_begin = h.off_arc_begin; g->off_fail = h.off_fail; g->off_bw = h.off_bw; g->off_arc_cls = h.off_arc_cls;
     g->off_arc_w = h.off_arc_w; g->off_arc_dst = h.off_arc_dst; g->off_strec = h.off_strec; g->off_tokent = h.off_tokent;
     g->n_tokent = h.n_tokent; g->off_rsrec = h.off_rsrec; g->off_rsent = h.off_rsent; g->n_rsent = h.n_rsent;
-    g->d_max = h.d_max;
+    g->d_max = h.d_max; g->off_final = h.off_final;
     // the sections named by the header must lie inside the blob
     const int64_t B = static_cast<int64_t>(g->blob.size());
     const int32_t offs[] = {g->off_arc_begin, g->off_fail, g->off_bw, g->off_arc_cls, g->off_arc_w, g->off_arc_dst,
-                            g->off_strec, g->off_tokent, g->off_rsrec, g->off_rsent};
+                            g->off_strec, g->off_tokent, g->off_rsrec, g->off_rsent, g->off_final};
     for (int32_t o : offs)
       if (o < 0 || o > B || (o & 15)) { delete g; return TB_ERR_INVALID_ARG; }
     if (g->class_map_hash != tb_hash_class_map(g->case_class.data(), g->vocab)) { delete g; return TB_ERR_INVALID_ARG; }

@@ -74,6 +74,7 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
   g->off_arc_cls = append_section(g->blob, g->arc_class);
   g->off_arc_w = append_section(g->blob, g->arc_w);
   g->off_arc_dst = append_section(g->blob, g->arc_dst);
+  g->off_final = append_section(g->blob, g->state_final);
   {  // per-state records and token-expanded arcs (tokens of a class in ascending id order)
     std::vector<int32_t> ctb(n_classes + 1, 0), ctk(vocab);
     for (int32_t v = 0; v < vocab; ++v) ctb[g->case_class[v] + 1]++;

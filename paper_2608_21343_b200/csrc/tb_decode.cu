@@ -475,6 +475,29 @@ int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
+// End of stream: every hypothesis that stops in a graph state is charged that state's final weight,
+// score' = fl(score + fl(lambda * final(state))).  Unbound slots, state -1 and empty places (-inf) stay as they are.
+__global__ void k_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,
+                                const int32_t* states, int32_t* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * K) return;
+  const TbSlotRec rec = slots[i / K];
+  const int32_t s = states[i];
+  if (rec.n_states <= 0 || s < 0) return;
+  if (s >= rec.n_states) { atomicOr(status, TB_STATUS_BAD_STATE); return; }
+  const float fin = reinterpret_cast<const float*>(arena + rec.blob_off + rec.off_final)[s];
+  const float sc = scores[i];
+  if (sc == -INFINITY) return;
+  scores[i] = __fadd_rn(sc, __fmul_rn(rec.lambda, fin));
+}
+
+int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,
+                            const int32_t* states, int32_t* status, cudaStream_t stream) {
+  const int n = B * K;
+  k_final_weights<<<(n + 127) / 128, 128, 0, stream>>>(slots, arena, B, K, scores, states, status);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
                            cudaStream_t stream) {
   k_publish_slot<<<1, 32, 0, stream>>>(slots, sstate, slot, rec);

@@ -21,6 +21,7 @@ struct tb_graph {
   // Device blob: sections at 16-byte aligned offsets, all ids graph-local.
   std::vector<unsigned char> blob;
   int32_t off_arc_begin = 0, off_fail = 0, off_bw = 0, off_arc_cls = 0, off_arc_w = 0, off_arc_dst = 0;
+  int32_t off_final = 0;                               // state_final as a blob section (end-of-stream weights)
   int32_t off_strec = 0, off_tokent = 0, n_tokent = 0;
   int32_t off_rsrec = 0, off_rsent = 0, n_rsent = 0;  // resolved per-state lists (n_rsent < 0: not built)
   float d_max = 0.0f;                                  // largest |sum of suffix-link weights| over all states
@@ -79,7 +80,8 @@ struct TbSlotRec {
   int32_t n_tokent, blob_bytes;
   int32_t off_rsrec, off_rsent, n_rsent;  // resolved lists; n_rsent < 0: the graph has none
   float d_max;
-  int32_t pad[12];
+  int32_t off_final;   // per-state final weights (within the blob)
+  int32_t pad[11];
 };
 static_assert(sizeof(TbSlotRec) == 128, "slot record is 128 bytes");
 

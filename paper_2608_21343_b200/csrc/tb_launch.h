@@ -45,6 +45,8 @@ int tb_launch_greedy_fast(const TbDecodeParams& p, int32_t max_cache_bytes, int3
 int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
+int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,
+                            const int32_t* states, int32_t* status, cudaStream_t stream);
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
                            cudaStream_t stream);
 

@@ -121,3 +121,45 @@ def test_streaming_with_registered_models(tb):
     for i, p in enumerate(data["phrases"]):
         ref = O.greedy_rnnt(oracle_graph(w, p), data["logits"][i])
         assert toks[i] == list(ref["tokens"])
+
+
+def test_final_weights_after_greedy_and_beam(tb):
+    # greedy: the charge on out_scores / out_states equals the oracle's; beam: on the [B, K] arrays, empty places kept
+    w = W.get_workload(2, B=5, T=140)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    lists = list(data["phrases"])
+    lists[3] = None
+    batch = tb.tb_batch_create(w.V, cc, w.B, arena_bytes=4 << 20, max_beam=4)
+    for i, p in enumerate(lists):
+        tb.tb_batch_bind_stream(batch, i, None if p is None else tb.tb_graph_compile(p, w.V, case_class=cc, lam=0.5))
+    out = tb.tb_greedy_decode(batch, to_device(data["logits"]))
+    before = out["scores"].clone()
+    tb.tb_apply_final_weights(batch, out["scores"], out["states"])
+    torch.cuda.synchronize()
+    changed = 0
+    for i, p in enumerate(lists):
+        g = oracle_graph(w, p, lam=0.5)
+        want = O.apply_final_weight(g, int(out["states"][i]), float(before[i]))
+        assert np.float32(out["scores"][i].item()) == want
+        changed += float(before[i]) != float(want)
+    assert float(out["scores"][3]) == float(before[3])
+    # every state of one graph, as a [1, K] call per group of four states
+    g = oracle_graph(w, lists[0], lam=0.5)
+    n = g.n_states
+    states = torch.arange(0, 4 * (n // 4), dtype=torch.int32, device="cuda:0").reshape(-1, 4)
+    for r in range(0, states.shape[0], 97):
+        sc = torch.tensor([[1.5, float("-inf"), -2.25, 0.0]], device="cuda:0")
+        st = states[r:r + 1].contiguous()
+        tb.tb_apply_final_weights(batch, sc, st)
+        torch.cuda.synchronize()
+        for k in range(4):
+            if k == 1:
+                assert float(sc[0, k]) == float("-inf")
+            else:
+                assert np.float32(sc[0, k].item()) == O.apply_final_weight(g, int(st[0, k]), [1.5, 0, -2.25, 0.0][k])
+    assert tb.tb_batch_status(batch) == 0
+    bad = torch.tensor([[10 ** 6]], dtype=torch.int32, device="cuda:0")
+    tb.tb_apply_final_weights(batch, torch.zeros((1, 1), device="cuda:0"), bad)
+    assert tb.tb_batch_status(batch) == 2            # TB_STATUS_BAD_STATE: a state outside the graph is reported, not used
+    assert tb.tb_batch_status(batch) == 0            # (reading the word clears it)
