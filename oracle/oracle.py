@@ -91,6 +91,10 @@ def lib():
         _lib.orc_beam_step.restype = None
         _lib.orc_beam_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int32,
                                        C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.orc_beam_decode_merge.restype = C.c_int
+        _lib.orc_beam_decode_merge.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
+                                               C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.orc_beam_decode.restype = C.c_int
         _lib.orc_beam_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -273,8 +277,9 @@ def beam_step(graph, rows_logits: np.ndarray, scores, states, live):
     return par, tok
 
 
-def beam_decode(graph, logits: np.ndarray, K: int, max_len=None):
+def beam_decode(graph, logits: np.ndarray, K: int, max_len=None, merge: bool = False):
     """Frame-synchronous beam decode of one stream.  logits [T, E, V+1].
+    merge: hypotheses with equal token sequences are merged at every frame start (the best is kept).
 
     Returns dict(tokens=list of K arrays, lens, scores, states, tree [T*E, K, 2])."""
     T, E, V1 = logits.shape
@@ -285,9 +290,9 @@ def beam_decode(graph, logits: np.ndarray, K: int, max_len=None):
     states = np.zeros(K, dtype=np.int32)
     tree = np.zeros((T * E, K, 2), dtype=np.int32)
     st = _strides3(logits)
-    rc = lib().orc_beam_decode(graph.handle if graph is not None else None, _ptr(logits), _dtype_code(logits),
-                               T, E, V1 - 1, _ptr(st), K, max_len, _ptr(out_tokens), _ptr(lens),
-                               _ptr(scores), _ptr(states), _ptr(tree))
+    rc = lib().orc_beam_decode_merge(graph.handle if graph is not None else None, _ptr(logits), _dtype_code(logits),
+                                     T, E, V1 - 1, _ptr(st), K, max_len, 1 if merge else 0, _ptr(out_tokens),
+                                     _ptr(lens), _ptr(scores), _ptr(states), _ptr(tree))
     assert rc == 0
     return dict(tokens=[out_tokens[k, :min(lens[k], max_len)].copy() for k in range(K)], lens=lens,
                 scores=scores, states=states, tree=tree)

@@ -506,9 +506,17 @@ void orc_beam_step(const orc_graph *g, const void *logits, int dtype, const int6
  * pairs to tree [T*E, K, 2].  Results per final slot j: token sequence (backtrace, carried
  * candidates skipped, blanks dropped) in out_tokens[j*max_len ...], its length, score, state.
  */
-int orc_beam_decode(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
-                    const int64_t *strides, int32_t K, int32_t max_len, int32_t *out_tokens,
-                    int32_t *out_lens, float *out_scores, int32_t *out_states, int32_t *tree) {
+/*
+ * merge != 0 (Sec. 2.3: stored hypotheses are anchors for continuing, merging and pruning): at the start of
+ * every frame, hypotheses that have emitted the same token sequence are one transcript reached by different
+ * alignments; the best of them (the first in selection order) is kept, the others become empty places.
+ * READING: merging happens where the hypotheses are in the same situation -- all live, at a frame start -- so
+ * that equal sequences have equal futures and keeping the best loses nothing (the result is, per token
+ * sequence, the best alignment, as long as the beam is wide enough).
+ */
+int orc_beam_decode_merge(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
+                          const int64_t *strides, int32_t K, int32_t max_len, int32_t merge, int32_t *out_tokens,
+                          int32_t *out_lens, float *out_scores, int32_t *out_states, int32_t *tree) {
   float *scores = (float *)malloc((size_t)K * sizeof(float));
   int32_t *states = (int32_t *)malloc((size_t)K * sizeof(int32_t));
   uint8_t *live = (uint8_t *)malloc((size_t)K);
@@ -519,14 +527,40 @@ int orc_beam_decode(const orc_graph *g, const void *logits, int dtype, int32_t T
   for (int32_t k = 0; k < K; ++k) { scores[k] = -INFINITY; states[k] = -1; live[k] = 0; }
   scores[0] = 0.0f; states[0] = g ? 0 : -1; live[0] = 1;
   int64_t step = 0;
+  /* the token sequence of every hypothesis, kept explicitly for the merge */
+  const int64_t cap = (int64_t)T * E + 1;
+  int32_t *seq = (int32_t *)malloc((size_t)K * cap * sizeof(int32_t));
+  int32_t *seq2 = (int32_t *)malloc((size_t)K * cap * sizeof(int32_t));
+  int32_t *len = (int32_t *)calloc((size_t)K, sizeof(int32_t));
+  int32_t *len2 = (int32_t *)calloc((size_t)K, sizeof(int32_t));
   for (int32_t t = 0; t < T; ++t) {
+    if (merge) {
+      for (int32_t k = 1; k < K; ++k) {
+        if (scores[k] == -INFINITY) continue;
+        for (int32_t j = 0; j < k; ++j) {
+          if (scores[j] == -INFINITY || len[j] != len[k]) continue;
+          if (memcmp(seq + j * cap, seq + k * cap, (size_t)len[k] * sizeof(int32_t)) != 0) continue;
+          scores[k] = -INFINITY; states[k] = -1; live[k] = 0;
+          break;
+        }
+      }
+    }
     for (int32_t k = 0; k < K; ++k) live[k] = (uint8_t)(scores[k] != -INFINITY);
     for (int32_t e = 0; e < E; ++e, ++step) {
       for (int32_t k = 0; k < K; ++k) rows[k] = (int64_t)t * strides[0] + (int64_t)e * strides[1];
       orc_beam_step(g, logits, dtype, rows, strides[2], K, V, scores, states, live, par, tok);
       for (int32_t k = 0; k < K; ++k) { tree[(step * K + k) * 2] = par[k]; tree[(step * K + k) * 2 + 1] = tok[k]; }
+      for (int32_t k = 0; k < K; ++k) {
+        len2[k] = 0;
+        if (par[k] < 0) continue;
+        memcpy(seq2 + k * cap, seq + par[k] * cap, (size_t)len[par[k]] * sizeof(int32_t));
+        len2[k] = len[par[k]];
+        if (tok[k] >= 0 && tok[k] != V) seq2[k * cap + len2[k]++] = tok[k];
+      }
+      { int32_t *sw = seq; seq = seq2; seq2 = sw; sw = len; len = len2; len2 = sw; }
     }
   }
+  free(seq); free(seq2); free(len); free(len2);
   for (int32_t j = 0; j < K; ++j) {
     out_scores[j] = scores[j]; out_states[j] = states[j];
     int32_t n = 0, slot = j;
@@ -543,4 +577,11 @@ int orc_beam_decode(const orc_graph *g, const void *logits, int dtype, int32_t T
   }
   free(scores); free(states); free(live); free(rows); free(par); free(tok); free(rev);
   return ORC_OK;
+}
+
+int orc_beam_decode(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
+                    const int64_t *strides, int32_t K, int32_t max_len, int32_t *out_tokens,
+                    int32_t *out_lens, float *out_scores, int32_t *out_states, int32_t *tree) {
+  return orc_beam_decode_merge(g, logits, dtype, T, E, V, strides, K, max_len, 0, out_tokens, out_lens, out_scores,
+                               out_states, tree);
 }

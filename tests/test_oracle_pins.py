@@ -663,3 +663,36 @@ def test_final_weight_leaves_exactly_the_completed_phrases(seed):
                     want += 2.0 * completed_value(p)
         assert total == want, (h, total, want)
     assert float(O.apply_final_weight(None, -1, 3.5)) == 3.5 and float(O.apply_final_weight(g, -1, 3.5)) == 3.5
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_beam_with_merging_keeps_the_best_alignment_of_every_sequence(seed):
+    """With room for everything, merging equal token sequences at frame starts leaves, for every distinct
+    token sequence, exactly its best alignment (found by exhaustive enumeration), in score order."""
+    rng = np.random.default_rng(600 + seed)
+    V, T, E = 3, 3, 2
+    phrases = [[0, 1], [1], [2, 0, 1]][: 2 + seed % 2]
+    g = O.Graph(phrases, V)
+    br = Brute(phrases)
+    x = dyadic_logits(rng, (T, E, V + 1), q=1 << 16)
+    best = {}
+    for h, raw in _alignments(x, E, V):
+        sc = raw + br.G(h)
+        best[tuple(h)] = max(best.get(tuple(h), -np.inf), sc)
+    K = 13 ** 3
+    r = O.beam_decode(g, x, K, merge=True)
+    got = [(float(r["scores"][k]), tuple(int(v) for v in r["tokens"][k])) for k in range(K) if np.isfinite(r["scores"][k])]
+    # merging happens at frame starts, so the alignments of the last frame are still all there: reduce them
+    final = {}
+    for sc, h in got:
+        final[h] = max(final.get(h, -np.inf), sc)
+    assert final == best
+    # and before the last frame nothing is double: the number of survivors is what the last frame can make of
+    # the distinct sequences alive at its start
+    r2 = O.beam_decode(g, x[:T - 1], K, merge=True)
+    alive = [tuple(int(v) for v in r2["tokens"][k]) for k in range(K) if np.isfinite(r2["scores"][k])]
+    n_start = len(set(alive))
+    assert len(got) == 13 * n_start
+    # without merging the same run keeps every alignment
+    r0 = O.beam_decode(g, x, K)
+    assert int(np.isfinite(r0["scores"]).sum()) == K > len(got)
