@@ -55,6 +55,11 @@ extern "C" {
 #define TB_STATUS_STEP_LIMIT 4      /* a decode loop hit its static iteration bound */
 #define TB_STATUS_WAIT_TIMEOUT 8    /* a bounded wait inside a kernel ran out */
 
+/* tb_beam_step, new_frame */
+#define TB_FRAME_SAME 0       /* another row of the current frame */
+#define TB_FRAME_NEW 1        /* first row of a frame: every hypothesis with a score becomes live */
+#define TB_FRAME_NEW_MERGE 2  /* as TB_FRAME_NEW, after hypotheses with equal token sequences were merged */
+
 /* tb_batch_set_flags */
 #define TB_FLAG_GENERAL_KERNELS 1   /* always use the general decode kernel (any layout), never the pipelined one */
 
@@ -317,7 +322,12 @@ int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots,
                     int32_t *out_tokens, int32_t *out_frames, int32_t *out_durs, int32_t *out_counts,
                     float *out_scores, int32_t *out_states, int32_t *out_cursors, void *stream);
 
-/* Forget the hypothesis tree (step counter = 0).  Call before the first step of an utterance. */
+/*
+ * Forget the hypothesis tree (step counter = 0) and the per-hypothesis record of emitted token sequences (every
+ * hypothesis starts from the empty sequence).  Call before the first step of an utterance; the clearing is
+ * ordered on the device's default stream.  Across the chunks of one utterance simply keep calling
+ * tb_beam_step: scores, states, liveness (the caller's arrays), the tree and the sequence records carry over.
+ */
 int tb_beam_reset(tb_batch *b);
 
 /*
@@ -334,7 +344,12 @@ int tb_beam_reset(tb_batch *b);
  *   logits         device; hypothesis k of stream i reads the vocab+1 contiguous elements
  *                  at element offset i*stream_stride + k*hyp_stride (hyp_stride 0: all
  *                  hypotheses of a stream share one row)
- *   new_frame      non-zero: before expanding, every hypothesis with score > -inf becomes live
+ *   new_frame      TB_FRAME_SAME, TB_FRAME_NEW (before expanding, every hypothesis with score > -inf becomes
+ *                  live) or TB_FRAME_NEW_MERGE (Sec. 2.3, merging: first, hypotheses of a stream that have
+ *                  emitted the same token sequence -- one transcript reached by different alignments -- are
+ *                  merged: the first in slot order, i.e. the best of the previous step, stays, the others
+ *                  become empty places; then as TB_FRAME_NEW).  Sequences are compared by length, graph
+ *                  state and a 64-bit hash kept per hypothesis inside the batch from tb_beam_reset on.
  *   scores/states/live  device float / int32 / uint8 [B, K], updated in place
  *   out_parent/out_token  device int32 [B, K]
  * Errors: TB_ERR_INVALID_ARG (K > max_beam, tree full, ...), TB_ERR_CUDA.

@@ -23,6 +23,7 @@ _lib = C.CDLL(LIB_PATH)
 TB_OK = 0
 TB_ERR_INVALID_ARG, TB_ERR_OOM, TB_ERR_CUDA, TB_ERR_ARENA_FULL, TB_ERR_BAD_SLOT, TB_ERR_DEVICE_STATUS = -1, -2, -3, -4, -5, -6
 TB_ERR_IO = -7
+TB_FRAME_SAME, TB_FRAME_NEW, TB_FRAME_NEW_MERGE = 0, 1, 2
 TB_BF16, TB_F32 = 0, 1
 
 
@@ -382,15 +383,16 @@ def tb_beam_reset(batch: Batch):
     _check(_lib.tb_beam_reset(batch.handle), "tb_beam_reset")
 
 
-def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_stride: int, new_frame: bool,
+def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_stride: int, new_frame,
                  scores: torch.Tensor, states: torch.Tensor, live: torch.Tensor, out_parent: torch.Tensor,
                  out_token: torch.Tensor, stream=None, offset: int = 0):
     """logits: any tensor; hypothesis k of stream i reads vocab+1 contiguous elements at element
-    offset ``offset + i*stream_stride + k*hyp_stride``.  scores/states/live [B, K] are updated in place."""
+    offset ``offset + i*stream_stride + k*hyp_stride``.  scores/states/live [B, K] are updated in place.
+    new_frame: False / True, or one of TB_FRAME_SAME / TB_FRAME_NEW / TB_FRAME_NEW_MERGE."""
     B, K = scores.shape
     ptr = _vp(logits.data_ptr() + offset * logits.element_size())
     _check(_lib.tb_beam_step(batch.handle, ptr, _logit_dtype(logits), B, K, stream_stride, hyp_stride,
-                             1 if new_frame else 0, _dp(scores), _dp(states), _dp(live), _dp(out_parent),
+                             int(new_frame), _dp(scores), _dp(states), _dp(live), _dp(out_parent),
                              _dp(out_token), _stream(stream)), "tb_beam_step")
 
 

@@ -78,6 +78,9 @@ struct tb_batch {
   uint32_t flags = 0;
   int32_t* d_status = nullptr;
   int2* d_tree = nullptr;
+  unsigned long long* d_hyp_hash = nullptr;   // [2][n_slots * max_beam]: token-sequence hash of every beam hypothesis, ping-pong
+  int32_t* d_hyp_len = nullptr;               // [2][n_slots * max_beam]: its length
+  int64_t beam_steps = 0;                     // steps since tb_beam_reset (selects the ping-pong half)
   int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
   ArenaAllocator alloc;
   std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
@@ -105,7 +108,7 @@ static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len);
   for (auto& s : b->staging) {
     if (s.host) cudaFreeHost(s.host);
     if (s.done) cudaEventDestroy(s.done);
@@ -150,7 +153,12 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   ok = ok && cudaMalloc(&b->d_status, sizeof(int32_t)) == cudaSuccess;
   if (ok && max_tree_steps > 0)
     ok = cudaMalloc(&b->d_tree, sizeof(int2) * static_cast<size_t>(max_tree_steps) * n_slots * max_beam) == cudaSuccess;
+  const size_t n_hyp = static_cast<size_t>(n_slots) * max_beam;
+  ok = ok && cudaMalloc(&b->d_hyp_hash, 2 * n_hyp * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_hyp_len, 2 * n_hyp * sizeof(int32_t)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); destroy_batch(b); return TB_ERR_OOM; }
+  ok = ok && cudaMemset(b->d_hyp_hash, 0, 2 * n_hyp * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMemset(b->d_hyp_len, 0, 2 * n_hyp * sizeof(int32_t)) == cudaSuccess;
   // every slot starts unbound: n_states = 0, streaming state = {-1, 0, 0, 0, 0, 0}
   std::vector<TbSlotState> init(n_slots);
   for (auto& s : init) { std::memset(&s, 0, sizeof s); s.state = -1; }
@@ -408,6 +416,17 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
 extern "C" int tb_beam_reset(tb_batch* b) {
   if (!b) return TB_ERR_INVALID_ARG;
   b->tree_steps = 0; b->tree_B = 0; b->tree_K = 0;
+  // every hypothesis starts from the empty token sequence (hash 0, length 0): stream-ordered on the default stream,
+  // like the caller's own initialisation of the score / state arrays
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  b->beam_steps = 0;
+  if (cudaMemset(b->d_hyp_hash, 0, 2 * n_hyp * sizeof(unsigned long long)) != cudaSuccess ||
+      cudaMemset(b->d_hyp_len, 0, 2 * n_hyp * sizeof(int32_t)) != cudaSuccess) {
+    cudaGetLastError();
+    return TB_ERR_CUDA;
+  }
   return TB_OK;
 }
 
@@ -423,12 +442,21 @@ extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t 
   TbBeamParams p;
   std::memset(&p, 0, sizeof p);
   p.logits = logits; p.dtype = dtype; p.B = B; p.K = K; p.V = b->vocab; p.C = b->n_classes;
-  p.new_frame = new_frame; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = hyp_stride;
+  if (new_frame < 0 || new_frame > TB_FRAME_NEW_MERGE) return TB_ERR_INVALID_ARG;
+  {
+    const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+    const size_t in = (b->beam_steps & 1) ? n_hyp : 0, out = (b->beam_steps & 1) ? 0 : n_hyp;
+    p.hash_in = b->d_hyp_hash + in; p.hash_out = b->d_hyp_hash + out;
+    p.len_in = b->d_hyp_len + in; p.len_out = b->d_hyp_len + out;
+    p.merge = new_frame == TB_FRAME_NEW_MERGE ? 1 : 0;
+  }
+  p.new_frame = new_frame != 0; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = hyp_stride;
   p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;
   p.tree = b->d_tree; p.slots = b->d_slots; p.arena = b->arena; p.cls = b->d_cls; p.status = b->d_status;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   int rc = tb_launch_beam_step(p, static_cast<cudaStream_t>(stream_));
+  if (rc == TB_OK) b->beam_steps++;
   if (rc == TB_OK && b->d_tree) { b->tree_steps++; b->tree_B = B; b->tree_K = K; }
   return rc;
 }

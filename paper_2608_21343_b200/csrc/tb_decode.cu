@@ -217,6 +217,8 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   __shared__ float h_score[TB_MAX_BEAM];
   __shared__ int32_t h_state[TB_MAX_BEAM];
   __shared__ uint8_t h_live[TB_MAX_BEAM];
+  __shared__ unsigned long long h_hash[TB_MAX_BEAM];   // identity of the hypothesis' token sequence
+  __shared__ int32_t h_len[TB_MAX_BEAM];
   __shared__ BeamKey sel[TB_MAX_BEAM];
 
   const int b = blockIdx.x;
@@ -248,8 +250,23 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     h_score[threadIdx.x] = sc;
     h_state[threadIdx.x] = p.states[o];
     h_live[threadIdx.x] = p.new_frame ? static_cast<uint8_t>(sc != -INFINITY) : p.live[o];
+    h_hash[threadIdx.x] = p.hash_in[o];
+    h_len[threadIdx.x] = p.len_in[o];
   }
   __syncthreads();
+  if (p.merge) {
+    // hypotheses that have emitted the same token sequence are one transcript: the first in selection order (the
+    // best) stays, the others become empty places before anything is expanded
+    bool dup = false;
+    if (threadIdx.x < K && h_score[threadIdx.x] != -INFINITY) {
+      const int k = threadIdx.x;
+      for (int j = 0; j < k; ++j)
+        if (h_score[j] != -INFINITY && h_len[j] == h_len[k] && h_hash[j] == h_hash[k] && h_state[j] == h_state[k]) { dup = true; break; }
+    }
+    __syncthreads();
+    if (dup) { h_score[threadIdx.x] = -INFINITY; h_state[threadIdx.x] = -1; h_live[threadIdx.x] = 0; }
+    __syncthreads();
+  }
 
   // all candidate values of the live hypotheses
   if (use_tv) {
@@ -385,6 +402,20 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     }
     p.scores[o] = sc; p.states[o] = state; p.live[o] = lv;
     p.out_parent[o] = parent; p.out_token[o] = token;
+    {
+      unsigned long long nh = 0ull;
+      int32_t nl = 0;
+      if (parent >= 0) {
+        nh = h_hash[parent]; nl = h_len[parent];
+        if (token >= 0 && token != V) {          // one more token: a 64-bit mix of the sequence so far and the token
+          nh = (nh ^ static_cast<unsigned long long>(token + 1)) * 0xff51afd7ed558ccdull;
+          nh ^= nh >> 33;
+          nh += 0x9e3779b97f4a7c15ull;
+          ++nl;
+        }
+      }
+      p.hash_out[o] = nh; p.len_out[o] = nl;
+    }
     if (p.tree) p.tree[(static_cast<int64_t>(p.step) * p.B + b) * K + r] = make_int2(parent, token);
   }
 }

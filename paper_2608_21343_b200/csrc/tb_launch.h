@@ -30,6 +30,9 @@ struct TbBeamParams {
   int64_t stream_stride, hyp_stride;
   float* scores; int32_t* states; uint8_t* live; int32_t* out_parent; int32_t* out_token;
   int2* tree;                // [steps, B, K] (parent, token) or null
+  // identity of every hypothesis' token sequence (64-bit hash and length), read from *_in, written to *_out
+  const unsigned long long* hash_in; unsigned long long* hash_out; const int32_t* len_in; int32_t* len_out;
+  int32_t merge;             // at this frame start, hypotheses with equal token sequences are merged first
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
 };
 

@@ -10,7 +10,7 @@ from helpers import SCORE_TOL, make_batch, oracle_graph, to_device, to_host
 pytestmark = pytest.mark.gpu
 
 
-def run_beam(tb, w, data, K, phrase_lists=None, batch=None):
+def run_beam(tb, w, data, K, phrase_lists=None, batch=None, merge=False):
     """Frame-synchronous driver: E = w.S rows per frame shared by all hypotheses of a stream.
     (batch: one made by the caller, with slot i bound unless phrase_lists[i] is None)"""
     phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
@@ -31,7 +31,8 @@ def run_beam(tb, w, data, K, phrase_lists=None, batch=None):
     sb, st, se, _ = logits.stride()
     for t in range(T):
         for e in range(E):
-            tb.tb_beam_step(batch, logits, sb, 0, e == 0, scores, states, live, par, tok, offset=t * st + e * se)
+            frame = (tb.TB_FRAME_NEW_MERGE if merge else tb.TB_FRAME_NEW) if e == 0 else tb.TB_FRAME_SAME
+            tb.tb_beam_step(batch, logits, sb, 0, frame, scores, states, live, par, tok, offset=t * st + e * se)
             tree.append(torch.stack([par, tok], dim=-1).clone())
     toks, lens = tb.tb_beam_backtrace(batch, B, K, T * E)
     assert tb.tb_batch_status(batch) == 0
@@ -40,10 +41,10 @@ def run_beam(tb, w, data, K, phrase_lists=None, batch=None):
                 tree=torch.stack(tree, dim=1).cpu().numpy(), tokens=toks.cpu().numpy(), lens=lens.cpu().numpy())
 
 
-def compare_beam(w, data, out, K, streams, phrase_lists=None):
+def compare_beam(w, data, out, K, streams, phrase_lists=None, merge=False):
     phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
     for i in streams:
-        ref = O.beam_decode(oracle_graph(w, phrase_lists[i]), data["logits"][i], K)
+        ref = O.beam_decode(oracle_graph(w, phrase_lists[i]), data["logits"][i], K, merge=merge)
         assert np.array_equal(out["tree"][i], ref["tree"]), f"stream {i}: (parent, token) tree"
         assert np.array_equal(out["states"][i], ref["states"]), f"stream {i}: states"
         assert np.array_equal(out["lens"][i], ref["lens"]), f"stream {i}: lengths"
@@ -61,6 +62,47 @@ def test_workload4_beam_reduced(tb):
     lists[2] = None
     out = run_beam(tb, w, data, w.K, lists)
     compare_beam(w, data, out, w.K, range(w.B), lists)
+
+
+def _competing_alignments(w, seed):
+    """Logits on which alignments of the same short transcript compete for the beam: a token costs about 2 against
+    blank in the first row of a frame, the second row closes the frame, noise of 0.3 decides the rest."""
+    rng = np.random.default_rng(seed)
+    x = (rng.standard_normal((w.B, w.T, w.S, w.V + 1)) * 0.3).astype(np.float32)
+    x[:, :, 0, w.V] += 2.0
+    x[:, :, 1:, :w.V] -= 2.0
+    return x
+
+
+@pytest.mark.parametrize("K", [8, 32])
+def test_beam_with_merging_of_equal_sequences(tb, K):
+    w = W.get_workload(1, B=4, T=12, S=2, V=8, n_plants=0)
+    data = W.batch_inputs(w)
+    data["logits"] = _competing_alignments(w, 5)
+    lists = [None, data["phrases"][1], None, data["phrases"][3]]
+    batch, _ = make_batch(tb, w, lists, lam=0.125, max_beam=K, max_tree_steps=w.T * w.S)
+    out = run_beam(tb, w, data, K, lists, batch=batch, merge=True)
+    changed = 0
+    for i in range(w.B):
+        g = oracle_graph(w, lists[i], lam=0.125)
+        ref = O.beam_decode(g, data["logits"][i], K, merge=True)
+        assert np.array_equal(out["tree"][i], ref["tree"]), f"stream {i}: (parent, token) tree"
+        assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"])
+        for k in range(K):
+            assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
+        fin = np.isfinite(ref["scores"])
+        assert np.array_equal(np.isfinite(out["scores"][i]), fin)
+        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
+        changed += not np.array_equal(ref["tree"], O.beam_decode(g, data["logits"][i], K)["tree"])
+    assert changed >= 3                       # on these inputs merging does change what the beam holds
+
+
+def test_beam_merging_is_off_unless_asked_for(tb):
+    w = W.get_workload(1, B=2, T=10, S=2, V=8, n_plants=0)
+    data = W.batch_inputs(w)
+    data["logits"] = _competing_alignments(w, 6)
+    out = run_beam(tb, w, data, 16, [None, None])
+    compare_beam(w, data, out, 16, range(w.B), [None, None])
 
 
 @pytest.mark.parametrize("K", [1, 2, 7])
