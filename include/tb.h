@@ -324,8 +324,8 @@ int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots,
 
 /*
  * Forget the hypothesis tree (step counter = 0) and the per-hypothesis record of emitted token sequences (every
- * hypothesis starts from the empty sequence).  Call before the first step of an utterance; the clearing is
- * ordered on the device's default stream.  Across the chunks of one utterance simply keep calling
+ * hypothesis starts from the empty sequence).  Call before the first step of an utterance (host bookkeeping only:
+ * no device work, so it may sit inside a stream capture).  Across the chunks of one utterance simply keep calling
  * tb_beam_step: scores, states, liveness (the caller's arrays), the tree and the sequence records carry over.
  */
 int tb_beam_reset(tb_batch *b);

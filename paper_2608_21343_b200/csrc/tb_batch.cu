@@ -416,17 +416,8 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
 extern "C" int tb_beam_reset(tb_batch* b) {
   if (!b) return TB_ERR_INVALID_ARG;
   b->tree_steps = 0; b->tree_B = 0; b->tree_K = 0;
-  // every hypothesis starts from the empty token sequence (hash 0, length 0): stream-ordered on the default stream,
-  // like the caller's own initialisation of the score / state arrays
-  DeviceGuard guard(b->device);
-  if (!guard.ok) return TB_ERR_CUDA;
-  const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  // every hypothesis starts from the empty token sequence: the first step after this ignores the stored records
   b->beam_steps = 0;
-  if (cudaMemset(b->d_hyp_hash, 0, 2 * n_hyp * sizeof(unsigned long long)) != cudaSuccess ||
-      cudaMemset(b->d_hyp_len, 0, 2 * n_hyp * sizeof(int32_t)) != cudaSuccess) {
-    cudaGetLastError();
-    return TB_ERR_CUDA;
-  }
   return TB_OK;
 }
 
@@ -449,6 +440,7 @@ extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t 
     p.hash_in = b->d_hyp_hash + in; p.hash_out = b->d_hyp_hash + out;
     p.len_in = b->d_hyp_len + in; p.len_out = b->d_hyp_len + out;
     p.merge = new_frame == TB_FRAME_NEW_MERGE ? 1 : 0;
+    p.fresh = b->beam_steps == 0 ? 1 : 0;
   }
   p.new_frame = new_frame != 0; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = hyp_stride;
   p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;

@@ -250,8 +250,8 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     h_score[threadIdx.x] = sc;
     h_state[threadIdx.x] = p.states[o];
     h_live[threadIdx.x] = p.new_frame ? static_cast<uint8_t>(sc != -INFINITY) : p.live[o];
-    h_hash[threadIdx.x] = p.hash_in[o];
-    h_len[threadIdx.x] = p.len_in[o];
+    h_hash[threadIdx.x] = p.fresh ? 0ull : p.hash_in[o];
+    h_len[threadIdx.x] = p.fresh ? 0 : p.len_in[o];
   }
   __syncthreads();
   if (p.merge) {
