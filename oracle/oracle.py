@@ -91,10 +91,10 @@ def lib():
         _lib.orc_beam_step.restype = None
         _lib.orc_beam_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_int32,
                                        C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
-        _lib.orc_beam_decode_merge.restype = C.c_int
-        _lib.orc_beam_decode_merge.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
-                                               C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
-                                               C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.orc_beam_decode_opts.restype = C.c_int
+        _lib.orc_beam_decode_opts.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
+                                              C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p,
+                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.orc_beam_decode.restype = C.c_int
         _lib.orc_beam_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -277,9 +277,10 @@ def beam_step(graph, rows_logits: np.ndarray, scores, states, live):
     return par, tok
 
 
-def beam_decode(graph, logits: np.ndarray, K: int, max_len=None, merge: bool = False):
+def beam_decode(graph, logits: np.ndarray, K: int, max_len=None, merge: bool = False, prune_delta: float = -1.0):
     """Frame-synchronous beam decode of one stream.  logits [T, E, V+1].
     merge: hypotheses with equal token sequences are merged at every frame start (the best is kept).
+    prune_delta >= 0: at every frame start hypotheses scoring below best - prune_delta are dropped.
 
     Returns dict(tokens=list of K arrays, lens, scores, states, tree [T*E, K, 2])."""
     T, E, V1 = logits.shape
@@ -290,9 +291,9 @@ def beam_decode(graph, logits: np.ndarray, K: int, max_len=None, merge: bool = F
     states = np.zeros(K, dtype=np.int32)
     tree = np.zeros((T * E, K, 2), dtype=np.int32)
     st = _strides3(logits)
-    rc = lib().orc_beam_decode_merge(graph.handle if graph is not None else None, _ptr(logits), _dtype_code(logits),
-                                     T, E, V1 - 1, _ptr(st), K, max_len, 1 if merge else 0, _ptr(out_tokens),
-                                     _ptr(lens), _ptr(scores), _ptr(states), _ptr(tree))
+    rc = lib().orc_beam_decode_opts(graph.handle if graph is not None else None, _ptr(logits), _dtype_code(logits),
+                                    T, E, V1 - 1, _ptr(st), K, max_len, 1 if merge else 0, float(prune_delta),
+                                    _ptr(out_tokens), _ptr(lens), _ptr(scores), _ptr(states), _ptr(tree))
     assert rc == 0
     return dict(tokens=[out_tokens[k, :min(lens[k], max_len)].copy() for k in range(K)], lens=lens,
                 scores=scores, states=states, tree=tree)

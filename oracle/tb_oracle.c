@@ -513,10 +513,15 @@ void orc_beam_step(const orc_graph *g, const void *logits, int dtype, const int6
  * READING: merging happens where the hypotheses are in the same situation -- all live, at a frame start -- so
  * that equal sequences have equal futures and keeping the best loses nothing (the result is, per token
  * sequence, the best alignment, as long as the beam is wide enough).
+ * prune_delta >= 0 (Sec. 2.3: ... and pruning): after the merge, still at the frame start, every hypothesis
+ * whose score is below (best score - prune_delta), one rounded subtraction, becomes an empty place.
+ * READING: the paper names pruning only; a threshold relative to the best hypothesis is the usual rule.
+ * A negative prune_delta switches it off.
  */
-int orc_beam_decode_merge(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
-                          const int64_t *strides, int32_t K, int32_t max_len, int32_t merge, int32_t *out_tokens,
-                          int32_t *out_lens, float *out_scores, int32_t *out_states, int32_t *tree) {
+int orc_beam_decode_opts(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
+                         const int64_t *strides, int32_t K, int32_t max_len, int32_t merge, float prune_delta,
+                         int32_t *out_tokens, int32_t *out_lens, float *out_scores, int32_t *out_states,
+                         int32_t *tree) {
   float *scores = (float *)malloc((size_t)K * sizeof(float));
   int32_t *states = (int32_t *)malloc((size_t)K * sizeof(int32_t));
   uint8_t *live = (uint8_t *)malloc((size_t)K);
@@ -544,6 +549,13 @@ int orc_beam_decode_merge(const orc_graph *g, const void *logits, int dtype, int
           break;
         }
       }
+    }
+    if (prune_delta >= 0.0f) {
+      float best = -INFINITY;
+      for (int32_t k = 0; k < K; ++k) if (scores[k] > best) best = scores[k];
+      float floor_ = best - prune_delta;
+      for (int32_t k = 0; k < K; ++k)
+        if (scores[k] != -INFINITY && scores[k] < floor_) { scores[k] = -INFINITY; states[k] = -1; live[k] = 0; }
     }
     for (int32_t k = 0; k < K; ++k) live[k] = (uint8_t)(scores[k] != -INFINITY);
     for (int32_t e = 0; e < E; ++e, ++step) {
@@ -582,6 +594,6 @@ int orc_beam_decode_merge(const orc_graph *g, const void *logits, int dtype, int
 int orc_beam_decode(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t E, int32_t V,
                     const int64_t *strides, int32_t K, int32_t max_len, int32_t *out_tokens,
                     int32_t *out_lens, float *out_scores, int32_t *out_states, int32_t *tree) {
-  return orc_beam_decode_merge(g, logits, dtype, T, E, V, strides, K, max_len, 0, out_tokens, out_lens, out_scores,
-                               out_states, tree);
+  return orc_beam_decode_opts(g, logits, dtype, T, E, V, strides, K, max_len, 0, -1.0f, out_tokens, out_lens,
+                              out_scores, out_states, tree);
 }

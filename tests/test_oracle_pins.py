@@ -696,3 +696,50 @@ def test_beam_with_merging_keeps_the_best_alignment_of_every_sequence(seed):
     # without merging the same run keeps every alignment
     r0 = O.beam_decode(g, x, K)
     assert int(np.isfinite(r0["scores"]).sum()) == K > len(got)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_beam_pruning_reductions_and_brute_force(seed):
+    """Pruning at frame starts against what does not use the beam code: a threshold of infinity changes nothing;
+    a threshold of 0 with one row per frame leaves one hypothesis per frame, i.e. the beam of one (greedy);
+    and with room for everything the survivors are the alignments whose prefixes, frame by frame, stayed
+    within the threshold of the best surviving prefix (set recursion over exhaustive enumeration)."""
+    rng = np.random.default_rng(700 + seed)
+    V, T, E = 3, 3, 2
+    phrases = [[0, 1], [1], [2, 0, 1]][: 2 + seed % 2]
+    g = O.Graph(phrases, V)
+    br = Brute(phrases)
+    x = dyadic_logits(rng, (T, E, V + 1), q=1 << 16)
+    K = 13 ** 3
+    r_inf = O.beam_decode(g, x, K, prune_delta=float("inf"))
+    r_off = O.beam_decode(g, x, K)
+    assert np.array_equal(r_inf["tree"], r_off["tree"]) and np.array_equal(r_inf["scores"], r_off["scores"])
+    x1 = np.ascontiguousarray(x[:, :1])                         # one row per frame: every step starts a frame
+    r0 = O.beam_decode(g, x1, 5, prune_delta=0.0)
+    r1 = O.beam_decode(g, x1, 1)
+    assert list(r0["tokens"][0]) == list(r1["tokens"][0]) and r0["scores"][0] == r1["scores"][0]
+    # brute force: per frame, extend every surviving history by every alignment of that frame, then prune
+    delta = 1.5
+    per_frame = []
+    for t in range(T):
+        opts = []
+
+        def rec(e, toks, raw):
+            if e == E:
+                opts.append((toks, raw)); return
+            opts.append((toks, raw + [float(x[t, e, V])]))
+            for v in range(V):
+                rec(e + 1, toks + [v], raw + [float(x[t, e, v])])
+        rec(0, [], [])
+        per_frame.append(opts)
+    alive = [((), 0.0)]                                         # (history, raw logit sum); the bonus comes from Brute
+    for t in range(T):
+        total = [(h, raw + br.G(list(h))) for h, raw in alive]
+        best = max(s for _, s in total)
+        alive = [(h, raw) for (h, raw), (_, s) in zip(alive, total) if s >= best - delta]
+        alive = [(h + tuple(toks), raw + sum(rw)) for h, raw in alive for toks, rw in per_frame[t]]
+    want = sorted(((raw + br.G(list(h)), h) for h, raw in alive), key=lambda p: (-p[0], p[1]))
+    r = O.beam_decode(g, x, K, prune_delta=delta)
+    got = [(float(r["scores"][k]), tuple(int(v) for v in r["tokens"][k])) for k in range(K) if np.isfinite(r["scores"][k])]
+    assert sorted(got, key=lambda p: (-p[0], p[1])) == want
+    assert 0 < len(got) < K
