@@ -359,6 +359,15 @@ int tb_beam_step(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t 
                  int32_t *out_parent, int32_t *out_token, void *stream);
 
 /*
+ * Pruning of the beam (Sec. 2.3 names it; the rule here is the usual threshold against the best hypothesis):
+ * with delta >= 0, every tb_beam_step that starts a frame (TB_FRAME_NEW, TB_FRAME_NEW_MERGE) first -- after
+ * the merge, if one was asked for -- turns every hypothesis of a stream whose score is below
+ * fl(best score of the stream - delta) into an empty place.  A negative delta (the default) switches it off;
+ * +inf prunes nothing.  Errors: TB_ERR_INVALID_ARG (NULL, NaN).
+ */
+int tb_batch_set_beam_prune(tb_batch *b, float delta);
+
+/*
  * End of stream: charge every hypothesis the final weight of the graph state it stops in (Sec. 2.2 para. 2
  * lists a final weight per state; it is the loan of the unfinished partial match, negated, so a finished
  * hypothesis keeps the bonus of the phrases it completed and nothing else):

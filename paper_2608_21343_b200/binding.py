@@ -77,6 +77,7 @@ _SIGS = {
     "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
     "tb_apply_final_weights": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
+    "tb_batch_set_beam_prune": (C.c_int, [_vp, C.c_float]),
     "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
                                            _vp, _vp, _vp]),
 }
@@ -394,6 +395,10 @@ def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_str
     _check(_lib.tb_beam_step(batch.handle, ptr, _logit_dtype(logits), B, K, stream_stride, hyp_stride,
                              int(new_frame), _dp(scores), _dp(states), _dp(live), _dp(out_parent),
                              _dp(out_token), _stream(stream)), "tb_beam_step")
+
+
+def tb_batch_set_beam_prune(batch: Batch, delta: float):
+    _check(_lib.tb_batch_set_beam_prune(batch.handle, float(delta)), "tb_batch_set_beam_prune")
 
 
 def tb_apply_final_weights(batch: Batch, scores: torch.Tensor, states: torch.Tensor, stream=None):

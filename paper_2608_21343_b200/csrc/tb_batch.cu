@@ -81,6 +81,7 @@ struct tb_batch {
   unsigned long long* d_hyp_hash = nullptr;   // [2][n_slots * max_beam]: token-sequence hash of every beam hypothesis, ping-pong
   int32_t* d_hyp_len = nullptr;               // [2][n_slots * max_beam]: its length
   int64_t beam_steps = 0;                     // steps since tb_beam_reset (selects the ping-pong half)
+  float beam_prune_delta = -1.0f;             // >= 0: prune at frame starts (tb_batch_set_beam_prune)
   int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
   ArenaAllocator alloc;
   std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
@@ -383,6 +384,12 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
 }
 
+extern "C" int tb_batch_set_beam_prune(tb_batch* b, float delta) {
+  if (!b || delta != delta) return TB_ERR_INVALID_ARG;
+  b->beam_prune_delta = delta >= 0.0f ? delta : -1.0f;
+  return TB_OK;
+}
+
 extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* scores, const int32_t* states,
                                       void* stream_) {
   if (!b || !scores || !states || B < 1 || B > b->n_slots || K < 1) return TB_ERR_INVALID_ARG;
@@ -441,6 +448,7 @@ extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t 
     p.len_in = b->d_hyp_len + in; p.len_out = b->d_hyp_len + out;
     p.merge = new_frame == TB_FRAME_NEW_MERGE ? 1 : 0;
     p.fresh = b->beam_steps == 0 ? 1 : 0;
+    p.prune_delta = new_frame != 0 ? b->beam_prune_delta : -1.0f;
   }
   p.new_frame = new_frame != 0; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = hyp_stride;
   p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;

@@ -267,6 +267,19 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     if (dup) { h_score[threadIdx.x] = -INFINITY; h_state[threadIdx.x] = -1; h_live[threadIdx.x] = 0; }
     __syncthreads();
   }
+  if (p.prune_delta >= 0.0f) {
+    // still at the frame start: whatever scores below the best by more than the threshold becomes an empty place
+    bool drop = false;
+    if (threadIdx.x < K) {
+      float best = -INFINITY;
+      for (int j = 0; j < K; ++j) best = fmaxf(best, h_score[j]);
+      const float sc = h_score[threadIdx.x];
+      drop = sc != -INFINITY && sc < __fsub_rn(best, p.prune_delta);
+    }
+    __syncthreads();
+    if (drop) { h_score[threadIdx.x] = -INFINITY; h_state[threadIdx.x] = -1; h_live[threadIdx.x] = 0; }
+    __syncthreads();
+  }
 
   // all candidate values of the live hypotheses
   if (use_tv) {

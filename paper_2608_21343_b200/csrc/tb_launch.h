@@ -33,6 +33,7 @@ struct TbBeamParams {
   // identity of every hypothesis' token sequence (64-bit hash and length), read from *_in, written to *_out
   const unsigned long long* hash_in; unsigned long long* hash_out; const int32_t* len_in; int32_t* len_out;
   int32_t merge;             // at this frame start, hypotheses with equal token sequences are merged first
+  float prune_delta;         // >= 0: at a frame start, hypotheses scoring below best - prune_delta are dropped
   int32_t fresh;             // first step after a reset: every hypothesis has the empty sequence, *_in is not read
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
 };

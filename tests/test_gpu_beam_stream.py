@@ -10,13 +10,15 @@ from helpers import SCORE_TOL, make_batch, oracle_graph, to_device, to_host
 pytestmark = pytest.mark.gpu
 
 
-def run_beam(tb, w, data, K, phrase_lists=None, batch=None, merge=False):
+def run_beam(tb, w, data, K, phrase_lists=None, batch=None, merge=False, prune_delta=None):
     """Frame-synchronous driver: E = w.S rows per frame shared by all hypotheses of a stream.
     (batch: one made by the caller, with slot i bound unless phrase_lists[i] is None)"""
     phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
     B, T, E, Wd = data["logits"].shape
     if batch is None:
         batch, _ = make_batch(tb, w, phrase_lists, max_beam=K, max_tree_steps=T * E)
+    if prune_delta is not None:
+        tb.tb_batch_set_beam_prune(batch, prune_delta)
     logits = to_device(data["logits"])
     dev = logits.device
     scores = torch.full((B, K), float("-inf"), device=dev)
@@ -95,6 +97,31 @@ def test_beam_with_merging_of_equal_sequences(tb, K):
         assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
         changed += not np.array_equal(ref["tree"], O.beam_decode(g, data["logits"][i], K)["tree"])
     assert changed >= 3                       # on these inputs merging does change what the beam holds
+
+
+@pytest.mark.parametrize("delta,merge", [(0.5, False), (1.5, True), (0.0, True), (float("inf"), False)])
+def test_beam_with_pruning(tb, delta, merge):
+    w = W.get_workload(1, B=4, T=12, S=2, V=8, n_plants=0)
+    data = W.batch_inputs(w)
+    data["logits"] = _competing_alignments(w, 7)
+    lists = [None, data["phrases"][1], None, data["phrases"][3]]
+    K = 16
+    batch, _ = make_batch(tb, w, lists, lam=0.125, max_beam=K, max_tree_steps=w.T * w.S)
+    out = run_beam(tb, w, data, K, lists, batch=batch, merge=merge, prune_delta=delta)
+    changed = 0
+    for i in range(w.B):
+        g = oracle_graph(w, lists[i], lam=0.125)
+        ref = O.beam_decode(g, data["logits"][i], K, merge=merge, prune_delta=delta)
+        assert np.array_equal(out["tree"][i], ref["tree"]), f"stream {i}: (parent, token) tree"
+        assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"])
+        fin = np.isfinite(ref["scores"])
+        assert np.array_equal(np.isfinite(out["scores"][i]), fin)
+        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
+        changed += not np.array_equal(ref["tree"], O.beam_decode(g, data["logits"][i], K, merge=merge)["tree"])
+    assert (changed >= 2) == (delta < 10)     # a finite threshold bites on these inputs, an infinite one never
+    tb.tb_batch_set_beam_prune(batch, -1.0)
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_set_beam_prune(batch, float("nan"))
 
 
 def test_beam_merging_is_off_unless_asked_for(tb):
