@@ -226,9 +226,20 @@ def side_measurement(args):
             graph_ms = timed(cg.replay, max(2, args.steps // 5), 1)
         except Exception as exc:  # noqa: BLE001
             graph_ms = f"capture failed: {exc}"
+        # ... and the whole utterance in one launch (each stream's block loops over its expansions)
+        l4 = logits.view(B, T, E, -1)
+
+        def run_fused():
+            scores.fill_(float("-inf")); scores[:, 0] = 0.0
+            states.fill_(-1); states[:, 0] = 0
+            tb.tb_beam_reset(batch)
+            tb.tb_beam_frames(batch, l4, False, scores, states, live, par, tok)
+        fused_ms = timed(run_fused, max(2, args.steps // 5), 1)
+        assert tb.tb_batch_status(batch) == 0
         print(json.dumps({"metric": "beam_decode_frames_per_s_K4_B32", "value": B * T / (ms * 1e-3), "unit": UNIT,
                           "ms_per_decode": ms, "us_per_beam_step": ms * 1e3 / (T * E), "n_gpus": 1,
-                          "cuda_graph_ms_per_decode": graph_ms,
+                          "cuda_graph_ms_per_decode": graph_ms, "one_launch_ms_per_decode": fused_ms,
+                          "one_launch_frames_per_s": B * T / (fused_ms * 1e-3),
                           "config": {"workload": w.name, "B": B, "K": K, "T": T, "E": E,
                                      "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
     elif args.workload == 5:

@@ -359,6 +359,19 @@ int tb_beam_step(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t 
                  int32_t *out_parent, int32_t *out_token, void *stream);
 
 /*
+ * T frames of E expansions each in ONE launch (Sec. 2.3: fully GPU-based decoding without a host round trip per
+ * step): exactly the sequence of tb_beam_step calls in which every hypothesis of stream i reads the row at element
+ * offset i*stream_stride + t*frame_stride + e*row_stride (hyp_stride 0) and the first row of every frame is given
+ * TB_FRAME_NEW, or TB_FRAME_NEW_MERGE when `merge` is non-zero; pruning as set by tb_batch_set_beam_prune.  Each
+ * stream's block loops over its own expansions.  The tree receives T*E steps; out_parent / out_token hold those of
+ * the last one.  A chunk of a longer utterance is one such call; the next call continues from the arrays.
+ * Errors: as tb_beam_step (the tree must have room for T*E more steps).
+ */
+int tb_beam_frames(tb_batch *b, const void *logits, int dtype, int32_t B, int32_t K, int32_t T, int32_t E,
+                   int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge, float *scores,
+                   int32_t *states, uint8_t *live, int32_t *out_parent, int32_t *out_token, void *stream);
+
+/*
  * Pruning of the beam (Sec. 2.3 names it; the rule here is the usual threshold against the best hypothesis):
  * with delta >= 0, every tb_beam_step that starts a frame (TB_FRAME_NEW, TB_FRAME_NEW_MERGE) first -- after
  * the merge, if one was asked for -- turns every hypothesis of a stream whose score is below

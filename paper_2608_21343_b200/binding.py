@@ -76,6 +76,8 @@ _SIGS = {
     "tb_beam_reset": (C.c_int, [_vp]),
     "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "tb_beam_frames": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
+                                 _vp]),
     "tb_apply_final_weights": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "tb_batch_set_beam_prune": (C.c_int, [_vp, C.c_float]),
     "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -395,6 +397,17 @@ def tb_beam_step(batch: Batch, logits: torch.Tensor, stream_stride: int, hyp_str
     _check(_lib.tb_beam_step(batch.handle, ptr, _logit_dtype(logits), B, K, stream_stride, hyp_stride,
                              int(new_frame), _dp(scores), _dp(states), _dp(live), _dp(out_parent),
                              _dp(out_token), _stream(stream)), "tb_beam_step")
+
+
+def tb_beam_frames(batch: Batch, logits: torch.Tensor, merge: bool, scores: torch.Tensor, states: torch.Tensor,
+                   live: torch.Tensor, out_parent: torch.Tensor, out_token: torch.Tensor, stream=None):
+    """logits [B, T, E, V+1] (any strides with a contiguous last dimension): T frames of E expansions in one launch."""
+    B, K = scores.shape
+    assert logits.dim() == 4 and logits.shape[0] == B and logits.stride(3) == 1
+    sb, st, se, _ = logits.stride()
+    _check(_lib.tb_beam_frames(batch.handle, _dp(logits), _logit_dtype(logits), B, K, logits.shape[1], logits.shape[2],
+                               sb, st, se, 1 if merge else 0, _dp(scores), _dp(states), _dp(live), _dp(out_parent),
+                               _dp(out_token), _stream(stream)), "tb_beam_frames")
 
 
 def tb_batch_set_beam_prune(batch: Batch, delta: float):

@@ -461,6 +461,42 @@ extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t 
   return rc;
 }
 
+extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_t B, int32_t K, int32_t T, int32_t E,
+                              int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge,
+                              float* scores, int32_t* states, uint8_t* live, int32_t* out_parent, int32_t* out_token,
+                              void* stream_) {
+  if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
+  if ((dtype != TB_BF16 && dtype != TB_F32) || B < 1 || B > b->n_slots || K < 1 || K > b->max_beam || T < 1 || E < 1 ||
+      static_cast<int64_t>(T) * E > (1 << 24))
+    return TB_ERR_INVALID_ARG;
+  const int32_t n_steps = T * E;
+  if (b->d_tree) {
+    if (b->tree_steps + n_steps > b->max_tree_steps) return TB_ERR_INVALID_ARG;
+    if (b->tree_steps > 0 && (b->tree_B != B || b->tree_K != K)) return TB_ERR_INVALID_ARG;
+  }
+  TbBeamParams p;
+  std::memset(&p, 0, sizeof p);
+  p.logits = logits; p.dtype = dtype; p.B = B; p.K = K; p.V = b->vocab; p.C = b->n_classes;
+  {
+    const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+    const size_t in = (b->beam_steps & 1) ? n_hyp : 0, out = (b->beam_steps & 1) ? 0 : n_hyp;
+    p.hash_in = b->d_hyp_hash + in; p.hash_out = b->d_hyp_hash + out;
+    p.len_in = b->d_hyp_len + in; p.len_out = b->d_hyp_len + out;
+    p.merge = merge ? 1 : 0;
+    p.fresh = b->beam_steps == 0 ? 1 : 0;
+    p.prune_delta = b->beam_prune_delta;
+  }
+  p.new_frame = 1; p.step = b->tree_steps; p.stream_stride = stream_stride; p.hyp_stride = 0;
+  p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;
+  p.tree = b->d_tree; p.slots = b->d_slots; p.arena = b->arena; p.cls = b->d_cls; p.status = b->d_status;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  int rc = tb_launch_beam_frames(p, T, E, frame_stride, row_stride, static_cast<cudaStream_t>(stream_));
+  if (rc == TB_OK) b->beam_steps += n_steps;
+  if (rc == TB_OK && b->d_tree) { b->tree_steps += n_steps; b->tree_B = B; b->tree_K = K; }
+  return rc;
+}
+
 extern "C" int tb_beam_backtrace(tb_batch* b, int32_t B, int32_t K, int32_t max_len, int32_t* out_tokens,
                                  int32_t* out_lens, void* stream_) {
   if (!b || !out_tokens || !out_lens || max_len < 1) return TB_ERR_INVALID_ARG;

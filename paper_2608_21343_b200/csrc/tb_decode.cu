@@ -59,6 +59,15 @@ __device__ inline void tokview_init(TokView& tv, unsigned char* mem, int V, int 
   }
   __syncthreads();
 }
+// The same tables, already filled by an earlier tokview_init of this block with the same arguments.
+__device__ inline void tokview_attach(TokView& tv, unsigned char* mem, int V, int C) {
+  tv.rootcw = reinterpret_cast<float*>(mem);
+  tv.rootdst = reinterpret_cast<int32_t*>(mem + 4 * static_cast<size_t>(C));
+  tv.tok_lb = reinterpret_cast<float*>(mem + 8 * static_cast<size_t>(C));
+  tv.tok_dst = reinterpret_cast<int32_t*>(mem + 8 * static_cast<size_t>(C) + 4 * static_cast<size_t>(V));
+  tv.cur_tok = reinterpret_cast<uint16_t*>(mem + 8 * static_cast<size_t>(C) + 8 * static_cast<size_t>(V));
+  tv.n = 0; tv.D = 0.0f;
+}
 // Block-wide: replace the scattered list by that of state s (the root's list is empty, D = 0).
 __device__ inline void tokview_enter(TokView& tv, const unsigned char* blob, const TbSlotRec& rec, int32_t s, int V,
                                      int32_t* status) {
@@ -198,8 +207,9 @@ struct BeamKey {  // order: value descending, token key ascending, parent ascend
   float v;
   int32_t tkey, par;
 };
+// One beam expansion of the block's stream (the body of k_beam_step; k_beam_frames calls it once per row).
 template <typename LT>
-__global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
+__device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int V = p.V, K = p.K, W = V + 1;
   float* cand = reinterpret_cast<float*>(dyn);                         // [K, V+1]
@@ -242,7 +252,10 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
     }
   }
   TokView tv;
-  if (use_tv) tokview_init(tv, aux, V, p.C, g);
+  if (use_tv) {
+    if (p.tv_ready) tokview_attach(tv, aux, V, p.C);      // a later step of the same launch: the root tables are there
+    else tokview_init(tv, aux, V, p.C, g);
+  }
 
   if (threadIdx.x < K) {
     const int64_t o = static_cast<int64_t>(b) * K + threadIdx.x;
@@ -433,6 +446,36 @@ __global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
   }
 }
 
+template <typename LT>
+__global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
+  beam_step_body<LT>(p);
+}
+
+// T frames of E rows in one launch: the block loops over the expansions of its stream; every hypothesis of the
+// stream reads row (t, e).  What a step leaves in global memory (scores, states, liveness, sequence records) is read
+// back in the next step by the thread that wrote it.
+template <typename LT>
+__global__ void __launch_bounds__(kThreads) k_beam_frames(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
+                                                          int64_t row_stride) {
+  for (int32_t t = 0; t < T; ++t) {
+    for (int32_t e = 0; e < E; ++e) {
+      const int32_t sidx = t * E + e;
+      TbBeamParams q = p;
+      q.logits = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
+      q.hyp_stride = 0;
+      q.new_frame = e == 0 ? 1 : 0;
+      q.merge = e == 0 ? p.merge : 0;
+      q.prune_delta = e == 0 ? p.prune_delta : -1.0f;
+      q.fresh = (p.fresh && sidx == 0) ? 1 : 0;
+      q.tv_ready = sidx > 0 ? 1 : 0;
+      q.step = p.step + sidx;
+      if (sidx & 1) { q.hash_in = p.hash_out; q.hash_out = const_cast<unsigned long long*>(p.hash_in); q.len_in = p.len_out; q.len_out = const_cast<int32_t*>(p.len_in); }
+      beam_step_body<LT>(q);
+      __syncthreads();
+    }
+  }
+}
+
 __global__ void k_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V,
                                  int32_t max_len, int32_t* out_tokens, int32_t* out_lens) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -508,6 +551,25 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
   } else {
     if ((rc = set_smem(k_beam_step<float>, smem)) != TB_OK) return rc;
     k_beam_step<float><<<p.B, kThreads, smem, stream>>>(p);
+  }
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
+                          cudaStream_t stream) {
+  TbBeamParams p = p_in;
+  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+  p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
+  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) + aux;
+  if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
+  int rc;
+  if (p.dtype == TB_BF16) {
+    if ((rc = set_smem(k_beam_frames<uint16_t>, smem)) != TB_OK) return rc;
+    k_beam_frames<uint16_t><<<p.B, kThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
+  } else {
+    if ((rc = set_smem(k_beam_frames<float>, smem)) != TB_OK) return rc;
+    k_beam_frames<float><<<p.B, kThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
   }
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }

@@ -34,6 +34,7 @@ struct TbBeamParams {
   const unsigned long long* hash_in; unsigned long long* hash_out; const int32_t* len_in; int32_t* len_out;
   int32_t merge;             // at this frame start, hypotheses with equal token sequences are merged first
   float prune_delta;         // >= 0: at a frame start, hypotheses scoring below best - prune_delta are dropped
+  int32_t tv_ready;          // set inside a multi-step launch: the block's root tables in shared memory are filled already
   int32_t fresh;             // first step after a reset: every hypothesis has the empty sequence, *_in is not read
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
 };
@@ -48,6 +49,8 @@ size_t tb_greedy_fast_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S
 int tb_launch_greedy_fast(const TbDecodeParams& p, int32_t max_cache_bytes, int32_t max_states, int32_t all_resolved,
                           void* scratch, size_t scratch_bytes, cudaStream_t stream);
 int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
+int tb_launch_beam_frames(const TbBeamParams& p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
+                          cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
 int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,

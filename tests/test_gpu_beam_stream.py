@@ -233,3 +233,66 @@ def test_streaming_rnnt_chunked_equals_offline(tb):
         assert toks[i] == list(zip(off["tokens"][i, :n], off["frames"][i, :n]))
         assert out["states"][i] == off["states"][i] and out["scores"][i] == off["scores"][i]
         assert out["cursors"][i] == w.T
+
+
+def run_beam_frames(tb, w, data, K, phrase_lists, batch, merge=False, chunks=(None,)):
+    """The same decode through tb_beam_frames: the whole utterance in one launch, or chunk by chunk."""
+    B, T, E, Wd = data["logits"].shape
+    logits = to_device(data["logits"])
+    dev = logits.device
+    scores = torch.full((B, K), float("-inf"), device=dev)
+    scores[:, 0] = 0.0
+    states = torch.full((B, K), -1, dtype=torch.int32, device=dev)
+    states[:, 0] = torch.tensor([0 if p is not None else -1 for p in phrase_lists], dtype=torch.int32, device=dev)
+    live = torch.zeros((B, K), dtype=torch.uint8, device=dev)
+    par = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tok = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tb.tb_beam_reset(batch)
+    t0 = 0
+    for n in chunks:
+        n = T - t0 if n is None else n
+        tb.tb_beam_frames(batch, logits[:, t0:t0 + n], merge, scores, states, live, par, tok)
+        t0 += n
+    assert t0 == T
+    toks, lens = tb.tb_beam_backtrace(batch, B, K, T * E)
+    assert tb.tb_batch_status(batch) == 0
+    torch.cuda.synchronize()
+    return dict(scores=scores.cpu().numpy(), states=states.cpu().numpy(), tokens=toks.cpu().numpy(), lens=lens.cpu().numpy(),
+                last=torch.stack([par, tok], dim=-1).cpu().numpy())
+
+
+@pytest.mark.parametrize("merge,chunks", [(False, (None,)), (True, (None,)), (True, (5, 1, 6)), (False, (1,) * 12)])
+def test_beam_frames_in_one_launch_equals_the_steps(tb, merge, chunks):
+    w = W.get_workload(1, B=4, T=12, S=2, V=8, n_plants=0)
+    data = W.batch_inputs(w)
+    data["logits"] = _competing_alignments(w, 8)
+    lists = [None, data["phrases"][1], None, data["phrases"][3]]
+    K = 16
+    batch, _ = make_batch(tb, w, lists, lam=0.125, max_beam=K, max_tree_steps=w.T * w.S)
+    tb.tb_batch_set_beam_prune(batch, 3.0)
+    out = run_beam_frames(tb, w, data, K, lists, batch, merge=merge, chunks=chunks)
+    for i in range(w.B):
+        ref = O.beam_decode(oracle_graph(w, lists[i], lam=0.125), data["logits"][i], K, merge=merge, prune_delta=3.0)
+        assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"])
+        assert np.array_equal(out["last"][i], ref["tree"][-1])
+        for k in range(K):
+            assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
+        fin = np.isfinite(ref["scores"])
+        assert np.array_equal(np.isfinite(out["scores"][i]), fin)
+        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
+
+
+def test_beam_frames_on_workload4_reduced(tb):
+    w = W.get_workload(4, B=5, T=60, n_plants=6)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[2] = None
+    batch, _ = make_batch(tb, w, lists, max_beam=w.K, max_tree_steps=w.T * w.S)
+    out = run_beam_frames(tb, w, data, w.K, lists, batch, chunks=(8,) * 7 + (4,))
+    for i in range(w.B):
+        ref = O.beam_decode(oracle_graph(w, lists[i]), data["logits"][i], w.K)
+        assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"])
+        for k in range(w.K):
+            assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
+        fin = np.isfinite(ref["scores"])
+        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
