@@ -208,8 +208,13 @@ struct BeamKey {  // order: value descending, token key ascending, parent ascend
   int32_t tkey, par;
 };
 // One beam expansion of the block's stream (the body of k_beam_step; k_beam_frames calls it once per row).
+constexpr int kBeamThreads = 512;   // threads of a beam block: more warps hide the latencies of its short dependent phases
+constexpr int kBeamPref = 5;   // elements of a shared row each thread may hold ahead of time (rows up to 5 * kBeamThreads wide)
+// xpre / xpre_valid: this thread's elements of the stream's shared row, fetched ahead by the previous step of the same
+// launch; next_row: where the next step's shared row starts (null: none), fetched while this step selects.
 template <typename LT>
-__device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
+__device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xpre)[kBeamPref], bool& xpre_valid,
+                                               const LT* next_row) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int V = p.V, K = p.K, W = V + 1;
   float* cand = reinterpret_cast<float*>(dyn);                         // [K, V+1]
@@ -223,7 +228,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
   __shared__ int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
   __shared__ int32_t h_beg[TB_MAX_BEAM], h_cnt[TB_MAX_BEAM];
   __shared__ float h_D[TB_MAX_BEAM];
-  __shared__ unsigned long long red64[kThreads / 32];
+  __shared__ unsigned long long red64[kBeamThreads / 32];
   __shared__ float h_score[TB_MAX_BEAM];
   __shared__ int32_t h_state[TB_MAX_BEAM];
   __shared__ uint8_t h_live[TB_MAX_BEAM];
@@ -240,14 +245,13 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
   const bool use_tv = bound && rec.n_rsent >= 0 && p.tokview;
   // rows shared by the hypotheses of a stream (hyp_stride 0) depend on nothing that is loaded below: fetch this
   // thread's elements now, so that their latency overlaps the loads of the slot record, states and lists
-  constexpr int kPref = 5;
-  const bool pref = use_tv && p.hyp_stride == 0 && W <= kPref * kThreads;
-  float xpre[kPref];
-  if (pref) {
+  constexpr int kPref = kBeamPref;
+  const bool pref = use_tv && p.hyp_stride == 0 && W <= kPref * kBeamThreads;
+  if (pref && !xpre_valid) {
     const LT* row0 = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
 #pragma unroll
     for (int j = 0; j < kPref; ++j) {
-      const int v = threadIdx.x + j * kThreads;
+      const int v = threadIdx.x + j * kBeamThreads;
       xpre[j] = v < W ? LogitLoad<LT>::at(row0 + v) : 0.0f;
     }
   }
@@ -258,13 +262,18 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
   }
 
   if (threadIdx.x < K) {
-    const int64_t o = static_cast<int64_t>(b) * K + threadIdx.x;
-    float sc = p.scores[o];
-    h_score[threadIdx.x] = sc;
-    h_state[threadIdx.x] = p.states[o];
-    h_live[threadIdx.x] = p.new_frame ? static_cast<uint8_t>(sc != -INFINITY) : p.live[o];
-    h_hash[threadIdx.x] = p.fresh ? 0ull : p.hash_in[o];
-    h_len[threadIdx.x] = p.fresh ? 0 : p.len_in[o];
+    if (p.tv_ready) {
+      // a later step of the same launch: the previous step left its hypotheses in shared memory
+      if (p.new_frame) h_live[threadIdx.x] = static_cast<uint8_t>(h_score[threadIdx.x] != -INFINITY);
+    } else {
+      const int64_t o = static_cast<int64_t>(b) * K + threadIdx.x;
+      float sc = p.scores[o];
+      h_score[threadIdx.x] = sc;
+      h_state[threadIdx.x] = p.states[o];
+      h_live[threadIdx.x] = p.new_frame ? static_cast<uint8_t>(sc != -INFINITY) : p.live[o];
+      h_hash[threadIdx.x] = p.fresh ? 0ull : p.hash_in[o];
+      h_len[threadIdx.x] = p.fresh ? 0 : p.len_in[o];
+    }
   }
   __syncthreads();
   if (p.merge) {
@@ -308,8 +317,8 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
     __syncthreads();
     const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
 #pragma unroll
-    for (int j = 0; j < (W + kThreads - 1) / kThreads && (!pref || j < kPref); ++j) {
-      const int v = threadIdx.x + j * kThreads;
+    for (int j = 0; j < (W + kBeamThreads - 1) / kBeamThreads && (!pref || j < kPref); ++j) {
+      const int v = threadIdx.x + j * kBeamThreads;
       if (v >= W) break;
       const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
       for (int k = 0; k < K; ++k) {
@@ -323,7 +332,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
     const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
     for (int k = 0; k < K; ++k) {
       if (h_score[k] == -INFINITY || !h_live[k]) continue;
-      for (int i = threadIdx.x; i < h_cnt[k]; i += kThreads) {
+      for (int i = threadIdx.x; i < h_cnt[k]; i += kBeamThreads) {
         const TbRsEnt e = ent[h_beg[k] + i];
         const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
         if (i < kBeamList) { hl_tok[k][i] = static_cast<uint16_t>(tk); hl_dst[k][i] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
@@ -341,7 +350,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
       const LT* row = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride +
                       static_cast<int64_t>(k) * p.hyp_stride;
       const float sc = h_score[k];
-      for (int v = threadIdx.x; v < W; v += kThreads) {
+      for (int v = threadIdx.x; v < W; v += kBeamThreads) {
         float x = LogitLoad<LT>::at(row + v);
         float val = (bound && v < V) ? __fadd_rn(x, __fmul_rn(g.lambda, bvec[__ldg(p.cls + v)])) : x;
         cand[static_cast<size_t>(k) * W + v] = __fadd_rn(sc, val);
@@ -362,20 +371,33 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
   };
   // best key below `limit` among this thread's candidates: tokens v = tid, tid + 256, ... of every live
   // hypothesis, plus (thread k) the carried candidate of a frozen hypothesis k
+  // the row of the next step is requested now: its trip from HBM overlaps the selection rounds
+  xpre_valid = false;
+  if (pref && next_row) {
+#pragma unroll
+    for (int j = 0; j < kPref; ++j) {
+      const int v = threadIdx.x + j * kBeamThreads;
+      xpre[j] = v < W ? LogitLoad<LT>::at(next_row + v) : 0.0f;
+    }
+    xpre_valid = true;
+  }
+  unsigned long long spare = 0ull;                            // this thread's second best key below the limit of its last scan
+  bool have_spare = false;
   auto scan_mine = [&](unsigned long long limit) -> unsigned long long {
-    unsigned long long m = 0ull;
+    unsigned long long m = 0ull, m2 = 0ull;
     for (int k = 0; k < K; ++k) {
       if (h_score[k] == -INFINITY) continue;
       if (!h_live[k]) {
-        if (threadIdx.x == k) { const unsigned long long kk = make_key(h_score[k], V + 1, k); if (kk < limit && kk > m) m = kk; }
+        if (threadIdx.x == k) { const unsigned long long kk = make_key(h_score[k], V + 1, k); if (kk < limit) { if (kk > m) { m2 = m; m = kk; } else if (kk > m2) m2 = kk; } }
         continue;
       }
       const float* ck = cand + static_cast<size_t>(k) * W;
-      for (int v = threadIdx.x; v < W; v += kThreads) {
+      for (int v = threadIdx.x; v < W; v += kBeamThreads) {
         const unsigned long long kk = make_key(ck[v], v, k);
-        if (kk < limit && kk > m) m = kk;
+        if (kk < limit) { if (kk > m) { m2 = m; m = kk; } else if (kk > m2) m2 = kk; }
       }
     }
+    spare = m2; have_spare = true;
     return m;
   };
   unsigned long long mine = scan_mine(~0ull);
@@ -387,7 +409,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
     __syncthreads();
     unsigned long long best = red64[0];
 #pragma unroll
-    for (int w2 = 1; w2 < kThreads / 32; ++w2) { const unsigned long long o = red64[w2]; if (o > best) best = o; }
+    for (int w2 = 1; w2 < kBeamThreads / 32; ++w2) { const unsigned long long o = red64[w2]; if (o > best) best = o; }
     __syncthreads();
     if (threadIdx.x == 0) {
       BeamKey c{-INFINITY, INT32_MAX, INT32_MAX};
@@ -398,18 +420,23 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
       }
       sel[r] = c;
     }
-    if (best != 0ull && mine == best) mine = scan_mine(best);   // this thread owned the pick: find its next best
+    if (best != 0ull && mine == best) {                          // this thread owned the pick: its next best
+      if (have_spare) { mine = spare; have_spare = false; }
+      else mine = scan_mine(best);
+    }
   }
   __syncthreads();
 
   // new hypotheses, the hypothesis tree
+  int32_t parent = -1, token = -1, state = -1;
+  uint8_t lv = 0;
+  float sc = -INFINITY;
+  unsigned long long nh = 0ull;
+  int32_t nl = 0;
   if (threadIdx.x < K) {
     const int r = threadIdx.x;
     const BeamKey c = sel[r];
     const int64_t o = static_cast<int64_t>(b) * K + r;
-    int32_t parent = -1, token = -1, state = -1;
-    uint8_t lv = 0;
-    float sc = -INFINITY;
     if (c.par != INT32_MAX) {
       parent = c.par; sc = c.v;
       token = (c.tkey == V + 1) ? -1 : c.tkey;
@@ -429,8 +456,6 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
     p.scores[o] = sc; p.states[o] = state; p.live[o] = lv;
     p.out_parent[o] = parent; p.out_token[o] = token;
     {
-      unsigned long long nh = 0ull;
-      int32_t nl = 0;
       if (parent >= 0) {
         nh = h_hash[parent]; nl = h_len[parent];
         if (token >= 0 && token != V) {          // one more token: a 64-bit mix of the sequence so far and the token
@@ -444,19 +469,30 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p) {
     }
     if (p.tree) p.tree[(static_cast<int64_t>(p.step) * p.B + b) * K + r] = make_int2(parent, token);
   }
+  // ... and in shared memory, for the next step of a launch that runs several (read by every thread above: wait)
+  __syncthreads();
+  if (threadIdx.x < K) {
+    h_score[threadIdx.x] = sc; h_state[threadIdx.x] = state; h_live[threadIdx.x] = lv;
+    h_hash[threadIdx.x] = nh; h_len[threadIdx.x] = nl;
+  }
 }
 
 template <typename LT>
-__global__ void __launch_bounds__(kThreads) k_beam_step(TbBeamParams p) {
-  beam_step_body<LT>(p);
+__global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
+  float xpre[kBeamPref];
+  bool xpre_valid = false;
+  beam_step_body<LT>(p, xpre, xpre_valid, static_cast<const LT*>(nullptr));
 }
 
 // T frames of E rows in one launch: the block loops over the expansions of its stream; every hypothesis of the
 // stream reads row (t, e).  What a step leaves in global memory (scores, states, liveness, sequence records) is read
 // back in the next step by the thread that wrote it.
 template <typename LT>
-__global__ void __launch_bounds__(kThreads) k_beam_frames(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
+__global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
                                                           int64_t row_stride) {
+  float xpre[kBeamPref];
+  bool xpre_valid = false;
+  const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(blockIdx.x) * p.stream_stride;
   for (int32_t t = 0; t < T; ++t) {
     for (int32_t e = 0; e < E; ++e) {
       const int32_t sidx = t * E + e;
@@ -470,7 +506,9 @@ __global__ void __launch_bounds__(kThreads) k_beam_frames(TbBeamParams p, int32_
       q.tv_ready = sidx > 0 ? 1 : 0;
       q.step = p.step + sidx;
       if (sidx & 1) { q.hash_in = p.hash_out; q.hash_out = const_cast<unsigned long long*>(p.hash_in); q.len_in = p.len_out; q.len_out = const_cast<int32_t*>(p.len_in); }
-      beam_step_body<LT>(q);
+      const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
+      const LT* next_row = nt < T ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
+      beam_step_body<LT>(q, xpre, xpre_valid, next_row);
       __syncthreads();
     }
   }
@@ -547,10 +585,10 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
   int rc;
   if (p.dtype == TB_BF16) {
     if ((rc = set_smem(k_beam_step<uint16_t>, smem)) != TB_OK) return rc;
-    k_beam_step<uint16_t><<<p.B, kThreads, smem, stream>>>(p);
+    k_beam_step<uint16_t><<<p.B, kBeamThreads, smem, stream>>>(p);
   } else {
     if ((rc = set_smem(k_beam_step<float>, smem)) != TB_OK) return rc;
-    k_beam_step<float><<<p.B, kThreads, smem, stream>>>(p);
+    k_beam_step<float><<<p.B, kBeamThreads, smem, stream>>>(p);
   }
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
@@ -566,10 +604,10 @@ int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_
   int rc;
   if (p.dtype == TB_BF16) {
     if ((rc = set_smem(k_beam_frames<uint16_t>, smem)) != TB_OK) return rc;
-    k_beam_frames<uint16_t><<<p.B, kThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
+    k_beam_frames<uint16_t><<<p.B, kBeamThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
   } else {
     if ((rc = set_smem(k_beam_frames<float>, smem)) != TB_OK) return rc;
-    k_beam_frames<float><<<p.B, kThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
+    k_beam_frames<float><<<p.B, kBeamThreads, smem, stream>>>(p, T, E, frame_stride, row_stride);
   }
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
