@@ -163,3 +163,37 @@ def test_final_weights_after_greedy_and_beam(tb):
     tb.tb_apply_final_weights(batch, torch.zeros((1, 1), device="cuda:0"), bad)
     assert tb.tb_batch_status(batch) == 2            # TB_STATUS_BAD_STATE: a state outside the graph is reported, not used
     assert tb.tb_batch_status(batch) == 0            # (reading the word clears it)
+
+
+def test_error_codes_of_the_beam_and_lifecycle_calls(tb):
+    w = W.get_workload(1, B=2, T=4, S=2, V=8, n_plants=0)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    K = 4
+    batch = tb.tb_batch_create(w.V, cc, 2, arena_bytes=1 << 20, max_beam=K, max_tree_steps=6)
+    logits = to_device(data["logits"])
+    dev = logits.device
+    scores = torch.full((2, K), float("-inf"), device=dev); scores[:, 0] = 0
+    states = torch.full((2, K), -1, dtype=torch.int32, device=dev)
+    live = torch.zeros((2, K), dtype=torch.uint8, device=dev)
+    par = torch.empty((2, K), dtype=torch.int32, device=dev); tok = torch.empty_like(par)
+
+    def code(fn, *a, **k):
+        with pytest.raises(tb.TbError) as e:
+            fn(*a, **k)
+        return e.value.code
+    tb.tb_beam_reset(batch)
+    assert code(tb.tb_beam_frames, batch, logits, False, scores, states, live, par, tok) == tb.TB_ERR_INVALID_ARG   # 8 steps, room for 6
+    tb.tb_beam_frames(batch, logits[:, :3], False, scores, states, live, par, tok)                                    # 6 steps fit
+    assert code(tb.tb_beam_frames, batch, logits[:, 3:], False, scores, states, live, par, tok) == tb.TB_ERR_INVALID_ARG
+    wide = torch.zeros((2, 8), device=dev)
+    assert code(tb.tb_beam_frames, batch, logits[:, :1], False, wide, torch.zeros((2, 8), dtype=torch.int32, device=dev),
+                torch.zeros((2, 8), dtype=torch.uint8, device=dev), torch.zeros((2, 8), dtype=torch.int32, device=dev),
+                torch.zeros((2, 8), dtype=torch.int32, device=dev)) == tb.TB_ERR_INVALID_ARG                          # K above max_beam
+    tb.tb_beam_reset(batch)
+    assert code(tb.tb_beam_step, batch, logits, logits.stride(0), 0, 3, scores, states, live, par, tok) == tb.TB_ERR_INVALID_ARG   # no such frame flag
+    three = torch.zeros((3, 1), device=dev)
+    assert code(tb.tb_apply_final_weights, batch, three, torch.zeros((3, 1), dtype=torch.int32, device=dev)) == tb.TB_ERR_INVALID_ARG   # more streams than slots
+    other = tb.tb_graph_compile([[1, 2]], w.V + 1)
+    assert code(tb.tb_batch_register_model, batch, other) == tb.TB_ERR_INVALID_ARG                                    # another vocabulary
+    assert tb.tb_batch_status(batch) == 0
