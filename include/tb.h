@@ -191,6 +191,8 @@ int tb_graph_load(const char *path, tb_graph **out);
  * graphs are dropped once `capacity_bytes` of host memory would be exceeded; a graph larger than that is
  * returned but not kept).  The returned graph is the caller's to release with tb_graph_free as usual; it
  * stays valid after the cache drops or is destroyed.  Calls on one cache may come from several threads.
+ * Graphs kept by a cache have their device blob page-locked (when a CUDA device is present), so binding them
+ * copies from the graph in place; the batch holds the graph until that copy is done.
  *   out_hit  host int32 or NULL.   Errors: as tb_graph_compile.
  * tb_cache_stats: any pointer may be NULL.
  */

@@ -60,11 +60,22 @@ struct Staging {
   size_t cap = 0;
   cudaEvent_t done = nullptr;
   bool pending = false;
+  tb_graph* held = nullptr;   // a pinned graph whose blob the pending copy reads: released once the copy is done
 };
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
+
+tb_graph::~tb_graph() {
+  if (pinned) { cudaHostUnregister(blob.data()); cudaGetLastError(); }
+}
+
+void tb_graph_pin(tb_graph* g) {
+  if (!g || g->pinned || g->blob.empty()) return;
+  if (cudaHostRegister(g->blob.data(), g->blob.size(), cudaHostRegisterDefault) == cudaSuccess) g->pinned = true;
+  else cudaGetLastError();
+}
 
 struct tb_batch {
   int device = 0;
@@ -111,6 +122,7 @@ static void destroy_batch(tb_batch* b) {
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
   cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len);
   for (auto& s : b->staging) {
+    if (s.held) tb_graph_free(s.held);
     if (s.host) cudaFreeHost(s.host);
     if (s.done) cudaEventDestroy(s.done);
   }
@@ -192,14 +204,20 @@ static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, siz
   b->next_staging = (b->next_staging + 1) % kStagingRing;
   bool ok = true;
   if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
-  if (ok && s.cap < g->blob.size()) {
+  if (s.held) { tb_graph_free(s.held); s.held = nullptr; }
+  if (ok && g->pinned) {
+    // the blob's pages are locked: the copy engine reads it in place; the graph is held until the copy is done
+    ok = cudaMemcpyAsync(b->arena + off, g->blob.data(), g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;
+    if (ok) { s.pending = true; s.held = const_cast<tb_graph*>(g); s.held->refs.fetch_add(1); }
+  } else if (ok && s.cap < g->blob.size()) {
     if (s.host) cudaFreeHost(s.host);
     s.host = nullptr; s.cap = 0;
     size_t want = round_up(g->blob.size() * 2, 1 << 16);
     ok = cudaMallocHost(&s.host, want) == cudaSuccess;
     if (ok) s.cap = want;
   }
-  if (ok) {
+  if (ok && !g->pinned) {
     std::memcpy(s.host, g->blob.data(), g->blob.size());
     ok = cudaMemcpyAsync(b->arena + off, s.host, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
     ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;

@@ -239,6 +239,7 @@ extern "C" int tb_cache_compile(tb_cache* c, const int32_t* phrase_tokens, const
         c->evictions++;
       }
       g->refs.fetch_add(1);
+      tb_graph_pin(g);                                            // it will be bound again: binds then copy from it in place
       c->lru.push_front({key, g, bytes});
       c->map[key] = c->lru.begin();
       c->used += bytes;

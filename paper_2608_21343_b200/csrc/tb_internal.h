@@ -25,8 +25,14 @@ struct tb_graph {
   int32_t off_strec = 0, off_tokent = 0, n_tokent = 0;
   int32_t off_rsrec = 0, off_rsent = 0, n_rsent = 0;  // resolved per-state lists (n_rsent < 0: not built)
   float d_max = 0.0f;                                  // largest |sum of suffix-link weights| over all states
-  std::atomic<int32_t> refs{1};                        // holders: the caller's handle, plus one per cache that keeps the graph
+  std::atomic<int32_t> refs{1};                        // holders: the caller's handle, one per cache that keeps the graph, one per copy in flight
+  bool pinned = false;                                 // the blob's pages are locked (tb_graph_pin): binds copy straight from it
+  ~tb_graph();
 };
+
+// Page-locks the blob of a graph that will be bound again and again (graphs kept by a cache), so that a bind can
+// hand it to the copy engine directly instead of going through the staging ring.  Does nothing without a device.
+void tb_graph_pin(tb_graph* g);
 
 // Two derived sections of the blob serve the pipelined kernel.  TbStateRec packs what a
 // suffix-link walk needs from one state into one 16-byte load; TbTokEnt lists, per state, its

@@ -99,6 +99,10 @@ def test_graphs_from_file_and_from_the_cache_decode_the_same(tb, tmp_path):
             g, hit = tb.tb_cache_compile(cache, p, w.V, case_class=cc)
             assert hit
         tb.tb_batch_bind_stream(batch, i, g)
+        g.free()                      # the caller's handle may go at once: a copy in flight keeps what it reads
+        if i == 2:
+            cache.destroy()           # ... and so may the cache that pinned the graph
+            cache = tb.tb_cache_create(8 << 20)
     cache.destroy()
     _decode_and_check(tb, w, batch, data, data["phrases"], "file / cache")
 
