@@ -316,16 +316,30 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
     }
     __syncthreads();
     const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+    if (pref) {
+      // the row sits in registers: every index below is a compile-time constant
 #pragma unroll
-    for (int j = 0; j < (W + kBeamThreads - 1) / kBeamThreads && (!pref || j < kPref); ++j) {
-      const int v = threadIdx.x + j * kBeamThreads;
-      if (v >= W) break;
-      const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
-      for (int k = 0; k < K; ++k) {
-        if (h_score[k] == -INFINITY || !h_live[k]) continue;
-        const float x = pref ? xpre[j < kPref ? j : 0] : LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
-        const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
-        cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+      for (int j = 0; j < kPref; ++j) {
+        const int v = threadIdx.x + j * kBeamThreads;
+        if (v < W) {
+          const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
+          const float x = xpre[j];
+          for (int k = 0; k < K; ++k) {
+            if (h_score[k] == -INFINITY || !h_live[k]) continue;
+            const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
+            cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+          }
+        }
+      }
+    } else {
+      for (int v = threadIdx.x; v < W; v += kBeamThreads) {
+        const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
+        for (int k = 0; k < K; ++k) {
+          if (h_score[k] == -INFINITY || !h_live[k]) continue;
+          const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
+          const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
+          cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+        }
       }
     }
     __syncthreads();
