@@ -11,6 +11,10 @@ happen once before the timed region (decoder-level registration in the paper's T
 Prints ONE JSON line.  With N > 1 (under torchrun) every rank decodes its own batch of 128
 independent streams (weak scaling, no collective on the data path; the only collective is the
 timing barrier / max).
+
+Side measurements, one JSON line each (not the headline): --workload 3 large lists, 4 beam decoding (step by
+step, under graph replay, and all expansions in one launch), 5 streaming TDT chunks with stream churn, 6 variative
+case-insensitive lists compiled from text, 7 model lifecycle sweep (cache: none / disk / memory / decoder).
 """
 from __future__ import annotations
 
