@@ -476,7 +476,10 @@ def main():
         p_ms, _ = timed(lambda: tb.tb_greedy_decode(plain, logits, out=out0), args.steps, args.warmup)
         p_ms /= args.steps
         result["unboosted"] = {"ms_per_step": p_ms, "frames_per_s": w.B * w.T / (p_ms * 1e-3),
-                               "boosted_overhead_pct": 100.0 * (total_ms / args.steps / p_ms - 1.0)}
+                               "boosted_overhead_pct": 100.0 * (total_ms / args.steps / p_ms - 1.0),
+                               # an unboosted decode streams every row once: the whole tensor over the launch time
+                               "all_rows_GBs": logits.numel() * logits.element_size() / (p_ms * 1e-3) / 1e9,
+                               "all_rows_frac_of_measured_peak": logits.numel() * logits.element_size() / (p_ms * 1e-3) / 1e9 / result["roofline"]["peak"]}
     if not args.no_extras and rank == 0:
         # end to end through the public call with host buffers: H2D of the logits, decode, D2H of results
         dl = torch.empty_like(logits)
