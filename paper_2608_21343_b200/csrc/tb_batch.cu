@@ -73,7 +73,8 @@ tb_graph::~tb_graph() {
 
 void tb_graph_pin(tb_graph* g) {
   if (!g || g->pinned || g->blob.empty()) return;
-  if (cudaHostRegister(g->blob.data(), g->blob.size(), cudaHostRegisterDefault) == cudaSuccess) g->pinned = true;
+  // (portable: whichever device's batch binds the graph later may copy from it)
+  if (cudaHostRegister(g->blob.data(), g->blob.size(), cudaHostRegisterPortable) == cudaSuccess) g->pinned = true;
   else cudaGetLastError();
 }
 
