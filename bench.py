@@ -324,7 +324,9 @@ def side_measurement(args):
                     elif mode == "memory":
                         tb.tb_batch_bind_stream(batch, sl, tb.tb_cache_compile(cache, p, w.V, case_class=cc)[0])
                     else:
-                        tb.tb_batch_bind_model(batch, sl, model_of[sid])
+                        break
+                if mode == "decoder" and bl:
+                    tb.tb_batch_bind_models(batch, [sl for sl, _, _ in bl], [model_of[sid] for _, sid, _ in bl])
                 tb.tb_stream_chunk(batch, dl, w.n_dur, dv)
                 torch.cuda.synchronize()
                 lat.append((time.perf_counter() - t0) * 1e3)
@@ -337,6 +339,54 @@ def side_measurement(args):
                          "frames_per_s": w.B * w.chunk * len(steady) / (float(steady.sum()) * 1e-3),
                          "binds_per_chunk": nb / len(steady)})
             batch.destroy()
+        # the same four levels around the offline decode of workload 2: every one of the 128 streams brings its own list
+        w2 = W.get_workload(2)
+        d2 = W.batch_inputs(w2)
+        cc2 = w2.vocab.case_class
+        l2 = torch.from_numpy(d2["logits"]).view(torch.bfloat16).to(dev)
+        flat2 = [flat(p) for p in d2["phrases"]]
+        rows2 = []
+        for mode in ("none", "disk", "memory", "decoder"):
+            batch = tb.tb_batch_create(w2.V, cc2, w2.B, arena_bytes=64 << 20)
+            cache, ids = None, []
+            if mode == "disk":
+                for i, p in enumerate(flat2):
+                    tb.tb_graph_save(tb.tb_graph_compile(p, w2.V, case_class=cc2), os.path.join(tmp, "w2_%d.tbg" % i))
+            elif mode == "memory":
+                cache = tb.tb_cache_create(1 << 30)
+                for p in flat2:
+                    tb.tb_cache_compile(cache, p, w2.V, case_class=cc2)
+            elif mode == "decoder":
+                ids = [tb.tb_batch_register_model(batch, tb.tb_graph_compile(p, w2.V, case_class=cc2)) for p in flat2]
+            out2 = tb.tb_greedy_decode(batch, l2)
+            torch.cuda.synchronize()
+            ts = []
+            all_slots = np.arange(w2.B, dtype=np.int32)
+            for _ in range(max(5, args.steps // 20)):
+                t0 = time.perf_counter()
+                for i, p in enumerate(flat2):
+                    if mode == "none":
+                        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, w2.V, case_class=cc2))
+                    elif mode == "disk":
+                        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_load(os.path.join(tmp, "w2_%d.tbg" % i)))
+                    elif mode == "memory":
+                        tb.tb_batch_bind_stream(batch, i, tb.tb_cache_compile(cache, p, w2.V, case_class=cc2)[0])
+                    else:
+                        break
+                if mode == "decoder":
+                    tb.tb_batch_bind_models(batch, all_slots, ids)
+                tb.tb_greedy_decode(batch, l2, out=out2)
+                torch.cuda.synchronize()
+                ts.append((time.perf_counter() - t0) * 1e3)
+            assert tb.tb_batch_status(batch) == 0
+            rows2.append({"cache": mode, "ms_per_batch": float(np.median(ts)), "frames_per_s": w2.B * w2.T / (float(np.median(ts)) * 1e-3)})
+            batch.destroy()
+        for r in rows2:
+            r["vs_decoder_level"] = r["frames_per_s"] / rows2[-1]["frames_per_s"]
+        print(json.dumps({"metric": "model_lifecycle_sweep_offline_greedy", "unit": UNIT, "n_gpus": 1, "rows": rows2,
+                          "config": {"workload": w2.name, "B": w2.B, "T": w2.T, "phrases_per_stream": 100,
+                                     "timed": "host wall clock per batch: obtain and bind all 128 streams' graphs, decode, synchronise"},
+                          "data": "synthetic"}))
         base = rows[-1]["frames_per_s"]
         for r in rows:
             r["vs_decoder_level"] = r["frames_per_s"] / base

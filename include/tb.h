@@ -250,6 +250,12 @@ int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *str
 int tb_batch_register_model(tb_batch *b, const tb_graph *g, int32_t *out_model_id, void *stream);
 int tb_batch_bind_model(tb_batch *b, int32_t slot, int32_t model_id, void *stream);
 int tb_batch_unregister_model(tb_batch *b, int32_t model_id);
+/*
+ * tb_batch_bind_model for n (slot, model id) pairs at once: one small launch per 256 pairs, which is what takes the
+ * update cost out of the decoding loop when many streams start together.  host int32 arrays; a slot may appear once.
+ * All pairs are checked before anything changes (TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG).
+ */
+int tb_batch_bind_models(tb_batch *b, int32_t n, const int32_t *slots, const int32_t *model_ids, void *stream);
 
 /*
  * Set behaviour flags of the batch (TB_FLAG_*; 0 = defaults).  With the defaults

@@ -65,6 +65,7 @@ _SIGS = {
     "tb_batch_register_model": (C.c_int, [_vp, _vp, C.POINTER(_i32), _vp]),
     "tb_batch_bind_model": (C.c_int, [_vp, _i32, _i32, _vp]),
     "tb_batch_unregister_model": (C.c_int, [_vp, _i32]),
+    "tb_batch_bind_models": (C.c_int, [_vp, _i32, _vp, _vp, _vp]),
     "tb_batch_create": (C.c_int, [_i32, _vp, _i32, _i32, _i32, C.c_size_t, C.c_int, C.POINTER(_vp)]),
     "tb_batch_destroy": (None, [_vp]),
     "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
@@ -251,6 +252,12 @@ def tb_batch_register_model(batch, graph: Graph, stream=None) -> int:
 
 def tb_batch_bind_model(batch, slot: int, model_id: int, stream=None):
     _check(_lib.tb_batch_bind_model(batch.handle, slot, model_id, _stream(stream)), "tb_batch_bind_model")
+
+
+def tb_batch_bind_models(batch, slots, model_ids, stream=None):
+    sl, ids = _host(slots, np.int32), _host(model_ids, np.int32)
+    assert sl.shape == ids.shape
+    _check(_lib.tb_batch_bind_models(batch.handle, len(sl), _hp(sl), _hp(ids), _stream(stream)), "tb_batch_bind_models")
 
 
 def tb_batch_unregister_model(batch, model_id: int):

@@ -110,6 +110,8 @@ struct tb_batch {
     uint8_t resolved = 1;
   };
   std::vector<Model> models;
+  TbSlotRec* d_model_recs = nullptr;                   // the registered models' records on the device, by model id
+  int32_t model_recs_cap = 0;
   std::vector<int32_t> slot_model;                     // registered model a slot is bound to, else -1
   Staging staging[kStagingRing];
   int next_staging = 0;
@@ -121,7 +123,7 @@ static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs);
   for (auto& s : b->staging) {
     if (s.held) tb_graph_free(s.held);
     if (s.host) cudaFreeHost(s.host);
@@ -284,7 +286,8 @@ extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* 
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   tb_batch::Model m;
-  int rc = upload_graph(b, g, static_cast<cudaStream_t>(stream_), &m.off, &m.bytes, &m.rec);
+  int rc;
+  rc = upload_graph(b, g, static_cast<cudaStream_t>(stream_), &m.off, &m.bytes, &m.rec);
   if (rc != TB_OK) return rc;
   m.live = true; m.n_states = g->n_states; m.cache_bytes = cache_bytes_of(g); m.resolved = g->n_rsent >= 0 ? 1 : 0;
   int32_t id = -1;
@@ -296,8 +299,58 @@ extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* 
     b->alloc.release(m.off, m.bytes);
     return TB_ERR_OOM;
   }
+  // the record also goes into the device table that tb_batch_bind_models reads (grown in powers of two; the old
+  // table is freed after a device-wide wait inside cudaFree, registration is not on the decoding loop)
+  if (id >= b->model_recs_cap) {
+    int32_t cap = b->model_recs_cap ? b->model_recs_cap : 256;
+    while (cap <= id) cap *= 2;
+    TbSlotRec* bigger = nullptr;
+    bool ok = cudaMalloc(&bigger, sizeof(TbSlotRec) * cap) == cudaSuccess;
+    ok = ok && cudaMemset(bigger, 0, sizeof(TbSlotRec) * cap) == cudaSuccess;
+    if (ok && b->model_recs_cap)
+      ok = cudaMemcpy(bigger, b->d_model_recs, sizeof(TbSlotRec) * b->model_recs_cap, cudaMemcpyDeviceToDevice) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); cudaFree(bigger); b->alloc.release(m.off, m.bytes); return TB_ERR_OOM; }
+    cudaFree(b->d_model_recs);
+    b->d_model_recs = bigger; b->model_recs_cap = cap;
+  }
+  rc = tb_launch_publish_model(b->d_model_recs, id, m.rec, static_cast<cudaStream_t>(stream_));
+  if (rc != TB_OK) { b->alloc.release(m.off, m.bytes); return rc; }
   b->models[id] = m;
   *out_model_id = id;
+  return TB_OK;
+}
+
+extern "C" int tb_batch_bind_models(tb_batch* b, int32_t n, const int32_t* slots, const int32_t* model_ids, void* stream_) {
+  if (!b || n < 0 || (n > 0 && (!slots || !model_ids))) return TB_ERR_INVALID_ARG;
+  // everything is checked before anything is changed
+  std::vector<uint8_t> seen(static_cast<size_t>(b->n_slots), 0);
+  for (int32_t i = 0; i < n; ++i) {
+    if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
+    if (seen[slots[i]]) return TB_ERR_INVALID_ARG;           // a slot twice in one call
+    seen[slots[i]] = 1;
+    const int32_t m = model_ids[i];
+    if (m < -1 || m >= static_cast<int32_t>(b->models.size()) || (m >= 0 && !b->models[m].live)) return TB_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  for (int32_t i0 = 0; i0 < n; i0 += TB_BIND_PAIRS) {
+    const int32_t cnt = n - i0 < TB_BIND_PAIRS ? n - i0 : TB_BIND_PAIRS;
+    int rc = tb_launch_bind_models(b->d_slots, b->d_sstate, b->d_model_recs, cnt, slots + i0, model_ids + i0,
+                                   static_cast<cudaStream_t>(stream_));
+    if (rc != TB_OK) return rc;
+    for (int32_t i = i0; i < i0 + cnt; ++i) {
+      const int32_t slot = slots[i], m = model_ids[i];
+      release_slot(b, slot);
+      if (m >= 0) {
+        b->models[m].users++;
+        b->slot_model[slot] = m;
+        b->slot_n_states[slot] = b->models[m].n_states; b->slot_cache_bytes[slot] = b->models[m].cache_bytes;
+        b->slot_resolved[slot] = b->models[m].resolved;
+      } else {
+        b->slot_n_states[slot] = 0; b->slot_cache_bytes[slot] = 0; b->slot_resolved[slot] = 1;
+      }
+    }
+  }
   return TB_OK;
 }
 

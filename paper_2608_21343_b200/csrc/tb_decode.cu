@@ -656,6 +656,38 @@ int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, 
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
+__global__ void k_publish_model(TbSlotRec* model_recs, int32_t model_id, TbSlotRec rec) {
+  if (threadIdx.x == 0) model_recs[model_id] = rec;
+}
+
+struct BindPairs { int32_t slot[TB_BIND_PAIRS]; int32_t model[TB_BIND_PAIRS]; };
+__global__ void k_bind_models(TbSlotRec* slots, TbSlotState* sstate, const TbSlotRec* model_recs, int32_t n, BindPairs pr) {
+  const int i = threadIdx.x;
+  if (i >= n) return;
+  TbSlotRec rec;
+  if (pr.model[i] >= 0) rec = model_recs[pr.model[i]];
+  else memset(&rec, 0, sizeof rec);
+  slots[pr.slot[i]] = rec;
+  TbSlotState st;
+  st.state = rec.n_states > 0 ? 0 : -1; st.t = 0; st.k = 0; st.score = 0.0f; st.n_emitted = 0;
+  st.chunk_base = 0; st.pad0 = 0; st.pad1 = 0;
+  sstate[pr.slot[i]] = st;
+}
+
+int tb_launch_publish_model(TbSlotRec* model_recs, int32_t model_id, const TbSlotRec& rec, cudaStream_t stream) {
+  k_publish_model<<<1, 32, 0, stream>>>(model_recs, model_id, rec);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_bind_models(TbSlotRec* slots, TbSlotState* sstate, const TbSlotRec* model_recs, int32_t n,
+                          const int32_t* slot_of, const int32_t* model_of, cudaStream_t stream) {
+  if (n < 1 || n > TB_BIND_PAIRS) return TB_ERR_INVALID_ARG;
+  BindPairs pr;
+  for (int i = 0; i < TB_BIND_PAIRS; ++i) { pr.slot[i] = i < n ? slot_of[i] : 0; pr.model[i] = i < n ? model_of[i] : -1; }
+  k_bind_models<<<1, TB_BIND_PAIRS, 0, stream>>>(slots, sstate, model_recs, n, pr);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
                            cudaStream_t stream) {
   k_publish_slot<<<1, 32, 0, stream>>>(slots, sstate, slot, rec);

@@ -53,6 +53,12 @@ int tb_launch_beam_frames(const TbBeamParams& p, int32_t T, int32_t E, int64_t f
                           cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
+// Registered models: their records live in a device table; tb_launch_bind_models points up to TB_BIND_PAIRS slots at
+// models of that table (id -1: unbound) and resets the slots' streaming state, in one launch.
+#define TB_BIND_PAIRS 256
+int tb_launch_publish_model(TbSlotRec* model_recs, int32_t model_id, const TbSlotRec& rec, cudaStream_t stream);
+int tb_launch_bind_models(TbSlotRec* slots, TbSlotState* sstate, const TbSlotRec* model_recs, int32_t n,
+                          const int32_t* slot_of, const int32_t* model_of, cudaStream_t stream);
 int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,
                             const int32_t* states, int32_t* status, cudaStream_t stream);
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,

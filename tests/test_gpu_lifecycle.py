@@ -201,3 +201,33 @@ def test_error_codes_of_the_beam_and_lifecycle_calls(tb):
     other = tb.tb_graph_compile([[1, 2]], w.V + 1)
     assert code(tb.tb_batch_register_model, batch, other) == tb.TB_ERR_INVALID_ARG                                    # another vocabulary
     assert tb.tb_batch_status(batch) == 0
+
+
+def test_binding_many_registered_models_at_once(tb):
+    w = W.get_workload(2, B=6, T=150)
+    data = W.batch_inputs(w)
+    cc = w.vocab.case_class
+    n_slots = 300                                       # more than one launch's worth of pairs
+    batch = tb.tb_batch_create(w.V, cc, n_slots, arena_bytes=4 << 20)
+    ids = [tb.tb_batch_register_model(batch, tb.tb_graph_compile(p, w.V, case_class=cc)) for p in data["phrases"]]
+    slots = list(range(n_slots))
+    models = [ids[i % 6] if i % 7 else -1 for i in range(n_slots)]
+    tb.tb_batch_bind_models(batch, slots, models)
+    lists = [None if models[i] < 0 else data["phrases"][models[i]] for i in range(6)]
+    _decode_and_check(tb, w, batch, data, lists, "bound at once")
+    # the last slots too: decode them through a strided view of the same logits
+    tb.tb_batch_bind_models(batch, [5, 0, 299], [ids[0], -1, ids[3]])
+    lists[5], lists[0] = data["phrases"][0], None
+    _decode_and_check(tb, w, batch, data, lists, "re-bound at once")
+
+    def code(*a):
+        with pytest.raises(tb.TbError) as e:
+            tb.tb_batch_bind_models(batch, *a)
+        return e.value.code
+    assert code([0, 1, 0], [ids[0], ids[1], ids[2]]) == tb.TB_ERR_INVALID_ARG      # a slot twice
+    assert code([0, 300], [ids[0], ids[1]]) == tb.TB_ERR_BAD_SLOT
+    assert code([0, 1], [ids[0], 77]) == tb.TB_ERR_INVALID_ARG
+    _decode_and_check(tb, w, batch, data, lists, "nothing changed by refused calls")
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_unregister_model(batch, ids[3])                               # slot 299 still uses it
+    tb.tb_batch_bind_models(batch, [], [])
