@@ -201,6 +201,12 @@ void tb_cache_destroy(tb_cache *c);
 int tb_cache_compile(tb_cache *c, const int32_t *phrase_tokens, const int64_t *phrase_offsets, int32_t n_phrases,
                      const float *token_weights, const int32_t *case_class, int32_t vocab, float lambda,
                      uint32_t flags, tb_graph **out, int32_t *out_hit);
+/* The same for tb_graph_compile_variative (the key holds the phrases' text, weights, tau, lambda and a checksum of
+ * the piece vocabulary). */
+int tb_cache_compile_variative(tb_cache *c, const uint8_t *phrase_chars, const int64_t *phrase_offsets,
+                               int32_t n_phrases, const float *phrase_weights, const uint8_t *piece_chars,
+                               const int64_t *piece_offsets, int32_t vocab, float tau, float lambda, uint32_t flags,
+                               tb_graph **out, int32_t *out_hit);
 int tb_cache_stats(tb_cache *c, int64_t *hits, int64_t *misses, int64_t *evictions, size_t *bytes_used,
                    int64_t *entries);
 

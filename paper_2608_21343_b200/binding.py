@@ -60,6 +60,8 @@ _SIGS = {
     "tb_cache_destroy": (None, [_vp]),
     "tb_cache_compile": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _i32, C.c_float, C.c_uint32, C.POINTER(_vp),
                                    C.POINTER(_i32)]),
+    "tb_cache_compile_variative": (C.c_int, [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _i32, C.c_float, C.c_float, C.c_uint32,
+                                             C.POINTER(_vp), C.POINTER(_i32)]),
     "tb_cache_stats": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(C.c_size_t),
                                  C.POINTER(_i64)]),
     "tb_batch_register_model": (C.c_int, [_vp, _vp, C.POINTER(_i32), _vp]),
@@ -240,6 +242,19 @@ def tb_cache_compile(cache: Cache, phrases, vocab: int, case_class=None, token_w
     h, hit = _vp(), _i32()
     _check(_lib.tb_cache_compile(cache.handle, _hp(toks), _hp(offs), n, _hp(w), _hp(cc), vocab, float(lam), flags,
                                  C.byref(h), C.byref(hit)), "tb_cache_compile")
+    return Graph(h), bool(hit.value)
+
+
+def tb_cache_compile_variative(cache: Cache, phrases, pieces, phrase_weights=None, tau: float = 1.0, lam: float = 1.0,
+                               flags: int = 0):
+    """Returns (graph, hit).  ``pieces`` may be the (bytes, offsets) pair made once by ``_flat_bytes``."""
+    pf, po = _flat_bytes(phrases)
+    vf, vo = pieces if isinstance(pieces, tuple) else _flat_bytes(pieces)
+    w = _host(phrase_weights, np.float32)
+    h, hit = _vp(), _i32()
+    _check(_lib.tb_cache_compile_variative(cache.handle, _hp(pf), _hp(po), len(phrases), _hp(w), _hp(vf), _hp(vo),
+                                           len(vo) - 1, float(tau), float(lam), flags, C.byref(h), C.byref(hit)),
+           "tb_cache_compile_variative")
     return Graph(h), bool(hit.value)
 
 

@@ -189,6 +189,39 @@ extern "C" int tb_cache_stats(tb_cache* c, int64_t* hits, int64_t* misses, int64
   return TB_OK;
 }
 
+// A hit hands out the cached graph with one more reference and makes it the most recently used.
+static bool cache_lookup(tb_cache* c, const std::string& key, tb_graph** out) {
+  std::lock_guard<std::mutex> lk(c->mu);
+  auto it = c->map.find(key);
+  if (it == c->map.end()) return false;
+  c->lru.splice(c->lru.begin(), c->lru, it->second);
+  it->second->g->refs.fetch_add(1);
+  *out = it->second->g;
+  c->hits++;
+  return true;
+}
+
+// Keeps a freshly compiled graph (the caller keeps its own reference), dropping the least recently used ones first.
+static void cache_insert(tb_cache* c, const std::string& key, tb_graph* g) {
+  const size_t bytes = graph_bytes(g) + key.size();
+  std::lock_guard<std::mutex> lk(c->mu);
+  c->misses++;
+  if (bytes > c->capacity || c->map.find(key) != c->map.end()) return;
+  while (c->used + bytes > c->capacity && !c->lru.empty()) {
+    auto& last = c->lru.back();
+    c->used -= last.bytes;
+    c->map.erase(last.key);
+    tb_graph_free(last.g);
+    c->lru.pop_back();
+    c->evictions++;
+  }
+  g->refs.fetch_add(1);
+  tb_graph_pin(g);                                              // it will be bound again: binds then copy from it in place
+  c->lru.push_front({key, g, bytes});
+  c->map[key] = c->lru.begin();
+  c->used += bytes;
+}
+
 extern "C" int tb_cache_compile(tb_cache* c, const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,
                                 const float* token_weights, const int32_t* case_class, int32_t vocab, float lambda,
                                 uint32_t flags, tb_graph** out, int32_t* out_hit) {
@@ -211,39 +244,51 @@ extern "C" int tb_cache_compile(tb_cache* c, const int32_t* phrase_tokens, const
     if (n_phrases > 0) key.append(reinterpret_cast<const char*>(phrase_offsets), sizeof(int64_t) * (static_cast<size_t>(n_phrases) + 1));
     if (n_tok) key.append(reinterpret_cast<const char*>(phrase_tokens), sizeof(int32_t) * n_tok);
     if (n_tok && token_weights) key.append(reinterpret_cast<const char*>(token_weights), sizeof(float) * n_tok);
-    {
-      std::lock_guard<std::mutex> lk(c->mu);
-      auto it = c->map.find(key);
-      if (it != c->map.end()) {
-        c->lru.splice(c->lru.begin(), c->lru, it->second);
-        it->second->g->refs.fetch_add(1);
-        *out = it->second->g;
-        if (out_hit) *out_hit = 1;
-        c->hits++;
-        return TB_OK;
-      }
-    }
+    if (cache_lookup(c, key, out)) { if (out_hit) *out_hit = 1; return TB_OK; }
     tb_graph* g = nullptr;
     int rc = tb_graph_compile(phrase_tokens, phrase_offsets, n_phrases, token_weights, case_class, vocab, lambda, flags, &g);
     if (rc != TB_OK) return rc;
-    const size_t bytes = graph_bytes(g) + key.size();
-    std::lock_guard<std::mutex> lk(c->mu);
-    c->misses++;
-    if (bytes <= c->capacity && c->map.find(key) == c->map.end()) {
-      while (c->used + bytes > c->capacity && !c->lru.empty()) {   // least recently used first
-        auto& last = c->lru.back();
-        c->used -= last.bytes;
-        c->map.erase(last.key);
-        tb_graph_free(last.g);
-        c->lru.pop_back();
-        c->evictions++;
-      }
-      g->refs.fetch_add(1);
-      tb_graph_pin(g);                                            // it will be bound again: binds then copy from it in place
-      c->lru.push_front({key, g, bytes});
-      c->map[key] = c->lru.begin();
-      c->used += bytes;
-    }
+    cache_insert(c, key, g);
+    *out = g;
+    return TB_OK;
+  } catch (const std::bad_alloc&) {
+    return TB_ERR_OOM;
+  }
+}
+
+extern "C" int tb_cache_compile_variative(tb_cache* c, const uint8_t* phrase_chars, const int64_t* phrase_offsets,
+                                          int32_t n_phrases, const float* phrase_weights, const uint8_t* piece_chars,
+                                          const int64_t* piece_offsets, int32_t vocab, float tau, float lambda,
+                                          uint32_t flags, tb_graph** out, int32_t* out_hit) {
+  if (!c || !out) return TB_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (out_hit) *out_hit = 0;
+  if (n_phrases < 0 || vocab < 1 || vocab > TB_MAX_VOCAB || !piece_offsets || piece_offsets[0] != 0 ||
+      piece_offsets[vocab] <= 0 || !piece_chars || (n_phrases > 0 && !phrase_offsets))
+    return TB_ERR_INVALID_ARG;
+  if (n_phrases > 0 && (phrase_offsets[0] != 0 || phrase_offsets[n_phrases] < 0 ||
+                        (phrase_offsets[n_phrases] > 0 && !phrase_chars)))
+    return TB_ERR_INVALID_ARG;
+  try {
+    const size_t n_ch = n_phrases > 0 ? static_cast<size_t>(phrase_offsets[n_phrases]) : 0;
+    const size_t n_pc = static_cast<size_t>(piece_offsets[vocab]);
+    std::string key("variative", 9);
+    const int32_t head[4] = {vocab, n_phrases, static_cast<int32_t>(flags), phrase_weights ? 1 : 0};
+    key.append(reinterpret_cast<const char*>(head), sizeof head);
+    key.append(reinterpret_cast<const char*>(&tau), sizeof tau);
+    key.append(reinterpret_cast<const char*>(&lambda), sizeof lambda);
+    // the vocabulary enters by a checksum of its spellings and boundaries (it is large and the same for every list)
+    const uint64_t vh = fnv1a(piece_offsets, sizeof(int64_t) * (static_cast<size_t>(vocab) + 1), fnv1a(piece_chars, n_pc));
+    key.append(reinterpret_cast<const char*>(&vh), sizeof vh);
+    if (n_phrases > 0) key.append(reinterpret_cast<const char*>(phrase_offsets), sizeof(int64_t) * (static_cast<size_t>(n_phrases) + 1));
+    if (n_ch) key.append(reinterpret_cast<const char*>(phrase_chars), n_ch);
+    if (n_phrases > 0 && phrase_weights) key.append(reinterpret_cast<const char*>(phrase_weights), sizeof(float) * static_cast<size_t>(n_phrases));
+    if (cache_lookup(c, key, out)) { if (out_hit) *out_hit = 1; return TB_OK; }
+    tb_graph* g = nullptr;
+    int rc = tb_graph_compile_variative(phrase_chars, phrase_offsets, n_phrases, phrase_weights, piece_chars, piece_offsets,
+                                        vocab, tau, lambda, flags, &g);
+    if (rc != TB_OK) return rc;
+    cache_insert(c, key, g);
     *out = g;
     return TB_OK;
   } catch (const std::bad_alloc&) {

@@ -274,3 +274,31 @@ def test_cache_is_safe_from_several_threads(tb):
     assert not errors
     st = cache.stats()
     assert st["hits"] + st["misses"] == 240 and st["entries"] == 8
+
+
+def test_cache_of_variative_lists(tb):
+    pieces = W.make_piece_vocab(3, letters=10, merged=60, max_len=4)
+    lists = [W.draw_string_phrases(30 + b, pieces, 40, 1, 4) for b in range(4)]
+    cache = tb.tb_cache_create(1 << 22)
+    first = []
+    for p in lists:
+        g, hit = tb.tb_cache_compile_variative(cache, p, pieces, tau=1.5)
+        assert not hit
+        _same_view(g.view(), tb.tb_graph_compile_variative(p, pieces, tau=1.5).view())
+        first.append(g)
+    for p, g0 in zip(lists, first):
+        g, hit = tb.tb_cache_compile_variative(cache, p, pieces, tau=1.5)
+        assert hit and g.handle.value == g0.handle.value
+    assert not tb.tb_cache_compile_variative(cache, lists[0], pieces, tau=0.5)[1]                    # tau is part of the key
+    assert not tb.tb_cache_compile_variative(cache, lists[0], pieces, tau=1.5, lam=2.0)[1]
+    assert not tb.tb_cache_compile_variative(cache, lists[0], pieces, tau=1.5, phrase_weights=[1.0] * 40)[1]
+    assert not tb.tb_cache_compile_variative(cache, lists[0], pieces[:-1] + [b"zz"], tau=1.5)[1]     # so is the vocabulary
+    assert not tb.tb_cache_compile_variative(cache, [p.upper() for p in lists[0]], pieces, tau=1.5)[1]   # the text as given
+    with pytest.raises(tb.TbError):
+        tb.tb_cache_compile_variative(cache, [b"\\x01"], pieces)
+    st = cache.stats()
+    assert st["hits"] == 4 and st["entries"] == 9
+    # token lists and text lists live side by side
+    w = W.get_workload(1)
+    assert not tb.tb_cache_compile(cache, W.stream_phrases(w, 0), w.V, case_class=w.vocab.case_class)[1]
+    assert tb.tb_cache_compile(cache, W.stream_phrases(w, 0), w.V, case_class=w.vocab.case_class)[1]
