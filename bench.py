@@ -479,8 +479,19 @@ def main():
     # the timed region alone can be shorter than one nvidia-smi sampling period)
     sampler = ClockSampler(local_rank)
     sampler.start()
+
+    def keep_busy(until, limit_s):
+        # untimed decodes, the same load as the timed ones, until the sampler has delivered enough lines
+        t_end = time.perf_counter() + limit_s
+        while not until() and time.perf_counter() < t_end:
+            for _ in range(20):
+                tb.tb_greedy_decode(batch, logits, out=out)
+            torch.cuda.synchronize()
+    keep_busy(lambda: len(sampler.rows) >= 1, 5.0)          # nvidia-smi takes a moment to come up
+    n_before = len(sampler.rows)
     timed(lambda: tb.tb_greedy_decode(batch, logits, out=out), max(50, args.steps), args.warmup)
     total_ms, each_ms = timed(lambda: tb.tb_greedy_decode(batch, logits, out=out), args.steps, args.warmup)
+    keep_busy(lambda: len(sampler.rows) - n_before >= 6, 3.0)   # the timed region can be shorter than a sampling period
     clocks = sampler.stop()
     assert tb.tb_batch_status(batch) == 0, "a kernel recorded a violated bound"
     job = sharding.job_throughput(w.B * w.T, total_ms / args.steps, device=dev)   # max over ranks of the time
