@@ -228,7 +228,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   __shared__ int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
   __shared__ int32_t h_beg[TB_MAX_BEAM], h_cnt[TB_MAX_BEAM];
   __shared__ float h_D[TB_MAX_BEAM];
-  __shared__ unsigned long long red64[kBeamThreads / 32];
+  __shared__ unsigned long long red64[2][kBeamThreads / 32];   // the warps' best keys, two copies used in turn by the selection rounds
   __shared__ float h_score[TB_MAX_BEAM];
   __shared__ int32_t h_state[TB_MAX_BEAM];
   __shared__ uint8_t h_live[TB_MAX_BEAM];
@@ -416,15 +416,15 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   };
   unsigned long long mine = scan_mine(~0ull);
   for (int r = 0; r < K; ++r) {
-    unsigned long long m = mine;
+    // the warp's best key: the largest high word, then the largest low word among the lanes that have it
+    const uint32_t hi = static_cast<uint32_t>(mine >> 32), lo = static_cast<uint32_t>(mine);
+    const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+    const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+    if (lane == 0) red64[r & 1][warp] = (static_cast<unsigned long long>(mh) << 32) | ml;
+    __syncthreads();                     // (one barrier per round: the next round writes the other copy)
+    unsigned long long best = red64[r & 1][0];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) { const unsigned long long o = __shfl_xor_sync(0xffffffffu, m, off); if (o > m) m = o; }
-    if (lane == 0) red64[warp] = m;
-    __syncthreads();
-    unsigned long long best = red64[0];
-#pragma unroll
-    for (int w2 = 1; w2 < kBeamThreads / 32; ++w2) { const unsigned long long o = red64[w2]; if (o > best) best = o; }
-    __syncthreads();
+    for (int w2 = 1; w2 < kBeamThreads / 32; ++w2) { const unsigned long long o = red64[r & 1][w2]; if (o > best) best = o; }
     if (threadIdx.x == 0) {
       BeamKey c{-INFINITY, INT32_MAX, INT32_MAX};
       if (best != 0ull) {
