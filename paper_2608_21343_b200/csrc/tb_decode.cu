@@ -561,7 +561,9 @@ __global__ void k_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t sl
 
 template <typename F>
 int set_smem(F* fn, size_t bytes) {
-  if (bytes > 48 * 1024) {
+  // (the default limit of 48 KB counts the kernel's static shared memory too -- up to 16 KB here -- so the opt-in
+  //  starts well below it)
+  if (bytes > 24 * 1024) {
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) != cudaSuccess) {
       cudaGetLastError();
       return TB_ERR_INVALID_ARG;

@@ -296,3 +296,16 @@ def test_beam_frames_on_workload4_reduced(tb):
             assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
         fin = np.isfinite(ref["scores"])
         assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
+
+
+@pytest.mark.parametrize("K", [8, 10, 12])
+def test_beam_widths_whose_shared_memory_straddles_the_default_limit(tb, K):
+    # V = 1024: K * (V + 1) floats plus the tables is 33-49 KB of dynamic shared memory, which together with the
+    # kernel's static 16 KB crosses the 48 KB a launch may use without opting in
+    w = W.get_workload(4, B=2, T=12, n_plants=2)
+    data = W.batch_inputs(w)
+    out = run_beam(tb, w, data, K)
+    compare_beam(w, data, out, K, range(w.B))
+    batch, _ = make_batch(tb, w, data["phrases"], max_beam=K, max_tree_steps=w.T * w.S)
+    fr = run_beam_frames(tb, w, data, K, data["phrases"], batch)
+    assert np.array_equal(fr["tokens"], out["tokens"]) and np.array_equal(fr["scores"], out["scores"])
