@@ -298,7 +298,7 @@ def test_beam_frames_on_workload4_reduced(tb):
         assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)
 
 
-@pytest.mark.parametrize("K", [8, 10, 12])
+@pytest.mark.parametrize("K", [8, 10, 12, 32])
 def test_beam_widths_whose_shared_memory_straddles_the_default_limit(tb, K):
     # V = 1024: K * (V + 1) floats plus the tables is 33-49 KB of dynamic shared memory, which together with the
     # kernel's static 16 KB crosses the 48 KB a launch may use without opting in
