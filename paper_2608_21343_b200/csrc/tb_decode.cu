@@ -218,7 +218,9 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   extern __shared__ __align__(16) unsigned char dyn[];
   const int V = p.V, K = p.K, W = V + 1;
   float* cand = reinterpret_cast<float*>(dyn);                         // [K, V+1]
-  unsigned char* aux = dyn + ((static_cast<size_t>(K) * W * sizeof(float) + 15) & ~size_t(15));
+  const int WW = (W + 31) >> 5;
+  uint32_t* ovr = reinterpret_cast<uint32_t*>(dyn + ((static_cast<size_t>(K) * W * sizeof(float) + 15) & ~size_t(15)));   // [K, WW] bits: the value in cand is a boosted one
+  unsigned char* aux = reinterpret_cast<unsigned char*>(ovr) + ((static_cast<size_t>(K) * WW * sizeof(uint32_t) + 15) & ~size_t(15));
   float* bvec = reinterpret_cast<float*>(aux);                         // [C]   (chain-walk path)
   int32_t* nvec = reinterpret_cast<int32_t*>(bvec + p.C);              // [C]
   __shared__ ChainSmem chain;
@@ -303,6 +305,16 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
     __syncthreads();
   }
 
+  auto make_key = [](float v, int tkey, int k) -> unsigned long long {
+    const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
+    const uint32_t hi = u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+    const uint32_t lo = 0xFFFFFFFFu - (static_cast<uint32_t>(tkey) * 32u + static_cast<uint32_t>(k));
+    return (static_cast<unsigned long long>(hi) << 32) | lo;
+  };
+  // this thread's two best candidates, when the sweep below has already looked at all of them
+  unsigned long long m1 = 0ull, m2 = 0ull;
+  bool swept = false;
+  auto offer = [&](unsigned long long kk) { if (kk > m1) { m2 = m1; m1 = kk; } else if (kk > m2) m2 = kk; };
   // all candidate values of the live hypotheses
   if (use_tv) {
     // every hypothesis at once: its state's record, then all plain values, then the listed tokens on top
@@ -314,8 +326,29 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
       h_beg[k] = r.begin; h_cnt[k] = r.count; h_D[k] = r.D;
       hl_n[k] = r.count <= kBeamList ? r.count : -1;
     }
+    for (int i = threadIdx.x; i < K * WW; i += kBeamThreads) ovr[i] = 0u;
     __syncthreads();
     const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+    // the boosted tokens of every hypothesis first: their values go to cand and are marked, so that the sweep over
+    // all candidates below leaves them alone -- and sees every candidate's final value, which lets each thread
+    // collect its best keys on the way instead of scanning cand again afterwards
+    {
+      const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
+      for (int k = 0; k < K; ++k) {
+        if (h_score[k] == -INFINITY || !h_live[k]) continue;
+        for (int i = threadIdx.x; i < h_cnt[k]; i += kBeamThreads) {
+          const TbRsEnt e = ent[h_beg[k] + i];
+          const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
+          if (i < kBeamList) { hl_tok[k][i] = static_cast<uint16_t>(tk); hl_dst[k][i] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
+          if (tk < V) {
+            const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + tk);
+            cand[static_cast<size_t>(k) * W + tk] = __fadd_rn(h_score[k], __fadd_rn(x, e.lb));
+            atomicOr(&ovr[k * WW + (tk >> 5)], 1u << (tk & 31));
+          }
+        }
+      }
+    }
+    __syncthreads();
     if (pref) {
       // the row sits in registers: every index below is a compile-time constant
 #pragma unroll
@@ -326,8 +359,15 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
           const float x = xpre[j];
           for (int k = 0; k < K; ++k) {
             if (h_score[k] == -INFINITY || !h_live[k]) continue;
-            const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
-            cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+            float c;
+            if ((ovr[k * WW + (v >> 5)] >> (v & 31)) & 1u) {
+              c = cand[static_cast<size_t>(k) * W + v];
+            } else {
+              const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
+              c = __fadd_rn(h_score[k], val);
+              cand[static_cast<size_t>(k) * W + v] = c;
+            }
+            offer(make_key(c, v, k));
           }
         }
       }
@@ -336,26 +376,22 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
         const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
         for (int k = 0; k < K; ++k) {
           if (h_score[k] == -INFINITY || !h_live[k]) continue;
-          const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
-          const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
-          cand[static_cast<size_t>(k) * W + v] = __fadd_rn(h_score[k], val);
+          float c;
+          if ((ovr[k * WW + (v >> 5)] >> (v & 31)) & 1u) {
+            c = cand[static_cast<size_t>(k) * W + v];
+          } else {
+            const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + v);
+            const float val = v < V ? __fadd_rn(x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], plain_w))) : x;
+            c = __fadd_rn(h_score[k], val);
+            cand[static_cast<size_t>(k) * W + v] = c;
+          }
+          offer(make_key(c, v, k));
         }
       }
     }
-    __syncthreads();
-    const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
-    for (int k = 0; k < K; ++k) {
-      if (h_score[k] == -INFINITY || !h_live[k]) continue;
-      for (int i = threadIdx.x; i < h_cnt[k]; i += kBeamThreads) {
-        const TbRsEnt e = ent[h_beg[k] + i];
-        const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
-        if (i < kBeamList) { hl_tok[k][i] = static_cast<uint16_t>(tk); hl_dst[k][i] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
-        if (tk < V) {
-          const float x = LogitLoad<LT>::at(base + static_cast<int64_t>(k) * p.hyp_stride + tk);
-          cand[static_cast<size_t>(k) * W + tk] = __fadd_rn(h_score[k], __fadd_rn(x, e.lb));
-        }
-      }
-    }
+    // a frozen hypothesis is carried as one candidate (thread k offers it)
+    if (threadIdx.x < K && h_score[threadIdx.x] != -INFINITY && !h_live[threadIdx.x]) offer(make_key(h_score[threadIdx.x], V + 1, threadIdx.x));
+    swept = true;
     __syncthreads();
   } else {
     for (int k = 0; k < K; ++k) {
@@ -377,12 +413,6 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   // parent ascending) is one 64-bit key: the order-preserving image of the value above the inverted
   // (token key, parent) pair; keys are distinct, 0 means "none".  Every thread keeps the best key among
   // its own candidates that has not been picked yet; after a round only the owner of the pick rescans.
-  auto make_key = [](float v, int tkey, int k) -> unsigned long long {
-    const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
-    const uint32_t hi = u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
-    const uint32_t lo = 0xFFFFFFFFu - (static_cast<uint32_t>(tkey) * 32u + static_cast<uint32_t>(k));
-    return (static_cast<unsigned long long>(hi) << 32) | lo;
-  };
   // best key below `limit` among this thread's candidates: tokens v = tid, tid + 256, ... of every live
   // hypothesis, plus (thread k) the carried candidate of a frozen hypothesis k
   // the row of the next step is requested now: its trip from HBM overlaps the selection rounds
@@ -414,7 +444,9 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
     spare = m2; have_spare = true;
     return m;
   };
-  unsigned long long mine = scan_mine(~0ull);
+  unsigned long long mine;
+  if (swept) { mine = m1; spare = m2; have_spare = true; }     // collected during the sweep
+  else mine = scan_mine(~0ull);
   for (int r = 0; r < K; ++r) {
     // the warp's best key: the largest high word, then the largest low word among the lanes that have it
     const uint32_t hi = static_cast<uint32_t>(mine >> 32), lo = static_cast<uint32_t>(mine);
@@ -596,7 +628,8 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
   size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
   if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
-  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) + aux;
+  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
+                      ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
   int rc;
   if (p.dtype == TB_BF16) {
@@ -615,7 +648,8 @@ int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_
   size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
   if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
-  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) + aux;
+  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
+                      ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
   int rc;
   if (p.dtype == TB_BF16) {
