@@ -208,7 +208,9 @@ struct BeamKey {  // order: value descending, token key ascending, parent ascend
   int32_t tkey, par;
 };
 // One beam expansion of the block's stream (the body of k_beam_step; k_beam_frames calls it once per row).
-constexpr int kBeamThreads = 512;   // threads of a beam block: more warps hide the latencies of its short dependent phases
+// threads of a beam block: more warps than the general kernel's hide the latencies of its short dependent phases; 17
+// warps take a row of 1025 logits (vocabularies of about a thousand pieces) in two strides instead of three
+constexpr int kBeamThreads = 544;
 constexpr int kBeamPref = 5;   // elements of a shared row each thread may hold ahead of time (rows up to 5 * kBeamThreads wide)
 // xpre / xpre_valid: this thread's elements of the stream's shared row, fetched ahead by the previous step of the same
 // launch; next_row: where the next step's shared row starts (null: none), fetched while this step selects.
