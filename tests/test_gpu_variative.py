@@ -97,3 +97,18 @@ def test_greedy_decode_variative_list_sizes(tb, n_phrases, letters, merged):
     assert tb.tb_batch_status(batch) == 0
     for b, g in enumerate(oracle_graphs(pieces, lists, 1.5)):
         check_greedy(out, b, O.greedy_rnnt(g, x[b]), f"variative {n_phrases} phrases")
+
+
+def test_variative_full_size_sampled_streams(tb):
+    # the configuration bench.py --workload 6 times (128 streams of 750 frames, lists cached in shared memory with
+    # the short ring), checked on sampled streams
+    B, T, S = 128, 750, 3
+    pieces = W.make_piece_vocab(6, letters=26, merged=560, max_len=5)
+    lists = [W.draw_string_phrases(6000 + b, pieces, 100, 1, 4) for b in range(B)]
+    x = np.stack([W.variative_stream_logits(6, b, pieces, lists[b], T, S) for b in range(B)])
+    batch = make_variative_batch(tb, pieces, lists, tau=1.0)
+    out = to_host(tb.tb_greedy_decode(batch, to_device(x)))
+    assert tb.tb_batch_status(batch) == 0
+    for b in (0, 41, 94, 127):
+        g = O.GraphFromArrays(var.build(lists[b], pieces, tau=1.0))
+        check_greedy(out, b, O.greedy_rnnt(g, x[b]), "variative full size")
