@@ -499,6 +499,38 @@ def test_beam_step_order_and_carry():
     assert scores[0] == 1.0 and np.isneginf(scores[1]) and list(states) == [0, -1, -1]
 
 
+def test_beam_step_equal_candidates_go_to_the_lower_parent():
+    """Hand-worked step for the last clause of the order (score, token id, parent): two live hypotheses with
+    equal scores and equal graph states read the same row, so every (token) candidate exists twice with the same
+    value; each pair must come out lower parent first.  A third hypothesis with a lower score whose row lifts one
+    of its candidates to the same value joins such a pair as the highest parent."""
+    V = 3
+    g = O.Graph([[0]], V)                                   # token 0 earns +1 at the root
+    row = np.array([0.0, 0.5, -4.0, 0.5], dtype=np.float32)  # values at the root: 1.0, 0.5, -4.0, blank 0.5
+    rows = np.stack([row, row, row, row])
+    scores = np.array([0.0, -np.inf, 0.0, -np.inf], dtype=np.float32)   # hypotheses 0 and 2, slot 1 and 3 empty
+    states = np.array([0, -1, 0, -1], dtype=np.int32)
+    live = np.array([1, 0, 1, 0], dtype=np.uint8)
+    par, tok = O.beam_step(g, rows, scores, states, live)
+    # 1.0: (0, tok 0) (2, tok 0);  0.5: (0, tok 1) (2, tok 1), then the blanks (0, 3) (2, 3) which no longer fit
+    assert list(tok) == [0, 0, 1, 1] and list(par) == [0, 2, 0, 2]
+    assert list(scores) == [1.0, 1.0, 0.5, 0.5] and list(states) == [1, 1, 0, 0] and list(live) == [1, 1, 1, 1]
+    # three parents in one tie: hypothesis 1 scores 0.25 less and its own row offers token 0 at 0.25 more
+    rows = np.stack([row, row + np.float32(0.25), row, row])
+    scores = np.array([0.0, -0.25, 0.0, -np.inf], dtype=np.float32)
+    states = np.array([0, 0, 0, -1], dtype=np.int32)
+    live = np.array([1, 1, 1, 0], dtype=np.uint8)
+    par, tok = O.beam_step(g, rows, scores, states, live)
+    assert list(tok) == [0, 0, 0, 1] and list(par) == [0, 1, 2, 0]
+    assert list(scores) == [1.0, 1.0, 1.0, 0.5]
+    # frozen hypotheses with equal scores are carried in parent order as well (their key is the same, V + 1)
+    scores = np.array([2.0, 2.0, 2.0, -np.inf], dtype=np.float32)
+    states = np.array([0, 1, 0, -1], dtype=np.int32)
+    live = np.array([0, 0, 0, 0], dtype=np.uint8)
+    par, tok = O.beam_step(g, rows, scores, states, live)
+    assert list(par) == [0, 1, 2, -1] and list(tok) == [-1, -1, -1, -1] and list(states) == [0, 1, 0, -1]
+
+
 # ---------------------------------------------------------------------------------------------
 # TDT and streaming
 # ---------------------------------------------------------------------------------------------
