@@ -10,7 +10,8 @@
  *
  * Conventions
  *   - Every call returns an int: TB_OK (0) or a negative TB_ERR_* code; tb_strerror() names
- *     it.  No exception crosses this boundary and the library keeps no global state.
+ *     it.  No exception crosses this boundary.  The library keeps no global state, with one
+ *     exception that its own comment describes: the fixed device array of tb_greedy_decode_noalloc.
  *   - "host" pointers are read or written by the CPU during the call.  "device" pointers are
  *     caller-owned device memory on the batch's GPU; the library never frees or resizes
  *     them.  The library owns only what tb_batch_create allocates (graph arena, slot table,
@@ -90,7 +91,7 @@ typedef struct {
   const float *arc_w;             /* [n_arcs] */
   const int32_t *state_fail;      /* [n_states] suffix-link target */
   const float *state_bw;          /* [n_states] suffix-link weight */
-  const float *state_final;       /* [n_states] final weight (exported, not applied) */
+  const float *state_final;       /* [n_states] final weight; charged by tb_apply_final_weights only */
   const uint8_t *state_depth;     /* [n_states] */
   const int32_t *case_class;      /* [vocab] token -> class */
 } tb_graph_view;

@@ -467,9 +467,43 @@ def tb_greedy_decode_noalloc(logits: torch.Tensor, out: dict, lengths=None, stre
     ``tokens`` / ``frames`` [B, T*S], ``counts`` / ``states`` [B] (int32), ``scores`` [B] (float32) and
     optionally ``status`` [1] (int32).  Calls that overlap on one GPU race on the shared array."""
     B, T, S, W = logits.shape
+    _check_noalloc_buffers(logits, out, lengths)
     st = _strides4(logits)
-    _check(_lib.tb_greedy_decode_noalloc(logits.device.index or 0, _dp(logits), _logit_dtype(logits), B, T, S, W - 1,
+    device = logits.device.index if logits.device.index is not None else torch.cuda.current_device()
+    _check(_lib.tb_greedy_decode_noalloc(device, _dp(logits), _logit_dtype(logits), B, T, S, W - 1,
                                          _hp(st), _dp(lengths), _dp(out["tokens"]), _dp(out["frames"]),
                                          _dp(out["counts"]), _dp(out["scores"]), _dp(out["states"]),
                                          _dp(out.get("status")), _stream(stream)), "tb_greedy_decode_noalloc")
     return out
+
+
+def _check_noalloc_buffers(logits: torch.Tensor, out: dict, lengths):
+    """The caller brings every output buffer of tb_greedy_decode_noalloc, and the kernel writes them without
+    knowing their sizes: a buffer that is too short, of another type, strided, or on another device is refused
+    here, before anything is launched.  Sizes and types are checked first (they need no GPU), devices last."""
+    B, T, S, _ = logits.shape
+    need = {"tokens": (torch.int32, B * T * S), "frames": (torch.int32, B * T * S), "counts": (torch.int32, B),
+            "states": (torch.int32, B), "scores": (torch.float32, B)}
+    if out.get("status") is not None:
+        need["status"] = (torch.int32, 1)
+    tensors = []
+    for name, (dt, n) in need.items():
+        t = out.get(name)
+        if not isinstance(t, torch.Tensor):
+            raise ValueError(f"tb_greedy_decode_noalloc: out[{name!r}] must be a preallocated tensor")
+        if t.dtype != dt:
+            raise ValueError(f"tb_greedy_decode_noalloc: out[{name!r}] must be {dt}, got {t.dtype}")
+        if not t.is_contiguous():
+            raise ValueError(f"tb_greedy_decode_noalloc: out[{name!r}] must be contiguous")
+        if t.numel() < n:
+            raise ValueError(f"tb_greedy_decode_noalloc: out[{name!r}] holds {t.numel()} elements, {n} are written")
+        tensors.append((name, t))
+    if lengths is not None:
+        if lengths.dtype != torch.int32 or not lengths.is_contiguous() or lengths.numel() < B:
+            raise ValueError("tb_greedy_decode_noalloc: lengths must be a contiguous int32 tensor of at least B elements")
+        tensors.append(("lengths", lengths))
+    if not logits.is_cuda:
+        raise ValueError("tb_greedy_decode_noalloc: logits must be on a CUDA device")
+    for name, t in tensors:
+        if t.device != logits.device:
+            raise ValueError(f"tb_greedy_decode_noalloc: {name} is on {t.device}, the logits are on {logits.device}")

@@ -22,7 +22,7 @@ struct GraphPtrs {
   float lambda;
 };
 
-// "Read the state and arc offsets of the model id and shift the pointers" (Sec. 2.2 para. 3).
+// The slot's record selects the stream's graph: per-slot offsets into the arena give the graph's arrays (Sec. 2.2 para. 3).
 __device__ __forceinline__ GraphPtrs graph_of(const unsigned char* arena, const TbSlotRec& r) {
   GraphPtrs g;
   const unsigned char* blob = arena + r.blob_off;
@@ -106,8 +106,8 @@ __device__ __forceinline__ ValId block_best(ValId x, ValId* scratch) {
   return scratch[nwarps];
 }
 
-// Dense bonus / next-state vectors over classes for state s (the "score vector over the
-// vocabulary" and next states of Sec. 2.2 para. 3, kept in shared memory, indexed by class).
+// Dense bonus / next-state vectors over classes for state s (what the scoring kernel of
+// Sec. 2.2 para. 3 hands the decoder per batch item; here kept in shared memory, indexed by class).
 // The chain s, fail(s), ... root is walked once; acc_j is the sum of the suffix-link weights
 // crossed before chain state j (float adds in walk order).  Classes are then filled from the
 // root end of the chain toward s, so the state closest to s wins.

@@ -48,24 +48,6 @@ constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr int kSegMinFrames = 128;  // streams at least this long are decoded as two segments (see the header)
 constexpr int kSegWarm = 16;        // frames the second segment decodes before the first frame it answers for
 
-#ifdef TB_PROFILE
-__device__ unsigned long long tb_prof[16];
-__device__ unsigned long long tb_prof_blk[4 * 1024];
-#define PROF_DECL() long long _pacc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; long long _pt = 0
-#define PROF_T0() _pt = clock64()
-#define PROF_ADD(slot) do { long long _n = clock64(); _pacc[slot] += _n - _pt; _pt = _n; } while (0)
-#define PROF_COUNT(slot) _pacc[slot] += 1
-#ifndef TB_PROF_PIPE
-#define TB_PROF_PIPE pipe
-#endif
-#define PROF_FLUSH() do { if ((threadIdx.x & 31) == 0 && pipe == TB_PROF_PIPE) { for (int _i = 0; _i < 16; ++_i) if (_pacc[_i]) atomicAdd(&tb_prof[_i], (unsigned long long)_pacc[_i]); } } while (0)
-#else
-#define PROF_DECL() do {} while (0)
-#define PROF_T0() do {} while (0)
-#define PROF_ADD(slot) do {} while (0)
-#define PROF_COUNT(slot) do {} while (0)
-#define PROF_FLUSH() do {} while (0)
-#endif
 
 // What a helper leaves for the decider about one row (32 bytes, read as two 16-byte loads).
 struct RowSummary {
@@ -470,9 +452,6 @@ __device__ __forceinline__ Pick warp_pick(ValId v, int next) {
 template <int NIT>
 __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   extern __shared__ __align__(128) unsigned char dyn[];
-#ifdef TB_PROFILE
-  const long long _kstart = clock64();
-#endif
   const TbDecodeParams& p = P.d;
   const int V = p.V, C = p.C, S = p.S, W = V + 1, nst = P.nst;
   const Smem so = carve(nst, P.slot_bytes, V, C, P.cache_bytes, P.npipes, P.own_lists);
@@ -610,15 +589,12 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   uint64_t* pfree = freeb + pst_base;
   const uint32_t psumm_a = summ_a + pst_base * kSumStageBytes;
 
-  PROF_DECL();
   if (vw == 4 || (seg && vw == 12)) {
     // ================================ producer ================================================
     int issued = pf0, st = 0, use = 0;
     for (int f = pf0; f < end; ++f) {
-      PROF_T0();
       if (flags[pipe]) break;
       if (use > 0 && !mbar_wait_parked(&pfree[st], (use - 1) & 1, flags, pipe, p.status)) break;
-      PROF_ADD(6);
       const unsigned char* src = base + static_cast<int64_t>(f) * frame_stride_bytes;
       const int lead = static_cast<int>(reinterpret_cast<uintptr_t>(src) & 15);
       const unsigned char* a0 = src - lead;
@@ -637,7 +613,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       if (++st == pnst) { st = 0; ++use; }
       __syncwarp();
     }
-    PROF_FLUSH();
     // no copy may be in flight when the block exits
     for (int f = max(pf0, issued - pnst); f < issued; ++f) {
       const int fl = f - pf0, fs = fl % pnst;
@@ -658,13 +633,10 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     int f = pf0 + fl;
     int lead = (lead0 + f * lead_step) & 15;
     for (; f < end;) {
-      PROF_T0();
       if (!mbar_wait_parked(&pfull[st], ph, flags, pipe, p.status)) break;
-      PROF_ADD(0);
       const unsigned char* slot = pring + static_cast<size_t>(st) * P.slot_bytes;
       summarize_row<NIT>(h, slot, lead + k * row_bytes, psumm_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
       if (lane == 0) mbar_arrive(&pfree[st]);
-      PROF_ADD(1);
       k += pnh;
       while (k >= S) {                                      // on to a later frame
         k -= S; ++f;
@@ -672,7 +644,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         if (++st == pnst) { st = 0; ph ^= 1u; }
       }
     }
-    PROF_FLUSH();
   } else if (vw == 0 || (seg && vw == 8)) {
     // ================================ decider =================================================
     // Works in rounds over a window of eight frames.  The warp is eight groups of four lanes; group q
@@ -728,7 +699,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     const bool fast_ok = bound && cached && resolved;       // the branch-free round reads lists from the cache only
     for (int it = 0; t < end; ++it) {
       if (it >= max_rounds) { if (lane == 0) atomicOr(p.status, TB_STATUS_STEP_LIMIT); break; }
-      PROF_T0();
       // ---- mode and this lane's row --------------------------------------------------------------------
       const bool allrows = !no_allrows && (L.n == 0 || (stable && L.n <= kAllRowsDeep));
       const bool wide = !allrows && L.n > kGroupDeep;
@@ -892,14 +862,10 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             if (lane == 0 && adv > 0) prog_publish(flags, t + 1);
           }
           spins = 0; no_allrows = false;
-          PROF_ADD(3);
-          PROF_COUNT(8);
-          PROF_COUNT(13);
           // the next round is of the same kind more often than not: straight back, without the loop's bookkeeping
           if (L.n > 0 && L.n <= kGroupDeep && !stable && t < end && it + 1 < max_rounds && !(chk_on && t >= f_mid)) { ++it; goto fast_again; }
           continue;
         }
-        PROF_COUNT(14);
       }
       // ---- the same for an all-rows round (root state, unbound stream, or a state that repeats itself): every
       // lane its own row, and the whole list of the state, if it has one
@@ -1019,12 +985,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             if (lane == 0 && fq > 0) prog_publish(flags, t + 1);
           }
           spins = 0;
-          PROF_ADD(3);
-          PROF_COUNT(8);
-          PROF_COUNT(13);
           continue;
         }
-        PROF_COUNT(14);
       }
       const int rq = wide ? 0 : q;                          // window frame of this lane
       const int rk = allrows ? ql : (rq == 0 ? k : 0);      // row of that frame
@@ -1036,7 +998,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + rq * lead_step) & 15) + rk * row_bytes;
       const bool in_row = rk < S && (rq > 0 || rk >= k);   // all-rows mode: rows before (t, k) are behind us
       const bool ready = in_row && t + rq < end && q1.w == static_cast<uint32_t>(t + rq) + 1u;
-      PROF_ADD(2);
       const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
       const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
       bool rescan = (q1.z & kSumOvf) != 0;
@@ -1093,7 +1054,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           if (v0 > wv || (v0 == wv && (e0.x & kTokMask) < (wdt & kTokMask))) { wv = v0; wdt = e0.x; }
         }
       }
-      PROF_ADD(3);
       // combine over the lanes that share the row
       if (L.n > 0 && !allrows) {
         if (wide) {
@@ -1115,7 +1075,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           }
         }
       }
-      PROF_ADD(15);
       int wtok = static_cast<int>((wdt & kTokMask) >> 1);
       int wnext = static_cast<int>(wdt >> TB_RS_TOK_BITS);
       {
@@ -1144,7 +1103,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         // ---- walk the window row by row, through tokens too, while the state stays what it is ----------
         const unsigned ready_all = __ballot_sync(0xffffffffu, ready && !rescan);
         const unsigned keep_all = __ballot_sync(0xffffffffu, wnext == s);
-        PROF_ADD(7);
         // Which rows the decode visits follows from the blank / token pattern alone while the state stays what
         // it is: in a frame, row j is visited when rows 0 .. j-1 selected tokens.  All of it is bit arithmetic
         // on the ballots (bit 4 q + j: row j of frame t + q); only the score is added up row by row.
@@ -1200,15 +1158,12 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           const unsigned resc_all = __ballot_sync(0xffffffffu, ready && rescan);
           if ((resc_all >> k) & 1u) no_allrows = true;
         }
-        PROF_ADD(4);
-        PROF_ADD(10);
       } else {
         // ---- the leading blanks, then the row after them --------------------------------------------------
         const unsigned blank_m = blank_all & 0x11111111u;   // one bit per group
         const unsigned stop_m = ~blank_m & 0x11111111u;
         int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : kWin;
         if (wide) nb = (blank_m & 1u) ? 1 : 0;
-        PROF_ADD(7);
         const int jl = wide ? 0 : 4 * min(nb, kWin - 1);
         const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
         const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
@@ -1221,7 +1176,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, 4 * r));
         adv = nb;
         progress = nb > 0;
-        PROF_ADD(4);
         bool took = false;                                  // the row after the blanks was consumed too
         if (!(wide && nb == 1) && nb < kWin && j_ready) {
           progress = true;
@@ -1231,7 +1185,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             tok = j_tok; tval = j_val; tnext = j_next;
           } else {
             // exact evaluation of that row by the whole warp from shared memory
-            PROF_COUNT(9);
             const uint32_t rrow = __shfl_sync(0xffffffffu, row_a, jl);
             for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = static_cast<int16_t>(i); }
             __syncwarp();
@@ -1279,11 +1232,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           nv += nb + (took ? 1 : 0);
         }
         if (adv > 0 && (tok == V || k == S)) k = 0;
-        PROF_ADD(10);
       }
-      PROF_COUNT(8);
       if (!progress) {                                      // the current row is not summarised yet: poll
-        PROF_COUNT(12);
         if (++spins > kSpinLimit || ((spins & 255u) == 0u && flags[pipe])) {
           if (spins > kSpinLimit) { flags[0] = 1; flags[1] = 1; if (lane == 0) atomicOr(p.status, TB_STATUS_WAIT_TIMEOUT); }
           failed = true; break;
@@ -1301,7 +1251,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       t += adv;
       st += adv; if (st >= nst) st -= nst;
       lead = (lead + adv * lead_step) & 15;
-      PROF_ADD(5);
       if (tok != V) stable = (tnext == s);                  // the last token left the state unchanged
       if (tok != V && bound && tnext != s) {
         s = tnext;
@@ -1333,17 +1282,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const int rec_state = *reinterpret_cast<const volatile int*>(trace + t);
         if (rec_state == s) { tc = t; break; }
       }
-      PROF_ADD(11);
     }
-    PROF_FLUSH();
-#ifdef TB_PROFILE
-    if (lane == 0 && blockIdx.x < 1024) {
-      tb_prof_blk[4 * blockIdx.x] = _pacc[2] + _pacc[3] + _pacc[4] + _pacc[5] + _pacc[7] + _pacc[10] + _pacc[11];
-      tb_prof_blk[4 * blockIdx.x + 1] = clock64() - _kstart;
-      tb_prof_blk[4 * blockIdx.x + 2] = n_out;
-      tb_prof_blk[4 * blockIdx.x + 3] = _pacc[9];
-    }
-#endif
     if ((n_out & 31) != 0) {                  // the tokens still staged
       __syncwarp();
       const int2 e = emit_buf[lane];
@@ -1403,16 +1342,6 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
 
 }  // namespace
 
-#ifdef TB_PROFILE
-extern "C" int tb_debug_prof(unsigned long long* out16, int reset) {
-  if (cudaMemcpyFromSymbol(out16, tb_prof, sizeof(unsigned long long) * 16) != cudaSuccess) return -1;
-  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(tb_prof, z, sizeof z); }
-  return 0;
-}
-extern "C" int tb_debug_prof_blk(unsigned long long* out, int n) {
-  return cudaMemcpyFromSymbol(out, tb_prof_blk, sizeof(unsigned long long) * 4 * n) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 namespace {
 // scratch layout of the two-segment decode: tokens+frames, values, frame-start records

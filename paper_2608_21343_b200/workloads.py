@@ -309,9 +309,17 @@ class ChurnSchedule:
     total stream lengths, and the list of (slot, stream id, phrases) binds that must be applied
     before this chunk is decoded."""
 
-    def __init__(self, w: Workload):
+    def __init__(self, w: Workload, workers: int = 0):
+        """workers > 0: the inputs of the streams that come next are generated ahead of time on that many
+        threads (every stream has its own generator, so the bits do not depend on it)."""
         assert w.chunk > 0
         self.w = w
+        self._pool = None
+        self._ahead = {}
+        if workers > 0:
+            from concurrent.futures import ThreadPoolExecutor
+            self._pool = ThreadPoolExecutor(max_workers=workers)
+            self._n_ahead = 4 * workers
         self.next_stream = w.B
         self.stream_of = list(range(w.B))
         self.offset = [0] * w.B        # frames of the current stream already served
@@ -320,11 +328,31 @@ class ChurnSchedule:
         np_dt = np.float32 if w.dtype == "f32" else np.uint16
         self.zero_chunk = np.zeros((w.chunk, w.S, w.row_width), dtype=np_dt)
 
+    def _inputs(self, stream_id: int) -> dict:
+        if self._pool is None:
+            return stream_inputs(self.w, stream_id)
+        # stream ids are handed out in ascending order: keep the next few in flight
+        hi = max(stream_id + 1, min(self.next_stream, stream_id + 1) + self._n_ahead)
+        if stream_id < self.w.B:
+            hi = max(hi, self.w.B)          # the first chunk asks for all slots' streams at once
+        for sid in range(stream_id, hi):
+            if sid not in self._ahead:
+                self._ahead[sid] = self._pool.submit(stream_inputs, self.w, sid)
+        return self._ahead.pop(stream_id).result()
+
+    def close(self):
+        if self._pool is not None:
+            for f in self._ahead.values():
+                f.cancel()
+            self._pool.shutdown(wait=True)
+            self._pool = None
+            self._ahead = {}
+
     def next_chunk(self):
         w = self.w
         binds = []
         for slot in self.pending:
-            d = stream_inputs(w, self.stream_of[slot])
+            d = self._inputs(self.stream_of[slot])
             self.data[slot] = d
             self.offset[slot] = 0
             binds.append((slot, self.stream_of[slot], d["phrases"]))

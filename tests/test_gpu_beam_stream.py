@@ -145,13 +145,6 @@ def test_beam_other_widths_fp32(tb, K):
             assert out["lens"][i, 0] == n and np.array_equal(out["tokens"][i, 0, :n], ref["tokens"])
 
 
-def test_workload4_full_size_sampled_streams(tb):
-    w = W.get_workload(4)
-    data = W.batch_inputs(w)
-    out = run_beam(tb, w, data, w.K)
-    compare_beam(w, data, out, w.K, [0, 13, 31])
-
-
 def test_beam_step_frozen_and_empty(tb):
     """One step by hand: ordering of equal scores, a frozen hypothesis carried, empty places."""
     w = W.get_workload(1, B=1, T=1)
@@ -309,18 +302,3 @@ def test_beam_widths_whose_shared_memory_straddles_the_default_limit(tb, K):
     batch, _ = make_batch(tb, w, data["phrases"], max_beam=K, max_tree_steps=w.T * w.S)
     fr = run_beam_frames(tb, w, data, K, data["phrases"], batch)
     assert np.array_equal(fr["tokens"], out["tokens"]) and np.array_equal(fr["scores"], out["scores"])
-
-
-def test_workload4_full_size_in_one_launch_sampled_streams(tb):
-    # the configuration bench.py --workload 4 times through tb_beam_frames, checked on sampled streams
-    w = W.get_workload(4)
-    data = W.batch_inputs(w)
-    batch, _ = make_batch(tb, w, data["phrases"], max_beam=w.K, max_tree_steps=w.T * w.S)
-    out = run_beam_frames(tb, w, data, w.K, data["phrases"], batch)
-    for i in (0, 13, 31):
-        ref = O.beam_decode(oracle_graph(w, data["phrases"][i]), data["logits"][i], w.K)
-        assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"])
-        for k in range(w.K):
-            assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k])
-        fin = np.isfinite(ref["scores"])
-        assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL)

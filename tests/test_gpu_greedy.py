@@ -51,27 +51,6 @@ def test_workload2_reduced_and_unbound_mix(tb):
     assert out["states"][3] == -1
 
 
-def test_workload2_full_size_sampled_streams(tb):
-    """The benchmark's configuration (B=128, T=750, bf16): every stream decoded on the GPU,
-    a sample of streams decoded one by one by the oracle."""
-    w = W.get_workload(2)
-    data = W.batch_inputs(w)
-    batch, _ = make_batch(tb, w, data["phrases"])
-    logits = to_device(data["logits"])
-    out = to_host(tb.tb_greedy_decode(batch, logits))
-    assert tb.tb_batch_status(batch) == 0
-    for i in list(range(0, w.B, 9)) + [w.B - 1]:
-        ref = O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i])
-        check_greedy(out, i, ref, "w2")
-    # unboosted: every slot unbound
-    for i in range(w.B):
-        tb.tb_batch_bind_stream(batch, i, None)
-    out0 = to_host(tb.tb_greedy_decode(batch, logits))
-    for i in (0, 64, 127):
-        check_greedy(out0, i, O.greedy_rnnt(None, data["logits"][i]), "w2-unboosted")
-    assert (out0["states"] == -1).all()
-
-
 def test_workload3_large_lists(tb):
     w = W.get_workload(3, B=3, T=300)
     data = W.batch_inputs(w)

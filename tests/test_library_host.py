@@ -302,3 +302,33 @@ def test_cache_of_variative_lists(tb):
     w = W.get_workload(1)
     assert not tb.tb_cache_compile(cache, W.stream_phrases(w, 0), w.V, case_class=w.vocab.case_class)[1]
     assert tb.tb_cache_compile(cache, W.stream_phrases(w, 0), w.V, case_class=w.vocab.case_class)[1]
+
+
+def test_noalloc_binding_refuses_bad_buffers_before_any_launch(tb):
+    """tb_greedy_decode_noalloc writes into buffers the caller brings; the binding refuses a buffer that is too
+    short, of the wrong type or strided without touching a GPU (sizes and types are checked before devices)."""
+    import torch
+    B, T, S, V = 3, 5, 2, 8
+    logits = torch.zeros((B, T, S, V + 1), dtype=torch.float32)
+
+    def bufs():
+        return dict(tokens=torch.zeros((B, T * S), dtype=torch.int32), frames=torch.zeros((B, T * S), dtype=torch.int32),
+                    counts=torch.zeros(B, dtype=torch.int32), states=torch.zeros(B, dtype=torch.int32),
+                    scores=torch.zeros(B, dtype=torch.float32), status=torch.zeros(1, dtype=torch.int32))
+
+    o = bufs(); o["tokens"] = torch.zeros((B, T * S - 1), dtype=torch.int32)
+    with pytest.raises(ValueError, match="tokens.*elements"):
+        tb.tb_greedy_decode_noalloc(logits, o)
+    o = bufs(); o["scores"] = torch.zeros(B, dtype=torch.float64)
+    with pytest.raises(ValueError, match="scores.*float32"):
+        tb.tb_greedy_decode_noalloc(logits, o)
+    o = bufs(); o["frames"] = torch.zeros((B, 2 * T * S), dtype=torch.int32)[:, ::2]
+    with pytest.raises(ValueError, match="frames.*contiguous"):
+        tb.tb_greedy_decode_noalloc(logits, o)
+    o = bufs(); del o["counts"]
+    with pytest.raises(ValueError, match="counts"):
+        tb.tb_greedy_decode_noalloc(logits, o)
+    with pytest.raises(ValueError, match="lengths"):
+        tb.tb_greedy_decode_noalloc(logits, bufs(), lengths=torch.zeros(B - 1, dtype=torch.int32))
+    with pytest.raises(ValueError, match="CUDA"):           # everything else in order: the logits are not on a GPU
+        tb.tb_greedy_decode_noalloc(logits, bufs())

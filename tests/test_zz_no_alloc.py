@@ -4,8 +4,9 @@ tb_greedy_decode_noalloc exists for callers that are not allowed to allocate dev
 decode (a server that divided its memory budget up front, or a thread that cannot take the device-wide
 synchronisation of cudaMalloc): it keeps the kernel's working memory in a fixed array inside the library and
 decodes every stream as unbound.  Its results must equal those of tb_greedy_decode on a batch whose slots
-are all unbound -- tokens, frames, counts and states exactly, scores within the tolerance of the other
-parity tests -- on two calls in a row (the second call meets the array as the first one left it).
+are all unbound, and those of the CPU oracle decoding without a graph -- tokens, frames, counts and states
+exactly, scores within the tolerance of the other parity tests -- on two calls in a row (the second call meets
+the array as the first one left it).
 
 This file is collected last on purpose: if it fails, a run that stops at the first failure has already run
 every other test.  It passes alone in a fresh process as well as after the others.
@@ -14,8 +15,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_2608_21343_b200 import workloads as W
-from helpers import SCORE_TOL, to_device
+from helpers import SCORE_TOL, check_greedy, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +57,11 @@ def test_noalloc_matches_unbound_decode_twice(tb):
             out = tb.tb_greedy_decode_noalloc(lg, _out(w.B, w.T, w.S, dev))
             _same(out, rf)
             assert int(out["status"].item()) == 0 and (out["states"] == -1).all()
+            # and against the oracle, stream by stream (no graph: the unboosted decode)
+            host = {k: v.cpu().numpy() for k, v in out.items()}
+            lg_host = data["logits"] if call == 0 else data["logits"][::-1]
+            for i in range(w.B):
+                check_greedy(host, i, O.greedy_rnnt(None, np.ascontiguousarray(lg_host[i])), "noalloc")
     # a length vector and a strided view, still without a batch
     w = cases[0]
     data = W.batch_inputs(w)
@@ -63,8 +70,11 @@ def test_noalloc_matches_unbound_decode_twice(tb):
     view = big[..., 3:w.V + 4]
     lengths = torch.tensor([90, 0, 17, 1, 89, 45], dtype=torch.int32, device=dev)
     batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=1 << 16)
-    _same(tb.tb_greedy_decode_noalloc(view, _out(w.B, w.T, w.S, dev), lengths=lengths),
-          tb.tb_greedy_decode(batch, view, lengths=lengths))
+    out = tb.tb_greedy_decode_noalloc(view, _out(w.B, w.T, w.S, dev), lengths=lengths)
+    _same(out, tb.tb_greedy_decode(batch, view, lengths=lengths))
+    host = {k: v.cpu().numpy() for k, v in out.items()}
+    for i in range(w.B):
+        check_greedy(host, i, O.greedy_rnnt(None, data["logits"][i], int(lengths[i])), "noalloc-lengths")
 
 
 def test_noalloc_rejects_sizes_beyond_its_array(tb):
