@@ -62,7 +62,16 @@ extern "C" {
 #define TB_FRAME_NEW_MERGE 2  /* as TB_FRAME_NEW, after hypotheses with equal token sequences were merged */
 
 /* tb_batch_set_flags */
-#define TB_FLAG_GENERAL_KERNELS 1   /* always use the general decode kernel (any layout), never the pipelined one */
+#define TB_FLAG_GENERAL_KERNELS 1       /* always use the general decode kernel (any layout), never a pipelined one */
+#define TB_FLAG_ONE_BLOCK_PER_STREAM 2  /* pipelined greedy decode: never the segmented kernel, one block per stream */
+#define TB_FLAG_TEST_WAIT_TIMEOUT 4     /* self-test of the kernels' bounded waits: tb_greedy_decode (segmented kernel) withholds one
+                                           frame's summaries and waits only briefly, so the wait runs out: the call returns,
+                                           TB_STATUS_WAIT_TIMEOUT is set, the outputs of that call are undefined */
+
+/* tb_batch_last_greedy_kernel */
+#define TB_KERNEL_GENERAL 1     /* one block per stream, a block-wide argmax per visited row */
+#define TB_KERNEL_PIPELINED 2   /* one block per stream: rows staged in shared memory, at most two segments */
+#define TB_KERNEL_SEGMENTED 3   /* streams cut into segments decoded by many small pipelines on all SMs, then stitched */
 
 /* Limits of this build. */
 #define TB_MAX_VOCAB 8192           /* non-blank tokens */
@@ -266,12 +275,33 @@ int tb_batch_bind_models(tb_batch *b, int32_t n, const int32_t *slots, const int
 
 /*
  * Set behaviour flags of the batch (TB_FLAG_*; 0 = defaults).  With the defaults
- * tb_greedy_decode picks the pipelined kernel whenever the call fits it (bf16 logits, token
- * stride 1, the S rows of a frame contiguous, vocab <= 2048, S <= 4) and the general kernel
- * otherwise; both give identical results.  The paper has no counterpart of this call.
+ * tb_greedy_decode picks a pipelined kernel whenever the call fits it (bf16 logits, token
+ * stride 1, the S rows of a frame contiguous, vocab <= 2048, S <= 4) -- the segmented one when every
+ * bound graph carries resolved lists that fit a block's shared memory, else the one-block-per-stream
+ * one -- and the general kernel otherwise; all give identical results.  The paper has no counterpart
+ * of this call.
  * Errors: TB_ERR_INVALID_ARG (unknown bits).
  */
 int tb_batch_set_flags(tb_batch *b, uint32_t flags);
+
+/*
+ * Tuning of the segmented greedy kernel (no counterpart in the paper): how many decider warps (1..4) and helper
+ * warps a block holds, and how many blocks decode one stream; the stream is cut into blocks_per_stream *
+ * deciders_per_block segments (Sec. 2.2 para. 3 asks for one advance per stream and step; segments are a way to run
+ * several parts of a stream's decode at once, with identical results).  0 = chosen by the library from the GPU's
+ * size and the call's shape; deciders and helpers are given together or not at all.
+ * Errors: TB_ERR_INVALID_ARG.
+ */
+int tb_batch_set_greedy_plan(tb_batch *b, int32_t deciders_per_block, int32_t helpers_per_block,
+                             int32_t blocks_per_stream);
+
+/*
+ * Which kernel the last successful tb_greedy_decode of this batch launched (TB_KERNEL_*; 0 before the first), and
+ * for the segmented kernel its blocks per stream and deciders per block (host pointers, each may be NULL).  The
+ * three kernels give identical results; a caller that depends on the speed of one can assert it here.
+ */
+int tb_batch_last_greedy_kernel(const tb_batch *b, int32_t *kernel, int32_t *blocks_per_stream,
+                                int32_t *deciders_per_block);
 
 /*
  * Copy the device status word to *device_status (host) after synchronising `stream`, and

@@ -73,6 +73,8 @@ _SIGS = {
     "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
     "tb_batch_status": (C.c_int, [_vp, C.POINTER(_i32), _vp]),
     "tb_batch_set_flags": (C.c_int, [_vp, C.c_uint32]),
+    "tb_batch_set_greedy_plan": (C.c_int, [_vp, _i32, _i32, _i32]),
+    "tb_batch_last_greedy_kernel": (C.c_int, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
     "tb_greedy_decode": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_stream_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                   _vp, _vp, _vp]),
@@ -342,11 +344,28 @@ def tb_batch_bind_stream(batch: Batch, slot: int, graph, stream=None):
            "tb_batch_bind_stream")
 
 
+TB_STATUS_WALK_TOO_DEEP, TB_STATUS_BAD_STATE, TB_STATUS_STEP_LIMIT, TB_STATUS_WAIT_TIMEOUT = 1, 2, 4, 8
 TB_FLAG_GENERAL_KERNELS = 1
+TB_FLAG_ONE_BLOCK_PER_STREAM = 2
+TB_FLAG_TEST_WAIT_TIMEOUT = 4
+TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
 
 
 def tb_batch_set_flags(batch: Batch, flags: int):
     _check(_lib.tb_batch_set_flags(batch.handle, flags), "tb_batch_set_flags")
+
+
+def tb_batch_set_greedy_plan(batch: Batch, deciders_per_block: int = 0, helpers_per_block: int = 0,
+                             blocks_per_stream: int = 0):
+    _check(_lib.tb_batch_set_greedy_plan(batch.handle, deciders_per_block, helpers_per_block, blocks_per_stream),
+           "tb_batch_set_greedy_plan")
+
+
+def tb_batch_last_greedy_kernel(batch: Batch) -> dict:
+    k, nb, g = _i32(0), _i32(0), _i32(0)
+    _check(_lib.tb_batch_last_greedy_kernel(batch.handle, C.byref(k), C.byref(nb), C.byref(g)),
+           "tb_batch_last_greedy_kernel")
+    return dict(kernel=k.value, blocks_per_stream=nb.value, deciders_per_block=g.value)
 
 
 def tb_batch_status(batch: Batch, stream=None) -> int:

@@ -117,13 +117,22 @@ struct tb_batch {
   int next_staging = 0;
   void* seg_scratch = nullptr;      // working memory of the two-segment greedy decode (grown on demand)
   size_t seg_scratch_bytes = 0;
+  // working memory of the segmented greedy decode: zeroed when allocated and whenever the shape it is laid out for
+  // changes; never freed or moved once a stream capture has used it (a captured graph keeps the pointer)
+  void* sg_scratch = nullptr;
+  size_t sg_scratch_bytes = 0;
+  int32_t sg_shape[4] = {0, 0, 0, 0};   // streams, frames, rows per frame, segments of the layout in place
+  bool sg_captured = false;
+  int32_t plan_G = 0, plan_H = 0, plan_NB = 0;   // tb_batch_set_greedy_plan (0: automatic)
+  int32_t last_kernel = 0, last_NB = 0, last_G = 0;
+  int32_t n_sm = 0, max_smem = 0;
 };
 
 static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs);
   for (auto& s : b->staging) {
     if (s.held) tb_graph_free(s.held);
     if (s.host) cudaFreeHost(s.host);
@@ -429,6 +438,7 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   p.out_scores = out_scores; p.out_states = out_states;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (!(b->flags & TB_FLAG_GENERAL_KERNELS)) {
     int32_t max_cache = 0, max_states = 0, all_resolved = 1;
     for (int32_t i = 0; i < B; ++i) {
@@ -436,24 +446,81 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
       max_states = b->slot_n_states[i] > max_states ? b->slot_n_states[i] : max_states;
       if (!b->slot_resolved[i]) all_resolved = 0;
     }
+    // Working memory is never allocated while the caller's stream is being captured into a graph (allocation is
+    // not allowed there): the decode then runs with the block it has, or on a path that needs none.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (!(b->flags & TB_FLAG_ONE_BLOCK_PER_STREAM)) {
+      if (b->n_sm == 0) {
+        cudaDeviceGetAttribute(&b->n_sm, cudaDevAttrMultiProcessorCount, b->device);
+        cudaDeviceGetAttribute(&b->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, b->device);
+        cudaGetLastError();
+      }
+      TbSegPlan plan;
+      plan.force_G = b->plan_G; plan.force_H = b->plan_H; plan.force_NB = b->plan_NB;
+      plan.test_timeout = (b->flags & TB_FLAG_TEST_WAIT_TIMEOUT) ? 1 : 0;
+      if (plan.test_timeout && plan.force_G == 0) { plan.force_G = 2; plan.force_H = 8; }   // the self-test always takes this kernel
+      if (b->n_sm > 0 && tb_greedy_seg_plan(p, max_cache, all_resolved, b->n_sm, b->max_smem, &plan)) {
+        const int32_t nseg = plan.NB * plan.G;
+        const size_t want = tb_greedy_seg_scratch_bytes(B, T, S, nseg);
+        bool ok = true;
+        if (want > b->sg_scratch_bytes) {
+          ok = !capturing && !b->sg_captured && want <= (static_cast<size_t>(4) << 30);
+          if (ok) {
+            cudaFree(b->sg_scratch);                    // (waits for earlier work: one decode per batch at a time)
+            b->sg_scratch = nullptr; b->sg_scratch_bytes = 0; b->sg_shape[0] = 0;
+            if (cudaMalloc(&b->sg_scratch, want) == cudaSuccess) b->sg_scratch_bytes = want;
+            else { cudaGetLastError(); ok = false; }
+          }
+        }
+        if (ok && (b->sg_shape[0] != B || b->sg_shape[1] != T || b->sg_shape[2] != S || b->sg_shape[3] != nseg)) {
+          // another layout: what the last one left (launch numbers, records) would be misread
+          if (cudaMemsetAsync(b->sg_scratch, 0, want, stream) != cudaSuccess) { cudaGetLastError(); ok = false; }
+          else { b->sg_shape[0] = B; b->sg_shape[1] = T; b->sg_shape[2] = S; b->sg_shape[3] = nseg; }
+        }
+        if (ok) {
+          if (capturing) b->sg_captured = true;
+          rc = tb_launch_greedy_seg(p, max_cache, plan, b->sg_scratch, stream);
+          if (rc == TB_OK) { b->last_kernel = TB_KERNEL_SEGMENTED; b->last_NB = plan.NB; b->last_G = plan.G; }
+          return rc;
+        }
+      }
+    }
     // the two-segment decode keeps what its second segment produces in scratch memory of the batch; growing it
     // frees the old block first (cudaFree waits for earlier work), so one decode per batch at a time
     const size_t want = tb_greedy_fast_scratch_bytes(B, T, S);
-    // (never while the caller's stream is being captured into a graph: allocation is not allowed there; the decode
-    // then runs with the block it has, or with one segment per stream)
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream_), &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
-    if (cap == cudaStreamCaptureStatusNone && want > b->seg_scratch_bytes && want <= (static_cast<size_t>(1) << 30)) {
+    if (!capturing && want > b->seg_scratch_bytes && want <= (static_cast<size_t>(1) << 30)) {
       cudaFree(b->seg_scratch);
       b->seg_scratch = nullptr; b->seg_scratch_bytes = 0;
       if (cudaMalloc(&b->seg_scratch, want) == cudaSuccess) b->seg_scratch_bytes = want;
       else cudaGetLastError();
     }
-    rc = tb_launch_greedy_fast(p, max_cache, max_states, all_resolved, b->seg_scratch, b->seg_scratch_bytes,
-                               static_cast<cudaStream_t>(stream_));
+    rc = tb_launch_greedy_fast(p, max_cache, max_states, all_resolved, b->seg_scratch, b->seg_scratch_bytes, stream);
+    if (rc == TB_OK) { b->last_kernel = TB_KERNEL_PIPELINED; b->last_NB = 1; b->last_G = 0; }
     if (rc != 1) return rc;
   }
-  return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+  rc = tb_launch_decode_general(p, stream);
+  if (rc == TB_OK) { b->last_kernel = TB_KERNEL_GENERAL; b->last_NB = 1; b->last_G = 0; }
+  return rc;
+}
+
+extern "C" int tb_batch_set_greedy_plan(tb_batch* b, int32_t deciders_per_block, int32_t helpers_per_block,
+                                        int32_t blocks_per_stream) {
+  if (!b || deciders_per_block < 0 || helpers_per_block < 0 || blocks_per_stream < 0) return TB_ERR_INVALID_ARG;
+  if ((deciders_per_block == 0) != (helpers_per_block == 0)) return TB_ERR_INVALID_ARG;
+  if (deciders_per_block > 4 || (deciders_per_block + helpers_per_block) > 20) return TB_ERR_INVALID_ARG;
+  b->plan_G = deciders_per_block; b->plan_H = helpers_per_block; b->plan_NB = blocks_per_stream;
+  return TB_OK;
+}
+
+extern "C" int tb_batch_last_greedy_kernel(const tb_batch* b, int32_t* kernel, int32_t* blocks_per_stream,
+                                           int32_t* deciders_per_block) {
+  if (!b) return TB_ERR_INVALID_ARG;
+  if (kernel) *kernel = b->last_kernel;
+  if (blocks_per_stream) *blocks_per_stream = b->last_NB;
+  if (deciders_per_block) *deciders_per_block = b->last_G;
+  return TB_OK;
 }
 
 extern "C" int tb_batch_set_beam_prune(tb_batch* b, float delta) {
@@ -471,7 +538,7 @@ extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* 
 }
 
 extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {
-  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS))) return TB_ERR_INVALID_ARG;
+  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT))) return TB_ERR_INVALID_ARG;
   b->flags = flags;
   return TB_OK;
 }

@@ -48,6 +48,18 @@ int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
 size_t tb_greedy_fast_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S);
 int tb_launch_greedy_fast(const TbDecodeParams& p, int32_t max_cache_bytes, int32_t max_states, int32_t all_resolved,
                           void* scratch, size_t scratch_bytes, cudaStream_t stream);
+// The segmented kernel (tb_greedy_seg.cu): every stream cut into NB * G segments, NB blocks per stream with G decider
+// warps and H helper warps each.  force_*: non-zero values override the automatic choice (tuning).
+struct TbSegPlan {
+  int32_t G = 0, H = 0, NB = 0, smem = 0;
+  int32_t force_G = 0, force_H = 0, force_NB = 0;
+  int32_t test_timeout = 0;   // self-test: one frame is withheld and the waits are short, so a wait runs out
+};
+bool tb_greedy_seg_plan(const TbDecodeParams& p, int32_t max_cache_bytes, int32_t all_resolved, int32_t n_sm,
+                        int32_t max_smem, TbSegPlan* plan);
+size_t tb_greedy_seg_scratch_bytes(int32_t n_streams, int32_t frames, int32_t S, int32_t nseg_max);
+int tb_launch_greedy_seg(const TbDecodeParams& p, int32_t max_cache_bytes, const TbSegPlan& plan, void* scratch,
+                         cudaStream_t stream);
 int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
 int tb_launch_beam_frames(const TbBeamParams& p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
                           cudaStream_t stream);

@@ -156,23 +156,60 @@ def test_error_codes(tb):
 # the pipelined kernel (packed bf16) against the oracle and against the general kernel
 # ---------------------------------------------------------------------------------------------
 
-def both_kernels(tb, w, data, phrase_lists=None, weights=None, lam=None, lengths=None, logits=None, what=""):
+SEG_PLANS = [(2, 8, 0), (1, 3, 1), (3, 7, 2), (4, 9, 3)]    # deciders, helpers per block; blocks per stream (0: automatic)
+
+
+def both_kernels(tb, w, data, phrase_lists=None, weights=None, lam=None, lengths=None, logits=None, what="", plans=SEG_PLANS,
+                 expect_fast=None):
+    """Every kernel tb_greedy_decode can take -- the segmented one under several plans, the one-block-per-stream
+    pipelined one, the general one -- against the oracle, stream by stream; all must agree bit for bit."""
     phrase_lists = data["phrases"] if phrase_lists is None else phrase_lists
     batch, _ = make_batch(tb, w, phrase_lists, weights=weights, lam=lam)
     logits = to_device(data["logits"]) if logits is None else logits
     dl = None if lengths is None else torch.tensor(lengths, dtype=torch.int32, device="cuda:0")
-    fast = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
-    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
-    gen = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
-    tb.tb_batch_set_flags(batch, 0)
-    assert tb.tb_batch_status(batch) == 0
+    refs = []
     for i, p in enumerate(phrase_lists):
         g = oracle_graph(w, p, None if weights is None else weights[i], lam)
-        ref = O.greedy_rnnt(g, data["logits"][i], None if lengths is None else lengths[i])
-        check_greedy(fast, i, ref, what + " pipelined")
-        check_greedy(gen, i, ref, what + " general")
-        assert fast["scores"][i] == gen["scores"][i]
+        refs.append(O.greedy_rnnt(g, data["logits"][i], None if lengths is None else lengths[i]))
+    outs = {}
+    for plan in plans:
+        tb.tb_batch_set_greedy_plan(batch, *plan)
+        outs[f"segmented{plan}"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+        outs[f"segmented{plan} again"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))   # what the first launch left must not matter
+        if expect_fast is not None:
+            assert (tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_SEGMENTED) == expect_fast, plan
+    tb.tb_batch_set_greedy_plan(batch, 0, 0, 0)
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
+    fast = outs["pipelined"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+    if expect_fast is not None:
+        assert (tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_PIPELINED) == expect_fast
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
+    outs["general"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=dl))
+    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_GENERAL
+    tb.tb_batch_set_flags(batch, 0)
+    assert tb.tb_batch_status(batch) == 0
+    for name, out in outs.items():
+        for i, ref in enumerate(refs):
+            check_greedy(out, i, ref, f"{what} {name}")
+            assert out["scores"][i] == fast["scores"][i], (name, i)
     return fast
+
+
+def decode_every_way(tb, batch, logits, lengths, seed=0):
+    """Outputs of tb_greedy_decode on one batch under the default choice of kernel, a forced segmented plan (where the
+    call fits the segmented kernel; otherwise the library falls back by itself), the one-block-per-stream pipelined
+    kernel and the general kernel."""
+    outs = {"default": to_host(tb.tb_greedy_decode(batch, logits, lengths=lengths))}
+    tb.tb_batch_set_greedy_plan(batch, *SEG_PLANS[seed % len(SEG_PLANS)])
+    outs["segmented"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=lengths))
+    tb.tb_batch_set_greedy_plan(batch, 0, 0, 0)
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
+    outs["pipelined"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=lengths))
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
+    outs["general"] = to_host(tb.tb_greedy_decode(batch, logits, lengths=lengths))
+    tb.tb_batch_set_flags(batch, 0)
+    assert tb.tb_batch_status(batch) == 0
+    return outs
 
 
 @pytest.mark.parametrize("V,S,T", [(1024, 3, 150), (300, 4, 70), (256, 1, 90), (2048, 2, 40), (700, 3, 33)])
@@ -183,7 +220,7 @@ def test_pipelined_kernel_shapes(tb, V, S, T):
     lists[1] = None
     lists[4] = []
     lengths = [T, T - 1, 0, 1, T // 2, T, 3]
-    both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"V{V}S{S}")
+    both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"V{V}S{S}", expect_fast=V <= 2047)
 
 
 @pytest.mark.parametrize("lam", [0.5, 2.0, -1.0])
@@ -277,15 +314,12 @@ def test_pipelined_kernel_random_configurations(tb, seed):
     view.copy_(to_device(xb))
     lens = rng.integers(0, T + 1, size=B).astype(np.int32)
     dl = torch.from_numpy(lens).to("cuda:0")
-    fast = to_host(tb.tb_greedy_decode(batch, view, lengths=dl))
-    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
-    gen = to_host(tb.tb_greedy_decode(batch, view, lengths=dl))
-    assert tb.tb_batch_status(batch) == 0
+    outs = decode_every_way(tb, batch, view, dl, seed)
     for i, p in enumerate(lists):
         g = None if p is None else O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam)
         ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
-        check_greedy(fast, i, ref, f"seed{seed} pipelined V{V} S{S}")
-        check_greedy(gen, i, ref, f"seed{seed} general V{V} S{S}")
+        for name, out in outs.items():
+            check_greedy(out, i, ref, f"seed{seed} {name} V{V} S{S}")
 
 
 # ---------------------------------------------------------------------------------------------
@@ -329,15 +363,12 @@ def test_two_segment_decode_slow_to_meet(tb, seed):
         tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc, token_weights=weights[i], lam=lam))
     lens = np.array([T, T - 3, 128, T, 250 if T >= 250 else T], dtype=np.int32)
     dl = torch.from_numpy(lens).to("cuda:0")
-    out = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=dl))
-    tb.tb_batch_set_flags(batch, tb.TB_FLAG_GENERAL_KERNELS)
-    gen = to_host(tb.tb_greedy_decode(batch, to_device(xb), lengths=dl))
-    assert tb.tb_batch_status(batch) == 0
+    outs = decode_every_way(tb, batch, to_device(xb), dl, seed)
     for i, p in enumerate(lists):
         ref = O.greedy_rnnt(O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam), xb[i], int(lens[i]))
-        check_greedy(out, i, ref, f"seed {seed} pipelined")
-        check_greedy(gen, i, ref, f"seed {seed} general")
-        assert out["scores"][i] == gen["scores"][i]
+        for name, out in outs.items():
+            check_greedy(out, i, ref, f"seed {seed} {name}")
+            assert out["scores"][i] == outs["general"]["scores"][i]
 
 
 def test_two_segment_decode_repeats_and_rebinding(tb):
@@ -392,13 +423,13 @@ def test_pipelined_kernel_soak_against_oracle(tb, block):
         view = flat[shift:shift + xb.size].view(B, T, S, V + 1)
         view.copy_(to_device(xb))
         lens = rng.integers(max(0, T - 40), T + 1, size=B).astype(np.int32)
-        out = to_host(tb.tb_greedy_decode(batch, view, lengths=torch.from_numpy(lens).to("cuda:0")))
-        assert tb.tb_batch_status(batch) == 0
+        outs = decode_every_way(tb, batch, view, torch.from_numpy(lens).to("cuda:0"), seed)
         for i, p in enumerate(lists):
             g = None if p is None else O.Graph(p, V, case_class=cc, weights=weights[i], lam=lam)
             ref = O.greedy_rnnt(g, xb[i], int(lens[i]))
-            check_greedy(out, i, ref, f"seed {seed}")
-            assert float(out["scores"][i]) == float(ref["score"]), f"seed {seed} stream {i}: score bits"
+            for name, out in outs.items():
+                check_greedy(out, i, ref, f"seed {seed} {name}")
+                assert float(out["scores"][i]) == float(ref["score"]), f"seed {seed} stream {i} {name}: score bits"
 
 
 def test_greedy_decode_in_a_cuda_graph(tb):
@@ -452,9 +483,134 @@ def test_pipelined_kernel_masked_logits(tb, seed):
     batch = tb.tb_batch_create(V, cc, B, arena_bytes=8 << 20)
     for i, p in enumerate(lists):
         tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, V, case_class=cc))
-    out = to_host(tb.tb_greedy_decode(batch, to_device(xb)))
-    assert tb.tb_batch_status(batch) == 0
+    outs = decode_every_way(tb, batch, to_device(xb), None, seed)
     for i, p in enumerate(lists):
         ref = O.greedy_rnnt(O.Graph(p, V, case_class=cc), xb[i])
-        check_greedy(out, i, ref, f"masked seed {seed}")
-        assert float(out["scores"][i]) == float(ref["score"]) or (np.isinf(ref["score"]) and np.isinf(out["scores"][i]))
+        for name, out in outs.items():
+            check_greedy(out, i, ref, f"masked seed {seed} {name}")
+            assert float(out["scores"][i]) == float(ref["score"]) or (np.isinf(ref["score"]) and np.isinf(out["scores"][i]))
+
+
+# ---------------------------------------------------------------------------------------------
+# the segmented kernel: cut points, streams whose segments never meet, choice of kernel, reuse of its scratch memory
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("T", [47, 48, 49, 95, 96, 97, 143, 145, 191, 193, 400])
+def test_segmented_decode_cut_points(tb, T):
+    """Lengths on both sides of every multiple of the shortest segment (48 frames), so that the number of segments
+    and their cut points change from stream to stream within one launch."""
+    w = W.get_workload(2, B=7, T=T, n_phrases=60, n_plants=max(1, T // 25))
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[3] = None
+    lengths = [T, T - 1, max(0, T - 47), T, max(0, T - 48), max(0, T - 49), 1]
+    both_kernels(tb, w, data, phrase_lists=lists, lengths=lengths, what=f"cut points T{T}", expect_fast=True)
+
+
+def test_segmented_decode_segments_that_never_meet(tb):
+    """A list with a phrase that repeats one class makes the graph state loop on itself: the decode stays in that
+    state for most of the stream, a segment that starts in the root state hardly ever reaches it, and the first
+    segment ends up decoding almost everything (with another list on the same logits as a control)."""
+    w = W.get_workload(2, B=4, T=600, n_phrases=30, n_plants=0)
+    data = W.batch_inputs(w)
+    c = 5                                                     # class 5: tokens 15, 16, 17
+    loop = [[15] * 6, [15, 15], [15, 40, 41]]
+    lists = [loop + data["phrases"][0], data["phrases"][1], loop, None]
+    x = W.bf16_bits_to_f32(data["logits"])
+    x[:, :, :, 15:18] += 1.0                                  # the class is frequent enough to enter the loop, not to stay without it
+    data["logits"] = W.f32_to_bf16_bits(x)
+    fast = both_kernels(tb, w, data, phrase_lists=lists, what="never meet", expect_fast=True)
+    assert fast["counts"][0] > 2 * fast["counts"][1] and fast["counts"][2] > 2 * fast["counts"][3]
+
+
+def test_choice_of_greedy_kernel(tb):
+    """Which kernel a call gets: few streams -> segmented (many blocks per stream); a full batch -> one block per
+    stream; fp32 or a padded token stride -> general.  A silent fall-back would cost a factor, so it is observable."""
+    w = W.get_workload(2, B=8, T=200, n_phrases=40, n_plants=5)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    logits = to_device(data["logits"])
+    tb.tb_greedy_decode(batch, logits)
+    k = tb.tb_batch_last_greedy_kernel(batch)
+    assert k["kernel"] == tb.TB_KERNEL_SEGMENTED and k["blocks_per_stream"] * k["deciders_per_block"] >= 2
+    big = W.get_workload(2, B=128, T=60, n_phrases=20, n_plants=2)
+    dbig = W.batch_inputs(big)
+    bbatch, _ = make_batch(tb, big, dbig["phrases"])
+    tb.tb_greedy_decode(bbatch, to_device(dbig["logits"]))
+    assert tb.tb_batch_last_greedy_kernel(bbatch)["kernel"] == tb.TB_KERNEL_PIPELINED
+    tb.tb_greedy_decode(batch, logits.float())
+    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_GENERAL
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_set_greedy_plan(batch, 5, 4, 0)
+    with pytest.raises(tb.TbError):
+        tb.tb_batch_set_greedy_plan(batch, 2, 0, 0)
+
+
+def test_segmented_decode_reuses_its_scratch_memory(tb):
+    """Launches of different shapes on one batch (more streams, longer streams, another plan) and back: the working
+    memory is laid out anew each time and nothing of an earlier launch is taken for a record of this one."""
+    w = W.get_workload(2, B=6, T=300, n_phrases=50, n_plants=10)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    logits = to_device(data["logits"])
+    refs = [O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]) for i in range(w.B)]
+    refs150 = [O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i, :150]) for i in range(w.B)]
+    for plan, nb, T in [((2, 8, 3), 6, 300), ((2, 8, 3), 3, 300), ((3, 7, 2), 6, 150), ((2, 8, 3), 6, 300), ((1, 3, 4), 6, 300),
+                        ((2, 8, 3), 6, 300)]:
+        tb.tb_batch_set_greedy_plan(batch, *plan)
+        for _ in range(3):
+            out = to_host(tb.tb_greedy_decode(batch, logits[:nb, :T]))
+            assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_SEGMENTED
+            for i in range(nb):
+                check_greedy(out, i, (refs if T == 300 else refs150)[i], f"plan {plan} nb {nb} T {T}")
+    assert tb.tb_batch_status(batch) == 0
+
+
+def test_segmented_decode_in_a_cuda_graph(tb):
+    """The segmented decode captured once and replayed: every replay starts from what the previous one left in the
+    working memory (launch numbers advance on the device), with other logits in the same buffer each time."""
+    w = W.get_workload(2, B=5, T=260, n_phrases=50, n_plants=10)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    tb.tb_batch_set_greedy_plan(batch, 2, 8, 3)
+    logits = to_device(data["logits"]).clone()
+    out = tb.tb_greedy_decode(batch, logits)                  # allocates the working memory (not allowed while capturing)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        tb.tb_greedy_decode(batch, logits, out=out, stream=torch.cuda.current_stream())
+    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_SEGMENTED
+    for shift in (0, 1, 2):
+        rolled = np.roll(data["logits"], shift, axis=0)        # stream i now carries the logits of stream i - shift
+        logits.copy_(to_device(rolled))
+        for v in out.values():
+            v.zero_()
+        graph.replay()
+        host = to_host(out)
+        for i in range(w.B):
+            check_greedy(host, i, O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), rolled[i]), f"replay, shift {shift}")
+    assert tb.tb_batch_status(batch) == 0
+
+
+def test_a_bounded_wait_that_runs_out(tb):
+    """The kernels wait for each other's results with a limit on every wait.  The self-test flag makes one wait run
+    out on purpose (a frame's summaries are withheld, the limit is a few thousand polls): the call returns, the status
+    word carries TB_STATUS_WAIT_TIMEOUT, and the next ordinary decode on the same batch is bit-exact again."""
+    w = W.get_workload(2, B=6, T=200, n_phrases=40, n_plants=6)
+    data = W.batch_inputs(w)
+    batch, _ = make_batch(tb, w, data["phrases"])
+    logits = to_device(data["logits"])
+    refs = [O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]) for i in range(w.B)]
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_TEST_WAIT_TIMEOUT)
+    tb.tb_greedy_decode(batch, logits)
+    torch.cuda.synchronize()                                  # the launch ends by itself
+    status = tb.tb_batch_status(batch)
+    assert status & tb.TB_STATUS_WAIT_TIMEOUT, status
+    assert tb.tb_batch_status(batch) == 0                     # reading the status clears it
+    tb.tb_batch_set_flags(batch, 0)
+    for _ in range(2):
+        out = to_host(tb.tb_greedy_decode(batch, logits))
+        assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_SEGMENTED
+        for i in range(w.B):
+            check_greedy(out, i, refs[i], "after the timeout")
+    assert tb.tb_batch_status(batch) == 0
