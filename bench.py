@@ -278,6 +278,74 @@ def side_measurement(args):
                           "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
                           "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds), "data": "synthetic"}))
 
+    elif args.workload == 8:
+        # Streaming beam search (Sec. 2.3; Sec. 3.4 uses beam 32): the streaming workload's churn without duration
+        # logits, 2 expansions per frame, chunks of 8 frames through tb_beam_chunk; equal transcripts merged and the
+        # beam pruned at frame starts; a finished stream gets its final weights and a backtrace, a new one is compiled
+        # and bound.  Timed per chunk with the binds and the finishing calls inside the timed region.
+        rows = []
+        for K in (4, 32):
+            w = W.get_workload(5, B=args.streams or 128, S=2, n_dur=0)
+            E = w.S
+            sched = W.ChurnSchedule(w, workers=8)
+            batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=K, max_tree_steps=w.T * E, arena_bytes=256 << 20)
+            tb.tb_batch_set_beam_prune(batch, 10.0)
+            scores = torch.full((w.B, K), float("-inf"), device=dev)
+            states = torch.full((w.B, K), -1, dtype=torch.int32, device=dev)
+            live = torch.zeros((w.B, K), dtype=torch.uint8, device=dev)
+            par = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+            tok = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+            tb.tb_beam_reset_slots(batch)
+            served = np.zeros(w.B, dtype=np.int64)
+            total = np.zeros(w.B, dtype=np.int64)
+            n_chunks, lat, kern, n_done, frames = 30 + 2 * args.steps, [], [], 0, 0
+            bufs = []
+            for c in range(n_chunks):
+                chunk, lengths, bl = sched.next_chunk()
+                gs = [(sl, tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class)) for sl, _, p in bl]
+                for sl, _, _ in bl:
+                    served[sl] = 0
+                total[:] = lengths
+                left = np.clip(total - served, 0, w.chunk).astype(np.int32)
+                dl = torch.from_numpy(chunk).view(torch.bfloat16).to(dev)   # a fresh buffer per chunk: nothing stays in L2
+                dn = torch.from_numpy(left).to(dev)
+                bufs = (bufs + [dl])[-8:]
+                new = [sl for sl, _ in gs]
+                idx = torch.tensor(new, device=dev, dtype=torch.long) if new else None
+                torch.cuda.synchronize()
+                a, m0, m1, b = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+                a.record()
+                for sl, g in gs:
+                    tb.tb_batch_bind_stream(batch, sl, g)
+                if new:
+                    scores[idx] = float("-inf"); scores[idx, 0] = 0.0
+                    states[idx] = -1; states[idx, 0] = 0
+                    live[idx] = 0
+                    tb.tb_beam_reset_slots(batch, new)
+                m0.record()
+                tb.tb_beam_chunk(batch, dl, True, dn, scores, states, live, par, tok)
+                m1.record()
+                served += left
+                ended = [sl for sl in range(w.B) if left[sl] > 0 and served[sl] >= total[sl]]
+                if ended:
+                    tb.tb_apply_final_weights_slots(batch, ended, scores, states)
+                    tb.tb_beam_backtrace_slots(batch, w.B, K, 256)
+                b.record()
+                torch.cuda.synchronize()
+                lat.append(a.elapsed_time(b)); kern.append(m0.elapsed_time(m1))
+                n_done += len(ended); frames += int(left.sum())
+            assert tb.tb_batch_status(batch) == 0
+            sched.close()
+            lat, kern = np.array(lat[10:]), np.array(kern[10:])
+            rows.append({"K": K, "p50_ms": float(np.percentile(lat, 50)), "p99_ms": float(np.percentile(lat, 99)),
+                         "chunk_kernel_p50_ms": float(np.percentile(kern, 50)),
+                         "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
+                         "chunks": int(len(lat)), "streams_finished": n_done})
+        print(json.dumps({"metric": "streaming_beam_chunk_latency_ms", "unit": "ms", "higher_is_better": False, "n_gpus": 1,
+                          "rows": rows, "config": {"workload": "streaming_beam_churn", "slots": w.B, "chunk_frames": w.chunk,
+                                                   "expansions_per_frame": E, "merge": True, "prune_delta": 10.0,
+                                                   "binds_and_finishing_in_timed_region": True}, "data": "synthetic"}))
+
     elif args.workload == 7:
         # Model lifecycle sweep in the manner of the paper's speed table (128 streams; cache: none / disk / memory /
         # decoder): the streaming workload's churn with 128 slots, the same schedule for every mode; the timed region of
@@ -406,7 +474,7 @@ def main():
     ap.add_argument("--streams", type=int, default=0, help="override B (profiling captures use a small case)")
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
-    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7],
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7, 8],
                     help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists, 7 model lifecycle sweep: side measurements")
     args = ap.parse_args()
     if args.workload != 2:

@@ -417,6 +417,39 @@ int tb_beam_frames(tb_batch *b, const void *logits, int dtype, int32_t B, int32_
                    int32_t *states, uint8_t *live, int32_t *out_parent, int32_t *out_token, void *stream);
 
 /*
+ * Streaming beam decoding, slot by slot (Sec. 2.3: the hypotheses a stream holds at the end of a chunk -- their
+ * place in the flattened tree, accumulated scores and graph states -- are kept and are what the next chunk continues,
+ * merges and prunes; Sec. 2.2 para. 4: streams end and new ones start on their slots between chunks).
+ * Every slot has its own hypothesis tree (a ring of max_tree_steps * max_beam / K steps inside the batch's tree
+ * buffer) and its own position in it, so slots start, pause and end independently.  The caller's [n_slots, K] arrays
+ * hold scores, graph states and liveness as for tb_beam_step.  A session: tb_beam_reset_slots(b, 0, NULL) for all
+ * slots, or for the slots on which a new utterance starts (the caller also sets those slots' rows of the arrays:
+ * score 0 / -inf..., state 0 or -1, as for an utterance's first tb_beam_step); then per chunk tb_beam_chunk; when a
+ * stream has ended tb_apply_final_weights_slots and tb_beam_backtrace_slots give its result.  tb_beam_reset ends the
+ * session (tb_beam_step / tb_beam_frames refuse to run during one, and tb_beam_chunk after them without a reset).
+ *
+ * tb_beam_reset_slots: n = 0 resets every slot; else `slots` is a host int32 array of n slot indices.  Device work
+ *   on `stream` (position 0, empty token sequences).  Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG, TB_ERR_CUDA.
+ * tb_beam_chunk: for slot i, n_frames[i] (device int32 [n_slots], clamped to [0, chunk]; NULL: chunk) frames of E
+ *   expansions, exactly as tb_beam_frames does them for a whole batch (every hypothesis of slot i reads the row at
+ *   element offset i*stream_stride + t*frame_stride + e*row_stride; merge and pruning at frame starts); a slot with
+ *   n_frames 0 is left alone (its out_parent / out_token rows are not written).  K must stay the same from one
+ *   reset of all slots to the next.  Errors: TB_ERR_INVALID_ARG (no tree, K, a batch-wide tree in use), TB_ERR_CUDA.
+ * tb_beam_backtrace_slots: as tb_beam_backtrace, each slot walked back to the start of its own utterance; an
+ *   utterance longer than the slot's ring sets TB_STATUS_STEP_LIMIT and yields the tokens still in the ring.
+ * tb_apply_final_weights_slots: tb_apply_final_weights for the rows of the [n_slots, K] arrays that `slots` (host
+ *   int32 [n]) names.
+ */
+int tb_beam_reset_slots(tb_batch *b, int32_t n, const int32_t *slots, void *stream);
+int tb_beam_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots, int32_t K, int32_t chunk, int32_t E,
+                  int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge, const int32_t *n_frames,
+                  float *scores, int32_t *states, uint8_t *live, int32_t *out_parent, int32_t *out_token, void *stream);
+int tb_beam_backtrace_slots(tb_batch *b, int32_t n_slots, int32_t K, int32_t max_len, int32_t *out_tokens,
+                            int32_t *out_lens, void *stream);
+int tb_apply_final_weights_slots(tb_batch *b, int32_t n, const int32_t *slots, int32_t K, float *scores,
+                                 const int32_t *states, void *stream);
+
+/*
  * Pruning of the beam (Sec. 2.3 names it; the rule here is the usual threshold against the best hypothesis):
  * with delta >= 0, every tb_beam_step that starts a frame (TB_FRAME_NEW, TB_FRAME_NEW_MERGE) first -- after
  * the merge, if one was asked for -- turns every hypothesis of a stream whose score is below

@@ -84,6 +84,11 @@ _SIGS = {
     "tb_beam_frames": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
                                  _vp]),
     "tb_apply_final_weights": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
+    "tb_beam_reset_slots": (C.c_int, [_vp, _i32, _vp, _vp]),
+    "tb_beam_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
+                                _vp, _vp]),
+    "tb_beam_backtrace_slots": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "tb_apply_final_weights_slots": (C.c_int, [_vp, _i32, _vp, _i32, _vp, _vp, _vp]),
     "tb_batch_set_beam_prune": (C.c_int, [_vp, C.c_float]),
     "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
                                            _vp, _vp, _vp]),
@@ -449,6 +454,44 @@ def tb_beam_frames(batch: Batch, logits: torch.Tensor, merge: bool, scores: torc
     _check(_lib.tb_beam_frames(batch.handle, _dp(logits), _logit_dtype(logits), B, K, logits.shape[1], logits.shape[2],
                                sb, st, se, 1 if merge else 0, _dp(scores), _dp(states), _dp(live), _dp(out_parent),
                                _dp(out_token), _stream(stream)), "tb_beam_frames")
+
+
+def tb_beam_reset_slots(batch: Batch, slots=None, stream=None):
+    """A new utterance on ``slots`` (None: on every slot) for streaming beam decoding."""
+    if slots is None:
+        _check(_lib.tb_beam_reset_slots(batch.handle, 0, None, _stream(stream)), "tb_beam_reset_slots")
+        return
+    sl = _host(slots, np.int32)
+    if len(sl):
+        _check(_lib.tb_beam_reset_slots(batch.handle, len(sl), _hp(sl), _stream(stream)), "tb_beam_reset_slots")
+
+
+def tb_beam_chunk(batch: Batch, logits: torch.Tensor, merge: bool, n_frames, scores: torch.Tensor, states: torch.Tensor,
+                  live: torch.Tensor, out_parent: torch.Tensor, out_token: torch.Tensor, stream=None):
+    """logits [n_slots, chunk, E, vocab+1]; n_frames: device int32 [n_slots] (frames of this chunk each slot decodes)."""
+    B, T, E, W = logits.shape
+    K = scores.shape[1]
+    sb, st, se, sv = logits.stride()
+    assert sv == 1 and W == batch.vocab + 1
+    _check(_lib.tb_beam_chunk(batch.handle, _dp(logits), _logit_dtype(logits), B, K, T, E, sb, st, se, 1 if merge else 0,
+                              _dp(n_frames), _dp(scores), _dp(states), _dp(live), _dp(out_parent), _dp(out_token),
+                              _stream(stream)), "tb_beam_chunk")
+
+
+def tb_beam_backtrace_slots(batch: Batch, n_slots: int, K: int, max_len: int, stream=None):
+    dev = torch.device("cuda", batch.device)
+    toks = torch.zeros((n_slots, K, max_len), dtype=torch.int32, device=dev)
+    lens = torch.zeros((n_slots, K), dtype=torch.int32, device=dev)
+    _check(_lib.tb_beam_backtrace_slots(batch.handle, n_slots, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
+           "tb_beam_backtrace_slots")
+    return toks, lens
+
+
+def tb_apply_final_weights_slots(batch: Batch, slots, scores: torch.Tensor, states: torch.Tensor, stream=None):
+    sl = _host(slots, np.int32)
+    if len(sl):
+        _check(_lib.tb_apply_final_weights_slots(batch.handle, len(sl), _hp(sl), scores.shape[1], _dp(scores), _dp(states),
+                                                 _stream(stream)), "tb_apply_final_weights_slots")
 
 
 def tb_batch_set_beam_prune(batch: Batch, delta: float):

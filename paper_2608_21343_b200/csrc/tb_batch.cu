@@ -95,6 +95,8 @@ struct tb_batch {
   int64_t beam_steps = 0;                     // steps since tb_beam_reset (selects the ping-pong half)
   float beam_prune_delta = -1.0f;             // >= 0: prune at frame starts (tb_batch_set_beam_prune)
   int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
+  int32_t* d_slot_pos = nullptr;              // [n_slots] steps every slot has taken since its last reset (streaming beam decoding)
+  int32_t chunk_K = 0;                        // beam width of the streaming calls since the last reset of all slots (0: none yet)
   ArenaAllocator alloc;
   std::vector<std::pair<size_t, size_t>> slot_block;  // (offset, bytes); bytes == 0: none
   std::vector<int32_t> slot_cache_bytes;               // bytes of the sections the pipelined kernel caches
@@ -132,7 +134,7 @@ static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs); cudaFree(b->d_slot_pos);
   for (auto& s : b->staging) {
     if (s.held) tb_graph_free(s.held);
     if (s.host) cudaFreeHost(s.host);
@@ -181,6 +183,8 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   const size_t n_hyp = static_cast<size_t>(n_slots) * max_beam;
   ok = ok && cudaMalloc(&b->d_hyp_hash, 2 * n_hyp * sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMalloc(&b->d_hyp_len, 2 * n_hyp * sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(&b->d_slot_pos, static_cast<size_t>(n_slots) * sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaMemset(b->d_slot_pos, 0, static_cast<size_t>(n_slots) * sizeof(int32_t)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); destroy_batch(b); return TB_ERR_OOM; }
   ok = ok && cudaMemset(b->d_hyp_hash, 0, 2 * n_hyp * sizeof(unsigned long long)) == cudaSuccess;
   ok = ok && cudaMemset(b->d_hyp_len, 0, 2 * n_hyp * sizeof(int32_t)) == cudaSuccess;
@@ -562,6 +566,7 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
 extern "C" int tb_beam_reset(tb_batch* b) {
   if (!b) return TB_ERR_INVALID_ARG;
   b->tree_steps = 0; b->tree_B = 0; b->tree_K = 0;
+  b->chunk_K = 0;   // (a streaming session, if one was under way, is over: its per-slot trees are reused by the batch-wide one)
   // every hypothesis starts from the empty token sequence: the first step after this ignores the stored records
   b->beam_steps = 0;
   return TB_OK;
@@ -572,6 +577,7 @@ extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t 
                             int32_t* out_parent, int32_t* out_token, void* stream_) {
   if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
   if ((dtype != TB_BF16 && dtype != TB_F32) || B < 1 || B > b->n_slots || K < 1 || K > b->max_beam) return TB_ERR_INVALID_ARG;
+  if (b->chunk_K != 0) return TB_ERR_INVALID_ARG;   // a streaming session is under way: tb_beam_reset ends it
   if (b->d_tree) {
     if (b->tree_steps >= b->max_tree_steps) return TB_ERR_INVALID_ARG;
     if (b->tree_steps > 0 && (b->tree_B != B || b->tree_K != K)) return TB_ERR_INVALID_ARG;
@@ -609,6 +615,7 @@ extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_
       static_cast<int64_t>(T) * E > (1 << 24))
     return TB_ERR_INVALID_ARG;
   const int32_t n_steps = T * E;
+  if (b->chunk_K != 0) return TB_ERR_INVALID_ARG;   // a streaming session is under way: tb_beam_reset ends it
   if (b->d_tree) {
     if (b->tree_steps + n_steps > b->max_tree_steps) return TB_ERR_INVALID_ARG;
     if (b->tree_steps > 0 && (b->tree_B != B || b->tree_K != K)) return TB_ERR_INVALID_ARG;
@@ -634,6 +641,84 @@ extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_
   if (rc == TB_OK) b->beam_steps += n_steps;
   if (rc == TB_OK && b->d_tree) { b->tree_steps += n_steps; b->tree_B = B; b->tree_K = K; }
   return rc;
+}
+
+// ---- streaming beam decoding, slot by slot (Sec. 2.3) --------------------------------------------------------
+
+extern "C" int tb_beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots, void* stream_) {
+  if (!b || n < 0 || (n > 0 && !slots)) return TB_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < n; ++i) if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (n == 0) {   // every slot
+    b->chunk_K = 0;
+    return tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, b->n_slots, nullptr, 1, stream);
+  }
+  for (int32_t at = 0; at < n; at += TB_BIND_PAIRS) {
+    const int32_t m = n - at < TB_BIND_PAIRS ? n - at : TB_BIND_PAIRS;
+    const int rc = tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, m, slots + at, 0, stream);
+    if (rc != TB_OK) return rc;
+  }
+  return TB_OK;
+}
+
+extern "C" int tb_beam_chunk(tb_batch* b, const void* logits, int dtype, int32_t n_slots, int32_t K, int32_t chunk, int32_t E,
+                             int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge,
+                             const int32_t* n_frames, float* scores, int32_t* states, uint8_t* live, int32_t* out_parent,
+                             int32_t* out_token, void* stream_) {
+  if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
+  if ((dtype != TB_BF16 && dtype != TB_F32) || n_slots < 1 || n_slots > b->n_slots || K < 1 || K > b->max_beam || chunk < 1 ||
+      E < 1 || static_cast<int64_t>(chunk) * E > (1 << 24))
+    return TB_ERR_INVALID_ARG;
+  if (!b->d_tree || b->max_tree_steps < 1) return TB_ERR_INVALID_ARG;            // streaming needs the hypothesis tree
+  if (b->chunk_K != 0 && b->chunk_K != K) return TB_ERR_INVALID_ARG;             // one beam width between resets of all slots
+  if (b->tree_steps != 0) return TB_ERR_INVALID_ARG;                             // the tree is in use by tb_beam_step / tb_beam_frames
+  TbBeamParams p;
+  std::memset(&p, 0, sizeof p);
+  p.logits = logits; p.dtype = dtype; p.B = n_slots; p.K = K; p.V = b->vocab; p.C = b->n_classes;
+  p.merge = merge ? 1 : 0; p.prune_delta = b->beam_prune_delta; p.new_frame = 1;
+  p.stream_stride = stream_stride; p.hyp_stride = 0;
+  p.scores = scores; p.states = states; p.live = live; p.out_parent = out_parent; p.out_token = out_token;
+  p.tree = b->d_tree;
+  // each slot's ring: the tree buffer holds max_tree_steps * n_slots * max_beam entries, i.e. per slot
+  // max_tree_steps * max_beam / K steps of K entries (an entry index never leaves the slot's share)
+  p.tree_cap = static_cast<int32_t>(static_cast<int64_t>(b->max_tree_steps) * b->max_beam / K);
+  p.slots = b->d_slots; p.arena = b->arena; p.cls = b->d_cls; p.status = b->d_status;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  const int rc = tb_launch_beam_chunk(p, chunk, E, frame_stride, row_stride, n_frames, b->d_slot_pos, b->d_hyp_hash,
+                                      b->d_hyp_len, n_hyp, static_cast<cudaStream_t>(stream_));
+  if (rc == TB_OK) b->chunk_K = K;
+  return rc;
+}
+
+extern "C" int tb_beam_backtrace_slots(tb_batch* b, int32_t n_slots, int32_t K, int32_t max_len, int32_t* out_tokens,
+                                       int32_t* out_lens, void* stream_) {
+  if (!b || !out_tokens || !out_lens || max_len < 1 || n_slots < 1 || n_slots > b->n_slots) return TB_ERR_INVALID_ARG;
+  if (!b->d_tree || b->chunk_K != K) return TB_ERR_INVALID_ARG;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  const int32_t cap = static_cast<int32_t>(static_cast<int64_t>(b->max_tree_steps) * b->max_beam / K);
+  return tb_launch_beam_backtrace_slots(b->d_tree, cap, b->d_slot_pos, n_slots, K, b->vocab, max_len, out_tokens, out_lens,
+                                        b->d_status, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_apply_final_weights_slots(tb_batch* b, int32_t n, const int32_t* slots, int32_t K, float* scores,
+                                            const int32_t* states, void* stream_) {
+  if (!b || n < 1 || !slots || K < 1 || !scores || !states) return TB_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < n; ++i) if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  for (int32_t at = 0; at < n; at += TB_BIND_PAIRS) {
+    const int32_t m = n - at < TB_BIND_PAIRS ? n - at : TB_BIND_PAIRS;
+    const int rc = tb_launch_final_weights_slots(b->d_slots, b->arena, m, slots + at, K, scores, states, b->d_status,
+                                                 static_cast<cudaStream_t>(stream_));
+    if (rc != TB_OK) return rc;
+  }
+  return TB_OK;
 }
 
 extern "C" int tb_beam_backtrace(tb_batch* b, int32_t B, int32_t K, int32_t max_len, int32_t* out_tokens,

@@ -515,7 +515,11 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
       }
       p.hash_out[o] = nh; p.len_out[o] = nl;
     }
-    if (p.tree) p.tree[(static_cast<int64_t>(p.step) * p.B + b) * K + r] = make_int2(parent, token);
+    if (p.tree) {
+      const int64_t at = p.tree_cap > 0 ? static_cast<int64_t>(b) * p.tree_cap + (p.step % p.tree_cap)
+                                        : static_cast<int64_t>(p.step) * p.B + b;
+      p.tree[at * K + r] = make_int2(parent, token);
+    }
   }
   // ... and in shared memory, for the next step of a launch that runs several (read by every thread above: wait)
   __syncthreads();
@@ -559,6 +563,80 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, in
       beam_step_body<LT>(q, xpre, xpre_valid, next_row);
       __syncthreads();
     }
+  }
+}
+
+// A chunk of streaming beam decoding: slot by slot, n_frames[slot] frames (at most T) of E rows; each slot has its own
+// position in its own tree ring and its own parity of the sequence-record halves, so that slots start, pause and end
+// independently of each other (Sec. 2.3: hypotheses kept across chunks; Sec. 2.2 para. 4: slots re-bound in between).
+template <typename LT>
+__global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
+                                                         int64_t row_stride, const int32_t* n_frames, int32_t* slot_pos,
+                                                         unsigned long long* hash, int32_t* len, size_t n_hyp) {
+  float xpre[kBeamPref];
+  bool xpre_valid = false;
+  const int b = blockIdx.x;
+  const int32_t nf = n_frames ? max(0, min(T, n_frames[b])) : T;
+  const int32_t pos0 = slot_pos[b];
+  const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+  for (int32_t t = 0; t < nf; ++t) {
+    for (int32_t e = 0; e < E; ++e) {
+      const int32_t sidx = t * E + e;
+      TbBeamParams q = p;
+      q.logits = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
+      q.hyp_stride = 0;
+      q.new_frame = e == 0 ? 1 : 0;
+      q.merge = e == 0 ? p.merge : 0;
+      q.prune_delta = e == 0 ? p.prune_delta : -1.0f;
+      q.fresh = 0;
+      q.tv_ready = sidx > 0 ? 1 : 0;
+      q.step = pos0 + sidx;
+      const size_t in = ((pos0 + sidx) & 1) ? n_hyp : 0, out = ((pos0 + sidx) & 1) ? 0 : n_hyp;
+      q.hash_in = hash + in; q.hash_out = hash + out; q.len_in = len + in; q.len_out = len + out;
+      const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
+      const LT* next_row = nt < nf ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
+      beam_step_body<LT>(q, xpre, xpre_valid, next_row);
+      __syncthreads();
+    }
+  }
+  if (threadIdx.x == 0) slot_pos[b] = pos0 + nf * E;
+}
+
+struct SlotList { int32_t slot[TB_BIND_PAIRS]; };
+// A new utterance on some slots (or on all): position 0 in the slot's tree, every hypothesis' sequence empty.
+__global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
+                                   int32_t n, SlotList sl, int32_t all_slots) {
+  const int i = blockIdx.x;
+  if (i >= n) return;
+  const int slot = all_slots ? i : sl.slot[i];
+  if (threadIdx.x == 0) slot_pos[slot] = 0;
+  for (int k = threadIdx.x; k < max_beam; k += blockDim.x) {
+    const size_t o = static_cast<size_t>(slot) * max_beam + k;
+    hash[o] = 0ull; hash[n_hyp + o] = 0ull; len[o] = 0; len[n_hyp + o] = 0;
+  }
+}
+
+// The tokens of every hypothesis a slot holds, walked back through the slot's own ring to the start of its utterance.
+__global__ void k_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
+                                       int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_slots * K) return;
+  const int b = idx / K;
+  const int32_t pos = slot_pos[b];
+  if (pos > tree_cap && idx % K == 0) atomicOr(status, TB_STATUS_STEP_LIMIT);   // the utterance is longer than the ring: its start is gone
+  const int32_t first = max(0, pos - tree_cap);
+  int32_t n = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    int32_t slot = idx % K, at = n;
+    for (int32_t st = pos - 1; st >= first && slot >= 0; --st) {
+      const int2 e = tree[(static_cast<int64_t>(b) * tree_cap + (st % tree_cap)) * K + slot];
+      if (e.y >= 0 && e.y != V) {
+        if (pass == 0) ++n;
+        else { --at; if (at < max_len) out_tokens[static_cast<int64_t>(idx) * max_len + at] = e.y; }
+      }
+      slot = e.x;
+    }
+    if (pass == 0) out_lens[idx] = n;
   }
 }
 
@@ -729,5 +807,70 @@ int tb_launch_bind_models(TbSlotRec* slots, TbSlotState* sstate, const TbSlotRec
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
                            cudaStream_t stream) {
   k_publish_slot<<<1, 32, 0, stream>>>(slots, sstate, slot, rec);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+namespace {
+__global__ void k_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, SlotList sl, int32_t K,
+                                      float* scores, const int32_t* states, int32_t* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n * K) return;
+  const int slot = sl.slot[i / K];
+  const int64_t o = static_cast<int64_t>(slot) * K + i % K;
+  const TbSlotRec rec = slots[slot];
+  const float sc = scores[o];
+  const int32_t st = states[o];
+  if (rec.n_states <= 0 || st < 0 || sc == -INFINITY) return;
+  if (st >= rec.n_states) { atomicOr(status, TB_STATUS_BAD_STATE); return; }
+  const float fw = reinterpret_cast<const float*>(arena + rec.blob_off + rec.off_final)[st];
+  scores[o] = __fadd_rn(sc, __fmul_rn(rec.lambda, fw));
+}
+}  // namespace
+
+int tb_launch_beam_chunk(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
+                         const int32_t* n_frames, int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp,
+                         cudaStream_t stream) {
+  TbBeamParams p = p_in;
+  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
+  p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
+  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
+                      ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
+  if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
+  int rc;
+  if (p.dtype == TB_BF16) {
+    if ((rc = set_smem(k_beam_chunk<uint16_t>, smem)) != TB_OK) return rc;
+    k_beam_chunk<uint16_t><<<p.B, kBeamThreads, smem, stream>>>(p, T, E, frame_stride, row_stride, n_frames, slot_pos, hash, len, n_hyp);
+  } else {
+    if ((rc = set_smem(k_beam_chunk<float>, smem)) != TB_OK) return rc;
+    k_beam_chunk<float><<<p.B, kBeamThreads, smem, stream>>>(p, T, E, frame_stride, row_stride, n_frames, slot_pos, hash, len, n_hyp);
+  }
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
+                               int32_t n, const int32_t* slots, int32_t all_slots, cudaStream_t stream) {
+  if (n < 1 || (!all_slots && n > TB_BIND_PAIRS)) return TB_ERR_INVALID_ARG;
+  SlotList sl;
+  for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = (!all_slots && i < n) ? slots[i] : 0;
+  k_beam_reset_slots<<<n, 32, 0, stream>>>(slot_pos, hash, len, n_hyp, max_beam, n, sl, all_slots);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
+                                   int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status,
+                                   cudaStream_t stream) {
+  const int n = n_slots * K;
+  k_beam_backtrace_slots<<<(n + 127) / 128, 128, 0, stream>>>(tree, tree_cap, slot_pos, n_slots, K, V, max_len, out_tokens, out_lens, status);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, const int32_t* slot_list,
+                                  int32_t K, float* scores, const int32_t* states, int32_t* status, cudaStream_t stream) {
+  if (n < 1 || n > TB_BIND_PAIRS) return TB_ERR_INVALID_ARG;
+  SlotList sl;
+  for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = i < n ? slot_list[i] : 0;
+  const int total = n * K;
+  k_final_weights_slots<<<(total + 127) / 128, 128, 0, stream>>>(slots, arena, n, sl, K, scores, states, status);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }

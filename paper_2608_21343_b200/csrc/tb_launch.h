@@ -36,6 +36,9 @@ struct TbBeamParams {
   float prune_delta;         // >= 0: at a frame start, hypotheses scoring below best - prune_delta are dropped
   int32_t tv_ready;          // set inside a multi-step launch: the block's root tables in shared memory are filled already
   int32_t fresh;             // first step after a reset: every hypothesis has the empty sequence, *_in is not read
+  // streaming (tb_beam_chunk): every slot keeps its own ring of tree_cap steps, tree[slot][step % tree_cap][K]; 0: the
+  // tree is [steps, B, K] for the whole batch
+  int32_t tree_cap;
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
 };
 
@@ -63,6 +66,18 @@ int tb_launch_greedy_seg(const TbDecodeParams& p, int32_t max_cache_bytes, const
 int tb_launch_beam_step(const TbBeamParams& p, cudaStream_t stream);
 int tb_launch_beam_frames(const TbBeamParams& p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
                           cudaStream_t stream);
+// Streaming beam decoding, slot by slot (tb_beam_chunk and friends).  slot_pos: device [n_slots], steps each slot has
+// taken since its last reset; hash / len: both halves of the per-hypothesis sequence records, n_hyp entries apart.
+int tb_launch_beam_chunk(const TbBeamParams& p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
+                         const int32_t* n_frames, int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp,
+                         cudaStream_t stream);
+int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
+                               int32_t n, const int32_t* slots, int32_t all_slots, cudaStream_t stream);
+int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
+                                   int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status,
+                                   cudaStream_t stream);
+int tb_launch_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, const int32_t* slot_list,
+                                  int32_t K, float* scores, const int32_t* states, int32_t* status, cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
 // Registered models: their records live in a device table; tb_launch_bind_models points up to TB_BIND_PAIRS slots at

@@ -1,0 +1,118 @@
+"""GPU parity for streaming beam decoding (tb_beam_reset_slots / tb_beam_chunk / tb_beam_backtrace_slots /
+tb_apply_final_weights_slots) against the CPU oracle: streams of different lengths come and go on their slots
+(Sec. 2.2 para. 4), every slot keeps its hypotheses -- tree, scores, graph states -- from chunk to chunk (Sec. 2.3),
+equal transcripts are merged and the beam is pruned at frame starts, and a finished stream is charged its final
+weights.  The oracle decodes each stream on its own, whole, with the same options."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2608_21343_b200 import workloads as W
+from helpers import SCORE_TOL, oracle_graph, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=False):
+    """Chunks of w.chunk frames over w.B slots with stream churn; returns the number of streams checked."""
+    E = w.S
+    sched = W.ChurnSchedule(w)
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=K, max_tree_steps=w.T * E, arena_bytes=32 << 20)
+    if prune_delta is not None:
+        tb.tb_batch_set_beam_prune(batch, prune_delta)
+    dev = torch.device("cuda:0")
+    scores = torch.full((w.B, K), float("-inf"), device=dev)
+    states = torch.full((w.B, K), -1, dtype=torch.int32, device=dev)
+    live = torch.zeros((w.B, K), dtype=torch.uint8, device=dev)
+    par = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+    tok = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+    tb.tb_beam_reset_slots(batch)                        # a new session: every slot at the start of an utterance
+    slot = [None] * w.B
+    served = np.zeros(w.B, dtype=np.int64)
+    checked = 0
+    for c in range(n_chunks):
+        chunk, lengths, binds = sched.next_chunk()
+        new = []
+        for s, _sid, phrases in binds:
+            g = tb.tb_graph_compile(phrases, w.V, case_class=w.vocab.case_class)
+            tb.tb_batch_bind_stream(batch, s, g)
+            slot[s] = dict(phrases=phrases, logits=sched.data[s]["logits"], length=int(sched.data[s]["length"]))
+            served[s] = 0
+            new.append(s)
+        if new:
+            idx = torch.tensor(new, device=dev)
+            scores[idx] = float("-inf")
+            scores[idx, 0] = 0.0
+            states[idx] = -1
+            states[idx, 0] = 0
+            live[idx] = 0
+            tb.tb_beam_reset_slots(batch, new)
+        left = np.clip(np.array([slot[s]["length"] for s in range(w.B)]) - served, 0, w.chunk).astype(np.int32)
+        tb.tb_beam_chunk(batch, to_device(chunk), merge, torch.from_numpy(left).to(dev), scores, states, live, par, tok)
+        served += left
+        ended = [s for s in range(w.B) if left[s] > 0 and served[s] >= slot[s]["length"]]
+        if check_partial and c % 3 == 1:
+            # the running result of a stream in mid-utterance: the oracle on the frames decoded so far
+            s = int(np.argmax(served * (served < np.array([slot[i]["length"] for i in range(w.B)]))))
+            toks, lens = tb.tb_beam_backtrace_slots(batch, w.B, K, w.T * E)
+            ref = O.beam_decode(oracle_graph(w, slot[s]["phrases"]), slot[s]["logits"][:served[s]], K, merge=merge,
+                                prune_delta=-1.0 if prune_delta is None else prune_delta)
+            assert np.array_equal(lens[s].cpu().numpy(), ref["lens"]), (c, s)
+            assert np.array_equal(states[s].cpu().numpy(), ref["states"]), (c, s)
+        if ended:
+            tb.tb_apply_final_weights_slots(batch, ended, scores, states)
+            toks, lens = tb.tb_beam_backtrace_slots(batch, w.B, K, w.T * E)
+            torch.cuda.synchronize()
+            h_tok, h_len, h_sc, h_st = toks.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), states.cpu().numpy()
+            for s in ended:
+                g = oracle_graph(w, slot[s]["phrases"])
+                ref = O.beam_decode(g, slot[s]["logits"][:slot[s]["length"]], K, merge=merge,
+                                    prune_delta=-1.0 if prune_delta is None else prune_delta)
+                assert np.array_equal(h_len[s], ref["lens"]), (c, s, "lengths")
+                assert np.array_equal(h_st[s], ref["states"]), (c, s, "states")
+                for k in range(K):
+                    assert np.array_equal(h_tok[s, k, :ref["lens"][k]], ref["tokens"][k]), (c, s, k)
+                    if np.isfinite(ref["scores"][k]):
+                        want = O.apply_final_weight(g, int(ref["states"][k]), ref["scores"][k])
+                        assert abs(float(h_sc[s, k]) - float(want)) <= SCORE_TOL, (c, s, k, "score")
+                    else:
+                        assert not np.isfinite(h_sc[s, k])
+                checked += 1
+    assert tb.tb_batch_status(batch) == 0
+    return checked
+
+
+@pytest.mark.parametrize("K,merge,prune", [(4, True, 8.0), (32, True, 8.0), (4, False, None), (32, False, 2.0)])
+def test_streaming_beam_with_churn(tb, K, merge, prune):
+    """The streaming workload's shape in small: 10 slots, chunks of 8 frames, 2 expansions per frame, streams of
+    20-70 frames that end in the middle of chunks, lists of 10-60 phrases compiled and bound as streams arrive."""
+    w = W.get_workload(5, B=10, T=70, T_lo=20, S=2, n_dur=0, n_phrases=60, n_phrases_lo=10)
+    n = run_streaming_beam(tb, w, K, n_chunks=24, merge=merge, prune_delta=prune, check_partial=True)
+    assert n >= 2 * w.B                                     # every slot saw several streams
+
+
+def test_streaming_beam_refuses_to_mix_with_the_batch_wide_tree(tb):
+    w = W.get_workload(5, B=3, T=16, T_lo=16, S=2, n_dur=0, n_phrases=10, n_phrases_lo=10)
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=4, max_tree_steps=64, arena_bytes=1 << 20)
+    dev = torch.device("cuda:0")
+    logits = torch.zeros((w.B, 8, 2, w.V + 1), dtype=torch.bfloat16, device=dev)
+    scores = torch.zeros((w.B, 4), device=dev)
+    states = torch.full((w.B, 4), -1, dtype=torch.int32, device=dev)
+    live = torch.zeros((w.B, 4), dtype=torch.uint8, device=dev)
+    par = torch.empty((w.B, 4), dtype=torch.int32, device=dev)
+    tok = torch.empty((w.B, 4), dtype=torch.int32, device=dev)
+    tb.tb_beam_reset_slots(batch)
+    tb.tb_beam_chunk(batch, logits, False, None, scores, states, live, par, tok)
+    with pytest.raises(tb.TbError):                        # a batch-wide step in the middle of a streaming session
+        tb.tb_beam_frames(batch, logits, False, scores, states, live, par, tok)
+    with pytest.raises(tb.TbError):                        # another beam width in the same session
+        tb.tb_beam_chunk(batch, logits, False, None, scores[:, :2].contiguous(), states[:, :2].contiguous(),
+                         live[:, :2].contiguous(), par[:, :2].contiguous(), tok[:, :2].contiguous())
+    with pytest.raises(tb.TbError):
+        tb.tb_beam_reset_slots(batch, [w.B])
+    tb.tb_beam_reset(batch)                                # ends the session
+    tb.tb_beam_frames(batch, logits, False, scores, states, live, par, tok)
+    with pytest.raises(tb.TbError):                        # and the other way round
+        tb.tb_beam_chunk(batch, logits, False, None, scores, states, live, par, tok)
+    torch.cuda.synchronize()
