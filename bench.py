@@ -251,6 +251,7 @@ def side_measurement(args):
         sched = W.ChurnSchedule(w)
         batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
         n_chunks, lat, binds, t_compile = 40 + 10 * args.steps, [], 0, 0.0
+        host_us = []
         bufs = []
         for c in range(n_chunks):
             chunk, lengths, bl = sched.next_chunk()
@@ -262,11 +263,16 @@ def side_measurement(args):
             bufs = (bufs + [dl])[-8:]
             torch.cuda.synchronize()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            th = time.perf_counter()
             a.record()
-            for sl, g in gs:
-                tb.tb_batch_bind_stream(batch, sl, g)
+            if args.single_binds:
+                for sl, g in gs:
+                    tb.tb_batch_bind_stream(batch, sl, g)
+            else:
+                tb.tb_batch_bind_streams(batch, [sl for sl, _ in gs], [g for _, g in gs])   # one copy, one launch
             tb.tb_stream_chunk(batch, dl, w.n_dur, dv)
             b.record()
+            host_us.append((time.perf_counter() - th) * 1e6)
             torch.cuda.synchronize()
             lat.append(a.elapsed_time(b))
             binds += len(bl)
@@ -274,9 +280,12 @@ def side_measurement(args):
         print(json.dumps({"metric": "streaming_tdt_chunk_latency_ms", "p50": float(np.percentile(lat, 50)),
                           "p99": float(np.percentile(lat, 99)), "unit": "ms", "higher_is_better": False, "n_gpus": 1,
                           "config": {"workload": w.name, "slots": w.B, "chunk_frames": w.chunk, "chunks": len(lat),
-                                     "binds_in_timed_region": True, "rebinds": binds - w.B},
+                                     "binds_in_timed_region": True, "rebinds": binds - w.B,
+                                     "binds": "one by one" if args.single_binds else "tb_batch_bind_streams (one copy + one launch per chunk)"},
                           "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
-                          "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds), "data": "synthetic"}))
+                          "host_issue_us_p50": float(np.percentile(np.array(host_us[10:]), 50)),
+                          "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds),
+                          "data": "synthetic"}))
 
     elif args.workload == 8:
         # Streaming beam search (Sec. 2.3; Sec. 3.4 uses beam 32): the streaming workload's churn without duration
@@ -315,8 +324,7 @@ def side_measurement(args):
                 torch.cuda.synchronize()
                 a, m0, m1, b = (torch.cuda.Event(enable_timing=True) for _ in range(4))
                 a.record()
-                for sl, g in gs:
-                    tb.tb_batch_bind_stream(batch, sl, g)
+                tb.tb_batch_bind_streams(batch, [sl for sl, _ in gs], [g for _, g in gs])
                 if new:
                     scores[idx] = float("-inf"); scores[idx, 0] = 0.0
                     states[idx] = -1; states[idx, 0] = 0
@@ -473,6 +481,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--streams", type=int, default=0, help="override B (profiling captures use a small case)")
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
+    ap.add_argument("--single-binds", action="store_true", help="workload 5: bind new streams one by one instead of in one call")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7, 8],
                     help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists, 7 model lifecycle sweep: side measurements")

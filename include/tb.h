@@ -245,10 +245,29 @@ void tb_batch_destroy(tb_batch *b);
  * on `stream`; the slot's offsets are published and its streaming state is reset (state =
  * root or -1, frame cursor 0, score 0) in stream order.  The previous graph's arena space is
  * reused by later binds.  g must have been compiled with the batch's vocab and class map.
+ * Ordering: the previous graph's arena block goes back to the free list when this call returns, and a later bind
+ * may overwrite it; a bind (this call, tb_batch_bind_streams, tb_batch_bind_model(s), tb_batch_register_model) must
+ * therefore be enqueued on the same stream as, or be ordered by an event after, every decode call that still reads
+ * the slot's previous graph.  Issuing all calls on one batch to one stream satisfies this.
  * Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG (vocab / class map mismatch),
  * TB_ERR_ARENA_FULL (nothing was changed), TB_ERR_CUDA.
  */
 int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *stream);
+
+/*
+ * tb_batch_bind_stream for n slots at once (Sec. 2.2 para. 4: between two chunks several streams end and start): the
+ * graphs are packed into one arena block and travel, with their slot records, in ONE host-to-device copy (graphs kept
+ * by a tb_cache are page-locked and go in one copy each, straight from where they are) followed by one small launch.  graphs[i] == NULL
+ * unbinds slots[i].  A slot may appear once.  Everything is checked before anything changes.  A group of more than
+ * 4 MB of graphs goes in parts of that size, and when the arena has no contiguous room for a part its slots are
+ * bound one by one (an error then leaves the earlier ones bound).
+ *   slots   host int32 [n];   graphs  host array of n graph pointers (each may be freed when the call returns)
+ * Ordering: as for tb_batch_bind_stream -- a bind must be enqueued on the stream (or ordered by an event) after the
+ * decode calls that still read the slots' previous graphs: their arena blocks go back to the free list at once and
+ * the next bind may overwrite them.
+ * Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG (a slot twice, vocab / class map mismatch), TB_ERR_ARENA_FULL, TB_ERR_CUDA.
+ */
+int tb_batch_bind_streams(tb_batch *b, int32_t n, const int32_t *slots, const tb_graph *const *graphs, void *stream);
 
 /*
  * Decoder-level registration (Sec. 2.2 para. 5: models known before a recognition session are registered with

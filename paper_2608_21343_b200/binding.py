@@ -71,6 +71,7 @@ _SIGS = {
     "tb_batch_create": (C.c_int, [_i32, _vp, _i32, _i32, _i32, C.c_size_t, C.c_int, C.POINTER(_vp)]),
     "tb_batch_destroy": (None, [_vp]),
     "tb_batch_bind_stream": (C.c_int, [_vp, _i32, _vp, _vp]),
+    "tb_batch_bind_streams": (C.c_int, [_vp, _i32, _vp, _vp, _vp]),
     "tb_batch_status": (C.c_int, [_vp, C.POINTER(_i32), _vp]),
     "tb_batch_set_flags": (C.c_int, [_vp, C.c_uint32]),
     "tb_batch_set_greedy_plan": (C.c_int, [_vp, _i32, _i32, _i32]),
@@ -354,6 +355,16 @@ TB_FLAG_GENERAL_KERNELS = 1
 TB_FLAG_ONE_BLOCK_PER_STREAM = 2
 TB_FLAG_TEST_WAIT_TIMEOUT = 4
 TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
+
+
+def tb_batch_bind_streams(batch: Batch, slots, graphs, stream=None):
+    """Bind graphs[i] (None: unbind) to slots[i], all in one copy and one launch."""
+    sl = _host(slots, np.int32)
+    assert len(sl) == len(graphs)
+    if len(sl) == 0:
+        return
+    arr = (_vp * len(graphs))(*[None if g is None else g.handle for g in graphs])
+    _check(_lib.tb_batch_bind_streams(batch.handle, len(sl), _hp(sl), arr, _stream(stream)), "tb_batch_bind_streams")
 
 
 def tb_batch_set_flags(batch: Batch, flags: int):

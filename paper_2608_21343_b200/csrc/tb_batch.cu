@@ -13,6 +13,7 @@ namespace {
 
 constexpr size_t kArenaAlign = 256;
 constexpr int kStagingRing = 4;
+constexpr size_t kGroupBytes = 4u << 20;   // graphs a group bind packs into one copy (larger groups go in parts)
 
 struct DeviceGuard {  // makes the batch's device current for the duration of a call
   int prev = -1;
@@ -61,6 +62,7 @@ struct Staging {
   cudaEvent_t done = nullptr;
   bool pending = false;
   tb_graph* held = nullptr;   // a pinned graph whose blob the pending copy reads: released once the copy is done
+  std::vector<tb_graph*> held_more;   // the same for a group bind (tb_batch_bind_streams)
 };
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -137,6 +139,7 @@ static void destroy_batch(tb_batch* b) {
   cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs); cudaFree(b->d_slot_pos);
   for (auto& s : b->staging) {
     if (s.held) tb_graph_free(s.held);
+    for (tb_graph* h : s.held_more) tb_graph_free(h);
     if (s.host) cudaFreeHost(s.host);
     if (s.done) cudaEventDestroy(s.done);
   }
@@ -207,6 +210,20 @@ extern "C" void tb_batch_destroy(tb_batch* b) {
   destroy_batch(b);
 }
 
+// The slot record of graph g when its blob sits at byte offset `off` of the arena.
+static void fill_record(const tb_graph* g, size_t off, TbSlotRec* rec_out) {
+  TbSlotRec& rec = *rec_out;
+  std::memset(&rec, 0, sizeof rec);
+  rec.blob_off = static_cast<int64_t>(off);
+  rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
+  rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
+  rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
+  rec.off_final = g->off_final;
+  rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
+  rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
+  rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
+}
+
 // Copies a graph's blob into a fresh arena block (through the pinned staging ring, on `stream`) and fills the
 // slot record that points at it.
 static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, size_t* off_out, size_t* bytes_out,
@@ -221,6 +238,8 @@ static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, siz
   bool ok = true;
   if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
   if (s.held) { tb_graph_free(s.held); s.held = nullptr; }
+  for (tb_graph* h : s.held_more) tb_graph_free(h);
+  s.held_more.clear();
   if (ok && g->pinned) {
     // the blob's pages are locked: the copy engine reads it in place; the graph is held until the copy is done
     ok = cudaMemcpyAsync(b->arena + off, g->blob.data(), g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
@@ -240,16 +259,7 @@ static int upload_graph(tb_batch* b, const tb_graph* g, cudaStream_t stream, siz
     s.pending = ok;
   }
   if (!ok) { cudaGetLastError(); b->alloc.release(off, bytes); return TB_ERR_CUDA; }
-  TbSlotRec& rec = *rec_out;
-  std::memset(&rec, 0, sizeof rec);
-  rec.blob_off = static_cast<int64_t>(off);
-  rec.off_arc_begin = g->off_arc_begin; rec.off_fail = g->off_fail; rec.off_bw = g->off_bw;
-  rec.off_arc_cls = g->off_arc_cls; rec.off_arc_w = g->off_arc_w; rec.off_arc_dst = g->off_arc_dst;
-  rec.off_strec = g->off_strec; rec.off_tokent = g->off_tokent;
-  rec.off_final = g->off_final;
-  rec.n_tokent = g->n_tokent; rec.blob_bytes = static_cast<int32_t>(g->blob.size());
-  rec.off_rsrec = g->off_rsrec; rec.off_rsent = g->off_rsent; rec.n_rsent = g->n_rsent; rec.d_max = g->d_max;
-  rec.n_states = g->n_states; rec.n_arcs = g->n_arcs; rec.max_depth = g->max_depth; rec.lambda = g->lambda;
+  fill_record(g, off, rec_out);
   *off_out = off; *bytes_out = bytes;
   return TB_OK;
 }
@@ -293,6 +303,109 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
   return TB_OK;
 }
 
+// Several slots at once (the streams that start between two chunks): the graphs go into ONE arena block, packed
+// next to each other in one pinned staging block together with their slot records, so that the whole update is one
+// host-to-device copy and one small launch, whatever the number of streams.
+extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slots, const tb_graph* const* graphs,
+                                     void* stream_) {
+  if (!b || n < 0 || (n > 0 && (!slots || !graphs))) return TB_ERR_INVALID_ARG;
+  if (n == 0) return TB_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // everything is checked before anything changes
+  std::vector<uint8_t> seen(static_cast<size_t>(b->n_slots), 0);
+  size_t total = 0;
+  int32_t first_part = n;                                             // a group beyond a few MB goes in several parts
+  for (int32_t i = 0; i < n; ++i) {
+    if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
+    if (seen[slots[i]]) return TB_ERR_INVALID_ARG;
+    seen[slots[i]] = 1;
+    const tb_graph* g = graphs[i];
+    if (g && (g->vocab != b->vocab || g->class_map_hash != b->class_map_hash)) return TB_ERR_INVALID_ARG;
+    if (g && first_part == n) {
+      if (total > 0 && total + g->blob.size() > kGroupBytes) first_part = i;
+      else total += round_up(g->blob.size(), kArenaAlign);
+    }
+  }
+  if (first_part < n) {
+    // (the parts' staging blocks stay small; an error in a later part leaves the earlier parts bound)
+    int rc = tb_batch_bind_streams(b, first_part, slots, graphs, stream_);
+    if (rc == TB_OK) rc = tb_batch_bind_streams(b, n - first_part, slots + first_part, graphs + first_part, stream_);
+    return rc;
+  }
+  const size_t tail_off = total;                                      // records, then slot indices, behind the graphs
+  const size_t tail = round_up(static_cast<size_t>(n) * (sizeof(TbSlotRec) + sizeof(int32_t)), kArenaAlign);
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  size_t base = 0;
+  if (!b->alloc.alloc(total + tail, &base)) {
+    // no contiguous room for the group (a fragmented or nearly full arena): one by one, each in the first hole that fits
+    for (int32_t i = 0; i < n; ++i) {
+      const int rc = tb_batch_bind_stream(b, slots[i], graphs[i], stream_);
+      if (rc != TB_OK) return rc;
+    }
+    return TB_OK;
+  }
+  Staging& s = b->staging[b->next_staging];
+  b->next_staging = (b->next_staging + 1) % kStagingRing;
+  bool ok = true;
+  if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
+  if (s.held) { tb_graph_free(s.held); s.held = nullptr; }
+  for (tb_graph* h : s.held_more) tb_graph_free(h);
+  s.held_more.clear();
+  // graphs whose image is page-locked (those kept by a cache) are copied from where they are; only
+  // the others pass through the staging block, which also carries the records
+  bool any_pinned = false;
+  for (int32_t i = 0; i < n; ++i) any_pinned = any_pinned || (graphs[i] && graphs[i]->pinned);
+  if (ok && s.cap < total + tail) {
+    if (s.host) cudaFreeHost(s.host);
+    s.host = nullptr; s.cap = 0;
+    const size_t want = round_up((total + tail) * 2, 1 << 20);
+    ok = cudaMallocHost(&s.host, want) == cudaSuccess;
+    if (ok) s.cap = want;
+  }
+  if (!ok) { cudaGetLastError(); b->alloc.release(base, total + tail); return TB_ERR_CUDA; }
+  TbSlotRec* recs = reinterpret_cast<TbSlotRec*>(s.host + tail_off);
+  int32_t* slot_of = reinterpret_cast<int32_t*>(s.host + tail_off + static_cast<size_t>(n) * sizeof(TbSlotRec));
+  std::vector<std::pair<size_t, size_t>> blocks(static_cast<size_t>(n), {0, 0});
+  size_t at = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const tb_graph* g = graphs[i];
+    slot_of[i] = slots[i];
+    if (!g) { std::memset(&recs[i], 0, sizeof(TbSlotRec)); continue; }
+    if (g->pinned) {
+      ok = ok && cudaMemcpyAsync(b->arena + base + at, g->blob.data(), g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+      if (ok) { tb_graph* h = const_cast<tb_graph*>(g); h->refs.fetch_add(1); s.held_more.push_back(h); }
+    } else {
+      std::memcpy(s.host + at, g->blob.data(), g->blob.size());
+      if (any_pinned)   // (a mixed group: every staged graph is its own copy)
+        ok = ok && cudaMemcpyAsync(b->arena + base + at, s.host + at, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    }
+    fill_record(g, base + at, &recs[i]);
+    blocks[i] = {base + at, round_up(g->blob.size(), kArenaAlign)};
+    at += blocks[i].second;
+  }
+  if (any_pinned) ok = ok && cudaMemcpyAsync(b->arena + base + tail_off, s.host + tail_off, tail, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  else ok = ok && cudaMemcpyAsync(b->arena + base, s.host, total + tail, cudaMemcpyHostToDevice, stream) == cudaSuccess;   // graphs and records in one copy
+  ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;
+  s.pending = ok;
+  int rc = ok ? tb_launch_publish_slots(b->d_slots, b->d_sstate, n, reinterpret_cast<const TbSlotRec*>(b->arena + base + tail_off),
+                                        reinterpret_cast<const int32_t*>(b->arena + base + tail_off + static_cast<size_t>(n) * sizeof(TbSlotRec)),
+                                        stream)
+              : TB_ERR_CUDA;
+  if (rc != TB_OK) { cudaGetLastError(); b->alloc.release(base, total + tail); return rc; }
+  // the records' part of the block is free again (whatever reuses it is enqueued after the launch that reads it)
+  b->alloc.release(base + tail_off, tail);
+  for (int32_t i = 0; i < n; ++i) {
+    const tb_graph* g = graphs[i];
+    release_slot(b, slots[i]);
+    b->slot_block[slots[i]] = blocks[i];
+    b->slot_n_states[slots[i]] = g ? g->n_states : 0;
+    b->slot_cache_bytes[slots[i]] = !g ? 0 : cache_bytes_of(g);
+    b->slot_resolved[slots[i]] = (!g || g->n_rsent >= 0) ? 1 : 0;
+  }
+  return TB_OK;
+}
+
 extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* out_model_id, void* stream_) {
   if (!b || !g || !out_model_id) return TB_ERR_INVALID_ARG;
   *out_model_id = -1;
@@ -320,6 +433,9 @@ extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* 
     TbSlotRec* bigger = nullptr;
     bool ok = cudaMalloc(&bigger, sizeof(TbSlotRec) * cap) == cudaSuccess;
     ok = ok && cudaMemset(bigger, 0, sizeof(TbSlotRec) * cap) == cudaSuccess;
+    // records published on `stream` by earlier registrations must have landed before the table is copied (the
+    // caller's stream does not synchronise with the legacy stream the copy below runs on)
+    ok = ok && cudaStreamSynchronize(static_cast<cudaStream_t>(stream_)) == cudaSuccess;
     if (ok && b->model_recs_cap)
       ok = cudaMemcpy(bigger, b->d_model_recs, sizeof(TbSlotRec) * b->model_recs_cap, cudaMemcpyDeviceToDevice) == cudaSuccess;
     if (!ok) { cudaGetLastError(); cudaFree(bigger); b->alloc.release(m.off, m.bytes); return TB_ERR_OOM; }

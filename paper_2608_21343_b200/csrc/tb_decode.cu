@@ -811,6 +811,18 @@ int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, 
 }
 
 namespace {
+// Many slots published at once: the records and their slot indices were copied to the device with the graphs.
+__global__ void k_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n, const TbSlotRec* recs, const int32_t* slot_of) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const TbSlotRec rec = recs[i];
+  slots[slot_of[i]] = rec;
+  TbSlotState st;
+  st.state = rec.n_states > 0 ? 0 : -1; st.t = 0; st.k = 0; st.score = 0.0f; st.n_emitted = 0;
+  st.chunk_base = 0; st.pad0 = 0; st.pad1 = 0;
+  sstate[slot_of[i]] = st;
+}
+
 __global__ void k_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, SlotList sl, int32_t K,
                                       float* scores, const int32_t* states, int32_t* status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -872,5 +884,12 @@ int tb_launch_final_weights_slots(const TbSlotRec* slots, const unsigned char* a
   for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = i < n ? slot_list[i] : 0;
   const int total = n * K;
   k_final_weights_slots<<<(total + 127) / 128, 128, 0, stream>>>(slots, arena, n, sl, K, scores, states, status);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n, const TbSlotRec* recs, const int32_t* slot_of,
+                            cudaStream_t stream) {
+  if (n < 1) return TB_ERR_INVALID_ARG;
+  k_publish_slots<<<(n + 63) / 64, 64, 0, stream>>>(slots, sstate, n, recs, slot_of);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }

@@ -88,6 +88,9 @@ int tb_launch_bind_models(TbSlotRec* slots, TbSlotState* sstate, const TbSlotRec
                           const int32_t* slot_of, const int32_t* model_of, cudaStream_t stream);
 int tb_launch_final_weights(const TbSlotRec* slots, const unsigned char* arena, int32_t B, int32_t K, float* scores,
                             const int32_t* states, int32_t* status, cudaStream_t stream);
+// n slots at once: recs / slot_of are device arrays (uploaded together with the graphs they describe).
+int tb_launch_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n, const TbSlotRec* recs, const int32_t* slot_of,
+                            cudaStream_t stream);
 int tb_launch_publish_slot(TbSlotRec* slots, TbSlotState* sstate, int32_t slot, const TbSlotRec& rec,
                            cudaStream_t stream);
 

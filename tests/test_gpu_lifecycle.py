@@ -231,3 +231,51 @@ def test_binding_many_registered_models_at_once(tb):
     with pytest.raises(tb.TbError):
         tb.tb_batch_unregister_model(batch, ids[3])                               # slot 299 still uses it
     tb.tb_batch_bind_models(batch, [], [])
+
+
+def test_binding_many_streams_at_once(tb):
+    """tb_batch_bind_streams: several slots get new lists (or lose theirs) in one copy and one launch; the result is
+    what the same binds one by one give, other slots are untouched, and a small arena falls back to single binds."""
+    w = W.get_workload(2, B=8, T=100, n_phrases=40, n_plants=6)
+    data = W.batch_inputs(w)
+    logits = to_device(data["logits"])
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=4 << 20)
+    graphs = [tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class) for p in data["phrases"]]
+    tb.tb_batch_bind_streams(batch, list(range(w.B)), graphs)
+    out = to_host(tb.tb_greedy_decode(batch, logits))
+    for i in range(w.B):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]), "all at once")
+    # a second round: three slots swap lists, one is unbound, the rest stay
+    other = [W.stream_phrases(w, 50 + i) for i in range(3)]
+    tb.tb_batch_bind_streams(batch, [6, 1, 4, 2], [tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class) for p in other] + [None])
+    lists = list(data["phrases"])
+    lists[6], lists[1], lists[4], lists[2] = other[0], other[1], other[2], None
+    out = to_host(tb.tb_greedy_decode(batch, logits))
+    for i in range(w.B):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, lists[i]), data["logits"][i]), "second round")
+    assert out["states"][2] == -1
+    # streaming state is reset by the bind, as with a single bind
+    valid = torch.full((w.B,), w.T, dtype=torch.int32, device="cuda:0")
+    tb.tb_stream_chunk(batch, logits[:, :8], 0, valid)
+    tb.tb_batch_bind_streams(batch, [0, 3], [graphs[0], graphs[3]])
+    ch = to_host(tb.tb_stream_chunk(batch, logits[:, :8], 0, valid))
+    assert ch["cursors"][0] == 8 and ch["cursors"][3] == 8 and ch["cursors"][1] == 16
+    # errors: checked before anything changes
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_batch_bind_streams(batch, [0, 0], [graphs[0], graphs[1]])
+    assert e.value.code == tb.TB_ERR_INVALID_ARG
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_batch_bind_streams(batch, [0, w.B], [graphs[0], graphs[1]])
+    assert e.value.code == tb.TB_ERR_BAD_SLOT
+    # many rounds into a small arena: space is handed back, and when no contiguous block fits the group the binds
+    # still succeed one by one
+    small = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=360 << 10)
+    for r in range(12):
+        sl = [(r + j) % w.B for j in range(4)]
+        tb.tb_batch_bind_streams(small, sl, [graphs[(r + 2 * j) % w.B] for j in range(4)])
+    tb.tb_batch_bind_streams(small, list(range(w.B)), [None] * w.B)
+    tb.tb_batch_bind_streams(small, [0, 1, 2, 3, 4], graphs[:5])
+    out = to_host(tb.tb_greedy_decode(small, logits))
+    for i in range(5):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]), "small arena")
+    assert tb.tb_batch_status(batch) == 0 and tb.tb_batch_status(small) == 0
