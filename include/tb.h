@@ -64,6 +64,10 @@ extern "C" {
 /* tb_batch_set_flags */
 #define TB_FLAG_GENERAL_KERNELS 1       /* always use the general decode kernel (any layout), never a pipelined one */
 #define TB_FLAG_ONE_BLOCK_PER_STREAM 2  /* pipelined greedy decode: never the segmented kernel, one block per stream */
+#define TB_FLAG_LOG_SOFTMAX 8           /* tb_greedy_decode and tb_stream_chunk (RNNT rows) normalise every visited row first:
+                                           value(v) = fl(fl(x_v - L) + fl(lambda * bonus)), L = m + log(sum_v exp(x_v - m)) over the
+                                           row's vocab+1 entries, computed in float inside the selection kernel (Sec. 2.2 para. 3:
+                                           one fused scoring operation); runs on the general kernel */
 #define TB_FLAG_TEST_WAIT_TIMEOUT 4     /* self-test of the kernels' bounded waits: tb_greedy_decode (segmented kernel) withholds one
                                            frame's summaries and waits only briefly, so the wait runs out: the call returns,
                                            TB_STATUS_WAIT_TIMEOUT is set, the outputs of that call are undefined */

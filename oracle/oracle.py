@@ -84,6 +84,13 @@ def lib():
         _lib.orc_greedy_rnnt.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                          C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        _lib.orc_row_lse.restype = C.c_double
+        _lib.orc_row_lse.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int32]
+        _lib.orc_greedy_rnnt_lsm.restype = C.c_int64
+        _lib.orc_greedy_rnnt_lsm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_void_p,
+                                             C.POINTER(C.c_double), C.POINTER(C.c_int32), C.POINTER(C.c_int64),
+                                             C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         _lib.orc_stream_chunk.restype = C.c_int64
         _lib.orc_stream_chunk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_int32, C.c_int32,
                                           C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
@@ -243,6 +250,40 @@ def greedy_rnnt(graph, logits: np.ndarray, length=None):
                               T, S, V1 - 1, _ptr(st), length, _ptr(toks), _ptr(frs),
                               C.byref(score), C.byref(state))
     return dict(tokens=toks[:n].copy(), frames=frs[:n].copy(), score=np.float32(score.value), state=state.value)
+
+
+def row_lse(row: np.ndarray) -> float:
+    """log sum exp of one row [V+1] (float32 or bf16 bits), in double."""
+    row = np.ascontiguousarray(row)
+    return float(lib().orc_row_lse(_ptr(row), _dtype_code(row), 0, 1, row.shape[0] - 1))
+
+
+def greedy_rnnt_lsm(graph, logits: np.ndarray, length=None, follow=None, eps: float = 0.0):
+    """Greedy RNNT on log-softmax scores (double).  follow = (tokens, frames) of another decoder: its choices are
+    taken wherever they are within eps of this decoder's (counted in ``followed``); a larger difference stops the
+    decode (``first_mismatch`` = index of the visited row, else -1).
+
+    Returns dict(tokens, frames, score (float64), state, followed, first_mismatch, rows)."""
+    T, S, V1 = logits.shape
+    length = T if length is None else int(length)
+    toks = np.zeros(T * S, dtype=np.int32)
+    frs = np.zeros(T * S, dtype=np.int32)
+    score = C.c_double()
+    state = C.c_int32()
+    nf, mm, rows = C.c_int64(), C.c_int64(), C.c_int64()
+    st = _strides3(logits)
+    if follow is None:
+        ft = ff = None
+        n_follow = -1
+    else:
+        ft = np.ascontiguousarray(follow[0], dtype=np.int32)
+        ff = np.ascontiguousarray(follow[1], dtype=np.int32)
+        n_follow = len(ft)
+    n = lib().orc_greedy_rnnt_lsm(graph.handle if graph is not None else None, _ptr(logits), _dtype_code(logits), T, S,
+                                  V1 - 1, _ptr(st), length, _ptr(ft), _ptr(ff), n_follow, float(eps), _ptr(toks), _ptr(frs),
+                                  C.byref(score), C.byref(state), C.byref(nf), C.byref(mm), C.byref(rows))
+    return dict(tokens=toks[:n].copy(), frames=frs[:n].copy(), score=score.value, state=state.value,
+                followed=nf.value, first_mismatch=mm.value, rows=rows.value)
 
 
 def stream_chunk(graph, logits: np.ndarray, n_dur: int, t0: int, valid_frames: int, st: StreamState):

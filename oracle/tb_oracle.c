@@ -383,6 +383,90 @@ int64_t orc_greedy_rnnt(const orc_graph *g, const void *logits, int dtype, int32
 }
 
 /* ------------------------------------------------------------------------------------ */
+/* Greedy RNNT on normalised scores: log-softmax fused into the selection                  */
+/* (Sec. 2.2 para. 3 speaks of one fused scoring operation; READING: the paper does not say  */
+/* whether the joint output is normalised before the bonus is added -- this variant does it). */
+/* ------------------------------------------------------------------------------------ */
+
+/* log sum exp of the V+1 entries of one row, in double: L = m + log(sum_v exp(x_v - m)), m = max_v x_v. */
+double orc_row_lse(const void *logits, int dtype, int64_t row, int64_t stride_v, int32_t V) {
+  double m = -INFINITY;
+  for (int32_t v = 0; v <= V; ++v) {
+    double x = (double)logit_at(logits, dtype, row + v * stride_v);
+    if (x > m) m = x;
+  }
+  if (m == -INFINITY) return -INFINITY;
+  double sum = 0.0;
+  for (int32_t v = 0; v <= V; ++v) sum += exp((double)logit_at(logits, dtype, row + v * stride_v) - m);
+  return m + log(sum);
+}
+
+/*
+ * As orc_greedy_rnnt, on val(v) = (x_v - L(row)) + lambda * bonus(s, v), everything after the float bonus
+ * term in double: the bonus term is the float product fl(lambda * bonus) of the un-normalised decode, the
+ * normalised logit x_v - L and the sum are double, the score is a double sum.  L is the same for every entry of
+ * a row, so in exact arithmetic the selected tokens are those of the un-normalised decode and the score is lower
+ * by the sum of L over the visited rows.
+ *
+ * follow_tokens / follow_frames (n_follow >= 0): another decoder's output to be checked against this one.  At
+ * every visited row the other decoder's action there (its next token if that token's frame is the current frame,
+ * else blank) is compared with this decoder's choice; where they differ and the two values are closer than eps
+ * the other decoder's action is taken (and counted in *n_followed), so that one near-tie does not make the rest
+ * of the stream incomparable; where they differ by eps or more the decode stops and *first_mismatch receives the
+ * index of the visited row (else -1).  n_follow < 0: a free decode.
+ */
+int64_t orc_greedy_rnnt_lsm(const orc_graph *g, const void *logits, int dtype, int32_t T, int32_t S, int32_t V,
+                            const int64_t *strides, int32_t len, const int32_t *follow_tokens,
+                            const int32_t *follow_frames, int64_t n_follow, double eps, int32_t *out_tokens,
+                            int32_t *out_frames, double *out_score, int32_t *out_state, int64_t *n_followed,
+                            int64_t *first_mismatch, int64_t *rows_visited) {
+  int32_t s = g ? 0 : -1, t = 0, k = 0;
+  double score = 0.0;
+  int64_t n = 0, rows = 0, followed = 0;
+  if (first_mismatch) *first_mismatch = -1;
+  if (len > T) len = T;
+  while (t < len) {
+    int64_t row = (int64_t)t * strides[0] + (int64_t)k * strides[1];
+    double L = orc_row_lse(logits, dtype, row, strides[2], V);
+    int32_t best = -1, best_next = -1;
+    double bv = 0.0;
+    for (int32_t v = 0; v <= V; ++v) {
+      float x = logit_at(logits, dtype, row + v * strides[2]);
+      int32_t nv;
+      float lam_b = boosted(g, s, v, V, 0.0f, &nv);          /* fl(0 + fl(lambda * bonus)): the float bonus term alone */
+      double val = ((double)x - L) + (double)lam_b;
+      if (best < 0 || val > bv) { best = v; bv = val; best_next = nv; }
+    }
+    int32_t tok = best, nx = best_next;
+    double val = bv;
+    if (n_follow >= 0) {
+      int32_t want = (n < n_follow && follow_frames[n] == t) ? follow_tokens[n] : V;
+      if (want < 0 || want > V) want = V;
+      if (want != best) {
+        float xw = logit_at(logits, dtype, row + want * strides[2]);
+        int32_t nw;
+        float lam_w = boosted(g, s, want, V, 0.0f, &nw);
+        double vw = ((double)xw - L) + (double)lam_w;
+        if (bv - vw < eps) { tok = want; nx = nw; val = vw; followed++; }
+        else { if (first_mismatch) *first_mismatch = rows; break; }
+      }
+    }
+    rows++;
+    score += val;
+    if (tok == V) { t++; k = 0; }
+    else {
+      out_tokens[n] = tok; out_frames[n] = t; n++;
+      s = nx; k++;
+      if (k == S) { t++; k = 0; }
+    }
+  }
+  *out_score = score; *out_state = s;
+  if (n_followed) *n_followed = followed;
+  if (rows_visited) *rows_visited = rows;
+  return n;
+}
+
+/* ------------------------------------------------------------------------------------ */
 /* Streaming greedy, RNNT or TDT, one slot, one chunk (Sec. 2.3: state kept across chunks) */
 /* ------------------------------------------------------------------------------------ */
 

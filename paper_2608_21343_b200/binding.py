@@ -354,6 +354,7 @@ TB_STATUS_WALK_TOO_DEEP, TB_STATUS_BAD_STATE, TB_STATUS_STEP_LIMIT, TB_STATUS_WA
 TB_FLAG_GENERAL_KERNELS = 1
 TB_FLAG_ONE_BLOCK_PER_STREAM = 2
 TB_FLAG_TEST_WAIT_TIMEOUT = 4
+TB_FLAG_LOG_SOFTMAX = 8
 TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
 
 

@@ -559,7 +559,8 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (!(b->flags & TB_FLAG_GENERAL_KERNELS)) {
+  p.normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;   // (only the general kernel normalises)
+  if (!(b->flags & (TB_FLAG_GENERAL_KERNELS | TB_FLAG_LOG_SOFTMAX))) {
     int32_t max_cache = 0, max_states = 0, all_resolved = 1;
     for (int32_t i = 0; i < B; ++i) {
       max_cache = b->slot_cache_bytes[i] > max_cache ? b->slot_cache_bytes[i] : max_cache;
@@ -658,7 +659,7 @@ extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* 
 }
 
 extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {
-  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT))) return TB_ERR_INVALID_ARG;
+  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT | TB_FLAG_LOG_SOFTMAX))) return TB_ERR_INVALID_ARG;
   b->flags = flags;
   return TB_OK;
 }
@@ -672,6 +673,8 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
   if (rc != TB_OK) return rc;
   if (!valid_frames || !out_tokens || !out_frames || !out_counts || !out_scores || !out_states) return TB_ERR_INVALID_ARG;
   p.lengths = valid_frames; p.persistent = 1;
+  p.normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;
+  if (p.normalize && n_dur != 0) return TB_ERR_INVALID_ARG;   // normalisation is defined for the token logits of an RNNT row
   p.out_tokens = out_tokens; p.out_frames = out_frames; p.out_durs = out_durs; p.out_counts = out_counts;
   p.out_scores = out_scores; p.out_states = out_states; p.out_cursors = out_cursors;
   DeviceGuard guard(b->device);

@@ -96,6 +96,7 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
   float* bvec = reinterpret_cast<float*>(dyn);
   int32_t* nvec = reinterpret_cast<int32_t*>(dyn + sizeof(float) * p.C);
   __shared__ StepSmem sm;
+  __shared__ float fred[kThreads / 32];
 
   const int b = blockIdx.x;
   const TbSlotRec rec = p.slots[b];
@@ -137,9 +138,35 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
       built_for = s;
     }
     const LT* row = base + static_cast<int64_t>(t - t0) * p.st + static_cast<int64_t>(k) * p.ss;
+    float lse = 0.0f;
+    if (p.normalize) {
+      // log-softmax fused into the selection: L = m + log(sum_v exp(x_v - m)) over the row's V+1 entries, in
+      // float with a fixed order of additions (per thread by index, then lanes, then warps), so that a launch
+      // repeats bit for bit; every entry becomes x_v - L before its bonus is added
+      float m = -INFINITY;
+      for (int v = threadIdx.x; v <= V; v += kThreads) m = fmaxf(m, LogitLoad<LT>::at(row + static_cast<int64_t>(v) * p.sv));
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+      if ((threadIdx.x & 31) == 0) fred[threadIdx.x >> 5] = m;
+      __syncthreads();
+      m = fred[0];
+      for (int w2 = 1; w2 < kThreads / 32; ++w2) m = fmaxf(m, fred[w2]);
+      __syncthreads();
+      float sum = 0.0f;
+      for (int v = threadIdx.x; v <= V; v += kThreads) sum = __fadd_rn(sum, expf(__fsub_rn(LogitLoad<LT>::at(row + static_cast<int64_t>(v) * p.sv), m)));
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, off));
+      if ((threadIdx.x & 31) == 0) fred[threadIdx.x >> 5] = sum;
+      __syncthreads();
+      sum = fred[0];
+      for (int w2 = 1; w2 < kThreads / 32; ++w2) sum = __fadd_rn(sum, fred[w2]);
+      __syncthreads();
+      lse = m == -INFINITY ? 0.0f : __fadd_rn(m, logf(sum));
+    }
     ValId best{-INFINITY, INT32_MAX};
     for (int v = threadIdx.x; v <= V; v += kThreads) {
       float x = LogitLoad<LT>::at(row + static_cast<int64_t>(v) * p.sv);
+      if (p.normalize) x = __fsub_rn(x, lse);
       float val = x;
       if (bound && v < V) {
         if (use_tv) {
