@@ -126,17 +126,24 @@ __device__ __forceinline__ void fetch_row(unsigned char* buf, const unsigned cha
   const int off = static_cast<int>(reinterpret_cast<uintptr_t>(rowp) & 15);
   const unsigned char* a0 = rowp - off;
   const int nchunks = (off + row_bytes + 15) >> 4;
-  const bool guard = a0 < lo || a0 + 16 * nchunks > hi;
-  const uint32_t buf_a = smem_u32(buf);
-  for (int c = lane; c < nchunks; c += 32) {
-    const unsigned char* a = a0 + 16 * c;
-    if (!guard || (a >= lo && a + 16 <= hi)) {
-      cp_async16(buf_a + 16u * c, a);
-    } else {
-      for (int e = 0; e < 8; ++e) {
-        uint16_t x = 0xFF80u;
-        if (a + 2 * e >= lo && a + 2 * e + 2 <= hi) x = *reinterpret_cast<const uint16_t*>(a + 2 * e);
-        *reinterpret_cast<uint16_t*>(buf + 16 * c + 2 * e) = x;
+  const uint32_t buf_a = smem_u32(buf) + 16u * lane;
+  const unsigned char* a = a0 + 16 * lane;
+  if (a0 >= lo && a0 + 16 * nchunks <= hi) {
+    // (a row of up to 2048 elements and its lead of up to 14 bytes are at most 257 pieces: nine per lane)
+#pragma unroll
+    for (int j = 0; j < 9; ++j)
+      if (lane + 32 * j < nchunks) cp_async16(buf_a + 512u * j, a + 512 * j);
+  } else {
+    for (int c = lane; c < nchunks; c += 32) {
+      const unsigned char* ac = a0 + 16 * c;
+      if (ac >= lo && ac + 16 <= hi) {
+        cp_async16(smem_u32(buf) + 16u * c, ac);
+      } else {
+        for (int e = 0; e < 8; ++e) {
+          uint16_t x = 0xFF80u;
+          if (ac + 2 * e >= lo && ac + 2 * e + 2 <= hi) x = *reinterpret_cast<const uint16_t*>(ac + 2 * e);
+          *reinterpret_cast<uint16_t*>(buf + 16 * c + 2 * e) = x;
+        }
       }
     }
   }
