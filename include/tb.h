@@ -68,6 +68,8 @@ extern "C" {
                                            value(v) = fl(fl(x_v - L) + fl(lambda * bonus)), L = m + log(sum_v exp(x_v - m)) over the
                                            row's vocab+1 entries, computed in float inside the selection kernel (Sec. 2.2 para. 3:
                                            one fused scoring operation); runs on the general kernel */
+#define TB_FLAG_BEAM_WHOLE_ROWS 16      /* tb_beam_frames / tb_beam_chunk: no pre-pass that reduces every row to its best tokens; every
+                                           step looks at all vocab+1 entries of its row (identical results) */
 #define TB_FLAG_TEST_WAIT_TIMEOUT 4     /* self-test of the kernels' bounded waits: tb_greedy_decode (segmented kernel) withholds one
                                            frame's summaries and waits only briefly, so the wait runs out: the call returns,
                                            TB_STATUS_WAIT_TIMEOUT is set, the outputs of that call are undefined */

@@ -355,6 +355,7 @@ TB_FLAG_GENERAL_KERNELS = 1
 TB_FLAG_ONE_BLOCK_PER_STREAM = 2
 TB_FLAG_TEST_WAIT_TIMEOUT = 4
 TB_FLAG_LOG_SOFTMAX = 8
+TB_FLAG_BEAM_WHOLE_ROWS = 16
 TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
 
 

@@ -97,6 +97,8 @@ struct tb_batch {
   int64_t beam_steps = 0;                     // steps since tb_beam_reset (selects the ping-pong half)
   float beam_prune_delta = -1.0f;             // >= 0: prune at frame starts (tb_batch_set_beam_prune)
   int32_t tree_steps = 0, tree_B = 0, tree_K = 0;
+  TbTopEnt* d_top = nullptr;                  // rows reduced ahead of a multi-step beam launch (grown on demand)
+  size_t d_top_bytes = 0;
   int32_t* d_slot_pos = nullptr;              // [n_slots] steps every slot has taken since its last reset (streaming beam decoding)
   int32_t chunk_K = 0;                        // beam width of the streaming calls since the last reset of all slots (0: none yet)
   ArenaAllocator alloc;
@@ -136,7 +138,7 @@ static void destroy_batch(tb_batch* b) {
   if (!b) return;
   cudaDeviceSynchronize();
   cudaFree(b->arena); cudaFree(b->d_slots); cudaFree(b->d_sstate); cudaFree(b->d_cls);
-  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs); cudaFree(b->d_slot_pos);
+  cudaFree(b->d_status); cudaFree(b->d_tree); cudaFree(b->seg_scratch); cudaFree(b->sg_scratch); cudaFree(b->d_hyp_hash); cudaFree(b->d_hyp_len); cudaFree(b->d_model_recs); cudaFree(b->d_slot_pos); cudaFree(b->d_top);
   for (auto& s : b->staging) {
     if (s.held) tb_graph_free(s.held);
     for (tb_graph* h : s.held_more) tb_graph_free(h);
@@ -659,7 +661,8 @@ extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* 
 }
 
 extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {
-  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT | TB_FLAG_LOG_SOFTMAX))) return TB_ERR_INVALID_ARG;
+  if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT | TB_FLAG_LOG_SOFTMAX |
+                                              TB_FLAG_BEAM_WHOLE_ROWS))) return TB_ERR_INVALID_ARG;
   b->flags = flags;
   return TB_OK;
 }
@@ -680,6 +683,32 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
+}
+
+// The beam pre-pass for a launch that covers T * E rows per stream: reduces every row to its few best root-boosted
+// tokens (tb_launch_beam_topm) into memory of the batch and points the step parameters at the result.  Skipped (the
+// steps then look at whole rows) when the batch asks for it, when the memory would have to grow while the stream is
+// being captured, or when it cannot be had.
+static void beam_prepass(tb_batch* b, TbBeamParams* p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
+                         const int32_t* n_frames, cudaStream_t stream) {
+  p->top_base = nullptr; p->top_row = nullptr; p->top_m = 0;
+  if (b->flags & (TB_FLAG_GENERAL_KERNELS | TB_FLAG_BEAM_WHOLE_ROWS)) return;
+  if (2 * (b->vocab + 1) > (1 << TB_RS_TOK_BITS) || b->vocab > 0xFFFE) return;   // (the steps' token view has the same limit)
+  const int32_t M = 2 * p->K + 8;
+  const size_t want = static_cast<size_t>(p->B) * T * E * (M + 1) * sizeof(TbTopEnt);
+  if (want > b->d_top_bytes) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return; }
+    if (cap != cudaStreamCaptureStatusNone || want > (static_cast<size_t>(2) << 30)) return;
+    cudaFree(b->d_top);
+    b->d_top = nullptr; b->d_top_bytes = 0;
+    if (cudaMalloc(&b->d_top, want) != cudaSuccess) { cudaGetLastError(); return; }
+    b->d_top_bytes = want;
+  }
+  if (tb_launch_beam_topm(p->logits, p->dtype, p->B, T, E, p->V, p->C, p->stream_stride, frame_stride, row_stride, n_frames,
+                          b->d_slots, b->arena, b->d_cls, M, b->d_top, stream) != TB_OK)
+    return;
+  p->top_base = b->d_top; p->top_m = M;
 }
 
 extern "C" int tb_beam_reset(tb_batch* b) {
@@ -756,6 +785,7 @@ extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_
   p.tree = b->d_tree; p.slots = b->d_slots; p.arena = b->arena; p.cls = b->d_cls; p.status = b->d_status;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
+  beam_prepass(b, &p, T, E, frame_stride, row_stride, nullptr, static_cast<cudaStream_t>(stream_));
   int rc = tb_launch_beam_frames(p, T, E, frame_stride, row_stride, static_cast<cudaStream_t>(stream_));
   if (rc == TB_OK) b->beam_steps += n_steps;
   if (rc == TB_OK && b->d_tree) { b->tree_steps += n_steps; b->tree_B = B; b->tree_K = K; }
@@ -808,6 +838,7 @@ extern "C" int tb_beam_chunk(tb_batch* b, const void* logits, int dtype, int32_t
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  beam_prepass(b, &p, chunk, E, frame_stride, row_stride, n_frames, static_cast<cudaStream_t>(stream_));
   const int rc = tb_launch_beam_chunk(p, chunk, E, frame_stride, row_stride, n_frames, b->d_slot_pos, b->d_hyp_hash,
                                       b->d_hyp_len, n_hyp, static_cast<cudaStream_t>(stream_));
   if (rc == TB_OK) b->chunk_K = K;

@@ -42,6 +42,12 @@ struct TokView {
 __host__ __device__ inline size_t tokview_bytes(int V, int C) {
   return static_cast<size_t>(C) * 8 + static_cast<size_t>(V) * 8 + ((static_cast<size_t>(V) * 2 + 8 + 15) & ~size_t(15));
 }
+// The beam kernels' auxiliary shared memory behind the candidate arrays: class vectors or the token view.
+__host__ __device__ inline size_t beam_aux_bytes(int V, int C, int tokview) {
+  size_t a = static_cast<size_t>(C) * 8;
+  if (tokview && tokview_bytes(V, C) > a) a = tokview_bytes(V, C);
+  return (a + 15) & ~size_t(15);
+}
 __device__ inline void tokview_init(TokView& tv, unsigned char* mem, int V, int C, const GraphPtrs& g) {
   tv.rootcw = reinterpret_cast<float*>(mem);
   tv.rootdst = reinterpret_cast<int32_t*>(mem + 4 * static_cast<size_t>(C));
@@ -242,8 +248,9 @@ constexpr int kBeamPref = 5;   // elements of a shared row each thread may hold 
 // xpre / xpre_valid: this thread's elements of the stream's shared row, fetched ahead by the previous step of the same
 // launch; next_row: where the next step's shared row starts (null: none), fetched while this step selects.
 template <typename LT>
-__device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xpre)[kBeamPref], bool& xpre_valid,
-                                               const LT* next_row) {
+__device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)[kBeamPref], bool& xpre_valid,
+                                               const LT* next_row, TbTopEnt& tpre, bool& tpre_valid,
+                                               const TbTopEnt* next_top) {
   extern __shared__ __align__(16) unsigned char dyn[];
   const int V = p.V, K = p.K, W = V + 1;
   float* cand = reinterpret_cast<float*>(dyn);                         // [K, V+1]
@@ -266,6 +273,12 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   __shared__ unsigned long long h_hash[TB_MAX_BEAM];   // identity of the hypothesis' token sequence
   __shared__ int32_t h_len[TB_MAX_BEAM];
   __shared__ BeamKey sel[TB_MAX_BEAM];
+  __shared__ int32_t sel_dst[TB_MAX_BEAM];      // compact path: the graph state a selected candidate leads to
+  __shared__ int32_t cp_n, cp_flag;             // compact path: candidates laid out; 0 = this step cannot take it
+  __shared__ int32_t cp_off[TB_MAX_BEAM + 1];   // compact path: where each hypothesis' listed candidates start
+  __shared__ int32_t rec_ready;                 // the hypotheses' list records in h_beg / h_cnt / h_D are those of their current states
+  __shared__ TbTopEnt ttop[2 * TB_MAX_BEAM + 9]; // this step's reduced row
+  __shared__ float root_wmax;                   // largest |root arc weight| of the stream's graph (filled with the root tables)
 
   const int b = blockIdx.x;
   const TbSlotRec rec = p.slots[b];
@@ -277,19 +290,30 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   // rows shared by the hypotheses of a stream (hyp_stride 0) depend on nothing that is loaded below: fetch this
   // thread's elements now, so that their latency overlaps the loads of the slot record, states and lists
   constexpr int kPref = kBeamPref;
-  const bool pref = use_tv && p.hyp_stride == 0 && W <= kPref * kBeamThreads;
+  const bool pref = (use_tv || (!bound && p.top_row != nullptr)) && p.hyp_stride == 0 && W <= kPref * kBeamThreads;
   if (pref && !xpre_valid) {
     const LT* row0 = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
 #pragma unroll
     for (int j = 0; j < kPref; ++j) {
       const int v = threadIdx.x + j * kBeamThreads;
-      xpre[j] = v < W ? LogitLoad<LT>::at(row0 + v) : 0.0f;
+      if (v < W) xpre[j] = LogitLoad<LT>::raw(row0 + v);
     }
   }
   TokView tv;
   if (use_tv) {
     if (p.tv_ready) tokview_attach(tv, aux, V, p.C);      // a later step of the same launch: the root tables are there
-    else tokview_init(tv, aux, V, p.C, g);
+    else {
+      tokview_init(tv, aux, V, p.C, g);
+      if (warp == 0) {
+        float r = 0.0f;
+        for (int c = lane; c < p.C; c += 32) r = fmaxf(r, fabsf(tv.rootcw[c]));
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, off));
+        if (lane == 0) root_wmax = r;
+      }
+    }
+  } else if (!p.tv_ready && threadIdx.x == 0) {
+    root_wmax = 0.0f;
   }
 
   if (threadIdx.x < K) {
@@ -344,8 +368,209 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   unsigned long long m1 = 0ull, m2 = 0ull;
   bool swept = false;
   auto offer = [&](unsigned long long kk) { if (kk > m1) { m2 = m1; m1 = kk; } else if (kk > m2) m2 = kk; };
+  // ---- the compact path ---------------------------------------------------------------------------------
+  // With the row reduced ahead of time to its top_m root-boosted tokens (k_beam_topm), a hypothesis' candidates are
+  // its blank, the tokens its graph state lists (exact values from their entries) and the first tokens of that
+  // short list which the state does not list (exact values from the list's logits): a few dozen per hypothesis
+  // instead of vocab + 1.  Every token outside the list has y <= y_next, hence a value of at most
+  // score + y_next + lambda * D plus roundings; the step is valid when the K-th selected candidate clears that
+  // bound for every hypothesis by a margin that dominates the roundings.  Otherwise (or with a very long list)
+  // the step is done again the long way below.
+  bool compact_done = false;
+  bool row_staged = false;      // the compact path put this step's row into shared memory and asked for the next one (in xpre)
+  float* xrow_s = reinterpret_cast<float*>(aux + beam_aux_bytes(V, p.C, p.tokview));
+  if (p.top_row != nullptr && p.hyp_stride == 0 && (use_tv || !bound) && p.top_m <= 2 * TB_MAX_BEAM + 8) {
+    unsigned long long* ckey = reinterpret_cast<unsigned long long*>(cand);
+    const int M = p.top_m;
+    float* xrow = xrow_s;                                     // [W] this step's row, staged
+    // the candidate arrays share the whole-row path's value array: keys, target states, then the warps' picks
+    const int wsel_bytes = (kBeamThreads / 32) * TB_MAX_BEAM * 12;
+    const int cap = (static_cast<int>(static_cast<size_t>(K) * W * sizeof(float)) - wsel_bytes - 16) / 12 & ~1;
+    int32_t* cdst = reinterpret_cast<int32_t*>(ckey + cap);
+    const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+    const bool recs_at_hand = p.tv_ready && rec_ready;        // left by the previous step of this launch
+    if (threadIdx.x < K && !recs_at_hand) {
+      const int k = threadIdx.x;
+      h_beg[k] = 0; h_cnt[k] = 0; h_D[k] = 0.0f;
+      if (bound && h_score[k] != -INFINITY) {
+        int32_t st = h_state[k];
+        if (st < 0 || st >= rec.n_states) { atomicOr(p.status, TB_STATUS_BAD_STATE); st = 0; }
+        const TbRsRec r = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[st];
+        h_beg[k] = r.begin; h_cnt[k] = r.count; h_D[k] = r.D;
+      }
+    }
+    for (int i = threadIdx.x; i < K * WW; i += kBeamThreads) ovr[i] = 0u;
+    // the row and its reduced form, asked for during the previous step (or now), go to shared memory
+    if (pref) {
+#pragma unroll
+      for (int j = 0; j < kPref; ++j) { const int v = threadIdx.x + j * kBeamThreads; if (v < W) xrow[v] = LogitLoad<LT>::widen(xpre[j]); }
+    }
+    if (threadIdx.x <= M) ttop[threadIdx.x] = tpre_valid ? tpre : p.top_row[threadIdx.x];
+    __syncthreads();
+    // the next step's row and reduced row are requested now: their trip overlaps the rest of this step
+    row_staged = pref;
+    xpre_valid = false;
+    if (pref && next_row) {
+#pragma unroll
+      for (int j = 0; j < kPref; ++j) {
+        const int v = threadIdx.x + j * kBeamThreads;
+        if (v < W) xpre[j] = LogitLoad<LT>::raw(next_row + v);      // (the load alone: widened when it is used)
+      }
+      xpre_valid = true;
+    }
+    tpre_valid = false;
+    if (next_top) { if (threadIdx.x <= M) tpre = next_top[threadIdx.x]; tpre_valid = true; }
+    // (one warp doing a narrow beam's few dozen candidates by itself, with warp-wide synchronisation only, was
+    // measured slower than the whole block: 8.4 against 6.9 ms per utterance at K = 4)
+    const int cth = static_cast<int>(threadIdx.x), cnt = kBeamThreads;
+    {
+      if (cth == 0) {
+        int at = 0;
+        for (int k = 0; k < K; ++k) {
+          cp_off[k] = at;
+          const bool lv = h_score[k] != -INFINITY && h_live[k];
+          hl_n[k] = !lv ? 0 : (h_cnt[k] <= kBeamList ? h_cnt[k] : -1);
+          if (lv) at += h_cnt[k];
+        }
+        cp_off[K] = at;
+        cp_flag = at + K * (M + 1) <= cap ? 1 : 0;
+        cp_n = at + K * (M + 1);
+      }
+      __syncthreads();
+      if (cp_flag) {
+        const int n_listed = cp_off[K], n = cp_n;
+        // the listed tokens of every hypothesis, all hypotheses at once: exact values; marked, so that the walk over
+        // the reduced row leaves them out.  Candidate slots that stay unused hold key 0 (none).
+        if (bound) {
+          const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
+          // (eight entries per thread are requested before the first is used: one trip to L2 for all of them)
+          for (int q0 = cth; q0 < n_listed; q0 += 8 * cnt) {
+            TbRsEnt e8[8];
+            int k8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int q = q0 + j * cnt;
+              int k = 0;
+              if (q < n_listed) {
+                while (q >= cp_off[k + 1]) ++k;
+                e8[j] = ent[h_beg[k] + (q - cp_off[k])];
+              }
+              k8[j] = k;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int q = q0 + j * cnt;
+              if (q >= n_listed) continue;
+              const int k = k8[j], i = q - cp_off[k];
+              const TbRsEnt e = e8[j];
+              const int tk = static_cast<int>((e.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
+              if (i < kBeamList) { hl_tok[k][i] = static_cast<uint16_t>(tk); hl_dst[k][i] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS); }
+              unsigned long long key = 0ull;
+              if (tk < V) {
+                const float x = pref ? xrow[tk] : LogitLoad<LT>::at(base + tk);
+                key = make_key(__fadd_rn(h_score[k], __fadd_rn(x, e.lb)), tk, k);
+                atomicOr(&ovr[k * WW + (tk >> 5)], 1u << (tk & 31));
+              }
+              ckey[q] = key; cdst[q] = static_cast<int32_t>(e.dst_tok >> TB_RS_TOK_BITS);
+            }
+          }
+        }
+        __syncthreads();
+        // blank, the first unlisted tokens of the reduced row, and the frozen hypotheses' carried candidates
+        for (int pr = cth; pr < K * (M + 1); pr += cnt) {
+          const int k = pr / (M + 1), j = pr - k * (M + 1);
+          unsigned long long key = 0ull;
+          int32_t dst = -1;
+          if (h_score[k] != -INFINITY) {
+            const TbTopEnt t = ttop[j];
+            if (!h_live[k]) {
+              if (j == M) { key = make_key(h_score[k], V + 1, k); dst = h_state[k]; }
+            } else if (j == M) {
+              key = make_key(__fadd_rn(h_score[k], t.x), V, k); dst = h_state[k];
+            } else {
+              const int tk = static_cast<int>(t.tok_cls & 0xFFFFu), cl = static_cast<int>(t.tok_cls >> 16);
+              if (tk < V && !((ovr[k * WW + (tk >> 5)] >> (tk & 31)) & 1u)) {     // (tk >= V: the row has fewer tokens)
+                const float val = bound ? __fadd_rn(t.x, __fmul_rn(g.lambda, __fadd_rn(h_D[k], tv.rootcw[cl]))) : t.x;
+                key = make_key(__fadd_rn(h_score[k], val), tk, k);
+                dst = bound ? tv.rootdst[cl] : -1;
+              }
+            }
+          }
+          ckey[n_listed + pr] = key; cdst[n_listed + pr] = dst;
+        }
+        __syncthreads();
+        {
+          // Selection in two levels, without a block-wide barrier per round: every warp picks the K best of the
+          // candidates it looks at (indices warp * 32 + lane, + the block size, ...) in K warp-wide rounds and
+          // leaves them, best first, in shared memory; warp 0 then merges the warps' lists, one lane per list.
+          unsigned long long* wkey = reinterpret_cast<unsigned long long*>(cdst + cap);            // [warps][K] (key); behind the targets
+          int32_t* widx = reinterpret_cast<int32_t*>(wkey + (kBeamThreads / 32) * TB_MAX_BEAM);   // [warps][K] where in ckey
+          {
+            unsigned long long lim = ~0ull;
+            for (int r = 0; r < K; ++r) {
+              unsigned long long a = 0ull;
+              int ai = -1;
+              for (int i = threadIdx.x; i < n; i += kBeamThreads) { const unsigned long long kk = ckey[i]; if (kk < lim && kk > a) { a = kk; ai = i; } }
+              const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+              const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+              const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+              const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+              if (best != 0ull && a == best) { wkey[warp * TB_MAX_BEAM + r] = best; widx[warp * TB_MAX_BEAM + r] = ai; }
+              if (best == 0ull && lane == 0) { wkey[warp * TB_MAX_BEAM + r] = 0ull; widx[warp * TB_MAX_BEAM + r] = -1; }
+              lim = best;                                       // (0 once nothing is left: the later rounds find nothing either)
+            }
+          }
+          __syncthreads();
+          if (warp == 0) {
+            // lane w walks warp w's list from its head; a round takes the largest head
+            int ptr = 0;
+            for (int r = 0; r < K; ++r) {
+              const unsigned long long a = (lane < kBeamThreads / 32 && ptr < K) ? wkey[lane * TB_MAX_BEAM + ptr] : 0ull;
+              const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+              const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+              const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+              const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+              if (best == 0ull) {
+                if (lane == 0) { sel[r] = BeamKey{-INFINITY, INT32_MAX, INT32_MAX}; sel_dst[r] = -1; }
+              } else if (a == best) {
+                const uint32_t l2 = 0xFFFFFFFFu - static_cast<uint32_t>(best & 0xFFFFFFFFull);
+                BeamKey c;
+                c.v = __uint_as_float(mh ^ ((mh >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+                c.tkey = static_cast<int32_t>(l2 >> 5); c.par = static_cast<int32_t>(l2 & 31u);
+                sel[r] = c; sel_dst[r] = cdst[widx[lane * TB_MAX_BEAM + ptr]];
+                ++ptr;
+              }
+            }
+          }
+        }
+        __syncthreads();
+        if (cth == 0) {
+          // does the K-th pick clear everything that was not looked at?
+          const float y_next = ttop[M].y;
+          int ok = 1;
+          if (y_next != -INFINITY) {
+            const float c_k = sel[K - 1].par != INT32_MAX ? sel[K - 1].v : -INFINITY;
+            for (int k = 0; k < K; ++k) {
+              if (h_score[k] == -INFINITY || !h_live[k]) continue;
+              const float lamD = bound ? g.lambda * h_D[k] : 0.0f;
+              const float scale = fabsf(h_score[k]) + fabsf(y_next) + 2.0f * (bound ? fabsf(g.lambda) * (fabsf(h_D[k]) + root_wmax) : 0.0f);
+              const float ub = (h_score[k] + y_next) + lamD + scale * 3.814697265625e-6f + 1e-30f;      // 2^-18 of the scale
+              if (!(c_k > ub)) ok = 0;
+            }
+          }
+          cp_flag = ok;
+        }
+      }
+    }
+    __syncthreads();
+    compact_done = cp_flag != 0;
+  }
+  if (threadIdx.x == 0) rec_ready = 0;      // (set again below, once the new hypotheses' records have been fetched)
+
   // all candidate values of the live hypotheses
-  if (use_tv) {
+  if (compact_done) {
+    // (nothing to lay out)
+  } else if (use_tv) {
     // every hypothesis at once: its state's record, then all plain values, then the listed tokens on top
     if (threadIdx.x < K) {
       const int k = threadIdx.x;
@@ -385,7 +610,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
         const int v = threadIdx.x + j * kBeamThreads;
         if (v < W) {
           const float plain_w = v < V ? tv.rootcw[__ldg(p.cls + v)] : 0.0f;
-          const float x = xpre[j];
+          const float x = row_staged ? xrow_s[v] : LogitLoad<LT>::widen(xpre[j]);
           for (int k = 0; k < K; ++k) {
             if (h_score[k] == -INFINITY || !h_live[k]) continue;
             float c;
@@ -445,14 +670,18 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
   // best key below `limit` among this thread's candidates: tokens v = tid, tid + 256, ... of every live
   // hypothesis, plus (thread k) the carried candidate of a frozen hypothesis k
   // the row of the next step is requested now: its trip from HBM overlaps the selection rounds
-  xpre_valid = false;
-  if (pref && next_row) {
+  if (!compact_done && !row_staged) {
+    xpre_valid = false;
+    if (pref && next_row) {
 #pragma unroll
-    for (int j = 0; j < kPref; ++j) {
-      const int v = threadIdx.x + j * kBeamThreads;
-      xpre[j] = v < W ? LogitLoad<LT>::at(next_row + v) : 0.0f;
+      for (int j = 0; j < kPref; ++j) {
+        const int v = threadIdx.x + j * kBeamThreads;
+        if (v < W) xpre[j] = LogitLoad<LT>::raw(next_row + v);
+      }
+      xpre_valid = true;
     }
-    xpre_valid = true;
+    tpre_valid = false;
+    if (next_top) { if (threadIdx.x <= p.top_m) tpre = next_top[threadIdx.x]; tpre_valid = true; }
   }
   unsigned long long spare = 0ull;                            // this thread's second best key below the limit of its last scan
   bool have_spare = false;
@@ -473,10 +702,11 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
     spare = m2; have_spare = true;
     return m;
   };
-  unsigned long long mine;
-  if (swept) { mine = m1; spare = m2; have_spare = true; }     // collected during the sweep
+  unsigned long long mine = 0ull;
+  if (compact_done) { /* picked already */ }
+  else if (swept) { mine = m1; spare = m2; have_spare = true; }     // collected during the sweep
   else mine = scan_mine(~0ull);
-  for (int r = 0; r < K; ++r) {
+  for (int r = 0; r < K && !compact_done; ++r) {
     // the warp's best key: the largest high word, then the largest low word among the lanes that have it
     const uint32_t hi = static_cast<uint32_t>(mine >> 32), lo = static_cast<uint32_t>(mine);
     const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
@@ -517,7 +747,9 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
       token = (c.tkey == V + 1) ? -1 : c.tkey;
       state = h_state[parent];
       if (token >= 0 && token != V) {
-        if (use_tv && hl_n[parent] >= 0) {
+        if (compact_done) {
+          state = sel_dst[r];
+        } else if (use_tv && hl_n[parent] >= 0) {
           int nx = tv.rootdst[__ldg(p.cls + token)];          // a pick that the parent's list does not hold is a plain token
           for (int i = 0; i < hl_n[parent]; ++i)
             if (hl_tok[parent][i] == token) { nx = hl_dst[parent][i]; break; }
@@ -548,19 +780,31 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, float (&xp
       p.tree[at * K + r] = make_int2(parent, token);
     }
   }
+  // the list record of every new hypothesis' state, for the next step's compact path: fetched now, so that its trip
+  // to L2 is over when that step starts
+  TbRsRec nrec{0, 0, 0.0f, 0.0f};
+  int rec_ok = 1;
+  if (threadIdx.x < K && p.top_row != nullptr && use_tv && sc != -INFINITY) {
+    if (state >= 0 && state < rec.n_states) nrec = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[state];
+    else rec_ok = 0;                                        // (the next step reports it)
+  }
   // ... and in shared memory, for the next step of a launch that runs several (read by every thread above: wait)
-  __syncthreads();
+  const int all_ok = __syncthreads_and(rec_ok);
   if (threadIdx.x < K) {
     h_score[threadIdx.x] = sc; h_state[threadIdx.x] = state; h_live[threadIdx.x] = lv;
     h_hash[threadIdx.x] = nh; h_len[threadIdx.x] = nl;
+    if (p.top_row != nullptr) { h_beg[threadIdx.x] = nrec.begin; h_cnt[threadIdx.x] = nrec.count; h_D[threadIdx.x] = nrec.D; }
   }
+  if (threadIdx.x == 0) rec_ready = (p.top_row != nullptr && (use_tv || !bound) && all_ok) ? 1 : 0;
 }
 
 template <typename LT>
 __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
-  float xpre[kBeamPref];
+  LT xpre[kBeamPref] = {};
   bool xpre_valid = false;
-  beam_step_body<LT>(p, xpre, xpre_valid, static_cast<const LT*>(nullptr));
+  TbTopEnt tpre{0.0f, 0.0f, 0u};
+  bool tpre_valid = false;
+  beam_step_body<LT>(p, xpre, xpre_valid, static_cast<const LT*>(nullptr), tpre, tpre_valid, nullptr);
 }
 
 // T frames of E rows in one launch: the block loops over the expansions of its stream; every hypothesis of the
@@ -569,8 +813,10 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
 template <typename LT>
 __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
                                                           int64_t row_stride) {
-  float xpre[kBeamPref];
+  LT xpre[kBeamPref] = {};
   bool xpre_valid = false;
+  TbTopEnt tpre{0.0f, 0.0f, 0u};
+  bool tpre_valid = false;
   const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(blockIdx.x) * p.stream_stride;
   for (int32_t t = 0; t < T; ++t) {
     for (int32_t e = 0; e < E; ++e) {
@@ -584,12 +830,90 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, in
       q.fresh = (p.fresh && sidx == 0) ? 1 : 0;
       q.tv_ready = sidx > 0 ? 1 : 0;
       q.step = p.step + sidx;
+      q.top_row = p.top_base ? p.top_base + (static_cast<int64_t>(blockIdx.x) * T * E + sidx) * (p.top_m + 1) : nullptr;
       if (sidx & 1) { q.hash_in = p.hash_out; q.hash_out = const_cast<unsigned long long*>(p.hash_in); q.len_in = p.len_out; q.len_out = const_cast<int32_t*>(p.len_in); }
       const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
       const LT* next_row = nt < T ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
-      beam_step_body<LT>(q, xpre, xpre_valid, next_row);
+      const TbTopEnt* next_top = (nt < T && q.top_row) ? q.top_row + (p.top_m + 1) : nullptr;
+      beam_step_body<LT>(q, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
       __syncthreads();
     }
+  }
+}
+
+// Beam pre-pass: one warp per logit row, independent of every hypothesis.  With the rows of a stream shared by its
+// hypotheses, the order of a row's tokens that no hypothesis' state boosts is, up to rounding, the order of their
+// root-boosted values y -- so a step only needs the first few of them (see the compact path of beam_step_body).
+constexpr int kTopWarps = 8;
+template <typename LT>
+__global__ void __launch_bounds__(kTopWarps * 32) k_beam_topm(const LT* logits, int32_t B, int32_t T, int32_t E, int32_t V, int32_t C,
+                                                            int64_t stream_stride, int64_t frame_stride, int64_t row_stride,
+                                                            const int32_t* n_frames, const TbSlotRec* slots, const unsigned char* arena,
+                                                            const int32_t* cls, int32_t top_m, TbTopEnt* out) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  float* rootcw = reinterpret_cast<float*>(dyn);                                  // [C] root arc weight per class
+  float* ybuf = reinterpret_cast<float*>(dyn) + C;                                // [kTopWarps][V]
+  const int rows_per_stream = T * E, blocks_per_stream = (rows_per_stream + kTopWarps - 1) / kTopWarps;
+  const int b = blockIdx.x / blocks_per_stream, r0 = (blockIdx.x - b * blocks_per_stream) * kTopWarps;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const TbSlotRec rec = slots[b];
+  const bool bound = rec.n_states > 0;
+  const GraphPtrs g = graph_of(arena, rec);
+  for (int c = threadIdx.x; c < C; c += blockDim.x) rootcw[c] = 0.0f;
+  __syncthreads();
+  if (bound) {
+    const int e = g.arc_begin[1];
+    for (int a = g.arc_begin[0] + threadIdx.x; a < e; a += blockDim.x) {
+      const int c = g.arc_cls[a];
+      if (c >= 0 && c < C) rootcw[c] = __fadd_rn(0.0f, g.arc_w[a]);
+    }
+  }
+  __syncthreads();
+  const int r = r0 + warp;
+  if (r >= rows_per_stream) return;
+  const int t = r / E, e = r - t * E;
+  if (n_frames && t >= n_frames[b]) return;
+  const LT* row = logits + static_cast<int64_t>(b) * stream_stride + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
+  TbTopEnt* o = out + (static_cast<int64_t>(b) * rows_per_stream + r) * (top_m + 1);
+  float* y = ybuf + static_cast<size_t>(warp) * V;
+  // y of every token, this lane's best (value, lowest token) on the way
+  float bv = -INFINITY;
+  int bi = INT32_MAX;
+  for (int v = lane; v < V; v += 32) {
+    const float x = LogitLoad<LT>::at(row + v);
+    const float yv = bound ? __fadd_rn(x, __fmul_rn(g.lambda, rootcw[__ldg(cls + v)])) : x;
+    y[v] = yv;
+    if (yv > bv) { bv = yv; bi = v; }
+  }
+  if (bi == INT32_MAX && lane < V) bi = lane;                 // every value of the strip is -inf: still a token
+  __syncwarp();
+  for (int m = 0; m <= top_m; ++m) {
+    // the warp's best: largest value, then lowest token
+    const uint32_t u = __float_as_uint(bv + 0.0f);
+    const uint32_t key = bi == INT32_MAX ? 0u : (u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u));
+    const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+    const uint32_t imin = __reduce_min_sync(0xffffffffu, (key == kmax && bi != INT32_MAX) ? static_cast<uint32_t>(bi) : 0xFFFFFFFFu);
+    const bool none = imin == 0xFFFFFFFFu;                    // fewer than m + 1 tokens in the row
+    if (m == top_m) {
+      if (lane == 0) { o[m].y = none ? -INFINITY : y[imin]; o[m].x = LogitLoad<LT>::at(row + V); o[m].tok_cls = 0u; }
+      break;
+    }
+    if (lane == 0) {
+      if (none) { o[m].y = -INFINITY; o[m].x = -INFINITY; o[m].tok_cls = 0xFFFFu; }
+      else { o[m].y = y[imin]; o[m].x = LogitLoad<LT>::at(row + imin); o[m].tok_cls = imin | (static_cast<uint32_t>(__ldg(cls + imin)) << 16); }
+    }
+    if (!none && static_cast<uint32_t>(bi) == imin) {
+      // the owner takes it out and looks for its next best
+      y[bi] = __int_as_float(0x7FC00000);                     // (a NaN: never greater than anything, never chosen again)
+      bv = -INFINITY; bi = INT32_MAX;
+      int first_left = INT32_MAX;
+      for (int v = lane; v < V; v += 32) {
+        const float yv = y[v];
+        if (yv == yv) { if (first_left == INT32_MAX) first_left = v; if (yv > bv) { bv = yv; bi = v; } }
+      }
+      if (bi == INT32_MAX) bi = first_left;                   // only -inf values left in the strip
+    }
+    __syncwarp();
   }
 }
 
@@ -600,8 +924,10 @@ template <typename LT>
 __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
                                                          int64_t row_stride, const int32_t* n_frames, int32_t* slot_pos,
                                                          unsigned long long* hash, int32_t* len, size_t n_hyp) {
-  float xpre[kBeamPref];
+  LT xpre[kBeamPref] = {};
   bool xpre_valid = false;
+  TbTopEnt tpre{0.0f, 0.0f, 0u};
+  bool tpre_valid = false;
   const int b = blockIdx.x;
   const int32_t nf = n_frames ? max(0, min(T, n_frames[b])) : T;
   const int32_t pos0 = slot_pos[b];
@@ -618,11 +944,13 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int
       q.fresh = 0;
       q.tv_ready = sidx > 0 ? 1 : 0;
       q.step = pos0 + sidx;
+      q.top_row = p.top_base ? p.top_base + (static_cast<int64_t>(b) * T * E + sidx) * (p.top_m + 1) : nullptr;
       const size_t in = ((pos0 + sidx) & 1) ? n_hyp : 0, out = ((pos0 + sidx) & 1) ? 0 : n_hyp;
       q.hash_in = hash + in; q.hash_out = hash + out; q.len_in = len + in; q.len_out = len + out;
       const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
       const LT* next_row = nt < nf ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
-      beam_step_body<LT>(q, xpre, xpre_valid, next_row);
+      const TbTopEnt* next_top = (nt < nf && q.top_row) ? q.top_row + (p.top_m + 1) : nullptr;
+      beam_step_body<LT>(q, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
       __syncthreads();
     }
   }
@@ -732,9 +1060,8 @@ int tb_launch_decode_general(const TbDecodeParams& p_in, cudaStream_t stream) {
 
 int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
   TbBeamParams p = p_in;
-  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
-  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t aux = beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(p.V + 1) * sizeof(float);   // + the staged row
   const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
                       ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
@@ -752,9 +1079,8 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
 int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
                           cudaStream_t stream) {
   TbBeamParams p = p_in;
-  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
-  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t aux = beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(p.V + 1) * sizeof(float);   // + the staged row
   const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
                       ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
@@ -870,9 +1196,8 @@ int tb_launch_beam_chunk(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t
                          const int32_t* n_frames, int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp,
                          cudaStream_t stream) {
   TbBeamParams p = p_in;
-  size_t aux = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
-  if (p.tokview && tokview_bytes(p.V, p.C) > aux) aux = tokview_bytes(p.V, p.C);
+  const size_t aux = beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(p.V + 1) * sizeof(float);   // + the staged row
   const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
                       ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
@@ -918,5 +1243,24 @@ int tb_launch_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n, co
                             cudaStream_t stream) {
   if (n < 1) return TB_ERR_INVALID_ARG;
   k_publish_slots<<<(n + 63) / 64, 64, 0, stream>>>(slots, sstate, n, recs, slot_of);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_beam_topm(const void* logits, int dtype, int32_t B, int32_t T, int32_t E, int32_t V, int32_t C,
+                        int64_t stream_stride, int64_t frame_stride, int64_t row_stride, const int32_t* n_frames,
+                        const TbSlotRec* slots, const unsigned char* arena, const int32_t* cls, int32_t top_m,
+                        TbTopEnt* out, cudaStream_t stream) {
+  const size_t smem = (static_cast<size_t>(C) + static_cast<size_t>(kTopWarps) * V) * sizeof(float);
+  const int blocks = B * ((T * E + kTopWarps - 1) / kTopWarps);
+  int rc;
+  if (dtype == TB_BF16) {
+    if ((rc = set_smem(k_beam_topm<uint16_t>, smem)) != TB_OK) return rc;
+    k_beam_topm<uint16_t><<<blocks, kTopWarps * 32, smem, stream>>>(static_cast<const uint16_t*>(logits), B, T, E, V, C, stream_stride,
+                                                                  frame_stride, row_stride, n_frames, slots, arena, cls, top_m, out);
+  } else {
+    if ((rc = set_smem(k_beam_topm<float>, smem)) != TB_OK) return rc;
+    k_beam_topm<float><<<blocks, kTopWarps * 32, smem, stream>>>(static_cast<const float*>(logits), B, T, E, V, C, stream_stride,
+                                                               frame_stride, row_stride, n_frames, slots, arena, cls, top_m, out);
+  }
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }

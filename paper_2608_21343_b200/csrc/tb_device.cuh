@@ -39,11 +39,16 @@ __device__ __forceinline__ GraphPtrs graph_of(const unsigned char* arena, const 
 template <typename LT> struct LogitLoad;
 template <> struct LogitLoad<float> {
   static __device__ __forceinline__ float at(const float* p) { return __ldg(p); }
+  // the load alone (nothing waits for it until the value is widened), and the widening
+  static __device__ __forceinline__ float raw(const float* p) { return __ldg(p); }
+  static __device__ __forceinline__ float widen(float r) { return r; }
 };
 template <> struct LogitLoad<uint16_t> {  // bf16 bits, widened exactly
   static __device__ __forceinline__ float at(const uint16_t* p) {
     return __uint_as_float(static_cast<uint32_t>(__ldg(p)) << 16);
   }
+  static __device__ __forceinline__ uint16_t raw(const uint16_t* p) { return __ldg(p); }
+  static __device__ __forceinline__ float widen(uint16_t r) { return __uint_as_float(static_cast<uint32_t>(r) << 16); }
 };
 
 // Index of the arc of state u labelled with class c, or -1 (arcs are sorted by class).

@@ -24,6 +24,15 @@ struct TbDecodeParams {
   int32_t* status;
 };
 
+// What the beam pre-pass leaves per logit row: the top_m tokens (blank excluded) with the largest root-boosted value
+// y = fl(x + fl(lambda * w_root(class))), best first (ties: lowest token), and in entry top_m the value y of the next one
+// (-inf if there is none) together with the row's blank logit in x.
+struct TbTopEnt {
+  float y;
+  float x;            // the token's logit (entry top_m: the blank logit)
+  uint32_t tok_cls;   // token | class << 16
+};
+
 struct TbBeamParams {
   const void* logits; int dtype;
   int32_t B, K, V, C, new_frame, step;
@@ -40,6 +49,11 @@ struct TbBeamParams {
   // streaming (tb_beam_chunk): every slot keeps its own ring of tree_cap steps, tree[slot][step % tree_cap][K]; 0: the
   // tree is [steps, B, K] for the whole batch
   int32_t tree_cap;
+  // rows reduced ahead of the steps (tb_launch_beam_topm): per row top_m + 1 entries of 12 bytes, see TbTopEnt; null: none.
+  // top_rows: this step's row (set per step inside a multi-step launch); top_base / strides: where the launch finds them
+  const struct TbTopEnt* top_row;
+  const struct TbTopEnt* top_base;
+  int32_t top_m;
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
 };
 
@@ -79,6 +93,12 @@ int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int
                                    cudaStream_t stream);
 int tb_launch_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, const int32_t* slot_list,
                                   int32_t K, float* scores, const int32_t* states, int32_t* status, cudaStream_t stream);
+// Reduces every row of [B, T, E] (element strides given) to its TbTopEnt entries: out[((b * T + t) * E + e) * (top_m + 1)].
+// n_frames: device [B] or null (rows of frames at or beyond it are skipped).
+int tb_launch_beam_topm(const void* logits, int dtype, int32_t B, int32_t T, int32_t E, int32_t V, int32_t C,
+                        int64_t stream_stride, int64_t frame_stride, int64_t row_stride, const int32_t* n_frames,
+                        const TbSlotRec* slots, const unsigned char* arena, const int32_t* cls, int32_t top_m,
+                        TbTopEnt* out, cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
                              int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
 // Registered models: their records live in a device table; tb_launch_bind_models points up to TB_BIND_PAIRS slots at

@@ -302,3 +302,33 @@ def test_beam_widths_whose_shared_memory_straddles_the_default_limit(tb, K):
     batch, _ = make_batch(tb, w, data["phrases"], max_beam=K, max_tree_steps=w.T * w.S)
     fr = run_beam_frames(tb, w, data, K, data["phrases"], batch)
     assert np.array_equal(fr["tokens"], out["tokens"]) and np.array_equal(fr["scores"], out["scores"])
+
+
+@pytest.mark.parametrize("K", [4, 16])
+def test_beam_frames_when_the_reduced_rows_do_not_suffice(tb, K):
+    """tb_beam_frames reduces every row to its few best tokens ahead of the steps and redoes a step on the whole row
+    when those cannot be shown to hold the K best candidates.  Flat rows (all tokens equal, or equal but for a few)
+    force that second path at almost every step; rows with a clear order in between take the short one.  Both,
+    with and without the pre-pass, against the oracle."""
+    w = W.get_workload(4, B=4, T=30, V=256, n_phrases=30, n_plants=3)
+    data = W.batch_inputs(w)
+    x = W.bf16_bits_to_f32(data["logits"])
+    x[:, 0::3, :, :w.V] = 0.0                                         # every token the same
+    x[:, 1::3, :, :w.V] = np.round(x[:, 1::3, :, :w.V])               # a handful of distinct values
+    x[:, :, :, w.V] = 0.25                                            # blank close to the tokens: tokens do get emitted
+    data["logits"] = W.f32_to_bf16_bits(x)
+    lists = [data["phrases"][0], None, data["phrases"][2], data["phrases"][3]]
+    refs = [O.beam_decode(oracle_graph(w, lists[i]), data["logits"][i], K, merge=True) for i in range(w.B)]
+    for flags in (0, tb.TB_FLAG_BEAM_WHOLE_ROWS):
+        batch, _ = make_batch(tb, w, lists, max_beam=K, max_tree_steps=w.T * w.S)
+        tb.tb_batch_set_flags(batch, flags)
+        out = run_beam_frames(tb, w, data, K, lists, batch, merge=True, chunks=(7, 23))
+        for i in range(w.B):
+            ref = refs[i]
+            assert np.array_equal(out["states"][i], ref["states"]) and np.array_equal(out["lens"][i], ref["lens"]), (flags, i)
+            assert np.array_equal(out["last"][i], ref["tree"][-1]), (flags, i)
+            for k in range(K):
+                assert np.array_equal(out["tokens"][i, k, :ref["lens"][k]], ref["tokens"][k]), (flags, i, k)
+            fin = np.isfinite(ref["scores"])
+            assert np.array_equal(np.isfinite(out["scores"][i]), fin)
+            assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL), (flags, i)
