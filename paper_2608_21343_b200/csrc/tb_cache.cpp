@@ -18,7 +18,7 @@
 namespace {
 
 constexpr uint32_t kMagic = 0x31474254u;   // "TBG1"
-constexpr uint32_t kVersion = 2;
+constexpr uint32_t kVersion = 3;
 
 // FNV-1a style checksum over 8-byte words (the tail byte by byte): detects damage, is not cryptographic
 uint64_t fnv1a(const void* p, size_t n, uint64_t h = 1469598103934665603ull) {
@@ -44,7 +44,7 @@ struct FileHeader {
   float d_max;
   int32_t off_final;
   uint64_t blob_bytes;
-  uint64_t payload_hash;   // of everything after the header
+  uint64_t payload_hash;   // of the header (this field taken as zero) followed by everything after it
 };
 
 template <typename T>
@@ -58,6 +58,13 @@ bool take(const unsigned char*& p, const unsigned char* end, std::vector<T>& v, 
   if (n) std::memcpy(v.data(), p, n * sizeof(T));
   p += n * sizeof(T);
   return true;
+}
+
+// Checksum of a file: the header with its checksum field zero, then the payload.
+uint64_t file_hash(const FileHeader& h0, const std::string& payload) {
+  std::string all(reinterpret_cast<const char*>(&h0), sizeof h0);
+  all.append(payload);
+  return fnv1a(all.data(), all.size());
 }
 
 size_t graph_bytes(const tb_graph* g) {
@@ -84,7 +91,8 @@ extern "C" int tb_graph_save(const tb_graph* g, const char* path) {
     h.off_arc_w = g->off_arc_w; h.off_arc_dst = g->off_arc_dst; h.off_strec = g->off_strec; h.off_tokent = g->off_tokent;
     h.n_tokent = g->n_tokent; h.off_rsrec = g->off_rsrec; h.off_rsent = g->off_rsent; h.n_rsent = g->n_rsent;
     h.d_max = g->d_max; h.off_final = g->off_final; h.blob_bytes = g->blob.size();
-    h.payload_hash = fnv1a(payload.data(), payload.size());
+    h.payload_hash = 0;
+    h.payload_hash = file_hash(h, payload);                  // header (with this field zero) and payload together
     std::FILE* f = std::fopen(path, "wb");
     if (!f) return TB_ERR_IO;
     bool ok = std::fwrite(&h, sizeof h, 1, f) == 1;
@@ -119,7 +127,12 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
     // a file that is not one of ours, was cut short or was altered is refused as a whole
     if (h.magic != kMagic || h.version != kVersion) return TB_ERR_INVALID_ARG;
     if (h.n_states < 1 || h.n_arcs < 0 || h.vocab < 1 || h.vocab > TB_MAX_VOCAB || h.n_classes < 1) return TB_ERR_INVALID_ARG;
-    if (h.payload_hash != fnv1a(payload.data(), payload.size())) return TB_ERR_INVALID_ARG;
+    {
+      FileHeader h0 = h;
+      h0.payload_hash = 0;
+      if (h.payload_hash != file_hash(h0, payload)) return TB_ERR_INVALID_ARG;
+    }
+    if (h.max_depth < 0 || h.max_depth > TB_MAX_PHRASE_LEN || h.n_tokent < 0) return TB_ERR_INVALID_ARG;
     g = new tb_graph();
     const unsigned char* p = reinterpret_cast<const unsigned char*>(payload.data());
     const unsigned char* end = p + payload.size();
@@ -142,6 +155,55 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
                             g->off_strec, g->off_tokent, g->off_rsrec, g->off_rsent, g->off_final};
     for (int32_t o : offs)
       if (o < 0 || o > B || (o & 15)) { delete g; return TB_ERR_INVALID_ARG; }
+    // ... with their whole extent, and what the kernels index with must stay inside the arrays
+    {
+      const int64_t Ns = h.n_states, As = h.n_arcs, Te = h.n_tokent, Re = h.n_rsent;
+      bool in = g->off_arc_begin + 4 * (Ns + 1) <= B && g->off_fail + 4 * Ns <= B && g->off_bw + 4 * Ns <= B &&
+                g->off_arc_cls + 4 * As <= B && g->off_arc_w + 4 * As <= B && g->off_arc_dst + 4 * As <= B &&
+                g->off_final + 4 * Ns <= B && g->off_strec + 16 * Ns <= B && g->off_tokent + 16 * Te <= B;
+      if (Re >= 0) in = in && g->off_rsrec + 16 * Ns <= B && g->off_rsent + 8 * Re <= B;
+      in = in && g->state_arc_begin[0] == 0 && g->state_arc_begin[Ns] == As;
+      for (int64_t u = 0; in && u < Ns; ++u)
+        in = g->state_arc_begin[u] <= g->state_arc_begin[u + 1] && g->state_fail[u] >= 0 && g->state_fail[u] < Ns;
+      for (int64_t a = 0; in && a < As; ++a)
+        in = g->arc_dst[a] >= 0 && g->arc_dst[a] < Ns && g->arc_class[a] >= 0 && g->arc_class[a] < h.n_classes;
+      if (!in) { delete g; return TB_ERR_INVALID_ARG; }
+      // the device-side copies of the same tables, and the derived records
+      const unsigned char* bl = g->blob.data();
+      auto i32 = [&](int32_t off, int64_t i) { int32_t v; std::memcpy(&v, bl + off + 4 * i, 4); return v; };
+      in = i32(g->off_arc_begin, 0) == 0 && i32(g->off_arc_begin, Ns) == As;
+      for (int64_t u = 0; in && u < Ns; ++u) {
+        const int32_t f = i32(g->off_fail, u);
+        in = i32(g->off_arc_begin, u) <= i32(g->off_arc_begin, u + 1) && f >= 0 && f < Ns;
+        TbStateRec sr;
+        std::memcpy(&sr, bl + g->off_strec + 16 * u, 16);
+        in = in && sr.tok_begin >= 0 && sr.tok_begin <= sr.tok_end && sr.tok_end <= Te && sr.fail >= 0 && sr.fail < Ns;
+      }
+      for (int64_t a = 0; in && a < As; ++a) {
+        const int32_t d = i32(g->off_arc_dst, a), c = i32(g->off_arc_cls, a);
+        in = d >= 0 && d < Ns && c >= 0 && c < h.n_classes;
+      }
+      for (int64_t e = 0; in && e < Te; ++e) {
+        TbTokEnt te;
+        std::memcpy(&te, bl + g->off_tokent + 16 * e, 16);
+        in = static_cast<int32_t>(te.tok_cls & 0xffffu) < h.vocab && te.dst >= 0 && te.dst < Ns;
+      }
+      if (Re >= 0) {
+        in = in && Re <= TB_RS_MAX_ENTRIES && h.vocab + 1 <= (1 << (TB_RS_TOK_BITS - 1));
+        for (int64_t u = 0; in && u < Ns; ++u) {
+          TbRsRec rr;
+          std::memcpy(&rr, bl + g->off_rsrec + 16 * u, 16);
+          in = rr.begin >= 0 && rr.count >= 0 && static_cast<int64_t>(rr.begin) + rr.count <= Re;
+        }
+        for (int64_t e = 0; in && e < Re; ++e) {
+          TbRsEnt re;
+          std::memcpy(&re, bl + g->off_rsent + 8 * e, 8);
+          const uint32_t tok2 = re.dst_tok & ((1u << TB_RS_TOK_BITS) - 1), dst = re.dst_tok >> TB_RS_TOK_BITS;
+          in = tok2 <= 2u * static_cast<uint32_t>(h.vocab) && (tok2 & 1u) == 0 && dst < static_cast<uint32_t>(Ns);
+        }
+      }
+      if (!in) { delete g; return TB_ERR_INVALID_ARG; }
+    }
     if (g->class_map_hash != tb_hash_class_map(g->case_class.data(), g->vocab)) { delete g; return TB_ERR_INVALID_ARG; }
     *out = g;
     return TB_OK;

@@ -193,6 +193,57 @@ def test_graph_load_refuses_damaged_files(tb, tmp_path):
     with pytest.raises(tb.TbError) as e:
         tb.tb_graph_load(str(tmp_path / "missing.tbg"))
     assert e.value.code == tb.TB_ERR_IO
+
+    # a file whose checksum is right but whose tables point outside themselves is refused as well
+    HDR, HASH_AT = 112, 104
+
+    def checksum(data):
+        h, m = 1469598103934665603, (1 << 64) - 1
+        i = 0
+        while i + 8 <= len(data):
+            h = ((h ^ int.from_bytes(data[i:i + 8], "little")) * 1099511628211) & m
+            h ^= h >> 29
+            i += 8
+        for c in data[i:]:
+            h = ((h ^ c) * 1099511628211) & m
+        return h
+
+    def resealed(b):
+        b = bytearray(b)
+        b[HASH_AT:HASH_AT + 8] = bytes(8)
+        b[HASH_AT:HASH_AT + 8] = checksum(bytes(b)).to_bytes(8, "little")
+        return bytes(b)
+    assert resealed(raw) == raw                                           # the checksum as this test computes it
+    hv = g.view()
+    N, A = hv["n_states"], hv["n_arcs"]
+    field = {"n_states": 8, "max_depth": 24, "off_arc_begin": 40, "off_strec": 64, "off_tokent": 68, "n_tokent": 72,
+             "off_rsrec": 76, "off_rsent": 80, "n_rsent": 84}
+
+    def with_i32(at, value):
+        b = bytearray(raw)
+        b[at:at + 4] = int(value).to_bytes(4, "little", signed=True)
+        return resealed(b)
+    n_tokent = int.from_bytes(raw[72:76], "little")
+    blob_bytes = int.from_bytes(raw[96:104], "little")
+    bad = [with_i32(field["max_depth"], 4096),                            # deeper than any phrase may be
+           with_i32(field["off_strec"], (blob_bytes - 16) & ~15),          # a section that runs off the end of the blob
+           with_i32(field["n_tokent"], n_tokent + (1 << 20)),
+           with_i32(field["n_rsent"], 1 << 17),
+           with_i32(HDR + 4 * (N + 1) + 4 * A, N),                        # first arc target: one past the last state
+           with_i32(HDR + 4 * (N + 1) + 4 * A, -1),
+           with_i32(HDR + 4 * (N + 1) + 3 * 4 * A + 4, N + 7),            # suffix link of state 1
+           with_i32(HDR + 4, 1 << 30)]                                          # arc ranges that go backwards
+    for data in bad:
+        assert code(data) == tb.TB_ERR_INVALID_ARG
+    # the same in the device copy of a table: suffix link of state 1 inside the blob
+    blob_at = len(raw) - blob_bytes
+    off_fail = int.from_bytes(raw[44:48], "little")
+    assert code(with_i32(blob_at + off_fail + 4, N)) == tb.TB_ERR_INVALID_ARG
+    off_rsent = int.from_bytes(raw[80:84], "little")
+    n_rsent = int.from_bytes(raw[84:88], "little", signed=True)
+    assert n_rsent > 0
+    ent = int.from_bytes(raw[blob_at + off_rsent:blob_at + off_rsent + 4], "little")
+    assert code(with_i32(blob_at + off_rsent, (ent & 0xfff) | ((N + 3) << 12))) == tb.TB_ERR_INVALID_ARG
     with pytest.raises(tb.TbError) as e:
         tb.tb_graph_save(g, str(tmp_path / "no_such_dir" / "g.tbg"))
     assert e.value.code == tb.TB_ERR_IO
