@@ -248,11 +248,12 @@ def side_measurement(args):
                                      "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
     elif args.workload == 5:
         w = W.get_workload(5, **({"B": args.streams} if args.streams else {}))
-        sched = W.ChurnSchedule(w)
+        sched = W.ChurnSchedule(w, workers=8)            # (the next chunks' inputs are drawn by worker threads)
         batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
         n_chunks, lat, binds, t_compile = 40 + 10 * args.steps, [], 0, 0.0
         host_us = []
         bufs = []
+        outs = None
         for c in range(n_chunks):
             chunk, lengths, bl = sched.next_chunk()
             t0 = time.perf_counter()
@@ -270,7 +271,7 @@ def side_measurement(args):
                     tb.tb_batch_bind_stream(batch, sl, g)
             else:
                 tb.tb_batch_bind_streams(batch, [sl for sl, _ in gs], [g for _, g in gs])   # one copy, one launch
-            tb.tb_stream_chunk(batch, dl, w.n_dur, dv)
+            outs = tb.tb_stream_chunk(batch, dl, w.n_dur, dv, out=outs)          # the result tensors are allocated once
             b.record()
             host_us.append((time.perf_counter() - th) * 1e6)
             torch.cuda.synchronize()

@@ -208,7 +208,10 @@ int tb_graph_load(const char *path, tb_graph **out);
  * returned but not kept).  The returned graph is the caller's to release with tb_graph_free as usual; it
  * stays valid after the cache drops or is destroyed.  Calls on one cache may come from several threads.
  * Graphs kept by a cache have their device blob page-locked (when a CUDA device is present), so binding them
- * copies from the graph in place; the batch holds the graph until that copy is done.
+ * copies from the graph in place; the batch holds the graph until that copy is done.  The same holds for every graph
+ * compiled or loaded after the process has created its first batch: their device blobs are placed in a pool of
+ * page-locked host memory (up to 1 GB, in pieces of 32 MB; blobs over 16 MB and whatever does not fit stay on the heap
+ * and are staged at bind time).
  *   out_hit  host int32 or NULL.   Errors: as tb_graph_compile.
  * tb_cache_stats: any pointer may be NULL.
  */
@@ -247,8 +250,8 @@ void tb_batch_destroy(tb_batch *b);
  * Attach graph g to `slot`, or detach with g == NULL (model id -1: zero bonus, state -1;
  * Sec. 2.2 para. 3).  Adding and removing lists while other streams keep running is Sec. 2.2
  * para. 4; here the slot index is the stable id, and no other slot's graph moves or changes.
- * The graph is copied through pinned host memory with an asynchronous host-to-device copy
- * on `stream`; the slot's offsets are published and its streaming state is reset (state =
+ * The graph is copied with an asynchronous host-to-device copy on `stream` (from its own page-locked blob, or
+ * through page-locked staging memory of the batch when its blob is on the heap); the slot's offsets are published and its streaming state is reset (state =
  * root or -1, frame cursor 0, score 0) in stream order.  The previous graph's arena space is
  * reused by later binds.  g must have been compiled with the batch's vocab and class map.
  * Ordering: the previous graph's arena block goes back to the free list when this call returns, and a later bind
@@ -262,8 +265,9 @@ int tb_batch_bind_stream(tb_batch *b, int32_t slot, const tb_graph *g, void *str
 
 /*
  * tb_batch_bind_stream for n slots at once (Sec. 2.2 para. 4: between two chunks several streams end and start): the
- * graphs are packed into one arena block and travel, with their slot records, in ONE host-to-device copy (graphs kept
- * by a tb_cache are page-locked and go in one copy each, straight from where they are) followed by one small launch.  graphs[i] == NULL
+ * graphs are packed into one arena block; heap-held graphs travel, with all slot records, in ONE host-to-device copy,
+ * page-locked graphs straight from where they are (one copy per run of graphs that are neighbours in the pool, which
+ * graphs compiled one after the other usually are), followed by one small launch.  graphs[i] == NULL
  * unbinds slots[i].  A slot may appear once.  Everything is checked before anything changes.  A group of more than
  * 4 MB of graphs goes in parts of that size, and when the arena has no contiguous room for a part its slots are
  * bound one by one (an error then leaves the earlier ones bound).

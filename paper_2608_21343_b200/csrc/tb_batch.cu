@@ -3,7 +3,10 @@
 // asynchronous host-to-device copies through pinned staging, and the C-ABI entry points that
 // validate arguments and launch the decode kernels.
 #include <cstring>
+#include <atomic>
+#include <iterator>
 #include <map>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -70,14 +73,99 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 }  // namespace
 
 tb_graph::~tb_graph() {
-  if (pinned) { cudaHostUnregister(blob.data()); cudaGetLastError(); }
+  if (registered) { cudaHostUnregister(blob.data()); cudaGetLastError(); }
 }
 
 void tb_graph_pin(tb_graph* g) {
   if (!g || g->pinned || g->blob.empty()) return;
   // (portable: whichever device's batch binds the graph later may copy from it)
-  if (cudaHostRegister(g->blob.data(), g->blob.size(), cudaHostRegisterPortable) == cudaSuccess) g->pinned = true;
+  if (cudaHostRegister(g->blob.data(), g->blob.size(), cudaHostRegisterPortable) == cudaSuccess) g->pinned = g->registered = true;
   else cudaGetLastError();
+}
+
+// ---- the pool of page-locked memory for graph images (see tb_internal.h) ---------------------------------------
+namespace {
+constexpr size_t kPoolChunk = static_cast<size_t>(32) << 20;     // allocated from the driver in pieces of this size
+constexpr size_t kPoolMax = static_cast<size_t>(1) << 30;        // the pool never takes more than this
+constexpr size_t kPoolLargest = static_cast<size_t>(16) << 20;   // larger images stay on the heap
+struct PinnedPool {
+  std::mutex mu;
+  struct Chunk {
+    unsigned char* base;
+    size_t bytes;
+    std::map<size_t, size_t> free_blocks;                          // offset -> bytes, neighbours coalesced
+  };
+  std::vector<Chunk> chunks;
+  size_t total = 0;
+  std::atomic<bool> armed{false};
+  bool closed = false;                                             // the driver refused a chunk: no further attempts
+};
+PinnedPool& pinned_pool() {
+  static PinnedPool* pool = new PinnedPool();                      // (never destroyed: graphs may be freed during exit)
+  return *pool;
+}
+}  // namespace
+
+void tb_pinned_pool_arm() { pinned_pool().armed.store(true); }
+
+void* tb_pinned_alloc(size_t bytes) {
+  PinnedPool& pool = pinned_pool();
+  if (!pool.armed.load() || bytes == 0 || bytes > kPoolLargest) return nullptr;
+  const size_t want = round_up(bytes, kArenaAlign);
+  std::lock_guard<std::mutex> lock(pool.mu);
+  for (int pass = 0; pass < 2; ++pass) {
+    for (auto& c : pool.chunks)
+      for (auto it = c.free_blocks.begin(); it != c.free_blocks.end(); ++it) {
+        if (it->second < want) continue;
+        const size_t off = it->first, rest = it->second - want;
+        c.free_blocks.erase(it);
+        if (rest) c.free_blocks[off + want] = rest;
+        return c.base + off;
+      }
+    if (pass == 1 || pool.closed || pool.total + kPoolChunk > kPoolMax) return nullptr;
+    void* base = nullptr;
+    if (cudaHostAlloc(&base, kPoolChunk, cudaHostAllocPortable) != cudaSuccess) {
+      cudaGetLastError();
+      pool.closed = true;
+      return nullptr;
+    }
+    PinnedPool::Chunk c;
+    c.base = static_cast<unsigned char*>(base); c.bytes = kPoolChunk;
+    c.free_blocks[0] = kPoolChunk;
+    pool.chunks.push_back(std::move(c));
+    pool.total += kPoolChunk;
+  }
+  return nullptr;
+}
+
+bool tb_pinned_owns(const void* p) {
+  PinnedPool& pool = pinned_pool();
+  if (!pool.armed.load() || !p) return false;
+  std::lock_guard<std::mutex> lock(pool.mu);
+  const unsigned char* q = static_cast<const unsigned char*>(p);
+  for (auto& c : pool.chunks)
+    if (q >= c.base && q < c.base + c.bytes) return true;
+  return false;
+}
+
+bool tb_pinned_free(void* p, size_t bytes) {
+  PinnedPool& pool = pinned_pool();
+  if (!pool.armed.load() || !p) return false;
+  std::lock_guard<std::mutex> lock(pool.mu);
+  unsigned char* q = static_cast<unsigned char*>(p);
+  for (auto& c : pool.chunks) {
+    if (q < c.base || q >= c.base + c.bytes) continue;
+    size_t off = static_cast<size_t>(q - c.base), n = round_up(bytes, kArenaAlign);
+    auto next = c.free_blocks.lower_bound(off);
+    if (next != c.free_blocks.begin()) {
+      auto prev = std::prev(next);
+      if (prev->first + prev->second == off) { off = prev->first; n += prev->second; c.free_blocks.erase(prev); }
+    }
+    if (next != c.free_blocks.end() && off + n == next->first) { n += next->second; c.free_blocks.erase(next); }
+    c.free_blocks[off] = n;
+    return true;
+  }
+  return false;
 }
 
 struct tb_batch {
@@ -202,6 +290,7 @@ extern "C" int tb_batch_create(int32_t vocab, const int32_t* case_class, int32_t
   ok = ok && cudaMemset(b->d_status, 0, sizeof(int32_t)) == cudaSuccess;
   for (auto& s : b->staging) ok = ok && cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) { cudaGetLastError(); destroy_batch(b); return TB_ERR_CUDA; }
+  tb_pinned_pool_arm();   // from now on this process keeps the images of the graphs it compiles in page-locked memory
   *out = b;
   return TB_OK;
 }
@@ -370,14 +459,29 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   int32_t* slot_of = reinterpret_cast<int32_t*>(s.host + tail_off + static_cast<size_t>(n) * sizeof(TbSlotRec));
   std::vector<std::pair<size_t, size_t>> blocks(static_cast<size_t>(n), {0, 0});
   size_t at = 0;
+  // page-locked images that lie next to each other in host memory (graphs compiled one after the other sit side by
+  // side in the pool, at the spacing the arena uses) travel in one copy
+  const unsigned char* run_src = nullptr;
+  size_t run_at = 0, run_span = 0, run_bytes = 0;
+  auto flush_run = [&]() {
+    if (run_src) ok = ok && cudaMemcpyAsync(b->arena + base + run_at, run_src, run_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    run_src = nullptr;
+  };
   for (int32_t i = 0; i < n; ++i) {
     const tb_graph* g = graphs[i];
     slot_of[i] = slots[i];
     if (!g) { std::memset(&recs[i], 0, sizeof(TbSlotRec)); continue; }
     if (g->pinned) {
-      ok = ok && cudaMemcpyAsync(b->arena + base + at, g->blob.data(), g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
-      if (ok) { tb_graph* h = const_cast<tb_graph*>(g); h->refs.fetch_add(1); s.held_more.push_back(h); }
+      if (!(run_src && !g->registered && g->blob.data() == run_src + run_span && at == run_at + run_span)) {
+        flush_run();
+        run_src = g->blob.data(); run_at = at; run_span = 0;
+      }
+      run_bytes = run_span + g->blob.size();
+      run_span += round_up(g->blob.size(), kArenaAlign);
+      if (g->registered) flush_run();                                  // (registered memory ends with the image)
+      tb_graph* h = const_cast<tb_graph*>(g); h->refs.fetch_add(1); s.held_more.push_back(h);
     } else {
+      flush_run();
       std::memcpy(s.host + at, g->blob.data(), g->blob.size());
       if (any_pinned)   // (a mixed group: every staged graph is its own copy)
         ok = ok && cudaMemcpyAsync(b->arena + base + at, s.host + at, g->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
@@ -386,6 +490,7 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
     blocks[i] = {base + at, round_up(g->blob.size(), kArenaAlign)};
     at += blocks[i].second;
   }
+  flush_run();
   if (any_pinned) ok = ok && cudaMemcpyAsync(b->arena + base + tail_off, s.host + tail_off, tail, cudaMemcpyHostToDevice, stream) == cudaSuccess;
   else ok = ok && cudaMemcpyAsync(b->arena + base, s.host, total + tail, cudaMemcpyHostToDevice, stream) == cudaSuccess;   // graphs and records in one copy
   ok = ok && cudaEventRecord(s.done, stream) == cudaSuccess;

@@ -47,12 +47,13 @@ struct FileHeader {
   uint64_t payload_hash;   // of the header (this field taken as zero) followed by everything after it
 };
 
-template <typename T>
-void put(std::string& out, const std::vector<T>& v) {
-  out.append(reinterpret_cast<const char*>(v.data()), v.size() * sizeof(T));
+template <typename Vec>
+void put(std::string& out, const Vec& v) {
+  out.append(reinterpret_cast<const char*>(v.data()), v.size() * sizeof(typename Vec::value_type));
 }
-template <typename T>
-bool take(const unsigned char*& p, const unsigned char* end, std::vector<T>& v, size_t n) {
+template <typename Vec>
+bool take(const unsigned char*& p, const unsigned char* end, Vec& v, size_t n) {
+  using T = typename Vec::value_type;
   if (static_cast<size_t>(end - p) < n * sizeof(T)) return false;
   v.resize(n);
   if (n) std::memcpy(v.data(), p, n * sizeof(T));
@@ -205,6 +206,7 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
       if (!in) { delete g; return TB_ERR_INVALID_ARG; }
     }
     if (g->class_map_hash != tb_hash_class_map(g->case_class.data(), g->vocab)) { delete g; return TB_ERR_INVALID_ARG; }
+    g->pinned = tb_pinned_owns(g->blob.data());
     *out = g;
     return TB_OK;
   } catch (const std::bad_alloc&) {

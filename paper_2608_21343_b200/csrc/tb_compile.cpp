@@ -67,14 +67,14 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
   g->class_map_hash = tb_hash_class_map(case_class, vocab);
 
   // ---- device blob ---------------------------------------------------------------------------
-  g->blob.clear();
-  g->off_arc_begin = append_section(g->blob, g->state_arc_begin);
-  g->off_fail = append_section(g->blob, g->state_fail);
-  g->off_bw = append_section(g->blob, g->state_bw);
-  g->off_arc_cls = append_section(g->blob, g->arc_class);
-  g->off_arc_w = append_section(g->blob, g->arc_w);
-  g->off_arc_dst = append_section(g->blob, g->arc_dst);
-  g->off_final = append_section(g->blob, g->state_final);
+  std::vector<unsigned char> blob;   // built here, then moved into its final place in one piece
+  g->off_arc_begin = append_section(blob, g->state_arc_begin);
+  g->off_fail = append_section(blob, g->state_fail);
+  g->off_bw = append_section(blob, g->state_bw);
+  g->off_arc_cls = append_section(blob, g->arc_class);
+  g->off_arc_w = append_section(blob, g->arc_w);
+  g->off_arc_dst = append_section(blob, g->arc_dst);
+  g->off_final = append_section(blob, g->state_final);
   {  // per-state records and token-expanded arcs (tokens of a class in ascending id order)
     std::vector<int32_t> ctb(n_classes + 1, 0), ctk(vocab);
     for (int32_t v = 0; v < vocab; ++v) ctb[g->case_class[v] + 1]++;
@@ -94,8 +94,8 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
       recs[u].fail = g->state_fail[u];
       recs[u].bw = g->state_bw[u];
     }
-    g->off_strec = append_section(g->blob, recs);
-    g->off_tokent = append_section(g->blob, ents);
+    g->off_strec = append_section(blob, recs);
+    g->off_tokent = append_section(blob, ents);
     g->n_tokent = static_cast<int32_t>(ents.size());
 
     // resolved lists (see TbRsRec): the walk the kernels would do, done once here in float
@@ -138,15 +138,18 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
       rrecs[s].bmag = std::fabs(lambda) * (std::fabs(acc) + root_w_max);
     }
     if (fits) {
-      g->off_rsrec = append_section(g->blob, rrecs);
-      g->off_rsent = append_section(g->blob, rents);
+      g->off_rsrec = append_section(blob, rrecs);
+      g->off_rsent = append_section(blob, rents);
       g->n_rsent = static_cast<int32_t>(rents.size());
     } else {
       g->off_rsrec = g->off_rsent = 0;
       g->n_rsent = -1;
     }
   }
-  g->blob.resize(align16(g->blob.size()) + 16);  // tail padding so vector loads may overrun a section
+  blob.resize(align16(blob.size()) + 16);  // tail padding so vector loads may overrun a section
+  g->blob = TbImage();
+  g->blob.assign(blob.begin(), blob.end());
+  g->pinned = tb_pinned_owns(g->blob.data());
 }
 
 static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,

@@ -9,6 +9,34 @@
 
 #include "tb.h"
 
+// Page-locked host memory for graph images.  A process that decodes (one that has created a batch) keeps the device
+// image of every graph it compiles or loads in one pool of page-locked memory, so that a bind is a plain
+// host-to-device copy from where the image already is: no staging copy on the path between "a stream starts" and
+// "its first chunk is decoded".  Before the first batch exists (a process that only compiles), when the pool is full,
+// or without a device, the image lives on the heap and binds go through the batch's staging ring.
+void tb_pinned_pool_arm();                       // called when a batch has been created
+void* tb_pinned_alloc(size_t bytes);             // nullptr: not from the pool (use the heap)
+bool tb_pinned_free(void* p, size_t bytes);      // false: p is not the pool's
+bool tb_pinned_owns(const void* p);
+
+template <typename T>
+struct TbImageAlloc {
+  using value_type = T;
+  TbImageAlloc() = default;
+  template <typename U> TbImageAlloc(const TbImageAlloc<U>&) {}
+  T* allocate(size_t n) {
+    void* p = tb_pinned_alloc(n * sizeof(T));
+    if (!p) p = ::operator new(n * sizeof(T));
+    return static_cast<T*>(p);
+  }
+  void deallocate(T* p, size_t n) {
+    if (!tb_pinned_free(p, n * sizeof(T))) ::operator delete(p);
+  }
+  template <typename U> bool operator==(const TbImageAlloc<U>&) const { return true; }
+  template <typename U> bool operator!=(const TbImageAlloc<U>&) const { return false; }
+};
+using TbImage = std::vector<unsigned char, TbImageAlloc<unsigned char>>;
+
 // A compiled graph: the canonical flat arrays (what tb_graph_view exposes) plus the
 // position-independent byte blob that is copied into the device arena.
 struct tb_graph {
@@ -19,19 +47,21 @@ struct tb_graph {
   std::vector<uint8_t> state_depth;
   uint64_t class_map_hash = 0;  // to reject a bind against a batch with another class map
   // Device blob: sections at 16-byte aligned offsets, all ids graph-local.
-  std::vector<unsigned char> blob;
+  TbImage blob;                                        // (allocated once, at its final size: see TbImageAlloc)
   int32_t off_arc_begin = 0, off_fail = 0, off_bw = 0, off_arc_cls = 0, off_arc_w = 0, off_arc_dst = 0;
   int32_t off_final = 0;                               // state_final as a blob section (end-of-stream weights)
   int32_t off_strec = 0, off_tokent = 0, n_tokent = 0;
   int32_t off_rsrec = 0, off_rsent = 0, n_rsent = 0;  // resolved per-state lists (n_rsent < 0: not built)
   float d_max = 0.0f;                                  // largest |sum of suffix-link weights| over all states
   std::atomic<int32_t> refs{1};                        // holders: the caller's handle, one per cache that keeps the graph, one per copy in flight
-  bool pinned = false;                                 // the blob's pages are locked (tb_graph_pin): binds copy straight from it
+  bool pinned = false;                                 // the blob's pages are locked (it sits in the pool, or tb_graph_pin registered it): binds copy straight from it
+  bool registered = false;                             // ... by tb_graph_pin: to be unregistered
   ~tb_graph();
 };
 
-// Page-locks the blob of a graph that will be bound again and again (graphs kept by a cache), so that a bind can
-// hand it to the copy engine directly instead of going through the staging ring.  Does nothing without a device.
+// Page-locks the blob of a graph that will be bound again and again (graphs kept by a cache) if it is not in the
+// page-locked pool already, so that a bind can hand it to the copy engine directly instead of going through the
+// staging ring.  Does nothing without a device.
 void tb_graph_pin(tb_graph* g);
 
 // Two derived sections of the blob serve the pipelined kernel.  TbStateRec packs what a
