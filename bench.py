@@ -36,10 +36,14 @@ from paper_2608_21343_b200 import workloads as W  # noqa: E402
 
 METRIC = "boosted_greedy_decode_frames_per_s_B128"
 UNIT = "frames/s"
-# DRAM read + write bytes per logits row of the decode kernel, from an ncu capture of a 32-stream launch
-# (160.2 MB for 72000 rows: each stream's second segment re-reads 16 warm-up frames, and what it emits goes
-# through scratch memory); the kernel runs one block per stream, so traffic scales with the stream count.
-NCU_DRAM_BYTES_PER_ROW = 2233.0
+# DRAM read + write bytes per logits row of k_greedy_fast, from an ncu capture of one 32-stream launch
+# (155.37 MB read + 5.68 MB written for 72000 rows: each stream's second segment re-reads 16 warm-up frames, and
+# what it emits goes through scratch memory); the kernel runs one block per stream, so traffic scales with the
+# stream count.  Captured with the command recorded in profiles/greedy_fast_small_case_B32_counters.md
+# (`python bench.py --streams 32 --steps 2 --warmup 3 --no-extras --one-block-per-stream` under
+# `ncu --clock-control none -k regex:k_greedy_fast -s 4 -c 1 ...`) on the kernel as of the commit that split its
+# row-summary code into tb_fast_common.cuh; to be re-captured whenever tb_greedy_fast.cu or that header changes.
+NCU_DRAM_BYTES_PER_ROW = 2237.0
 
 
 def load_peaks():
@@ -484,6 +488,8 @@ def main():
     ap.add_argument("--frames", type=int, default=0, help="override T (profiling captures use a small case)")
     ap.add_argument("--single-binds", action="store_true", help="workload 5: bind new streams one by one instead of in one call")
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
+    ap.add_argument("--one-block-per-stream", action="store_true",
+                    help="never the segmented kernel (small-case captures of k_greedy_fast: fewer streams would otherwise select it)")
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7, 8],
                     help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists, 7 model lifecycle sweep: side measurements")
     args = ap.parse_args()
@@ -529,9 +535,16 @@ def main():
     for i, g in enumerate(graphs):
         tb.tb_batch_bind_stream(batch, i, g)
     plain = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=1 << 20, device=local_rank)  # all unbound
+    if args.one_block_per_stream:
+        tb.tb_batch_set_flags(batch, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
+        tb.tb_batch_set_flags(plain, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
     out = tb.tb_greedy_decode(batch, logits)
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
+    ran = tb.tb_batch_last_greedy_kernel(batch)       # which kernel the library chose for this shape
+    kernel_name = {tb.TB_KERNEL_PIPELINED: "k_greedy_fast", tb.TB_KERNEL_SEGMENTED: "k_greedy_seg",
+                   tb.TB_KERNEL_GENERAL: "k_decode_general"}[ran["kernel"]]
+    fast = ran["kernel"] == tb.TB_KERNEL_PIPELINED
 
     def barrier():
         torch.cuda.synchronize()
@@ -593,13 +606,14 @@ def main():
         "gpu_launches": args.steps * 1,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S,
-                     "traffic_note": "ncu dram read+write of a 32-stream launch scaled by streams",
-                     "peak_kind": f"of {peak_kind}", "kernel": "k_greedy_fast (one launch per decode)",
+                     "traffic": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S if fast else None,
+                     "traffic_note": "ncu dram read+write of a 32-stream launch scaled by streams" if fast else "captured for k_greedy_fast only",
+                     "peak_kind": f"of {peak_kind}",
+                     "kernel": f"{kernel_name} (one launch per decode; {ran['blocks_per_stream']} block(s) per stream)",
                      "rows_visited": visited, "bytes_per_row": row_bytes,
                      "all_rows_GBs": streamed, "all_rows_frac": streamed / peak,
-                     "measured_GBs": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S / (kern_ms * 1e-3) / 1e9,
-                     "measured_frac": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S / (kern_ms * 1e-3) / 1e9 / peak,
+                     "measured_GBs": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S / (kern_ms * 1e-3) / 1e9 if fast else None,
+                     "measured_frac": NCU_DRAM_BYTES_PER_ROW * w.B * w.T * w.S / (kern_ms * 1e-3) / 1e9 / peak if fast else None,
                      "frac_of_nominal_8000": achieved / 8000.0},
         "ms_per_step_median": float(np.median(each_ms)), "ms_per_step_min": float(np.min(each_ms)),
         "ns_per_visited_row_per_stream": kern_ms * 1e6 / (visited / w.B),

@@ -106,7 +106,14 @@ PinnedPool& pinned_pool() {
 }
 }  // namespace
 
-void tb_pinned_pool_arm() { pinned_pool().armed.store(true); }
+void tb_pinned_pool_arm() {
+  PinnedPool& pool = pinned_pool();
+  if (pool.armed.exchange(true)) return;
+  // the first piece is taken now (page-locking 32 MB takes tens of milliseconds, which belongs to start-up and not
+  // to the first compile after it)
+  void* p = tb_pinned_alloc(kArenaAlign);
+  if (p) tb_pinned_free(p, kArenaAlign);
+}
 
 void* tb_pinned_alloc(size_t bytes) {
   PinnedPool& pool = pinned_pool();
