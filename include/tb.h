@@ -61,6 +61,11 @@ extern "C" {
 #define TB_FRAME_NEW 1        /* first row of a frame: every hypothesis with a score becomes live */
 #define TB_FRAME_NEW_MERGE 2  /* as TB_FRAME_NEW, after hypotheses with equal token sequences were merged */
 
+/* tb_graph_compile, tb_graph_compile_variative, tb_cache_compile(_variative): flags */
+#define TB_COMPILE_PAGEABLE 1           /* keep the graph's device blob in ordinary host memory even when the process has its pool of
+                                           page-locked memory (see tb_cache_compile): for lists compiled in bulk and seldom bound; a
+                                           bind then stages the blob through page-locked memory of the batch */
+
 /* tb_batch_set_flags */
 #define TB_FLAG_GENERAL_KERNELS 1       /* always use the general decode kernel (any layout), never a pipelined one */
 #define TB_FLAG_ONE_BLOCK_PER_STREAM 2  /* pipelined greedy decode: never the segmented kernel, one block per stream */
@@ -127,7 +132,7 @@ const char *tb_strerror(int code);
  *   case_class     host int32 [vocab] or NULL (= identity, case-sensitive): tokens with the
  *                  same class are case variants of each other; classes are >= 0
  *   lambda         boosting weight of this list (Sec. 2.2 para. 2), finite
- *   flags          must be 0
+ *   flags          0, or TB_COMPILE_PAGEABLE
  *   out            receives the graph; free it with tb_graph_free
  * Empty phrases are skipped.  Errors: TB_ERR_INVALID_ARG (token outside [0, vocab), bad
  * weight or class, phrase longer than TB_MAX_PHRASE_LEN, vocab outside [1, TB_MAX_VOCAB]),

@@ -25,6 +25,7 @@ TB_ERR_INVALID_ARG, TB_ERR_OOM, TB_ERR_CUDA, TB_ERR_ARENA_FULL, TB_ERR_BAD_SLOT,
 TB_ERR_IO = -7
 TB_FRAME_SAME, TB_FRAME_NEW, TB_FRAME_NEW_MERGE = 0, 1, 2
 TB_BF16, TB_F32 = 0, 1
+TB_COMPILE_PAGEABLE = 1
 
 
 class TbError(RuntimeError):

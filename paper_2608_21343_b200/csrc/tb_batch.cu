@@ -100,11 +100,14 @@ struct PinnedPool {
   std::atomic<bool> armed{false};
   bool closed = false;                                             // the driver refused a chunk: no further attempts
 };
+thread_local bool g_pool_bypass = false;
 PinnedPool& pinned_pool() {
   static PinnedPool* pool = new PinnedPool();                      // (never destroyed: graphs may be freed during exit)
   return *pool;
 }
 }  // namespace
+
+void tb_pinned_bypass(bool on) { g_pool_bypass = on; }
 
 void tb_pinned_pool_arm() {
   PinnedPool& pool = pinned_pool();
@@ -117,7 +120,7 @@ void tb_pinned_pool_arm() {
 
 void* tb_pinned_alloc(size_t bytes) {
   PinnedPool& pool = pinned_pool();
-  if (!pool.armed.load() || bytes == 0 || bytes > kPoolLargest) return nullptr;
+  if (!pool.armed.load() || g_pool_bypass || bytes == 0 || bytes > kPoolLargest) return nullptr;
   const size_t want = round_up(bytes, kArenaAlign);
   std::lock_guard<std::mutex> lock(pool.mu);
   for (int pass = 0; pass < 2; ++pass) {

@@ -58,6 +58,13 @@ extern "C" const char* tb_strerror(int code) {
   }
 }
 
+// TB_COMPILE_PAGEABLE: while one of these lives, this thread's images go to the heap.
+struct PoolBypass {
+  bool on;
+  explicit PoolBypass(bool o) : on(o) { if (on) tb_pinned_bypass(true); }
+  ~PoolBypass() { if (on) tb_pinned_bypass(false); }
+};
+
 // What every front end shares: from the flat arc / state arrays to the device blob (Sec. 2.2 para. 2), with the
 // per-state records, token-expanded arcs and resolved lists the kernels read.
 static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab, int32_t n_classes, float lambda) {
@@ -297,7 +304,8 @@ extern "C" int tb_graph_compile(const int32_t* phrase_tokens, const int64_t* phr
                                 float lambda, uint32_t flags, tb_graph** out) {
   if (!out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
-  if (flags != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda)) return TB_ERR_INVALID_ARG;
+  if ((flags & ~static_cast<uint32_t>(TB_COMPILE_PAGEABLE)) != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda)) return TB_ERR_INVALID_ARG;
+  PoolBypass bypass((flags & TB_COMPILE_PAGEABLE) != 0);
   if (n_phrases > 0 && (!phrase_offsets || (phrase_offsets[n_phrases] > 0 && !phrase_tokens))) return TB_ERR_INVALID_ARG;
   try {
     tb_graph* g = new tb_graph();
@@ -532,9 +540,10 @@ extern "C" int tb_graph_compile_variative(const uint8_t* phrase_chars, const int
                                           uint32_t flags, tb_graph** out) {
   if (!out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
-  if (flags != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda) ||
+  if ((flags & ~static_cast<uint32_t>(TB_COMPILE_PAGEABLE)) != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda) ||
       !std::isfinite(tau) || tau < 0.0f)
     return TB_ERR_INVALID_ARG;
+  PoolBypass bypass((flags & TB_COMPILE_PAGEABLE) != 0);
   if (n_phrases > 0 && (!phrase_offsets || (phrase_offsets[n_phrases] > 0 && !phrase_chars))) return TB_ERR_INVALID_ARG;
   try {
     tb_graph* g = new tb_graph();

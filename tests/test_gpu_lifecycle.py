@@ -279,3 +279,53 @@ def test_binding_many_streams_at_once(tb):
     for i in range(5):
         check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]), "small arena")
     assert tb.tb_batch_status(batch) == 0 and tb.tb_batch_status(small) == 0
+
+
+def test_graph_images_in_page_locked_memory_and_on_the_heap(tb):
+    """Once a batch exists, compiled and loaded graphs keep their device image in the library's pool of page-locked
+    memory and binds copy from there; TB_COMPILE_PAGEABLE keeps an image on the heap, and binds stage it.  Both kinds,
+    mixed in one group and one by one, must decode the same; images are released and their room is reused; more
+    images than one piece of the pool holds spill into further pieces."""
+    w = W.get_workload(2, B=8, T=100, n_phrases=40, n_plants=6)
+    data = W.batch_inputs(w)
+    logits = to_device(data["logits"])
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=8 << 20)
+    refs = [O.greedy_rnnt(oracle_graph(w, data["phrases"][i]), data["logits"][i]) for i in range(w.B)]
+
+    def graphs(kind):
+        return [tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class,
+                                    flags=tb.TB_COMPILE_PAGEABLE if (kind == "heap" or (kind == "mixed" and i % 3 == 1)) else 0)
+                for i, p in enumerate(data["phrases"])]
+    for kind in ("pool", "heap", "mixed"):
+        for grouped in (True, False):
+            gs = graphs(kind)
+            tb.tb_batch_bind_streams(batch, list(range(w.B)), [None] * w.B)
+            if grouped:
+                tb.tb_batch_bind_streams(batch, list(range(w.B)), gs)
+            else:
+                for i, g in enumerate(gs):
+                    tb.tb_batch_bind_stream(batch, i, g)
+            del gs                                           # the copies in flight hold the graphs they read
+            out = to_host(tb.tb_greedy_decode(batch, logits))
+            for i in range(w.B):
+                check_greedy(out, i, refs[i], f"{kind}, grouped={grouped}")
+    # a long series of lists of different sizes, kept alive in a window: images come and go, room is reused, and the
+    # total (about 60 MB alive at the peak) needs more than one 32 MB piece
+    wl = W.get_workload(5, B=4)
+    big = tb.tb_batch_create(wl.V, wl.vocab.case_class, 4, arena_bytes=16 << 20)
+    alive = []
+    for r in range(700):
+        g = tb.tb_graph_compile(W.stream_phrases(wl, r % 97), wl.V, case_class=wl.vocab.case_class)
+        alive.append(g)
+        if len(alive) > 450:
+            del alive[:200]
+        if r % 50 == 49:
+            tb.tb_batch_bind_streams(big, [0, 1, 2, 3], alive[-4:])
+    torch.cuda.synchronize()
+    assert tb.tb_batch_status(big) == 0
+    # what was bound last decodes as its list says (no image was overwritten by a later one)
+    lists = [W.stream_phrases(wl, r % 97) for r in range(696, 700)]
+    x = np.stack([np.ascontiguousarray(W.stream_inputs(wl, i)["logits"][:60, :, : wl.V + 1]) for i in range(4)])
+    out = to_host(tb.tb_greedy_decode(big, to_device(x)))
+    for i in range(4):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(wl, lists[i]), x[i]), "after many images")

@@ -85,7 +85,8 @@ def test_compile_error_codes(tb):
     assert code([[0, 1]], 0) == tb.TB_ERR_INVALID_ARG
     assert code([[0, 1]], 100000) == tb.TB_ERR_INVALID_ARG
     assert code([[0] * 300], 4) == tb.TB_ERR_INVALID_ARG
-    assert code([[0, 1]], 4, flags=1) == tb.TB_ERR_INVALID_ARG
+    assert code([[0, 1]], 4, flags=2) == tb.TB_ERR_INVALID_ARG
+    tb.tb_graph_compile([[0, 1]], 4, flags=tb.TB_COMPILE_PAGEABLE)       # the one flag there is
     g = tb.tb_graph_compile([], 4).view()
     assert g["n_states"] == 1 and g["n_arcs"] == 0
 
@@ -142,7 +143,7 @@ def test_variative_compile_error_codes(tb):
     assert code([b"a" * 256], pieces) == tb.TB_ERR_INVALID_ARG
     assert code([b"ab"], pieces + [b""]) == tb.TB_ERR_INVALID_ARG             # an empty piece
     assert code([b"ab"], pieces + [b"a" * 33]) == tb.TB_ERR_INVALID_ARG       # a piece longer than TB_MAX_PIECE_LEN
-    assert code([b"ab"], pieces, flags=1) == tb.TB_ERR_INVALID_ARG
+    assert code([b"ab"], pieces, flags=2) == tb.TB_ERR_INVALID_ARG
     g = tb.tb_graph_compile_variative([], pieces).view()
     assert g["n_states"] == 1 and g["n_arcs"] == 0
     g = tb.tb_graph_compile_variative([b"AB"], pieces, tau=0.0).view()      # the hand-worked list, given in upper case
