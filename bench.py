@@ -309,6 +309,7 @@ def side_measurement(args):
             live = torch.zeros((w.B, K), dtype=torch.uint8, device=dev)
             par = torch.empty((w.B, K), dtype=torch.int32, device=dev)
             tok = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+            bt = (torch.zeros((w.B, K, 256), dtype=torch.int32, device=dev), torch.zeros((w.B, K), dtype=torch.int32, device=dev))
             tb.tb_beam_reset_slots(batch)
             served = np.zeros(w.B, dtype=np.int64)
             total = np.zeros(w.B, dtype=np.int64)
@@ -325,16 +326,11 @@ def side_measurement(args):
                 dn = torch.from_numpy(left).to(dev)
                 bufs = (bufs + [dl])[-8:]
                 new = [sl for sl, _ in gs]
-                idx = torch.tensor(new, device=dev, dtype=torch.long) if new else None
                 torch.cuda.synchronize()
                 a, m0, m1, b = (torch.cuda.Event(enable_timing=True) for _ in range(4))
                 a.record()
-                tb.tb_batch_bind_streams(batch, [sl for sl, _ in gs], [g for _, g in gs])
-                if new:
-                    scores[idx] = float("-inf"); scores[idx, 0] = 0.0
-                    states[idx] = -1; states[idx, 0] = 0
-                    live[idx] = 0
-                    tb.tb_beam_reset_slots(batch, new)
+                tb.tb_batch_bind_streams(batch, new, [g for _, g in gs])
+                tb.tb_beam_start_slots(batch, new, scores, states, live)     # the new slots' beams, set up by the library
                 m0.record()
                 tb.tb_beam_chunk(batch, dl, True, dn, scores, states, live, par, tok)
                 m1.record()
@@ -342,7 +338,7 @@ def side_measurement(args):
                 ended = [sl for sl in range(w.B) if left[sl] > 0 and served[sl] >= total[sl]]
                 if ended:
                     tb.tb_apply_final_weights_slots(batch, ended, scores, states)
-                    tb.tb_beam_backtrace_slots(batch, w.B, K, 256)
+                    tb.tb_beam_backtrace_slots(batch, w.B, K, 256, out=bt)
                 b.record()
                 torch.cuda.synchronize()
                 lat.append(a.elapsed_time(b)); kern.append(m0.elapsed_time(m1))

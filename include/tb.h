@@ -464,6 +464,10 @@ int tb_beam_frames(tb_batch *b, const void *logits, int dtype, int32_t B, int32_
  *
  * tb_beam_reset_slots: n = 0 resets every slot; else `slots` is a host int32 array of n slot indices.  Device work
  *   on `stream` (position 0, empty token sequences).  Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG, TB_ERR_CUDA.
+ * tb_beam_start_slots: tb_beam_reset_slots, which in the same launch also sets up those slots' rows of the caller's
+ *   device arrays scores / states / live [n_slots, K] for an utterance's first step: hypothesis 0 with score 0 in state 0
+ *   (state -1 on a slot without a graph, so call it after the slot's bind, on the same stream), the others with score
+ *   -inf and state -1, live 0.  Errors: as tb_beam_reset_slots; TB_ERR_INVALID_ARG for K outside [1, max_beam].
  * tb_beam_chunk: for slot i, n_frames[i] (device int32 [n_slots], clamped to [0, chunk]; NULL: chunk) frames of E
  *   expansions, exactly as tb_beam_frames does them for a whole batch (every hypothesis of slot i reads the row at
  *   element offset i*stream_stride + t*frame_stride + e*row_stride; merge and pruning at frame starts); a slot with
@@ -475,6 +479,8 @@ int tb_beam_frames(tb_batch *b, const void *logits, int dtype, int32_t B, int32_
  *   int32 [n]) names.
  */
 int tb_beam_reset_slots(tb_batch *b, int32_t n, const int32_t *slots, void *stream);
+int tb_beam_start_slots(tb_batch *b, int32_t n, const int32_t *slots, int32_t K, float *scores, int32_t *states, uint8_t *live,
+                        void *stream);
 int tb_beam_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots, int32_t K, int32_t chunk, int32_t E,
                   int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge, const int32_t *n_frames,
                   float *scores, int32_t *states, uint8_t *live, int32_t *out_parent, int32_t *out_token, void *stream);

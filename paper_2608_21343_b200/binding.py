@@ -87,6 +87,7 @@ _SIGS = {
                                  _vp]),
     "tb_apply_final_weights": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp]),
     "tb_beam_reset_slots": (C.c_int, [_vp, _i32, _vp, _vp]),
+    "tb_beam_start_slots": (C.c_int, [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "tb_beam_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp]),
     "tb_beam_backtrace_slots": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
@@ -480,6 +481,15 @@ def tb_beam_reset_slots(batch: Batch, slots=None, stream=None):
         _check(_lib.tb_beam_reset_slots(batch.handle, len(sl), _hp(sl), _stream(stream)), "tb_beam_reset_slots")
 
 
+def tb_beam_start_slots(batch: Batch, slots, scores: torch.Tensor, states: torch.Tensor, live: torch.Tensor, stream=None):
+    """tb_beam_reset_slots that also sets up the slots' rows of scores / states / live [n_slots, K] (None: every slot)."""
+    sl = None if slots is None else _host(slots, np.int32)
+    if sl is not None and len(sl) == 0:
+        return
+    _check(_lib.tb_beam_start_slots(batch.handle, 0 if sl is None else len(sl), _hp(sl), scores.shape[1], _dp(scores),
+                                    _dp(states), _dp(live), _stream(stream)), "tb_beam_start_slots")
+
+
 def tb_beam_chunk(batch: Batch, logits: torch.Tensor, merge: bool, n_frames, scores: torch.Tensor, states: torch.Tensor,
                   live: torch.Tensor, out_parent: torch.Tensor, out_token: torch.Tensor, stream=None):
     """logits [n_slots, chunk, E, vocab+1]; n_frames: device int32 [n_slots] (frames of this chunk each slot decodes)."""
@@ -492,10 +502,17 @@ def tb_beam_chunk(batch: Batch, logits: torch.Tensor, merge: bool, n_frames, sco
                               _stream(stream)), "tb_beam_chunk")
 
 
-def tb_beam_backtrace_slots(batch: Batch, n_slots: int, K: int, max_len: int, stream=None):
+def tb_beam_backtrace_slots(batch: Batch, n_slots: int, K: int, max_len: int, stream=None, out=None):
+    """out: (tokens int32 [n_slots, K, max_len], lens int32 [n_slots, K]) to write into instead of new tensors."""
     dev = torch.device("cuda", batch.device)
-    toks = torch.zeros((n_slots, K, max_len), dtype=torch.int32, device=dev)
-    lens = torch.zeros((n_slots, K), dtype=torch.int32, device=dev)
+    if out is not None:
+        toks, lens = out
+        if tuple(toks.shape) != (n_slots, K, max_len) or tuple(lens.shape) != (n_slots, K) or toks.dtype != torch.int32 \
+                or lens.dtype != torch.int32 or not toks.is_contiguous() or not lens.is_contiguous():
+            raise ValueError("out must be contiguous int32 tensors [n_slots, K, max_len] and [n_slots, K]")
+    else:
+        toks = torch.zeros((n_slots, K, max_len), dtype=torch.int32, device=dev)
+        lens = torch.zeros((n_slots, K), dtype=torch.int32, device=dev)
     _check(_lib.tb_beam_backtrace_slots(batch.handle, n_slots, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
            "tb_beam_backtrace_slots")
     return toks, lens

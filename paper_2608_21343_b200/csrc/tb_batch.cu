@@ -909,7 +909,9 @@ extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_
 
 // ---- streaming beam decoding, slot by slot (Sec. 2.3) --------------------------------------------------------
 
-extern "C" int tb_beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots, void* stream_) {
+// tb_beam_reset_slots, and tb_beam_start_slots (which also sets up the slots' rows of the caller's arrays).
+static int beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots, int32_t K, float* scores, int32_t* states,
+                            uint8_t* live, void* stream_) {
   if (!b || n < 0 || (n > 0 && !slots)) return TB_ERR_INVALID_ARG;
   for (int32_t i = 0; i < n; ++i) if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
   DeviceGuard guard(b->device);
@@ -918,14 +920,26 @@ extern "C" int tb_beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots,
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (n == 0) {   // every slot
     b->chunk_K = 0;
-    return tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, b->n_slots, nullptr, 1, stream);
+    return tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, b->n_slots, nullptr, 1,
+                                      b->d_slots, K, scores, states, live, stream);
   }
   for (int32_t at = 0; at < n; at += TB_BIND_PAIRS) {
     const int32_t m = n - at < TB_BIND_PAIRS ? n - at : TB_BIND_PAIRS;
-    const int rc = tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, m, slots + at, 0, stream);
+    const int rc = tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, m, slots + at, 0,
+                                              b->d_slots, K, scores, states, live, stream);
     if (rc != TB_OK) return rc;
   }
   return TB_OK;
+}
+
+extern "C" int tb_beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots, void* stream_) {
+  return beam_reset_slots(b, n, slots, 0, nullptr, nullptr, nullptr, stream_);
+}
+
+extern "C" int tb_beam_start_slots(tb_batch* b, int32_t n, const int32_t* slots, int32_t K, float* scores, int32_t* states,
+                                   uint8_t* live, void* stream_) {
+  if (!b || !scores || !states || !live || K < 1 || K > b->max_beam) return TB_ERR_INVALID_ARG;
+  return beam_reset_slots(b, n, slots, K, scores, states, live, stream_);
 }
 
 extern "C" int tb_beam_chunk(tb_batch* b, const void* logits, int dtype, int32_t n_slots, int32_t K, int32_t chunk, int32_t E,

@@ -959,8 +959,11 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int
 
 struct SlotList { int32_t slot[TB_BIND_PAIRS]; };
 // A new utterance on some slots (or on all): position 0 in the slot's tree, every hypothesis' sequence empty.
+// With `scores` given, the slots' rows of the caller's [n_slots, K] arrays are set up as well: hypothesis 0 with score 0
+// in the root state (state -1 on an unbound slot), the others empty.
 __global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
-                                   int32_t n, SlotList sl, int32_t all_slots) {
+                                   int32_t n, SlotList sl, int32_t all_slots, const TbSlotRec* slots, int32_t K,
+                                   float* scores, int32_t* states, uint8_t* live) {
   const int i = blockIdx.x;
   if (i >= n) return;
   const int slot = all_slots ? i : sl.slot[i];
@@ -968,6 +971,15 @@ __global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, 
   for (int k = threadIdx.x; k < max_beam; k += blockDim.x) {
     const size_t o = static_cast<size_t>(slot) * max_beam + k;
     hash[o] = 0ull; hash[n_hyp + o] = 0ull; len[o] = 0; len[n_hyp + o] = 0;
+  }
+  if (scores) {
+    const bool bound = slots[slot].n_states > 0;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+      const size_t o = static_cast<size_t>(slot) * K + k;
+      scores[o] = k == 0 ? 0.0f : -INFINITY;
+      states[o] = (k == 0 && bound) ? 0 : -1;
+      live[o] = 0;
+    }
   }
 }
 
@@ -1213,11 +1225,12 @@ int tb_launch_beam_chunk(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t
 }
 
 int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
-                               int32_t n, const int32_t* slots, int32_t all_slots, cudaStream_t stream) {
+                               int32_t n, const int32_t* slots, int32_t all_slots, const TbSlotRec* slot_recs, int32_t K,
+                               float* scores, int32_t* states, uint8_t* live, cudaStream_t stream) {
   if (n < 1 || (!all_slots && n > TB_BIND_PAIRS)) return TB_ERR_INVALID_ARG;
   SlotList sl;
   for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = (!all_slots && i < n) ? slots[i] : 0;
-  k_beam_reset_slots<<<n, 32, 0, stream>>>(slot_pos, hash, len, n_hyp, max_beam, n, sl, all_slots);
+  k_beam_reset_slots<<<n, 32, 0, stream>>>(slot_pos, hash, len, n_hyp, max_beam, n, sl, all_slots, slot_recs, K, scores, states, live);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 

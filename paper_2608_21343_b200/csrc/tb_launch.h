@@ -87,7 +87,8 @@ int tb_launch_beam_chunk(const TbBeamParams& p, int32_t T, int32_t E, int64_t fr
                          const int32_t* n_frames, int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp,
                          cudaStream_t stream);
 int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
-                               int32_t n, const int32_t* slots, int32_t all_slots, cudaStream_t stream);
+                               int32_t n, const int32_t* slots, int32_t all_slots, const TbSlotRec* slot_recs, int32_t K,
+                               float* scores, int32_t* states, uint8_t* live, cudaStream_t stream);
 int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
                                    int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status,
                                    cudaStream_t stream);

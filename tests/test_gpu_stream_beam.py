@@ -40,7 +40,8 @@ def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=Fal
             slot[s] = dict(phrases=phrases, logits=sched.data[s]["logits"], length=int(sched.data[s]["length"]))
             served[s] = 0
             new.append(s)
-        if new:
+        if new and c % 2 == 0:
+            # the caller sets up the new slots' rows itself ...
             idx = torch.tensor(new, device=dev)
             scores[idx] = float("-inf")
             scores[idx, 0] = 0.0
@@ -48,6 +49,13 @@ def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=Fal
             states[idx, 0] = 0
             live[idx] = 0
             tb.tb_beam_reset_slots(batch, new)
+        elif new:
+            # ... or lets the library do it in the same launch (garbage first, to see that every entry is written)
+            idx = torch.tensor(new, device=dev)
+            scores[idx] = 123.0
+            states[idx] = 7
+            live[idx] = 1
+            tb.tb_beam_start_slots(batch, new, scores, states, live)
         left = np.clip(np.array([slot[s]["length"] for s in range(w.B)]) - served, 0, w.chunk).astype(np.int32)
         tb.tb_beam_chunk(batch, to_device(chunk), merge, torch.from_numpy(left).to(dev), scores, states, live, par, tok)
         served += left
