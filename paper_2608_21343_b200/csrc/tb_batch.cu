@@ -382,6 +382,7 @@ static void release_slot(tb_batch* b, int32_t slot) {
 }
 
 extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g, void* stream_) {
+  TbRange range_("tb_batch_bind_stream");
   if (!b) return TB_ERR_INVALID_ARG;
   if (slot < 0 || slot >= b->n_slots) return TB_ERR_BAD_SLOT;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -409,6 +410,7 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
 // host-to-device copy and one small launch, whatever the number of streams.
 extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slots, const tb_graph* const* graphs,
                                      void* stream_) {
+  TbRange range_("tb_batch_bind_streams");
   if (!b || n < 0 || (n > 0 && (!slots || !graphs))) return TB_ERR_INVALID_ARG;
   if (n == 0) return TB_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -524,6 +526,7 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
 }
 
 extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* out_model_id, void* stream_) {
+  TbRange range_("tb_batch_register_model");
   if (!b || !g || !out_model_id) return TB_ERR_INVALID_ARG;
   *out_model_id = -1;
   DeviceGuard guard(b->device);
@@ -567,6 +570,7 @@ extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* 
 }
 
 extern "C" int tb_batch_bind_models(tb_batch* b, int32_t n, const int32_t* slots, const int32_t* model_ids, void* stream_) {
+  TbRange range_("tb_batch_bind_models");
   if (!b || n < 0 || (n > 0 && (!slots || !model_ids))) return TB_ERR_INVALID_ARG;
   // everything is checked before anything is changed
   std::vector<uint8_t> seen(static_cast<size_t>(b->n_slots), 0);
@@ -666,6 +670,7 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
                                 const int64_t* strides, const int32_t* lengths, int32_t* out_tokens,
                                 int32_t* out_frames, int32_t* out_counts, float* out_scores, int32_t* out_states,
                                 void* stream_) {
+  TbRange range_("tb_greedy_decode");
   TbDecodeParams p;
   int rc = fill_decode_params(b, logits, dtype, B, T, S, 0, strides, &p);
   if (rc != TB_OK) return rc;
@@ -786,6 +791,7 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
                                int32_t S, int32_t n_dur, const int64_t* strides, const int32_t* valid_frames,
                                int32_t* out_tokens, int32_t* out_frames, int32_t* out_durs, int32_t* out_counts,
                                float* out_scores, int32_t* out_states, int32_t* out_cursors, void* stream_) {
+  TbRange range_("tb_stream_chunk");
   TbDecodeParams p;
   int rc = fill_decode_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, &p);
   if (rc != TB_OK) return rc;
@@ -838,6 +844,7 @@ extern "C" int tb_beam_reset(tb_batch* b) {
 extern "C" int tb_beam_step(tb_batch* b, const void* logits, int dtype, int32_t B, int32_t K, int64_t stream_stride,
                             int64_t hyp_stride, int32_t new_frame, float* scores, int32_t* states, uint8_t* live,
                             int32_t* out_parent, int32_t* out_token, void* stream_) {
+  TbRange range_("tb_beam_step");
   if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
   if ((dtype != TB_BF16 && dtype != TB_F32) || B < 1 || B > b->n_slots || K < 1 || K > b->max_beam) return TB_ERR_INVALID_ARG;
   if (b->chunk_K != 0) return TB_ERR_INVALID_ARG;   // a streaming session is under way: tb_beam_reset ends it
@@ -873,6 +880,7 @@ extern "C" int tb_beam_frames(tb_batch* b, const void* logits, int dtype, int32_
                               int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge,
                               float* scores, int32_t* states, uint8_t* live, int32_t* out_parent, int32_t* out_token,
                               void* stream_) {
+  TbRange range_("tb_beam_frames");
   if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
   if ((dtype != TB_BF16 && dtype != TB_F32) || B < 1 || B > b->n_slots || K < 1 || K > b->max_beam || T < 1 || E < 1 ||
       static_cast<int64_t>(T) * E > (1 << 24))
@@ -946,6 +954,7 @@ extern "C" int tb_beam_chunk(tb_batch* b, const void* logits, int dtype, int32_t
                              int64_t stream_stride, int64_t frame_stride, int64_t row_stride, int32_t merge,
                              const int32_t* n_frames, float* scores, int32_t* states, uint8_t* live, int32_t* out_parent,
                              int32_t* out_token, void* stream_) {
+  TbRange range_("tb_beam_chunk");
   if (!b || !logits || !scores || !states || !live || !out_parent || !out_token) return TB_ERR_INVALID_ARG;
   if ((dtype != TB_BF16 && dtype != TB_F32) || n_slots < 1 || n_slots > b->n_slots || K < 1 || K > b->max_beam || chunk < 1 ||
       E < 1 || static_cast<int64_t>(chunk) * E > (1 << 24))
@@ -976,6 +985,7 @@ extern "C" int tb_beam_chunk(tb_batch* b, const void* logits, int dtype, int32_t
 
 extern "C" int tb_beam_backtrace_slots(tb_batch* b, int32_t n_slots, int32_t K, int32_t max_len, int32_t* out_tokens,
                                        int32_t* out_lens, void* stream_) {
+  TbRange range_("tb_beam_backtrace_slots");
   if (!b || !out_tokens || !out_lens || max_len < 1 || n_slots < 1 || n_slots > b->n_slots) return TB_ERR_INVALID_ARG;
   if (!b->d_tree || b->chunk_K != K) return TB_ERR_INVALID_ARG;
   DeviceGuard guard(b->device);
@@ -1002,6 +1012,7 @@ extern "C" int tb_apply_final_weights_slots(tb_batch* b, int32_t n, const int32_
 
 extern "C" int tb_beam_backtrace(tb_batch* b, int32_t B, int32_t K, int32_t max_len, int32_t* out_tokens,
                                  int32_t* out_lens, void* stream_) {
+  TbRange range_("tb_beam_backtrace");
   if (!b || !out_tokens || !out_lens || max_len < 1) return TB_ERR_INVALID_ARG;
   if (!b->d_tree || b->tree_steps == 0 || b->tree_B != B || b->tree_K != K) return TB_ERR_INVALID_ARG;
   DeviceGuard guard(b->device);

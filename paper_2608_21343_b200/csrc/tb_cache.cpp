@@ -106,6 +106,7 @@ extern "C" int tb_graph_save(const tb_graph* g, const char* path) {
 }
 
 extern "C" int tb_graph_load(const char* path, tb_graph** out) {
+  TbRange range_("tb_graph_load");
   if (!out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
   if (!path) return TB_ERR_INVALID_ARG;
@@ -289,6 +290,7 @@ static void cache_insert(tb_cache* c, const std::string& key, tb_graph* g) {
 extern "C" int tb_cache_compile(tb_cache* c, const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,
                                 const float* token_weights, const int32_t* case_class, int32_t vocab, float lambda,
                                 uint32_t flags, tb_graph** out, int32_t* out_hit) {
+  TbRange range_("tb_cache_compile");
   if (!c || !out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
   if (out_hit) *out_hit = 0;

@@ -302,6 +302,7 @@ static int compile_impl(const int32_t* phrase_tokens, const int64_t* phrase_offs
 extern "C" int tb_graph_compile(const int32_t* phrase_tokens, const int64_t* phrase_offsets, int32_t n_phrases,
                                 const float* token_weights, const int32_t* case_class, int32_t vocab,
                                 float lambda, uint32_t flags, tb_graph** out) {
+  TbRange range_("tb_graph_compile");
   if (!out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
   if ((flags & ~static_cast<uint32_t>(TB_COMPILE_PAGEABLE)) != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda)) return TB_ERR_INVALID_ARG;
@@ -538,6 +539,7 @@ extern "C" int tb_graph_compile_variative(const uint8_t* phrase_chars, const int
                                           const float* phrase_weights, const uint8_t* piece_chars,
                                           const int64_t* piece_offsets, int32_t vocab, float tau, float lambda,
                                           uint32_t flags, tb_graph** out) {
+  TbRange range_("tb_graph_compile_variative");
   if (!out) return TB_ERR_INVALID_ARG;
   *out = nullptr;
   if ((flags & ~static_cast<uint32_t>(TB_COMPILE_PAGEABLE)) != 0 || vocab < 1 || vocab > TB_MAX_VOCAB || n_phrases < 0 || !std::isfinite(lambda) ||

@@ -7,7 +7,17 @@
 #include <cstdint>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "tb.h"
+
+// A named range around a library call for timeline tools (NVTX; costs a pointer test when no tool is attached).
+struct TbRange {
+  explicit TbRange(const char* name) { nvtxRangePushA(name); }
+  ~TbRange() { nvtxRangePop(); }
+  TbRange(const TbRange&) = delete;
+  TbRange& operator=(const TbRange&) = delete;
+};
 
 // Page-locked host memory for graph images.  A process that decodes (one that has created a batch) keeps the device
 // image of every graph it compiles or loads in one pool of page-locked memory, so that a bind is a plain

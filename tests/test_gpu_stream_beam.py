@@ -124,3 +124,39 @@ def test_streaming_beam_refuses_to_mix_with_the_batch_wide_tree(tb):
     with pytest.raises(tb.TbError):                        # and the other way round
         tb.tb_beam_chunk(batch, logits, False, None, scores, states, live, par, tok)
     torch.cuda.synchronize()
+
+
+def test_an_utterance_longer_than_the_tree_ring_is_reported(tb):
+    """A slot's hypothesis tree is a ring of max_tree_steps steps.  An utterance that outgrows it keeps decoding
+    correctly (scores, states); its backtrace raises TB_STATUS_STEP_LIMIT and yields the tokens still in the ring: the
+    tail of each transcript."""
+    w = W.get_workload(5, B=2, T=24, T_lo=24, S=2, n_dur=0, n_phrases=30, n_phrases_lo=30)
+    K, E, cap = 4, 2, 12
+    dev = torch.device("cuda:0")
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=K, max_tree_steps=cap, arena_bytes=4 << 20)
+    data = [W.stream_inputs(w, i) for i in range(w.B)]
+    for i, d in enumerate(data):
+        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(d["phrases"], w.V, case_class=w.vocab.case_class))
+    scores = torch.empty((w.B, K), device=dev)
+    states = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+    live = torch.empty((w.B, K), dtype=torch.uint8, device=dev)
+    par = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+    tok = torch.empty((w.B, K), dtype=torch.int32, device=dev)
+    tb.tb_beam_start_slots(batch, None, scores, states, live)
+    x = np.stack([d["logits"][:24] for d in data])                      # [2, 24, E, V + 1]
+    for c in range(3):                                                  # three chunks of 8 frames = 48 steps per slot
+        tb.tb_beam_chunk(batch, to_device(np.ascontiguousarray(x[:, 8 * c:8 * c + 8])), False, None, scores, states, live, par, tok)
+    toks, lens = tb.tb_beam_backtrace_slots(batch, w.B, K, 64)
+    torch.cuda.synchronize()
+    status = tb.tb_batch_status(batch)
+    assert status & tb.TB_STATUS_STEP_LIMIT, status
+    toks, lens = toks.cpu().numpy(), lens.cpu().numpy()
+    for i in range(w.B):
+        ref = O.beam_decode(oracle_graph(w, data[i]["phrases"]), x[i], K, merge=False, prune_delta=-1.0)
+        assert np.array_equal(states[i].cpu().numpy(), ref["states"])
+        assert np.allclose(scores[i].cpu().numpy(), ref["scores"], atol=SCORE_TOL)
+        for k in range(K):
+            n = int(lens[i, k])
+            assert n <= ref["lens"][k]
+            assert np.array_equal(toks[i, k, :n], ref["tokens"][k][ref["lens"][k] - n:ref["lens"][k]]), (i, k)
+        assert lens[i].max() <= cap
