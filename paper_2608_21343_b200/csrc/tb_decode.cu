@@ -241,6 +241,43 @@ struct BeamKey {  // order: value descending, token key ascending, parent ascend
   int32_t tkey, par;
 };
 // One beam expansion of the block's stream (the body of k_beam_step; k_beam_frames calls it once per row).
+// The K largest of the keys ckey[first], ckey[first + stride], ... (those below n; 0 = no candidate) that this warp's
+// lanes look at, R per lane: out_key[r] / out_idx[r] for r < K, best first (key 0, index -1 once nothing is left).
+// Every lane keeps its keys sorted in registers, so a round is two warp-wide integer maxima over the lanes' heads;
+// the lane that holds the winner finds its index again (one of its R places in the array) and moves up its other keys.
+template <int R>
+__device__ __forceinline__ void warp_top_keys(const unsigned long long* ckey, int n, int first, int stride, int K, int lane,
+                                              unsigned long long* out_key, int32_t* out_idx) {
+  unsigned long long ck[R];
+#pragma unroll
+  for (int j = 0; j < R; ++j) { const int i = first + stride * j; ck[j] = i < n ? ckey[i] : 0ull; }
+  auto ce = [&](int a, int b) { const bool sw = ck[b] > ck[a]; const unsigned long long hi = sw ? ck[b] : ck[a], lo = sw ? ck[a] : ck[b]; ck[a] = hi; ck[b] = lo; };
+  if (R == 2) { ce(0, 1); }
+  if (R == 4) { ce(0, 1); ce(2, 3); ce(0, 2); ce(1, 3); ce(1, 2); }
+  if (R == 8) {
+    ce(0, 1); ce(2, 3); ce(4, 5); ce(6, 7); ce(0, 2); ce(1, 3); ce(4, 6); ce(5, 7); ce(1, 2); ce(5, 6);
+    ce(0, 4); ce(1, 5); ce(2, 6); ce(3, 7); ce(2, 4); ce(3, 5); ce(1, 2); ce(3, 4); ce(5, 6);
+  }
+  for (int r = 0; r < K; ++r) {
+    const unsigned long long a = ck[0];
+    const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+    const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+    const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+    const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+    if (best == 0ull) {
+      if (lane == 0) { out_key[r] = 0ull; out_idx[r] = -1; }
+    } else if (a == best) {
+      int idx = -1;
+#pragma unroll
+      for (int j = 0; j < R; ++j) { const int i = first + stride * j; if (i < n && ckey[i] == best) idx = i; }
+      out_key[r] = best; out_idx[r] = idx;
+#pragma unroll
+      for (int j = 0; j + 1 < R; ++j) ck[j] = ck[j + 1];
+      ck[R - 1] = 0ull;
+    }
+  }
+}
+
 // threads of a beam block: more warps than the general kernel's hide the latencies of its short dependent phases; 17
 // warps take a row of 1025 logits (vocabularies of about a thousand pieces) in two strides instead of three
 constexpr int kBeamThreads = 544;
@@ -389,14 +426,42 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)
     int32_t* cdst = reinterpret_cast<int32_t*>(ckey + cap);
     const LT* base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
     const bool recs_at_hand = p.tv_ready && rec_ready;        // left by the previous step of this launch
-    if (threadIdx.x < K && !recs_at_hand) {
-      const int k = threadIdx.x;
-      h_beg[k] = 0; h_cnt[k] = 0; h_D[k] = 0.0f;
-      if (bound && h_score[k] != -INFINITY) {
-        int32_t st = h_state[k];
-        if (st < 0 || st >= rec.n_states) { atomicOr(p.status, TB_STATUS_BAD_STATE); st = 0; }
-        const TbRsRec r = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[st];
-        h_beg[k] = r.begin; h_cnt[k] = r.count; h_D[k] = r.D;
+    if (warp == 0) {
+      // lane k: hypothesis k's list record (fetched now unless the previous step left it), then where its listed
+      // candidates start in the candidate array: a prefix sum over the warp (K <= 32)
+      const int k = lane;
+      int cntk = 0;
+      bool lv = false;
+      if (k < K) {
+        if (!recs_at_hand) {
+          int32_t beg = 0;
+          float Dk = 0.0f;
+          if (bound && h_score[k] != -INFINITY) {
+            int32_t st = h_state[k];
+            if (st < 0 || st >= rec.n_states) { atomicOr(p.status, TB_STATUS_BAD_STATE); st = 0; }
+            const TbRsRec r = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec)[st];
+            beg = r.begin; cntk = r.count; Dk = r.D;
+          }
+          h_beg[k] = beg; h_cnt[k] = cntk; h_D[k] = Dk;
+        } else {
+          cntk = h_cnt[k];
+        }
+        lv = h_score[k] != -INFINITY && h_live[k];
+        hl_n[k] = !lv ? 0 : (cntk <= kBeamList ? cntk : -1);
+      }
+      const int c = lv ? cntk : 0;
+      int incl = c;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (k < K) cp_off[k] = incl - c;
+      const int total = __shfl_sync(0xffffffffu, incl, 31);
+      if (lane == 0) {
+        cp_off[K] = total;
+        cp_flag = total + K * (M + 1) <= cap ? 1 : 0;
+        cp_n = total + K * (M + 1);
       }
     }
     for (int i = threadIdx.x; i < K * WW; i += kBeamThreads) ovr[i] = 0u;
@@ -424,19 +489,6 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)
     // measured slower than the whole block: 8.4 against 6.9 ms per utterance at K = 4)
     const int cth = static_cast<int>(threadIdx.x), cnt = kBeamThreads;
     {
-      if (cth == 0) {
-        int at = 0;
-        for (int k = 0; k < K; ++k) {
-          cp_off[k] = at;
-          const bool lv = h_score[k] != -INFINITY && h_live[k];
-          hl_n[k] = !lv ? 0 : (h_cnt[k] <= kBeamList ? h_cnt[k] : -1);
-          if (lv) at += h_cnt[k];
-        }
-        cp_off[K] = at;
-        cp_flag = at + K * (M + 1) <= cap ? 1 : 0;
-        cp_n = at + K * (M + 1);
-      }
-      __syncthreads();
       if (cp_flag) {
         const int n_listed = cp_off[K], n = cp_n;
         // the listed tokens of every hypothesis, all hypotheses at once: exact values; marked, so that the walk over
@@ -500,65 +552,90 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)
         }
         __syncthreads();
         {
-          // Selection in two levels, without a block-wide barrier per round: every warp picks the K best of the
-          // candidates it looks at (indices warp * 32 + lane, + the block size, ...) in K warp-wide rounds and
-          // leaves them, best first, in shared memory; warp 0 then merges the warps' lists, one lane per list.
+          // Selection (warp_top_keys).  A thread takes its candidates (indices thread, thread + block size, ...) into
+          // registers once and keeps them sorted; a round is then two warp-wide integer maxima over the lanes' best.
+          // Few candidates (narrow beams): warp 0 alone.  Many: every warp picks the K best of its candidates and
+          // leaves them, best first, in shared memory; warp 0 then merges the warps' lists, one lane per list, the
+          // head of each in a register.
           unsigned long long* wkey = reinterpret_cast<unsigned long long*>(cdst + cap);            // [warps][K] (key); behind the targets
           int32_t* widx = reinterpret_cast<int32_t*>(wkey + (kBeamThreads / 32) * TB_MAX_BEAM);   // [warps][K] where in ckey
-          {
-            unsigned long long lim = ~0ull;
-            for (int r = 0; r < K; ++r) {
-              unsigned long long a = 0ull;
-              int ai = -1;
-              for (int i = threadIdx.x; i < n; i += kBeamThreads) { const unsigned long long kk = ckey[i]; if (kk < lim && kk > a) { a = kk; ai = i; } }
-              const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
-              const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
-              const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
-              const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
-              if (best != 0ull && a == best) { wkey[warp * TB_MAX_BEAM + r] = best; widx[warp * TB_MAX_BEAM + r] = ai; }
-              if (best == 0ull && lane == 0) { wkey[warp * TB_MAX_BEAM + r] = 0ull; widx[warp * TB_MAX_BEAM + r] = -1; }
-              lim = best;                                       // (0 once nothing is left: the later rounds find nothing either)
+          constexpr int kSelRegs = 8;
+          const bool solo = n <= 32 * kSelRegs;
+          auto put_sel = [&](int r, unsigned long long best, int idx) {
+            const uint32_t mh = static_cast<uint32_t>(best >> 32);
+            const uint32_t l2 = 0xFFFFFFFFu - static_cast<uint32_t>(best & 0xFFFFFFFFull);
+            BeamKey c;
+            c.v = __uint_as_float(mh ^ ((mh >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+            c.tkey = static_cast<int32_t>(l2 >> 5); c.par = static_cast<int32_t>(l2 & 31u);
+            if (best == 0ull) c = BeamKey{-INFINITY, INT32_MAX, INT32_MAX};
+            sel[r] = c; sel_dst[r] = best == 0ull ? -1 : cdst[idx];
+          };
+          if (solo) {
+            if (warp == 0) {
+              if (n <= 32 * 4) warp_top_keys<4>(ckey, n, lane, 32, K, lane, wkey, widx);
+              else warp_top_keys<8>(ckey, n, lane, 32, K, lane, wkey, widx);
+              __syncwarp();
+              if (lane < K) put_sel(lane, wkey[lane], widx[lane]);
             }
-          }
-          __syncthreads();
-          if (warp == 0) {
-            // lane w walks warp w's list from its head; a round takes the largest head
-            int ptr = 0;
-            for (int r = 0; r < K; ++r) {
-              const unsigned long long a = (lane < kBeamThreads / 32 && ptr < K) ? wkey[lane * TB_MAX_BEAM + ptr] : 0ull;
-              const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
-              const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
-              const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
-              const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
-              if (best == 0ull) {
-                if (lane == 0) { sel[r] = BeamKey{-INFINITY, INT32_MAX, INT32_MAX}; sel_dst[r] = -1; }
-              } else if (a == best) {
-                const uint32_t l2 = 0xFFFFFFFFu - static_cast<uint32_t>(best & 0xFFFFFFFFull);
-                BeamKey c;
-                c.v = __uint_as_float(mh ^ ((mh >> 31) ? 0x80000000u : 0xFFFFFFFFu));
-                c.tkey = static_cast<int32_t>(l2 >> 5); c.par = static_cast<int32_t>(l2 & 31u);
-                sel[r] = c; sel_dst[r] = cdst[widx[lane * TB_MAX_BEAM + ptr]];
-                ++ptr;
+          } else {
+            if (n <= kBeamThreads * 2) {
+              warp_top_keys<2>(ckey, n, static_cast<int>(threadIdx.x), kBeamThreads, K, lane, wkey + warp * TB_MAX_BEAM, widx + warp * TB_MAX_BEAM);
+            } else if (n <= kBeamThreads * 4) {
+              warp_top_keys<4>(ckey, n, static_cast<int>(threadIdx.x), kBeamThreads, K, lane, wkey + warp * TB_MAX_BEAM, widx + warp * TB_MAX_BEAM);
+            } else if (n <= kBeamThreads * 8) {
+              warp_top_keys<8>(ckey, n, static_cast<int>(threadIdx.x), kBeamThreads, K, lane, wkey + warp * TB_MAX_BEAM, widx + warp * TB_MAX_BEAM);
+            } else {
+              // (more candidates than the registers take: rounds over the array in shared memory)
+              unsigned long long lim = ~0ull;
+              for (int r = 0; r < K; ++r) {
+                unsigned long long a = 0ull;
+                int ai = -1;
+                for (int ii = threadIdx.x; ii < n; ii += kBeamThreads) { const unsigned long long kk = ckey[ii]; if (kk < lim && kk > a) { a = kk; ai = ii; } }
+                const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+                const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+                const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+                const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+                if (best != 0ull && a == best) { wkey[warp * TB_MAX_BEAM + r] = best; widx[warp * TB_MAX_BEAM + r] = ai; }
+                if (best == 0ull && lane == 0) { wkey[warp * TB_MAX_BEAM + r] = 0ull; widx[warp * TB_MAX_BEAM + r] = -1; }
+                lim = best;                                       // (0 once nothing is left: the later rounds find nothing either)
+              }
+            }
+            __syncthreads();
+            if (warp == 0) {
+              // lane w walks warp w's list from its head, which it keeps in a register; a round takes the largest head
+              int ptr = 0;
+              unsigned long long hk = lane < kBeamThreads / 32 ? wkey[lane * TB_MAX_BEAM] : 0ull;
+              for (int r = 0; r < K; ++r) {
+                const uint32_t hi = static_cast<uint32_t>(hk >> 32), lo = static_cast<uint32_t>(hk);
+                const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+                const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+                const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+                if (best == 0ull) {
+                  if (lane == 0) put_sel(r, 0ull, -1);
+                } else if (hk == best) {
+                  put_sel(r, best, widx[lane * TB_MAX_BEAM + ptr]);
+                  ++ptr;
+                  hk = ptr < K ? wkey[lane * TB_MAX_BEAM + ptr] : 0ull;
+                }
               }
             }
           }
-        }
-        __syncthreads();
-        if (cth == 0) {
-          // does the K-th pick clear everything that was not looked at?
-          const float y_next = ttop[M].y;
-          int ok = 1;
-          if (y_next != -INFINITY) {
-            const float c_k = sel[K - 1].par != INT32_MAX ? sel[K - 1].v : -INFINITY;
-            for (int k = 0; k < K; ++k) {
-              if (h_score[k] == -INFINITY || !h_live[k]) continue;
+          if (warp == 0) {
+            // does the K-th pick clear everything that was not looked at?  Lane k answers for hypothesis k.
+            __syncwarp();
+            const float y_next = ttop[M].y;
+            bool okk = true;
+            if (y_next != -INFINITY && lane < K && h_score[lane] != -INFINITY && h_live[lane]) {
+              const int k = lane;
+              const float c_k = sel[K - 1].par != INT32_MAX ? sel[K - 1].v : -INFINITY;
               const float lamD = bound ? g.lambda * h_D[k] : 0.0f;
               const float scale = fabsf(h_score[k]) + fabsf(y_next) + 2.0f * (bound ? fabsf(g.lambda) * (fabsf(h_D[k]) + root_wmax) : 0.0f);
               const float ub = (h_score[k] + y_next) + lamD + scale * 3.814697265625e-6f + 1e-30f;      // 2^-18 of the scale
-              if (!(c_k > ub)) ok = 0;
+              okk = c_k > ub;
             }
+            const bool all_ok = __all_sync(0xffffffffu, okk);
+            if (lane == 0) cp_flag = all_ok ? 1 : 0;
           }
-          cp_flag = ok;
         }
       }
     }
