@@ -284,8 +284,40 @@ constexpr int kBeamThreads = 544;
 constexpr int kBeamPref = 5;   // elements of a shared row each thread may hold ahead of time (rows up to 5 * kBeamThreads wide)
 // xpre / xpre_valid: this thread's elements of the stream's shared row, fetched ahead by the previous step of the same
 // launch; next_row: where the next step's shared row starts (null: none), fetched while this step selects.
+// What a beam block keeps in shared memory besides its candidate arrays: the stream's hypotheses from step to step,
+// and the working set of a step.
+constexpr int kTeamMaxK = 8;   // (= kFastMaxK, needed here already)
+struct BeamShared {
+  ChainSmem chain;
+  // token-view path: per hypothesis a copy of its state's short list, to find the next state of a pick
+  uint16_t hl_tok[TB_MAX_BEAM][kBeamList];
+  int32_t hl_dst[TB_MAX_BEAM][kBeamList];
+  int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
+  int32_t h_beg[TB_MAX_BEAM], h_cnt[TB_MAX_BEAM];
+  float h_D[TB_MAX_BEAM];
+  unsigned long long red64[2][kBeamThreads / 32];   // the warps' best keys, two copies used in turn by the selection rounds
+  float h_score[TB_MAX_BEAM];
+  int32_t h_state[TB_MAX_BEAM];
+  uint8_t h_live[TB_MAX_BEAM];
+  unsigned long long h_hash[TB_MAX_BEAM];   // identity of the hypothesis' token sequence
+  int32_t h_len[TB_MAX_BEAM];
+  BeamKey sel[TB_MAX_BEAM];
+  int32_t sel_dst[TB_MAX_BEAM];      // compact path: the graph state a selected candidate leads to
+  int32_t cp_n, cp_flag;             // compact path: candidates laid out; 0 = this step cannot take it
+  int32_t cp_off[TB_MAX_BEAM + 1];   // compact path: where each hypothesis' listed candidates start
+  int32_t rec_ready;                 // the hypotheses' list records in h_beg / h_cnt / h_D are those of their current states
+  TbTopEnt ttop[2 * TB_MAX_BEAM + 9]; // this step's reduced row
+  float root_wmax;                   // largest |root arc weight| of the stream's graph (filled with the root tables)
+  int32_t fast_done;                 // narrow beams: steps the team has just taken
+  // narrow beams, between the team's warps: the hypotheses a step works on, each worker's picks and bound term
+  float f_sc[kTeamMaxK]; int32_t f_st[kTeamMaxK]; uint8_t f_lv[kTeamMaxK];
+  unsigned long long f_key[kTeamMaxK][kTeamMaxK]; int32_t f_dst[kTeamMaxK][kTeamMaxK];
+  float f_ub[kTeamMaxK];
+  volatile int32_t f_cmd, f_fail;    // 1: the run ends here / a worker met a list it cannot take
+};
+
 template <typename LT>
-__device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)[kBeamPref], bool& xpre_valid,
+__device__ __forceinline__ void beam_step_body(const TbBeamParams& p, BeamShared& sh, LT (&xpre)[kBeamPref], bool& xpre_valid,
                                                const LT* next_row, TbTopEnt& tpre, bool& tpre_valid,
                                                const TbTopEnt* next_top) {
   extern __shared__ __align__(16) unsigned char dyn[];
@@ -296,26 +328,17 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, LT (&xpre)
   unsigned char* aux = reinterpret_cast<unsigned char*>(ovr) + ((static_cast<size_t>(K) * WW * sizeof(uint32_t) + 15) & ~size_t(15));
   float* bvec = reinterpret_cast<float*>(aux);                         // [C]   (chain-walk path)
   int32_t* nvec = reinterpret_cast<int32_t*>(bvec + p.C);              // [C]
-  __shared__ ChainSmem chain;
-  // token-view path: per hypothesis a copy of its state's short list, to find the next state of a pick
-  __shared__ uint16_t hl_tok[TB_MAX_BEAM][kBeamList];
-  __shared__ int32_t hl_dst[TB_MAX_BEAM][kBeamList];
-  __shared__ int32_t hl_n[TB_MAX_BEAM];                                 // -1: list too long, walk the chain instead
-  __shared__ int32_t h_beg[TB_MAX_BEAM], h_cnt[TB_MAX_BEAM];
-  __shared__ float h_D[TB_MAX_BEAM];
-  __shared__ unsigned long long red64[2][kBeamThreads / 32];   // the warps' best keys, two copies used in turn by the selection rounds
-  __shared__ float h_score[TB_MAX_BEAM];
-  __shared__ int32_t h_state[TB_MAX_BEAM];
-  __shared__ uint8_t h_live[TB_MAX_BEAM];
-  __shared__ unsigned long long h_hash[TB_MAX_BEAM];   // identity of the hypothesis' token sequence
-  __shared__ int32_t h_len[TB_MAX_BEAM];
-  __shared__ BeamKey sel[TB_MAX_BEAM];
-  __shared__ int32_t sel_dst[TB_MAX_BEAM];      // compact path: the graph state a selected candidate leads to
-  __shared__ int32_t cp_n, cp_flag;             // compact path: candidates laid out; 0 = this step cannot take it
-  __shared__ int32_t cp_off[TB_MAX_BEAM + 1];   // compact path: where each hypothesis' listed candidates start
-  __shared__ int32_t rec_ready;                 // the hypotheses' list records in h_beg / h_cnt / h_D are those of their current states
-  __shared__ TbTopEnt ttop[2 * TB_MAX_BEAM + 9]; // this step's reduced row
-  __shared__ float root_wmax;                   // largest |root arc weight| of the stream's graph (filled with the root tables)
+  ChainSmem& chain = sh.chain;
+  auto& hl_tok = sh.hl_tok; auto& hl_dst = sh.hl_dst; auto& hl_n = sh.hl_n;
+  auto& h_beg = sh.h_beg; auto& h_cnt = sh.h_cnt; auto& h_D = sh.h_D;
+  auto& red64 = sh.red64;
+  auto& h_score = sh.h_score; auto& h_state = sh.h_state; auto& h_live = sh.h_live; auto& h_hash = sh.h_hash; auto& h_len = sh.h_len;
+  auto& sel = sh.sel; auto& sel_dst = sh.sel_dst;
+  int32_t& cp_n = sh.cp_n; int32_t& cp_flag = sh.cp_flag;
+  auto& cp_off = sh.cp_off;
+  int32_t& rec_ready = sh.rec_ready;
+  auto& ttop = sh.ttop;
+  float& root_wmax = sh.root_wmax;
 
   const int b = blockIdx.x;
   const TbSlotRec rec = p.slots[b];
@@ -881,7 +904,368 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
   bool xpre_valid = false;
   TbTopEnt tpre{0.0f, 0.0f, 0u};
   bool tpre_valid = false;
-  beam_step_body<LT>(p, xpre, xpre_valid, static_cast<const LT*>(nullptr), tpre, tpre_valid, nullptr);
+  __shared__ BeamShared sh;
+  beam_step_body<LT>(p, sh, xpre, xpre_valid, static_cast<const LT*>(nullptr), tpre, tpre_valid, nullptr);
+}
+
+
+// ---- narrow beams: steps taken by a small team of warps ------------------------------------------------------------
+// With K <= 8 and the rows reduced ahead of the steps, a step has a few dozen candidates, and the block-wide step body
+// spends its time in block-wide barriers between short phases.  beam_fast_run lets K + 1 warps take such steps, one
+// after the other, while the block's other warps wait: warp 0 coordinates (it holds the stream's hypotheses in
+// registers, lane k: hypothesis k), warp k + 1 works for hypothesis k.  Per step
+//   worker k     : the hypothesis' list record, its listed tokens (exact values; logits from the row, which arrives
+//                  in shared memory by asynchronous copies the coordinator issues two steps ahead), blank, the first
+//                  unlisted tokens of the reduced row or the carried hypothesis -- at most 32 * kFastRL + 32
+//                  candidates in registers --, its K best of them in K rounds of two warp-wide integer maxima;
+//   barrier of the team (a named barrier, not the block's);
+//   coordinator  : the K best of the workers' picks, the same bound check as the block-wide compact path, the new
+//                  hypotheses, and, where the next step begins a frame, merging and pruning;
+//   barrier of the team; then the workers go on while the coordinator writes the step's results to global memory
+//                  and asks for the row after the next.
+// A step the team cannot take (a list of more than 32 * kFastRL tokens, the bound not cleared) is left untouched: the
+// run ends before it, the hypotheses go back to shared memory, and the whole block does that step with
+// beam_step_body.  Same arithmetic, same order of candidates, hence the same results bit for bit.
+constexpr int kFastMaxK = 8;      // widest beam of the team's steps
+constexpr int kFastRL = 3;        // a worker lane's registers for listed tokens (lists of up to 32 * kFastRL tokens)
+constexpr int kFastR = kFastRL + 1;
+
+__device__ __forceinline__ unsigned long long beam_key(float v, int tkey, int k) {
+  const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
+  const uint32_t hi = u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+  const uint32_t lo = 0xFFFFFFFFu - (static_cast<uint32_t>(tkey) * 32u + static_cast<uint32_t>(k));
+  return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+__device__ __forceinline__ float beam_key_value(unsigned long long key) {
+  const uint32_t mh = static_cast<uint32_t>(key >> 32);
+  return __uint_as_float(mh ^ ((mh >> 31) ? 0x80000000u : 0xFFFFFFFFu));
+}
+__device__ __forceinline__ unsigned long long shfl_u64(unsigned long long v, int src) {
+  const uint32_t lo = __shfl_sync(0xffffffffu, static_cast<uint32_t>(v), src);
+  const uint32_t hi = __shfl_sync(0xffffffffu, static_cast<uint32_t>(v >> 32), src);
+  return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+__device__ __forceinline__ void beam_cp_async16(unsigned char* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem))), "l"(src) : "memory");
+}
+__device__ __forceinline__ void beam_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void beam_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+template <typename LT> __device__ __forceinline__ float beam_smem_logit(const unsigned char* row, int idx);
+template <> __device__ __forceinline__ float beam_smem_logit<uint16_t>(const unsigned char* row, int idx) {
+  return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row + 2 * idx)) << 16);
+}
+template <> __device__ __forceinline__ float beam_smem_logit<float>(const unsigned char* row, int idx) {
+  return *reinterpret_cast<const float*>(row + 4 * idx);
+}
+// Starts the copy of one row (its 16-byte aligned superset) into buf; a 16-byte piece that is not wholly inside the
+// tensor [lo, hi) is assembled from the elements that are.
+template <typename LT>
+__device__ __forceinline__ void beam_fetch_row(unsigned char* buf, const LT* row, int W, const unsigned char* lo,
+                                               const unsigned char* hi, int lane) {
+  const unsigned char* rp = reinterpret_cast<const unsigned char*>(row);
+  const int off = static_cast<int>(reinterpret_cast<uintptr_t>(rp) & 15);
+  const unsigned char* a0 = rp - off;
+  const int nchunks = (off + W * static_cast<int>(sizeof(LT)) + 15) >> 4;
+  for (int c = lane; c < nchunks; c += 32) {
+    const unsigned char* ac = a0 + 16 * c;
+    if (ac >= lo && ac + 16 <= hi) {
+      beam_cp_async16(buf + 16 * c, ac);
+    } else {
+      for (int e = 0; e < 16; e += static_cast<int>(sizeof(LT)))
+        if (ac + e >= lo && ac + e + sizeof(LT) <= hi) *reinterpret_cast<LT*>(buf + 16 * c + e) = *reinterpret_cast<const LT*>(ac + e);
+    }
+  }
+}
+__host__ __device__ inline size_t beam_ring_bytes(int V, int elem) {   // two row buffers of the lone-warp steps
+  const size_t one = ((static_cast<size_t>(V + 1) * elem + 16 + 15) & ~size_t(15)) + 16;
+  return 2 * one + 16;
+}
+
+__device__ __forceinline__ void beam_team_barrier(int n_threads) { asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory"); }
+
+// Takes the steps sidx, sidx + 1, ... of the block's stream as long as it can; returns (on warp 0) how many it took.
+// Called by warps 0 .. K; the hypotheses are read from and left in sh.h_*.  hashA / hashB, lenA / lenB: the two halves
+// of the sequence records; step s writes half ((par0 + s) & 1 ? A : B).
+template <typename LT>
+__device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& sh, unsigned char* dyn, int32_t sidx, const int32_t n_steps,
+                                             const int32_t E, const int64_t frame_stride, const int64_t row_stride,
+                                             const int32_t rows_per_stream, const int32_t step_base, unsigned long long* hashA,
+                                             unsigned long long* hashB, int32_t* lenA, int32_t* lenB, const int32_t par0) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.x, K = p.K, V = p.V, W = V + 1, M = p.top_m, WW = (W + 31) >> 5;
+  const int team = 32 * (K + 1);
+  const TbSlotRec rec = p.slots[b];
+  const bool bound = rec.n_states > 0;
+  const GraphPtrs g = graph_of(p.arena, rec);
+  const unsigned char* blob = p.arena + rec.blob_off;
+  uint32_t* ovr = reinterpret_cast<uint32_t*>(dyn + ((static_cast<size_t>(K) * W * sizeof(float) + 15) & ~size_t(15)));
+  unsigned char* aux = reinterpret_cast<unsigned char*>(ovr) + ((static_cast<size_t>(K) * WW * sizeof(uint32_t) + 15) & ~size_t(15));
+  unsigned char* ring = aux + beam_aux_bytes(V, p.C, p.tokview) + static_cast<size_t>(W) * sizeof(float);
+  ring += (16 - (reinterpret_cast<uintptr_t>(ring) & 15)) & 15;
+  const int row_buf = static_cast<int>((beam_ring_bytes(V, sizeof(LT)) - 16) / 2);
+  const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
+  auto row_of = [&](int s) -> const LT* {
+    const int t = s / E, e = s - t * E;
+    return stream_base + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
+  };
+
+  if (warp > 0) {
+    // ================================ worker: hypothesis k ================================
+    const int k = warp - 1;
+    TokView tv;
+    tokview_attach(tv, aux, V, p.C);
+    const TbTopEnt* top0 = p.top_base + static_cast<int64_t>(b) * rows_per_stream * (M + 1);
+    const TbRsRec* rsrec = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec);
+    const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
+    uint32_t* ovr_k = ovr + k * WW;
+    beam_team_barrier(team);                                   // the coordinator has set up the first step
+    for (;; ++sidx) {
+      if (sh.f_cmd != 0) break;
+      TbTopEnt tt{-INFINITY, -INFINITY, 0xFFFFu};
+      if (lane <= M) tt = top0[static_cast<int64_t>(sidx) * (M + 1) + lane];
+      const float sc1 = sh.f_sc[k];
+      const int32_t st1 = sh.f_st[k];
+      const bool lv1 = sh.f_lv[k] != 0;
+      unsigned long long ck[kFastR];
+      int32_t cd[kFastR];
+#pragma unroll
+      for (int j = 0; j < kFastR; ++j) { ck[j] = 0ull; cd[j] = -1; }
+      float D = 0.0f;
+      if (sc1 != -INFINITY) {
+        int32_t beg = 0, cnt = 0;
+        if (bound) {
+          int32_t sx = st1;
+          if (sx < 0 || sx >= rec.n_states) { if (lane == 0) atomicOr(p.status, TB_STATUS_BAD_STATE); sx = 0; }
+          const TbRsRec r = rsrec[sx];
+          beg = r.begin; cnt = r.count; D = r.D;
+        }
+        const unsigned char* rowb = ring + (sidx & 1) * row_buf + (reinterpret_cast<uintptr_t>(row_of(sidx)) & 15);
+        if (lv1) {
+          if (cnt > 32 * kFastRL) { if (lane == 0) sh.f_fail = 1; cnt = 0; }
+          for (int i = lane; i < WW; i += 32) ovr_k[i] = 0u;
+          __syncwarp();
+          // the listed tokens: exact values
+#pragma unroll
+          for (int j = 0; j < kFastRL; ++j) {
+            const int i = lane + 32 * j;
+            if (i < cnt) {
+              const TbRsEnt en = ent[beg + i];
+              const int tk = static_cast<int>((en.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
+              if (tk < V) {
+                const float x = beam_smem_logit<LT>(rowb, tk);
+                ck[j] = beam_key(__fadd_rn(sc1, __fadd_rn(x, en.lb)), tk, k);
+                cd[j] = static_cast<int32_t>(en.dst_tok >> TB_RS_TOK_BITS);
+                atomicOr(&ovr_k[tk >> 5], 1u << (tk & 31));
+              }
+            }
+          }
+          __syncwarp();
+          // blank and the first unlisted tokens of the reduced row: lane j looks at its entry j
+          if (lane == M) {
+            ck[kFastRL] = beam_key(__fadd_rn(sc1, tt.x), V, k); cd[kFastRL] = st1;
+          } else if (lane < M) {
+            const int tk = static_cast<int>(tt.tok_cls & 0xFFFFu), cl = static_cast<int>(tt.tok_cls >> 16);
+            if (tk < V && !((ovr_k[tk >> 5] >> (tk & 31)) & 1u)) {     // (tk >= V: the row has fewer tokens)
+              const float val = bound ? __fadd_rn(tt.x, __fmul_rn(g.lambda, __fadd_rn(D, tv.rootcw[cl]))) : tt.x;
+              ck[kFastRL] = beam_key(__fadd_rn(sc1, val), tk, k);
+              cd[kFastRL] = bound ? tv.rootdst[cl] : -1;
+            }
+          }
+        } else if (lane == M) {
+          ck[kFastRL] = beam_key(sc1, V + 1, k); cd[kFastRL] = st1;      // a frozen hypothesis is carried
+        }
+      }
+      // the K best of this hypothesis' candidates: lane r ends up with pick r
+      unsigned long long mykey = 0ull;
+      int32_t mydst = -1;
+      for (int r = 0; r < K; ++r) {
+        unsigned long long a = ck[0];
+        int aj = 0;
+#pragma unroll
+        for (int jj = 1; jj < kFastR; ++jj) { const bool bt = ck[jj] > a; a = bt ? ck[jj] : a; aj = bt ? jj : aj; }
+        const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+        const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+        const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+        const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+        if (best == 0ull) break;                                  // (uniform: nothing left; the later picks stay empty)
+        const bool mine = a == best;
+        const unsigned who = __ballot_sync(0xffffffffu, mine);
+        int32_t dw = cd[0];
+#pragma unroll
+        for (int jj = 1; jj < kFastR; ++jj) dw = jj == aj ? cd[jj] : dw;
+        const int32_t dsel = __shfl_sync(0xffffffffu, dw, __ffs(who) - 1);
+        if (lane == r) { mykey = best; mydst = dsel; }
+        if (mine) {
+#pragma unroll
+          for (int jj = 0; jj < kFastR; ++jj) ck[jj] = jj == aj ? 0ull : ck[jj];
+        }
+      }
+      if (lane < K) { sh.f_key[k][lane] = mykey; sh.f_dst[k][lane] = mydst; }
+      {
+        // what the K-th pick of the step has to clear on behalf of this hypothesis (-inf: nothing)
+        const float y_next = __shfl_sync(0xffffffffu, tt.y, M);
+        if (lane == 0) {
+          float ub = -INFINITY;
+          if (y_next != -INFINITY && sc1 != -INFINITY && lv1) {
+            const float lamD = bound ? g.lambda * D : 0.0f;
+            const float scale = fabsf(sc1) + fabsf(y_next) + 2.0f * (bound ? fabsf(g.lambda) * (fabsf(D) + sh.root_wmax) : 0.0f);
+            ub = (sc1 + y_next) + lamD + scale * 3.814697265625e-6f + 1e-30f;      // 2^-18 of the scale
+          }
+          sh.f_ub[k] = ub;
+        }
+      }
+      beam_team_barrier(team);                                 // picks are in place
+      beam_team_barrier(team);                                 // the coordinator has set up the next step (or ended the run)
+    }
+    return 0;
+  }
+
+  // ================================ coordinator ================================
+  float sc = -INFINITY;
+  int32_t st = -1, hl = 0;
+  bool lv = false;
+  unsigned long long hh = 0ull;
+  if (lane < K) { sc = sh.h_score[lane]; st = sh.h_state[lane]; lv = sh.h_live[lane] != 0; hh = sh.h_hash[lane]; hl = sh.h_len[lane]; }
+  // the working copy of the hypotheses for step s: after the frame start's liveness, merging and pruning
+  float sc1 = sc;
+  int32_t st1 = st;
+  bool lv1 = lv;
+  auto frame_start = [&](int s) {
+    sc1 = sc; st1 = st; lv1 = lv;
+    if (s % E != 0) return;
+    lv1 = sc1 != -INFINITY;
+    if (p.merge) {
+      bool dup = false;
+      for (int j = 0; j + 1 < K; ++j) {
+        const float sj = __shfl_sync(0xffffffffu, sc, j);
+        const int32_t lj = __shfl_sync(0xffffffffu, hl, j), stj = __shfl_sync(0xffffffffu, st, j);
+        const unsigned long long hj = shfl_u64(hh, j);
+        if (lane > j && lane < K && sc != -INFINITY && sj != -INFINITY && lj == hl && hj == hh && stj == st) dup = true;
+      }
+      if (dup) { sc1 = -INFINITY; st1 = -1; lv1 = false; }
+    }
+    if (p.prune_delta >= 0.0f) {
+      float best = sc1;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, o));
+      if (lane < K && sc1 != -INFINITY && sc1 < __fsub_rn(best, p.prune_delta)) { sc1 = -INFINITY; st1 = -1; lv1 = false; }
+    }
+  };
+  auto publish = [&]() { if (lane < K) { sh.f_sc[lane] = sc1; sh.f_st[lane] = st1; sh.f_lv[lane] = lv1 ? 1 : 0; } };
+  frame_start(sidx);
+  publish();
+  if (lane == 0) { sh.f_cmd = 0; sh.f_fail = 0; }
+  beam_fetch_row<LT>(ring + (sidx & 1) * row_buf, row_of(sidx), W, p.tensor_lo, p.tensor_hi, lane);
+  if (sidx + 1 < n_steps) beam_fetch_row<LT>(ring + ((sidx + 1) & 1) * row_buf, row_of(sidx + 1), W, p.tensor_lo, p.tensor_hi, lane);
+  beam_cp_async_commit();
+  beam_cp_async_wait<0>();
+  __syncwarp();
+  beam_team_barrier(team);
+  int done = 0;
+  for (;; ++sidx) {
+    beam_team_barrier(team);                                   // the workers' picks are in place
+    // ---- the K best of K * K picks: lane i looks at picks i and i + 32
+    unsigned long long c0 = 0ull, c1 = 0ull;
+    int32_t d0 = -1, d1 = -1;
+    if (lane < K * K) { c0 = sh.f_key[lane / K][lane % K]; d0 = sh.f_dst[lane / K][lane % K]; }
+    if (lane + 32 < K * K) { c1 = sh.f_key[(lane + 32) / K][(lane + 32) % K]; d1 = sh.f_dst[(lane + 32) / K][(lane + 32) % K]; }
+    unsigned long long mykey = 0ull;
+    int32_t mydst = -1;
+    for (int r = 0; r < K; ++r) {
+      const bool second = c1 > c0;
+      const unsigned long long a = second ? c1 : c0;
+      const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+      const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
+      const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+      const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
+      if (best == 0ull) break;
+      const bool mine = a == best;
+      const unsigned who = __ballot_sync(0xffffffffu, mine);
+      const int32_t dsel = __shfl_sync(0xffffffffu, second ? d1 : d0, __ffs(who) - 1);
+      if (lane == r) { mykey = best; mydst = dsel; }
+      if (mine) { if (second) c1 = 0ull; else c0 = 0ull; }
+    }
+    // ---- does the K-th pick clear everything that was not looked at?
+    bool ok = sh.f_fail == 0;
+    {
+      const unsigned long long key_last = shfl_u64(mykey, K - 1);
+      const float c_k = key_last != 0ull ? beam_key_value(key_last) : -INFINITY;
+      bool okk = true;
+      if (lane < K) { const float ub = sh.f_ub[lane]; okk = ub == -INFINITY || c_k > ub; }
+      ok = ok && __all_sync(0xffffffffu, okk);
+    }
+    if (!ok) {
+      if (lane == 0) sh.f_cmd = 1;
+      __syncwarp();
+      beam_team_barrier(team);
+      break;
+    }
+    // ---- the new hypotheses
+    int32_t parent = -1, token = -1, nstate = -1, nl = 0;
+    bool nlv = false;
+    float nsc = -INFINITY;
+    unsigned long long nh = 0ull;
+    {
+      const uint32_t l2 = 0xFFFFFFFFu - static_cast<uint32_t>(mykey & 0xFFFFFFFFull);
+      const int par_l = mykey != 0ull ? static_cast<int>(l2 & 31u) : 0;
+      const int32_t pst = __shfl_sync(0xffffffffu, st1, par_l), pl = __shfl_sync(0xffffffffu, hl, par_l);
+      const int plv = __shfl_sync(0xffffffffu, lv1 ? 1 : 0, par_l);
+      const unsigned long long ph = shfl_u64(hh, par_l);
+      if (lane < K && mykey != 0ull) {
+        const int tkey = static_cast<int>(l2 >> 5);
+        parent = par_l; nsc = beam_key_value(mykey);
+        token = tkey == V + 1 ? -1 : tkey;
+        nstate = pst;
+        nh = ph; nl = pl;
+        if (token >= 0 && token != V) {
+          nstate = mydst; nlv = plv != 0;
+          nh = (nh ^ static_cast<unsigned long long>(token + 1)) * 0xff51afd7ed558ccdull;
+          nh ^= nh >> 33;
+          nh += 0x9e3779b97f4a7c15ull;
+          ++nl;
+        }
+      }
+    }
+    sc = nsc; st = nstate; lv = nlv; hh = nh; hl = nl;
+    ++done;
+    const bool last = sidx + 1 >= n_steps;
+    if (!last) { frame_start(sidx + 1); publish(); }
+    if (lane == 0 && last) sh.f_cmd = 1;
+    beam_cp_async_wait<0>();                                   // the next step's row (asked for a step ago) is there
+    __syncwarp();
+    beam_team_barrier(team);                                   // the workers go on
+    // ---- off the critical path: this step's results, the row after the next
+    if (lane < K) {
+      const int64_t o = static_cast<int64_t>(b) * K + lane;
+      p.scores[o] = nsc; p.states[o] = nstate; p.live[o] = nlv ? 1 : 0;
+      p.out_parent[o] = parent; p.out_token[o] = token;
+      const bool odd = ((par0 + sidx) & 1) != 0;
+      (odd ? hashA : hashB)[o] = nh; (odd ? lenA : lenB)[o] = nl;
+      if (p.tree) {
+        const int32_t step = step_base + sidx;
+        const int64_t at = p.tree_cap > 0 ? static_cast<int64_t>(b) * p.tree_cap + (step % p.tree_cap)
+                                          : static_cast<int64_t>(step) * p.B + b;
+        p.tree[at * K + lane] = make_int2(parent, token);
+      }
+    }
+    if (last) break;
+    if (sidx + 2 < n_steps) beam_fetch_row<LT>(ring + (sidx & 1) * row_buf, row_of(sidx + 2), W, p.tensor_lo, p.tensor_hi, lane);
+    beam_cp_async_commit();
+  }
+  beam_cp_async_wait<0>();
+  if (lane < K) { sh.h_score[lane] = sc; sh.h_state[lane] = st; sh.h_live[lane] = lv ? 1 : 0; sh.h_hash[lane] = hh; sh.h_len[lane] = hl; }
+  if (lane == 0) sh.rec_ready = 0;
+  __syncwarp();
+  return done;
+}
+
+// Whether the team's steps apply to this launch and this block's stream.
+template <typename LT>
+__device__ __forceinline__ bool beam_fast_applies(const TbBeamParams& p) {
+  if (p.K > kFastMaxK || p.top_base == nullptr || p.tensor_lo == nullptr || p.top_m + 1 > 32) return false;
+  const TbSlotRec& rec = p.slots[blockIdx.x];
+  return rec.n_states <= 0 || (rec.n_rsent >= 0 && p.tokview);
 }
 
 // T frames of E rows in one launch: the block loops over the expansions of its stream; every hypothesis of the
@@ -890,14 +1274,33 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
 template <typename LT>
 __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
                                                           int64_t row_stride) {
+  __shared__ BeamShared sh;
   LT xpre[kBeamPref] = {};
   bool xpre_valid = false;
   TbTopEnt tpre{0.0f, 0.0f, 0u};
   bool tpre_valid = false;
   const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(blockIdx.x) * p.stream_stride;
-  for (int32_t t = 0; t < T; ++t) {
-    for (int32_t e = 0; e < E; ++e) {
-      const int32_t sidx = t * E + e;
+  extern __shared__ __align__(16) unsigned char dyn_all[];
+  const bool fast = beam_fast_applies<LT>(p);
+  int32_t skip = 0, backoff = 0;              // steps until the team tries again after a step it could not take
+  for (int32_t sidx = 0; sidx < T * E; ++sidx) {
+    if (fast && sidx > 0 && skip-- <= 0) {
+      if (threadIdx.x < 32 * (p.K + 1)) {
+        const int d = beam_fast_run<LT>(p, sh, dyn_all, sidx, T * E, E, frame_stride, row_stride, T * E, p.step,
+                                        const_cast<unsigned long long*>(p.hash_in), p.hash_out, const_cast<int32_t*>(p.len_in), p.len_out, 0);
+        if (threadIdx.x == 0) sh.fast_done = d;
+      }
+      __syncthreads();
+      const int d = sh.fast_done;
+      __syncthreads();                          // (read by everyone before a later run writes it again)
+      sidx += d;
+      backoff = d == 0 ? min(2 * backoff + 1, 32) : 0;
+      skip = backoff;
+      xpre_valid = false; tpre_valid = false;
+      if (sidx >= T * E) break;
+    }
+    {
+      const int32_t t = sidx / E, e = sidx - t * E;
       TbBeamParams q = p;
       q.logits = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
       q.hyp_stride = 0;
@@ -912,7 +1315,7 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, in
       const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
       const LT* next_row = nt < T ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
       const TbTopEnt* next_top = (nt < T && q.top_row) ? q.top_row + (p.top_m + 1) : nullptr;
-      beam_step_body<LT>(q, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
+      beam_step_body<LT>(q, sh, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
       __syncthreads();
     }
   }
@@ -1001,6 +1404,7 @@ template <typename LT>
 __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int32_t T, int32_t E, int64_t frame_stride,
                                                          int64_t row_stride, const int32_t* n_frames, int32_t* slot_pos,
                                                          unsigned long long* hash, int32_t* len, size_t n_hyp) {
+  __shared__ BeamShared sh;
   LT xpre[kBeamPref] = {};
   bool xpre_valid = false;
   TbTopEnt tpre{0.0f, 0.0f, 0u};
@@ -1009,9 +1413,27 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int
   const int32_t nf = n_frames ? max(0, min(T, n_frames[b])) : T;
   const int32_t pos0 = slot_pos[b];
   const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
-  for (int32_t t = 0; t < nf; ++t) {
-    for (int32_t e = 0; e < E; ++e) {
-      const int32_t sidx = t * E + e;
+  extern __shared__ __align__(16) unsigned char dyn_all[];
+  const bool fast = beam_fast_applies<LT>(p);
+  int32_t skip = 0, backoff = 0;
+  for (int32_t sidx = 0; sidx < nf * E; ++sidx) {
+    if (fast && sidx > 0 && skip-- <= 0) {
+      if (threadIdx.x < 32 * (p.K + 1)) {
+        const int d = beam_fast_run<LT>(p, sh, dyn_all, sidx, nf * E, E, frame_stride, row_stride, T * E, pos0, hash, hash + n_hyp,
+                                        len, len + n_hyp, pos0);
+        if (threadIdx.x == 0) sh.fast_done = d;
+      }
+      __syncthreads();
+      const int d = sh.fast_done;
+      __syncthreads();
+      sidx += d;
+      backoff = d == 0 ? min(2 * backoff + 1, 32) : 0;
+      skip = backoff;
+      xpre_valid = false; tpre_valid = false;
+      if (sidx >= nf * E) break;
+    }
+    {
+      const int32_t t = sidx / E, e = sidx - t * E;
       TbBeamParams q = p;
       q.logits = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
       q.hyp_stride = 0;
@@ -1027,7 +1449,7 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int
       const int32_t nt = e + 1 < E ? t : t + 1, ne = e + 1 < E ? e + 1 : 0;
       const LT* next_row = nt < nf ? stream_base + static_cast<int64_t>(nt) * frame_stride + static_cast<int64_t>(ne) * row_stride : nullptr;
       const TbTopEnt* next_top = (nt < nf && q.top_row) ? q.top_row + (p.top_m + 1) : nullptr;
-      beam_step_body<LT>(q, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
+      beam_step_body<LT>(q, sh, xpre, xpre_valid, next_row, tpre, tpre_valid, next_top);
       __syncthreads();
     }
   }
@@ -1165,13 +1587,29 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
+// The team steps of narrow beams (beam_fast_run) read rows through two buffers behind the block's other shared
+// memory and need the extent of the logits tensor; without either (a wide beam, odd strides) they stay off.
+static void beam_fast_setup(TbBeamParams* p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride, size_t* smem) {
+  p->tensor_lo = nullptr; p->tensor_hi = nullptr;
+  if (p->K > kFastMaxK || !p->top_base || p->stream_stride < 0 || frame_stride < 0 || row_stride < 0) return;
+  const size_t elem = p->dtype == TB_BF16 ? 2 : 4;
+  const size_t more = beam_ring_bytes(p->V, static_cast<int>(elem)) + 16;
+  if (*smem + more > 200 * 1024) return;
+  *smem += more;
+  const int64_t last = static_cast<int64_t>(p->B - 1) * p->stream_stride + static_cast<int64_t>(T - 1) * frame_stride +
+                       static_cast<int64_t>(E - 1) * row_stride + p->V;
+  p->tensor_lo = static_cast<const unsigned char*>(p->logits);
+  p->tensor_hi = p->tensor_lo + static_cast<size_t>(last + 1) * elem;
+}
+
 int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
                           cudaStream_t stream) {
   TbBeamParams p = p_in;
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
   const size_t aux = beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(p.V + 1) * sizeof(float);   // + the staged row
-  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
-                      ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
+  size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
+                ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
+  beam_fast_setup(&p, T, E, frame_stride, row_stride, &smem);
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
   int rc;
   if (p.dtype == TB_BF16) {
@@ -1287,8 +1725,9 @@ int tb_launch_beam_chunk(const TbBeamParams& p_in, int32_t T, int32_t E, int64_t
   TbBeamParams p = p_in;
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
   const size_t aux = beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(p.V + 1) * sizeof(float);   // + the staged row
-  const size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
-                      ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
+  size_t smem = ((static_cast<size_t>(p.K) * (p.V + 1) * sizeof(float) + 15) & ~size_t(15)) +
+                ((static_cast<size_t>(p.K) * ((p.V + 1 + 31) >> 5) * sizeof(uint32_t) + 15) & ~size_t(15)) + aux;
+  beam_fast_setup(&p, T, E, frame_stride, row_stride, &smem);
   if (smem > 200 * 1024) return TB_ERR_INVALID_ARG;
   int rc;
   if (p.dtype == TB_BF16) {

@@ -55,6 +55,8 @@ struct TbBeamParams {
   const struct TbTopEnt* top_base;
   int32_t top_m;
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
+  // first / one-past-last byte of the logits tensor of a multi-step launch (set by the launcher; null: not known)
+  const unsigned char* tensor_lo; const unsigned char* tensor_hi;
 };
 
 int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
