@@ -916,19 +916,18 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
 // registers, lane k: hypothesis k), warp k + 1 works for hypothesis k.  Per step
 //   worker k     : the hypothesis' list record, its listed tokens (exact values; logits from the row, which arrives
 //                  in shared memory by asynchronous copies the coordinator issues two steps ahead), blank, the first
-//                  unlisted tokens of the reduced row or the carried hypothesis -- at most 32 * kFastRL + 32
-//                  candidates in registers --, its K best of them in K rounds of two warp-wide integer maxima;
+//                  unlisted tokens of the reduced row or the carried hypothesis, every lane keeping the three best
+//                  of those it sees in registers; the K best of them in K rounds of two warp-wide integer maxima;
 //   barrier of the team (a named barrier, not the block's);
 //   coordinator  : the K best of the workers' picks, the same bound check as the block-wide compact path, the new
 //                  hypotheses, and, where the next step begins a frame, merging and pruning;
 //   barrier of the team; then the workers go on while the coordinator writes the step's results to global memory
 //                  and asks for the row after the next.
-// A step the team cannot take (a list of more than 32 * kFastRL tokens, the bound not cleared) is left untouched: the
+// A step the team cannot take (the bound not cleared, more than three picks due to one lane) is left untouched: the
 // run ends before it, the hypotheses go back to shared memory, and the whole block does that step with
 // beam_step_body.  Same arithmetic, same order of candidates, hence the same results bit for bit.
 constexpr int kFastMaxK = 8;      // widest beam of the team's steps
-constexpr int kFastRL = 3;        // a worker lane's registers for listed tokens (lists of up to 32 * kFastRL tokens)
-constexpr int kFastR = kFastRL + 1;
+constexpr int kFastMaxList = 2048; // longest list of boosted tokens a worker takes
 
 __device__ __forceinline__ unsigned long long beam_key(float v, int tkey, int k) {
   const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
@@ -1027,10 +1026,17 @@ __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& 
       const float sc1 = sh.f_sc[k];
       const int32_t st1 = sh.f_st[k];
       const bool lv1 = sh.f_lv[k] != 0;
-      unsigned long long ck[kFastR];
-      int32_t cd[kFastR];
-#pragma unroll
-      for (int j = 0; j < kFastR; ++j) { ck[j] = 0ull; cd[j] = -1; }
+      // a lane keeps the three best of the candidates it sees, best first (a step's K picks hardly ever include more
+      // than three of one lane's; if they might, the step is left to the whole block)
+      unsigned long long m0 = 0ull, m1 = 0ull, m2 = 0ull;
+      int32_t e0 = -1, e1 = -1, e2 = -1;
+      int n_seen = 0;
+      auto offer = [&](unsigned long long kk, int32_t dd) {
+        ++n_seen;
+        if (kk > m0) { m2 = m1; e2 = e1; m1 = m0; e1 = e0; m0 = kk; e0 = dd; }
+        else if (kk > m1) { m2 = m1; e2 = e1; m1 = kk; e1 = dd; }
+        else if (kk > m2) { m2 = kk; e2 = dd; }
+      };
       float D = 0.0f;
       if (sc1 != -INFINITY) {
         int32_t beg = 0, cnt = 0;
@@ -1042,20 +1048,18 @@ __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& 
         }
         const unsigned char* rowb = ring + (sidx & 1) * row_buf + (reinterpret_cast<uintptr_t>(row_of(sidx)) & 15);
         if (lv1) {
-          if (cnt > 32 * kFastRL) { if (lane == 0) sh.f_fail = 1; cnt = 0; }
+          if (cnt > kFastMaxList) { if (lane == 0) sh.f_fail = 1; cnt = 0; }
           for (int i = lane; i < WW; i += 32) ovr_k[i] = 0u;
           __syncwarp();
           // the listed tokens: exact values
-#pragma unroll
-          for (int j = 0; j < kFastRL; ++j) {
-            const int i = lane + 32 * j;
+          for (int i0 = 0; i0 < cnt; i0 += 32) {
+            const int i = i0 + lane;
             if (i < cnt) {
               const TbRsEnt en = ent[beg + i];
               const int tk = static_cast<int>((en.dst_tok & ((1u << TB_RS_TOK_BITS) - 1u)) >> 1);   // padding entries carry token V
               if (tk < V) {
                 const float x = beam_smem_logit<LT>(rowb, tk);
-                ck[j] = beam_key(__fadd_rn(sc1, __fadd_rn(x, en.lb)), tk, k);
-                cd[j] = static_cast<int32_t>(en.dst_tok >> TB_RS_TOK_BITS);
+                offer(beam_key(__fadd_rn(sc1, __fadd_rn(x, en.lb)), tk, k), static_cast<int32_t>(en.dst_tok >> TB_RS_TOK_BITS));
                 atomicOr(&ovr_k[tk >> 5], 1u << (tk & 31));
               }
             }
@@ -1063,44 +1067,36 @@ __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& 
           __syncwarp();
           // blank and the first unlisted tokens of the reduced row: lane j looks at its entry j
           if (lane == M) {
-            ck[kFastRL] = beam_key(__fadd_rn(sc1, tt.x), V, k); cd[kFastRL] = st1;
+            offer(beam_key(__fadd_rn(sc1, tt.x), V, k), st1);
           } else if (lane < M) {
             const int tk = static_cast<int>(tt.tok_cls & 0xFFFFu), cl = static_cast<int>(tt.tok_cls >> 16);
             if (tk < V && !((ovr_k[tk >> 5] >> (tk & 31)) & 1u)) {     // (tk >= V: the row has fewer tokens)
               const float val = bound ? __fadd_rn(tt.x, __fmul_rn(g.lambda, __fadd_rn(D, tv.rootcw[cl]))) : tt.x;
-              ck[kFastRL] = beam_key(__fadd_rn(sc1, val), tk, k);
-              cd[kFastRL] = bound ? tv.rootdst[cl] : -1;
+              offer(beam_key(__fadd_rn(sc1, val), tk, k), bound ? tv.rootdst[cl] : -1);
             }
           }
         } else if (lane == M) {
-          ck[kFastRL] = beam_key(sc1, V + 1, k); cd[kFastRL] = st1;      // a frozen hypothesis is carried
+          offer(beam_key(sc1, V + 1, k), st1);                             // a frozen hypothesis is carried
         }
       }
       // the K best of this hypothesis' candidates: lane r ends up with pick r
       unsigned long long mykey = 0ull;
       int32_t mydst = -1;
+      int taken = 0;
       for (int r = 0; r < K; ++r) {
-        unsigned long long a = ck[0];
-        int aj = 0;
-#pragma unroll
-        for (int jj = 1; jj < kFastR; ++jj) { const bool bt = ck[jj] > a; a = bt ? ck[jj] : a; aj = bt ? jj : aj; }
-        const uint32_t hi = static_cast<uint32_t>(a >> 32), lo = static_cast<uint32_t>(a);
+        const uint32_t hi = static_cast<uint32_t>(m0 >> 32), lo = static_cast<uint32_t>(m0);
         const uint32_t mh = __reduce_max_sync(0xffffffffu, hi);
         const uint32_t ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
         const unsigned long long best = (static_cast<unsigned long long>(mh) << 32) | ml;
         if (best == 0ull) break;                                  // (uniform: nothing left; the later picks stay empty)
-        const bool mine = a == best;
+        const bool mine = m0 == best;
         const unsigned who = __ballot_sync(0xffffffffu, mine);
-        int32_t dw = cd[0];
-#pragma unroll
-        for (int jj = 1; jj < kFastR; ++jj) dw = jj == aj ? cd[jj] : dw;
-        const int32_t dsel = __shfl_sync(0xffffffffu, dw, __ffs(who) - 1);
+        const int32_t dsel = __shfl_sync(0xffffffffu, e0, __ffs(who) - 1);
         if (lane == r) { mykey = best; mydst = dsel; }
-        if (mine) {
-#pragma unroll
-          for (int jj = 0; jj < kFastR; ++jj) ck[jj] = jj == aj ? 0ull : ck[jj];
-        }
+        if (mine) { m0 = m1; e0 = e1; m1 = m2; e1 = e2; m2 = 0ull; e2 = -1; ++taken; }
       }
+      // a lane whose three kept candidates were all picked while it had seen more: a fourth might have been due
+      if (__any_sync(0xffffffffu, taken == 3 && n_seen > 3) && lane == 0) sh.f_fail = 1;
       if (lane < K) { sh.f_key[k][lane] = mykey; sh.f_dst[k][lane] = mydst; }
       {
         // what the K-th pick of the step has to clear on behalf of this hypothesis (-inf: nothing)
