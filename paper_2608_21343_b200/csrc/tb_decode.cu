@@ -928,6 +928,7 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_step(TbBeamParams p) {
 // beam_step_body.  Same arithmetic, same order of candidates, hence the same results bit for bit.
 constexpr int kFastMaxK = 8;      // widest beam of the team's steps
 constexpr int kFastMaxList = 2048; // longest list of boosted tokens a worker takes
+constexpr int kFastRecCache = 48 << 10;   // shared memory for a copy of the stream's list records (graphs of up to 3072 states)
 
 __device__ __forceinline__ unsigned long long beam_key(float v, int tkey, int k) {
   const uint32_t u = __float_as_uint(v + 0.0f);             // -0 folded into +0: equal values, equal keys
@@ -981,6 +982,27 @@ __host__ __device__ inline size_t beam_ring_bytes(int V, int elem) {   // two ro
   return 2 * one + 16;
 }
 
+// Where the team keeps a copy of the stream's list records (16 bytes per graph state), behind the row buffers.
+template <typename LT>
+__device__ __forceinline__ TbRsRec* beam_rec_cache(const TbBeamParams& p, unsigned char* dyn) {
+  const int W = p.V + 1, WW = (W + 31) >> 5;
+  unsigned char* ovr = dyn + ((static_cast<size_t>(p.K) * W * sizeof(float) + 15) & ~size_t(15));
+  unsigned char* aux = ovr + ((static_cast<size_t>(p.K) * WW * sizeof(uint32_t) + 15) & ~size_t(15));
+  unsigned char* ring = aux + beam_aux_bytes(p.V, p.C, p.tokview) + static_cast<size_t>(W) * sizeof(float);
+  ring += (16 - (reinterpret_cast<uintptr_t>(ring) & 15)) & 15;
+  return reinterpret_cast<TbRsRec*>(ring + beam_ring_bytes(p.V, sizeof(LT)));
+}
+// Block-wide, once per launch: fills that copy if the stream's records fit.  Returns whether they do.
+template <typename LT>
+__device__ __forceinline__ bool beam_rec_cache_fill(const TbBeamParams& p, unsigned char* dyn) {
+  const TbSlotRec& rec = p.slots[blockIdx.x];
+  if (rec.n_states <= 0 || rec.n_rsent < 0 || static_cast<int64_t>(rec.n_states) * 16 > p.rec_cache_bytes) return false;
+  const uint4* src = reinterpret_cast<const uint4*>(p.arena + rec.blob_off + rec.off_rsrec);
+  uint4* dst = reinterpret_cast<uint4*>(beam_rec_cache<LT>(p, dyn));
+  for (int i = threadIdx.x; i < rec.n_states; i += blockDim.x) dst[i] = src[i];
+  return true;                                                  // (the barriers of the launch's first step come before any use)
+}
+
 __device__ __forceinline__ void beam_team_barrier(int n_threads) { asm volatile("bar.sync 1, %0;" ::"r"(n_threads) : "memory"); }
 
 // Takes the steps sidx, sidx + 1, ... of the block's stream as long as it can; returns (on warp 0) how many it took.
@@ -990,7 +1012,8 @@ template <typename LT>
 __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& sh, unsigned char* dyn, int32_t sidx, const int32_t n_steps,
                                              const int32_t E, const int64_t frame_stride, const int64_t row_stride,
                                              const int32_t rows_per_stream, const int32_t step_base, unsigned long long* hashA,
-                                             unsigned long long* hashB, int32_t* lenA, int32_t* lenB, const int32_t par0) {
+                                             unsigned long long* hashB, int32_t* lenA, int32_t* lenB, const int32_t par0,
+                                             const bool recs_cached) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int b = blockIdx.x, K = p.K, V = p.V, W = V + 1, M = p.top_m, WW = (W + 31) >> 5;
   const int team = 32 * (K + 1);
@@ -1015,7 +1038,7 @@ __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& 
     TokView tv;
     tokview_attach(tv, aux, V, p.C);
     const TbTopEnt* top0 = p.top_base + static_cast<int64_t>(b) * rows_per_stream * (M + 1);
-    const TbRsRec* rsrec = reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec);
+    const TbRsRec* rsrec = recs_cached ? beam_rec_cache<LT>(p, dyn) : reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec);
     const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
     uint32_t* ovr_k = ovr + k * WW;
     beam_team_barrier(team);                                   // the coordinator has set up the first step
@@ -1278,12 +1301,14 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_frames(TbBeamParams p, in
   const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(blockIdx.x) * p.stream_stride;
   extern __shared__ __align__(16) unsigned char dyn_all[];
   const bool fast = beam_fast_applies<LT>(p);
+  const bool recs_cached = fast && beam_rec_cache_fill<LT>(p, dyn_all);
   int32_t skip = 0, backoff = 0;              // steps until the team tries again after a step it could not take
   for (int32_t sidx = 0; sidx < T * E; ++sidx) {
     if (fast && sidx > 0 && skip-- <= 0) {
       if (threadIdx.x < 32 * (p.K + 1)) {
         const int d = beam_fast_run<LT>(p, sh, dyn_all, sidx, T * E, E, frame_stride, row_stride, T * E, p.step,
-                                        const_cast<unsigned long long*>(p.hash_in), p.hash_out, const_cast<int32_t*>(p.len_in), p.len_out, 0);
+                                        const_cast<unsigned long long*>(p.hash_in), p.hash_out, const_cast<int32_t*>(p.len_in), p.len_out, 0,
+                                        recs_cached);
         if (threadIdx.x == 0) sh.fast_done = d;
       }
       __syncthreads();
@@ -1411,12 +1436,13 @@ __global__ void __launch_bounds__(kBeamThreads) k_beam_chunk(TbBeamParams p, int
   const LT* stream_base = reinterpret_cast<const LT*>(p.logits) + static_cast<int64_t>(b) * p.stream_stride;
   extern __shared__ __align__(16) unsigned char dyn_all[];
   const bool fast = beam_fast_applies<LT>(p);
+  const bool recs_cached = fast && beam_rec_cache_fill<LT>(p, dyn_all);
   int32_t skip = 0, backoff = 0;
   for (int32_t sidx = 0; sidx < nf * E; ++sidx) {
     if (fast && sidx > 0 && skip-- <= 0) {
       if (threadIdx.x < 32 * (p.K + 1)) {
         const int d = beam_fast_run<LT>(p, sh, dyn_all, sidx, nf * E, E, frame_stride, row_stride, T * E, pos0, hash, hash + n_hyp,
-                                        len, len + n_hyp, pos0);
+                                        len, len + n_hyp, pos0, recs_cached);
         if (threadIdx.x == 0) sh.fast_done = d;
       }
       __syncthreads();
@@ -1586,12 +1612,14 @@ int tb_launch_beam_step(const TbBeamParams& p_in, cudaStream_t stream) {
 // The team steps of narrow beams (beam_fast_run) read rows through two buffers behind the block's other shared
 // memory and need the extent of the logits tensor; without either (a wide beam, odd strides) they stay off.
 static void beam_fast_setup(TbBeamParams* p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride, size_t* smem) {
-  p->tensor_lo = nullptr; p->tensor_hi = nullptr;
+  p->tensor_lo = nullptr; p->tensor_hi = nullptr; p->rec_cache_bytes = 0;
   if (p->K > kFastMaxK || !p->top_base || p->stream_stride < 0 || frame_stride < 0 || row_stride < 0) return;
   const size_t elem = p->dtype == TB_BF16 ? 2 : 4;
   const size_t more = beam_ring_bytes(p->V, static_cast<int>(elem)) + 16;
   if (*smem + more > 200 * 1024) return;
   *smem += more;
+  p->rec_cache_bytes = 0;
+  if (*smem + kFastRecCache <= 200 * 1024) { p->rec_cache_bytes = kFastRecCache; *smem += kFastRecCache; }
   const int64_t last = static_cast<int64_t>(p->B - 1) * p->stream_stride + static_cast<int64_t>(T - 1) * frame_stride +
                        static_cast<int64_t>(E - 1) * row_stride + p->V;
   p->tensor_lo = static_cast<const unsigned char*>(p->logits);

@@ -57,6 +57,7 @@ struct TbBeamParams {
   const TbSlotRec* slots; const unsigned char* arena; const int32_t* cls; int32_t* status;
   // first / one-past-last byte of the logits tensor of a multi-step launch (set by the launcher; null: not known)
   const unsigned char* tensor_lo; const unsigned char* tensor_hi;
+  int32_t rec_cache_bytes;   // shared memory set aside for a copy of the stream's list records (narrow beams; 0: none)
 };
 
 int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
