@@ -1041,11 +1041,13 @@ __device__ __forceinline__ int beam_fast_run(const TbBeamParams& p, BeamShared& 
     const TbRsRec* rsrec = recs_cached ? beam_rec_cache<LT>(p, dyn) : reinterpret_cast<const TbRsRec*>(blob + rec.off_rsrec);
     const TbRsEnt* ent = reinterpret_cast<const TbRsEnt*>(blob + rec.off_rsent);
     uint32_t* ovr_k = ovr + k * WW;
+    TbTopEnt tnext{-INFINITY, -INFINITY, 0xFFFFu};
+    if (lane <= M) tnext = top0[static_cast<int64_t>(sidx) * (M + 1) + lane];
     beam_team_barrier(team);                                   // the coordinator has set up the first step
     for (;; ++sidx) {
       if (sh.f_cmd != 0) break;
-      TbTopEnt tt{-INFINITY, -INFINITY, 0xFFFFu};
-      if (lane <= M) tt = top0[static_cast<int64_t>(sidx) * (M + 1) + lane];
+      const TbTopEnt tt = tnext;                               // (lane j: entry j of this step's reduced row, asked for a step ago)
+      if (sidx + 1 < n_steps && lane <= M) tnext = top0[static_cast<int64_t>(sidx + 1) * (M + 1) + lane];
       const float sc1 = sh.f_sc[k];
       const int32_t st1 = sh.f_st[k];
       const bool lv1 = sh.f_lv[k] != 0;
