@@ -332,3 +332,65 @@ def test_beam_frames_when_the_reduced_rows_do_not_suffice(tb, K):
             fin = np.isfinite(ref["scores"])
             assert np.array_equal(np.isfinite(out["scores"][i]), fin)
             assert np.all(np.abs(out["scores"][i][fin] - ref["scores"][fin]) <= SCORE_TOL), (flags, i)
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_beam_frames_random_configurations(tb, block):
+    """Random small configurations of tb_beam_frames against the oracle: beams of 1 to 32 (narrow ones are decoded by a
+    team of warps, wide ones by the whole block), vocabularies of 4 to 1024, 1-3 expansions per frame, fp32 and bf16,
+    bound and unbound streams, with and without merging and pruning, each decode cut into random chunks."""
+    for seed in range(30 * block, 30 * block + 30):
+        rng = np.random.default_rng(41000 + seed)
+        V = int(rng.choice([4, 8, 30, 200, 1024]))
+        B, T, E = int(rng.integers(1, 5)), int(rng.integers(2, 40)), int(rng.integers(1, 4))
+        K = int(rng.choice([1, 2, 3, 4, 5, 8, 16, 32]))
+        f32 = bool(rng.integers(0, 2))
+        cc = (np.arange(V) // int(rng.integers(1, 4))).astype(np.int32)
+        lists = [None if rng.random() < 0.3 else
+                 [[int(t) for t in rng.integers(0, V, size=rng.integers(1, 5))] for _ in range(int(rng.integers(1, 12)))]
+                 for _ in range(B)]
+        lam = float(rng.choice([0.125, 0.5, 1.0]))
+        x = (rng.standard_normal((B, T, E, V + 1)) * float(rng.choice([0.05, 0.3, 1.0]))).astype(np.float32)
+        x[:, :, 0, V] += 2.0
+        if E > 1:
+            x[:, :, 1:, :V] -= 2.0
+        x = W.round_to_dtype(x, "f32" if f32 else "bf16")
+        xs = x if f32 else W.to_storage(x, "bf16")
+        merge = bool(rng.integers(0, 4) != 0)
+        delta = float(rng.choice([0.5, 2.0, 8.0])) if rng.random() < 0.5 else None
+        batch = tb.tb_batch_create(V, cc, B, arena_bytes=8 << 20, max_beam=K, max_tree_steps=T * E)
+        if delta is not None:
+            tb.tb_batch_set_beam_prune(batch, delta)
+        for i, p in enumerate(lists):
+            tb.tb_batch_bind_stream(batch, i, None if p is None else tb.tb_graph_compile(p, V, case_class=cc, lam=lam))
+        t = to_device(xs)
+        dev = t.device
+        scores = torch.full((B, K), float("-inf"), device=dev)
+        scores[:, 0] = 0.0
+        states = torch.full((B, K), -1, dtype=torch.int32, device=dev)
+        states[:, 0] = torch.tensor([0 if p is not None else -1 for p in lists], dtype=torch.int32, device=dev)
+        live = torch.zeros((B, K), dtype=torch.uint8, device=dev)
+        par = torch.empty((B, K), dtype=torch.int32, device=dev)
+        tok = torch.empty((B, K), dtype=torch.int32, device=dev)
+        tb.tb_beam_reset(batch)
+        t0 = 0
+        while t0 < T:
+            n = int(rng.integers(1, T - t0 + 1))
+            tb.tb_beam_frames(batch, t[:, t0:t0 + n], merge, scores, states, live, par, tok)
+            t0 += n
+        toks, lens = tb.tb_beam_backtrace(batch, B, K, T * E)
+        torch.cuda.synchronize()
+        assert tb.tb_batch_status(batch) == 0, seed
+        sc, stt, toks, lens = scores.cpu().numpy(), states.cpu().numpy(), toks.cpu().numpy(), lens.cpu().numpy()
+        last = torch.stack([par, tok], dim=-1).cpu().numpy()
+        for i in range(B):
+            g = None if lists[i] is None else O.Graph(lists[i], V, case_class=cc, lam=lam)
+            ref = O.beam_decode(g, xs[i], K, merge=merge, prune_delta=-1.0 if delta is None else delta)
+            fin = np.isfinite(ref["scores"])
+            what = (seed, i, dict(V=V, T=T, E=E, K=K, f32=f32, merge=merge, delta=delta))
+            assert np.array_equal(stt[i], ref["states"]) and np.array_equal(lens[i], ref["lens"]), what
+            assert np.array_equal(last[i], ref["tree"][-1]), what
+            assert np.array_equal(np.isfinite(sc[i]), fin) and np.all(np.abs(sc[i][fin] - ref["scores"][fin]) <= SCORE_TOL), what
+            for k in range(K):
+                assert np.array_equal(toks[i, k, :ref["lens"][k]], ref["tokens"][k]), what
+        batch.destroy()
