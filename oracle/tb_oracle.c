@@ -32,7 +32,9 @@
  * beam decoding with K smaller than the number of alignments on large inputs, TDT with
  * durations that vary from row to row (pinned by a hand-worked case and by the reductions
  * "all durations 0 = the RNNT rule" and "all durations d = the unit case on every d-th
- * frame"), and the stream-churn schedule.
+ * frame"), and the stream-churn schedule.  The order of equal beam candidates (value, token, parent) has a
+ * hand-worked pin of its own; the normalised decode (orc_row_lse, orc_greedy_rnnt_lsm) is pinned against a
+ * library log-sum-exp, closed forms, exact shifts of whole rows and the un-normalised decode.
  *
  * Arithmetic: potentials in double, each stored value rounded once to float; every
  * run-time sum is a float add in the order written, compiled with -ffp-contract=off so
