@@ -1379,23 +1379,29 @@ __global__ void __launch_bounds__(kTopWarps * 32) k_beam_topm(const LT* logits, 
   const LT* row = logits + static_cast<int64_t>(b) * stream_stride + static_cast<int64_t>(t) * frame_stride + static_cast<int64_t>(e) * row_stride;
   TbTopEnt* o = out + (static_cast<int64_t>(b) * rows_per_stream + r) * (top_m + 1);
   float* y = ybuf + static_cast<size_t>(warp) * V;
-  // y of every token, this lane's best (value, lowest token) on the way
-  float bv = -INFINITY;
-  int bi = INT32_MAX;
+  // y of every token; on the way every lane keeps the three best of its strip (value descending, token ascending:
+  // the strip is walked in ascending token order, so a strict comparison keeps the lower token among equals)
+  float v0 = -INFINITY, v1 = -INFINITY, v2 = -INFINITY;
+  int i0 = INT32_MAX, i1 = INT32_MAX, i2 = INT32_MAX;
+  int n_strip = 0;
+#pragma unroll 4
   for (int v = lane; v < V; v += 32) {
     const float x = LogitLoad<LT>::at(row + v);
     const float yv = bound ? __fadd_rn(x, __fmul_rn(g.lambda, rootcw[__ldg(cls + v)])) : x;
     y[v] = yv;
-    if (yv > bv) { bv = yv; bi = v; }
+    ++n_strip;
+    if (yv > v0 || i0 == INT32_MAX) { v2 = v1; i2 = i1; v1 = v0; i1 = i0; v0 = yv; i0 = v; }
+    else if (yv > v1 || i1 == INT32_MAX) { v2 = v1; i2 = i1; v1 = yv; i1 = v; }
+    else if (yv > v2 || i2 == INT32_MAX) { v2 = yv; i2 = v; }
   }
-  if (bi == INT32_MAX && lane < V) bi = lane;                 // every value of the strip is -inf: still a token
   __syncwarp();
+  int n_taken = 0;      // of this lane's strip
   for (int m = 0; m <= top_m; ++m) {
     // the warp's best: largest value, then lowest token
-    const uint32_t u = __float_as_uint(bv + 0.0f);
-    const uint32_t key = bi == INT32_MAX ? 0u : (u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u));
+    const uint32_t u = __float_as_uint(v0 + 0.0f);
+    const uint32_t key = i0 == INT32_MAX ? 0u : (u ^ ((u >> 31) ? 0xFFFFFFFFu : 0x80000000u));
     const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
-    const uint32_t imin = __reduce_min_sync(0xffffffffu, (key == kmax && bi != INT32_MAX) ? static_cast<uint32_t>(bi) : 0xFFFFFFFFu);
+    const uint32_t imin = __reduce_min_sync(0xffffffffu, (key == kmax && i0 != INT32_MAX) ? static_cast<uint32_t>(i0) : 0xFFFFFFFFu);
     const bool none = imin == 0xFFFFFFFFu;                    // fewer than m + 1 tokens in the row
     if (m == top_m) {
       if (lane == 0) { o[m].y = none ? -INFINITY : y[imin]; o[m].x = LogitLoad<LT>::at(row + V); o[m].tok_cls = 0u; }
@@ -1405,16 +1411,22 @@ __global__ void __launch_bounds__(kTopWarps * 32) k_beam_topm(const LT* logits, 
       if (none) { o[m].y = -INFINITY; o[m].x = -INFINITY; o[m].tok_cls = 0xFFFFu; }
       else { o[m].y = y[imin]; o[m].x = LogitLoad<LT>::at(row + imin); o[m].tok_cls = imin | (static_cast<uint32_t>(__ldg(cls + imin)) << 16); }
     }
-    if (!none && static_cast<uint32_t>(bi) == imin) {
-      // the owner takes it out and looks for its next best
-      y[bi] = __int_as_float(0x7FC00000);                     // (a NaN: never greater than anything, never chosen again)
-      bv = -INFINITY; bi = INT32_MAX;
-      int first_left = INT32_MAX;
-      for (int v = lane; v < V; v += 32) {
-        const float yv = y[v];
-        if (yv == yv) { if (first_left == INT32_MAX) first_left = v; if (yv > bv) { bv = yv; bi = v; } }
+    if (!none && static_cast<uint32_t>(i0) == imin) {
+      // the owner takes it out: its next best moves up; when the three it kept are used up and the strip holds
+      // more, it looks through the strip again
+      y[i0] = __int_as_float(0x7FC00000);                     // (a NaN: never greater than anything, never chosen again)
+      ++n_taken;
+      v0 = v1; i0 = i1; v1 = v2; i1 = i2; v2 = -INFINITY; i2 = INT32_MAX;
+      if (i0 == INT32_MAX && n_taken < n_strip) {
+        for (int v = lane; v < V; v += 32) {
+          const float yv = y[v];
+          if (yv == yv) {
+            if (yv > v0 || i0 == INT32_MAX) { v2 = v1; i2 = i1; v1 = v0; i1 = i0; v0 = yv; i0 = v; }
+            else if (yv > v1 || i1 == INT32_MAX) { v2 = v1; i2 = i1; v1 = yv; i1 = v; }
+            else if (yv > v2 || i2 == INT32_MAX) { v2 = yv; i2 = v; }
+          }
+        }
       }
-      if (bi == INT32_MAX) bi = first_left;                   // only -inf values left in the strip
     }
     __syncwarp();
   }
