@@ -509,7 +509,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, BeamShared
     tpre_valid = false;
     if (next_top) { if (threadIdx.x <= M) tpre = next_top[threadIdx.x]; tpre_valid = true; }
     // (one warp doing a narrow beam's few dozen candidates by itself, with warp-wide synchronisation only, was
-    // measured slower than the whole block: 8.4 against 6.9 ms per utterance at K = 4)
+    // measured slower than the whole block; narrow beams are taken by a team of warps instead, see beam_fast_run)
     const int cth = static_cast<int>(threadIdx.x), cnt = kBeamThreads;
     {
       if (cp_flag) {
@@ -977,7 +977,7 @@ __device__ __forceinline__ void beam_fetch_row(unsigned char* buf, const LT* row
     }
   }
 }
-__host__ __device__ inline size_t beam_ring_bytes(int V, int elem) {   // two row buffers of the lone-warp steps
+__host__ __device__ inline size_t beam_ring_bytes(int V, int elem) {   // two row buffers of the team steps
   const size_t one = ((static_cast<size_t>(V + 1) * elem + 16 + 15) & ~size_t(15)) + 16;
   return 2 * one + 16;
 }
