@@ -117,7 +117,10 @@ def _host(a, dtype):
 
 
 def _hp(a):
-    return None if a is None else a.ctypes.data_as(_vp)
+    # (the address from the array interface: numpy's .ctypes helper object costs several microseconds per call)
+    if a is None or isinstance(a, C.Array):        # (a ctypes array is passed as it is)
+        return a
+    return _vp(a.__array_interface__["data"][0])
 
 
 def _dp(t):
@@ -363,12 +366,13 @@ TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
 
 def tb_batch_bind_streams(batch: Batch, slots, graphs, stream=None):
     """Bind graphs[i] (None: unbind) to slots[i], all in one copy and one launch."""
-    sl = _host(slots, np.int32)
-    assert len(sl) == len(graphs)
-    if len(sl) == 0:
+    n = len(graphs)
+    assert len(slots) == n
+    if n == 0:
         return
-    arr = (_vp * len(graphs))(*[None if g is None else g.handle for g in graphs])
-    _check(_lib.tb_batch_bind_streams(batch.handle, len(sl), _hp(sl), arr, _stream(stream)), "tb_batch_bind_streams")
+    sl = (_i32 * n)(*[int(x) for x in slots])
+    arr = (_vp * n)(*[None if g is None else g.handle for g in graphs])
+    _check(_lib.tb_batch_bind_streams(batch.handle, n, sl, arr, _stream(stream)), "tb_batch_bind_streams")
 
 
 def tb_batch_set_flags(batch: Batch, flags: int):
@@ -398,7 +402,7 @@ def tb_batch_status(batch: Batch, stream=None) -> int:
 
 def _strides4(t: torch.Tensor):
     assert t.dim() == 4
-    return np.array(t.stride(), dtype=np.int64)
+    return (_i64 * 4)(*t.stride())
 
 
 def tb_greedy_decode(batch: Batch, logits: torch.Tensor, lengths=None, out=None, stream=None) -> dict:
