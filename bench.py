@@ -273,9 +273,10 @@ def side_measurement(args):
             if args.single_binds:
                 for sl, g in gs:
                     tb.tb_batch_bind_stream(batch, sl, g)
+                outs = tb.tb_stream_chunk(batch, dl, w.n_dur, dv, out=outs)      # the result tensors are allocated once
             else:
-                tb.tb_batch_bind_streams(batch, [sl for sl, _ in gs], [g for _, g in gs])   # one copy, one launch
-            outs = tb.tb_stream_chunk(batch, dl, w.n_dur, dv, out=outs)          # the result tensors are allocated once
+                # the new streams' binds (one copy, one launch) and the chunk in one call
+                outs = tb.tb_stream_chunk_binds(batch, [sl for sl, _ in gs], [g for _, g in gs], dl, w.n_dur, dv, out=outs)
             b.record()
             host_us.append((time.perf_counter() - th) * 1e6)
             torch.cuda.synchronize()
@@ -286,7 +287,7 @@ def side_measurement(args):
                           "p99": float(np.percentile(lat, 99)), "unit": "ms", "higher_is_better": False, "n_gpus": 1,
                           "config": {"workload": w.name, "slots": w.B, "chunk_frames": w.chunk, "chunks": len(lat),
                                      "binds_in_timed_region": True, "rebinds": binds - w.B,
-                                     "binds": "one by one" if args.single_binds else "tb_batch_bind_streams (one copy + one launch per chunk)"},
+                                     "binds": "one by one" if args.single_binds else "tb_stream_chunk_binds (binds in one copy + one launch, then the chunk, one call)"},
                           "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
                           "host_issue_us_p50": float(np.percentile(np.array(host_us[10:]), 50)),
                           "graph_compile_ms_per_list": 1e3 * t_compile / max(1, binds),

@@ -402,6 +402,20 @@ int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots,
                     float *out_scores, int32_t *out_states, int32_t *out_cursors, void *stream);
 
 /*
+ * The streams that start with a chunk and the chunk itself in one call (Sec. 2.2 para. 4, Sec. 2.3): first
+ * tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream), then tb_stream_chunk with the remaining
+ * arguments, both enqueued on `stream`.  A server that gets its new streams' lists with the audio saves one trip
+ * through its language binding per chunk; nothing else differs from the two calls made one after the other.
+ * n_binds may be 0 (bind_slots / bind_graphs are then not read).  If the binds fail the chunk is not decoded.
+ * Errors: those of the two calls.
+ */
+int tb_stream_chunk_binds(tb_batch *b, int32_t n_binds, const int32_t *bind_slots, const tb_graph *const *bind_graphs,
+                          const void *logits, int dtype, int32_t n_slots, int32_t chunk, int32_t S, int32_t n_dur,
+                          const int64_t *strides, const int32_t *valid_frames, int32_t *out_tokens, int32_t *out_frames,
+                          int32_t *out_durs, int32_t *out_counts, float *out_scores, int32_t *out_states,
+                          int32_t *out_cursors, void *stream);
+
+/*
  * Forget the hypothesis tree (step counter = 0) and the per-hypothesis record of emitted token sequences (every
  * hypothesis starts from the empty sequence).  Call before the first step of an utterance (host bookkeeping only:
  * no device work, so it may sit inside a stream capture).  Across the chunks of one utterance simply keep calling

@@ -80,6 +80,8 @@ _SIGS = {
     "tb_greedy_decode": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_stream_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                   _vp, _vp, _vp]),
+    "tb_stream_chunk_binds": (C.c_int, [_vp, _i32, _vp, _vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                                        _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_reset": (C.c_int, [_vp]),
     "tb_beam_step": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_beam_backtrace": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
@@ -444,6 +446,32 @@ def tb_stream_chunk(batch: Batch, logits: torch.Tensor, n_dur: int, valid_frames
                                 _dp(valid_frames), _dp(out["tokens"]), _dp(out["frames"]), _dp(out.get("durs")),
                                 _dp(out["counts"]), _dp(out["scores"]), _dp(out["states"]), _dp(out.get("cursors")),
                                 _stream(stream)), "tb_stream_chunk")
+    return out
+
+
+def tb_stream_chunk_binds(batch: Batch, slots, graphs, logits: torch.Tensor, n_dur: int, valid_frames: torch.Tensor,
+                          out=None, stream=None) -> dict:
+    """tb_batch_bind_streams(batch, slots, graphs) followed by tb_stream_chunk(batch, logits, ...), in one call."""
+    n, chunk, S, W = logits.shape
+    if W != batch.vocab + 1 + n_dur:
+        raise ValueError("last dimension must be vocab + 1 + n_dur")
+    nb = len(graphs)
+    assert len(slots) == nb
+    dev = logits.device
+    if out is None:
+        out = dict(tokens=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   frames=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   durs=torch.empty((n, chunk * S), dtype=torch.int32, device=dev),
+                   counts=torch.empty(n, dtype=torch.int32, device=dev),
+                   scores=torch.empty(n, dtype=torch.float32, device=dev),
+                   states=torch.empty(n, dtype=torch.int32, device=dev),
+                   cursors=torch.empty(n, dtype=torch.int32, device=dev))
+    sl = (_i32 * nb)(*[int(x) for x in slots]) if nb else None
+    arr = (_vp * nb)(*[None if g is None else g.handle for g in graphs]) if nb else None
+    _check(_lib.tb_stream_chunk_binds(batch.handle, nb, sl, arr, _dp(logits), _logit_dtype(logits), n, chunk, S, n_dur,
+                                      _strides4(logits), _dp(valid_frames), _dp(out["tokens"]), _dp(out["frames"]),
+                                      _dp(out.get("durs")), _dp(out["counts"]), _dp(out["scores"]), _dp(out["states"]),
+                                      _dp(out.get("cursors")), _stream(stream)), "tb_stream_chunk_binds")
     return out
 
 

@@ -806,6 +806,20 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
 }
 
+extern "C" int tb_stream_chunk_binds(tb_batch* b, int32_t n_binds, const int32_t* bind_slots, const tb_graph* const* bind_graphs,
+                                     const void* logits, int dtype, int32_t n_slots, int32_t chunk, int32_t S, int32_t n_dur,
+                                     const int64_t* strides, const int32_t* valid_frames, int32_t* out_tokens,
+                                     int32_t* out_frames, int32_t* out_durs, int32_t* out_counts, float* out_scores,
+                                     int32_t* out_states, int32_t* out_cursors, void* stream_) {
+  if (!b || n_binds < 0) return TB_ERR_INVALID_ARG;
+  if (n_binds > 0) {
+    const int rc = tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream_);
+    if (rc != TB_OK) return rc;
+  }
+  return tb_stream_chunk(b, logits, dtype, n_slots, chunk, S, n_dur, strides, valid_frames, out_tokens, out_frames, out_durs,
+                         out_counts, out_scores, out_states, out_cursors, stream_);
+}
+
 // The beam pre-pass for a launch that covers T * E rows per stream: reduces every row to its few best root-boosted
 // tokens (tb_launch_beam_topm) into memory of the batch and points the step parameters at the result.  Skipped (the
 // steps then look at whole rows) when the batch asks for it, when the memory would have to grow while the stream is

@@ -260,7 +260,21 @@ def test_binding_many_streams_at_once(tb):
     tb.tb_batch_bind_streams(batch, [0, 3], [graphs[0], graphs[3]])
     ch = to_host(tb.tb_stream_chunk(batch, logits[:, :8], 0, valid))
     assert ch["cursors"][0] == 8 and ch["cursors"][3] == 8 and ch["cursors"][1] == 16
+    # binds and chunk in one call: the same as the two calls
+    tb.tb_batch_bind_streams(batch, [0, 3], [graphs[0], graphs[3]])
+    want = to_host(tb.tb_stream_chunk(batch, logits[:, :8], 0, valid))
+    got = to_host(tb.tb_stream_chunk_binds(batch, [0, 3], [graphs[0], graphs[3]], logits[:, :8], 0, valid))
+    for i in (0, 3):
+        n = int(want["counts"][i])
+        assert int(got["counts"][i]) == n and np.array_equal(got["tokens"][i, :n], want["tokens"][i, :n])
+        assert got["scores"][i] == want["scores"][i] and got["states"][i] == want["states"][i] and got["cursors"][i] == 8
+    assert got["cursors"][1] == want["cursors"][1] + 8                    # the other slots went on
+    more = to_host(tb.tb_stream_chunk_binds(batch, [], [], logits[:, 8:16], 0, valid))      # no binds: a plain chunk
+    assert more["cursors"][0] == 16
     # errors: checked before anything changes
+    with pytest.raises(tb.TbError) as e:
+        tb.tb_stream_chunk_binds(batch, [0, 0], [graphs[0], graphs[1]], logits[:, :8], 0, valid)
+    assert e.value.code == tb.TB_ERR_INVALID_ARG
     with pytest.raises(tb.TbError) as e:
         tb.tb_batch_bind_streams(batch, [0, 0], [graphs[0], graphs[1]])
     assert e.value.code == tb.TB_ERR_INVALID_ARG
