@@ -339,7 +339,7 @@ def side_measurement(args):
                 ended = [sl for sl in range(w.B) if left[sl] > 0 and served[sl] >= total[sl]]
                 if ended:
                     tb.tb_apply_final_weights_slots(batch, ended, scores, states)
-                    tb.tb_beam_backtrace_slots(batch, w.B, K, 256, out=bt)
+                    tb.tb_beam_backtrace_slot_list(batch, ended, K, 256, out=bt)    # the transcripts of the streams that ended
                 b.record()
                 torch.cuda.synchronize()
                 lat.append(a.elapsed_time(b)); kern.append(m0.elapsed_time(m1))

@@ -489,6 +489,9 @@ int tb_beam_frames(tb_batch *b, const void *logits, int dtype, int32_t B, int32_
  *   reset of all slots to the next.  Errors: TB_ERR_INVALID_ARG (no tree, K, a batch-wide tree in use), TB_ERR_CUDA.
  * tb_beam_backtrace_slots: as tb_beam_backtrace, each slot walked back to the start of its own utterance; an
  *   utterance longer than the slot's ring sets TB_STATUS_STEP_LIMIT and yields the tokens still in the ring.
+ * tb_beam_backtrace_slot_list: the same for the n slots that `slots` (host int32 [n]) names, e.g. those whose streams
+ *   have just ended: out_tokens device int32 [n, K, max_len], out_lens device int32 [n, K], row i for slots[i].
+ *   Errors: TB_ERR_BAD_SLOT, TB_ERR_INVALID_ARG, TB_ERR_CUDA.
  * tb_apply_final_weights_slots: tb_apply_final_weights for the rows of the [n_slots, K] arrays that `slots` (host
  *   int32 [n]) names.
  */
@@ -500,6 +503,8 @@ int tb_beam_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots, i
                   float *scores, int32_t *states, uint8_t *live, int32_t *out_parent, int32_t *out_token, void *stream);
 int tb_beam_backtrace_slots(tb_batch *b, int32_t n_slots, int32_t K, int32_t max_len, int32_t *out_tokens,
                             int32_t *out_lens, void *stream);
+int tb_beam_backtrace_slot_list(tb_batch *b, int32_t n, const int32_t *slots, int32_t K, int32_t max_len, int32_t *out_tokens,
+                                int32_t *out_lens, void *stream);
 int tb_apply_final_weights_slots(tb_batch *b, int32_t n, const int32_t *slots, int32_t K, float *scores,
                                  const int32_t *states, void *stream);
 

@@ -93,6 +93,7 @@ _SIGS = {
     "tb_beam_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp,
                                 _vp, _vp]),
     "tb_beam_backtrace_slots": (C.c_int, [_vp, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "tb_beam_backtrace_slot_list": (C.c_int, [_vp, _i32, _vp, _i32, _i32, _vp, _vp, _vp]),
     "tb_apply_final_weights_slots": (C.c_int, [_vp, _i32, _vp, _i32, _vp, _vp, _vp]),
     "tb_batch_set_beam_prune": (C.c_int, [_vp, C.c_float]),
     "tb_greedy_decode_noalloc": (C.c_int, [C.c_int, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
@@ -548,6 +549,26 @@ def tb_beam_backtrace_slots(batch: Batch, n_slots: int, K: int, max_len: int, st
     _check(_lib.tb_beam_backtrace_slots(batch.handle, n_slots, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
            "tb_beam_backtrace_slots")
     return toks, lens
+
+
+def tb_beam_backtrace_slot_list(batch: Batch, slots, K: int, max_len: int, stream=None, out=None):
+    """Transcripts of the slots in ``slots`` only: (tokens int32 [n, K, max_len], lens int32 [n, K]); ``out``: tensors of
+    at least that many rows to write into (their first n rows are used)."""
+    n = len(slots)
+    dev = torch.device("cuda", batch.device)
+    if out is not None:
+        toks, lens = out
+        if toks.dim() != 3 or toks.shape[0] < n or tuple(toks.shape[1:]) != (K, max_len) or lens.shape[0] < n or lens.shape[1] != K \
+                or toks.dtype != torch.int32 or lens.dtype != torch.int32 or not toks.is_contiguous() or not lens.is_contiguous():
+            raise ValueError("out must be contiguous int32 tensors [>= n, K, max_len] and [>= n, K]")
+    else:
+        toks = torch.zeros((n, K, max_len), dtype=torch.int32, device=dev)
+        lens = torch.zeros((n, K), dtype=torch.int32, device=dev)
+    if n:
+        sl = (_i32 * n)(*[int(x) for x in slots])
+        _check(_lib.tb_beam_backtrace_slot_list(batch.handle, n, sl, K, max_len, _dp(toks), _dp(lens), _stream(stream)),
+               "tb_beam_backtrace_slot_list")
+    return toks[:n], lens[:n]
 
 
 def tb_apply_final_weights_slots(batch: Batch, slots, scores: torch.Tensor, states: torch.Tensor, stream=None):

@@ -943,11 +943,13 @@ static int beam_reset_slots(tb_batch* b, int32_t n, const int32_t* slots, int32_
   if (n == 0) {   // every slot
     b->chunk_K = 0;
     return tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, b->n_slots, nullptr, 1,
-                                      b->d_slots, K, scores, states, live, stream);
+                                      b->d_slots, K, scores, states, live, stream);   // (every record of both halves, whatever the width)
   }
   for (int32_t at = 0; at < n; at += TB_BIND_PAIRS) {
     const int32_t m = n - at < TB_BIND_PAIRS ? n - at : TB_BIND_PAIRS;
-    const int rc = tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, b->max_beam, m, slots + at, 0,
+    // a slot's records sit at slot * (the session's beam width): the width of the chunks so far, else the one given
+    const int32_t stride = b->chunk_K > 0 ? b->chunk_K : (K > 0 ? K : b->max_beam);
+    const int rc = tb_launch_beam_reset_slots(b->d_slot_pos, b->d_hyp_hash, b->d_hyp_len, n_hyp, stride, m, slots + at, 0,
                                               b->d_slots, K, scores, states, live, stream);
     if (rc != TB_OK) return rc;
   }
@@ -1006,7 +1008,28 @@ extern "C" int tb_beam_backtrace_slots(tb_batch* b, int32_t n_slots, int32_t K, 
   if (!guard.ok) return TB_ERR_CUDA;
   const int32_t cap = static_cast<int32_t>(static_cast<int64_t>(b->max_tree_steps) * b->max_beam / K);
   return tb_launch_beam_backtrace_slots(b->d_tree, cap, b->d_slot_pos, n_slots, K, b->vocab, max_len, out_tokens, out_lens,
-                                        b->d_status, static_cast<cudaStream_t>(stream_));
+                                        b->d_status, b->d_hyp_len, static_cast<size_t>(b->n_slots) * b->max_beam, nullptr,
+                                        static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int tb_beam_backtrace_slot_list(tb_batch* b, int32_t n, const int32_t* slots, int32_t K, int32_t max_len,
+                                           int32_t* out_tokens, int32_t* out_lens, void* stream_) {
+  TbRange range_("tb_beam_backtrace_slot_list");
+  if (!b || !out_tokens || !out_lens || max_len < 1 || n < 1 || !slots) return TB_ERR_INVALID_ARG;
+  for (int32_t i = 0; i < n; ++i) if (slots[i] < 0 || slots[i] >= b->n_slots) return TB_ERR_BAD_SLOT;
+  if (!b->d_tree || b->chunk_K != K) return TB_ERR_INVALID_ARG;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  const int32_t cap = static_cast<int32_t>(static_cast<int64_t>(b->max_tree_steps) * b->max_beam / K);
+  for (int32_t at = 0; at < n; at += TB_BIND_PAIRS) {
+    const int32_t m = n - at < TB_BIND_PAIRS ? n - at : TB_BIND_PAIRS;
+    const int rc = tb_launch_beam_backtrace_slots(b->d_tree, cap, b->d_slot_pos, m, K, b->vocab, max_len,
+                                                  out_tokens + static_cast<int64_t>(at) * K * max_len, out_lens + static_cast<int64_t>(at) * K,
+                                                  b->d_status, b->d_hyp_len, static_cast<size_t>(b->n_slots) * b->max_beam, slots + at,
+                                                  static_cast<cudaStream_t>(stream_));
+    if (rc != TB_OK) return rc;
+  }
+  return TB_OK;
 }
 
 extern "C" int tb_apply_final_weights_slots(tb_batch* b, int32_t n, const int32_t* slots, int32_t K, float* scores,
@@ -1031,6 +1054,9 @@ extern "C" int tb_beam_backtrace(tb_batch* b, int32_t B, int32_t K, int32_t max_
   if (!b->d_tree || b->tree_steps == 0 || b->tree_B != B || b->tree_K != K) return TB_ERR_INVALID_ARG;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
-  return tb_launch_beam_backtrace(b->d_tree, b->tree_steps, B, K, b->vocab, max_len, out_tokens, out_lens,
+  // the sequence records the last step wrote: their lengths are the transcripts' lengths
+  const size_t n_hyp = static_cast<size_t>(b->n_slots) * b->max_beam;
+  const int32_t* len_cur = b->beam_steps > 0 ? b->d_hyp_len + (((b->beam_steps - 1) & 1) ? 0 : n_hyp) : nullptr;
+  return tb_launch_beam_backtrace(b->d_tree, b->tree_steps, B, K, b->vocab, max_len, out_tokens, out_lens, len_cur,
                                   static_cast<cudaStream_t>(stream_));
 }

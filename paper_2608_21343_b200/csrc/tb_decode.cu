@@ -1496,7 +1496,7 @@ struct SlotList { int32_t slot[TB_BIND_PAIRS]; };
 // A new utterance on some slots (or on all): position 0 in the slot's tree, every hypothesis' sequence empty.
 // With `scores` given, the slots' rows of the caller's [n_slots, K] arrays are set up as well: hypothesis 0 with score 0
 // in the root state (state -1 on an unbound slot), the others empty.
-__global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
+__global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,   // (max_beam: records per slot)
                                    int32_t n, SlotList sl, int32_t all_slots, const TbSlotRec* slots, int32_t K,
                                    float* scores, int32_t* states, uint8_t* live) {
   const int i = blockIdx.x;
@@ -1519,47 +1519,72 @@ __global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, 
 }
 
 // The tokens of every hypothesis a slot holds, walked back through the slot's own ring to the start of its utterance.
-__global__ void k_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
-                                       int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= n_slots * K) return;
-  const int b = idx / K;
-  const int32_t pos = slot_pos[b];
-  if (pos > tree_cap && idx % K == 0) atomicOr(status, TB_STATUS_STEP_LIMIT);   // the utterance is longer than the ring: its start is gone
-  const int32_t first = max(0, pos - tree_cap);
+// Backtrace of one stream's K hypotheses by one warp (lane k: hypothesis k).  The walk from the last step back to the
+// first is a chain of dependent loads; the warp therefore brings the tree's nodes of 32 steps at a time into shared
+// memory (coalesced, one trip) and the lanes follow their chains there.  The number of tokens of a hypothesis is its
+// sequence record's length, so the tokens are written from the back in one walk; only where part of the utterance
+// has left the ring (or no record is at hand) a first walk counts what is still there.
+// RING: the stream's own ring of tree_cap steps at position slot_pos[slot] (streaming), sequence records in the half
+// of len_base that the slot's last step wrote; else the batch-wide tree [n_steps, B, K] with the records at len_cur.
+// sl / use_list: the slots to walk (output row i belongs to sl.slot[i]); else slot = block index.
+constexpr int kBtSteps = 32;
+template <bool RING>
+__global__ void __launch_bounds__(32) k_beam_backtrace_warp(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_steps,
+                                                           int32_t B, int32_t K, int32_t V, int32_t max_len, int32_t* out_tokens,
+                                                           int32_t* out_lens, int32_t* status, const int32_t* len_base,
+                                                           size_t n_hyp, const int32_t* len_cur, SlotList sl, int32_t use_list) {
+  extern __shared__ int2 bt_stage[];                         // [kBtSteps][K]
+  const int lane = threadIdx.x;
+  const int b = use_list ? sl.slot[blockIdx.x] : blockIdx.x;
+  const int32_t pos = RING ? slot_pos[b] : n_steps;
+  const int32_t first = RING ? max(0, pos - tree_cap) : 0;
+  const bool cut = RING && pos > tree_cap;
+  if (cut && lane == 0) atomicOr(status, TB_STATUS_STEP_LIMIT);   // the utterance is longer than the ring: its start is gone
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * K + lane;
+  const int32_t* lens = RING ? (pos > 0 ? len_base + (((pos - 1) & 1) ? 0 : n_hyp) : nullptr) : len_cur;
+  const bool count_first = cut || (lens == nullptr && pos > 0);
   int32_t n = 0;
-  for (int pass = 0; pass < 2; ++pass) {
-    int32_t slot = idx % K, at = n;
-    for (int32_t st = pos - 1; st >= first && slot >= 0; --st) {
-      const int2 e = tree[(static_cast<int64_t>(b) * tree_cap + (st % tree_cap)) * K + slot];
-      if (e.y >= 0 && e.y != V) {
-        if (pass == 0) ++n;
-        else { --at; if (at < max_len) out_tokens[static_cast<int64_t>(idx) * max_len + at] = e.y; }
-      }
-      slot = e.x;
-    }
-    if (pass == 0) out_lens[idx] = n;
+  if (!count_first && lane < K) {
+    n = lens ? lens[static_cast<int64_t>(b) * K + lane] : 0;
+    out_lens[row] = n;
   }
-}
-
-__global__ void k_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V,
-                                 int32_t max_len, int32_t* out_tokens, int32_t* out_lens) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= B * K) return;
-  const int b = idx / K;
-  // pass 1: length; pass 2: fill from the back
-  int32_t n = 0;
-  for (int pass = 0; pass < 2; ++pass) {
-    int32_t slot = idx % K, pos = n;
-    for (int32_t st = n_steps - 1; st >= 0 && slot >= 0; --st) {
-      const int2 e = tree[(static_cast<int64_t>(st) * B + b) * K + slot];
-      if (e.y >= 0 && e.y != V) {
-        if (pass == 0) ++n;
-        else { --pos; if (pos < max_len) out_tokens[static_cast<int64_t>(idx) * max_len + pos] = e.y; }
+  for (int pass = count_first ? 0 : 1; pass < 2; ++pass) {
+    int32_t cur = lane < K ? lane : -1, at = n;
+    for (int32_t hi = pos; hi > first; hi -= kBtSteps) {
+      if (!__any_sync(0xffffffffu, cur >= 0 && (pass == 0 || at > 0))) break;
+      const int32_t lo = max(first, hi - kBtSteps), cnt = hi - lo;
+      // (eight nodes per lane are requested before the first is stored: one trip for all of them)
+      for (int e0 = 0; e0 < cnt * K; e0 += 32 * 8) {
+        int2 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int e = e0 + 32 * u + lane;
+          if (e < cnt * K) {
+            const int j = e / K, kk = e - j * K;
+            const int32_t st = lo + j;
+            const int64_t node = RING ? (static_cast<int64_t>(b) * tree_cap + (st % tree_cap)) * K + kk
+                                      : (static_cast<int64_t>(st) * B + b) * K + kk;
+            v[u] = tree[node];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int e = e0 + 32 * u + lane;
+          if (e < cnt * K) bt_stage[e] = v[u];
+        }
       }
-      slot = e.x;
+      __syncwarp();
+      for (int j = cnt - 1; j >= 0 && cur >= 0; --j) {
+        const int2 e = bt_stage[j * K + cur];
+        if (e.y >= 0 && e.y != V) {
+          if (pass == 0) ++n;
+          else { --at; if (at >= 0 && at < max_len) out_tokens[row * max_len + at] = e.y; }
+        }
+        cur = e.x;
+      }
+      __syncwarp();
     }
-    if (pass == 0) out_lens[idx] = n;
+    if (pass == 0 && lane < K) out_lens[row] = n;
   }
 }
 
@@ -1661,9 +1686,11 @@ int tb_launch_beam_frames(const TbBeamParams& p_in, int32_t T, int32_t E, int64_
 }
 
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
-                             int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream) {
-  const int n = B * K;
-  k_beam_backtrace<<<(n + 127) / 128, 128, 0, stream>>>(tree, n_steps, B, K, V, max_len, out_tokens, out_lens);
+                             int32_t* out_tokens, int32_t* out_lens, const int32_t* len_cur, cudaStream_t stream) {
+  SlotList none;
+  for (int i = 0; i < TB_BIND_PAIRS; ++i) none.slot[i] = 0;
+  k_beam_backtrace_warp<false><<<B, 32, kBtSteps * K * sizeof(int2), stream>>>(tree, 0, nullptr, n_steps, B, K, V, max_len, out_tokens,
+                                                                              out_lens, nullptr, nullptr, 0, len_cur, none, 0);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
@@ -1790,9 +1817,14 @@ int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int3
 
 int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
                                    int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status,
-                                   cudaStream_t stream) {
-  const int n = n_slots * K;
-  k_beam_backtrace_slots<<<(n + 127) / 128, 128, 0, stream>>>(tree, tree_cap, slot_pos, n_slots, K, V, max_len, out_tokens, out_lens, status);
+                                   const int32_t* len_base, size_t n_hyp, const int32_t* slot_list, cudaStream_t stream) {
+  // slot_list (host, n_slots entries, at most TB_BIND_PAIRS): the slots to walk; null: slots 0 .. n_slots-1
+  if (slot_list && n_slots > TB_BIND_PAIRS) return TB_ERR_INVALID_ARG;
+  SlotList sl;
+  for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = (slot_list && i < n_slots) ? slot_list[i] : 0;
+  k_beam_backtrace_warp<true><<<n_slots, 32, kBtSteps * K * sizeof(int2), stream>>>(tree, tree_cap, slot_pos, 0, n_slots, K, V, max_len,
+                                                                                   out_tokens, out_lens, status, len_base, n_hyp, nullptr,
+                                                                                   sl, slot_list ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 

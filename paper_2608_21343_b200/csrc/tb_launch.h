@@ -89,12 +89,12 @@ int tb_launch_beam_frames(const TbBeamParams& p, int32_t T, int32_t E, int64_t f
 int tb_launch_beam_chunk(const TbBeamParams& p, int32_t T, int32_t E, int64_t frame_stride, int64_t row_stride,
                          const int32_t* n_frames, int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp,
                          cudaStream_t stream);
-int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t max_beam,
+int tb_launch_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, int32_t* len, size_t n_hyp, int32_t rec_stride,
                                int32_t n, const int32_t* slots, int32_t all_slots, const TbSlotRec* slot_recs, int32_t K,
                                float* scores, int32_t* states, uint8_t* live, cudaStream_t stream);
 int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_slots, int32_t K,
                                    int32_t V, int32_t max_len, int32_t* out_tokens, int32_t* out_lens, int32_t* status,
-                                   cudaStream_t stream);
+                                   const int32_t* len_base, size_t n_hyp, const int32_t* slot_list, cudaStream_t stream);
 int tb_launch_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, const int32_t* slot_list,
                                   int32_t K, float* scores, const int32_t* states, int32_t* status, cudaStream_t stream);
 // Reduces every row of [B, T, E] (element strides given) to its TbTopEnt entries: out[((b * T + t) * E + e) * (top_m + 1)].
@@ -104,7 +104,7 @@ int tb_launch_beam_topm(const void* logits, int dtype, int32_t B, int32_t T, int
                         const TbSlotRec* slots, const unsigned char* arena, const int32_t* cls, int32_t top_m,
                         TbTopEnt* out, cudaStream_t stream);
 int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32_t K, int32_t V, int32_t max_len,
-                             int32_t* out_tokens, int32_t* out_lens, cudaStream_t stream);
+                             int32_t* out_tokens, int32_t* out_lens, const int32_t* len_cur, cudaStream_t stream);
 // Registered models: their records live in a device table; tb_launch_bind_models points up to TB_BIND_PAIRS slots at
 // models of that table (id -1: unbound) and resets the slots' streaming state, in one launch.
 #define TB_BIND_PAIRS 256

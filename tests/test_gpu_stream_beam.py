@@ -71,8 +71,11 @@ def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=Fal
         if ended:
             tb.tb_apply_final_weights_slots(batch, ended, scores, states)
             toks, lens = tb.tb_beam_backtrace_slots(batch, w.B, K, w.T * E)
+            some_t, some_l = tb.tb_beam_backtrace_slot_list(batch, ended, K, w.T * E)      # ... and of the ended slots only
             torch.cuda.synchronize()
             h_tok, h_len, h_sc, h_st = toks.cpu().numpy(), lens.cpu().numpy(), scores.cpu().numpy(), states.cpu().numpy()
+            for i, s in enumerate(ended):
+                assert np.array_equal(some_l[i].cpu().numpy(), h_len[s]) and np.array_equal(some_t[i].cpu().numpy(), h_tok[s]), (c, s)
             for s in ended:
                 g = oracle_graph(w, slot[s]["phrases"])
                 ref = O.beam_decode(g, slot[s]["logits"][:slot[s]["length"]], K, merge=merge,
