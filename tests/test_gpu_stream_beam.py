@@ -14,11 +14,11 @@ from helpers import SCORE_TOL, oracle_graph, to_device
 pytestmark = pytest.mark.gpu
 
 
-def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=False):
+def run_streaming_beam(tb, w, K, n_chunks, merge, prune_delta, check_partial=False, max_beam=None):
     """Chunks of w.chunk frames over w.B slots with stream churn; returns the number of streams checked."""
     E = w.S
     sched = W.ChurnSchedule(w)
-    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=K, max_tree_steps=w.T * E, arena_bytes=32 << 20)
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=max_beam or K, max_tree_steps=w.T * E, arena_bytes=32 << 20)
     if prune_delta is not None:
         tb.tb_batch_set_beam_prune(batch, prune_delta)
     dev = torch.device("cuda:0")
@@ -101,6 +101,14 @@ def test_streaming_beam_with_churn(tb, K, merge, prune):
     w = W.get_workload(5, B=10, T=70, T_lo=20, S=2, n_dur=0, n_phrases=60, n_phrases_lo=10)
     n = run_streaming_beam(tb, w, K, n_chunks=24, merge=merge, prune_delta=prune, check_partial=True)
     assert n >= 2 * w.B                                     # every slot saw several streams
+
+
+def test_streaming_beam_narrower_than_the_batch_allows(tb):
+    """A session may use a beam narrower than the batch was created for: the per-slot records (tree ring, sequence
+    hashes and lengths) are then laid out at the session's width, also when single slots restart."""
+    w = W.get_workload(5, B=6, T=50, T_lo=15, S=2, n_dur=0, n_phrases=40, n_phrases_lo=10)
+    n = run_streaming_beam(tb, w, 3, n_chunks=20, merge=True, prune_delta=6.0, check_partial=True, max_beam=8)
+    assert n >= w.B
 
 
 def test_streaming_beam_refuses_to_mix_with_the_batch_wide_tree(tb):
