@@ -583,6 +583,7 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, BeamShared
           unsigned long long* wkey = reinterpret_cast<unsigned long long*>(cdst + cap);            // [warps][K] (key); behind the targets
           int32_t* widx = reinterpret_cast<int32_t*>(wkey + (kBeamThreads / 32) * TB_MAX_BEAM);   // [warps][K] where in ckey
           constexpr int kSelRegs = 8;
+          constexpr int kRadixMinK = 9;       // beams at least this wide (wider than the teams of warps take) find their picks by radix selection
           const bool solo = n <= 32 * kSelRegs;
           auto put_sel = [&](int r, unsigned long long best, int idx) {
             const uint32_t mh = static_cast<uint32_t>(best >> 32);
@@ -599,6 +600,91 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, BeamShared
               else warp_top_keys<8>(ckey, n, lane, 32, K, lane, wkey, widx);
               __syncwarp();
               if (lane < K) put_sel(lane, wkey[lane], widx[lane]);
+            }
+          } else if (K >= kRadixMinK) {
+            // Wide beams: K rounds at two levels cost more than finding the K-th largest key first.  The keys are 64-bit
+            // numbers, all different; the K-th largest is found digit by digit (8 bits at a time, from the highest
+            // digit in which the candidates differ) with a histogram in shared memory, the keys at or above it are
+            // collected, and one warp orders them by counting, for each, the keys above it.
+            int* hist = reinterpret_cast<int*>(wkey);                     // [256]
+            int* ctl = hist + 256;                                        // digit, its count, rank left, collected
+            unsigned long long* okey = reinterpret_cast<unsigned long long*>(ctl + 8);   // [K] the collected keys
+            int32_t* oidx = reinterpret_cast<int32_t*>(okey + TB_MAX_BEAM);              // [K] where they sit in ckey
+            uint32_t hmax = 0u, hmin = 0xFFFFFFFFu;
+            for (int ii = threadIdx.x; ii < n; ii += kBeamThreads) {
+              const unsigned long long kk = ckey[ii];
+              if (kk != 0ull) { const uint32_t h = static_cast<uint32_t>(kk >> 32); hmax = max(hmax, h); hmin = min(hmin, h); }
+            }
+            hmax = __reduce_max_sync(0xffffffffu, hmax);
+            hmin = __reduce_min_sync(0xffffffffu, hmin);
+            if (lane == 0) { red64[0][warp] = hmax; red64[1][warp] = hmin; }
+            if (threadIdx.x == 0) ctl[3] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int w2 = 0; w2 < kBeamThreads / 32; ++w2) {
+              hmax = max(hmax, static_cast<uint32_t>(red64[0][w2])); hmin = min(hmin, static_cast<uint32_t>(red64[1][w2]));
+            }
+            unsigned long long t_low = 1ull;                               // keys at or above this are the picks
+            if (hmax != 0u) {
+              const uint32_t diff = hmax ^ hmin;
+              int shift = diff == 0u ? 24 : 32 + ((31 - __clz(diff)) >> 3) * 8;
+              unsigned long long prefix = shift + 8 >= 64 ? 0ull : ((static_cast<unsigned long long>(hmax) << 32) >> (shift + 8));
+              int want = K;
+              for (;;) {
+                if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+                __syncthreads();
+                for (int ii = threadIdx.x; ii < n; ii += kBeamThreads) {
+                  const unsigned long long kk = ckey[ii];
+                  if (kk != 0ull && (shift + 8 >= 64 || (kk >> (shift + 8)) == prefix)) atomicAdd(&hist[static_cast<int>((kk >> shift) & 255ull)], 1);
+                }
+                __syncthreads();
+                if (warp == 0) {
+                  // lane l looks at digits 255 - 8 l ... 248 - 8 l; the digit of the K-th key is the first at which
+                  // the count of keys with that digit or a higher one reaches the rank wanted
+                  int c[8], mine_total = 0;
+#pragma unroll
+                  for (int d = 0; d < 8; ++d) { c[d] = hist[255 - (8 * lane + d)]; mine_total += c[d]; }
+                  int incl = mine_total;
+#pragma unroll
+                  for (int o = 1; o < 32; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                  const int total = __shfl_sync(0xffffffffu, incl, 31);
+                  const unsigned reach = __ballot_sync(0xffffffffu, incl >= want);
+                  if (total < want) {
+                    if (lane == 0) ctl[0] = -1;                           // fewer candidates than places: all of them
+                  } else if (lane == __ffs(reach) - 1) {
+                    int above = incl - mine_total, d = 0;
+                    while (above + c[d] < want) { above += c[d]; ++d; }
+                    ctl[0] = 255 - (8 * lane + d); ctl[1] = c[d]; ctl[2] = want - above;
+                  }
+                }
+                __syncthreads();
+                const int digit = ctl[0];
+                if (digit < 0) break;
+                const int cD = ctl[1];
+                want = ctl[2];
+                prefix = (prefix << 8) | static_cast<unsigned long long>(digit);
+                if (want == cD || shift == 0) { t_low = prefix << shift; break; }
+                shift -= 8;
+              }
+              for (int ii = threadIdx.x; ii < n; ii += kBeamThreads) {
+                const unsigned long long kk = ckey[ii];
+                if (kk != 0ull && kk >= t_low) {
+                  const int pos = atomicAdd(&ctl[3], 1);
+                  if (pos < TB_MAX_BEAM) { okey[pos] = kk; oidx[pos] = ii; }
+                }
+              }
+            }
+            __syncthreads();
+            if (warp == 0) {
+              const int cnt = min(ctl[3], K);
+              if (lane < cnt) {
+                const unsigned long long mine = okey[lane];
+                int rank = 0;
+                for (int j2 = 0; j2 < cnt; ++j2) rank += okey[j2] > mine ? 1 : 0;
+                put_sel(rank, mine, oidx[lane]);
+              } else if (lane < K) {
+                put_sel(lane, 0ull, -1);
+              }
             }
           } else {
             if (n <= kBeamThreads * 2) {
