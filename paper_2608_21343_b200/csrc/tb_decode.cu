@@ -527,7 +527,9 @@ __device__ __forceinline__ void beam_step_body(const TbBeamParams& p, BeamShared
               const int q = q0 + j * cnt;
               int k = 0;
               if (q < n_listed) {
-                while (q >= cp_off[k + 1]) ++k;
+                // the hypothesis whose listed candidates include place q: the last k with cp_off[k] <= q (bisection)
+                int hi_k = K;
+                while (hi_k - k > 1) { const int mid = (k + hi_k) >> 1; if (cp_off[mid] <= q) k = mid; else hi_k = mid; }
                 e8[j] = ent[h_beg[k] + (q - cp_off[k])];
               }
               k8[j] = k;
