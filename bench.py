@@ -252,7 +252,7 @@ def side_measurement(args):
                                      "note": "one tb_beam_step call per expansion, driven from the host"}, "data": "synthetic"}))
     elif args.workload == 5:
         w = W.get_workload(5, **({"B": args.streams} if args.streams else {}))
-        sched = W.ChurnSchedule(w, workers=8)            # (the next chunks' inputs are drawn by worker threads)
+        sched = W.ChurnSchedule(w)                       # (inputs drawn by this thread: worker threads would compete with the timed calls for the interpreter)
         batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
         n_chunks, lat, binds, t_compile = 40 + 10 * args.steps, [], 0, 0.0
         host_us = []
@@ -302,7 +302,7 @@ def side_measurement(args):
         for K in (4, 32):
             w = W.get_workload(5, B=args.streams or 128, S=2, n_dur=0)
             E = w.S
-            sched = W.ChurnSchedule(w, workers=8)
+            sched = W.ChurnSchedule(w)
             batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, max_beam=K, max_tree_steps=w.T * E, arena_bytes=256 << 20)
             tb.tb_batch_set_beam_prune(batch, 10.0)
             scores = torch.full((w.B, K), float("-inf"), device=dev)
