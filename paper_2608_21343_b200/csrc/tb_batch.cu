@@ -452,9 +452,14 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   b->next_staging = (b->next_staging + 1) % kStagingRing;
   bool ok = true;
   if (s.pending) { ok = cudaEventSynchronize(s.done) == cudaSuccess; s.pending = false; }
-  if (s.held) { tb_graph_free(s.held); s.held = nullptr; }
-  for (tb_graph* h : s.held_more) tb_graph_free(h);
-  s.held_more.clear();
+  // the graphs this entry's last copies read are let go when the call returns: after this call's copies and launch
+  // have been issued, not before them
+  struct LetGo {
+    std::vector<tb_graph*> graphs;
+    ~LetGo() { for (tb_graph* h : graphs) tb_graph_free(h); }
+  } let_go;
+  let_go.graphs.swap(s.held_more);
+  if (s.held) { let_go.graphs.push_back(s.held); s.held = nullptr; }
   // graphs whose image is page-locked (those kept by a cache) are copied from where they are; only
   // the others pass through the staging block, which also carries the records
   bool any_pinned = false;
