@@ -630,6 +630,27 @@ def main():
                                # an unboosted decode streams every row once: the whole tensor over the launch time
                                "all_rows_GBs": logits.numel() * logits.element_size() / (p_ms * 1e-3) / 1e9,
                                "all_rows_frac_of_measured_peak": logits.numel() * logits.element_size() / (p_ms * 1e-3) / 1e9 / result["roofline"]["peak"]}
+    if not args.no_extras and rank == 0 and w.B >= 64:
+        # the same streams in smaller batches (the first 16 / 32 of them): with most SMs free, tb_greedy_decode cuts
+        # every stream into segments decoded by several blocks at once (k_greedy_seg); reported beside the headline,
+        # not part of it
+        small = {}
+        for nb_ in (16, 32):
+            sb_ = tb.tb_batch_create(w.V, w.vocab.case_class, nb_, arena_bytes=16 << 20, device=local_rank)
+            for i in range(nb_):
+                tb.tb_batch_bind_stream(sb_, i, graphs[i])
+            lg_ = logits[:nb_]
+            o_ = tb.tb_greedy_decode(sb_, lg_)
+            ran_ = tb.tb_batch_last_greedy_kernel(sb_)
+            ms_, _ = timed(lambda: tb.tb_greedy_decode(sb_, lg_, out=o_), max(20, args.steps // 4), args.warmup)
+            ms_ /= max(20, args.steps // 4)
+            same_ = all(int(o_["counts"][i]) == int(counts[i]) for i in range(nb_))      # (the same decode as in the full batch)
+            small[str(nb_)] = {"ms_per_step": ms_, "frames_per_s": nb_ * w.T / (ms_ * 1e-3), "blocks_per_stream": ran_["blocks_per_stream"],
+                               "kernel": {tb.TB_KERNEL_PIPELINED: "k_greedy_fast", tb.TB_KERNEL_SEGMENTED: "k_greedy_seg",
+                                          tb.TB_KERNEL_GENERAL: "k_decode_general"}[ran_["kernel"]],
+                               "same_token_counts_as_in_full_batch": bool(same_)}
+            sb_.destroy()
+        result["smaller_batches"] = small
     if not args.no_extras and rank == 0:
         # end to end through the public call with host buffers: H2D of the logits, decode, D2H of results
         dl = torch.empty_like(logits)
