@@ -652,6 +652,22 @@ def main():
             sb_.destroy()
         result["smaller_batches"] = small
     if not args.no_extras and rank == 0:
+        # the same decode with every row log-softmax normalised inside the selection (TB_FLAG_LOG_SOFTMAX): the
+        # helpers also leave each row's normaliser; reported beside the headline, not part of it
+        base_flags = tb.TB_FLAG_ONE_BLOCK_PER_STREAM if args.one_block_per_stream else 0
+        tb.tb_batch_set_flags(batch, base_flags | tb.TB_FLAG_LOG_SOFTMAX)
+        on_ = tb.tb_greedy_decode(batch, logits)
+        ran_ = tb.tb_batch_last_greedy_kernel(batch)
+        n_ms, _ = timed(lambda: tb.tb_greedy_decode(batch, logits, out=on_), max(20, args.steps // 4), args.warmup)
+        n_ms /= max(20, args.steps // 4)
+        valid_ = torch.arange(out["tokens"].shape[1], device=dev)[None, :] < out["counts"][:, None]
+        result["log_softmax"] = {"ms_per_step": n_ms, "frames_per_s": w.B * w.T / (n_ms * 1e-3),
+                                 "kernel": {tb.TB_KERNEL_PIPELINED: "k_greedy_fast", tb.TB_KERNEL_SEGMENTED: "k_greedy_seg",
+                                            tb.TB_KERNEL_GENERAL: "k_decode_general"}[ran_["kernel"]],
+                                 "same_tokens_as_unnormalised": bool(torch.equal(on_["counts"], out["counts"]) and torch.equal(
+                                     torch.where(valid_, on_["tokens"], 0), torch.where(valid_, out["tokens"], 0)))}
+        tb.tb_batch_set_flags(batch, base_flags)
+    if not args.no_extras and rank == 0:
         # end to end through the public call with host buffers: H2D of the logits, decode, D2H of results
         dl = torch.empty_like(logits)
         host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}

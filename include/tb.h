@@ -69,10 +69,16 @@ extern "C" {
 /* tb_batch_set_flags */
 #define TB_FLAG_GENERAL_KERNELS 1       /* always use the general decode kernel (any layout), never a pipelined one */
 #define TB_FLAG_ONE_BLOCK_PER_STREAM 2  /* pipelined greedy decode: never the segmented kernel, one block per stream */
-#define TB_FLAG_LOG_SOFTMAX 8           /* tb_greedy_decode and tb_stream_chunk (RNNT rows) normalise every visited row first:
-                                           value(v) = fl(fl(x_v - L) + fl(lambda * bonus)), L = m + log(sum_v exp(x_v - m)) over the
-                                           row's vocab+1 entries, computed in float inside the selection kernel (Sec. 2.2 para. 3:
-                                           one fused scoring operation); runs on the general kernel */
+#define TB_FLAG_LOG_SOFTMAX 8           /* tb_greedy_decode and tb_stream_chunk (RNNT rows) score every visited row by its log-softmax:
+                                           L = m + log(sum_v exp(x_v - m)) over the row's vocab+1 entries, computed in float inside
+                                           the selection kernel (Sec. 2.2 para. 3: one fused scoring operation).  The general kernel
+                                           (any layout; streaming chunks) takes L off every entry before the bonus is added:
+                                           value(v) = fl(fl(x_v - L) + fl(lambda * bonus)).  The pipelined kernels (packed bf16 rows)
+                                           take it off after the selection, L being common to a row's candidates: the row is
+                                           decided on fl(x_v + fl(lambda * bonus)) exactly as without the flag, and adds
+                                           fl(that value - L) to the score.  Either way tokens can differ from a decode in exact
+                                           arithmetic only where two candidates are closer than the float roundings, and scores
+                                           by a few float roundings per visited row */
 #define TB_FLAG_BEAM_WHOLE_ROWS 16      /* tb_beam_frames / tb_beam_chunk: no pre-pass that reduces every row to its best tokens; every
                                            step looks at all vocab+1 entries of its row (identical results) */
 #define TB_FLAG_TEST_WAIT_TIMEOUT 4     /* self-test of the kernels' bounded waits: tb_greedy_decode (segmented kernel) withholds one

@@ -686,8 +686,8 @@ extern "C" int tb_greedy_decode(tb_batch* b, const void* logits, int dtype, int3
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  p.normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;   // (only the general kernel normalises)
-  if (!(b->flags & (TB_FLAG_GENERAL_KERNELS | TB_FLAG_LOG_SOFTMAX))) {
+  p.normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;
+  if (!(b->flags & TB_FLAG_GENERAL_KERNELS)) {
     int32_t max_cache = 0, max_states = 0, all_resolved = 1;
     for (int32_t i = 0; i < B; ++i) {
       max_cache = b->slot_cache_bytes[i] > max_cache ? b->slot_cache_bytes[i] : max_cache;

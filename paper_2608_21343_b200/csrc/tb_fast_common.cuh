@@ -26,7 +26,8 @@ struct RowSummary {
 };
 constexpr uint32_t kSumOvf = 1u << 16, kSumGap = 1u << 17;
 // Summaries of one ring stage are kSMax * 32 bytes; stages are spaced 16 bytes further apart so that the
-// decider's lanes (one stage each) read their 16-byte halves from distinct shared-memory banks.
+// decider's lanes (one stage each) read their 16-byte halves from distinct shared-memory banks.  A decode that
+// normalises its rows keeps the stage's kSMax normalisers (floats) in those 16 bytes.
 constexpr int kSumStageBytes = kSMax * 32 + 16;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -82,6 +83,16 @@ __device__ __forceinline__ uint4 lds_v4_volatile(uint32_t a) {
   uint4 v;
   asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
   return v;
+}
+__device__ __forceinline__ float lds_f32_volatile(uint32_t a) {
+  float v;
+  asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ float exp2f_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ void sts_v4_volatile(uint32_t a, uint4 v) {
   asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -146,9 +157,12 @@ __device__ __forceinline__ void load_row(const HelperCtx& h, const unsigned char
 
 // Row in registers -> summary at shared address out_a (see RowSummary).  rowp: the row's first element (the few exact
 // candidate values are re-read from there), p: elements of the first 16-byte block that precede the row.
-template <int NIT>
+// NORM: the row's log-softmax normaliser L = M + log(sum_v exp(x_v - M)) over its V + 1 entries (M: their maximum)
+// is computed as well, in float with a fixed order of additions, and stored at shared address lse_a before the
+// summary's sequence word (0 for a row without a finite entry).
+template <int NIT, bool NORM = false>
 __device__ __forceinline__ void finish_row(const HelperCtx& h, RowRegs<NIT>& r, const unsigned char* rowp, int p,
-                                           uint32_t out_a, uint32_t seq, int lane) {
+                                           uint32_t out_a, uint32_t seq, int lane, uint32_t lse_a = 0u) {
   const int V = h.V;
   uint32_t (&w)[4 * NIT] = r.w;
   // What the 16-byte blocks hold beyond this row's tokens is masked to -inf: the p elements before the row in
@@ -198,6 +212,28 @@ __device__ __forceinline__ void finish_row(const HelperCtx& h, RowRegs<NIT>& r, 
     m = __ushort_as_bfloat16(static_cast<unsigned short>(ub));
   }
   const float mf = __bfloat162float(m);
+  float lse = 0.0f;
+  if constexpr (NORM) {
+    // sum_v 2^(x_v * log2(e) - c) with c = fl(M * log2(e)): one fused multiply-add and one exponential per entry; what
+    // the rounding of c scales the sum by (2^(c - M * log2(e)), the same for every entry) is taken off the logarithm
+    const float xbl = row_at(rowp, V);
+    const float M = fmaxf(mf, xbl);
+    const float kL2e = 1.4426950408889634f;
+    const float c = __fmul_rn(M, kL2e), nc = -c;
+    float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4 * NIT; ++i) {
+      acc0 = __fadd_rn(acc0, exp2f_approx(__fmaf_rn(__uint_as_float(w[i] << 16), kL2e, nc)));
+      acc1 = __fadd_rn(acc1, exp2f_approx(__fmaf_rn(__uint_as_float(w[i] & 0xFFFF0000u), kL2e, nc)));
+    }
+    float acc = __fadd_rn(acc0, acc1);
+    if (tail_ok) acc = __fadd_rn(acc, exp2f_approx(__fmaf_rn(bf16_bits_to_float(tail_bits), kL2e, nc)));
+    if (lane == 0) acc = __fadd_rn(acc, exp2f_approx(__fmaf_rn(xbl, kL2e, nc)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+    const float c_lo = __fmaf_rn(M, kL2e, nc);                       // M * log2(e) - c, exactly
+    lse = (M == -INFINITY) ? 0.0f : __fadd_rn(M, __fsub_rn(logf(acc), __fmul_rn(c_lo, 0.6931471805599453f)));
+  }
   // Every token whose root-boosted value can reach that of the raw maximum has x >= m - dbeta;
   // gamma keeps a strict margin over all roundings.  thr is rounded down.
   const float gamma = (fabsf(mf) + fabsf(h.beta_max) + fabsf(h.beta_min)) * 0.0009765625f + 1e-30f;
@@ -266,6 +302,7 @@ __device__ __forceinline__ void finish_row(const HelperCtx& h, RowRegs<NIT>& r, 
     r.packed = static_cast<uint32_t>(id1) | (ovf ? kSumOvf : 0u) | ((r.y1 - r.y2b > tau) ? kSumGap : 0u);
     r.seq = seq;
     if (!ovf || lane == 0) {
+      if constexpr (NORM) asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(lse_a), "f"(lse) : "memory");
       // first half, fence, then the half that carries the sequence word
       sts_v4_volatile(out_a, make_uint4(__float_as_uint(r.y1), __float_as_uint(r.y2b), __float_as_uint(r.xb), __float_as_uint(r.x1)));
       __threadfence_block();
@@ -276,12 +313,12 @@ __device__ __forceinline__ void finish_row(const HelperCtx& h, RowRegs<NIT>& r, 
 }
 
 // Both steps at once, for a row that sits in shared memory (every block readable).
-template <int NIT>
+template <int NIT, bool NORM = false>
 __device__ __forceinline__ void summarize_row(const HelperCtx& h, const unsigned char* slot, int off_bytes,
-                                              uint32_t out_a, uint32_t seq, int lane) {
+                                              uint32_t out_a, uint32_t seq, int lane, uint32_t lse_a = 0u) {
   RowRegs<NIT> r;
   load_row<NIT>(h, slot, off_bytes, lane, nullptr, nullptr, r);
-  finish_row<NIT>(h, r, slot + off_bytes, (off_bytes & 15) >> 1, out_a, seq, lane);
+  finish_row<NIT, NORM>(h, r, slot + off_bytes, (off_bytes & 15) >> 1, out_a, seq, lane, lse_a);
 }
 
 // The tokens boosted by the non-root part of the suffix chain of the current state, as 8-byte

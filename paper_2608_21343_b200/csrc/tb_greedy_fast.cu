@@ -190,7 +190,7 @@ __device__ __forceinline__ void build_list(const TbStateRec* strec, const TbTokE
 __device__ __forceinline__ void prog_publish(volatile int* flags, int v) { flags[2] = v; }
 
 
-template <int NIT>
+template <int NIT, bool NORM>
 __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
   extern __shared__ __align__(128) unsigned char dyn[];
   const TbDecodeParams& p = P.d;
@@ -376,7 +376,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
     for (; f < end;) {
       if (!mbar_wait_parked(&pfull[st], ph, flags, pipe, p.status)) break;
       const unsigned char* slot = pring + static_cast<size_t>(st) * P.slot_bytes;
-      summarize_row<NIT>(h, slot, lead + k * row_bytes, psumm_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane);
+      summarize_row<NIT, NORM>(h, slot, lead + k * row_bytes, psumm_a + st * kSumStageBytes + k * 32, static_cast<uint32_t>(f) + 1u, lane,
+                               psumm_a + st * kSumStageBytes + kSMax * 32 + 4 * k);
       if (lane == 0) mbar_arrive(&pfree[st]);
       k += pnh;
       while (k >= S) {                                      // on to a later frame
@@ -459,6 +460,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const uint32_t row_a = ring_a + stq * P.slot_bytes + ((lead + q * lead_step) & 15) + rk * row_bytes;
         const bool ready = t + q < end && q1.w == static_cast<uint32_t>(t + q) + 1u;
         const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+        const float lse = NORM ? lds_f32_volatile(summ_a + stq * kSumStageBytes + kSMax * 32u + 4u * rk) : 0.0f;
         const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
         // this lane's entries ql, ql + 4, ...: the cached lists are sorted by token, so within a lane a strict
         // comparison keeps the lowest token among equal values; bit 0 of an entry word is free (2 * token) and
@@ -542,11 +544,14 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
         const uint32_t j_tn = __shfl_sync(0xffffffffu, (static_cast<uint32_t>(wnext) << TB_RS_TOK_BITS) | static_cast<uint32_t>(wtok), jl);
         const int j_tok = static_cast<int>(j_tn & kTokMask), j_next = static_cast<int>(j_tn >> TB_RS_TOK_BITS);
-        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
-        const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
-        const float xb2 = __shfl_sync(0xffffffffu, xb, 8), xb3 = __shfl_sync(0xffffffffu, xb, 12);
-        const float xb4 = __shfl_sync(0xffffffffu, xb, 16), xb5 = __shfl_sync(0xffffffffu, xb, 20);
-        const float xb6 = __shfl_sync(0xffffffffu, xb, 24), xb7 = __shfl_sync(0xffffffffu, xb, 28);
+        // what a row adds to the score: its selected value, less the row's normaliser when rows are normalised (the
+        // normaliser is common to all candidates of a row, so it is taken off after the selection)
+        const float xbs = NORM ? __fsub_rn(xb, lse) : xb;
+        const float j_val = __shfl_sync(0xffffffffu, NORM ? __fsub_rn(wv, lse) : wv, jl);
+        const float xb0 = __shfl_sync(0xffffffffu, xbs, 0), xb1 = __shfl_sync(0xffffffffu, xbs, 4);
+        const float xb2 = __shfl_sync(0xffffffffu, xbs, 8), xb3 = __shfl_sync(0xffffffffu, xbs, 12);
+        const float xb4 = __shfl_sync(0xffffffffu, xbs, 16), xb5 = __shfl_sync(0xffffffffu, xbs, 20);
+        const float xb6 = __shfl_sync(0xffffffffu, xbs, 24), xb7 = __shfl_sync(0xffffffffu, xbs, 28);
         const bool took = nb < kWin && j_ready;             // the row after the blanks selects a token
         const bool rare = (nb == 0 && !took) || (took && j_rescan) || (took && (j_next < 0 || j_next >= rec.n_states));
         if (!rare) {
@@ -576,7 +581,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           const int tnext = took ? j_next : s;
           n_out += took ? 1 : 0;
           if (rec_on) {
-            if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xb;
+            if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xbs;
             if (took && lane == 0) vlog[nv + nb] = j_val;
             if (lane < adv && t + lane + 1 >= f_mid)
               trace[t + lane + 1] = make_int4(lane >= nb ? tnext : s, n_out - ((took && lane < nb) ? 1 : 0), nv + lane + 1, 0);
@@ -616,6 +621,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const uint4 q1 = lds_v4_volatile(sum_a + 16u);
         const uint4 q0 = lds_v4_volatile(sum_a);
         const float xb = __uint_as_float(q0.z);
+        const float lse = NORM ? lds_f32_volatile(summ_a + stq * kSumStageBytes + kSMax * 32u + 4u * min(ql, kSMax - 1)) : 0.0f;
         // the plain winner: at the root (no list) it is the row's winner
         float wv = __fadd_rn(__uint_as_float(q0.w), __fmul_rn(lam, __fadd_rn(L.D, __uint_as_float(q1.x))));
         int wtok = static_cast<int>(q1.z & 0xFFFFu), wnext = bound ? static_cast<int>(q1.y) : -1;
@@ -682,7 +688,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
           const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * (fq & 7))) & 0xFu) : 0;
           const unsigned upto = 0xFFFFFFFFu >> (31 - lane);
           const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
-          const float val = mine_t ? wv : xb;
+          const float val = NORM ? __fsub_rn(mine_t ? wv : xb, lse) : (mine_t ? wv : xb);
           if (rec_on) {
             if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
             if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
@@ -740,6 +746,8 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
       const bool in_row = rk < S && (rq > 0 || rk >= k);   // all-rows mode: rows before (t, k) are behind us
       const bool ready = in_row && t + rq < end && q1.w == static_cast<uint32_t>(t + rq) + 1u;
       const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+      const float lse = NORM ? lds_f32_volatile(summ_a + stq * kSumStageBytes + kSMax * 32u + 4u * min(rk, kSMax - 1)) : 0.0f;
+      const float xbs = NORM ? __fsub_rn(xb, lse) : xb;
       const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
       bool rescan = (q1.z & kSumOvf) != 0;
       // ---- the tokens the state's chain boosts: exact values; the lanes that share a row split the list
@@ -869,7 +877,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         const int pos = fq < kWin ? __popc(((tm | (fq == 0 ? pre : 0u)) >> (4 * fq)) & 0xFu) : 0;
         const unsigned upto = 0xFFFFFFFFu >> (31 - lane);                       // bits 0 .. lane
         const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
-        const float val = mine_t ? wv : xb;
+        const float val = NORM ? __fsub_rn(mine_t ? wv : xb, lse) : (mine_t ? wv : xb);
         if (rec_on) {
           if (mine_c) vlog[nv + __popc(cm & upto) - 1] = val;
           if (((cl >> lane) & 1u) && t + q + 1 >= f_mid)
@@ -906,15 +914,16 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         int nb = stop_m ? (__ffs(stop_m) - 1) >> 2 : kWin;
         if (wide) nb = (blank_m & 1u) ? 1 : 0;
         const int jl = wide ? 0 : 4 * min(nb, kWin - 1);
-        const float xb0 = __shfl_sync(0xffffffffu, xb, 0), xb1 = __shfl_sync(0xffffffffu, xb, 4);
+        const float xb0 = __shfl_sync(0xffffffffu, xbs, 0), xb1 = __shfl_sync(0xffffffffu, xbs, 4);
         const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
         const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
         const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
-        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+        const float j_val = __shfl_sync(0xffffffffu, NORM ? __fsub_rn(wv, lse) : wv, jl);
+        const float j_lse = NORM ? __shfl_sync(0xffffffffu, lse, jl) : 0.0f;
         const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
         if (nb > 0) score = __fadd_rn(score, xb0);
         if (nb > 1) score = __fadd_rn(score, xb1);
-        for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xb, 4 * r));
+        for (int r = 2; r < nb; ++r) score = __fadd_rn(score, __shfl_sync(0xffffffffu, xbs, 4 * r));
         adv = nb;
         progress = nb > 0;
         bool took = false;                                  // the row after the blanks was consumed too
@@ -943,7 +952,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
             __syncwarp();
             for (int i = lane; i < L.n; i += 32) { const int tk = (lds_v2(L.addr + 8u * i).x & kTokMask) >> 1; if (tk < V) tokidx[tk] = -1; }
             const Pick pk = warp_pick(best, bn);
-            tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
+            tok = pk.win.i; tval = NORM ? __fsub_rn(pk.win.v, j_lse) : pk.win.v; tnext = pk.next;
             if (tok == V) { score = __fadd_rn(score, tval); ++adv; }   // blank after all: that frame is passed too
           }
           if (tok != V) {
@@ -964,7 +973,7 @@ __global__ void __launch_bounds__(kThreadsF, 1) k_greedy_fast(FastParams P) {
         }
         if (rec_on) {
           // the values in visiting order, and the frame starts t + 1 .. t + adv this round reached
-          if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xb;
+          if ((lane & 3) == 0 && q < nb) vlog[nv + q] = xbs;
           if (took && lane == 0) vlog[nv + nb] = tval;
           if (lane < adv && t + lane + 1 >= f_mid) {
             const bool viatok = lane >= nb && tok != V;     // reached because the token closed its frame
@@ -1164,7 +1173,9 @@ int tb_launch_greedy_fast(const TbDecodeParams& d, int32_t max_cache_bytes, int3
   const Smem so = carve(nst, P.slot_bytes, d.V, d.C, P.cache_bytes, P.npipes, P.own_lists);
   if (so.total > budget) return 1;
   const int nit = (d.V + 255) / 256;
-  void (*fn)(FastParams) = nit <= 1 ? k_greedy_fast<1> : nit <= 2 ? k_greedy_fast<2> : nit <= 4 ? k_greedy_fast<4> : k_greedy_fast<8>;
+  void (*fn)(FastParams) = nit <= 1 ? k_greedy_fast<1, false> : nit <= 2 ? k_greedy_fast<2, false> : nit <= 4 ? k_greedy_fast<4, false> : k_greedy_fast<8, false>;
+  // rows normalised inside the selection (log-softmax): the helpers also leave every row's normaliser
+  if (d.normalize) fn = nit <= 1 ? k_greedy_fast<1, true> : nit <= 2 ? k_greedy_fast<2, true> : nit <= 4 ? k_greedy_fast<4, true> : k_greedy_fast<8, true>;
   if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess) {
     cudaGetLastError();
     return 1;

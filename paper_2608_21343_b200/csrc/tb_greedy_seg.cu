@@ -206,7 +206,7 @@ __device__ __forceinline__ void eval_list_all(uint32_t laddr, int first, int ste
 
 // One frame (S rows) reduced by a warp that is not a helper by trade: a decider whose own rows are not ready yet.
 // Two buffers: the next row is on its way while the current one is reduced.
-template <int NIT>
+template <int NIT, bool NORM>
 __device__ __noinline__ void summarize_frame(const HelperCtx h, unsigned char* bufs, int row_buf, const unsigned char* frame0,
                                              int row_bytes, int S, const unsigned char* lo, const unsigned char* hi,
                                              uint32_t out_a, uint32_t seq, int lane) {
@@ -216,7 +216,8 @@ __device__ __noinline__ void summarize_frame(const HelperCtx h, unsigned char* b
     if (k + 1 < S) { fetch_row(bufs + ((k + 1) & 1) * row_buf, rowp + row_bytes, row_bytes, lo, hi, lane); cp_async_wait<1>(); }
     else cp_async_wait<0>();
     __syncwarp();
-    summarize_row<NIT>(h, bufs + (k & 1) * row_buf, static_cast<int>(reinterpret_cast<uintptr_t>(rowp) & 15), out_a + k * 32, seq, lane);
+    summarize_row<NIT, NORM>(h, bufs + (k & 1) * row_buf, static_cast<int>(reinterpret_cast<uintptr_t>(rowp) & 15), out_a + k * 32, seq, lane,
+                             out_a + kSMax * 32 + 4 * k);
   }
 }
 
@@ -225,7 +226,7 @@ struct PipeInfo {   // one per pipeline of the block, in shared memory
   int32_t pad0, pad1;
 };
 
-template <int NIT>
+template <int NIT, bool NORM>
 __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
   extern __shared__ __align__(128) unsigned char dyn[];
   const TbDecodeParams& p = P.d;
@@ -384,9 +385,10 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         if (ng >= 0) cp_async_wait<1>(); else cp_async_wait<0>();
         __syncwarp();
         if (cf != P.withhold_frame)
-        summarize_row<NIT>(h, bufs + cb * so.row_buf, coff,
-                           summ_a + cg * kRingBytes + (cf & (kRing - 1)) * kSumStageBytes + ck * 32,
-                           static_cast<uint32_t>(cf) + 1u, lane);
+        summarize_row<NIT, NORM>(h, bufs + cb * so.row_buf, coff,
+                                 summ_a + cg * kRingBytes + (cf & (kRing - 1)) * kSumStageBytes + ck * 32,
+                                 static_cast<uint32_t>(cf) + 1u, lane,
+                                 summ_a + cg * kRingBytes + (cf & (kRing - 1)) * kSumStageBytes + kSMax * 32 + 4 * ck);
       }
       const bool had = cg >= 0;
       cg = ng; cf = nf; ck = nk; cb = nb_; coff = noff;
@@ -476,7 +478,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
           if (f >= end) continue;
           helped = true;
           if (f == P.withhold_frame) continue;
-          summarize_frame<NIT>(h, dyn + so.rows + (H + pipe) * kRowBufs * so.row_buf, so.row_buf,
+          summarize_frame<NIT, NORM>(h, dyn + so.rows + (H + pipe) * kRowBufs * so.row_buf, so.row_buf,
                                base + static_cast<int64_t>(f) * fsb, row_bytes, S, P.tensor_lo, P.tensor_hi,
                                summ_a + g * kRingBytes + (f & (kRing - 1)) * kSumStageBytes, static_cast<uint32_t>(f) + 1u, lane);
         }
@@ -496,6 +498,8 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         const unsigned char* rowp = base + static_cast<int64_t>(min(fq, end - 1)) * fsb + rk * row_bytes;
         const bool ready = fq < end && q1.w == static_cast<uint32_t>(fq) + 1u;
         const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+        // rows normalised: the row's normaliser comes off what the row adds to the score, after the selection
+        const float lse = NORM ? lds_f32_volatile(sring + (fq & (kRing - 1)) * kSumStageBytes + kSMax * 32u + 4u * rk) : 0.0f;
         const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
         // this lane's entries ql, ql + 4, ...: sorted by token, so a strict comparison keeps the lowest token
         float wv = -INFINITY;
@@ -538,7 +542,8 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
         const uint32_t j_tn = __shfl_sync(0xffffffffu, (static_cast<uint32_t>(wnext) << TB_RS_TOK_BITS) | static_cast<uint32_t>(wtok), jl);
         const int j_tok = static_cast<int>(j_tn & kTokMask), j_next = static_cast<int>(j_tn >> TB_RS_TOK_BITS);
-        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+        const float j_val = __shfl_sync(0xffffffffu, NORM ? __fsub_rn(wv, lse) : wv, jl);
+        const float xbs = NORM ? __fsub_rn(xb, lse) : xb;
         const bool took = nb < kWin && j_ready;             // the row after the blanks selects a token
         const bool rare = (nb == 0 && !took) || (took && j_rescan) || (took && (j_next < 0 || j_next >= rec.n_states));
         if (!rare) {
@@ -558,7 +563,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
           const int tnext = took ? j_next : s;
           n_out += took ? 1 : 0;
           // the values in visiting order, and the frame starts t + 1 .. t + adv this round reached
-          if ((lane & 3) == 0 && q < nb && nv + q < out_cap) vlog[nv + q] = xb;
+          if ((lane & 3) == 0 && q < nb && nv + q < out_cap) vlog[nv + q] = xbs;
           if (took && lane == 0 && nv + nb < out_cap) vlog[nv + nb] = j_val;
           if (lane < adv) TB_TRACE_PUT(t + lane + 1, lane >= nb ? tnext : s, n_out - ((took && lane < nb) ? 1 : 0), nv + lane + 1);
           nv += nb + (took ? 1 : 0);
@@ -587,6 +592,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         const uint4 q1 = lds_v4_volatile(sum_a + 16u);
         const uint4 q0 = lds_v4_volatile(sum_a);
         const float xb = __uint_as_float(q0.z);
+        const float lse = NORM ? lds_f32_volatile(sring + (fq & (kRing - 1)) * kSumStageBytes + kSMax * 32u + 4u * rkq) : 0.0f;
         // the plain winner: at the root (no list) it is the row's winner
         float wv = __fadd_rn(__uint_as_float(q0.w), __fmul_rn(lam, __fadd_rn(Lc.D, __uint_as_float(q1.x))));
         int wtok = static_cast<int>(q1.z & 0xFFFFu), wnext = bound ? static_cast<int>(q1.y) : -1;
@@ -639,7 +645,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
           const int pos = fcl < kWin ? __popc(((tm | (fcl == 0 ? pre : 0u)) >> (4 * (fcl & 7))) & 0xFu) : 0;
           const unsigned upto = 0xFFFFFFFFu >> (31 - lane);
           const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
-          const float val = mine_t ? wv : xb;
+          const float val = NORM ? __fsub_rn(mine_t ? wv : xb, lse) : (mine_t ? wv : xb);
           {
             const int vi = nv + __popc(cm & upto) - 1;
             if (mine_c && vi < out_cap) vlog[vi] = val;
@@ -685,6 +691,8 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
       const bool in_row = rk < S && (rq > 0 || rk >= k);   // all-rows mode: rows before (t, k) are behind us
       const bool ready = in_row && fq < end && q1.w == static_cast<uint32_t>(fq) + 1u;
       const float y1 = __uint_as_float(q0.x), y2b = __uint_as_float(q0.y), xb = __uint_as_float(q0.z), x1 = __uint_as_float(q0.w);
+      const float lse = NORM ? lds_f32_volatile(sring + (fq & (kRing - 1)) * kSumStageBytes + kSMax * 32u + 4u * min(rk, kSMax - 1)) : 0.0f;
+      const float xbs = NORM ? __fsub_rn(xb, lse) : xb;
       const uint32_t id1x2 = 2u * (q1.z & 0xFFFFu);
       bool rescan = (q1.z & kSumOvf) != 0;
       // ---- the tokens the state's chain boosts: exact values; the lanes that share a row split the list
@@ -762,7 +770,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         const int pos = fcl < kWin ? __popc(((tm | (fcl == 0 ? pre : 0u)) >> (4 * fcl)) & 0xFu) : 0;
         const unsigned upto = 0xFFFFFFFFu >> (31 - lane);                       // bits 0 .. lane
         const bool mine_c = (cm >> lane) & 1u, mine_t = (tm >> lane) & 1u;
-        const float val = mine_t ? wv : xb;
+        const float val = NORM ? __fsub_rn(mine_t ? wv : xb, lse) : (mine_t ? wv : xb);
         {
           const int vi = nv + __popc(cm & upto) - 1;
           if (mine_c && vi < out_cap) vlog[vi] = val;
@@ -802,7 +810,8 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         const bool j_ready = __shfl_sync(0xffffffffu, ready, jl);
         const bool j_rescan = __shfl_sync(0xffffffffu, rescan, jl);
         const int j_tok = __shfl_sync(0xffffffffu, wtok, jl);
-        const float j_val = __shfl_sync(0xffffffffu, wv, jl);
+        const float j_val = __shfl_sync(0xffffffffu, NORM ? __fsub_rn(wv, lse) : wv, jl);
+        const float j_lse = NORM ? __shfl_sync(0xffffffffu, lse, jl) : 0.0f;
         const int j_next = __shfl_sync(0xffffffffu, wnext, jl);
         adv = nb;
         progress = nb > 0;
@@ -836,7 +845,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
               if (better(c2, best)) { best = c2; bn = bound ? nx : -1; }
             }
             const Pick pk = warp_pick(best, bn);
-            tok = pk.win.i; tval = pk.win.v; tnext = pk.next;
+            tok = pk.win.i; tval = NORM ? __fsub_rn(pk.win.v, j_lse) : pk.win.v; tnext = pk.next;
             if (tok == V) ++adv;                              // blank after all: that frame is passed too
           }
           if (tok != V) {
@@ -856,7 +865,7 @@ __global__ void __launch_bounds__(kMaxThreadsS, 1) k_greedy_seg(SegParams P) {
         }
         {
           // the values in visiting order, and the frame starts t + 1 .. t + adv this round reached
-          if ((lane & 3) == 0 && q < nb && nv + q < out_cap) vlog[nv + q] = xb;
+          if ((lane & 3) == 0 && q < nb && nv + q < out_cap) vlog[nv + q] = xbs;
           if (took && lane == 0 && nv + nb < out_cap) vlog[nv + nb] = tval;
           if (lane < adv) {
             const bool viatok = lane >= nb && tok != V;     // reached because the token closed its frame
@@ -1099,7 +1108,9 @@ int tb_launch_greedy_seg(const TbDecodeParams& d, int32_t max_cache_bytes, const
   P.done = reinterpret_cast<uint32_t*>(sb + l.done);
   P.epoch = reinterpret_cast<uint32_t*>(sb + l.epoch);
   const int nit = (d.V + 255) / 256;
-  void (*fn)(SegParams) = nit <= 1 ? k_greedy_seg<1> : nit <= 2 ? k_greedy_seg<2> : nit <= 4 ? k_greedy_seg<4> : k_greedy_seg<8>;
+  void (*fn)(SegParams) = nit <= 1 ? k_greedy_seg<1, false> : nit <= 2 ? k_greedy_seg<2, false> : nit <= 4 ? k_greedy_seg<4, false> : k_greedy_seg<8, false>;
+  // rows normalised inside the selection (log-softmax): the helpers also leave every row's normaliser
+  if (d.normalize) fn = nit <= 1 ? k_greedy_seg<1, true> : nit <= 2 ? k_greedy_seg<2, true> : nit <= 4 ? k_greedy_seg<4, true> : k_greedy_seg<8, true>;
   if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem) != cudaSuccess) {
     cudaGetLastError();
     return TB_ERR_CUDA;

@@ -46,13 +46,24 @@ def test_normalised_greedy_decode(tb, dtype):
     lengths = [200, 199, 1, 0, 200, 150, 200, 200, 77, 200]
     out = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"]), lengths=torch.tensor(lengths, dtype=torch.int32, device="cuda:0")))
     assert tb.tb_batch_status(batch) == 0
-    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_GENERAL
+    # packed bf16 rows: a pipelined kernel (its helpers leave every row's normaliser, and the selection takes it off
+    # the selected value; ten streams: the segmented one); anything else: the general kernel, which normalises every
+    # entry before the bonus
+    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == (tb.TB_KERNEL_SEGMENTED if dtype == "bf16" else tb.TB_KERNEL_GENERAL)
     followed = rows = 0
     for i in range(w.B):
         f, r = compare(out, i, oracle_graph(w, lists[i]), data["logits"][i], lengths[i])
         followed += f
         rows += r
     assert followed <= 0.02 * rows                     # near-ties are the exception (they are counted, not ignored)
+    if dtype == "bf16":
+        # the same decode on the general kernel meets the same bar, and differs from the pipelined one by roundings only
+        tb.tb_batch_set_flags(batch, tb.TB_FLAG_LOG_SOFTMAX | tb.TB_FLAG_GENERAL_KERNELS)
+        gen = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"]), lengths=torch.tensor(lengths, dtype=torch.int32, device="cuda:0")))
+        assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == tb.TB_KERNEL_GENERAL
+        for i in range(w.B):
+            compare(gen, i, oracle_graph(w, lists[i]), data["logits"][i], lengths[i])
+        assert np.allclose(gen["scores"], out["scores"], rtol=0, atol=2e-3)
     # in exact arithmetic the tokens are those of the un-normalised decode: on these inputs almost every stream agrees
     tb.tb_batch_set_flags(batch, 0)
     plain = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"]), lengths=torch.tensor(lengths, dtype=torch.int32, device="cuda:0")))
@@ -66,7 +77,8 @@ def test_normalised_streaming_chunks_equal_the_offline_decode(tb):
     w = W.get_workload(2, B=4, T=64, n_phrases=40, n_plants=5)
     data = W.batch_inputs(w)
     batch, _ = make_batch(tb, w, data["phrases"])
-    tb.tb_batch_set_flags(batch, tb.TB_FLAG_LOG_SOFTMAX)
+    # (streaming chunks run on the general kernel; so does the offline decode they are compared with bit for bit)
+    tb.tb_batch_set_flags(batch, tb.TB_FLAG_LOG_SOFTMAX | tb.TB_FLAG_GENERAL_KERNELS)
     logits = to_device(data["logits"])
     off = to_host(tb.tb_greedy_decode(batch, logits))
     valid = torch.full((w.B,), w.T, dtype=torch.int32, device="cuda:0")
@@ -84,3 +96,37 @@ def test_normalised_streaming_chunks_equal_the_offline_decode(tb):
     tdt = torch.zeros((w.B, 8, w.S, w.V + 6), dtype=torch.bfloat16, device="cuda:0")
     with pytest.raises(tb.TbError):
         tb.tb_stream_chunk(batch, tdt, 5, valid)
+
+
+@pytest.mark.parametrize("wl,B,T,one_block", [(2, 16, 750, False), (2, 16, 750, True), (2, 3, 100, False), (2, 3, 100, True),
+                                               (3, 3, 300, True)])
+def test_normalised_decode_on_the_pipelined_kernels(tb, wl, B, T, one_block):
+    """The benchmark's workload (and a short case, and large lists that the decider walks in the arena) with rows
+    normalised, on the segmented kernel and on the one-block-per-stream kernel with one and two segments: bound and
+    unbound slots, ragged lengths; every stream against the oracle's normalised decode."""
+    w = W.get_workload(wl, B=B, T=T)
+    data = W.batch_inputs(w)
+    lists = list(data["phrases"])
+    lists[1] = None
+    batch, _ = make_batch(tb, w, lists)
+    base = tb.TB_FLAG_ONE_BLOCK_PER_STREAM if one_block else 0
+    tb.tb_batch_set_flags(batch, base | tb.TB_FLAG_LOG_SOFTMAX)
+    lengths = np.full(B, T, dtype=np.int32)
+    lengths[2] = T - 37
+    out = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"]), lengths=torch.from_numpy(lengths).to("cuda:0")))
+    assert tb.tb_batch_status(batch) == 0
+    ran = tb.tb_batch_last_greedy_kernel(batch)["kernel"]
+    assert ran == (tb.TB_KERNEL_PIPELINED if one_block else tb.TB_KERNEL_SEGMENTED)   # (large lists: always one block per stream)
+    followed = rows = 0
+    for i in range(B):
+        f, r = compare(out, i, oracle_graph(w, lists[i]), data["logits"][i], int(lengths[i]))
+        followed += f
+        rows += r
+    assert followed <= 0.02 * rows
+    # the tokens are those of the un-normalised decode (the normaliser is taken off after the selection)
+    tb.tb_batch_set_flags(batch, base)
+    plain = to_host(tb.tb_greedy_decode(batch, to_device(data["logits"]), lengths=torch.from_numpy(lengths).to("cuda:0")))
+    assert tb.tb_batch_last_greedy_kernel(batch)["kernel"] == ran
+    assert np.array_equal(plain["counts"], out["counts"]) and np.array_equal(plain["states"], out["states"])
+    for i in range(B):
+        assert np.array_equal(plain["tokens"][i, :plain["counts"][i]], out["tokens"][i, :out["counts"][i]])
