@@ -1616,12 +1616,13 @@ __global__ void k_beam_reset_slots(int32_t* slot_pos, unsigned long long* hash, 
 // of len_base that the slot's last step wrote; else the batch-wide tree [n_steps, B, K] with the records at len_cur.
 // sl / use_list: the slots to walk (output row i belongs to sl.slot[i]); else slot = block index.
 constexpr int kBtSteps = 32;
+constexpr int kBtBufs = 4;         // stages in flight: the copies of the next three are under way while one is walked
 template <bool RING>
 __global__ void __launch_bounds__(32) k_beam_backtrace_warp(const int2* tree, int32_t tree_cap, const int32_t* slot_pos, int32_t n_steps,
                                                            int32_t B, int32_t K, int32_t V, int32_t max_len, int32_t* out_tokens,
                                                            int32_t* out_lens, int32_t* status, const int32_t* len_base,
                                                            size_t n_hyp, const int32_t* len_cur, SlotList sl, int32_t use_list) {
-  extern __shared__ int2 bt_stage[];                         // [kBtSteps][K]
+  extern __shared__ __align__(16) int2 bt_stage[];           // [kBtBufs][kBtSteps][K]
   const int lane = threadIdx.x;
   const int b = use_list ? sl.slot[blockIdx.x] : blockIdx.x;
   const int32_t pos = RING ? slot_pos[b] : n_steps;
@@ -1636,34 +1637,45 @@ __global__ void __launch_bounds__(32) k_beam_backtrace_warp(const int2* tree, in
     n = lens ? lens[static_cast<int64_t>(b) * K + lane] : 0;
     out_lens[row] = n;
   }
+  // A stage is the nodes of up to kBtSteps consecutive steps, [step][K], brought in by asynchronous copies: 16 bytes
+  // (two nodes) each when K is even (a step's K nodes are contiguous and then start on a 16-byte boundary), else 8.
+  const bool wide = (K & 1) == 0 && (reinterpret_cast<uintptr_t>(tree) & 15) == 0;
+  const int per_step = wide ? K >> 1 : K;                    // copies per step
+  const uint32_t stage_a = static_cast<uint32_t>(__cvta_generic_to_shared(bt_stage));
+  const int n_stages = (pos - first + kBtSteps - 1) / kBtSteps;
+  const int ps_shift = (per_step & (per_step - 1)) == 0 ? 31 - __clz(per_step) : -1;   // copies per step a power of two: shifts
+  auto fetch = [&](int sidx) {                               // stage sidx holds steps [lo, hi), hi = pos - sidx * kBtSteps
+    if (sidx < n_stages) {
+      const int32_t hi = pos - sidx * kBtSteps, lo = max(first, hi - kBtSteps), cnt = hi - lo;
+      const uint32_t dst0 = stage_a + static_cast<uint32_t>(sidx % kBtBufs) * (kBtSteps * K * 8u);
+      const int32_t r0 = RING ? lo % tree_cap : 0;           // ring position of the stage's first step
+      const int2* base = RING ? tree + static_cast<int64_t>(b) * tree_cap * K : tree + static_cast<int64_t>(b) * K;
+      const int64_t step_stride = RING ? K : static_cast<int64_t>(B) * K;
+      const int total = cnt * per_step;
+      for (int e = lane; e < total; e += 32) {
+        const int j = ps_shift >= 0 ? e >> ps_shift : e / per_step;
+        const int c = e - j * per_step;
+        int32_t sj = RING ? r0 + j : lo + j;
+        if (RING && sj >= tree_cap) sj -= tree_cap;
+        const int2* src = base + sj * step_stride;
+        if (wide) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (j * K + 2 * c) * 8u), "l"(src + 2 * c) : "memory");
+        else asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst0 + (j * K + c) * 8u), "l"(src + c) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");      // (one group per call, empty beyond the last stage)
+  };
   for (int pass = count_first ? 0 : 1; pass < 2; ++pass) {
     int32_t cur = lane < K ? lane : -1, at = n;
-    for (int32_t hi = pos; hi > first; hi -= kBtSteps) {
-      if (!__any_sync(0xffffffffu, cur >= 0 && (pass == 0 || at > 0))) break;
-      const int32_t lo = max(first, hi - kBtSteps), cnt = hi - lo;
-      // (eight nodes per lane are requested before the first is stored: one trip for all of them)
-      for (int e0 = 0; e0 < cnt * K; e0 += 32 * 8) {
-        int2 v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int e = e0 + 32 * u + lane;
-          if (e < cnt * K) {
-            const int j = e / K, kk = e - j * K;
-            const int32_t st = lo + j;
-            const int64_t node = RING ? (static_cast<int64_t>(b) * tree_cap + (st % tree_cap)) * K + kk
-                                      : (static_cast<int64_t>(st) * B + b) * K + kk;
-            v[u] = tree[node];
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int e = e0 + 32 * u + lane;
-          if (e < cnt * K) bt_stage[e] = v[u];
-        }
-      }
+    for (int sidx = 0; sidx < kBtBufs - 1; ++sidx) fetch(sidx);
+    for (int sidx = 0; sidx < n_stages; ++sidx) {
+      fetch(sidx + kBtBufs - 1);
+      asm volatile("cp.async.wait_group %0;" ::"n"(kBtBufs - 1) : "memory");
       __syncwarp();
+      if (!__any_sync(0xffffffffu, cur >= 0 && (pass == 0 || at > 0))) break;
+      const int32_t hi = pos - sidx * kBtSteps, lo = max(first, hi - kBtSteps), cnt = hi - lo;
+      const int2* stg = bt_stage + static_cast<size_t>(sidx % kBtBufs) * (kBtSteps * K);
       for (int j = cnt - 1; j >= 0 && cur >= 0; --j) {
-        const int2 e = bt_stage[j * K + cur];
+        const int2 e = stg[j * K + cur];
         if (e.y >= 0 && e.y != V) {
           if (pass == 0) ++n;
           else { --at; if (at >= 0 && at < max_len) out_tokens[row * max_len + at] = e.y; }
@@ -1672,6 +1684,8 @@ __global__ void __launch_bounds__(32) k_beam_backtrace_warp(const int2* tree, in
       }
       __syncwarp();
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncwarp();
     if (pass == 0 && lane < K) out_lens[row] = n;
   }
 }
@@ -1777,7 +1791,7 @@ int tb_launch_beam_backtrace(const int2* tree, int32_t n_steps, int32_t B, int32
                              int32_t* out_tokens, int32_t* out_lens, const int32_t* len_cur, cudaStream_t stream) {
   SlotList none;
   for (int i = 0; i < TB_BIND_PAIRS; ++i) none.slot[i] = 0;
-  k_beam_backtrace_warp<false><<<B, 32, kBtSteps * K * sizeof(int2), stream>>>(tree, 0, nullptr, n_steps, B, K, V, max_len, out_tokens,
+  k_beam_backtrace_warp<false><<<B, 32, kBtBufs * kBtSteps * K * sizeof(int2), stream>>>(tree, 0, nullptr, n_steps, B, K, V, max_len, out_tokens,
                                                                               out_lens, nullptr, nullptr, 0, len_cur, none, 0);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
@@ -1910,7 +1924,7 @@ int tb_launch_beam_backtrace_slots(const int2* tree, int32_t tree_cap, const int
   if (slot_list && n_slots > TB_BIND_PAIRS) return TB_ERR_INVALID_ARG;
   SlotList sl;
   for (int i = 0; i < TB_BIND_PAIRS; ++i) sl.slot[i] = (slot_list && i < n_slots) ? slot_list[i] : 0;
-  k_beam_backtrace_warp<true><<<n_slots, 32, kBtSteps * K * sizeof(int2), stream>>>(tree, tree_cap, slot_pos, 0, n_slots, K, V, max_len,
+  k_beam_backtrace_warp<true><<<n_slots, 32, kBtBufs * kBtSteps * K * sizeof(int2), stream>>>(tree, tree_cap, slot_pos, 0, n_slots, K, V, max_len,
                                                                                    out_tokens, out_lens, status, len_base, n_hyp, nullptr,
                                                                                    sl, slot_list ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
