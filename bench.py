@@ -37,13 +37,14 @@ from paper_2608_21343_b200 import workloads as W  # noqa: E402
 METRIC = "boosted_greedy_decode_frames_per_s_B128"
 UNIT = "frames/s"
 # DRAM read + write bytes per logits row of k_greedy_fast, from an ncu capture of one 32-stream launch
-# (155.37 MB read + 5.68 MB written for 72000 rows: each stream's second segment re-reads 16 warm-up frames, and
+# (155.53 MB read + 3.83 MB written for 72000 rows: each stream's second segment re-reads 16 warm-up frames, and
 # what it emits goes through scratch memory); the kernel runs one block per stream, so traffic scales with the
 # stream count.  Captured with the command recorded in profiles/greedy_fast_small_case_B32_counters.md
 # (`python bench.py --streams 32 --steps 2 --warmup 3 --no-extras --one-block-per-stream` under
-# `ncu --clock-control none -k regex:k_greedy_fast -s 4 -c 1 ...`) on the kernel as of the commit that split its
-# row-summary code into tb_fast_common.cuh; to be re-captured whenever tb_greedy_fast.cu or that header changes.
-NCU_DRAM_BYTES_PER_ROW = 2237.0
+# `ncu --clock-control none -k regex:k_greedy_fast -s 4 -c 1 ...`) on the kernel as of the commit that made it a
+# template over "rows normalised or not" (the plain instance; the earlier captures read 2233 and 2237); to be
+# re-captured whenever tb_greedy_fast.cu or tb_fast_common.cuh changes.
+NCU_DRAM_BYTES_PER_ROW = 2213.0
 
 
 def load_peaks():
@@ -543,6 +544,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip unboosted / e2e / cpu legs (profiling)")
     ap.add_argument("--one-block-per-stream", action="store_true",
                     help="never the segmented kernel (small-case captures of k_greedy_fast: fewer streams would otherwise select it)")
+    ap.add_argument("--log-softmax", action="store_true",
+                    help="the timed decode normalises every visited row (TB_FLAG_LOG_SOFTMAX): a side measurement and profiling captures, not the headline")
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4, 5, 6, 7, 8],
                     help="2 = the headline (default); 3 large lists, 4 beam, 5 streaming TDT with churn, 6 variative lists, 7 model lifecycle sweep: side measurements")
     args = ap.parse_args()
@@ -588,9 +591,10 @@ def main():
     for i, g in enumerate(graphs):
         tb.tb_batch_bind_stream(batch, i, g)
     plain = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=1 << 20, device=local_rank)  # all unbound
-    if args.one_block_per_stream:
-        tb.tb_batch_set_flags(batch, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
-        tb.tb_batch_set_flags(plain, tb.TB_FLAG_ONE_BLOCK_PER_STREAM)
+    main_flags = (tb.TB_FLAG_ONE_BLOCK_PER_STREAM if args.one_block_per_stream else 0) | (tb.TB_FLAG_LOG_SOFTMAX if args.log_softmax else 0)
+    if main_flags:
+        tb.tb_batch_set_flags(batch, main_flags)
+        tb.tb_batch_set_flags(plain, main_flags)
     out = tb.tb_greedy_decode(batch, logits)
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
@@ -654,7 +658,7 @@ def main():
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "T": w.T, "S": w.S, "V": w.V, "logits": w.dtype,
-                   "phrases_per_stream": w.n_phrases, "l2": "inputs (590 MB per step) larger than L2, no flush",
+                   "phrases_per_stream": w.n_phrases, "log_softmax": bool(args.log_softmax), "l2": "inputs (590 MB per step) larger than L2, no flush",
                    "parallelism": f"replicas x{world}, streams partitioned, no collective"},
         "gpu_launches": args.steps * 1,
         "clocks": clocks,
@@ -707,7 +711,7 @@ def main():
                                "same_token_counts_as_in_full_batch": bool(same_)}
             sb_.destroy()
         result["smaller_batches"] = small
-    if not args.no_extras and rank == 0:
+    if not args.no_extras and rank == 0 and not args.log_softmax:
         # the same decode with every row log-softmax normalised inside the selection (TB_FLAG_LOG_SOFTMAX): the
         # helpers also leave each row's normaliser; reported beside the headline, not part of it
         base_flags = tb.TB_FLAG_ONE_BLOCK_PER_STREAM if args.one_block_per_stream else 0
