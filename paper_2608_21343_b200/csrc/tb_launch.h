@@ -15,7 +15,7 @@ struct TbDecodeParams {
   const int32_t* lengths;    // device [n_streams] or null
   int32_t persistent;        // 0: offline greedy (fresh state); 1: streaming (TbSlotState)
   int32_t tokview;           // set by the launcher: shared memory is sized for the token view of resolved lists
-  int32_t normalize;         // general kernel only: every visited row is log-softmax normalised before the bonus is added
+  int32_t normalize;         // every visited row is scored by its log-softmax (general kernel: before the bonus is added; pipelined kernels: the normaliser comes off the selected value)
   int32_t* out_tokens; int32_t* out_frames; int32_t* out_durs; int32_t* out_counts;
   float* out_scores; int32_t* out_states; int32_t* out_cursors;
   int32_t out_cap;           // tokens per stream the output arrays can hold
