@@ -1484,6 +1484,10 @@ __global__ void __launch_bounds__(kTopWarps * 32) k_beam_topm(const LT* logits, 
   }
   __syncwarp();
   int n_taken = 0;      // of this lane's strip
+  // The rounds only note which token won and its y (the owner's registers hold both); the logit and the class of the
+  // picks are looked up afterwards by all lanes at once, so that no round waits for a trip to memory.
+  float* pick_y = reinterpret_cast<float*>(ybuf + static_cast<size_t>(kTopWarps) * V) + static_cast<size_t>(warp) * 2 * (top_m + 1);
+  int32_t* pick_i = reinterpret_cast<int32_t*>(pick_y + (top_m + 1));
   for (int m = 0; m <= top_m; ++m) {
     // the warp's best: largest value, then lowest token
     const uint32_t u = __float_as_uint(v0 + 0.0f);
@@ -1491,32 +1495,38 @@ __global__ void __launch_bounds__(kTopWarps * 32) k_beam_topm(const LT* logits, 
     const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
     const uint32_t imin = __reduce_min_sync(0xffffffffu, (key == kmax && i0 != INT32_MAX) ? static_cast<uint32_t>(i0) : 0xFFFFFFFFu);
     const bool none = imin == 0xFFFFFFFFu;                    // fewer than m + 1 tokens in the row
-    if (m == top_m) {
-      if (lane == 0) { o[m].y = none ? -INFINITY : y[imin]; o[m].x = LogitLoad<LT>::at(row + V); o[m].tok_cls = 0u; }
-      break;
-    }
-    if (lane == 0) {
-      if (none) { o[m].y = -INFINITY; o[m].x = -INFINITY; o[m].tok_cls = 0xFFFFu; }
-      else { o[m].y = y[imin]; o[m].x = LogitLoad<LT>::at(row + imin); o[m].tok_cls = imin | (static_cast<uint32_t>(__ldg(cls + imin)) << 16); }
-    }
-    if (!none && static_cast<uint32_t>(i0) == imin) {
-      // the owner takes it out: its next best moves up; when the three it kept are used up and the strip holds
-      // more, it looks through the strip again
-      y[i0] = __int_as_float(0x7FC00000);                     // (a NaN: never greater than anything, never chosen again)
-      ++n_taken;
-      v0 = v1; i0 = i1; v1 = v2; i1 = i2; v2 = -INFINITY; i2 = INT32_MAX;
-      if (i0 == INT32_MAX && n_taken < n_strip) {
-        for (int v = lane; v < V; v += 32) {
-          const float yv = y[v];
-          if (yv == yv) {
-            if (yv > v0 || i0 == INT32_MAX) { v2 = v1; i2 = i1; v1 = v0; i1 = i0; v0 = yv; i0 = v; }
-            else if (yv > v1 || i1 == INT32_MAX) { v2 = v1; i2 = i1; v1 = yv; i1 = v; }
-            else if (yv > v2 || i2 == INT32_MAX) { v2 = yv; i2 = v; }
+    if (none) {
+      if (lane == 0) { pick_y[m] = -INFINITY; pick_i[m] = -1; }
+    } else if (static_cast<uint32_t>(i0) == imin) {
+      pick_y[m] = v0; pick_i[m] = i0;
+      if (m < top_m) {
+        // the owner takes it out: its next best moves up; when the three it kept are used up and the strip holds
+        // more, it looks through the strip again
+        y[i0] = __int_as_float(0x7FC00000);                   // (a NaN: never greater than anything, never chosen again)
+        ++n_taken;
+        v0 = v1; i0 = i1; v1 = v2; i1 = i2; v2 = -INFINITY; i2 = INT32_MAX;
+        if (i0 == INT32_MAX && n_taken < n_strip) {
+          for (int v = lane; v < V; v += 32) {
+            const float yv = y[v];
+            if (yv == yv) {
+              if (yv > v0 || i0 == INT32_MAX) { v2 = v1; i2 = i1; v1 = v0; i1 = i0; v0 = yv; i0 = v; }
+              else if (yv > v1 || i1 == INT32_MAX) { v2 = v1; i2 = i1; v1 = yv; i1 = v; }
+              else if (yv > v2 || i2 == INT32_MAX) { v2 = yv; i2 = v; }
+            }
           }
         }
       }
     }
     __syncwarp();
+  }
+  for (int m = lane; m <= top_m; m += 32) {
+    const int i = pick_i[m];
+    TbTopEnt e;
+    e.y = pick_y[m];
+    if (m == top_m) { e.x = LogitLoad<LT>::at(row + V); e.tok_cls = 0u; }
+    else if (i < 0) { e.x = -INFINITY; e.tok_cls = 0xFFFFu; }
+    else { e.x = LogitLoad<LT>::at(row + i); e.tok_cls = static_cast<uint32_t>(i) | (static_cast<uint32_t>(__ldg(cls + i)) << 16); }
+    o[m] = e;
   }
 }
 
@@ -1951,7 +1961,8 @@ int tb_launch_beam_topm(const void* logits, int dtype, int32_t B, int32_t T, int
                         int64_t stream_stride, int64_t frame_stride, int64_t row_stride, const int32_t* n_frames,
                         const TbSlotRec* slots, const unsigned char* arena, const int32_t* cls, int32_t top_m,
                         TbTopEnt* out, cudaStream_t stream) {
-  const size_t smem = (static_cast<size_t>(C) + static_cast<size_t>(kTopWarps) * V) * sizeof(float);
+  // root weights per class, every warp's y values, every warp's picks (value and token, top_m + 1 each)
+  const size_t smem = (static_cast<size_t>(C) + static_cast<size_t>(kTopWarps) * V + static_cast<size_t>(kTopWarps) * 2 * (top_m + 1)) * sizeof(float);
   const int blocks = B * ((T * E + kTopWarps - 1) / kTopWarps);
   int rc;
   if (dtype == TB_BF16) {
