@@ -81,6 +81,8 @@ extern "C" {
                                            by a few float roundings per visited row */
 #define TB_FLAG_BEAM_WHOLE_ROWS 16      /* tb_beam_frames / tb_beam_chunk: no pre-pass that reduces every row to its best tokens; every
                                            step looks at all vocab+1 entries of its row (identical results) */
+#define TB_FLAG_COPIED_BINDS 32         /* tb_stream_chunk_binds: always bind ahead of the chunk's launch (copies + a small launch), never
+                                           inside it */
 #define TB_FLAG_TEST_WAIT_TIMEOUT 4     /* self-test of the kernels' bounded waits: tb_greedy_decode (segmented kernel) withholds one
                                            frame's summaries and waits only briefly, so the wait runs out: the call returns,
                                            TB_STATUS_WAIT_TIMEOUT is set, the outputs of that call are undefined */
@@ -408,13 +410,22 @@ int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots,
                     float *out_scores, int32_t *out_states, int32_t *out_cursors, void *stream);
 
 /*
- * The streams that start with a chunk and the chunk itself in one call (Sec. 2.2 para. 4, Sec. 2.3): first
- * tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream), then tb_stream_chunk with the remaining
- * arguments, both enqueued on `stream`.  A server that gets its new streams' lists with the audio saves one trip
- * through its language binding per chunk; nothing else differs from the two calls made one after the other.
- * n_binds may be 0 (bind_slots / bind_graphs are then not read).  If the binds fail the chunk is not decoded.
- * Errors: those of the two calls.
+ * The streams that start with a chunk and the chunk itself in one call (Sec. 2.2 para. 4, Sec. 2.3): the result is
+ * that of tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream) followed by tb_stream_chunk with the
+ * remaining arguments, both on `stream`.  The chunk's arguments are checked first: a chunk that would be refused
+ * binds nothing.  n_binds may be 0 (bind_slots / bind_graphs are then not read).  If the binds fail the chunk is not
+ * decoded.  Errors: those of the two calls.
+ *
+ * Up to 8 binds per call ride on the chunk's own launch: when every graph's image lies in the library's page-locked
+ * memory (graphs compiled or loaded after the first tb_batch_create, without TB_COMPILE_PAGEABLE, not handed out by
+ * a cache), the bound slots are among the chunk's n_slots, and `stream` is not being captured, the call reserves
+ * the arena blocks, and the thread block that decodes a re-bound slot first reads the new image from host memory in
+ * place into its arena block, stores the slot's record and starts the stream afresh, while all other slots' blocks
+ * decode already: no copy is enqueued and no second launch is made.  The library holds the graphs until that
+ * launch has completed, as for a copy.  Anything else goes the ordinary way (copies and a small launch ahead of the
+ * chunk).  tb_batch_bind_counts tells how many binds went which way.
  */
+int tb_batch_bind_counts(const tb_batch *b, int64_t *out_pulled, int64_t *out_copied);   /* binds of tb_stream_chunk_binds so far: inside the chunk's launch / ahead of it */
 int tb_stream_chunk_binds(tb_batch *b, int32_t n_binds, const int32_t *bind_slots, const tb_graph *const *bind_graphs,
                           const void *logits, int dtype, int32_t n_slots, int32_t chunk, int32_t S, int32_t n_dur,
                           const int64_t *strides, const int32_t *valid_frames, int32_t *out_tokens, int32_t *out_frames,

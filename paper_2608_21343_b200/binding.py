@@ -77,6 +77,7 @@ _SIGS = {
     "tb_batch_set_flags": (C.c_int, [_vp, C.c_uint32]),
     "tb_batch_set_greedy_plan": (C.c_int, [_vp, _i32, _i32, _i32]),
     "tb_batch_last_greedy_kernel": (C.c_int, [_vp, C.POINTER(_i32), C.POINTER(_i32), C.POINTER(_i32)]),
+    "tb_batch_bind_counts": (C.c_int, [_vp, C.POINTER(_i64), C.POINTER(_i64)]),
     "tb_greedy_decode": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "tb_stream_chunk": (C.c_int, [_vp, _vp, C.c_int, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
                                   _vp, _vp, _vp]),
@@ -364,6 +365,7 @@ TB_FLAG_ONE_BLOCK_PER_STREAM = 2
 TB_FLAG_TEST_WAIT_TIMEOUT = 4
 TB_FLAG_LOG_SOFTMAX = 8
 TB_FLAG_BEAM_WHOLE_ROWS = 16
+TB_FLAG_COPIED_BINDS = 32
 TB_KERNEL_GENERAL, TB_KERNEL_PIPELINED, TB_KERNEL_SEGMENTED = 1, 2, 3
 
 
@@ -393,6 +395,13 @@ def tb_batch_last_greedy_kernel(batch: Batch) -> dict:
     _check(_lib.tb_batch_last_greedy_kernel(batch.handle, C.byref(k), C.byref(nb), C.byref(g)),
            "tb_batch_last_greedy_kernel")
     return dict(kernel=k.value, blocks_per_stream=nb.value, deciders_per_block=g.value)
+
+
+def tb_batch_bind_counts(batch: Batch) -> dict:
+    """Binds of tb_stream_chunk_binds so far: carried out inside the chunk's launch / ahead of it."""
+    pulled, copied = _i64(0), _i64(0)
+    _check(_lib.tb_batch_bind_counts(batch.handle, C.byref(pulled), C.byref(copied)), "tb_batch_bind_counts")
+    return dict(pulled=pulled.value, copied=copied.value)
 
 
 def tb_batch_status(batch: Batch, stream=None) -> int:

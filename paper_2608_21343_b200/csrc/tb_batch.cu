@@ -92,6 +92,7 @@ struct PinnedPool {
   std::mutex mu;
   struct Chunk {
     unsigned char* base;
+    unsigned char* dev_base;                                       // the same memory as kernels address it, or null
     size_t bytes;
     std::map<size_t, size_t> free_blocks;                          // offset -> bytes, neighbours coalesced
   };
@@ -134,13 +135,18 @@ void* tb_pinned_alloc(size_t bytes) {
       }
     if (pass == 1 || pool.closed || pool.total + kPoolChunk > kPoolMax) return nullptr;
     void* base = nullptr;
-    if (cudaHostAlloc(&base, kPoolChunk, cudaHostAllocPortable) != cudaSuccess) {
+    if (cudaHostAlloc(&base, kPoolChunk, cudaHostAllocPortable | cudaHostAllocMapped) != cudaSuccess) {
       cudaGetLastError();
       pool.closed = true;
       return nullptr;
     }
     PinnedPool::Chunk c;
     c.base = static_cast<unsigned char*>(base); c.bytes = kPoolChunk;
+    // kernels may read the piece in place (a bind that the decoding kernel carries out itself) where the device
+    // addresses it like the host does -- unified addressing --, which is what makes the address good on every device
+    void* dev = nullptr;
+    if (cudaHostGetDevicePointer(&dev, base, 0) != cudaSuccess) { cudaGetLastError(); dev = nullptr; }
+    c.dev_base = dev == base ? static_cast<unsigned char*>(dev) : nullptr;
     c.free_blocks[0] = kPoolChunk;
     pool.chunks.push_back(std::move(c));
     pool.total += kPoolChunk;
@@ -156,6 +162,16 @@ bool tb_pinned_owns(const void* p) {
   for (auto& c : pool.chunks)
     if (q >= c.base && q < c.base + c.bytes) return true;
   return false;
+}
+
+const unsigned char* tb_pinned_device_ptr(const void* p) {
+  PinnedPool& pool = pinned_pool();
+  if (!pool.armed.load() || !p) return nullptr;
+  std::lock_guard<std::mutex> lock(pool.mu);
+  const unsigned char* q = static_cast<const unsigned char*>(p);
+  for (auto& c : pool.chunks)
+    if (q >= c.base && q < c.base + c.bytes) return c.dev_base ? c.dev_base + (q - c.base) : nullptr;
+  return nullptr;
 }
 
 bool tb_pinned_free(void* p, size_t bytes) {
@@ -230,6 +246,7 @@ struct tb_batch {
   int32_t plan_G = 0, plan_H = 0, plan_NB = 0;   // tb_batch_set_greedy_plan (0: automatic)
   int32_t last_kernel = 0, last_NB = 0, last_G = 0;
   int32_t n_sm = 0, max_smem = 0;
+  int64_t n_pulled_binds = 0, n_copied_binds = 0;   // tb_stream_chunk_binds: binds carried out by the chunk's launch / ahead of it
 };
 
 static void destroy_batch(tb_batch* b) {
@@ -530,6 +547,67 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   return TB_OK;
 }
 
+// A group of binds prepared for the streaming chunk launch that follows to carry out itself (see TbInlineBinds): room in
+// the arena, the records, the host's bookkeeping -- no copy, no launch.  Taken when every graph's image sits in the
+// page-locked pool at an address the device can read, the group is small enough for the launch's parameters, and the
+// stream is not being captured (a captured launch would keep the host addresses).  Returns false, with nothing
+// changed, when the group has to go the ordinary way (tb_batch_bind_streams, which also reports what is wrong with it).
+// *used: the staging entry that holds the graphs until the launch is done; the caller records its event after the
+// launch.  let_go: graphs of that entry's previous use, to be released after the launch has been issued.
+static bool prepare_pulled_binds(tb_batch* b, int32_t n, const int32_t* slots, const tb_graph* const* graphs, cudaStream_t stream,
+                                 TbInlineBinds* ib, Staging** used, std::vector<tb_graph*>* let_go) {
+  if (n < 1 || n > TB_INLINE_BINDS || !slots || !graphs) return false;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (cap != cudaStreamCaptureStatusNone) return false;
+  size_t total = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    if (slots[i] < 0 || slots[i] >= b->n_slots) return false;
+    for (int32_t j = 0; j < i; ++j)
+      if (slots[j] == slots[i]) return false;
+    const tb_graph* g = graphs[i];
+    ib->slot[i] = slots[i]; ib->src[i] = nullptr; ib->bytes[i] = 0;
+    if (!g) continue;
+    if (g->vocab != b->vocab || g->class_map_hash != b->class_map_hash) return false;
+    if (!g->pinned || g->registered || g->blob.size() > static_cast<size_t>(INT32_MAX)) return false;
+    ib->src[i] = tb_pinned_device_ptr(g->blob.data());
+    if (!ib->src[i]) return false;
+    ib->bytes[i] = static_cast<int32_t>(g->blob.size());
+    total += round_up(g->blob.size(), kArenaAlign);
+  }
+  size_t base = 0;
+  if (total > 0 && !b->alloc.alloc(total, &base)) return false;
+  Staging& s = b->staging[b->next_staging];
+  b->next_staging = (b->next_staging + 1) % kStagingRing;
+  if (s.pending) {
+    if (cudaEventSynchronize(s.done) != cudaSuccess) { cudaGetLastError(); if (total) b->alloc.release(base, total); return false; }
+    s.pending = false;
+  }
+  let_go->swap(s.held_more);
+  if (s.held) { let_go->push_back(s.held); s.held = nullptr; }
+  size_t at = 0;
+  for (int32_t i = 0; i < n; ++i) {
+    const tb_graph* g = graphs[i];
+    std::pair<size_t, size_t> block{0, 0};
+    if (g) {
+      fill_record(g, base + at, &ib->rec[i]);
+      block = {base + at, round_up(g->blob.size(), kArenaAlign)};
+      at += block.second;
+      tb_graph* h = const_cast<tb_graph*>(g); h->refs.fetch_add(1); s.held_more.push_back(h);
+    } else {
+      std::memset(&ib->rec[i], 0, sizeof(TbSlotRec));
+    }
+    release_slot(b, slots[i]);                       // (after the group's room was taken: the new blocks are none of the old)
+    b->slot_block[slots[i]] = block;
+    b->slot_n_states[slots[i]] = g ? g->n_states : 0;
+    b->slot_cache_bytes[slots[i]] = !g ? 0 : cache_bytes_of(g);
+    b->slot_resolved[slots[i]] = (!g || g->n_rsent >= 0) ? 1 : 0;
+  }
+  ib->n = n; ib->arena = b->arena; ib->slots = b->d_slots;
+  *used = &s;
+  return true;
+}
+
 extern "C" int tb_batch_register_model(tb_batch* b, const tb_graph* g, int32_t* out_model_id, void* stream_) {
   TbRange range_("tb_batch_register_model");
   if (!b || !g || !out_model_id) return TB_ERR_INVALID_ARG;
@@ -787,8 +865,23 @@ extern "C" int tb_apply_final_weights(tb_batch* b, int32_t B, int32_t K, float* 
 
 extern "C" int tb_batch_set_flags(tb_batch* b, uint32_t flags) {
   if (!b || (flags & ~static_cast<uint32_t>(TB_FLAG_GENERAL_KERNELS | TB_FLAG_ONE_BLOCK_PER_STREAM | TB_FLAG_TEST_WAIT_TIMEOUT | TB_FLAG_LOG_SOFTMAX |
-                                              TB_FLAG_BEAM_WHOLE_ROWS))) return TB_ERR_INVALID_ARG;
+                                              TB_FLAG_BEAM_WHOLE_ROWS | TB_FLAG_COPIED_BINDS))) return TB_ERR_INVALID_ARG;
   b->flags = flags;
+  return TB_OK;
+}
+
+static int stream_chunk_params(tb_batch* b, const void* logits, int dtype, int32_t n_slots, int32_t chunk, int32_t S, int32_t n_dur,
+                               const int64_t* strides, const int32_t* valid_frames, int32_t* out_tokens, int32_t* out_frames,
+                               int32_t* out_durs, int32_t* out_counts, float* out_scores, int32_t* out_states,
+                               int32_t* out_cursors, TbDecodeParams* p) {
+  int rc = fill_decode_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, p);
+  if (rc != TB_OK) return rc;
+  if (!valid_frames || !out_tokens || !out_frames || !out_counts || !out_scores || !out_states) return TB_ERR_INVALID_ARG;
+  p->lengths = valid_frames; p->persistent = 1;
+  p->normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;
+  if (p->normalize && n_dur != 0) return TB_ERR_INVALID_ARG;   // normalisation is defined for the token logits of an RNNT row
+  p->out_tokens = out_tokens; p->out_frames = out_frames; p->out_durs = out_durs; p->out_counts = out_counts;
+  p->out_scores = out_scores; p->out_states = out_states; p->out_cursors = out_cursors;
   return TB_OK;
 }
 
@@ -798,14 +891,9 @@ extern "C" int tb_stream_chunk(tb_batch* b, const void* logits, int dtype, int32
                                float* out_scores, int32_t* out_states, int32_t* out_cursors, void* stream_) {
   TbRange range_("tb_stream_chunk");
   TbDecodeParams p;
-  int rc = fill_decode_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, &p);
+  const int rc = stream_chunk_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, valid_frames, out_tokens, out_frames,
+                                     out_durs, out_counts, out_scores, out_states, out_cursors, &p);
   if (rc != TB_OK) return rc;
-  if (!valid_frames || !out_tokens || !out_frames || !out_counts || !out_scores || !out_states) return TB_ERR_INVALID_ARG;
-  p.lengths = valid_frames; p.persistent = 1;
-  p.normalize = (b->flags & TB_FLAG_LOG_SOFTMAX) ? 1 : 0;
-  if (p.normalize && n_dur != 0) return TB_ERR_INVALID_ARG;   // normalisation is defined for the token logits of an RNNT row
-  p.out_tokens = out_tokens; p.out_frames = out_frames; p.out_durs = out_durs; p.out_counts = out_counts;
-  p.out_scores = out_scores; p.out_states = out_states; p.out_cursors = out_cursors;
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
   return tb_launch_decode_general(p, static_cast<cudaStream_t>(stream_));
@@ -816,13 +904,53 @@ extern "C" int tb_stream_chunk_binds(tb_batch* b, int32_t n_binds, const int32_t
                                      const int64_t* strides, const int32_t* valid_frames, int32_t* out_tokens,
                                      int32_t* out_frames, int32_t* out_durs, int32_t* out_counts, float* out_scores,
                                      int32_t* out_states, int32_t* out_cursors, void* stream_) {
+  TbRange range_("tb_stream_chunk_binds");
   if (!b || n_binds < 0) return TB_ERR_INVALID_ARG;
+  // the chunk's arguments are checked before any bind changes anything
+  TbDecodeParams p;
+  int rc = stream_chunk_params(b, logits, dtype, n_slots, chunk, S, n_dur, strides, valid_frames, out_tokens, out_frames,
+                               out_durs, out_counts, out_scores, out_states, out_cursors, &p);
+  if (rc != TB_OK) return rc;
+  DeviceGuard guard(b->device);
+  if (!guard.ok) return TB_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (n_binds > 0) {
-    const int rc = tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream_);
+    // every bound slot must be one the chunk decodes, or its bind could not ride on the chunk's launch
+    bool in_chunk = true;
+    for (int32_t i = 0; i < n_binds && bind_slots; ++i) in_chunk = in_chunk && bind_slots[i] < n_slots;
+    TbInlineBinds ib;
+    Staging* used = nullptr;
+    std::vector<tb_graph*> let_go;
+    if (in_chunk && !(b->flags & TB_FLAG_COPIED_BINDS) &&
+        prepare_pulled_binds(b, n_binds, bind_slots, bind_graphs, stream, &ib, &used, &let_go)) {
+      rc = tb_launch_decode_general(p, stream, &ib);
+      if (rc == TB_OK && cudaEventRecord(used->done, stream) == cudaSuccess) used->pending = true;
+      else if (rc == TB_OK) { cudaGetLastError(); cudaStreamSynchronize(stream); }   // (no event: the graphs are let go only after the launch is done)
+      if (rc != TB_OK) {
+        // the launch did not happen: the slots it would have bound are left unbound, on both sides
+        for (int32_t i = 0; i < n_binds; ++i) {
+          release_slot(b, bind_slots[i]);
+          b->slot_n_states[bind_slots[i]] = 0; b->slot_cache_bytes[bind_slots[i]] = 0; b->slot_resolved[bind_slots[i]] = 1;
+          cudaMemsetAsync(b->d_slots + bind_slots[i], 0, sizeof(TbSlotRec), stream);
+        }
+        cudaGetLastError();
+      } else {
+        b->n_pulled_binds += n_binds;
+      }
+      for (tb_graph* h : let_go) tb_graph_free(h);
+      return rc;
+    }
+    rc = tb_batch_bind_streams(b, n_binds, bind_slots, bind_graphs, stream_);
     if (rc != TB_OK) return rc;
+    b->n_copied_binds += n_binds;
   }
-  return tb_stream_chunk(b, logits, dtype, n_slots, chunk, S, n_dur, strides, valid_frames, out_tokens, out_frames, out_durs,
-                         out_counts, out_scores, out_states, out_cursors, stream_);
+  return tb_launch_decode_general(p, stream);
+}
+
+extern "C" int tb_batch_bind_counts(const tb_batch* b, int64_t* out_pulled, int64_t* out_copied) {
+  if (!b || !out_pulled || !out_copied) return TB_ERR_INVALID_ARG;
+  *out_pulled = b->n_pulled_binds; *out_copied = b->n_copied_binds;
+  return TB_OK;
 }
 
 // The beam pre-pass for a launch that covers T * E rows per stream: reduces every row to its few best root-boosted

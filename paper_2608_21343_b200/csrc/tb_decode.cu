@@ -97,7 +97,7 @@ __device__ inline void tokview_enter(TokView& tv, const unsigned char* blob, con
 }
 
 template <typename LT>
-__global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
+__global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p, TbInlineBinds ib) {
   extern __shared__ __align__(16) unsigned char dyn[];
   float* bvec = reinterpret_cast<float*>(dyn);
   int32_t* nvec = reinterpret_cast<int32_t*>(dyn + sizeof(float) * p.C);
@@ -105,7 +105,44 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
   __shared__ float fred[kThreads / 32];
 
   const int b = blockIdx.x;
-  const TbSlotRec rec = p.slots[b];
+  TbSlotRec rec = p.slots[b];
+  // A bind that travels with this launch (streaming chunks): the block of a re-bound slot brings the new graph's
+  // image from page-locked host memory into its arena block itself, then stores the slot's new record; every other
+  // block is on its way already.
+  bool rebound = false;
+  if (ib.n > 0) {
+    int hit = -1;
+#pragma unroll
+    for (int i = 0; i < TB_INLINE_BINDS; ++i)
+      if (i < ib.n && ib.slot[i] == b) hit = i;
+    if (hit >= 0) {
+      const unsigned char* src = nullptr;
+      int32_t bytes = 0;
+#pragma unroll
+      for (int i = 0; i < TB_INLINE_BINDS; ++i)
+        if (hit == i) { src = ib.src[i]; bytes = ib.bytes[i]; rec = ib.rec[i]; }
+      rebound = true;
+      const uint4* s16 = reinterpret_cast<const uint4*>(src);
+      uint4* d16 = reinterpret_cast<uint4*>(ib.arena + rec.blob_off);
+      const int n16 = (bytes + 15) >> 4;             // (both blocks are padded to the arena's granule)
+      for (int j0 = 0; j0 < n16; j0 += 8 * kThreads) {
+        uint4 v[8];                                    // eight loads per thread on their way across the bus at once
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = j0 + u * kThreads + threadIdx.x;
+          if (j < n16) v[u] = s16[j];
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = j0 + u * kThreads + threadIdx.x;
+          if (j < n16) d16[j] = v[u];
+        }
+      }
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x == 0) ib.slots[b] = rec;
+    }
+  }
   const bool bound = rec.n_states > 0;
   const GraphPtrs g = graph_of(p.arena, rec);
   const unsigned char* blob = p.arena + rec.blob_off;
@@ -119,7 +156,8 @@ __global__ void __launch_bounds__(kThreads) k_decode_general(TbDecodeParams p) {
   int32_t t0 = 0, end, s, t, k, n_total = 0;
   float score;
   if (p.persistent) {
-    const TbSlotState st = p.sstate[b];
+    TbSlotState st = p.sstate[b];
+    if (rebound) { st.state = rec.n_states > 0 ? 0 : -1; st.t = 0; st.k = 0; st.score = 0.0f; st.n_emitted = 0; st.chunk_base = 0; }
     t0 = st.chunk_base; s = st.state; t = st.t; k = st.k; score = st.score; n_total = st.n_emitted;
     int32_t valid = p.lengths ? p.lengths[b] : INT32_MAX;
     end = min(t0 + p.frames, valid);
@@ -1725,8 +1763,11 @@ int set_smem(F* fn, size_t bytes) {
 
 }  // namespace
 
-int tb_launch_decode_general(const TbDecodeParams& p_in, cudaStream_t stream) {
+int tb_launch_decode_general(const TbDecodeParams& p_in, cudaStream_t stream, const TbInlineBinds* binds) {
   TbDecodeParams p = p_in;
+  TbInlineBinds ib;
+  if (binds) ib = *binds; else ib.n = 0;
+  if (ib.n < 0 || ib.n > TB_INLINE_BINDS || (ib.n > 0 && (!p.persistent || !ib.arena || !ib.slots))) return TB_ERR_INVALID_ARG;
   size_t smem = static_cast<size_t>(p.C) * (sizeof(float) + sizeof(int32_t));
   // graphs with resolved lists exist only for vocabularies whose token view fits comfortably
   p.tokview = 2 * (p.V + 1) <= (1 << TB_RS_TOK_BITS) ? 1 : 0;
@@ -1734,10 +1775,10 @@ int tb_launch_decode_general(const TbDecodeParams& p_in, cudaStream_t stream) {
   int rc;
   if (p.dtype == TB_BF16) {
     if ((rc = set_smem(k_decode_general<uint16_t>, smem)) != TB_OK) return rc;
-    k_decode_general<uint16_t><<<p.n_streams, kThreads, smem, stream>>>(p);
+    k_decode_general<uint16_t><<<p.n_streams, kThreads, smem, stream>>>(p, ib);
   } else {
     if ((rc = set_smem(k_decode_general<float>, smem)) != TB_OK) return rc;
-    k_decode_general<float><<<p.n_streams, kThreads, smem, stream>>>(p);
+    k_decode_general<float><<<p.n_streams, kThreads, smem, stream>>>(p, ib);
   }
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }

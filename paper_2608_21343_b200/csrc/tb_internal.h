@@ -28,6 +28,9 @@ void tb_pinned_pool_arm();                       // called when a batch has been
 void* tb_pinned_alloc(size_t bytes);             // nullptr: not from the pool (use the heap)
 bool tb_pinned_free(void* p, size_t bytes);      // false: p is not the pool's
 bool tb_pinned_owns(const void* p);
+// The address at which kernels of the current device can read the pool memory at host address p (the pool's pieces
+// are mapped into the device's address space when they are taken), or null when p is not the pool's or not mapped.
+const unsigned char* tb_pinned_device_ptr(const void* p);
 void tb_pinned_bypass(bool on);                  // this thread's next images go to the heap (TB_COMPILE_PAGEABLE)
 
 template <typename T>

@@ -60,7 +60,22 @@ struct TbBeamParams {
   int32_t rec_cache_bytes;   // shared memory set aside for a copy of the stream's list records (narrow beams; 0: none)
 };
 
-int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream);
+// Binds that a streaming chunk launch carries out itself (tb_stream_chunk_binds): the block of slot[i] first copies
+// the graph image of bytes[i] bytes from src[i] -- page-locked host memory, read in place -- to its arena block
+// (rec[i].blob_off), stores rec[i] as the slot's record and starts the slot's stream afresh; all other blocks start
+// at once.  bytes 0: the slot becomes unbound (rec all zero).
+#define TB_INLINE_BINDS 8
+struct TbInlineBinds {
+  int32_t n;
+  int32_t slot[TB_INLINE_BINDS];
+  int32_t bytes[TB_INLINE_BINDS];
+  const unsigned char* src[TB_INLINE_BINDS];
+  unsigned char* arena;       // (writable views of what the decode parameters hold as read-only)
+  TbSlotRec* slots;
+  TbSlotRec rec[TB_INLINE_BINDS];
+};
+
+int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream, const TbInlineBinds* binds = nullptr);
 // Returns TB_OK when it launched, 1 when the call is outside what the pipelined kernel covers.
 // max_cache_bytes: the largest cacheable list section among the slots decoded; max_states: their largest state count.
 // all_resolved: non-zero when every bound graph among them carries resolved per-state lists.

@@ -171,22 +171,33 @@ def test_beam_step_frozen_and_empty(tb):
     assert rp.tolist() == [0, 0, 0] and rt.tolist() == [0, 4, V]
 
 
-def run_stream(tb, w, n_chunks, weights_lam=None):
-    """Streaming decode with stream churn on both sides; compares after every chunk."""
+def run_stream(tb, w, n_chunks, weights_lam=None, in_chunk=False, flags=0, counts=None):
+    """Streaming decode with stream churn on both sides; compares after every chunk.  in_chunk: the new streams'
+    binds travel with the chunk call (tb_stream_chunk_binds) instead of one tb_batch_bind_stream each."""
     sched_gpu = W.ChurnSchedule(w)
     batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=8 << 20)
+    tb.tb_batch_set_flags(batch, flags)
     slots = [dict(graph=None, st=None, t0=0) for _ in range(w.B)]
     n_binds = 0
     for c in range(n_chunks):
         chunk, lengths, binds = sched_gpu.next_chunk()
+        new = []
         for slot, stream_id, phrases in binds:
             g = tb.tb_graph_compile(phrases, w.V, case_class=w.vocab.case_class)
-            tb.tb_batch_bind_stream(batch, slot, g)
+            if in_chunk:
+                new.append((slot, g))
+            else:
+                tb.tb_batch_bind_stream(batch, slot, g)
             og = oracle_graph(w, phrases)
             slots[slot] = dict(graph=og, st=O.StreamState(0, 0, 0, 0.0, 0), t0=0)
             n_binds += 1
-        out = to_host(tb.tb_stream_chunk(batch, to_device(chunk), w.n_dur,
-                                         torch.from_numpy(lengths).to("cuda:0")))
+        if in_chunk:
+            out = to_host(tb.tb_stream_chunk_binds(batch, [sl for sl, _ in new], [g for _, g in new], to_device(chunk), w.n_dur,
+                                                   torch.from_numpy(lengths).to("cuda:0")))
+            del new                                   # (the library holds the graphs for as long as it reads them)
+        else:
+            out = to_host(tb.tb_stream_chunk(batch, to_device(chunk), w.n_dur,
+                                             torch.from_numpy(lengths).to("cuda:0")))
         for i in range(w.B):
             sl = slots[i]
             ref = O.stream_chunk(sl["graph"], chunk[i], w.n_dur, sl["t0"], int(lengths[i]), sl["st"])
@@ -199,6 +210,8 @@ def run_stream(tb, w, n_chunks, weights_lam=None):
             assert out["states"][i] == sl["st"].state and out["cursors"][i] == sl["st"].t, (c, i)
             assert abs(float(out["scores"][i]) - float(sl["st"].score)) <= SCORE_TOL, (c, i)
     assert tb.tb_batch_status(batch) == 0
+    if counts is not None:
+        counts.update(tb.tb_batch_bind_counts(batch))
     return n_binds
 
 
@@ -206,6 +219,20 @@ def test_workload5_streaming_tdt_with_churn_reduced(tb):
     w = W.get_workload(5, B=12, T=90, T_lo=20, n_phrases=60, n_phrases_lo=10)
     n_binds = run_stream(tb, w, n_chunks=30)
     assert n_binds > 2 * w.B          # slots were refilled while others kept running
+
+
+def test_streaming_binds_carried_out_by_the_chunk_launch(tb):
+    """tb_stream_chunk_binds: the first chunk's twelve binds exceed what a launch carries and go ahead of it; the
+    refills afterwards (a few per chunk) are carried out by the chunk's own launch -- the re-bound slot's block reads
+    the image from host memory -- and the decode is the oracle's, chunk by chunk, as with single binds."""
+    w = W.get_workload(5, B=12, T=90, T_lo=20, n_phrases=60, n_phrases_lo=10)
+    counts = {}
+    n_binds = run_stream(tb, w, n_chunks=40, in_chunk=True, counts=counts)
+    assert counts["copied"] == w.B and counts["pulled"] == n_binds - w.B and counts["pulled"] > w.B
+    # the same with the switch that keeps every bind ahead of the launch
+    counts = {}
+    n_binds = run_stream(tb, w, n_chunks=12, in_chunk=True, flags=tb.TB_FLAG_COPIED_BINDS, counts=counts)
+    assert counts["pulled"] == 0 and counts["copied"] == n_binds
 
 
 def test_streaming_rnnt_chunked_equals_offline(tb):

@@ -126,12 +126,19 @@ def test_workload5_full_size_with_churn(tb):
                 graphs = list(ex.map(lambda b: tb.tb_graph_compile(b[2], w.V, case_class=w.vocab.case_class), binds))
                 ographs = list(ex.map(lambda b: oracle_graph(w, b[2]), binds))
                 for (slot, _sid, _phr), g, og in zip(binds, graphs, ographs):
-                    tb.tb_batch_bind_stream(batch, slot, g)
+                    if c % 2:
+                        tb.tb_batch_bind_stream(batch, slot, g)
                     slots[slot] = dict(graph=og, st=O.StreamState(0, 0, 0, 0.0, 0))
                     t0[slot] = 0
                     n_binds += 1
                     n_refills += c > 0
-                out = to_host(tb.tb_stream_chunk(batch, to_device(chunk), w.n_dur, torch.from_numpy(lengths).to("cuda:0")))
+                if c % 2:
+                    out = to_host(tb.tb_stream_chunk(batch, to_device(chunk), w.n_dur, torch.from_numpy(lengths).to("cuda:0")))
+                else:
+                    # every other chunk brings its binds along (the first one all 512, ahead of the launch; refills of up
+                    # to eight slots inside the launch)
+                    out = to_host(tb.tb_stream_chunk_binds(batch, [bd[0] for bd in binds], graphs, to_device(chunk), w.n_dur,
+                                                           torch.from_numpy(lengths).to("cuda:0")))
 
                 def one(i):
                     sl = slots[i]
@@ -153,6 +160,8 @@ def test_workload5_full_size_with_churn(tb):
         sched.close()
     assert tb.tb_batch_status(batch) == 0
     assert n_binds == w.B + n_refills and n_refills > 300 and n_tokens > 100000
+    counts = tb.tb_batch_bind_counts(batch)
+    assert counts["pulled"] > 100 and counts["copied"] >= w.B      # both ways of tb_stream_chunk_binds were taken
 
 
 def _coarse(x):

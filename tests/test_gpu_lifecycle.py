@@ -271,6 +271,29 @@ def test_binding_many_streams_at_once(tb):
     assert got["cursors"][1] == want["cursors"][1] + 8                    # the other slots went on
     more = to_host(tb.tb_stream_chunk_binds(batch, [], [], logits[:, 8:16], 0, valid))      # no binds: a plain chunk
     assert more["cursors"][0] == 16
+    assert tb.tb_batch_bind_counts(batch) == dict(pulled=2, copied=0)     # the two binds rode on the chunk's launch
+    # a graph on the heap cannot be read by the kernel in place: the group goes ahead of the launch; a slot that is
+    # unbound in the same call as another is bound: carried out by the launch; and the result is the same every way
+    heap = tb.tb_graph_compile(data["phrases"][5], w.V, case_class=w.vocab.case_class, flags=tb.TB_COMPILE_PAGEABLE)
+    a_ = to_host(tb.tb_stream_chunk_binds(batch, [5, 6], [heap, None], logits[:, :8], 0, valid))
+    assert tb.tb_batch_bind_counts(batch) == dict(pulled=2, copied=2)
+    b_ = to_host(tb.tb_stream_chunk_binds(batch, [5, 6], [graphs[5], None], logits[:, :8], 0, valid))
+    assert tb.tb_batch_bind_counts(batch) == dict(pulled=4, copied=2)
+    ref5 = O.stream_chunk(oracle_graph(w, data["phrases"][5]), data["logits"][5][:8], 0, 0, w.T, O.StreamState(0, 0, 0, 0.0, 0))
+    ref6 = O.stream_chunk(None, data["logits"][6][:8], 0, 0, w.T, O.StreamState(-1, 0, 0, 0.0, 0))
+    for got_ in (a_, b_):
+        for i, ref in ((5, ref5), (6, ref6)):
+            n = int(got_["counts"][i])
+            assert n == len(ref["tokens"]) and np.array_equal(got_["tokens"][i, :n], ref["tokens"]) and got_["cursors"][i] == 8
+        assert got_["states"][6] == -1 and a_["scores"][5] == b_["scores"][5]
+    # a chunk that is refused binds nothing
+    with pytest.raises(tb.TbError):
+        tb.tb_stream_chunk_binds(batch, [7], [graphs[0]], logits[:, :8], 0, None)        # no frame counts: the chunk is refused
+    assert tb.tb_batch_bind_counts(batch) == dict(pulled=4, copied=2)
+    # slots beyond the chunk's are bound ahead of the launch
+    tb.tb_stream_chunk_binds(batch, [7], [graphs[7]], logits[:4, :8], 0, valid[:4])
+    assert tb.tb_batch_bind_counts(batch) == dict(pulled=4, copied=3)
+    assert tb.tb_batch_status(batch) == 0
     # errors: checked before anything changes
     with pytest.raises(tb.TbError) as e:
         tb.tb_stream_chunk_binds(batch, [0, 0], [graphs[0], graphs[1]], logits[:, :8], 0, valid)
