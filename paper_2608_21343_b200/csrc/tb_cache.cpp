@@ -18,7 +18,7 @@
 namespace {
 
 constexpr uint32_t kMagic = 0x31474254u;   // "TBG1"
-constexpr uint32_t kVersion = 3;
+constexpr uint32_t kVersion = 4;
 
 // FNV-1a style checksum over 8-byte words (the tail byte by byte): detects damage, is not cryptographic
 uint64_t fnv1a(const void* p, size_t n, uint64_t h = 1469598103934665603ull) {
@@ -162,8 +162,10 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
       const int64_t Ns = h.n_states, As = h.n_arcs, Te = h.n_tokent, Re = h.n_rsent;
       bool in = g->off_arc_begin + 4 * (Ns + 1) <= B && g->off_fail + 4 * Ns <= B && g->off_bw + 4 * Ns <= B &&
                 g->off_arc_cls + 4 * As <= B && g->off_arc_w + 4 * As <= B && g->off_arc_dst + 4 * As <= B &&
-                g->off_final + 4 * Ns <= B && g->off_strec + 16 * Ns <= B && g->off_tokent + 16 * Te <= B;
-      if (Re >= 0) in = in && g->off_rsrec + 16 * Ns <= B && g->off_rsent + 8 * Re <= B;
+                g->off_final + 4 * Ns <= B;
+      // a graph carries either resolved lists or per-state records with token-expanded arcs, never both
+      if (Re >= 0) in = in && g->off_rsrec + 16 * Ns <= B && g->off_rsent + 8 * Re <= B && Te == 0 && g->off_strec == 0 && g->off_tokent == 0;
+      else in = in && g->off_strec + 16 * Ns <= B && g->off_tokent + 16 * Te <= B;
       in = in && g->state_arc_begin[0] == 0 && g->state_arc_begin[Ns] == As;
       for (int64_t u = 0; in && u < Ns; ++u)
         in = g->state_arc_begin[u] <= g->state_arc_begin[u + 1] && g->state_fail[u] >= 0 && g->state_fail[u] < Ns;
@@ -177,9 +179,11 @@ extern "C" int tb_graph_load(const char* path, tb_graph** out) {
       for (int64_t u = 0; in && u < Ns; ++u) {
         const int32_t f = i32(g->off_fail, u);
         in = i32(g->off_arc_begin, u) <= i32(g->off_arc_begin, u + 1) && f >= 0 && f < Ns;
-        TbStateRec sr;
-        std::memcpy(&sr, bl + g->off_strec + 16 * u, 16);
-        in = in && sr.tok_begin >= 0 && sr.tok_begin <= sr.tok_end && sr.tok_end <= Te && sr.fail >= 0 && sr.fail < Ns;
+        if (Re < 0) {
+          TbStateRec sr;
+          std::memcpy(&sr, bl + g->off_strec + 16 * u, 16);
+          in = in && sr.tok_begin >= 0 && sr.tok_begin <= sr.tok_end && sr.tok_end <= Te && sr.fail >= 0 && sr.fail < Ns;
+        }
       }
       for (int64_t a = 0; in && a < As; ++a) {
         const int32_t d = i32(g->off_arc_dst, a), c = i32(g->off_arc_cls, a);

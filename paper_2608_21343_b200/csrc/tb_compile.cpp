@@ -82,28 +82,12 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
   g->off_arc_w = append_section(blob, g->arc_w);
   g->off_arc_dst = append_section(blob, g->arc_dst);
   g->off_final = append_section(blob, g->state_final);
-  {  // per-state records and token-expanded arcs (tokens of a class in ascending id order)
+  {  // the tokens of every class, in ascending id order
     std::vector<int32_t> ctb(n_classes + 1, 0), ctk(vocab);
     for (int32_t v = 0; v < vocab; ++v) ctb[g->case_class[v] + 1]++;
     for (int32_t c = 0; c < n_classes; ++c) ctb[c + 1] += ctb[c];
     std::vector<int32_t> fill(ctb.begin(), ctb.end() - 1);
     for (int32_t v = 0; v < vocab; ++v) ctk[fill[g->case_class[v]]++] = v;
-    std::vector<TbStateRec> recs(N);
-    std::vector<TbTokEnt> ents;
-    for (int32_t u = 0; u < N; ++u) {
-      recs[u].tok_begin = static_cast<int32_t>(ents.size());
-      for (int32_t a = g->state_arc_begin[u]; a < g->state_arc_begin[u + 1]; ++a) {
-        const int32_t c = g->arc_class[a];
-        for (int32_t j = ctb[c]; j < ctb[c + 1]; ++j)
-          ents.push_back({static_cast<uint32_t>(ctk[j]) | (static_cast<uint32_t>(c) << 16), g->arc_w[a], g->arc_dst[a], 0});
-      }
-      recs[u].tok_end = static_cast<int32_t>(ents.size());
-      recs[u].fail = g->state_fail[u];
-      recs[u].bw = g->state_bw[u];
-    }
-    g->off_strec = append_section(blob, recs);
-    g->off_tokent = append_section(blob, ents);
-    g->n_tokent = static_cast<int32_t>(ents.size());
 
     // resolved lists (see TbRsRec): the walk the kernels would do, done once here in float
     float root_w_max = 0.0f;
@@ -145,10 +129,30 @@ static void finalize_graph(tb_graph* g, const int32_t* case_class, int32_t vocab
       rrecs[s].bmag = std::fabs(lambda) * (std::fabs(acc) + root_w_max);
     }
     if (fits) {
+      // (the kernels read these lists and nothing else beyond the flat arrays: the image carries no per-state records)
+      g->off_strec = g->off_tokent = 0;
+      g->n_tokent = 0;
       g->off_rsrec = append_section(blob, rrecs);
       g->off_rsent = append_section(blob, rents);
       g->n_rsent = static_cast<int32_t>(rents.size());
     } else {
+      // too large for resolved lists: per-state records and token-expanded arcs, which the kernels walk instead
+      std::vector<TbStateRec> recs(N);
+      std::vector<TbTokEnt> ents;
+      for (int32_t u = 0; u < N; ++u) {
+        recs[u].tok_begin = static_cast<int32_t>(ents.size());
+        for (int32_t a = g->state_arc_begin[u]; a < g->state_arc_begin[u + 1]; ++a) {
+          const int32_t c = g->arc_class[a];
+          for (int32_t j = ctb[c]; j < ctb[c + 1]; ++j)
+            ents.push_back({static_cast<uint32_t>(ctk[j]) | (static_cast<uint32_t>(c) << 16), g->arc_w[a], g->arc_dst[a], 0});
+        }
+        recs[u].tok_end = static_cast<int32_t>(ents.size());
+        recs[u].fail = g->state_fail[u];
+        recs[u].bw = g->state_bw[u];
+      }
+      g->off_strec = append_section(blob, recs);
+      g->off_tokent = append_section(blob, ents);
+      g->n_tokent = static_cast<int32_t>(ents.size());
       g->off_rsrec = g->off_rsent = 0;
       g->n_rsent = -1;
     }
