@@ -224,7 +224,8 @@ int tb_graph_load(const char *path, tb_graph **out);
  * copies from the graph in place; the batch holds the graph until that copy is done.  The same holds for every graph
  * compiled or loaded after the process has created its first batch: their device blobs are placed in a pool of
  * page-locked host memory (up to 1 GB, in pieces of 32 MB; blobs over 16 MB and whatever does not fit stay on the heap
- * and are staged at bind time).
+ * and are staged at bind time).  The pool's pieces are also mapped into the devices' address space, so that a
+ * kernel can read a blob where it lies (tb_stream_chunk_binds uses that).
  *   out_hit  host int32 or NULL.   Errors: as tb_graph_compile.
  * tb_cache_stats: any pointer may be NULL.
  */

@@ -135,17 +135,22 @@ void* tb_pinned_alloc(size_t bytes) {
       }
     if (pass == 1 || pool.closed || pool.total + kPoolChunk > kPoolMax) return nullptr;
     void* base = nullptr;
+    bool mapped = true;
     if (cudaHostAlloc(&base, kPoolChunk, cudaHostAllocPortable | cudaHostAllocMapped) != cudaSuccess) {
       cudaGetLastError();
-      pool.closed = true;
-      return nullptr;
+      mapped = false;                                                // (page-locked without a device mapping still serves the copies)
+      if (cudaHostAlloc(&base, kPoolChunk, cudaHostAllocPortable) != cudaSuccess) {
+        cudaGetLastError();
+        pool.closed = true;
+        return nullptr;
+      }
     }
     PinnedPool::Chunk c;
     c.base = static_cast<unsigned char*>(base); c.bytes = kPoolChunk;
     // kernels may read the piece in place (a bind that the decoding kernel carries out itself) where the device
     // addresses it like the host does -- unified addressing --, which is what makes the address good on every device
     void* dev = nullptr;
-    if (cudaHostGetDevicePointer(&dev, base, 0) != cudaSuccess) { cudaGetLastError(); dev = nullptr; }
+    if (!mapped || cudaHostGetDevicePointer(&dev, base, 0) != cudaSuccess) { cudaGetLastError(); dev = nullptr; }
     c.dev_base = dev == base ? static_cast<unsigned char*>(dev) : nullptr;
     c.free_blocks[0] = kPoolChunk;
     pool.chunks.push_back(std::move(c));
