@@ -264,8 +264,10 @@ void tb_batch_destroy(tb_batch *b);
  * Attach graph g to `slot`, or detach with g == NULL (model id -1: zero bonus, state -1;
  * Sec. 2.2 para. 3).  Adding and removing lists while other streams keep running is Sec. 2.2
  * para. 4; here the slot index is the stable id, and no other slot's graph moves or changes.
- * The graph is copied with an asynchronous host-to-device copy on `stream` (from its own page-locked blob, or
- * through page-locked staging memory of the batch when its blob is on the heap); the slot's offsets are published and its streaming state is reset (state =
+ * The graph reaches the arena on `stream`: a blob in the library's page-locked pool is read in place by a small
+ * launch that also publishes the slot's record (no copy is enqueued); any other blob is copied with an asynchronous
+ * host-to-device copy (from its own page-locked memory when a cache keeps it, else through page-locked staging
+ * memory of the batch); the slot's offsets are published and its streaming state is reset (state =
  * root or -1, frame cursor 0, score 0) in stream order.  The previous graph's arena space is
  * reused by later binds.  g must have been compiled with the batch's vocab and class map.
  * Ordering: the previous graph's arena block goes back to the free list when this call returns, and a later bind

@@ -403,6 +403,37 @@ static void release_slot(tb_batch* b, int32_t slot) {
   b->slot_model[slot] = -1;
 }
 
+static bool prepare_pulled_binds(tb_batch* b, int32_t n, const int32_t* slots, const tb_graph* const* graphs, cudaStream_t stream,
+                                 TbInlineBinds* ib, Staging** used, std::vector<tb_graph*>* let_go);
+
+// Binds of up to TB_INLINE_BINDS graphs whose images lie in the page-locked pool, carried out by one launch that
+// reads the images in place (no copy is enqueued; the graphs are held until the launch's event).  False, with nothing
+// changed, when the group has to go the ordinary way.
+static bool bind_by_pull(tb_batch* b, int32_t n, const int32_t* slots, const tb_graph* const* graphs, cudaStream_t stream) {
+  if (b->flags & TB_FLAG_COPIED_BINDS) return false;
+  bool any = false;
+  for (int32_t i = 0; i < n && graphs; ++i) any = any || graphs[i] != nullptr;
+  if (!any) return false;                              // (slots that only lose their graph need no image: the small launch does)
+  TbInlineBinds ib;
+  Staging* used = nullptr;
+  std::vector<tb_graph*> let_go;
+  if (!prepare_pulled_binds(b, n, slots, graphs, stream, &ib, &used, &let_go)) return false;
+  int rc = tb_launch_pull_binds(ib, b->d_sstate, stream);
+  if (rc == TB_OK && cudaEventRecord(used->done, stream) == cudaSuccess) used->pending = true;
+  else { cudaGetLastError(); cudaStreamSynchronize(stream); }     // (no event, or no launch: nothing reads the graphs once this returns)
+  if (rc != TB_OK) {
+    // the launch did not happen: the copies and the small launch do the same job from the same blocks
+    bool ok = true;
+    for (int32_t i = 0; i < n; ++i)
+      if (graphs[i]) ok = ok && cudaMemcpyAsync(b->arena + ib.rec[i].blob_off, graphs[i]->blob.data(), graphs[i]->blob.size(), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    for (int32_t i = 0; i < n; ++i) ok = ok && tb_launch_publish_slot(b->d_slots, b->d_sstate, slots[i], ib.rec[i], stream) == TB_OK;
+    if (!ok) cudaGetLastError();
+    cudaStreamSynchronize(stream);
+  }
+  for (tb_graph* h : let_go) tb_graph_free(h);
+  return true;
+}
+
 extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g, void* stream_) {
   TbRange range_("tb_batch_bind_stream");
   if (!b) return TB_ERR_INVALID_ARG;
@@ -410,6 +441,7 @@ extern "C" int tb_batch_bind_stream(tb_batch* b, int32_t slot, const tb_graph* g
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
+  if (g && bind_by_pull(b, 1, &slot, &g, stream)) return TB_OK;
   TbSlotRec rec;
   std::memset(&rec, 0, sizeof rec);
   size_t off = 0, bytes = 0;
@@ -461,6 +493,18 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   const size_t tail = round_up(static_cast<size_t>(n) * (sizeof(TbSlotRec) + sizeof(int32_t)), kArenaAlign);
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
+  // graphs in the page-locked pool: a launch reads their images in place, eight binds at a time (what is left when a
+  // group cannot go that way -- a graph on the heap, no room -- goes the ordinary way below)
+  if (n <= 4 * TB_INLINE_BINDS) {
+    int32_t done = 0;
+    while (done < n) {
+      const int32_t m = n - done < TB_INLINE_BINDS ? n - done : TB_INLINE_BINDS;
+      if (!bind_by_pull(b, m, slots + done, graphs + done, stream)) break;
+      done += m;
+    }
+    if (done == n) return TB_OK;
+    if (done > 0) return tb_batch_bind_streams(b, n - done, slots + done, graphs + done, stream_);
+  }
   size_t base = 0;
   if (!b->alloc.alloc(total + tail, &base)) {
     // no contiguous room for the group (a fragmented or nearly full arena): one by one, each in the first hole that fits

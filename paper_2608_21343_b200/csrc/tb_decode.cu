@@ -1921,6 +1921,45 @@ __global__ void k_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n
   sstate[slot_of[i]] = st;
 }
 
+// Binds carried out by one launch (see TbInlineBinds): block i brings the image of bind i from page-locked host
+// memory, read in place, into its arena block, then stores the slot's record and starts the slot's stream afresh.
+constexpr int kPullThreads = 512;
+__global__ void __launch_bounds__(kPullThreads) k_pull_binds(TbInlineBinds ib, TbSlotState* sstate) {
+  const int i = blockIdx.x;
+  const unsigned char* src = nullptr;
+  int32_t bytes = 0, slot = -1;
+  TbSlotRec rec;
+#pragma unroll
+  for (int j = 0; j < TB_INLINE_BINDS; ++j)
+    if (i == j) { src = ib.src[j]; bytes = ib.bytes[j]; slot = ib.slot[j]; rec = ib.rec[j]; }
+  if (i >= ib.n || slot < 0) return;
+  const uint4* s16 = reinterpret_cast<const uint4*>(src);
+  uint4* d16 = reinterpret_cast<uint4*>(ib.arena + rec.blob_off);
+  const int n16 = (bytes + 15) >> 4;               // (both blocks are padded to the arena's granule)
+  for (int j0 = 0; j0 < n16; j0 += 8 * kPullThreads) {
+    uint4 v[8];                                      // eight loads per thread on their way across the bus at once
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + u * kPullThreads + threadIdx.x;
+      if (j < n16) v[u] = s16[j];
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int j = j0 + u * kPullThreads + threadIdx.x;
+      if (j < n16) d16[j] = v[u];
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    ib.slots[slot] = rec;
+    TbSlotState st;
+    st.state = rec.n_states > 0 ? 0 : -1; st.t = 0; st.k = 0; st.score = 0.0f; st.n_emitted = 0;
+    st.chunk_base = 0; st.pad0 = 0; st.pad1 = 0;
+    sstate[slot] = st;
+  }
+}
+
 __global__ void k_final_weights_slots(const TbSlotRec* slots, const unsigned char* arena, int32_t n, SlotList sl, int32_t K,
                                       float* scores, const int32_t* states, int32_t* status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -1995,6 +2034,12 @@ int tb_launch_publish_slots(TbSlotRec* slots, TbSlotState* sstate, int32_t n, co
                             cudaStream_t stream) {
   if (n < 1) return TB_ERR_INVALID_ARG;
   k_publish_slots<<<(n + 63) / 64, 64, 0, stream>>>(slots, sstate, n, recs, slot_of);
+  return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+
+int tb_launch_pull_binds(const TbInlineBinds& ib, TbSlotState* sstate, cudaStream_t stream) {
+  if (ib.n < 1 || ib.n > TB_INLINE_BINDS || !ib.arena || !ib.slots || !sstate) return TB_ERR_INVALID_ARG;
+  k_pull_binds<<<ib.n, kPullThreads, 0, stream>>>(ib, sstate);
   return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 

@@ -76,6 +76,8 @@ struct TbInlineBinds {
 };
 
 int tb_launch_decode_general(const TbDecodeParams& p, cudaStream_t stream, const TbInlineBinds* binds = nullptr);
+// The same binds carried out by a launch of their own (tb_batch_bind_stream(s) for graphs in the page-locked pool).
+int tb_launch_pull_binds(const TbInlineBinds& binds, TbSlotState* sstate, cudaStream_t stream);
 // Returns TB_OK when it launched, 1 when the call is outside what the pipelined kernel covers.
 // max_cache_bytes: the largest cacheable list section among the slots decoded; max_states: their largest state count.
 // all_resolved: non-zero when every bound graph among them carries resolved per-state lists.
