@@ -128,17 +128,24 @@ def _hp(a):
 
 
 def _dp(t):
+    # (an address as a plain int: ctypes converts it for a pointer argument; whatever is not a CUDA tensor is refused
+    # here, before its address could reach a kernel)
     if t is None:
         return None
-    if not (isinstance(t, torch.Tensor) and t.is_cuda):
+    if not t.is_cuda:
         raise TypeError("expected a CUDA tensor")
-    return _vp(t.data_ptr())
+    return t.data_ptr()
+
+
+_raw_current_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
 
 
 def _stream(stream):
     if stream is None:
+        if _raw_current_stream is not None:       # the current stream's handle without building a Stream object
+            return _raw_current_stream(torch.cuda.current_device())
         stream = torch.cuda.current_stream()
-    return _vp(stream.cuda_stream)
+    return stream.cuda_stream
 
 
 def _logit_dtype(t: torch.Tensor) -> int:
