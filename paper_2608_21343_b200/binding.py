@@ -127,6 +127,15 @@ def _hp(a):
     return _vp(a.__array_interface__["data"][0])
 
 
+def _slots(slots):
+    """A short list of slot indices as (n, host int32 array for the call)."""
+    if isinstance(slots, (list, tuple)):         # (the usual case: no numpy array is built for a handful of indices)
+        n = len(slots)
+        return n, ((_i32 * n)(*slots) if n else None)
+    a = _host(slots, np.int32)
+    return len(a), _hp(a)
+
+
 def _dp(t):
     # (an address as a plain int: ctypes converts it for a pointer argument; whatever is not a CUDA tensor is refused
     # here, before its address could reach a kernel)
@@ -525,17 +534,17 @@ def tb_beam_reset_slots(batch: Batch, slots=None, stream=None):
     if slots is None:
         _check(_lib.tb_beam_reset_slots(batch.handle, 0, None, _stream(stream)), "tb_beam_reset_slots")
         return
-    sl = _host(slots, np.int32)
-    if len(sl):
-        _check(_lib.tb_beam_reset_slots(batch.handle, len(sl), _hp(sl), _stream(stream)), "tb_beam_reset_slots")
+    n, sl = _slots(slots)
+    if n:
+        _check(_lib.tb_beam_reset_slots(batch.handle, n, sl, _stream(stream)), "tb_beam_reset_slots")
 
 
 def tb_beam_start_slots(batch: Batch, slots, scores: torch.Tensor, states: torch.Tensor, live: torch.Tensor, stream=None):
     """tb_beam_reset_slots that also sets up the slots' rows of scores / states / live [n_slots, K] (None: every slot)."""
-    sl = None if slots is None else _host(slots, np.int32)
-    if sl is not None and len(sl) == 0:
+    n, sl = (0, None) if slots is None else _slots(slots)
+    if slots is not None and n == 0:
         return
-    _check(_lib.tb_beam_start_slots(batch.handle, 0 if sl is None else len(sl), _hp(sl), scores.shape[1], _dp(scores),
+    _check(_lib.tb_beam_start_slots(batch.handle, n, sl, scores.shape[1], _dp(scores),
                                     _dp(states), _dp(live), _stream(stream)), "tb_beam_start_slots")
 
 
@@ -588,9 +597,9 @@ def tb_beam_backtrace_slot_list(batch: Batch, slots, K: int, max_len: int, strea
 
 
 def tb_apply_final_weights_slots(batch: Batch, slots, scores: torch.Tensor, states: torch.Tensor, stream=None):
-    sl = _host(slots, np.int32)
-    if len(sl):
-        _check(_lib.tb_apply_final_weights_slots(batch.handle, len(sl), _hp(sl), scores.shape[1], _dp(scores), _dp(states),
+    n, sl = _slots(slots)
+    if n:
+        _check(_lib.tb_apply_final_weights_slots(batch.handle, n, sl, scores.shape[1], _dp(scores), _dp(states),
                                                  _stream(stream)), "tb_apply_final_weights_slots")
 
 
