@@ -312,7 +312,7 @@ def side_measurement(args):
                                               "note": "chunk logits staged on the device before the loop, one buffer per chunk; binds and chunk call timed as above"},
                           "config": {"workload": w.name, "slots": w.B, "chunk_frames": w.chunk, "chunks": len(lat),
                                      "binds_in_timed_region": True, "rebinds": binds - w.B,
-                                     "binds": "one by one" if args.single_binds else "tb_stream_chunk_binds (up to 8 binds per chunk carried out by the chunk's own launch, larger groups by copies and a launch ahead of it)",
+                                     "binds": "one by one" if args.single_binds else "tb_stream_chunk_binds (up to 16 binds per chunk carried out by the chunk's own launch, larger groups by copies and a launch ahead of it)",
                                      "bind_counts": tb.tb_batch_bind_counts(batch)},
                           "frames_per_s_at_p50": w.B * w.chunk / (float(np.percentile(lat, 50)) * 1e-3),
                           "host_issue_us_p50": float(np.percentile(np.array(host_us[10:]), 50)),

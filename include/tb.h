@@ -419,7 +419,7 @@ int tb_stream_chunk(tb_batch *b, const void *logits, int dtype, int32_t n_slots,
  * binds nothing.  n_binds may be 0 (bind_slots / bind_graphs are then not read).  If the binds fail the chunk is not
  * decoded.  Errors: those of the two calls.
  *
- * Up to 8 binds per call ride on the chunk's own launch: when every graph's image lies in the library's page-locked
+ * Up to 16 binds per call ride on the chunk's own launch: when every graph's image lies in the library's page-locked
  * memory (graphs compiled or loaded after the first tb_batch_create, without TB_COMPILE_PAGEABLE, not handed out by
  * a cache), the bound slots are among the chunk's n_slots, and `stream` is not being captured, the call reserves
  * the arena blocks, and the thread block that decodes a re-bound slot first reads the new image from host memory in

@@ -493,7 +493,7 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   const size_t tail = round_up(static_cast<size_t>(n) * (sizeof(TbSlotRec) + sizeof(int32_t)), kArenaAlign);
   DeviceGuard guard(b->device);
   if (!guard.ok) return TB_ERR_CUDA;
-  // graphs in the page-locked pool: a launch reads their images in place, eight binds at a time (what is left when a
+  // graphs in the page-locked pool: a launch reads their images in place, TB_INLINE_BINDS binds at a time (what is left when a
   // group cannot go that way -- a graph on the heap, no room -- goes the ordinary way below)
   if (n <= 4 * TB_INLINE_BINDS) {
     int32_t done = 0;

@@ -64,7 +64,7 @@ struct TbBeamParams {
 // the graph image of bytes[i] bytes from src[i] -- page-locked host memory, read in place -- to its arena block
 // (rec[i].blob_off), stores rec[i] as the slot's record and starts the slot's stream afresh; all other blocks start
 // at once.  bytes 0: the slot becomes unbound (rec all zero).
-#define TB_INLINE_BINDS 8
+#define TB_INLINE_BINDS 16
 struct TbInlineBinds {
   int32_t n;
   int32_t slot[TB_INLINE_BINDS];

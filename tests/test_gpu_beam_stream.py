@@ -222,10 +222,10 @@ def test_workload5_streaming_tdt_with_churn_reduced(tb):
 
 
 def test_streaming_binds_carried_out_by_the_chunk_launch(tb):
-    """tb_stream_chunk_binds: the first chunk's twelve binds exceed what a launch carries and go ahead of it; the
+    """tb_stream_chunk_binds: the first chunk's twenty binds exceed what a launch carries and go ahead of it; the
     refills afterwards (a few per chunk) are carried out by the chunk's own launch -- the re-bound slot's block reads
     the image from host memory -- and the decode is the oracle's, chunk by chunk, as with single binds."""
-    w = W.get_workload(5, B=12, T=90, T_lo=20, n_phrases=60, n_phrases_lo=10)
+    w = W.get_workload(5, B=20, T=90, T_lo=20, n_phrases=60, n_phrases_lo=10)
     counts = {}
     n_binds = run_stream(tb, w, n_chunks=40, in_chunk=True, counts=counts)
     assert counts["copied"] == w.B and counts["pulled"] == n_binds - w.B and counts["pulled"] > w.B
