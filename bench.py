@@ -257,6 +257,8 @@ def side_measurement(args):
         batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=256 << 20)
         n_chunks, lat, binds, t_compile = 40 + 10 * args.steps, [], 0, 0.0
         host_us = []
+        ev5 = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+        ev5[0].record(); ev5[1].record(); torch.cuda.synchronize()
         bufs = []
         outs = None
         for c in range(n_chunks):
@@ -268,7 +270,7 @@ def side_measurement(args):
             dv = torch.from_numpy(lengths).to(dev)
             bufs = (bufs + [dl])[-8:]
             torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a, b = ev5                                     # (one pair of events for all chunks: every chunk ends with a synchronize)
             th = time.perf_counter()
             a.record()
             if args.single_binds:
@@ -342,6 +344,10 @@ def side_measurement(args):
             total = np.zeros(w.B, dtype=np.int64)
             n_chunks, lat, kern, n_done, frames = 30 + 2 * args.steps, [], [], 0, 0
             bufs = []
+            ev8 = tuple(torch.cuda.Event(enable_timing=True) for _ in range(4))
+            for e_ in ev8:
+                e_.record()
+            torch.cuda.synchronize()
             for c in range(n_chunks):
                 chunk, lengths, bl = sched.next_chunk()
                 gs = [(sl, tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class)) for sl, _, p in bl]
@@ -354,7 +360,7 @@ def side_measurement(args):
                 bufs = (bufs + [dl])[-8:]
                 new = [sl for sl, _ in gs]
                 torch.cuda.synchronize()
-                a, m0, m1, b = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+                a, m0, m1, b = ev8                          # (one set of events for all chunks: every chunk ends with a synchronize)
                 a.record()
                 tb.tb_batch_bind_streams(batch, new, [g for _, g in gs])
                 tb.tb_beam_start_slots(batch, new, scores, states, live)     # the new slots' beams, set up by the library
