@@ -233,6 +233,26 @@ def test_binding_many_registered_models_at_once(tb):
     tb.tb_batch_bind_models(batch, [], [])
 
 
+def test_binding_forty_streams_in_one_call(tb):
+    """tb_batch_bind_streams with more graphs than one binding launch carries (several launches of sixteen, each block
+    reading one image from page-locked memory in place), some of them on the heap (copied), some slots unbound."""
+    w = W.get_workload(2, B=40, T=60, n_phrases=30, n_plants=4)
+    data = W.batch_inputs(w)
+    logits = to_device(data["logits"])
+    batch = tb.tb_batch_create(w.V, w.vocab.case_class, w.B, arena_bytes=8 << 20)
+    lists = list(data["phrases"])
+    lists[7] = lists[23] = None
+    graphs = [None if p is None else tb.tb_graph_compile(p, w.V, case_class=w.vocab.case_class,
+                                                         flags=tb.TB_COMPILE_PAGEABLE if i in (18, 33) else 0) for i, p in enumerate(lists)]
+    tb.tb_batch_bind_streams(batch, list(range(w.B)), graphs)
+    del graphs                                           # (the library holds what it still reads)
+    out = to_host(tb.tb_greedy_decode(batch, logits))
+    assert tb.tb_batch_status(batch) == 0
+    for i in range(w.B):
+        check_greedy(out, i, O.greedy_rnnt(oracle_graph(w, lists[i]), data["logits"][i]), "forty at once")
+    assert out["states"][7] == -1 and out["states"][23] == -1
+
+
 def test_binding_many_streams_at_once(tb):
     """tb_batch_bind_streams: several slots get new lists (or lose theirs) in one copy and one launch; the result is
     what the same binds one by one give, other slots are untouched, and a small arena falls back to single binds."""
