@@ -504,19 +504,20 @@ def side_measurement(args):
             torch.cuda.synchronize()
             ts = []
             all_slots = np.arange(w2.B, dtype=np.int32)
+            slot_list = list(range(w2.B))
             for _ in range(max(5, args.steps // 20)):
                 t0 = time.perf_counter()
-                for i, p in enumerate(flat2):
-                    if mode == "none":
-                        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_compile(p, w2.V, case_class=cc2))
-                    elif mode == "disk":
-                        tb.tb_batch_bind_stream(batch, i, tb.tb_graph_load(os.path.join(tmp, "w2_%d.tbg" % i)))
-                    elif mode == "memory":
-                        tb.tb_batch_bind_stream(batch, i, tb.tb_cache_compile(cache, p, w2.V, case_class=cc2)[0])
-                    else:
-                        break
+                if mode == "none":
+                    gl = [tb.tb_graph_compile(p, w2.V, case_class=cc2) for p in flat2]
+                elif mode == "disk":
+                    gl = [tb.tb_graph_load(os.path.join(tmp, "w2_%d.tbg" % i)) for i in range(len(flat2))]
+                elif mode == "memory":
+                    gl = [tb.tb_cache_compile(cache, p, w2.V, case_class=cc2)[0] for p in flat2]
                 if mode == "decoder":
                     tb.tb_batch_bind_models(batch, all_slots, ids)
+                else:
+                    tb.tb_batch_bind_streams(batch, slot_list, gl)      # all 128 in one call
+                    gl = None
                 tb.tb_greedy_decode(batch, l2, out=out2)
                 torch.cuda.synchronize()
                 ts.append((time.perf_counter() - t0) * 1e3)

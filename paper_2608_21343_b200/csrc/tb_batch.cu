@@ -495,7 +495,7 @@ extern "C" int tb_batch_bind_streams(tb_batch* b, int32_t n, const int32_t* slot
   if (!guard.ok) return TB_ERR_CUDA;
   // graphs in the page-locked pool: a launch reads their images in place, TB_INLINE_BINDS binds at a time (what is left when a
   // group cannot go that way -- a graph on the heap, no room -- goes the ordinary way below)
-  if (n <= 4 * TB_INLINE_BINDS) {
+  {
     int32_t done = 0;
     while (done < n) {
       const int32_t m = n - done < TB_INLINE_BINDS ? n - done : TB_INLINE_BINDS;
